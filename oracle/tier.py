@@ -1,0 +1,157 @@
+"""Host-tier reference model and write admission.
+
+Reference model (Appendix D, "Reference model" and "Recency order of the host tier"):
+the tier starts empty and holds at most K_H chunks in recency order.  A reference to a
+resident chunk hits and moves it to the most-recent end.  A miss that is admitted
+inserts the chunk at the most-recent end, first evicting the least-recent chunk when
+K_H chunks are resident; a declined miss leaves the tier unchanged.
+
+Write rule (Eq. 6): a request with n prompt tokens of which the host holds the first h
+needs u = floor(n/b) - floor(h/b) new full chunks and save(r) = not (p_t and u > kappa),
+decided once per request.  p_t is 0 for plain offload (write-all), 1 for fixed write
+admission, and the pressure signal of Eq. 10 for capacity-conditioned admission:
+p_t = [ (A_t - 1) N_t beta > C_H ] and [ o_t >= theta and e_t > 0 ].  Copy-time
+deduplication falls out of the model: a resident chunk is a hit and is never copied.
+
+Readings taken where the paper is silent (integers only, virtual time in ms):
+  * windows are (now - W, now]; A_t counts distinct agents with a request in the window
+    including the current one; N_t is the mean of the last <= 256 prompt lengths
+    including the current one; e_t counts capacity evictions in the window before the
+    current request inserts anything; o_t uses the resident count at that same moment;
+  * C_H is taken as K_H * b * beta, so beta cancels: (A_t-1) * sum_len > K_H * b * count;
+  * slots come from a free stack that first yields 0, 1, 2, ...; an evicted chunk's slot
+    is the next one handed out;
+  * a request with more full chunks than K_H is refused and changes nothing.
+"""
+from collections import OrderedDict, deque
+
+WRITE_ALL = 0
+FILTER_FIXED = 1
+FILTER_CONDITIONED = 2
+
+
+class CapacityError(Exception):
+    pass
+
+
+class StepResult:
+    __slots__ = ("hit", "admit", "slot", "evicted", "save", "pressure", "new_chunks",
+                 "host_prefix_blocks")
+
+    def __init__(self):
+        self.hit = []
+        self.admit = []
+        self.slot = []
+        self.evicted = []        # (key, slot) in eviction order
+        self.save = True
+        self.pressure = False
+        self.new_chunks = 0
+        self.host_prefix_blocks = 0
+
+
+class HostTier:
+    def __init__(self, capacity_blocks, block_size, policy=WRITE_ALL, kappa_blocks=8,
+                 theta_percent=95, window_ms=60_000, len_window=256, telemetry=True):
+        self.K = int(capacity_blocks)
+        self.b = int(block_size)
+        self.policy = policy
+        self.kappa = int(kappa_blocks)
+        self.theta_percent = int(theta_percent)
+        self.window_ms = int(window_ms)
+        self.telemetry = telemetry
+        self.order = OrderedDict()                    # key -> slot, least recent first
+        self.free = list(range(self.K - 1, -1, -1))   # pop() yields 0, 1, 2, ...
+        self.agent_last = {}                          # agent -> time of latest request
+        self.lengths = deque(maxlen=int(len_window))
+        self.evict_times = deque()
+        self.stats = dict(requests=0, references=0, hits=0, admitted=0, declined=0,
+                          evicted=0, declined_requests=0, pressure_requests=0)
+
+    # ---- lookups that do not change recency -------------------------------------------
+    def __contains__(self, key):
+        return key in self.order
+
+    def slot_of(self, key):
+        return self.order[key]
+
+    def leading_run(self, keys):
+        n = 0
+        for k in keys:
+            if k not in self.order:
+                break
+            n += 1
+        return n
+
+    # ---- Eq. 10 ---------------------------------------------------------------------------
+    def _pressure(self, agent, n_tokens, now_ms):
+        self.agent_last[agent] = now_ms
+        self.lengths.append(int(n_tokens))
+        lo = now_ms - self.window_ms
+        while self.evict_times and self.evict_times[0] <= lo:
+            self.evict_times.popleft()
+        if self.policy == WRITE_ALL:
+            return False
+        if self.policy == FILTER_FIXED:
+            return True
+        active = sum(1 for t in self.agent_last.values() if t > lo)
+        estimate_exceeds = (active - 1) * sum(self.lengths) > self.K * self.b * len(self.lengths)
+        if not self.telemetry:
+            return estimate_exceeds
+        full = 100 * len(self.order) >= self.theta_percent * self.K
+        evicting = len(self.evict_times) > 0
+        return estimate_exceeds and full and evicting
+
+    # ---- one request ----------------------------------------------------------------------
+    def step(self, keys, n_tokens, agent, now_ms):
+        if len(keys) > self.K:
+            raise CapacityError("request references more blocks than the tier holds")
+        res = StepResult()
+        H = self.leading_run(keys)
+        res.host_prefix_blocks = H
+        res.pressure = self._pressure(agent, n_tokens, now_ms)
+        res.new_chunks = n_tokens // self.b - (H * self.b) // self.b
+        res.save = not (res.pressure and res.new_chunks > self.kappa)
+        st = self.stats
+        st["requests"] += 1
+        st["pressure_requests"] += int(res.pressure)
+        st["declined_requests"] += int(not res.save)
+        for k in keys:
+            st["references"] += 1
+            if k in self.order:
+                self.order.move_to_end(k)
+                res.hit.append(1); res.admit.append(0); res.slot.append(self.order[k])
+                st["hits"] += 1
+            elif res.save:
+                if len(self.order) >= self.K:
+                    vk, vs = self.order.popitem(last=False)
+                    self.free.append(vs)
+                    res.evicted.append((vk, vs))
+                    self.evict_times.append(now_ms)
+                    st["evicted"] += 1
+                s = self.free.pop()
+                self.order[k] = s
+                res.hit.append(0); res.admit.append(1); res.slot.append(s)
+                st["admitted"] += 1
+            else:
+                res.hit.append(0); res.admit.append(0); res.slot.append(-1)
+                st["declined"] += 1
+        return res
+
+
+def simulate_stream(stream, capacity, declined=frozenset()):
+    """Bare reference model over a flat stream of chunk keys.  ``declined`` holds the
+    reference indices whose miss is not inserted.  Returns the list of hit flags."""
+    order = OrderedDict()
+    hits = []
+    for i, k in enumerate(stream):
+        if k in order:
+            order.move_to_end(k)
+            hits.append(True)
+            continue
+        hits.append(False)
+        if i in declined:
+            continue
+        if len(order) >= capacity:
+            order.popitem(last=False)
+        order[k] = True
+    return hits

@@ -1,0 +1,132 @@
+"""Whole-trace driver: what one agent turn does to the two tiers and to the KV bytes.
+
+Per request (Section 4 and Appendix D for the order: lookup first, restore before
+compute, store after): hash the prompt's full blocks; G / H = leading runs resident in
+the GPU index / host tier; run the host-tier step (promotions, admission, insertions);
+reference the same keys in the GPU tier (harness-owned LRU of K_G blocks, ascending
+order, fresh blocks from a free stack, a partial tail takes a temporary block);
+load the host-covered blocks [G, H) into their GPU blocks; "prefill" = fill every block
+at or beyond max(G, H) that was not already GPU-resident with its payload; store the
+admitted blocks to their host slots.
+
+The GPU tier is never specified by the paper (it belongs to the serving engine); the
+model above is this build's reading.  KV payloads are a function of (block key, piece).
+"""
+from collections import OrderedDict
+
+import numpy as np
+
+from . import hash as ohash
+from . import storeload
+from .tier import HostTier
+
+
+class GpuTier:
+    """LRU of keyed GPU blocks with a free stack that first yields 0, 1, 2, ..."""
+
+    def __init__(self, num_blocks):
+        self.NB = int(num_blocks)
+        self.order = OrderedDict()                 # key -> block id, least recent first
+        self.free = list(range(self.NB - 1, -1, -1))
+
+    def __contains__(self, key):
+        return key in self.order
+
+    def _alloc(self):
+        if not self.free:
+            _, vb = self.order.popitem(last=False)
+            self.free.append(vb)
+        return self.free.pop()
+
+    def step(self, keys, need_tail):
+        """Reference ``keys`` in order.  Returns (was_resident[], block_id[], tail_block)."""
+        if len(keys) + int(need_tail) > self.NB:
+            raise ValueError("request does not fit the GPU cache")
+        resident, ids = [], []
+        for k in keys:
+            if k in self.order:
+                self.order.move_to_end(k)
+                resident.append(1)
+                ids.append(self.order[k])
+            else:
+                blk = self._alloc()
+                self.order[k] = blk
+                resident.append(0)
+                ids.append(blk)
+        tail = self._alloc() if need_tail else -1
+        return resident, ids, tail
+
+    def release(self, block_id):
+        if block_id >= 0:
+            self.free.append(block_id)
+
+
+class TraceOracle:
+    def __init__(self, shape, gpu_blocks, host_blocks, policy=0, kappa_blocks=8,
+                 theta_percent=95, window_ms=60_000, len_window=256, telemetry=True,
+                 payload=None, hash_base=ohash.HASH_BASE, hash_seed=ohash.HASH_SEED):
+        """``payload(keys, q, n_words) -> uint16[len(keys), n_words]`` enables full-bytes
+        mode (pool and tier held in numpy); None runs metadata only."""
+        self.shape = shape
+        self.b = shape.block_size
+        self.gpu = GpuTier(gpu_blocks)
+        self.host = HostTier(host_blocks, self.b, policy, kappa_blocks, theta_percent,
+                             window_ms, len_window, telemetry)
+        self.payload = payload
+        self.hash_base, self.hash_seed = hash_base, hash_seed
+        self.pool = self.tier = None
+        if payload is not None:
+            P = shape.piece_bytes
+            self.pool = [np.zeros((gpu_blocks, P), dtype=np.uint8)
+                         for _ in range(shape.pieces_per_block)]
+            self.tier = np.zeros((host_blocks, shape.pieces_per_block, P), dtype=np.uint8)
+        self.records = []
+        self.totals = dict(prompt_tokens=0, fresh_tokens=0, loaded_blocks=0, stored_blocks=0,
+                           gpu_hit_blocks=0, host_hit_blocks=0)
+
+    def turn(self, tokens, agent, now_ms):
+        n = len(tokens)
+        keys = ohash.hash_blocks(tokens, self.b, self.hash_seed, self.hash_base)
+        G = 0
+        for k in keys:
+            if k not in self.gpu:
+                break
+            G += 1
+        H = self.host.leading_run(keys)
+        host_slots = [self.host.slot_of(k) for k in keys[:H]]
+        res = self.host.step(keys, n, agent, now_ms)
+        resident, gpu_ids, tail = self.gpu.step(keys, n % self.b != 0)
+        cover = max(G, H)
+        lo, hi = (G, H) if H > G else (G, G)
+        fill = [j for j in range(cover, len(keys)) if not resident[j]]
+        if self.payload is not None:
+            storeload.load(self.pool, self.tier, host_slots[lo:hi], gpu_ids[lo:hi])
+            if fill:
+                W = self.shape.piece_bytes // 2
+                for q in range(self.shape.pieces_per_block):
+                    words = self.payload([keys[j] for j in fill], q, W)
+                    for r, j in enumerate(fill):
+                        self.pool[q][gpu_ids[j], :] = words[r].view(np.uint8)
+            storeload.store(self.pool, self.tier, gpu_ids, res.admit, res.slot)
+        self.gpu.release(tail)
+        rec = dict(agent=agent, now_ms=now_ms, n_tokens=n, keys=keys, G=G, H=H,
+                   new_chunks=res.new_chunks, pressure=res.pressure, save=res.save,
+                   hit=res.hit, admit=res.admit, slot=res.slot, evicted=res.evicted,
+                   gpu_resident=resident, gpu_block=gpu_ids, loaded=hi - lo,
+                   stored=sum(res.admit), fresh_tokens=n - cover * self.b, filled=len(fill))
+        t = self.totals
+        t["prompt_tokens"] += n
+        t["fresh_tokens"] += rec["fresh_tokens"]
+        t["loaded_blocks"] += rec["loaded"]
+        t["stored_blocks"] += rec["stored"]
+        t["gpu_hit_blocks"] += G
+        t["host_hit_blocks"] += H
+        self.records.append(rec)
+        return rec
+
+    def run(self, trace, limit=None):
+        for i, req in enumerate(trace.requests):
+            if limit is not None and i >= limit:
+                break
+            self.turn(trace.prompt(req), req.agent, req.time_ms)
+        return self.records

@@ -1,0 +1,269 @@
+"""Pins for oracle.tier and oracle.stackdist: Mattson inclusion (Eq. 4), Lemma 1,
+Proposition 1 and the write rule (Eq. 6 / Eq. 10), against brute force on tiny traces.
+The brute-force LRU below is written differently on purpose (timestamps + linear scan).
+"""
+import math
+import random
+
+import pytest
+
+from oracle import stackdist as sd
+from oracle import tier as ot
+
+
+def brute_lru(stream, K, declined=frozenset()):
+    """LRU by last-use timestamps; returns (hits, promoted_flags)."""
+    last_use = {}            # resident key -> timestamp of last promotion
+    hits, promoted = [], []
+    for i, k in enumerate(stream):
+        if k in last_use:
+            hits.append(True); promoted.append(True)
+            last_use[k] = i
+            continue
+        hits.append(False)
+        if i in declined:
+            promoted.append(False)
+            continue
+        if len(last_use) >= K:
+            victim = min(last_use, key=lambda x: last_use[x])
+            del last_use[victim]
+        last_use[k] = i
+        promoted.append(True)
+    return hits, promoted
+
+
+def rand_stream(rng, T, U):
+    return [rng.randrange(U) for _ in range(T)]
+
+
+def test_reuse_distance_hand_case():
+    #          a  b  c  a  b  b  d  c  a
+    stream = [1, 2, 3, 1, 2, 2, 4, 3, 1]
+    expect = [math.inf, math.inf, math.inf, 2, 2, 0, math.inf, 3, 3]
+    assert sd.reuse_distances_definition(stream) == expect
+    assert sd.reuse_distances(stream) == expect
+
+
+def test_fast_distances_equal_definition():
+    rng = random.Random(5)
+    for _ in range(100):
+        s = rand_stream(rng, rng.randrange(0, 80), rng.randrange(1, 15))
+        assert sd.reuse_distances(s) == sd.reuse_distances_definition(s)
+
+
+def test_mattson_inclusion_and_monotone_hits():
+    rng = random.Random(6)
+    for _ in range(150):
+        s = rand_stream(rng, rng.randrange(1, 120), rng.randrange(1, 20))
+        D = sd.reuse_distances(s)
+        prev = None
+        for K in range(1, 22):
+            model = ot.simulate_stream(s, K)
+            brute, _ = brute_lru(s, K)
+            assert model == brute
+            assert model == sd.predicted_hits(D, K)            # hit  <=>  D < K
+            if prev is not None:                                 # inclusion: hits grow with K
+                assert all((not p) or m for p, m in zip(prev, model))
+            prev = model
+        # a tier that holds everything hits every re-reference
+        assert ot.simulate_stream(s, 10**9) == [d != math.inf for d in D]
+        assert sd.working_set_full(D) == (max([d for d in D if d != math.inf], default=-1) + 1)
+
+
+def test_lemma1_resident_iff_promotions_below_capacity():
+    rng = random.Random(7)
+    for _ in range(300):
+        s = rand_stream(rng, rng.randrange(2, 60), rng.randrange(2, 10))
+        K = rng.randrange(1, 8)
+        declined = {i for i in range(len(s)) if rng.random() < 0.3}
+        hits, promoted = brute_lru(s, K, declined)
+        assert hits == ot.simulate_stream(s, K, declined)
+        for t, y in enumerate(s):
+            prev = [i for i in range(t) if s[i] == y]
+            if not prev:
+                continue
+            sref = prev[-1]
+            if not promoted[sref]:
+                continue
+            P = len({s[i] for i in range(sref + 1, t) if promoted[i] and s[i] != y})
+            assert hits[t] == (P < K)
+
+
+def test_proposition1_declinable_writes_lose_no_hit():
+    rng = random.Random(8)
+    for _ in range(300):
+        s = rand_stream(rng, rng.randrange(2, 70), rng.randrange(2, 12))
+        K = rng.randrange(1, 8)
+        D = sd.reuse_distances(s)
+        # next-reference distance of every reference (inf if never referenced again)
+        nxt = [math.inf] * len(s)
+        last = {}
+        for i, k in enumerate(s):
+            if k in last:
+                nxt[last[k]] = D[i]
+            last[k] = i
+        full = ot.simulate_stream(s, K)
+        eligible = [i for i in range(len(s)) if nxt[i] >= K]
+        declined = {i for i in eligible if rng.random() < 0.6}
+        restricted = ot.simulate_stream(s, K, declined)
+        assert all((not f) or r for f, r in zip(full, restricted))
+        assert sum(restricted) >= sum(full)
+
+
+def test_proposition1_coverage_never_shrinks():
+    rng = random.Random(9)
+    for _ in range(100):
+        # requests = prefixes of a few "agents", so coverage (leading run) is meaningful
+        reqs = []
+        for _ in range(rng.randrange(2, 10)):
+            a = rng.randrange(3)
+            n = rng.randrange(1, 8)
+            reqs.append([(a, j) for j in range(n)])
+        s = [k for r in reqs for k in r]
+        K = rng.randrange(1, 10)
+        D = sd.reuse_distances(s)
+        nxt = [math.inf] * len(s)
+        last = {}
+        for i, k in enumerate(s):
+            if k in last:
+                nxt[last[k]] = D[i]
+            last[k] = i
+        declined = {i for i in range(len(s)) if nxt[i] >= K and rng.random() < 0.5}
+        full = ot.simulate_stream(s, K)
+        rest = ot.simulate_stream(s, K, declined)
+        pos = 0
+        for r in reqs:
+            cf = sd.request_coverage(full[pos:pos + len(r)])
+            cr = sd.request_coverage(rest[pos:pos + len(r)])
+            assert cr >= cf
+            pos += len(r)
+
+
+def run_requests(tier, reqs, b=4):
+    out = []
+    for i, (agent, keys) in enumerate(reqs):
+        out.append(tier.step(keys, len(keys) * b + 1, agent, i * 1000))
+    return out
+
+
+def test_host_tier_equals_stream_model_under_write_all():
+    rng = random.Random(10)
+    for _ in range(100):
+        reqs = [(rng.randrange(4), [(a, j) for j in range(rng.randrange(0, 7))])
+                for a in [rng.randrange(4) for _ in range(rng.randrange(1, 12))]]
+        K = rng.randrange(7, 15)
+        t = ot.HostTier(K, 4)
+        res = run_requests(t, reqs)
+        s = [k for _, keys in reqs for k in keys]
+        flat = [h for r in res for h in r.hit]
+        assert [bool(h) for h in flat] == ot.simulate_stream(s, K)
+        # admit = miss (write-all), dedup = resident chunks are never copied
+        assert all(a == 1 - h for r in res for a, h in zip(r.admit, r.hit))
+        # slots of resident keys are unique and in range
+        slots = list(t.order.values())
+        assert len(set(slots)) == len(slots) and all(0 <= x < K for x in slots)
+        assert len(slots) + len(t.free) == K
+
+
+def test_slot_assignment_free_stack():
+    t = ot.HostTier(3, 4)
+    r = t.step(["a", "b", "c"], 13, 0, 0)
+    assert r.slot == [0, 1, 2] and r.evicted == []
+    r = t.step(["d"], 5, 1, 1)                 # evicts "a" (least recent), reuses slot 0
+    assert r.evicted == [("a", 0)] and r.slot == [0] and r.admit == [1]
+    r = t.step(["b", "e"], 9, 0, 2)            # b hits (slot 1); e evicts c (slot 2)
+    assert r.hit == [1, 0] and r.slot == [1, 2] and r.evicted == [("c", 2)]
+    assert r.host_prefix_blocks == 1 and r.new_chunks == 1
+
+
+def test_isolated_resident_chunk_hits_but_does_not_extend_coverage():
+    t = ot.HostTier(8, 4)
+    t.step(["a", "b", "c"], 12, 0, 0)
+    r = t.step(["a", "x", "c"], 12, 0, 1)
+    assert r.host_prefix_blocks == 1
+    assert r.hit == [1, 0, 1] and r.admit == [0, 1, 0]
+    assert r.new_chunks == 2
+
+
+def test_capacity_error_changes_nothing():
+    t = ot.HostTier(2, 4)
+    t.step(["a"], 4, 0, 0)
+    before = (list(t.order.items()), list(t.free), dict(t.stats))
+    with pytest.raises(ot.CapacityError):
+        t.step(["p", "q", "r"], 12, 0, 1)
+    assert before == (list(t.order.items()), list(t.free), dict(t.stats))
+
+
+def test_write_rule_endpoints_and_threshold():
+    keys = lambda a, n: [(a, j) for j in range(n)]
+    # u = floor(n/b) - floor(h/b): 10 blocks, host holds first 4 -> u = 6
+    for kappa, expect_save in [(5, False), (6, True), (7, True)]:
+        t = ot.HostTier(64, 4, policy=ot.FILTER_FIXED, kappa_blocks=kappa)
+        t.step(keys(0, 4), 16, 0, 0)           # u = 4 <= kappa: saved
+        assert all(k in t for k in keys(0, 4))
+        r = t.step(keys(0, 10), 43, 0, 1)
+        assert r.new_chunks == 6 and r.pressure and r.save == expect_save
+        assert r.hit[:4] == [1] * 4
+        assert r.admit[4:] == [int(expect_save)] * 6
+        if not expect_save:
+            assert r.slot[4:] == [-1] * 6 and r.evicted == []
+    # fixed admission: a long first prompt is declined, and stays declined as u only grows
+    t = ot.HostTier(64, 4, policy=ot.FILTER_FIXED, kappa_blocks=8)
+    for turn, n in enumerate([9, 10, 12]):
+        r = t.step(keys(1, n), n * 4, 1, turn)
+        assert not r.save and sum(r.admit) == 0
+    assert len(t.order) == 0
+    # kappa = infinity reproduces write-all; p == 0 reproduces write-all
+    rng = random.Random(11)
+    reqs = [(a, keys(a, rng.randrange(1, 9))) for a in [rng.randrange(3) for _ in range(30)]]
+    base = run_requests(ot.HostTier(10, 4), reqs)
+    for pol, kap in [(ot.FILTER_FIXED, 10**9), (ot.FILTER_CONDITIONED, 10**9), (ot.WRITE_ALL, 0)]:
+        other = run_requests(ot.HostTier(10, 4, policy=pol, kappa_blocks=kap), reqs)
+        assert [(r.hit, r.admit, r.slot, r.evicted) for r in base] == \
+               [(r.hit, r.admit, r.slot, r.evicted) for r in other]
+
+
+def test_conditioned_pressure_needs_estimate_and_full_evicting_tier():
+    b = 4
+    keys = lambda a, lo, hi: [(a, j) for j in range(lo, hi)]
+    # K = 8 blocks = 32 tokens of capacity.  Two agents with 5-block prompts: estimate
+    # (A-1)*mean = 1*20 tokens <= 32 -> never pressure, even once the tier evicts.
+    t = ot.HostTier(8, b, policy=ot.FILTER_CONDITIONED, kappa_blocks=2)
+    for i in range(6):
+        r = t.step(keys(i % 2, 0, 5) if i < 2 else keys(i, 0, 5), 20, i % 2, i)
+        assert not r.pressure and r.save
+    assert t.stats["evicted"] > 0
+    # Three agents with 5-block prompts: estimate 2*20 = 40 > 32.  Pressure engages only
+    # after the tier is >= 95 % full AND has evicted inside the window.
+    t = ot.HostTier(8, b, policy=ot.FILTER_CONDITIONED, kappa_blocks=2)
+    r0 = t.step(keys(0, 0, 5), 20, 0, 0)       # A=1: estimate 0
+    r1 = t.step(keys(1, 0, 5), 20, 1, 1)       # A=2: 20 <= 32; evicts 2 while inserting
+    r2 = t.step(keys(2, 0, 5), 20, 2, 2)       # A=3: 40 > 32, tier full (8/8), e_t = 2 > 0
+    assert (r0.pressure, r1.pressure, r2.pressure) == (False, False, True)
+    assert r1.evicted and len(r1.evicted) == 2
+    assert not r2.save and sum(r2.admit) == 0 and r2.new_chunks == 5
+    # a small extension of a resident prefix is still saved under pressure
+    r3 = t.step(keys(1, 0, 6), 24, 1, 3)
+    assert r3.pressure and r3.host_prefix_blocks == 5 and r3.new_chunks == 1 and r3.save
+    assert r3.admit == [0, 0, 0, 0, 0, 1]
+    # evictions older than the window no longer count: pressure subsides
+    r4 = t.step(keys(2, 0, 5), 20, 2, 3 + 60_000)
+    assert not r4.pressure and r4.save
+    # agents outside the window drop out of A_t (only agent 2 is recent now)
+    assert sum(1 for v in t.agent_last.values() if v > 3 + 60_000 - t.window_ms) == 1
+
+
+def test_conditioned_without_telemetry_uses_estimate_alone():
+    b = 4
+    keys = lambda a: [(a, j) for j in range(5)]
+    t = ot.HostTier(8, b, policy=ot.FILTER_CONDITIONED, kappa_blocks=2, telemetry=False)
+    flags = [t.step(keys(a), 20, a, a).pressure for a in range(3)]
+    assert flags == [False, False, True]      # third request: 2*20 > 32 although nothing evicted
+    assert len(t.order) == 8 or len(t.order) == 10 - 2
+
+
+def test_length_window_keeps_last_256():
+    t = ot.HostTier(4, 4, policy=ot.FILTER_CONDITIONED, len_window=3)
+    for i, n in enumerate([100, 200, 300, 400]):
+        t.step([], n, 0, i)
+    assert list(t.lengths) == [200, 300, 400]
