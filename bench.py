@@ -1,0 +1,529 @@
+#!/usr/bin/env python
+"""Benchmark of the paged-KV offload hot path on B200 (store/load microbench workload with
+Qwen3-30B-A3B-shaped KV: 48 layers, 4 KV heads, head_dim 128, bf16, block 16).
+
+One step = one pass of the whole path over one batch: two requests of `--blocks` blocks
+each.  Request 1 resubmits the previous step's prompt (its KV is host-resident and gone
+from the GPU): hash -> match -> tier step (all hits) -> load every block into freshly
+drawn, uniform-random pool blocks.  Request 2 is a new prompt: hash -> match (nothing) ->
+tier step (every block admitted, evicting the oldest prompt) -> store from uniform-random
+pool blocks.  Bytes moved per step = 2 * blocks * 1.5 MiB.
+
+  value  whole-step GB/s with the tier in HBM and tokens resident on the device (the
+         on-device gather/scatter, HBM roofline);
+  e2e    the same step through the same calls with the tier in pinned host memory and the
+         tokens in pinned host memory (host-link roofline; H2D/D2H bytes inside the timing).
+
+`--impl reference` times the CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "kv_store_load_gbps"
+UNIT = "GB/s"
+WORKLOAD = "c1_store_load_microbench_qwen3_30b_a3b"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="eakv", choices=["eakv", "reference"])
+    ap.add_argument("--blocks", type=int, default=4096, help="blocks per request")
+    ap.add_argument("--pool-blocks", type=int, default=65536)
+    ap.add_argument("--link", default="staged", choices=["zero_copy", "staged"],
+                    help="host-link strategy of the e2e arm")
+    ap.add_argument("--copy-path", default="vector", choices=["vector", "bulk"])
+    ap.add_argument("--copy-ctas", type=int, default=0)
+    ap.add_argument("--host-ctas", type=int, default=0)
+    ap.add_argument("--staging-mib", type=int, default=64)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--sweep", action="store_true",
+                    help="also print the 1..4096-block curve (contiguous/random ids, masks)")
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------
+# the step
+# ------------------------------------------------------------------------------------------
+class Arm:
+    """One configuration of the path (device tier or pinned-host tier) over a shared pool."""
+
+    def __init__(self, args, pool, shape, torch, eakv, *, host_tier, device):
+        self.torch, self.eakv = torch, eakv
+        self.m = args.blocks
+        self.b = shape.block_size
+        self.n_tokens = self.m * self.b
+        self.host_tier = host_tier
+        self.device = device
+        kw = dict(copy_path=eakv.COPY_BULK if args.copy_path == "bulk" else eakv.COPY_VECTOR,
+                  max_call_blocks=max(16384, self.m))
+        if host_tier:
+            kw.update(tier_location=eakv.TIER_PINNED_HOST,
+                      link_strategy=eakv.LINK_STAGED if args.link == "staged" else eakv.LINK_ZERO_COPY,
+                      staging_bytes=args.staging_mib << 20, copy_ctas=args.host_ctas)
+            if args.link == "staged":
+                kw["copy_ctas"] = args.copy_ctas
+        else:
+            # the tier is a tensor of ours that the context adopts, so it can be inspected
+            self.tier_t = torch.empty((2 * self.m, shape.pieces_per_block, shape.piece_bytes // 2),
+                                      dtype=torch.int16, device=device)
+            kw.update(tier_location=eakv.TIER_DEVICE, link_strategy=eakv.LINK_ZERO_COPY,
+                      copy_ctas=args.copy_ctas, tier_memory=self.tier_t.data_ptr())
+        self.ctx = eakv.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads,
+                                head_dim=shape.head_dim, block_size=shape.block_size,
+                                gpu_blocks=pool.gpu_blocks, host_blocks=2 * self.m,
+                                kv_base=pool.kv_base, **kw)
+        self.block_bytes = self.ctx.block_bytes
+        self.stream = torch.cuda.current_stream(device)
+        self.seed = self.ctx.eakv_hash_seed()
+        self.keys_dev = torch.empty(self.m, dtype=torch.int64, device=device)
+        self.keys_host = torch.empty(self.m, dtype=torch.int64).pin_memory()
+        self.tok_dev = torch.empty(self.n_tokens, dtype=torch.int32, device=device)
+        self.kernel_ms = []          # (bytes, ms) per timed store/load launch
+        self.h2d = self.d2h = 0
+
+    def request(self, tokens, table, agent, now, timed_events=None):
+        """tokens: device int32 tensor (device arm) or pinned host tensor (e2e arm)."""
+        torch = self.torch
+        if tokens.device.type == "cpu":
+            self.tok_dev.copy_(tokens, non_blocking=True)
+            self.h2d += tokens.numel() * 4
+            tok = self.tok_dev
+        else:
+            tok = tokens
+        nblk = self.ctx.eakv_hash_blocks(tok.data_ptr(), self.n_tokens, self.seed,
+                                         self.keys_dev.data_ptr(), self.stream)
+        self.keys_host.copy_(self.keys_dev, non_blocking=True)
+        self.stream.synchronize()
+        self.d2h += nblk * 8
+        keys = self.keys_host.numpy().view(np.uint64)
+        G, H, _, slots = self.ctx.eakv_match(keys)
+        step = self.ctx.eakv_tier_step(keys, agent, self.n_tokens, now)
+        ev = None
+        if timed_events is not None:
+            ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+            ev[0].record(self.stream)
+        moved = 0
+        if H > 0:
+            self.ctx.eakv_load(slots[:H], table[:H], self.stream)
+            moved += H * self.block_bytes
+            self.h2d += H * self.block_bytes if self.host_tier else 0
+        n_admit = int(step["admit"].sum())
+        if n_admit:
+            self.ctx.eakv_store(table, step["admit"], step["slot"], self.stream)
+            moved += n_admit * self.block_bytes
+            self.d2h += n_admit * self.block_bytes if self.host_tier else 0
+        if ev is not None:
+            ev[1].record(self.stream)
+            timed_events.append((moved, ev))
+        return moved, H, n_admit
+
+    def step(self, s, prompts, tables, timed_events=None):
+        """prompts[s-1] was stored by the previous step; prompts[s] is new."""
+        moved = 0
+        a, _, _ = self.request(prompts[s - 1], tables[2 * s], agent=(s - 1) % 2, now=s * 1000,
+                               timed_events=timed_events)
+        b, _, _ = self.request(prompts[s], tables[2 * s + 1], agent=s % 2, now=s * 1000 + 500,
+                               timed_events=timed_events)
+        return a + b
+
+
+def run_arm(arm, prompts, tables, steps, warmup, dist, clocks=None):
+    torch = arm.torch
+    # prime: store prompt 0 so that step 1 has something to restore
+    arm.request(prompts[0], tables[0], agent=0, now=0)
+    for s in range(1, warmup + 1):
+        arm.step(s, prompts, tables)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    arm.h2d = arm.d2h = 0
+    launches0 = arm.ctx.eakv_get_stats()["kernel_launches"]
+    timed = []
+    if clocks:
+        clocks.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(arm.stream)
+    moved = 0
+    for s in range(warmup + 1, warmup + 1 + steps):
+        moved += arm.step(s, prompts, tables, timed_events=timed)
+    e1.record(arm.stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    clk = clocks.stop() if clocks else None
+    if dist is not None:
+        dist.barrier()
+    launches = arm.ctx.eakv_get_stats()["kernel_launches"] - launches0
+    kernel = [(b, ev[0].elapsed_time(ev[1])) for b, ev in timed if b > 0]
+    return dict(ms=ms, moved=moved, launches=launches, kernel=kernel, clocks=clk,
+                h2d=arm.h2d / steps, d2h=arm.d2h / steps)
+
+
+def pinned_link_peak(torch, device, gib=1, reps=5):
+    n = gib << 30
+    host = torch.empty(n, dtype=torch.uint8).pin_memory()
+    dev = torch.empty(n, dtype=torch.uint8, device=device)
+    out = {}
+    for name, (dst, src) in (("h2d", (dev, host)), ("d2h", (host, dev))):
+        best = 0.0
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); dst.copy_(src, non_blocking=True); e1.record()
+            torch.cuda.synchronize()
+            best = max(best, n / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+        out[name] = best
+    # both directions at once on two streams
+    s1, s2 = torch.cuda.Stream(device), torch.cuda.Stream(device)
+    host2 = torch.empty(n, dtype=torch.uint8).pin_memory()
+    dev2 = torch.empty(n, dtype=torch.uint8, device=device)
+    best = 0.0
+    for _ in range(reps):
+        torch.cuda.synchronize()
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        s1.wait_stream(torch.cuda.current_stream()); s2.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s1):
+            dev.copy_(host, non_blocking=True)
+        with torch.cuda.stream(s2):
+            host2.copy_(dev2, non_blocking=True)
+        torch.cuda.current_stream().wait_stream(s1); torch.cuda.current_stream().wait_stream(s2)
+        t1.record()
+        torch.cuda.synchronize()
+        best = max(best, 2 * n / (t0.elapsed_time(t1) * 1e-3) / 1e9)
+    out["bidir"] = best
+    return out
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle arm
+# ------------------------------------------------------------------------------------------
+def oracle_step_rate(seconds, blocks=128, pool_blocks=512, steps_cap=10**9):
+    """The oracle, as it stands, on the same step with `blocks` blocks per request and a
+    host-resident pool of `pool_blocks`; returns (GB/s, steps run, seconds)."""
+    from eakv_workloads import SHAPES
+    from oracle import hash as ohash, storeload
+    from oracle.tier import HostTier
+    shape = SHAPES["qwen3_30b_a3b"]
+    rng = np.random.default_rng(1)
+    b, P, Q = shape.block_size, shape.piece_bytes, shape.pieces_per_block
+    pool = [rng.integers(0, 256, size=(pool_blocks, P), dtype=np.uint8) for _ in range(Q)]
+    tier_mem = np.zeros((2 * blocks, Q, P), dtype=np.uint8)
+    tier = HostTier(2 * blocks, b)
+    prompts = {}
+
+    def prompt(s):
+        if s not in prompts:
+            prompts[s] = rng.integers(0, 151936, size=blocks * b, dtype=np.int32)
+        return prompts[s]
+
+    def request(tokens, table, agent, now):
+        keys = ohash.hash_blocks(tokens.tolist(), b)
+        H = tier.leading_run(keys)
+        slots = [tier.slot_of(k) for k in keys[:H]]
+        res = tier.step(keys, len(tokens), agent, now)
+        storeload.load(pool, tier_mem, slots, table[:H])
+        storeload.store(pool, tier_mem, table, res.admit, res.slot)
+        return (H + sum(res.admit)) * shape.block_bytes
+
+    request(prompt(0), rng.permutation(pool_blocks)[:blocks], 0, 0)
+    t0 = time.perf_counter()
+    moved, s = 0, 0
+    while True:
+        s += 1
+        moved += request(prompt(s - 1), rng.permutation(pool_blocks)[:blocks], (s - 1) % 2, s * 1000)
+        moved += request(prompt(s), rng.permutation(pool_blocks)[:blocks], s % 2, s * 1000 + 500)
+        prompts.pop(s - 1, None)
+        dt = time.perf_counter() - t0
+        if dt >= seconds or s >= steps_cap:
+            break
+    return moved / dt / 1e9, s, dt
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    blocks = 128
+    # warm-up steps, then K timed steps of the bounded sample
+    oracle_step_rate(0.0, blocks=blocks, steps_cap=max(1, min(args.warmup, 2)))
+    gbps, steps, dt = oracle_step_rate(1e9, blocks=blocks, steps_cap=args.steps)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbps, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+        "data": "synthetic", "gpu_launches": 0,
+        "config": {"workload": WORKLOAD, "blocks_per_request": blocks,
+                   "note": "CPU oracle on a bounded sample of the step (128 blocks per request)"},
+        "cpu_baseline": {"value": gbps, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"{steps} steps x 2 requests x {blocks} blocks (1.5 MiB each)"},
+        "e2e": {"value": gbps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from eakv_workloads import SHAPES
+    from paper_2609_33762_b200 import eakv
+    from paper_2609_33762_b200.harness import PagedPool
+    from paper_2609_33762_b200.multi import aggregate_over_ranks, init_distributed
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the eakv path has no CPU fallback")
+    if not os.path.exists(os.path.join(ROOT, "paper_2609_33762_b200", "libeakv.so")):
+        from paper_2609_33762_b200 import build
+        build.build()
+    eakv.lib()
+
+    rank, world, local_rank, dist = init_distributed(args.gpus)
+    device = torch.device(f"cuda:{local_rank}")
+    torch.cuda.set_device(device)
+    shape = SHAPES["qwen3_30b_a3b"]
+    m = args.blocks
+
+    # paged pool, as large as fits (200k blocks = 293 GiB do not fit one GPU)
+    free, _total = torch.cuda.mem_get_info(device)
+    reserve = 2 * m * shape.block_bytes + (4 << 30) + 2 * (args.staging_mib << 20) * 2
+    nb = min(args.pool_blocks, int((free - reserve) // shape.block_bytes))
+    nb = max(nb, 2 * m)
+    pool = PagedPool(shape, nb, device, fill=lambda q, t: t.random_())
+    torch.cuda.synchronize()
+
+    total_steps = args.steps + args.warmup + 1
+    rng = np.random.default_rng(1 + rank)
+    tok_np = rng.integers(0, 151936, size=(total_steps + 1, m * shape.block_size), dtype=np.int32)
+    prompts_dev = [torch.from_numpy(tok_np[i]).to(device) for i in range(total_steps + 1)]
+    prompts_host = [torch.from_numpy(tok_np[i]).pin_memory() for i in range(total_steps + 1)]
+    # fresh uniform-random block ids per request, without replacement
+    tables = [rng.permutation(nb)[:m].astype(np.int32) for _ in range(2 * total_steps + 2)]
+
+    clocks = ClockSampler(local_rank) if rank == 0 else None
+
+    # ---- device-resident arm (value) ----
+    arm = Arm(args, pool, shape, torch, eakv, host_tier=False, device=device)
+    r = run_arm(arm, prompts_dev, tables, args.steps, args.warmup, dist, clocks)
+    check_ok = self_check(torch, arm, pool, tables, args, shape)
+    arm.ctx.close()
+    del arm
+    ms_max, moved_sum = aggregate_over_ranks(dist, r["ms"], r["moved"], device)
+    value = moved_sum / (ms_max * 1e-3) / 1e9
+
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    else:
+        peak, peak_src = 6650.0, "fallback"
+    kb = sum(b for b, _ in r["kernel"])
+    kms = sum(t for _, t in r["kernel"])
+    achieved = 2 * kb / (kms * 1e-3) / 1e9 if kms > 0 else 0.0
+    traffic = read_profile_traffic(shape, m)
+
+    # ---- end-to-end arm (pinned host tier, host tokens) ----
+    e2e = None
+    link = None
+    if not args.no_e2e:
+        link = pinned_link_peak(torch, device) if rank == 0 else None
+        arm = Arm(args, pool, shape, torch, eakv, host_tier=True, device=device)
+        e_steps = max(2, min(args.steps, 5))
+        re_ = run_arm(arm, prompts_host, tables, e_steps, min(args.warmup, 3), dist, None)
+        arm.ctx.close()
+        del arm
+        e_ms, e_moved = aggregate_over_ranks(dist, re_["ms"], re_["moved"], device)
+        e_val = e_moved / (e_ms * 1e-3) / 1e9
+        e2e = {"value": e_val, "unit": UNIT, "h2d_bytes_per_step": int(re_["h2d"]),
+               "d2h_bytes_per_step": int(re_["d2h"]), "steps": e_steps,
+               "ms_per_step": e_ms / e_steps, "link_strategy": args.link}
+        if link:
+            # load and store alternate, so the bound is the harmonic mean of the two directions
+            bound = 2.0 / (1.0 / link["h2d"] + 1.0 / link["d2h"])
+            e2e.update(host_link_peak_gbps=link, frac_of_link=e_val / bound / max(world, 1))
+
+    cpu = None
+    if rank == 0 and not args.no_cpu_baseline:
+        g, s, dt = oracle_step_rate(args.cpu_seconds)
+        cpu = {"value": g, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"{s} steps x 2 requests x 128 blocks of 1.5 MiB in {dt:.1f} s"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "blocks_per_request": m, "requests_per_step": 2,
+                       "pool_blocks": nb, "block_bytes": shape.block_bytes,
+                       "block_ids": "uniform-random without replacement", "admit_mask": "from tier step (all admitted)",
+                       "l2": "inputs larger than L2 (12 GiB moved per step)",
+                       "tokens_hashed_per_step": 2 * m * shape.block_size,
+                       "copy_path": args.copy_path, "self_check": check_ok},
+            "clocks": r["clocks"],
+            "e2e": e2e,
+            "gpu_launches": r["launches"],
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                         "kernel": "copy_blocks_vector_kernel" if args.copy_path == "vector" else "copy_blocks_bulk_kernel",
+                         "launches_timed": len(r["kernel"]),
+                         "frac_of_nominal_8TBs": achieved / 8000.0},
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+        if args.sweep:
+            sweep(args, torch, eakv, pool, shape, device)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def self_check(torch, arm, pool, tables, args, shape):
+    """After the timed region: the last stored prompt's slots must equal its pool blocks."""
+    s = args.warmup + args.steps
+    table = tables[2 * s + 1]
+    keys = arm.keys_host.numpy().view(np.uint64)         # keys of the last request
+    _, H, _, slots = arm.ctx.eakv_match(keys)
+    if H != len(keys):
+        return False
+    ok = True
+    for j in np.linspace(0, len(keys) - 1, 16).astype(int):
+        for q in (0, shape.pieces_per_block - 1):
+            ok &= bool(torch.equal(arm.tier_t[int(slots[j]), q], pool.pieces[q][int(table[j])]))
+    return bool(ok)
+
+
+def read_profile_traffic(shape, m):
+    """DRAM bytes per launch of the copy kernel from the committed ncu summary, if present:
+    a line `dram_bytes_per_block = <float>` in profiles/copy_blocks_vector_kernel.txt."""
+    path = os.path.join(ROOT, "profiles", "copy_blocks_vector_kernel.txt")
+    try:
+        for ln in open(path):
+            if ln.startswith("dram_bytes_per_block"):
+                return float(ln.split("=")[1]) * m
+    except OSError:
+        pass
+    return None
+
+
+def sweep(args, torch, eakv, pool, shape, device):
+    """Store/load curve: 1..4096 blocks per call, contiguous vs random ids, mask all-ones vs
+    Bernoulli(0.5), device tier vs host tier (both strategies)."""
+    rng = np.random.default_rng(7)
+    nb = pool.gpu_blocks
+    kh = 4096
+    rows = []
+    arms = [("hbm", dict(tier_location=eakv.TIER_DEVICE)),
+            ("host_zero_copy", dict(tier_location=eakv.TIER_PINNED_HOST, link_strategy=eakv.LINK_ZERO_COPY)),
+            ("host_staged", dict(tier_location=eakv.TIER_PINNED_HOST, link_strategy=eakv.LINK_STAGED,
+                                 staging_bytes=args.staging_mib << 20))]
+    for name, kw in arms:
+        ctx = eakv.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+                           block_size=shape.block_size, gpu_blocks=nb, host_blocks=kh,
+                           kv_base=pool.kv_base, **kw)
+        stream = torch.cuda.current_stream(device)
+        for m in (1, 2, 4, 8, 16, 32, 64, 128, 256, 512, 1024, 2048, 4096):
+            for ids in ("contiguous", "random"):
+                for mask in ("ones", "bernoulli"):
+                    reps = 20 if m <= 256 else 5
+                    for op in ("store", "load"):
+                        if op == "load" and mask != "ones":
+                            continue
+                        times, nbytes = [], 0
+                        for _ in range(reps):
+                            start = int(rng.integers(0, nb - m + 1))
+                            table = (np.arange(start, start + m) if ids == "contiguous"
+                                     else rng.permutation(nb)[:m]).astype(np.int32)
+                            slots = (np.arange(m) if ids == "contiguous" else rng.permutation(kh)[:m]).astype(np.int32)
+                            adm = None if mask == "ones" else (rng.random(m) < 0.5).astype(np.uint8)
+                            nbytes = (m if adm is None else int(adm.sum())) * shape.block_bytes
+                            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                            e0.record(stream)
+                            if op == "store":
+                                ctx.eakv_store(table, adm, slots, stream)
+                            else:
+                                ctx.eakv_load(slots, table, stream)
+                            e1.record(stream)
+                            torch.cuda.synchronize()
+                            if nbytes:
+                                times.append(nbytes / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+                        if times:
+                            rows.append(dict(arm=name, op=op, blocks=m, ids=ids, mask=mask,
+                                             gbps_median=float(np.median(times)), gbps_best=float(max(times))))
+        ctx.close()
+    for row in rows:
+        print(json.dumps({"sweep": row}), file=sys.stderr)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,227 @@
+/*
+ * eakv -- paged-KV offload path for concurrent agents on one B200 (sm_100a).
+ *
+ * The data path that EfficientAgent's host tier drives: every agent turn the prompt's
+ * token blocks get prefix-dependent keys, the longest cached prefix is located on the
+ * GPU and in a host tier, the host-covered part is restored into fresh paged blocks,
+ * and the turn's new blocks are written to the host tier under an LRU reference model
+ * with write admission.
+ *
+ * Conventions
+ *   - Every function returns an int status: EAKV_OK (0) or a negative EAKV_E_* code.
+ *     Nothing throws or aborts; on a validation failure no kernel is launched and no
+ *     state changes.  eakv_strerror() names a code; eakv_last_cuda_error() gives the
+ *     CUDA error text behind the most recent EAKV_E_CUDA of a context.
+ *   - "host" pointers are ordinary CPU memory (pageable is fine) and are fully consumed
+ *     before the call returns.  "device" pointers must be dereferenceable by kernels of
+ *     the context's GPU (device memory, or pinned host memory under unified addressing).
+ *   - The caller owns every buffer it passes.  The context owns its tier memory (unless
+ *     adopted, see eakv_config.tier_memory), staging buffers, argument rings and side
+ *     streams.
+ *   - cuda_stream is a cudaStream_t cast to void* (NULL = the legacy default stream).
+ *     hash/store/load only enqueue work: results are valid once the stream has reached
+ *     the point after the call.
+ *   - A context is not thread-safe.  Two calls of the same kind (hash, store, load) on
+ *     one context must be ordered with respect to each other (same stream, or an event
+ *     between them): each kind has one set of scratch / staging buffers.  A store and a
+ *     load may run concurrently on two streams when they touch different slots/blocks.
+ *   - Layouts: the paged pool is 2L separate arrays, kv_base[2*l] = layer l's K and
+ *     kv_base[2*l+1] = its V, each [gpu_blocks][block_size][kv_heads][head_dim] of
+ *     elem_bytes-sized elements; one such [block_size][kv_heads][head_dim] slab is a
+ *     "piece".  The tier is slot-major: [host_blocks][L][2][block_size][kv_heads][head_dim].
+ *     piece bytes must be a multiple of 16 and all base pointers 16-byte aligned.
+ */
+#ifndef EAKV_H
+#define EAKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define EAKV_OK           0
+#define EAKV_E_INVAL     -1   /* NULL pointer, bad shape, misaligned base, duplicate destination */
+#define EAKV_E_RANGE     -2   /* block id >= gpu_blocks or slot >= host_blocks (or negative) */
+#define EAKV_E_CAPACITY  -3   /* request larger than a tier, scratch or output buffer */
+#define EAKV_E_NOMEM     -4   /* host, pinned or device allocation failed */
+#define EAKV_E_CUDA      -5   /* a CUDA runtime call failed; see eakv_last_cuda_error */
+#define EAKV_E_TIMEOUT   -6   /* a bounded device-side wait gave up (bulk-copy path) */
+
+/* write admission (Section 4, Eq. 6): save(r) = not (p_t and u > kappa) */
+#define EAKV_POLICY_WRITE_ALL          0   /* p_t = 0: plain offload                      */
+#define EAKV_POLICY_FILTER_FIXED       1   /* p_t = 1: fixed write admission              */
+#define EAKV_POLICY_FILTER_CONDITIONED 2   /* p_t = pressure signal of Appendix D, Eq. 10 */
+
+/* how bytes cross the host link */
+#define EAKV_LINK_ZERO_COPY 0   /* kernels read/write the mapped pinned tier directly          */
+#define EAKV_LINK_STAGED    1   /* gather to HBM staging + copy engine on a side stream,
+                                   double-buffered against the next gather (and the mirror) */
+
+/* where the tier lives */
+#define EAKV_TIER_PINNED_HOST 0 /* the product configuration                                   */
+#define EAKV_TIER_DEVICE      1 /* tier in HBM: on-device gather/scatter, for the HBM roofline */
+
+/* which device code moves the bytes */
+#define EAKV_COPY_VECTOR 0      /* 16-byte vector loads/stores, coalesced                       */
+#define EAKV_COPY_BULK   1      /* 1-D bulk async copies through a shared-memory ring           */
+
+typedef struct eakv_ctx eakv_ctx;
+
+typedef struct eakv_config {
+    int32_t num_layers, kv_heads, head_dim, block_size, elem_bytes;
+    int64_t gpu_blocks;            /* NB: blocks in each of the 2L paged arrays                 */
+    int64_t host_blocks;           /* K_H = floor(C_H / (b * beta)): tier capacity in blocks    */
+    int64_t gpu_index_blocks;      /* K_G: blocks the GPU-tier LRU hands out (<= gpu_blocks);
+                                      0 = gpu_blocks                                             */
+    void* const* kv_base;          /* host array of 2L device pointers (copied at create)       */
+    uint64_t hash_base, hash_seed; /* B and S of the prefix hash; 0 = library defaults          */
+    int32_t policy;                /* EAKV_POLICY_*                                              */
+    int32_t kappa_blocks;          /* write threshold kappa, in blocks                           */
+    int32_t theta_percent;         /* occupancy threshold theta, in percent (paper: 95)          */
+    int32_t len_window;            /* prompt-length window, in requests (paper: 256)             */
+    int64_t window_ms;             /* activity / eviction window (paper: 60 s)                   */
+    int32_t telemetry;             /* 1: tier report available; 0: the estimate alone decides    */
+    int32_t link_strategy;         /* EAKV_LINK_*                                                */
+    int32_t tier_location;         /* EAKV_TIER_*                                                */
+    int32_t copy_path;             /* EAKV_COPY_*                                                */
+    int32_t copy_ctas;             /* CTAs of the copy kernels; 0 = auto                         */
+    int64_t staging_bytes;         /* per staging buffer (two per direction); 0 = 64 MiB         */
+    int64_t max_call_blocks;       /* entries per argument-ring slot; 0 = 16384                  */
+    int64_t hash_scratch_blocks;   /* block partials the hash scratch holds; 0 = 1 << 20        */
+    void*   tier_memory;           /* NULL: the context allocates the tier.  Else adopt this
+                                      buffer of host_blocks * block bytes (pinned host memory
+                                      for TIER_PINNED_HOST, device memory for TIER_DEVICE);
+                                      it must outlive the context                               */
+} eakv_config;
+
+typedef struct eakv_stats {
+    /* tier bookkeeping */
+    int64_t requests, references, hits, admitted, declined, evicted;
+    int64_t declined_requests, pressure_requests, resident;
+    /* data plane */
+    int64_t tokens_hashed, blocks_stored, blocks_loaded, bytes_stored, bytes_loaded;
+    int64_t kernel_launches, memcpy_calls;
+} eakv_stats;
+
+typedef struct eakv_step_info {
+    int64_t host_prefix_blocks;    /* H: leading blocks the host tier held before the step      */
+    int64_t new_chunks;            /* u = floor(n/b) - floor(h/b)                               */
+    int32_t pressure;              /* p_t                                                        */
+    int32_t save;                  /* save(r)                                                    */
+} eakv_step_info;
+
+/* Fill *cfg with zeros and the paper's controller defaults (Appendix D, parameter table:
+ * theta 0.95, 60 s windows, 256 lookups, kappa 8) and write-all policy. */
+int eakv_config_init(eakv_config* cfg);
+
+/* Create a context on the current CUDA device.  Allocates the tier (pinned + mapped, or
+ * device), staging buffers, argument rings, hash scratch and two side streams.
+ * Errors: EAKV_E_INVAL (bad shape/pointers), EAKV_E_NOMEM, EAKV_E_CUDA. */
+int eakv_create(const eakv_config* cfg, eakv_ctx** out);
+
+/* Wait for all work the context enqueued, then free everything it owns. */
+int eakv_destroy(eakv_ctx* ctx);
+
+/* Block keys (Section 3.2: a full chunk's key depends on its entire prefix; Section 4:
+ * only full chunks).  h_{-1} = parent_hash, h_i = (h_{i-1} * B + token_i + 1) mod 2^61-1,
+ * canonical in [0, p); key of block j = h after its last token; n_blocks = n_tokens /
+ * block_size, a partial tail has no key.  Pass the context's seed (hash_seed) as
+ * parent_hash for a fresh prompt, or block j-1's key with the tokens from j*block_size
+ * on to resume at a block boundary.
+ *   tokens_dev  device, int32[n_tokens], ids >= 0
+ *   hashes_dev  device, uint64[n_tokens / block_size] (written)
+ *   n_blocks_out host, may be NULL
+ * Asynchronous on cuda_stream.  Errors: EAKV_E_INVAL, EAKV_E_CUDA. */
+int eakv_hash_blocks(eakv_ctx* ctx, const int32_t* tokens_dev, int64_t n_tokens,
+                     uint64_t parent_hash, uint64_t* hashes_dev, int64_t* n_blocks_out,
+                     void* cuda_stream);
+
+/* The same for many prompts in one launch.  Prompt i is tokens_dev[offsets[i] ..
+ * offsets[i+1]) and starts from parents[i] (NULL: the seed for all).  Keys are packed:
+ * prompt i's keys start at block_offsets_out[i] = sum_{k<i} len_k / block_size.
+ *   offsets_host       host, int64[n_prompts + 1], non-decreasing
+ *   parents_host       host, uint64[n_prompts] or NULL
+ *   block_offsets_out  host, int64[n_prompts + 1] (written) or NULL
+ * Errors: EAKV_E_INVAL, EAKV_E_CAPACITY (more blocks than the hash scratch, or more
+ * prompts than max_call_blocks), EAKV_E_CUDA. */
+int eakv_hash_blocks_batched(eakv_ctx* ctx, const int32_t* tokens_dev,
+                             const int64_t* offsets_host, int64_t n_prompts,
+                             const uint64_t* parents_host, uint64_t* hashes_dev,
+                             int64_t* block_offsets_out, void* cuda_stream);
+
+/* Longest cached prefix (Section 2 "Exact-prefix reuse"; Appendix C "Prefix coverage
+ * from a reference stream"): G = leading keys resident in the GPU index, H = leading keys
+ * resident in the host tier; each walk stops at its first absent key.  The restore run is
+ * blocks [G, H) when H > G.  Does not change recency.
+ *   hashes_host       host, uint64[n_blocks]
+ *   gpu_block_ids_out host, int32[>= G] or NULL;  host_slots_out host, int32[>= H] or NULL
+ *                     (size them n_blocks) */
+int eakv_match(const eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
+               int64_t* gpu_prefix_blocks, int64_t* host_prefix_blocks,
+               int32_t* gpu_block_ids_out, int32_t* host_slots_out);
+
+/* One request against the host tier (Appendix D "Reference model" and "Recency order";
+ * write rule Eq. 6 with the pressure signal Eq. 10).  References the keys in order: a
+ * resident key hits and moves to the most-recent end; a miss is inserted at the
+ * most-recent end (evicting the least-recent key when full) if the request is saved,
+ * else declined.  The save decision is taken once, before the walk, from
+ * u = n_blocks - H.  admit[j] = 1 exactly for inserted keys: those are the blocks to
+ * pass to eakv_store with slot[j]; resident keys are never copied again (deduplication).
+ *   hit_out, admit_out  host, uint8[n_blocks];  slot_out host, int32[n_blocks] (-1 = declined)
+ *   evicted_keys_out / evicted_slots_out  host arrays of *n_evicted_inout entries or NULL;
+ *   n_evicted_inout  in: capacity of those arrays, out: evictions of this step
+ *                    (EAKV_E_CAPACITY, nothing changed, if capacity < n_blocks and non-NULL)
+ *   info_out  host or NULL
+ * Errors: EAKV_E_CAPACITY when n_blocks > host_blocks (nothing changes). */
+int eakv_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
+                   int64_t agent_id, int64_t n_tokens, int64_t now_ms,
+                   uint8_t* hit_out, uint8_t* admit_out, int32_t* slot_out,
+                   uint64_t* evicted_keys_out, int32_t* evicted_slots_out,
+                   int64_t* n_evicted_inout, eakv_step_info* info_out);
+
+/* The GPU tier's bookkeeping, which the paper leaves to the serving engine (Section 2):
+ * an LRU of gpu_index_blocks keyed blocks referenced in order; a non-resident key takes
+ * a block from a free stack (0, 1, 2, ... first; an evicted block is reused next).  With
+ * need_tail a further unkeyed block is taken for the partial tail; give it back with
+ * eakv_gpu_tier_release at the end of the turn.
+ *   resident_out host uint8[n_blocks]; block_out host int32[n_blocks]; tail_block_out host
+ * Errors: EAKV_E_CAPACITY when n_blocks + need_tail > gpu_index_blocks (nothing changes). */
+int eakv_gpu_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
+                       int32_t need_tail, uint8_t* resident_out, int32_t* block_out,
+                       int32_t* tail_block_out);
+int eakv_gpu_tier_release(eakv_ctx* ctx, int32_t block_id);
+
+/* Store (Section 2 host writes; Appendix D: copy only absent chunks, from their original
+ * GPU KV locations): for every j with admit_mask[j] != 0 copy all 2L pieces of pool block
+ * block_table[j] to tier slot host_slots[j].  admit_mask NULL = all admitted.
+ *   block_table, host_slots host int32[n_blocks]; admit_mask host uint8[n_blocks] or NULL
+ * Entries with admit 0 are ignored (their ids are not validated).  Asynchronous on
+ * cuda_stream; with EAKV_LINK_STAGED the copy-engine part runs on a side stream that
+ * cuda_stream waits for before the call's work counts as complete.
+ * Errors: EAKV_E_RANGE, EAKV_E_INVAL (two admitted entries share a slot), EAKV_E_CUDA. */
+int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_mask,
+               const int32_t* host_slots, int64_t n_blocks, void* cuda_stream);
+
+/* Load / restore (Section 3.1, the R * beta / B_H2D term of Eq. 3): copy all 2L pieces of
+ * tier slot host_slots[j] into pool block block_table[j], for every j.
+ * Errors: EAKV_E_RANGE, EAKV_E_INVAL (two entries share a destination block), EAKV_E_CUDA. */
+int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_table,
+              int64_t n_blocks, void* cuda_stream);
+
+/* Block the host until everything the context enqueued (side streams included) is done. */
+int eakv_sync(eakv_ctx* ctx);
+
+int eakv_get_stats(const eakv_ctx* ctx, eakv_stats* out);
+/* Base address of the tier (host pointer for TIER_PINNED_HOST, device pointer otherwise). */
+void* eakv_tier_ptr(const eakv_ctx* ctx);
+uint64_t eakv_hash_seed(const eakv_ctx* ctx);
+uint64_t eakv_hash_base(const eakv_ctx* ctx);
+const char* eakv_strerror(int code);
+const char* eakv_last_cuda_error(const eakv_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EAKV_H */

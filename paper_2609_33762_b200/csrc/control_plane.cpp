@@ -1,0 +1,162 @@
+#include "control_plane.h"
+
+namespace eakv {
+
+static inline uint64_t mix64(uint64_t x) {
+    x ^= x >> 31;
+    x *= 0x7fb5d329728ea185ull;
+    x ^= x >> 27;
+    x *= 0x81dadef4bc2dd44dull;
+    x ^= x >> 33;
+    return x;
+}
+
+KeyedLru::KeyedLru(int64_t capacity)
+    : cap_(capacity), resident_(0), key_(capacity), prev_(capacity, -1), next_(capacity, -1),
+      state_(capacity, 0), lru_(-1), mru_(-1) {
+    free_.reserve(capacity);
+    for (int64_t s = capacity - 1; s >= 0; --s) free_.push_back((int32_t)s);
+    size_t n = 16;
+    while (n < (size_t)capacity * 2 + 2) n <<= 1;
+    table_.assign(n, 0);
+    mask_ = n - 1;
+}
+
+size_t KeyedLru::home(uint64_t key) const { return (size_t)mix64(key) & mask_; }
+
+int32_t KeyedLru::find(uint64_t key) const {
+    size_t i = home(key);
+    while (true) {
+        int32_t v = table_[i];
+        if (v == 0) return -1;
+        if (key_[v - 1] == key) return v - 1;
+        i = (i + 1) & mask_;
+    }
+}
+
+void KeyedLru::table_put(uint64_t key, int32_t slot) {
+    size_t i = home(key);
+    while (table_[i] != 0) i = (i + 1) & mask_;
+    table_[i] = slot + 1;
+}
+
+// linear probing with backward-shift deletion
+void KeyedLru::table_erase(uint64_t key) {
+    size_t i = home(key);
+    while (true) {
+        int32_t v = table_[i];
+        if (v == 0) return;
+        if (key_[v - 1] == key) break;
+        i = (i + 1) & mask_;
+    }
+    size_t hole = i;
+    size_t j = (i + 1) & mask_;
+    while (table_[j] != 0) {
+        size_t h = home(key_[table_[j] - 1]);
+        // can the entry at j move into the hole?  yes unless its home lies cyclically in (hole, j]
+        bool stays = (hole <= j) ? (h > hole && h <= j) : (h > hole || h <= j);
+        if (!stays) {
+            table_[hole] = table_[j];
+            hole = j;
+        }
+        j = (j + 1) & mask_;
+    }
+    table_[hole] = 0;
+}
+
+void KeyedLru::unlink(int32_t s) {
+    int32_t p = prev_[s], n = next_[s];
+    if (p >= 0) next_[p] = n; else lru_ = n;
+    if (n >= 0) prev_[n] = p; else mru_ = p;
+    prev_[s] = next_[s] = -1;
+}
+
+void KeyedLru::push_mru(int32_t s) {
+    prev_[s] = mru_;
+    next_[s] = -1;
+    if (mru_ >= 0) next_[mru_] = s; else lru_ = s;
+    mru_ = s;
+}
+
+void KeyedLru::promote(int32_t s) {
+    if (mru_ == s) return;
+    unlink(s);
+    push_mru(s);
+}
+
+int32_t KeyedLru::evict_lru(uint64_t* victim_key) {
+    int32_t v = lru_;
+    *victim_key = key_[v];
+    table_erase(key_[v]);
+    unlink(v);
+    state_[v] = 0;
+    --resident_;
+    free_.push_back(v);
+    return v;
+}
+
+int32_t KeyedLru::insert(uint64_t key, bool* evicted, uint64_t* victim_key, int32_t* victim_slot) {
+    *evicted = false;
+    if (resident_ >= cap_ || free_.empty()) {
+        *victim_slot = evict_lru(victim_key);
+        *evicted = true;
+    }
+    int32_t s = free_.back();
+    free_.pop_back();
+    key_[s] = key;
+    state_[s] = 1;
+    table_put(key, s);
+    push_mru(s);
+    ++resident_;
+    return s;
+}
+
+int32_t KeyedLru::take_unkeyed(bool* evicted, uint64_t* victim_key, int32_t* victim_slot) {
+    *evicted = false;
+    if (free_.empty()) {
+        *victim_slot = evict_lru(victim_key);
+        *evicted = true;
+    }
+    int32_t s = free_.back();
+    free_.pop_back();
+    state_[s] = 2;
+    return s;
+}
+
+void KeyedLru::release_unkeyed(int32_t s) {
+    state_[s] = 0;
+    free_.push_back(s);
+}
+
+Admission::Admission(int32_t policy, int32_t kappa_blocks, int32_t theta_percent,
+                     int64_t window_ms, int32_t len_window, int32_t telemetry,
+                     int64_t host_blocks, int32_t block_size)
+    : policy_(policy), kappa_(kappa_blocks), theta_percent_(theta_percent),
+      telemetry_(telemetry), window_ms_(window_ms), host_blocks_(host_blocks),
+      len_window_(len_window), block_size_(block_size), length_sum_(0) {}
+
+bool Admission::pressure(int64_t agent, int64_t n_tokens, int64_t now_ms, int64_t resident_now) {
+    agent_last_[agent] = now_ms;
+    lengths_.push_back(n_tokens);
+    length_sum_ += n_tokens;
+    while ((int64_t)lengths_.size() > len_window_) {
+        length_sum_ -= lengths_.front();
+        lengths_.pop_front();
+    }
+    const int64_t lo = now_ms - window_ms_;
+    while (!evict_times_.empty() && evict_times_.front() <= lo) evict_times_.pop_front();
+    if (policy_ == 0) return false;
+    if (policy_ == 1) return true;
+    int64_t active = 0;
+    for (const auto& kv : agent_last_) active += kv.second > lo;
+    // 128-bit products: lengths and capacities are far below 2^63 but their product need not be
+    const __int128 lhs = (__int128)(active - 1) * (__int128)length_sum_;
+    const __int128 rhs = (__int128)host_blocks_ * block_size_ * (__int128)lengths_.size();
+    const bool estimate = lhs > rhs;
+    if (!telemetry_) return estimate;
+    const bool full = (__int128)100 * resident_now >= (__int128)theta_percent_ * host_blocks_;
+    const bool evicting = !evict_times_.empty();
+    return estimate && full && evicting;
+}
+
+}  // namespace eakv

@@ -1,0 +1,79 @@
+// Host-side control plane: keyed LRU tiers and write admission.  Integer-only.
+//
+// KeyedLru implements the paper's LRU reference model (Appendix D): residents in recency
+// order, hit -> most-recent end, admitted miss -> insert at the most-recent end after
+// evicting the least-recent resident when full.  Storage is flat: an open-addressing
+// table maps a 61-bit key to a slot; recency links live in arrays indexed by slot; free
+// slots come from a stack that first yields 0, 1, 2, ... and reuses an evicted slot next.
+#pragma once
+#include <cstdint>
+#include <deque>
+#include <unordered_map>
+#include <vector>
+
+namespace eakv {
+
+class KeyedLru {
+public:
+    explicit KeyedLru(int64_t capacity);
+
+    int64_t capacity() const { return cap_; }
+    int64_t resident() const { return resident_; }
+
+    // slot of key or -1; does not change recency
+    int32_t find(uint64_t key) const;
+    // move a resident slot to the most-recent end
+    void promote(int32_t slot);
+    // Insert an absent key at the most-recent end.  When full, first evicts the
+    // least-recent resident and reports it through (*victim_key, *victim_slot).
+    // Returns the slot given to key.  *evicted is set to whether an eviction happened.
+    int32_t insert(uint64_t key, bool* evicted, uint64_t* victim_key, int32_t* victim_slot);
+    // take an unkeyed slot (evicting the least-recent resident when none is free)
+    int32_t take_unkeyed(bool* evicted, uint64_t* victim_key, int32_t* victim_slot);
+    // give an unkeyed slot back to the free stack
+    void release_unkeyed(int32_t slot);
+    bool is_unkeyed_taken(int32_t slot) const { return state_[slot] == 2; }
+
+private:
+    void table_put(uint64_t key, int32_t slot);
+    void table_erase(uint64_t key);
+    size_t home(uint64_t key) const;
+    void unlink(int32_t slot);
+    void push_mru(int32_t slot);
+    int32_t evict_lru(uint64_t* victim_key);
+
+    int64_t cap_, resident_;
+    std::vector<uint64_t> key_;        // by slot
+    std::vector<int32_t> prev_, next_; // by slot; -1 ends
+    std::vector<uint8_t> state_;       // 0 free, 1 keyed resident, 2 unkeyed taken
+    int32_t lru_, mru_;
+    std::vector<int32_t> free_;        // stack
+    std::vector<int32_t> table_;       // slot + 1, 0 = empty
+    size_t mask_;
+};
+
+// Pressure signal of Eq. 10 over virtual time, all integers:
+//   estimate  (A_t - 1) * sum(len) > K_H * b * count     (beta cancels, C_H = K_H b beta)
+//   full      100 * resident >= theta_percent * K_H
+//   evicting  evictions in (now - window, now] > 0
+class Admission {
+public:
+    Admission(int32_t policy, int32_t kappa_blocks, int32_t theta_percent, int64_t window_ms,
+              int32_t len_window, int32_t telemetry, int64_t host_blocks, int32_t block_size);
+    // registers the request (agent activity, prompt length), expires old evictions and
+    // returns p_t; call once per request before the walk
+    bool pressure(int64_t agent, int64_t n_tokens, int64_t now_ms, int64_t resident_now);
+    void note_eviction(int64_t now_ms) { evict_times_.push_back(now_ms); }
+    int32_t kappa() const { return kappa_; }
+
+private:
+    int32_t policy_, kappa_, theta_percent_, telemetry_;
+    int64_t window_ms_, host_blocks_;
+    int32_t len_window_, block_size_;
+    std::unordered_map<int64_t, int64_t> agent_last_;
+    std::deque<int64_t> lengths_;
+    int64_t length_sum_;
+    std::deque<int64_t> evict_times_;
+};
+
+}  // namespace eakv

@@ -1,0 +1,222 @@
+// Gather / scatter of KV blocks between the paged pool and a slot-major tier.
+//
+// The pool is 2L independent arrays of pieces ([gpu_blocks][piece_bytes]); a tier slot is
+// the 2L pieces of one block back to back.  A work item is (entry j, piece q, 16-KiB
+// sub-range); consecutive items walk a slot contiguously, so the tier side streams while
+// the pool side jumps one piece at a time.  Nothing is reused: streaming cache hints.
+//
+// Vector path: a CTA takes one item per loop trip; each thread issues kCopyUnroll
+// independent 16-byte loads before its stores, so a full grid keeps >100 KiB per SM in
+// flight.  The same kernel serves an HBM tier (HBM roofline), a mapped pinned tier
+// (zero-copy over the host link; run it with few CTAs) and the HBM staging buffers of the
+// copy-engine strategy.
+#include "eakv_internal.h"
+
+namespace eakv {
+
+template <bool TO_TIER>
+__global__ void __launch_bounds__(kCopyThreads)
+copy_blocks_vector_kernel(CopyLaunch L) {
+    const int64_t items_per_entry = (int64_t)L.pieces * L.subs_per_piece;
+    const int64_t n_items = L.n_entries * items_per_entry;
+    const int units_per_piece = (int)(L.piece_bytes >> 4);
+    for (int64_t it = blockIdx.x; it < n_items; it += gridDim.x) {
+        const int64_t j = it / items_per_entry;
+        const int r = (int)(it - j * items_per_entry);
+        const int q = r / L.subs_per_piece;
+        const int sub = r - q * L.subs_per_piece;
+        const int2 e = __ldg(L.entries + j);
+        char* pool = reinterpret_cast<char*>(__ldg(reinterpret_cast<const unsigned long long*>(L.kv_base) + q)) + (int64_t)e.x * L.piece_bytes;
+        char* tier = L.tier_base + ((int64_t)e.y * L.pieces + q) * L.piece_bytes;
+        const int4* src = reinterpret_cast<const int4*>(TO_TIER ? pool : tier);
+        int4* dst = reinterpret_cast<int4*>(TO_TIER ? tier : pool);
+        const int unit0 = sub * (kCopyThreads * kCopyUnroll) + threadIdx.x;
+        int4 v[kCopyUnroll];
+#pragma unroll
+        for (int u = 0; u < kCopyUnroll; ++u) {
+            const int unit = unit0 + u * kCopyThreads;
+            if (unit < units_per_piece) v[u] = __ldcs(src + unit);
+        }
+#pragma unroll
+        for (int u = 0; u < kCopyUnroll; ++u) {
+            const int unit = unit0 + u * kCopyThreads;
+            if (unit < units_per_piece) __stcs(dst + unit, v[u]);
+        }
+    }
+}
+
+static int g_vector_ctas_per_sm = 0;
+
+cudaError_t copy_kernels_init() {
+    int a = 0, b = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+        &a, copy_blocks_vector_kernel<true>, kCopyThreads, 0);
+    if (e != cudaSuccess) return e;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+        &b, copy_blocks_vector_kernel<false>, kCopyThreads, 0);
+    if (e != cudaSuccess) return e;
+    g_vector_ctas_per_sm = a < b ? a : b;
+    if (g_vector_ctas_per_sm < 1) g_vector_ctas_per_sm = 1;
+    return cudaSuccess;
+}
+
+int copy_vector_ctas_per_sm() { return g_vector_ctas_per_sm; }
+
+cudaError_t launch_copy_vector(const CopyLaunch& L, bool to_tier, int ctas, cudaStream_t stream) {
+    if (L.n_entries <= 0) return cudaSuccess;
+    const int64_t n_items = L.n_entries * L.pieces * L.subs_per_piece;
+    if (ctas > n_items) ctas = (int)n_items;
+    if (ctas < 1) ctas = 1;
+    if (to_tier) copy_blocks_vector_kernel<true><<<ctas, kCopyThreads, 0, stream>>>(L);
+    else         copy_blocks_vector_kernel<false><<<ctas, kCopyThreads, 0, stream>>>(L);
+    return cudaGetLastError();
+}
+
+}  // namespace eakv
+
+// ---------------------------------------------------------------------------------------
+// Bulk path: one thread per CTA drives a ring of shared-memory stages with 1-D bulk async
+// copies (global -> shared completing on an mbarrier, shared -> global in bulk groups).
+// No multicast, no tensor maps; every address and size is a multiple of 16 bytes.
+// Every wait is bounded: on giving up the thread raises *error_flag, drains what it has
+// in flight (bounded again) and returns.
+// ---------------------------------------------------------------------------------------
+namespace eakv {
+
+constexpr int kBulkStages = 4;
+constexpr int kBulkStageBytes = kCopySubBytes;
+constexpr uint32_t kBulkSpinLimit = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kBulkSpinLimit; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if (i > 64) __nanosleep(32);
+    }
+    return false;
+}
+
+struct BulkItem { const char* src; char* dst; uint32_t bytes; };
+
+template <bool TO_TIER>
+__device__ __forceinline__ BulkItem bulk_decode(const CopyLaunch& L, int64_t it) {
+    const int64_t items_per_entry = (int64_t)L.pieces * L.subs_per_piece;
+    const int64_t j = it / items_per_entry;
+    const int r = (int)(it - j * items_per_entry);
+    const int q = r / L.subs_per_piece;
+    const int sub = r - q * L.subs_per_piece;
+    const int2 e = __ldg(L.entries + j);
+    const int64_t off = (int64_t)sub * kBulkStageBytes;
+    char* pool = reinterpret_cast<char*>(__ldg(reinterpret_cast<const unsigned long long*>(L.kv_base) + q)) +
+                 (int64_t)e.x * L.piece_bytes + off;
+    char* tier = L.tier_base + ((int64_t)e.y * L.pieces + q) * L.piece_bytes + off;
+    BulkItem b;
+    b.src = TO_TIER ? pool : tier;
+    b.dst = TO_TIER ? tier : pool;
+    const int64_t left = L.piece_bytes - off;
+    b.bytes = (uint32_t)(left < kBulkStageBytes ? left : kBulkStageBytes);
+    return b;
+}
+
+template <bool TO_TIER>
+__global__ void __launch_bounds__(32)
+copy_blocks_bulk_kernel(CopyLaunch L, int* error_flag) {
+    extern __shared__ __align__(128) unsigned char stage_mem[];
+    __shared__ __align__(8) uint64_t bars[kBulkStages];
+    if (threadIdx.x != 0) return;
+
+    const int64_t n_items = L.n_entries * L.pieces * L.subs_per_piece;
+    const int64_t first = blockIdx.x, stride = gridDim.x;
+    if (first >= n_items) return;
+    const int64_t n_my = (n_items - first + stride - 1) / stride;
+
+    for (int s = 0; s < kBulkStages; ++s)
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&bars[s])) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+
+    auto issue_load = [&](int64_t k) {
+        const BulkItem b = bulk_decode<TO_TIER>(L, first + k * stride);
+        const int s = (int)(k % kBulkStages);
+        const uint32_t bar = smem_u32(&bars[s]);
+        const uint32_t dst = smem_u32(stage_mem + (size_t)s * kBulkStageBytes);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                     :: "r"(bar), "r"(b.bytes) : "memory");
+        asm volatile(
+            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+            :: "r"(dst), "l"(b.src), "r"(b.bytes), "r"(bar) : "memory");
+    };
+
+    const int64_t prologue = n_my < kBulkStages ? n_my : kBulkStages;
+    for (int64_t k = 0; k < prologue; ++k) issue_load(k);
+    int64_t loads_issued = prologue;
+
+    bool ok = true;
+    int64_t k = 0;
+    for (; k < n_my; ++k) {
+        const int s = (int)(k % kBulkStages);
+        const uint32_t parity = (uint32_t)((k / kBulkStages) & 1);
+        if (!mbar_wait_bounded(smem_u32(&bars[s]), parity)) { ok = false; break; }
+        const BulkItem b = bulk_decode<TO_TIER>(L, first + k * stride);
+        const uint32_t src = smem_u32(stage_mem + (size_t)s * kBulkStageBytes);
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                     :: "l"(b.dst), "r"(src), "r"(b.bytes) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        if (k >= 1 && loads_issued < n_my) {
+            // all but the newest group have finished reading shared memory: stage of item k-1 is free
+            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            issue_load(loads_issued);
+            ++loads_issued;
+        }
+    }
+    if (!ok) {
+        atomicExch(error_flag, 1);
+        // drain the loads still in flight (bounded) so shared memory is quiescent on exit
+        for (int64_t d = k + 1; d < loads_issued; ++d) {
+            const int s = (int)(d % kBulkStages);
+            mbar_wait_bounded(smem_u32(&bars[s]), (uint32_t)((d / kBulkStages) & 1));
+        }
+    }
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+static int g_bulk_ctas_per_sm = 0;
+
+cudaError_t launch_copy_bulk(const CopyLaunch& L, bool to_tier, int ctas, int* error_flag,
+                             cudaStream_t stream) {
+    if (L.n_entries <= 0) return cudaSuccess;
+    const size_t smem = (size_t)kBulkStages * kBulkStageBytes;
+    if (g_bulk_ctas_per_sm == 0) {
+        cudaError_t e = cudaFuncSetAttribute(copy_blocks_bulk_kernel<true>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(copy_blocks_bulk_kernel<false>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&g_bulk_ctas_per_sm,
+                                                          copy_blocks_bulk_kernel<true>, 32, smem);
+        if (e != cudaSuccess) return e;
+        if (g_bulk_ctas_per_sm < 1) g_bulk_ctas_per_sm = 1;
+    }
+    // the auto grid of the vector path assumes its occupancy; rescale to this kernel's
+    const int per_sm_vec = copy_vector_ctas_per_sm();
+    if (per_sm_vec > 0 && ctas % per_sm_vec == 0 && ctas / per_sm_vec >= 100)
+        ctas = ctas / per_sm_vec * g_bulk_ctas_per_sm;
+    const int64_t n_items = L.n_entries * L.pieces * L.subs_per_piece;
+    if (ctas > n_items) ctas = (int)n_items;
+    if (ctas < 1) ctas = 1;
+    if (to_tier) copy_blocks_bulk_kernel<true><<<ctas, 32, smem, stream>>>(L, error_flag);
+    else         copy_blocks_bulk_kernel<false><<<ctas, 32, smem, stream>>>(L, error_flag);
+    return cudaGetLastError();
+}
+
+}  // namespace eakv

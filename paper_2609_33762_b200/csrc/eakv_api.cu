@@ -1,0 +1,808 @@
+// C-ABI of libeakv: argument validation, host control plane, stream/event choreography.
+// All data movement and hashing happens in the kernels of hash_kernels.cu /
+// copy_kernels.cu (and, for the staged strategy, the copy engines); there is no CPU
+// fallback: without a CUDA device eakv_create fails.
+#include "../../include/eakv.h"
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "control_plane.h"
+#include "eakv_internal.h"
+
+using namespace eakv;
+
+namespace {
+
+constexpr uint64_t P61 = (1ull << 61) - 1;
+constexpr uint64_t kDefaultBase = 6364136223846793005ull % P61;
+constexpr uint64_t kDefaultSeed = 0x9E3779B97F4A7C15ull % P61;
+constexpr int kRingSlots = 8;
+
+inline uint64_t mulmod_host(uint64_t a, uint64_t b) {
+    return (uint64_t)(((unsigned __int128)a * b) % P61);
+}
+
+struct RingSlot {
+    void* host = nullptr;     // pinned
+    void* dev = nullptr;
+    cudaEvent_t done = nullptr;   // recorded after the last consumer of the slot was enqueued
+};
+
+struct Staging {
+    char* buf[2] = {nullptr, nullptr};
+    cudaEvent_t ready[2] = {nullptr, nullptr};   // buffer filled
+    cudaEvent_t freed[2] = {nullptr, nullptr};   // buffer drained
+    cudaEvent_t start = nullptr;
+    cudaStream_t side = nullptr;
+    int next = 0;
+};
+
+}  // namespace
+
+struct eakv_ctx {
+    eakv_config cfg;
+    int device = 0;
+    int sm_count = 0;
+    int32_t pieces = 0;
+    int64_t piece_bytes = 0, block_bytes = 0;
+    uint64_t base = 0, seed = 0;
+
+    void** d_kv_base = nullptr;
+    char* tier = nullptr;
+    bool tier_owned = false;
+
+    KeyedLru* host_tier = nullptr;
+    KeyedLru* gpu_tier = nullptr;
+    Admission* adm = nullptr;
+    int64_t gpu_unkeyed = 0;
+    eakv_stats stats;
+
+    // hash
+    uint64_t* d_pow = nullptr;
+    uint64_t* d_partial = nullptr;
+    int* d_counters = nullptr;
+    int64_t hash_scratch_blocks = 0;
+    int64_t max_prompts = 0;
+
+    // argument rings
+    RingSlot ring[kRingSlots];
+    int ring_next = 0;
+    size_t ring_bytes = 0;
+    int64_t max_call_blocks = 0;
+
+    // staged strategy
+    Staging st_store, st_load;
+    int64_t staging_blocks = 0;
+
+    int* d_error_flag = nullptr;
+
+    // duplicate-destination checks
+    std::vector<uint32_t> slot_stamp, blk_stamp;
+    uint32_t epoch = 0;
+    std::vector<int2> scratch_entries;
+
+    std::string cuda_err;
+};
+
+namespace {
+
+int cuda_fail(eakv_ctx* c, cudaError_t e, const char* what) {
+    if (c) {
+        c->cuda_err = std::string(what) + ": " + cudaGetErrorString(e);
+    }
+    return EAKV_E_CUDA;
+}
+
+#define CU(call)                                                    \
+    do {                                                            \
+        cudaError_t _e = (call);                                    \
+        if (_e != cudaSuccess) return cuda_fail(ctx, _e, #call);    \
+    } while (0)
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) {
+            switched = cudaSetDevice(dev) == cudaSuccess;
+        }
+    }
+    ~DeviceGuard() {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+// Take the next ring slot; blocks only if its previous use (kRingSlots calls ago) is still
+// pending on the GPU.
+int ring_acquire(eakv_ctx* ctx, RingSlot** out) {
+    RingSlot* s = &ctx->ring[ctx->ring_next];
+    ctx->ring_next = (ctx->ring_next + 1) % kRingSlots;
+    CU(cudaEventSynchronize(s->done));
+    *out = s;
+    return EAKV_OK;
+}
+
+void free_all(eakv_ctx* c) {
+    if (!c) return;
+    for (auto& s : c->ring) {
+        if (s.host) cudaFreeHost(s.host);
+        if (s.dev) cudaFree(s.dev);
+        if (s.done) cudaEventDestroy(s.done);
+    }
+    for (Staging* st : {&c->st_store, &c->st_load}) {
+        for (int i = 0; i < 2; ++i) {
+            if (st->buf[i]) cudaFree(st->buf[i]);
+            if (st->ready[i]) cudaEventDestroy(st->ready[i]);
+            if (st->freed[i]) cudaEventDestroy(st->freed[i]);
+        }
+        if (st->start) cudaEventDestroy(st->start);
+        if (st->side) cudaStreamDestroy(st->side);
+    }
+    if (c->d_kv_base) cudaFree(c->d_kv_base);
+    if (c->d_pow) cudaFree(c->d_pow);
+    if (c->d_partial) cudaFree(c->d_partial);
+    if (c->d_counters) cudaFree(c->d_counters);
+    if (c->d_error_flag) cudaFree(c->d_error_flag);
+    if (c->tier && c->tier_owned) {
+        if (c->cfg.tier_location == EAKV_TIER_DEVICE) cudaFree(c->tier);
+        else cudaFreeHost(c->tier);
+    }
+    delete c->host_tier;
+    delete c->gpu_tier;
+    delete c->adm;
+    delete c;
+}
+
+int copy_ctas(const eakv_ctx* ctx, bool touches_host) {
+    if (ctx->cfg.copy_ctas > 0) return ctx->cfg.copy_ctas;
+    if (touches_host) return 32;   // a few SMs saturate the host link; leave the rest to the engine
+    return ctx->sm_count * copy_vector_ctas_per_sm();
+}
+
+int launch_copy(eakv_ctx* ctx, const int2* d_entries, int64_t n, char* tier_base, bool to_tier,
+                bool touches_host, cudaStream_t stream) {
+    CopyLaunch L;
+    L.entries = d_entries;
+    L.n_entries = n;
+    L.kv_base = ctx->d_kv_base;
+    L.tier_base = tier_base;
+    L.pieces = ctx->pieces;
+    L.piece_bytes = ctx->piece_bytes;
+    L.subs_per_piece = (int32_t)((ctx->piece_bytes + kCopySubBytes - 1) / kCopySubBytes);
+    cudaError_t e;
+    if (ctx->cfg.copy_path == EAKV_COPY_BULK)
+        e = launch_copy_bulk(L, to_tier, copy_ctas(ctx, touches_host), ctx->d_error_flag, stream);
+    else
+        e = launch_copy_vector(L, to_tier, copy_ctas(ctx, touches_host), stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "copy kernel launch");
+    ctx->stats.kernel_launches += 1;
+    return EAKV_OK;
+}
+
+// upload n entries through a ring slot, then run `body(device entries)`; records the slot's event
+template <class F>
+int with_entries(eakv_ctx* ctx, const int2* entries, int64_t n, cudaStream_t stream, F body) {
+    RingSlot* s = nullptr;
+    int rc = ring_acquire(ctx, &s);
+    if (rc != EAKV_OK) return rc;
+    std::memcpy(s->host, entries, (size_t)n * sizeof(int2));
+    CU(cudaMemcpyAsync(s->dev, s->host, (size_t)n * sizeof(int2), cudaMemcpyHostToDevice, stream));
+    ctx->stats.memcpy_calls += 1;
+    rc = body(static_cast<const int2*>(s->dev));
+    CU(cudaEventRecord(s->done, stream));
+    return rc;
+}
+
+int next_epoch(eakv_ctx* ctx) {
+    if (++ctx->epoch == 0) {   // wrapped: clear the stamps
+        std::fill(ctx->slot_stamp.begin(), ctx->slot_stamp.end(), 0u);
+        std::fill(ctx->blk_stamp.begin(), ctx->blk_stamp.end(), 0u);
+        ctx->epoch = 1;
+    }
+    return EAKV_OK;
+}
+
+// contiguous runs of host slots inside a chunk: [i0, i1) with slots e[i0].y, e[i0].y+1, ...
+template <class F>
+int for_slot_runs(const int2* e, int64_t n, F f) {
+    int64_t i0 = 0;
+    while (i0 < n) {
+        int64_t i1 = i0 + 1;
+        while (i1 < n && e[i1].y == e[i1 - 1].y + 1) ++i1;
+        int rc = f(i0, i1);
+        if (rc != EAKV_OK) return rc;
+        i0 = i1;
+    }
+    return EAKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int eakv_config_init(eakv_config* cfg) {
+    if (!cfg) return EAKV_E_INVAL;
+    std::memset(cfg, 0, sizeof(*cfg));
+    cfg->elem_bytes = 2;
+    cfg->policy = EAKV_POLICY_WRITE_ALL;
+    cfg->kappa_blocks = 8;
+    cfg->theta_percent = 95;
+    cfg->len_window = 256;
+    cfg->window_ms = 60000;
+    cfg->telemetry = 1;
+    cfg->link_strategy = EAKV_LINK_ZERO_COPY;
+    cfg->tier_location = EAKV_TIER_PINNED_HOST;
+    cfg->copy_path = EAKV_COPY_VECTOR;
+    return EAKV_OK;
+}
+
+int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
+    if (!cfg || !out) return EAKV_E_INVAL;
+    *out = nullptr;
+    if (cfg->num_layers <= 0 || cfg->kv_heads <= 0 || cfg->head_dim <= 0 || cfg->block_size <= 0 ||
+        cfg->elem_bytes <= 0 || cfg->gpu_blocks <= 0 || cfg->host_blocks <= 0 || !cfg->kv_base)
+        return EAKV_E_INVAL;
+    if (cfg->block_size > kHashMaxBlockSize) return EAKV_E_INVAL;
+    if (cfg->gpu_blocks > INT32_MAX || cfg->host_blocks > INT32_MAX) return EAKV_E_INVAL;
+    if (cfg->policy < 0 || cfg->policy > 2 || cfg->link_strategy < 0 || cfg->link_strategy > 1 ||
+        cfg->tier_location < 0 || cfg->tier_location > 1 || cfg->copy_path < 0 || cfg->copy_path > 1)
+        return EAKV_E_INVAL;
+    if (cfg->gpu_index_blocks < 0 || cfg->gpu_index_blocks > cfg->gpu_blocks) return EAKV_E_INVAL;
+    const int64_t piece = (int64_t)cfg->block_size * cfg->kv_heads * cfg->head_dim * cfg->elem_bytes;
+    if (piece % 16 != 0) return EAKV_E_INVAL;
+    const int pieces = 2 * cfg->num_layers;
+    for (int q = 0; q < pieces; ++q) {
+        if (!cfg->kv_base[q] || ((uintptr_t)cfg->kv_base[q] & 15)) return EAKV_E_INVAL;
+    }
+    if (cfg->tier_memory && ((uintptr_t)cfg->tier_memory & 15)) return EAKV_E_INVAL;
+
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) return EAKV_E_CUDA;
+
+    eakv_ctx* ctx = new (std::nothrow) eakv_ctx();
+    if (!ctx) return EAKV_E_NOMEM;
+    ctx->cfg = *cfg;
+    ctx->cfg.kv_base = nullptr;
+    std::memset(&ctx->stats, 0, sizeof(ctx->stats));
+    ctx->pieces = pieces;
+    ctx->piece_bytes = piece;
+    ctx->block_bytes = piece * pieces;
+    ctx->base = cfg->hash_base ? cfg->hash_base % P61 : kDefaultBase;
+    ctx->seed = cfg->hash_seed ? cfg->hash_seed % P61 : kDefaultSeed;
+    ctx->max_call_blocks = cfg->max_call_blocks > 0 ? cfg->max_call_blocks : 16384;
+    ctx->hash_scratch_blocks = cfg->hash_scratch_blocks > 0 ? cfg->hash_scratch_blocks : (1 << 20);
+    ctx->max_prompts = ctx->max_call_blocks;
+
+#define CUC(call)                                             \
+    do {                                                      \
+        cudaError_t _e = (call);                              \
+        if (_e != cudaSuccess) {                              \
+            int rc = (_e == cudaErrorMemoryAllocation) ? EAKV_E_NOMEM : EAKV_E_CUDA; \
+            std::fprintf(stderr, "eakv_create: %s: %s\n", #call, cudaGetErrorString(_e)); \
+            cudaGetLastError();                               \
+            free_all(ctx);                                    \
+            return rc;                                        \
+        }                                                     \
+    } while (0)
+
+    CUC(cudaGetDevice(&ctx->device));
+    CUC(cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device));
+    CUC(hash_kernels_init());
+    CUC(copy_kernels_init());
+
+    try {
+        ctx->host_tier = new KeyedLru(cfg->host_blocks);
+        ctx->gpu_tier = new KeyedLru(cfg->gpu_index_blocks ? cfg->gpu_index_blocks : cfg->gpu_blocks);
+        ctx->adm = new Admission(cfg->policy, cfg->kappa_blocks, cfg->theta_percent, cfg->window_ms,
+                                 cfg->len_window > 0 ? cfg->len_window : 256, cfg->telemetry,
+                                 cfg->host_blocks, cfg->block_size);
+        ctx->slot_stamp.assign((size_t)cfg->host_blocks, 0);
+        ctx->blk_stamp.assign((size_t)cfg->gpu_blocks, 0);
+    } catch (const std::bad_alloc&) {
+        free_all(ctx);
+        return EAKV_E_NOMEM;
+    }
+
+    // piece-array base pointers
+    CUC(cudaMalloc(&ctx->d_kv_base, sizeof(void*) * pieces));
+    CUC(cudaMemcpy(ctx->d_kv_base, cfg->kv_base, sizeof(void*) * pieces, cudaMemcpyHostToDevice));
+
+    // tier memory
+    const size_t tier_bytes = (size_t)cfg->host_blocks * (size_t)ctx->block_bytes;
+    if (cfg->tier_memory) {
+        ctx->tier = static_cast<char*>(cfg->tier_memory);
+    } else if (cfg->tier_location == EAKV_TIER_DEVICE) {
+        CUC(cudaMalloc(&ctx->tier, tier_bytes));
+        ctx->tier_owned = true;
+    } else {
+        CUC(cudaHostAlloc(&ctx->tier, tier_bytes, cudaHostAllocMapped | cudaHostAllocPortable));
+        ctx->tier_owned = true;
+    }
+
+    // hash: power table B^0..B^b, partial scratch, ticket counters
+    {
+        std::vector<uint64_t> pw((size_t)cfg->block_size + 1);
+        pw[0] = 1;
+        for (int e = 1; e <= cfg->block_size; ++e) pw[e] = mulmod_host(pw[e - 1], ctx->base);
+        CUC(cudaMalloc(&ctx->d_pow, pw.size() * 8));
+        CUC(cudaMemcpy(ctx->d_pow, pw.data(), pw.size() * 8, cudaMemcpyHostToDevice));
+        CUC(cudaMalloc(&ctx->d_partial, (size_t)ctx->hash_scratch_blocks * 8));
+        CUC(cudaMalloc(&ctx->d_counters, (size_t)ctx->max_prompts * sizeof(int)));
+        CUC(cudaMemset(ctx->d_counters, 0, (size_t)ctx->max_prompts * sizeof(int)));
+        CUC(cudaMalloc(&ctx->d_error_flag, sizeof(int)));
+        CUC(cudaMemset(ctx->d_error_flag, 0, sizeof(int)));
+    }
+
+    // argument rings: room for max_call_blocks copy entries, or the batched-hash descriptors
+    ctx->ring_bytes = std::max<size_t>((size_t)ctx->max_call_blocks * sizeof(HashPrompt) +
+                                           (size_t)ctx->max_call_blocks * sizeof(HashTile),
+                                       (size_t)1 << 16);
+    for (auto& s : ctx->ring) {
+        CUC(cudaHostAlloc(&s.host, ctx->ring_bytes, cudaHostAllocDefault));
+        CUC(cudaMalloc(&s.dev, ctx->ring_bytes));
+        CUC(cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming));
+    }
+
+    // staged strategy
+    if (cfg->link_strategy == EAKV_LINK_STAGED) {
+        int64_t sbytes = cfg->staging_bytes > 0 ? cfg->staging_bytes : (64ll << 20);
+        ctx->staging_blocks = std::max<int64_t>(1, sbytes / ctx->block_bytes);
+        ctx->staging_blocks = std::min(ctx->staging_blocks, ctx->max_call_blocks);
+        for (Staging* st : {&ctx->st_store, &ctx->st_load}) {
+            for (int i = 0; i < 2; ++i) {
+                CUC(cudaMalloc(&st->buf[i], (size_t)ctx->staging_blocks * ctx->block_bytes));
+                CUC(cudaEventCreateWithFlags(&st->ready[i], cudaEventDisableTiming));
+                CUC(cudaEventCreateWithFlags(&st->freed[i], cudaEventDisableTiming));
+            }
+            CUC(cudaEventCreateWithFlags(&st->start, cudaEventDisableTiming));
+            CUC(cudaStreamCreateWithFlags(&st->side, cudaStreamNonBlocking));
+        }
+    }
+    CUC(cudaDeviceSynchronize());
+#undef CUC
+    *out = ctx;
+    return EAKV_OK;
+}
+
+int eakv_sync(eakv_ctx* ctx) {
+    if (!ctx) return EAKV_E_INVAL;
+    DeviceGuard g(ctx->device);
+    CU(cudaDeviceSynchronize());
+    int flag = 0;
+    CU(cudaMemcpy(&flag, ctx->d_error_flag, sizeof(int), cudaMemcpyDeviceToHost));
+    if (flag != 0) {   // a bounded wait in the bulk-copy kernel gave up
+        CU(cudaMemset(ctx->d_error_flag, 0, sizeof(int)));
+        return EAKV_E_TIMEOUT;
+    }
+    return EAKV_OK;
+}
+
+int eakv_destroy(eakv_ctx* ctx) {
+    if (!ctx) return EAKV_E_INVAL;
+    DeviceGuard g(ctx->device);
+    cudaDeviceSynchronize();
+    free_all(ctx);
+    return EAKV_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// hashing
+// ------------------------------------------------------------------------------------------
+int eakv_hash_blocks(eakv_ctx* ctx, const int32_t* tokens_dev, int64_t n_tokens,
+                     uint64_t parent_hash, uint64_t* hashes_dev, int64_t* n_blocks_out,
+                     void* cuda_stream) {
+    if (!ctx || n_tokens < 0) return EAKV_E_INVAL;
+    const int b = ctx->cfg.block_size;
+    const int64_t nblk = n_tokens / b;
+    if (n_blocks_out) *n_blocks_out = nblk;
+    if (nblk == 0) return EAKV_OK;
+    if (!tokens_dev || !hashes_dev) return EAKV_E_INVAL;
+    if (((uintptr_t)tokens_dev & 3) || ((uintptr_t)hashes_dev & 7)) return EAKV_E_INVAL;
+    DeviceGuard g(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const bool generic = (b % 4) != 0;
+    const bool vec = !generic && (((uintptr_t)tokens_dev & 15) == 0);
+    const int tile_blocks = generic ? kHashThreads : std::max(1, kHashTileTokens / b);
+    // split at the scratch capacity; a later piece reads its parent from the previous key
+    const int64_t cap = ctx->hash_scratch_blocks;
+    int64_t done = 0;
+    while (done < nblk) {
+        const int64_t cur = std::min(cap, nblk - done);
+        HashLaunch L;
+        L.tokens = tokens_dev + done * b;
+        L.keys = hashes_dev + done;
+        L.partial = ctx->d_partial;
+        L.counters = ctx->d_counters;
+        L.pow_table = ctx->d_pow;
+        L.tiles = nullptr;
+        L.prompts = nullptr;
+        L.single_nblk = cur;
+        L.single_parent = parent_hash % P61;
+        L.single_parent_ptr = done ? hashes_dev + done - 1 : nullptr;
+        L.block_size = b;
+        L.tile_blocks = tile_blocks;
+        const int n_tiles = (int)((cur + tile_blocks - 1) / tile_blocks);
+        const bool piece_vec = vec && (((done * b) & 3) == 0);
+        cudaError_t e = launch_hash(L, n_tiles, generic, piece_vec, stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "hash kernel launch");
+        ctx->stats.kernel_launches += 1;
+        done += cur;
+    }
+    ctx->stats.tokens_hashed += nblk * b;
+    return EAKV_OK;
+}
+
+int eakv_hash_blocks_batched(eakv_ctx* ctx, const int32_t* tokens_dev,
+                             const int64_t* offsets_host, int64_t n_prompts,
+                             const uint64_t* parents_host, uint64_t* hashes_dev,
+                             int64_t* block_offsets_out, void* cuda_stream) {
+    if (!ctx || n_prompts < 0 || !offsets_host) return EAKV_E_INVAL;
+    const int b = ctx->cfg.block_size;
+    int64_t total_blocks = 0;
+    for (int64_t i = 0; i < n_prompts; ++i) {
+        if (offsets_host[i + 1] < offsets_host[i] || offsets_host[i] < 0) return EAKV_E_INVAL;
+        total_blocks += (offsets_host[i + 1] - offsets_host[i]) / b;
+    }
+    if (n_prompts > ctx->max_prompts || total_blocks > ctx->hash_scratch_blocks)
+        return EAKV_E_CAPACITY;
+    if (block_offsets_out) {
+        int64_t acc = 0;
+        for (int64_t i = 0; i < n_prompts; ++i) {
+            block_offsets_out[i] = acc;
+            acc += (offsets_host[i + 1] - offsets_host[i]) / b;
+        }
+        block_offsets_out[n_prompts] = acc;
+    }
+    if (total_blocks == 0) return EAKV_OK;
+    if (!tokens_dev || !hashes_dev) return EAKV_E_INVAL;
+    if (((uintptr_t)tokens_dev & 3) || ((uintptr_t)hashes_dev & 7)) return EAKV_E_INVAL;
+    DeviceGuard g(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const bool generic = (b % 4) != 0;
+    bool vec = !generic && (((uintptr_t)tokens_dev & 15) == 0);
+    const int tile_blocks = generic ? kHashThreads : std::max(1, kHashTileTokens / b);
+
+    int64_t n_tiles = 0;
+    for (int64_t i = 0; i < n_prompts; ++i) {
+        const int64_t nb = (offsets_host[i + 1] - offsets_host[i]) / b;
+        n_tiles += (nb + tile_blocks - 1) / tile_blocks;
+        if (nb > 0 && (offsets_host[i] & 3)) vec = false;
+    }
+    const size_t need = (size_t)n_prompts * sizeof(HashPrompt) + (size_t)n_tiles * sizeof(HashTile);
+    if (need > ctx->ring_bytes || n_tiles > INT32_MAX) return EAKV_E_CAPACITY;
+
+    RingSlot* s = nullptr;
+    int rc = ring_acquire(ctx, &s);
+    if (rc != EAKV_OK) return rc;
+    HashPrompt* hp = static_cast<HashPrompt*>(s->host);
+    HashTile* ht = reinterpret_cast<HashTile*>(hp + n_prompts);
+    int64_t acc = 0, t = 0;
+    for (int64_t i = 0; i < n_prompts; ++i) {
+        const int64_t nb = (offsets_host[i + 1] - offsets_host[i]) / b;
+        const int64_t tiles = (nb + tile_blocks - 1) / tile_blocks;
+        hp[i].tok_off = offsets_host[i];
+        hp[i].blk_off = acc;
+        hp[i].nblk = nb;
+        hp[i].parent = (parents_host ? parents_host[i] : ctx->seed) % P61;
+        hp[i].tiles = (int32_t)tiles;
+        hp[i].pad = 0;
+        for (int64_t k = 0; k < tiles; ++k) {
+            ht[t].prompt = (int32_t)i;
+            ht[t].first_block = (int32_t)(k * tile_blocks);
+            ++t;
+        }
+        acc += nb;
+    }
+    CU(cudaMemcpyAsync(s->dev, s->host, need, cudaMemcpyHostToDevice, stream));
+    ctx->stats.memcpy_calls += 1;
+    HashLaunch L;
+    L.tokens = tokens_dev;
+    L.keys = hashes_dev;
+    L.partial = ctx->d_partial;
+    L.counters = ctx->d_counters;
+    L.pow_table = ctx->d_pow;
+    L.prompts = static_cast<const HashPrompt*>(s->dev);
+    L.tiles = reinterpret_cast<const HashTile*>(L.prompts + n_prompts);
+    L.single_nblk = 0;
+    L.single_parent = 0;
+    L.single_parent_ptr = nullptr;
+    L.block_size = b;
+    L.tile_blocks = tile_blocks;
+    cudaError_t e = launch_hash(L, (int)n_tiles, generic, vec, stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "hash kernel launch");
+    ctx->stats.kernel_launches += 1;
+    CU(cudaEventRecord(s->done, stream));
+    ctx->stats.tokens_hashed += total_blocks * b;
+    return EAKV_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// control plane
+// ------------------------------------------------------------------------------------------
+int eakv_match(const eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
+               int64_t* gpu_prefix_blocks, int64_t* host_prefix_blocks,
+               int32_t* gpu_block_ids_out, int32_t* host_slots_out) {
+    if (!ctx || n_blocks < 0 || (n_blocks > 0 && !hashes_host)) return EAKV_E_INVAL;
+    int64_t G = 0, H = 0;
+    for (; G < n_blocks; ++G) {
+        const int32_t s = ctx->gpu_tier->find(hashes_host[G]);
+        if (s < 0) break;
+        if (gpu_block_ids_out) gpu_block_ids_out[G] = s;
+    }
+    for (; H < n_blocks; ++H) {
+        const int32_t s = ctx->host_tier->find(hashes_host[H]);
+        if (s < 0) break;
+        if (host_slots_out) host_slots_out[H] = s;
+    }
+    if (gpu_prefix_blocks) *gpu_prefix_blocks = G;
+    if (host_prefix_blocks) *host_prefix_blocks = H;
+    return EAKV_OK;
+}
+
+int eakv_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
+                   int64_t agent_id, int64_t n_tokens, int64_t now_ms,
+                   uint8_t* hit_out, uint8_t* admit_out, int32_t* slot_out,
+                   uint64_t* evicted_keys_out, int32_t* evicted_slots_out,
+                   int64_t* n_evicted_inout, eakv_step_info* info_out) {
+    if (!ctx || n_blocks < 0 || n_tokens < 0) return EAKV_E_INVAL;
+    if (n_blocks > 0 && (!hashes_host || !hit_out || !admit_out || !slot_out)) return EAKV_E_INVAL;
+    if (n_blocks > ctx->host_tier->capacity()) return EAKV_E_CAPACITY;
+    const bool want_evicted = evicted_keys_out || evicted_slots_out;
+    if (want_evicted && (!n_evicted_inout || *n_evicted_inout < n_blocks)) return EAKV_E_CAPACITY;
+
+    KeyedLru& T = *ctx->host_tier;
+    int64_t H = 0;
+    while (H < n_blocks && T.find(hashes_host[H]) >= 0) ++H;
+    const bool p = ctx->adm->pressure(agent_id, n_tokens, now_ms, T.resident());
+    const int b = ctx->cfg.block_size;
+    const int64_t u = n_tokens / b - (H * b) / b;
+    const bool save = !(p && u > ctx->adm->kappa());
+    eakv_stats& st = ctx->stats;
+    st.requests += 1;
+    st.pressure_requests += p;
+    st.declined_requests += !save;
+    int64_t n_ev = 0;
+    for (int64_t j = 0; j < n_blocks; ++j) {
+        const uint64_t key = hashes_host[j];
+        st.references += 1;
+        const int32_t s = T.find(key);
+        if (s >= 0) {
+            T.promote(s);
+            hit_out[j] = 1; admit_out[j] = 0; slot_out[j] = s;
+            st.hits += 1;
+        } else if (save) {
+            bool ev = false;
+            uint64_t vkey = 0;
+            int32_t vslot = -1;
+            const int32_t ns = T.insert(key, &ev, &vkey, &vslot);
+            if (ev) {
+                if (evicted_keys_out) evicted_keys_out[n_ev] = vkey;
+                if (evicted_slots_out) evicted_slots_out[n_ev] = vslot;
+                ++n_ev;
+                ctx->adm->note_eviction(now_ms);
+                st.evicted += 1;
+            }
+            hit_out[j] = 0; admit_out[j] = 1; slot_out[j] = ns;
+            st.admitted += 1;
+        } else {
+            hit_out[j] = 0; admit_out[j] = 0; slot_out[j] = -1;
+            st.declined += 1;
+        }
+    }
+    st.resident = T.resident();
+    if (n_evicted_inout) *n_evicted_inout = n_ev;
+    if (info_out) {
+        info_out->host_prefix_blocks = H;
+        info_out->new_chunks = u;
+        info_out->pressure = p;
+        info_out->save = save;
+    }
+    return EAKV_OK;
+}
+
+int eakv_gpu_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
+                       int32_t need_tail, uint8_t* resident_out, int32_t* block_out,
+                       int32_t* tail_block_out) {
+    if (!ctx || n_blocks < 0) return EAKV_E_INVAL;
+    if (n_blocks > 0 && (!hashes_host || !resident_out || !block_out)) return EAKV_E_INVAL;
+    if (need_tail && !tail_block_out) return EAKV_E_INVAL;
+    KeyedLru& T = *ctx->gpu_tier;
+    if (n_blocks + (need_tail ? 1 : 0) + ctx->gpu_unkeyed > T.capacity()) return EAKV_E_CAPACITY;
+    bool ev;
+    uint64_t vkey;
+    int32_t vslot;
+    for (int64_t j = 0; j < n_blocks; ++j) {
+        const int32_t s = T.find(hashes_host[j]);
+        if (s >= 0) {
+            T.promote(s);
+            resident_out[j] = 1;
+            block_out[j] = s;
+        } else {
+            resident_out[j] = 0;
+            block_out[j] = T.insert(hashes_host[j], &ev, &vkey, &vslot);
+        }
+    }
+    if (tail_block_out) *tail_block_out = -1;
+    if (need_tail) {
+        *tail_block_out = T.take_unkeyed(&ev, &vkey, &vslot);
+        ctx->gpu_unkeyed += 1;
+    }
+    return EAKV_OK;
+}
+
+int eakv_gpu_tier_release(eakv_ctx* ctx, int32_t block_id) {
+    if (!ctx) return EAKV_E_INVAL;
+    if (block_id < 0 || block_id >= ctx->gpu_tier->capacity()) return EAKV_E_RANGE;
+    if (!ctx->gpu_tier->is_unkeyed_taken(block_id)) return EAKV_E_INVAL;
+    ctx->gpu_tier->release_unkeyed(block_id);
+    ctx->gpu_unkeyed -= 1;
+    return EAKV_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// store / load
+// ------------------------------------------------------------------------------------------
+int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_mask,
+               const int32_t* host_slots, int64_t n_blocks, void* cuda_stream) {
+    if (!ctx || n_blocks < 0) return EAKV_E_INVAL;
+    if (n_blocks == 0) return EAKV_OK;
+    if (!block_table || !host_slots) return EAKV_E_INVAL;
+    // validate and compact before anything is enqueued
+    next_epoch(ctx);
+    std::vector<int2>& ent = ctx->scratch_entries;
+    ent.clear();
+    for (int64_t j = 0; j < n_blocks; ++j) {
+        if (admit_mask && !admit_mask[j]) continue;
+        const int32_t blk = block_table[j], slot = host_slots[j];
+        if (blk < 0 || blk >= ctx->cfg.gpu_blocks || slot < 0 || slot >= ctx->cfg.host_blocks)
+            return EAKV_E_RANGE;
+        if (ctx->slot_stamp[slot] == ctx->epoch) return EAKV_E_INVAL;
+        ctx->slot_stamp[slot] = ctx->epoch;
+        ent.push_back(make_int2(blk, slot));
+    }
+    const int64_t m = (int64_t)ent.size();
+    if (m == 0) return EAKV_OK;
+    DeviceGuard g(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const bool host_tier = ctx->cfg.tier_location == EAKV_TIER_PINNED_HOST;
+
+    if (ctx->cfg.link_strategy == EAKV_LINK_ZERO_COPY) {
+        for (int64_t i = 0; i < m; i += ctx->max_call_blocks) {
+            const int64_t cur = std::min(ctx->max_call_blocks, m - i);
+            int rc = with_entries(ctx, ent.data() + i, cur, stream, [&](const int2* d) {
+                return launch_copy(ctx, d, cur, ctx->tier, true, host_tier, stream);
+            });
+            if (rc != EAKV_OK) return rc;
+        }
+    } else {
+        Staging& S = ctx->st_store;
+        std::vector<int2> local;
+        for (int64_t i = 0; i < m; i += ctx->staging_blocks) {
+            const int64_t cur = std::min(ctx->staging_blocks, m - i);
+            const int sb = S.next;
+            S.next ^= 1;
+            local.resize((size_t)cur);
+            for (int64_t k = 0; k < cur; ++k) local[k] = make_int2(ent[i + k].x, (int)k);
+            CU(cudaStreamWaitEvent(stream, S.freed[sb], 0));
+            int rc = with_entries(ctx, local.data(), cur, stream, [&](const int2* d) {
+                return launch_copy(ctx, d, cur, S.buf[sb], true, false, stream);
+            });
+            if (rc != EAKV_OK) return rc;
+            CU(cudaEventRecord(S.ready[sb], stream));
+            CU(cudaStreamWaitEvent(S.side, S.ready[sb], 0));
+            rc = for_slot_runs(ent.data() + i, cur, [&](int64_t a, int64_t z) {
+                CU(cudaMemcpyAsync(ctx->tier + (int64_t)ent[i + a].y * ctx->block_bytes,
+                                   S.buf[sb] + a * ctx->block_bytes,
+                                   (size_t)(z - a) * ctx->block_bytes, cudaMemcpyDefault, S.side));
+                ctx->stats.memcpy_calls += 1;
+                return EAKV_OK;
+            });
+            if (rc != EAKV_OK) return rc;
+            CU(cudaEventRecord(S.freed[sb], S.side));
+        }
+        // the call's work is complete, in stream order, once both buffers are drained
+        CU(cudaStreamWaitEvent(stream, S.freed[0], 0));
+        CU(cudaStreamWaitEvent(stream, S.freed[1], 0));
+    }
+    ctx->stats.blocks_stored += m;
+    ctx->stats.bytes_stored += m * ctx->block_bytes;
+    return EAKV_OK;
+}
+
+int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_table,
+              int64_t n_blocks, void* cuda_stream) {
+    if (!ctx || n_blocks < 0) return EAKV_E_INVAL;
+    if (n_blocks == 0) return EAKV_OK;
+    if (!block_table || !host_slots) return EAKV_E_INVAL;
+    next_epoch(ctx);
+    std::vector<int2>& ent = ctx->scratch_entries;
+    ent.clear();
+    for (int64_t j = 0; j < n_blocks; ++j) {
+        const int32_t blk = block_table[j], slot = host_slots[j];
+        if (blk < 0 || blk >= ctx->cfg.gpu_blocks || slot < 0 || slot >= ctx->cfg.host_blocks)
+            return EAKV_E_RANGE;
+        if (ctx->blk_stamp[blk] == ctx->epoch) return EAKV_E_INVAL;
+        ctx->blk_stamp[blk] = ctx->epoch;
+        ent.push_back(make_int2(blk, slot));
+    }
+    const int64_t m = n_blocks;
+    DeviceGuard g(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const bool host_tier = ctx->cfg.tier_location == EAKV_TIER_PINNED_HOST;
+
+    if (ctx->cfg.link_strategy == EAKV_LINK_ZERO_COPY) {
+        for (int64_t i = 0; i < m; i += ctx->max_call_blocks) {
+            const int64_t cur = std::min(ctx->max_call_blocks, m - i);
+            int rc = with_entries(ctx, ent.data() + i, cur, stream, [&](const int2* d) {
+                return launch_copy(ctx, d, cur, ctx->tier, false, host_tier, stream);
+            });
+            if (rc != EAKV_OK) return rc;
+        }
+    } else {
+        Staging& S = ctx->st_load;
+        std::vector<int2> local;
+        // the side stream may read the tier only after what precedes this call on `stream`
+        CU(cudaEventRecord(S.start, stream));
+        CU(cudaStreamWaitEvent(S.side, S.start, 0));
+        for (int64_t i = 0; i < m; i += ctx->staging_blocks) {
+            const int64_t cur = std::min(ctx->staging_blocks, m - i);
+            const int sb = S.next;
+            S.next ^= 1;
+            CU(cudaStreamWaitEvent(S.side, S.freed[sb], 0));
+            int rc = for_slot_runs(ent.data() + i, cur, [&](int64_t a, int64_t z) {
+                CU(cudaMemcpyAsync(S.buf[sb] + a * ctx->block_bytes,
+                                   ctx->tier + (int64_t)ent[i + a].y * ctx->block_bytes,
+                                   (size_t)(z - a) * ctx->block_bytes, cudaMemcpyDefault, S.side));
+                ctx->stats.memcpy_calls += 1;
+                return EAKV_OK;
+            });
+            if (rc != EAKV_OK) return rc;
+            CU(cudaEventRecord(S.ready[sb], S.side));
+            CU(cudaStreamWaitEvent(stream, S.ready[sb], 0));
+            local.resize((size_t)cur);
+            for (int64_t k = 0; k < cur; ++k) local[k] = make_int2(ent[i + k].x, (int)k);
+            rc = with_entries(ctx, local.data(), cur, stream, [&](const int2* d) {
+                return launch_copy(ctx, d, cur, S.buf[sb], false, false, stream);
+            });
+            if (rc != EAKV_OK) return rc;
+            CU(cudaEventRecord(S.freed[sb], stream));
+        }
+    }
+    ctx->stats.blocks_loaded += m;
+    ctx->stats.bytes_loaded += m * ctx->block_bytes;
+    return EAKV_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+int eakv_get_stats(const eakv_ctx* ctx, eakv_stats* out) {
+    if (!ctx || !out) return EAKV_E_INVAL;
+    *out = ctx->stats;
+    out->resident = ctx->host_tier->resident();
+    return EAKV_OK;
+}
+
+void* eakv_tier_ptr(const eakv_ctx* ctx) { return ctx ? ctx->tier : nullptr; }
+uint64_t eakv_hash_seed(const eakv_ctx* ctx) { return ctx ? ctx->seed : 0; }
+uint64_t eakv_hash_base(const eakv_ctx* ctx) { return ctx ? ctx->base : 0; }
+
+const char* eakv_strerror(int code) {
+    switch (code) {
+        case EAKV_OK: return "ok";
+        case EAKV_E_INVAL: return "invalid argument";
+        case EAKV_E_RANGE: return "block id or slot out of range";
+        case EAKV_E_CAPACITY: return "request exceeds a capacity";
+        case EAKV_E_NOMEM: return "out of memory";
+        case EAKV_E_CUDA: return "CUDA runtime error";
+        case EAKV_E_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown error";
+    }
+}
+
+const char* eakv_last_cuda_error(const eakv_ctx* ctx) { return ctx ? ctx->cuda_err.c_str() : ""; }
+
+}  // extern "C"

@@ -1,0 +1,62 @@
+// Internal declarations shared by the C-ABI translation unit and the kernel files.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+
+namespace eakv {
+
+// ---- hash ---------------------------------------------------------------------------------
+constexpr int kHashThreads = 256;
+constexpr int kHashUnroll = 4;
+constexpr int kHashTileTokens = kHashThreads * kHashUnroll * 4;   // 4096 tokens per CTA tile
+constexpr int kHashMaxBlockSize = 4096;
+constexpr int kHashMaxSmem = 64 * 1024;
+
+struct HashTile { int32_t prompt; int32_t first_block; };
+struct HashPrompt {
+    int64_t tok_off;    // first token of the prompt in tokens[]
+    int64_t blk_off;    // first key of the prompt in keys[] (and partial[])
+    int64_t nblk;       // full blocks
+    uint64_t parent;    // h_{-1}
+    int32_t tiles;      // CTA tiles covering the prompt
+    int32_t pad;
+};
+struct HashLaunch {
+    const int32_t* tokens;
+    uint64_t* keys;
+    uint64_t* partial;              // scratch: per-block partial sums
+    int* counters;                  // scratch: one ticket counter per prompt, zero between launches
+    const uint64_t* pow_table;      // B^0 .. B^b
+    const HashTile* tiles;          // NULL: single prompt, tile i starts at block i * tile_blocks
+    const HashPrompt* prompts;
+    int64_t single_nblk;
+    uint64_t single_parent;
+    const uint64_t* single_parent_ptr;   // non-NULL: read the parent from device memory instead
+    int32_t block_size;
+    int32_t tile_blocks;
+};
+cudaError_t hash_kernels_init();
+cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool generic, bool vec, cudaStream_t stream);
+
+// ---- gather / scatter ---------------------------------------------------------------------
+constexpr int kCopyThreads = 256;
+constexpr int kCopyUnroll = 4;
+constexpr int kCopySubBytes = kCopyThreads * kCopyUnroll * 16;    // 16 KiB per CTA work item
+
+struct CopyLaunch {
+    const int2* entries;        // {pool block id, tier slot (or staging index)}
+    int64_t n_entries;
+    void* const* kv_base;       // device array of 2L piece-array base pointers
+    char* tier_base;            // slot-major destination/source
+    int32_t pieces;             // 2L
+    int32_t subs_per_piece;     // ceil(piece_bytes / kCopySubBytes)
+    int64_t piece_bytes;
+};
+// to_tier: pool -> tier (store/gather); else tier -> pool (load/scatter)
+cudaError_t launch_copy_vector(const CopyLaunch& L, bool to_tier, int ctas, cudaStream_t stream);
+cudaError_t launch_copy_bulk(const CopyLaunch& L, bool to_tier, int ctas, int* error_flag,
+                             cudaStream_t stream);
+cudaError_t copy_kernels_init();
+int copy_vector_ctas_per_sm();
+
+}  // namespace eakv

@@ -1,0 +1,277 @@
+// Block-key kernel: polynomial prefix hash mod p = 2^61 - 1 over token ids.
+//
+// h_i = h_{i-1} * B + x_i (x_i = token_i + 1) is a composition of affine maps, and every
+// full block contributes the same multiplier A = B^b, so the work splits in two:
+//   1. block partials  c_j = sum_k x_{jb+k} * B^{b-1-k} mod p, independent per block:
+//      coalesced 16-byte token loads, a 32x61-bit multiply-accumulate per token against a
+//      power table in shared memory, lazy reduction once per four tokens.  HBM/ALU bound.
+//   2. keys  h_j = h_{j-1} * A + c_j : a scan over affine pairs (a, c) with
+//      (a1,c1) o (a2,c2) = (a1 a2, c1 a2 + c2); each thread folds a run of blocks, a
+//      warp-level shuffle scan combines threads, shared memory combines warps.
+// Both run in one launch: each CTA publishes its tile's partials, takes a ticket on the
+// prompt's counter, and the CTA that draws the last ticket of a prompt runs that prompt's
+// scan.  No CTA ever waits for another, so there is no spin loop anywhere.
+#include "eakv_internal.h"
+
+namespace eakv {
+
+static constexpr uint64_t P61 = (1ull << 61) - 1;
+
+__device__ __forceinline__ uint64_t reduce_once(uint64_t r) {   // r < 2^63
+    r = (r & P61) + (r >> 61);
+    if (r >= P61) r -= P61;
+    return r;
+}
+
+__device__ __forceinline__ uint64_t mulmod61(uint64_t a, uint64_t b) {   // a, b < 2^61
+    const uint64_t lo = a * b;
+    const uint64_t hi = __umul64hi(a, b);                 // < 2^58
+    // 2^61 == 1 (mod p): value = (lo mod 2^61) + (lo >> 61) + hi * 8
+    return reduce_once((lo & P61) + ((hi << 3) | (lo >> 61)));
+}
+
+__device__ __forceinline__ uint64_t addmod61(uint64_t a, uint64_t b) {
+    uint64_t r = a + b;
+    if (r >= P61) r -= P61;
+    return r;
+}
+
+// sum of four (token+1) * power products, reduced to [0, p)
+__device__ __forceinline__ uint64_t dot4(int4 t, const uint64_t* __restrict__ pw, int e_first) {
+    // token k of the chunk multiplies B^(e_first - k)
+    const uint32_t x[4] = {(uint32_t)t.x + 1u, (uint32_t)t.y + 1u, (uint32_t)t.z + 1u,
+                           (uint32_t)t.w + 1u};
+    uint64_t s_lo = 0, s_hi = 0;
+    uint32_t carry = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint64_t w = pw[e_first - k];
+        const uint64_t lo = (uint64_t)x[k] * (uint32_t)w;           // < 2^64
+        const uint64_t hi = (uint64_t)x[k] * (uint32_t)(w >> 32);   // < 2^61
+        s_lo += lo;
+        carry += (s_lo < lo);
+        s_hi += hi;                                                 // < 2^63
+    }
+    // total = s_lo + carry * 2^64 + s_hi * 2^32;  2^64 == 8,  s_hi * 2^32 = (s_hi >> 29) * 2^61 + (s_hi & (2^29-1)) << 32
+    uint64_t r = (s_lo & P61) + (s_lo >> 61) + 8ull * carry + (s_hi >> 29) +
+                 ((s_hi & ((1ull << 29) - 1)) << 32);               // < 2^63
+    return reduce_once(r);
+}
+
+struct Pair { uint64_t a, c; };   // h -> h * a + c
+
+__device__ __forceinline__ Pair compose(Pair first, Pair second) {
+    Pair r;
+    r.a = mulmod61(first.a, second.a);
+    r.c = addmod61(mulmod61(first.c, second.a), second.c);
+    return r;
+}
+
+// Scan of one prompt's block partials into keys, by one whole CTA.
+//   partial[0..nblk) -> keys[0..nblk),  keys[j] = keys[j-1] * A + partial[j], keys[-1] = parent
+__device__ void scan_prompt(const uint64_t* partial, uint64_t* keys, int64_t nblk, uint64_t parent,
+                            uint64_t A, Pair* warp_tot /* smem [32] */) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
+    const int64_t per = (nblk + nthr - 1) / nthr;
+    const int64_t lo = min((int64_t)tid * per, nblk), hi = min(lo + per, nblk);
+    // fold this thread's run
+    Pair mine{1, 0};
+    for (int64_t j = lo; j < hi; ++j) {
+        const uint64_t c = __ldcg(partial + j);
+        mine.a = mulmod61(mine.a, A);
+        mine.c = addmod61(mulmod61(mine.c, A), c);
+    }
+    // inclusive warp scan over threads (earlier lanes apply first)
+    Pair inc = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        Pair up;
+        up.a = __shfl_up_sync(0xffffffffu, inc.a, d);
+        up.c = __shfl_up_sync(0xffffffffu, inc.c, d);
+        if (lane >= d) inc = compose(up, inc);
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        Pair w = lane < nwarp ? warp_tot[lane] : Pair{1, 0};
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            Pair up;
+            up.a = __shfl_up_sync(0xffffffffu, w.a, d);
+            up.c = __shfl_up_sync(0xffffffffu, w.c, d);
+            if (lane >= d) w = compose(up, w);
+        }
+        warp_tot[lane] = w;   // inclusive over warps
+    }
+    __syncthreads();
+    // exclusive prefix of this thread = (warps before) o (lanes before)
+    Pair exc;
+    exc.a = __shfl_up_sync(0xffffffffu, inc.a, 1);
+    exc.c = __shfl_up_sync(0xffffffffu, inc.c, 1);
+    if (lane == 0) exc = Pair{1, 0};
+    if (warp > 0) exc = compose(warp_tot[warp - 1], exc);
+    uint64_t h = addmod61(mulmod61(parent, exc.a), exc.c);
+    for (int64_t j = lo; j < hi; ++j) {
+        h = addmod61(mulmod61(h, A), __ldcg(partial + j));
+        keys[j] = h;
+    }
+    __syncthreads();
+}
+
+// tile = kHashTileChunks 16-byte chunks (or fewer at a prompt's end)
+template <bool VEC>
+__global__ void __launch_bounds__(kHashThreads)
+hash_blocks_kernel(HashLaunch L) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint64_t* pw = reinterpret_cast<uint64_t*>(smem_raw);             // [b + 1]
+    uint64_t* chunk_sum = pw + L.block_size + 1;                      // [tile chunks]
+    __shared__ Pair warp_tot[32];
+    __shared__ int is_last;
+
+    const int tid = threadIdx.x;
+    for (int e = tid; e <= L.block_size; e += blockDim.x) pw[e] = L.pow_table[e];
+
+    // which prompt and which run of blocks
+    int32_t p = 0;
+    int64_t first_blk = (int64_t)blockIdx.x * L.tile_blocks;
+    int64_t tok0 = 0, blk0 = 0, nblk = L.single_nblk;
+    uint64_t parent = L.single_parent;
+    int32_t tiles_in_prompt = gridDim.x;
+    if (L.tiles != nullptr) {
+        const HashTile t = L.tiles[blockIdx.x];
+        p = t.prompt;
+        first_blk = t.first_block;
+        const HashPrompt hp = L.prompts[p];
+        tok0 = hp.tok_off; blk0 = hp.blk_off; nblk = hp.nblk; parent = hp.parent;
+        tiles_in_prompt = hp.tiles;
+    } else if (L.single_parent_ptr != nullptr) {
+        parent = *L.single_parent_ptr;
+    }
+    const int64_t nb_tile = min((int64_t)L.tile_blocks, nblk - first_blk);
+    const int cpb = L.block_size >> 2;                                // chunks per block
+    const int n_chunks = (int)nb_tile * cpb;
+    const int32_t* tok = L.tokens + tok0 + first_blk * L.block_size;
+    __syncthreads();
+
+    // step 1a: per-chunk dot products
+    for (int c0 = 0; c0 < n_chunks; c0 += kHashThreads * kHashUnroll) {
+        int4 t[kHashUnroll];
+#pragma unroll
+        for (int u = 0; u < kHashUnroll; ++u) {
+            const int c = c0 + u * kHashThreads + tid;
+            if (c < n_chunks) {
+                if (VEC) {
+                    t[u] = __ldcs(reinterpret_cast<const int4*>(tok) + c);
+                } else {
+                    t[u].x = tok[4 * c]; t[u].y = tok[4 * c + 1];
+                    t[u].z = tok[4 * c + 2]; t[u].w = tok[4 * c + 3];
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kHashUnroll; ++u) {
+            const int c = c0 + u * kHashThreads + tid;
+            if (c < n_chunks) {
+                const int cib = c % cpb;
+                chunk_sum[c] = dot4(t[u], pw, L.block_size - 1 - 4 * cib);
+            }
+        }
+    }
+    __syncthreads();
+    // step 1b: per-block sums of chunk values -> partials in global scratch
+    uint64_t* partial = L.partial + blk0;
+    for (int j = tid; j < (int)nb_tile; j += blockDim.x) {
+        uint64_t s = 0;
+        const uint64_t* cs = chunk_sum + j * cpb;
+        for (int k = 0; k < cpb; ++k) s = addmod61(s, cs[k]);
+        __stcg(partial + first_blk + j, s);
+    }
+    // step 2: the CTA that draws the prompt's last ticket scans it
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int ticket = atomicAdd(L.counters + p, 1);
+        is_last = (ticket == tiles_in_prompt - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    scan_prompt(partial, L.keys + blk0, nblk, parent, pw[L.block_size], warp_tot);
+    if (tid == 0) L.counters[p] = 0;   // ready for the next launch
+}
+
+// Any block size (not a multiple of 4): one thread per block, same two steps.
+__global__ void __launch_bounds__(kHashThreads)
+hash_blocks_generic_kernel(HashLaunch L) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint64_t* pw = reinterpret_cast<uint64_t*>(smem_raw);
+    __shared__ Pair warp_tot[32];
+    __shared__ int is_last;
+    const int tid = threadIdx.x;
+    for (int e = tid; e <= L.block_size; e += blockDim.x) pw[e] = L.pow_table[e];
+    int32_t p = 0;
+    int64_t first_blk = (int64_t)blockIdx.x * L.tile_blocks;
+    int64_t tok0 = 0, blk0 = 0, nblk = L.single_nblk;
+    uint64_t parent = L.single_parent;
+    int32_t tiles_in_prompt = gridDim.x;
+    if (L.tiles != nullptr) {
+        const HashTile t = L.tiles[blockIdx.x];
+        p = t.prompt;
+        first_blk = t.first_block;
+        const HashPrompt hp = L.prompts[p];
+        tok0 = hp.tok_off; blk0 = hp.blk_off; nblk = hp.nblk; parent = hp.parent;
+        tiles_in_prompt = hp.tiles;
+    } else if (L.single_parent_ptr != nullptr) {
+        parent = *L.single_parent_ptr;
+    }
+    const int64_t nb_tile = min((int64_t)L.tile_blocks, nblk - first_blk);
+    __syncthreads();
+    uint64_t* partial = L.partial + blk0;
+    for (int64_t j = tid; j < nb_tile; j += blockDim.x) {
+        const int32_t* t = L.tokens + tok0 + (first_blk + j) * L.block_size;
+        uint64_t s = 0;
+        for (int k = 0; k < L.block_size; ++k)
+            s = addmod61(s, mulmod61((uint64_t)((uint32_t)t[k] + 1u), pw[L.block_size - 1 - k]));
+        __stcg(partial + first_blk + j, s);
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int ticket = atomicAdd(L.counters + p, 1);
+        is_last = (ticket == tiles_in_prompt - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    scan_prompt(partial, L.keys + blk0, nblk, parent, pw[L.block_size], warp_tot);
+    if (tid == 0) L.counters[p] = 0;
+}
+
+cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool generic, bool vec, cudaStream_t stream) {
+    if (n_tiles <= 0) return cudaSuccess;
+    if (generic) {
+        const size_t smem = (size_t)(L.block_size + 1) * 8;
+        hash_blocks_generic_kernel<<<n_tiles, kHashThreads, smem, stream>>>(L);
+    } else {
+        const size_t smem = (size_t)(L.block_size + 1) * 8 +
+                            (size_t)L.tile_blocks * (L.block_size / 4) * 8;
+        if (vec) hash_blocks_kernel<true><<<n_tiles, kHashThreads, smem, stream>>>(L);
+        else     hash_blocks_kernel<false><<<n_tiles, kHashThreads, smem, stream>>>(L);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t hash_kernels_init() {
+    // allow tiles whose chunk sums plus a large power table exceed the 48 KB default
+    cudaError_t e = cudaFuncSetAttribute(hash_blocks_kernel<true>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kHashMaxSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(hash_blocks_kernel<false>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kHashMaxSmem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(hash_blocks_generic_kernel,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, kHashMaxSmem);
+}
+
+}  // namespace eakv

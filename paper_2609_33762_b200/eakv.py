@@ -1,0 +1,294 @@
+"""ctypes binding of libeakv.so: same names as the C entry points, argument marshalling
+only.  Device buffers are passed as integer addresses (``tensor.data_ptr()``), host arrays
+as numpy arrays; a negative status raises ``EakvError``.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+OK, E_INVAL, E_RANGE, E_CAPACITY, E_NOMEM, E_CUDA, E_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
+POLICY_WRITE_ALL, POLICY_FILTER_FIXED, POLICY_FILTER_CONDITIONED = 0, 1, 2
+LINK_ZERO_COPY, LINK_STAGED = 0, 1
+TIER_PINNED_HOST, TIER_DEVICE = 0, 1
+COPY_VECTOR, COPY_BULK = 0, 1
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libeakv.so")
+_lib = None
+
+
+class EakvError(RuntimeError):
+    def __init__(self, code, where, detail=""):
+        self.code = code
+        msg = f"{where}: {lib().eakv_strerror(code).decode()} ({code})"
+        if detail:
+            msg += f": {detail}"
+        super().__init__(msg)
+
+
+class Config(C.Structure):
+    _fields_ = [
+        ("num_layers", C.c_int32), ("kv_heads", C.c_int32), ("head_dim", C.c_int32),
+        ("block_size", C.c_int32), ("elem_bytes", C.c_int32),
+        ("gpu_blocks", C.c_int64), ("host_blocks", C.c_int64), ("gpu_index_blocks", C.c_int64),
+        ("kv_base", C.POINTER(C.c_void_p)),
+        ("hash_base", C.c_uint64), ("hash_seed", C.c_uint64),
+        ("policy", C.c_int32), ("kappa_blocks", C.c_int32), ("theta_percent", C.c_int32),
+        ("len_window", C.c_int32), ("window_ms", C.c_int64), ("telemetry", C.c_int32),
+        ("link_strategy", C.c_int32), ("tier_location", C.c_int32), ("copy_path", C.c_int32),
+        ("copy_ctas", C.c_int32),
+        ("staging_bytes", C.c_int64), ("max_call_blocks", C.c_int64),
+        ("hash_scratch_blocks", C.c_int64), ("tier_memory", C.c_void_p),
+    ]
+
+
+class Stats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in (
+        "requests", "references", "hits", "admitted", "declined", "evicted",
+        "declined_requests", "pressure_requests", "resident",
+        "tokens_hashed", "blocks_stored", "blocks_loaded", "bytes_stored", "bytes_loaded",
+        "kernel_launches", "memcpy_calls")]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class StepInfo(C.Structure):
+    _fields_ = [("host_prefix_blocks", C.c_int64), ("new_chunks", C.c_int64),
+                ("pressure", C.c_int32), ("save", C.c_int32)]
+
+
+EXPORTS = [
+    "eakv_config_init", "eakv_create", "eakv_destroy", "eakv_hash_blocks",
+    "eakv_hash_blocks_batched", "eakv_match", "eakv_tier_step", "eakv_gpu_tier_step",
+    "eakv_gpu_tier_release", "eakv_store", "eakv_load", "eakv_sync", "eakv_get_stats",
+    "eakv_tier_ptr", "eakv_hash_seed", "eakv_hash_base", "eakv_strerror", "eakv_last_cuda_error",
+]
+
+
+def lib():
+    """Load libeakv.so (once).  Raises if it has not been built: there is no fallback."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2609_33762_b200.build` "
+            "(the eakv path has no CPU or PyTorch fallback)")
+    L = C.CDLL(_LIB_PATH)
+    vp, i32, i64, u64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64
+    L.eakv_config_init.argtypes = [C.POINTER(Config)]
+    L.eakv_create.argtypes = [C.POINTER(Config), C.POINTER(vp)]
+    L.eakv_destroy.argtypes = [vp]
+    L.eakv_hash_blocks.argtypes = [vp, vp, i64, u64, vp, C.POINTER(i64), vp]
+    L.eakv_hash_blocks_batched.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp]
+    L.eakv_match.argtypes = [vp, vp, i64, C.POINTER(i64), C.POINTER(i64), vp, vp]
+    L.eakv_tier_step.argtypes = [vp, vp, i64, i64, i64, i64, vp, vp, vp, vp, vp,
+                                 C.POINTER(i64), C.POINTER(StepInfo)]
+    L.eakv_gpu_tier_step.argtypes = [vp, vp, i64, i32, vp, vp, C.POINTER(i32)]
+    L.eakv_gpu_tier_release.argtypes = [vp, i32]
+    L.eakv_store.argtypes = [vp, vp, vp, vp, i64, vp]
+    L.eakv_load.argtypes = [vp, vp, vp, i64, vp]
+    L.eakv_sync.argtypes = [vp]
+    L.eakv_get_stats.argtypes = [vp, C.POINTER(Stats)]
+    L.eakv_tier_ptr.argtypes = [vp]
+    L.eakv_tier_ptr.restype = vp
+    L.eakv_hash_seed.argtypes = [vp]
+    L.eakv_hash_seed.restype = u64
+    L.eakv_hash_base.argtypes = [vp]
+    L.eakv_hash_base.restype = u64
+    L.eakv_strerror.argtypes = [C.c_int]
+    L.eakv_strerror.restype = C.c_char_p
+    L.eakv_last_cuda_error.argtypes = [vp]
+    L.eakv_last_cuda_error.restype = C.c_char_p
+    _lib = L
+    return L
+
+
+def _np(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a, a.ctypes.data_as(C.c_void_p)
+
+
+def _stream(s):
+    if s is None:
+        return None
+    return C.c_void_p(int(getattr(s, "cuda_stream", s)))
+
+
+class Context:
+    """Owns one eakv_ctx.  Method names mirror the C entry points."""
+
+    def __init__(self, *, num_layers, kv_heads, head_dim, block_size, gpu_blocks, host_blocks,
+                 kv_base, elem_bytes=2, gpu_index_blocks=0, hash_base=0, hash_seed=0,
+                 policy=POLICY_WRITE_ALL, kappa_blocks=8, theta_percent=95, len_window=256,
+                 window_ms=60_000, telemetry=1, link_strategy=LINK_ZERO_COPY,
+                 tier_location=TIER_PINNED_HOST, copy_path=COPY_VECTOR, copy_ctas=0,
+                 staging_bytes=0, max_call_blocks=0, hash_scratch_blocks=0, tier_memory=0):
+        L = lib()
+        cfg = Config()
+        L.eakv_config_init(C.byref(cfg))
+        ptrs = (C.c_void_p * len(kv_base))(*[int(p) for p in kv_base])
+        if len(kv_base) != 2 * num_layers:
+            raise ValueError("kv_base must hold 2 * num_layers device pointers")
+        cfg.num_layers, cfg.kv_heads, cfg.head_dim = num_layers, kv_heads, head_dim
+        cfg.block_size, cfg.elem_bytes = block_size, elem_bytes
+        cfg.gpu_blocks, cfg.host_blocks, cfg.gpu_index_blocks = gpu_blocks, host_blocks, gpu_index_blocks
+        cfg.kv_base = C.cast(ptrs, C.POINTER(C.c_void_p))
+        cfg.hash_base, cfg.hash_seed = hash_base, hash_seed
+        cfg.policy, cfg.kappa_blocks, cfg.theta_percent = policy, kappa_blocks, theta_percent
+        cfg.len_window, cfg.window_ms, cfg.telemetry = len_window, window_ms, telemetry
+        cfg.link_strategy, cfg.tier_location = link_strategy, tier_location
+        cfg.copy_path, cfg.copy_ctas = copy_path, copy_ctas
+        cfg.staging_bytes, cfg.max_call_blocks = staging_bytes, max_call_blocks
+        cfg.hash_scratch_blocks = hash_scratch_blocks
+        cfg.tier_memory = int(tier_memory) if tier_memory else None
+        self._h = C.c_void_p()
+        rc = L.eakv_create(C.byref(cfg), C.byref(self._h))
+        if rc != OK:
+            self._h = None
+            raise EakvError(rc, "eakv_create")
+        self.block_size = block_size
+        self.host_blocks = host_blocks
+        self.piece_bytes = block_size * kv_heads * head_dim * elem_bytes
+        self.block_bytes = 2 * num_layers * self.piece_bytes
+        self.tier_location = tier_location
+
+    # -- lifetime ---------------------------------------------------------------------------
+    def eakv_destroy(self):
+        if self._h:
+            lib().eakv_destroy(self._h)
+            self._h = None
+
+    close = eakv_destroy
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.eakv_destroy()
+
+    def __del__(self):
+        try:
+            self.eakv_destroy()
+        except Exception:
+            pass
+
+    def _check(self, rc, where):
+        if rc != OK:
+            detail = lib().eakv_last_cuda_error(self._h).decode() if rc == E_CUDA else ""
+            raise EakvError(rc, where, detail)
+
+    # -- hashing ----------------------------------------------------------------------------
+    def eakv_hash_blocks(self, tokens_dev, n_tokens, parent_hash, hashes_dev, stream=None):
+        n = C.c_int64(0)
+        rc = lib().eakv_hash_blocks(self._h, C.c_void_p(int(tokens_dev)), int(n_tokens),
+                                    C.c_uint64(int(parent_hash)), C.c_void_p(int(hashes_dev)),
+                                    C.byref(n), _stream(stream))
+        self._check(rc, "eakv_hash_blocks")
+        return n.value
+
+    def eakv_hash_blocks_batched(self, tokens_dev, offsets, parents, hashes_dev, stream=None):
+        off, off_p = _np(offsets, np.int64)
+        n_prompts = len(off) - 1
+        par_p = None
+        if parents is not None:
+            par, par_p = _np(parents, np.uint64)
+        out = np.zeros(n_prompts + 1, dtype=np.int64)
+        rc = lib().eakv_hash_blocks_batched(self._h, C.c_void_p(int(tokens_dev)), off_p, n_prompts,
+                                            par_p, C.c_void_p(int(hashes_dev)),
+                                            out.ctypes.data_as(C.c_void_p), _stream(stream))
+        self._check(rc, "eakv_hash_blocks_batched")
+        return out
+
+    # -- control plane ----------------------------------------------------------------------
+    def eakv_match(self, hashes):
+        h, hp = _np(hashes, np.uint64)
+        n = len(h)
+        G, H = C.c_int64(0), C.c_int64(0)
+        gids = np.full(n, -1, dtype=np.int32)
+        slots = np.full(n, -1, dtype=np.int32)
+        rc = lib().eakv_match(self._h, hp, n, C.byref(G), C.byref(H),
+                              gids.ctypes.data_as(C.c_void_p), slots.ctypes.data_as(C.c_void_p))
+        self._check(rc, "eakv_match")
+        return G.value, H.value, gids[:G.value], slots[:H.value]
+
+    def eakv_tier_step(self, hashes, agent_id, n_tokens, now_ms):
+        h, hp = _np(hashes, np.uint64)
+        n = len(h)
+        hit = np.zeros(n, dtype=np.uint8)
+        admit = np.zeros(n, dtype=np.uint8)
+        slot = np.zeros(n, dtype=np.int32)
+        ek = np.zeros(n, dtype=np.uint64)
+        es = np.zeros(n, dtype=np.int32)
+        nev = C.c_int64(n)
+        info = StepInfo()
+        vp = lambda a: a.ctypes.data_as(C.c_void_p)
+        rc = lib().eakv_tier_step(self._h, hp, n, int(agent_id), int(n_tokens), int(now_ms),
+                                  vp(hit), vp(admit), vp(slot), vp(ek), vp(es), C.byref(nev),
+                                  C.byref(info))
+        self._check(rc, "eakv_tier_step")
+        k = nev.value
+        return dict(hit=hit, admit=admit, slot=slot, evicted_keys=ek[:k], evicted_slots=es[:k],
+                    host_prefix_blocks=info.host_prefix_blocks, new_chunks=info.new_chunks,
+                    pressure=bool(info.pressure), save=bool(info.save))
+
+    def eakv_gpu_tier_step(self, hashes, need_tail):
+        h, hp = _np(hashes, np.uint64)
+        n = len(h)
+        res = np.zeros(n, dtype=np.uint8)
+        blk = np.zeros(n, dtype=np.int32)
+        tail = C.c_int32(-1)
+        rc = lib().eakv_gpu_tier_step(self._h, hp, n, int(bool(need_tail)),
+                                      res.ctypes.data_as(C.c_void_p),
+                                      blk.ctypes.data_as(C.c_void_p), C.byref(tail))
+        self._check(rc, "eakv_gpu_tier_step")
+        return res, blk, tail.value
+
+    def eakv_gpu_tier_release(self, block_id):
+        self._check(lib().eakv_gpu_tier_release(self._h, int(block_id)), "eakv_gpu_tier_release")
+
+    # -- data plane -------------------------------------------------------------------------
+    def eakv_store(self, block_table, admit_mask, host_slots, stream=None):
+        bt, btp = _np(block_table, np.int32)
+        hs, hsp = _np(host_slots, np.int32)
+        amp = None
+        if admit_mask is not None:
+            am, amp = _np(admit_mask, np.uint8)
+        rc = lib().eakv_store(self._h, btp, amp, hsp, len(bt), _stream(stream))
+        self._check(rc, "eakv_store")
+
+    def eakv_load(self, host_slots, block_table, stream=None):
+        bt, btp = _np(block_table, np.int32)
+        hs, hsp = _np(host_slots, np.int32)
+        rc = lib().eakv_load(self._h, hsp, btp, len(bt), _stream(stream))
+        self._check(rc, "eakv_load")
+
+    def eakv_sync(self):
+        self._check(lib().eakv_sync(self._h), "eakv_sync")
+
+    # -- introspection ----------------------------------------------------------------------
+    def eakv_get_stats(self):
+        s = Stats()
+        self._check(lib().eakv_get_stats(self._h, C.byref(s)), "eakv_get_stats")
+        return s.as_dict()
+
+    def eakv_tier_ptr(self):
+        return lib().eakv_tier_ptr(self._h)
+
+    def eakv_hash_seed(self):
+        return lib().eakv_hash_seed(self._h)
+
+    def eakv_hash_base(self):
+        return lib().eakv_hash_base(self._h)
+
+    def tier_host_view(self):
+        """numpy uint8 view [host_blocks, 2L, piece_bytes] of a pinned-host tier."""
+        if self.tier_location != TIER_PINNED_HOST:
+            raise ValueError("tier is not in host memory")
+        n = self.host_blocks * self.block_bytes
+        buf = (C.c_uint8 * n).from_address(self.eakv_tier_ptr())
+        return np.frombuffer(buf, dtype=np.uint8).reshape(
+            self.host_blocks, self.block_bytes // self.piece_bytes, self.piece_bytes)

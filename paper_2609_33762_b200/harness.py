@@ -1,0 +1,145 @@
+"""Agent-turn driver over the eakv C-ABI.  PyTorch supplies device memory and streams
+only; every step of the path (block keys, prefix match, tier bookkeeping, restore, store)
+runs inside libeakv.  The "prefill" of a real serving engine is replaced by writing each
+fresh block's synthetic payload into the paged pool.
+
+One turn (the order follows the paper: lookup at scheduling time, restore before compute,
+store after): hash -> match -> host tier step -> GPU tier step -> load blocks [G, H) ->
+fill fresh blocks -> store admitted blocks.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import eakv
+
+
+class PagedPool:
+    """2L paged arrays [gpu_blocks, piece_bytes] as int16 tensors on one CUDA device."""
+
+    def __init__(self, shape, gpu_blocks, device="cuda:0", fill=None):
+        self.shape = shape
+        self.gpu_blocks = int(gpu_blocks)
+        self.device = torch.device(device)
+        W = shape.piece_bytes // 2
+        self.words = W
+        alloc = torch.zeros if fill is None else torch.empty
+        self.pieces = [alloc((self.gpu_blocks, W), dtype=torch.int16, device=self.device)
+                       for _ in range(shape.pieces_per_block)]
+        if fill is not None:
+            for q, t in enumerate(self.pieces):
+                fill(q, t)
+
+    @property
+    def kv_base(self):
+        return [t.data_ptr() for t in self.pieces]
+
+
+class AgentServer:
+    def __init__(self, shape, gpu_blocks, host_blocks, payload, *, device="cuda:0",
+                 gpu_index_blocks=0, incremental_hash=False, data_plane=True, **ctx_kwargs):
+        """``payload(keys, q, n_words)`` returns the int16/uint16 words of piece q for the
+        blocks with these keys, as a numpy array or a tensor on ``device``."""
+        self.shape = shape
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        # data_plane=False runs keys, matching and both tiers' bookkeeping only; the pool is
+        # then a one-block placeholder and no KV bytes move
+        self.data_plane = data_plane
+        self.pool = PagedPool(shape, gpu_blocks if data_plane else 1, device)
+        if not data_plane and "tier_memory" not in ctx_kwargs:
+            # bookkeeping-only run: adopt a token buffer so no tier-sized memory is pinned
+            self._no_tier = torch.zeros(16, dtype=torch.uint8, device=self.device)
+            ctx_kwargs["tier_memory"] = self._no_tier.data_ptr()
+            ctx_kwargs["tier_location"] = eakv.TIER_DEVICE
+        self.ctx = eakv.Context(
+            num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+            block_size=shape.block_size, elem_bytes=shape.elem_bytes, gpu_blocks=gpu_blocks,
+            host_blocks=host_blocks, gpu_index_blocks=gpu_index_blocks, kv_base=self.pool.kv_base,
+            **ctx_kwargs)
+        self.payload = payload
+        self.incremental = incremental_hash
+        self.stream = torch.cuda.current_stream(self.device)
+        self.b = shape.block_size
+        self.seed = self.ctx.eakv_hash_seed()
+        self._agent_keys = {}          # agent -> np.uint64 keys of its previous prompt
+        self.records = []
+        self.totals = dict(prompt_tokens=0, fresh_tokens=0, loaded_blocks=0, stored_blocks=0,
+                           gpu_hit_blocks=0, host_hit_blocks=0)
+
+    def close(self):
+        self.ctx.close()
+
+    # -- block keys -------------------------------------------------------------------------
+    def block_keys(self, tokens: np.ndarray, agent) -> np.ndarray:
+        n = len(tokens)
+        nblk = n // self.b
+        prev = self._agent_keys.get(agent) if self.incremental else None
+        start = 0 if prev is None else min(len(prev), nblk)
+        out = np.empty(nblk, dtype=np.uint64)
+        if start:
+            out[:start] = prev[:start]
+        if nblk > start:
+            seg = np.ascontiguousarray(tokens[start * self.b: nblk * self.b], dtype=np.int32)
+            tok_dev = torch.from_numpy(seg).to(self.device, non_blocking=False)
+            keys_dev = torch.empty(nblk - start, dtype=torch.int64, device=self.device)
+            parent = int(out[start - 1]) if start else self.seed
+            got = self.ctx.eakv_hash_blocks(tok_dev.data_ptr(), len(seg), parent,
+                                            keys_dev.data_ptr(), self.stream)
+            assert got == nblk - start
+            out[start:] = keys_dev.cpu().numpy().view(np.uint64)
+        if self.incremental:
+            self._agent_keys[agent] = out
+        return out
+
+    # -- one request ------------------------------------------------------------------------
+    def turn(self, tokens, agent, now_ms):
+        tokens = np.asarray(tokens, dtype=np.int32)
+        n = len(tokens)
+        keys = self.block_keys(tokens, agent)
+        nblk = len(keys)
+        G, H, _gids, host_slots = self.ctx.eakv_match(keys)
+        step = self.ctx.eakv_tier_step(keys, agent, n, now_ms)
+        resident, blocks, tail = self.ctx.eakv_gpu_tier_step(keys, n % self.b != 0)
+        cover = max(G, H)
+        lo, hi = (G, H) if H > G else (G, G)
+        if hi > lo and self.data_plane:
+            self.ctx.eakv_load(host_slots[lo:hi], blocks[lo:hi], self.stream)
+        fill = [j for j in range(cover, nblk) if not resident[j]]
+        if fill and self.data_plane:
+            ids = torch.as_tensor(blocks[fill].astype(np.int64), device=self.device)
+            fkeys = keys[fill]
+            for q, piece in enumerate(self.pool.pieces):
+                w = self.payload(fkeys, q, self.pool.words)
+                if isinstance(w, np.ndarray):
+                    w = torch.from_numpy(w.view(np.int16)).to(self.device)
+                piece[ids] = w.view(torch.int16)
+        if self.data_plane and step["admit"].any():
+            self.ctx.eakv_store(blocks, step["admit"], step["slot"], self.stream)
+        if tail >= 0:
+            self.ctx.eakv_gpu_tier_release(tail)
+        rec = dict(agent=agent, now_ms=now_ms, n_tokens=n, keys=keys, G=G, H=H,
+                   new_chunks=step["new_chunks"], pressure=step["pressure"], save=step["save"],
+                   hit=step["hit"], admit=step["admit"], slot=step["slot"],
+                   evicted=list(zip(step["evicted_keys"].tolist(), step["evicted_slots"].tolist())),
+                   gpu_resident=resident, gpu_block=blocks, loaded=hi - lo,
+                   stored=int(step["admit"].sum()), fresh_tokens=n - cover * self.b,
+                   filled=len(fill))
+        t = self.totals
+        t["prompt_tokens"] += n
+        t["fresh_tokens"] += rec["fresh_tokens"]
+        t["loaded_blocks"] += rec["loaded"]
+        t["stored_blocks"] += rec["stored"]
+        t["gpu_hit_blocks"] += G
+        t["host_hit_blocks"] += H
+        self.records.append(rec)
+        return rec
+
+    def run(self, trace, limit=None):
+        for i, req in enumerate(trace.requests):
+            if limit is not None and i >= limit:
+                break
+            self.turn(trace.prompt(req), req.agent, req.time_ms)
+        self.ctx.eakv_sync()
+        return self.records

@@ -1,0 +1,138 @@
+"""GPU parity: eakv_hash_blocks / eakv_hash_blocks_batched against oracle.hash, bit-exact."""
+import numpy as np
+import pytest
+
+from oracle import hash as oh
+
+from gpu_util import gpu_keys, hash_ctx, require_gpu, torch
+
+pytestmark = pytest.mark.gpu
+P = (1 << 61) - 1
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _gpu():
+    require_gpu()
+
+
+@pytest.mark.parametrize("b", [16, 32, 4, 12, 10, 1, 1024, 256])
+def test_lengths_and_block_sizes(b):
+    rng = np.random.default_rng(b)
+    ctx = hash_ctx(b)
+    lengths = [0, 1, b - 1, b, b + 1, 31, 32, 33, 1023, 1024, 1025, 4095, 4096, 4097,
+               5 * 4096 + 3 * b + 1, 131072]
+    for n in lengths:
+        if n < 0:
+            continue
+        toks = rng.integers(0, 151936, size=n, dtype=np.int32)
+        assert gpu_keys(ctx, toks) == oh.hash_blocks(toks.tolist(), b), (b, n)
+    ctx.close()
+
+
+def test_extreme_token_ids_and_parents():
+    ctx = hash_ctx(16)
+    hi = np.full(16 * 40 + 5, 2**31 - 1, dtype=np.int32)
+    zero = np.zeros(16 * 40, dtype=np.int32)
+    for toks in (hi, zero):
+        for parent in (0, 1, P - 1, oh.HASH_SEED):
+            assert gpu_keys(ctx, toks, parent) == oh.hash_blocks(toks.tolist(), 16, parent)
+    # parents at or above p are reduced first
+    toks = np.arange(64, dtype=np.int32)
+    assert gpu_keys(ctx, toks, P + 5) == oh.hash_blocks(toks.tolist(), 16, 5)
+    ctx.close()
+
+
+def test_canonical_zero_key():
+    # pick the parent so that the first block's key is exactly 0 (never p)
+    b = 4
+    ctx = hash_ctx(b)
+    B = oh.HASH_BASE
+    toks = [7, 0, 151935, 3, 9, 9, 9, 9]
+    c = 0
+    for t in toks[:b]:
+        c = (c * B + t + 1) % P
+    parent = (-c * pow(pow(B, b, P), P - 2, P)) % P
+    keys = gpu_keys(ctx, toks, parent)
+    assert keys[0] == 0
+    assert keys == oh.hash_blocks(toks, b, parent)
+    ctx.close()
+
+
+def test_resume_and_unaligned_pointers():
+    b = 16
+    ctx = hash_ctx(b)
+    rng = np.random.default_rng(3)
+    toks = rng.integers(0, 151936, size=b * 300 + 7, dtype=np.int32)
+    full = oh.hash_blocks(toks.tolist(), b)
+    assert gpu_keys(ctx, toks) == full
+    for j in (1, 2, 255, 256, 257, 299):
+        assert gpu_keys(ctx, toks[j * b:], parent=full[j - 1]) == full[j:]
+    # token pointer only 4-byte aligned: scalar load path
+    for off in (1, 2, 3):
+        assert gpu_keys(ctx, toks, offset_tokens=off) == full
+    ctx.close()
+
+
+def test_scratch_smaller_than_prompt_chains_launches():
+    b = 16
+    ctx = hash_ctx(b, hash_scratch_blocks=300)
+    rng = np.random.default_rng(4)
+    toks = rng.integers(0, 151936, size=b * 1000 + 3, dtype=np.int32)
+    assert gpu_keys(ctx, toks) == oh.hash_blocks(toks.tolist(), b)
+    ctx.close()
+
+
+@pytest.mark.parametrize("b", [16, 32, 10])
+def test_batched_ragged(b):
+    ctx = hash_ctx(b)
+    rng = np.random.default_rng(5 + b)
+    lens = [0, 1, b - 1, b, 3 * b + 1, 4096, 4096 + b, 9000, 0, 70000, b * 256, 5]
+    if b % 4 == 0:
+        lens = [x - x % 4 if i % 2 == 0 else x for i, x in enumerate(lens)]   # some aligned starts
+    offsets = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    toks = rng.integers(0, 151936, size=int(offsets[-1]), dtype=np.int32)
+    parents = [int(x) for x in rng.integers(0, P, size=len(lens), dtype=np.uint64)]
+    dev = torch.from_numpy(toks).cuda()
+    total = sum(x // b for x in lens)
+    for par in (None, parents):
+        out = torch.full((total + 1,), -1, dtype=torch.int64, device="cuda")
+        boff = ctx.eakv_hash_blocks_batched(dev.data_ptr(), offsets, par, out.data_ptr())
+        torch.cuda.synchronize()
+        res = out.cpu().numpy()
+        assert res[total] == -1
+        assert boff.tolist() == np.concatenate([[0], np.cumsum([x // b for x in lens])]).tolist()
+        for i, n in enumerate(lens):
+            p = oh.HASH_SEED if par is None else par[i]
+            expect = oh.hash_blocks(toks[offsets[i]:offsets[i + 1]].tolist(), b, p)
+            got = [int(x) for x in res[boff[i]:boff[i + 1]].view(np.uint64)]
+            assert got == expect, (b, i, n)
+    ctx.close()
+
+
+def test_batched_many_prompts_back_to_back():
+    # ticket counters must return to zero after every launch
+    b = 16
+    ctx = hash_ctx(b)
+    rng = np.random.default_rng(6)
+    lens = rng.integers(0, 3000, size=200)
+    offsets = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    toks = rng.integers(0, 151936, size=int(offsets[-1]), dtype=np.int32)
+    dev = torch.from_numpy(toks).cuda()
+    total = int(sum(x // b for x in lens))
+    expect = []
+    for i in range(len(lens)):
+        expect += oh.hash_blocks(toks[offsets[i]:offsets[i + 1]].tolist(), b)
+    for _ in range(3):
+        out = torch.zeros(total, dtype=torch.int64, device="cuda")
+        ctx.eakv_hash_blocks_batched(dev.data_ptr(), offsets, None, out.data_ptr())
+        torch.cuda.synchronize()
+        assert [int(x) for x in out.cpu().numpy().view(np.uint64)] == expect
+    ctx.close()
+
+
+def test_custom_base_and_seed():
+    ctx = hash_ctx(16, hash_base=1234567891011, hash_seed=42)
+    assert ctx.eakv_hash_base() == 1234567891011 and ctx.eakv_hash_seed() == 42
+    toks = np.arange(100, dtype=np.int32)
+    assert gpu_keys(ctx, toks) == oh.hash_blocks(toks.tolist(), 16, 42, 1234567891011)
+    ctx.close()

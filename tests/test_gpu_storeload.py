@@ -1,0 +1,208 @@
+"""GPU parity: eakv_store / eakv_load against oracle.storeload, byte for byte, for both
+host-link strategies, both tier locations and both device copy paths."""
+import itertools
+
+import numpy as np
+import pytest
+
+from eakv_workloads import KVShape, SHAPES, counter_words_numpy, counter_words_torch
+from oracle import storeload as osl
+
+from gpu_util import make_ctx, require_gpu, torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _gpu():
+    require_gpu()
+
+
+def eakv():
+    from paper_2609_33762_b200 import eakv as m
+    return m
+
+
+def variants():
+    e = eakv()
+    out = []
+    for link, loc, path in itertools.product((e.LINK_ZERO_COPY, e.LINK_STAGED),
+                                             (e.TIER_PINNED_HOST, e.TIER_DEVICE),
+                                             (e.COPY_VECTOR, e.COPY_BULK)):
+        if path == e.COPY_BULK and loc == e.TIER_PINNED_HOST and link == e.LINK_ZERO_COPY:
+            continue      # bulk copies are only used on device-resident buffers
+        out.append(dict(link_strategy=link, tier_location=loc, copy_path=path))
+    return out
+
+
+def random_pool(rng, shape, nb):
+    return [rng.integers(0, 256, size=(nb, shape.piece_bytes), dtype=np.uint8)
+            for _ in range(shape.pieces_per_block)]
+
+
+def to_device(pool_np):
+    return [torch.from_numpy(a.view(np.int16).copy()).cuda() for a in pool_np]
+
+
+def pool_to_numpy(pool_dev):
+    return [t.cpu().numpy().view(np.uint8) for t in pool_dev]
+
+
+class Rig:
+    """Device pool + context + oracle mirror, with a tier both sides initialise equally."""
+
+    def __init__(self, shape, nb, kh, seed, **kw):
+        e = eakv()
+        self.shape, self.nb, self.kh = shape, nb, kh
+        rng = np.random.default_rng(seed)
+        self.rng = rng
+        self.pool_np = random_pool(rng, shape, nb)
+        self.pool_dev = to_device(self.pool_np)
+        self.tier_np = rng.integers(0, 256, size=(kh, shape.pieces_per_block, shape.piece_bytes),
+                                    dtype=np.uint8)
+        self.loc = kw.get("tier_location", e.TIER_PINNED_HOST)
+        if self.loc == e.TIER_DEVICE:
+            self.tier_dev = torch.from_numpy(self.tier_np.copy()).cuda()
+            kw["tier_memory"] = self.tier_dev.data_ptr()
+        else:
+            self.tier_host = torch.from_numpy(self.tier_np.copy()).pin_memory()
+            kw["tier_memory"] = self.tier_host.data_ptr()
+        self.ctx = make_ctx(shape, nb, kh, self.pool_dev, **kw)
+
+    def tier_bytes(self):
+        self.ctx.eakv_sync()
+        if self.loc == eakv().TIER_DEVICE:
+            return self.tier_dev.cpu().numpy()
+        return self.tier_host.numpy()
+
+    def check(self):
+        got_tier = self.tier_bytes()
+        assert np.array_equal(got_tier, self.tier_np)
+        for a, b in zip(pool_to_numpy(self.pool_dev), self.pool_np):
+            assert np.array_equal(a, b)
+
+    def store(self, table, admit, slots):
+        self.ctx.eakv_store(table, admit, slots)
+        osl.store(self.pool_np, self.tier_np, table, [1] * len(table) if admit is None else admit, slots)
+
+    def load(self, slots, table):
+        self.ctx.eakv_load(slots, table)
+        osl.load(self.pool_np, self.tier_np, slots, table)
+
+    def close(self):
+        self.ctx.close()
+
+
+SHAPE_CASES = {
+    "tiny": SHAPES["tiny"],                       # piece 4 KiB (one partial 16-KiB item)
+    "qwen": SHAPES["qwen3_30b_a3b"],              # piece 16 KiB
+    "llama": SHAPES["llama3_8b"],                 # piece 64 KiB (4 items per piece)
+    "ragged": KVShape(3, 5, 128, 16),             # piece 20 KiB (16 KiB + 4 KiB tail)
+    "small": KVShape(2, 3, 40, 2),                # piece 480 B
+}
+
+
+@pytest.mark.parametrize("kw", variants(), ids=lambda k: "-".join(f"{v}" for v in k.values()))
+@pytest.mark.parametrize("name", ["tiny", "qwen", "ragged", "small"])
+def test_store_load_parity(name, kw):
+    shape = SHAPE_CASES[name]
+    nb, kh = (96, 80) if shape.block_bytes <= (1 << 21) else (24, 20)
+    # small staging buffers so the staged strategy cycles through several chunks
+    rig = Rig(shape, nb, kh, seed=11, staging_bytes=5 * shape.block_bytes, **kw)
+    rng = rig.rng
+    # 1. masked store, unsorted ids and slots
+    m = min(nb, kh) - 3
+    table = rng.permutation(nb)[:m].astype(np.int32)
+    slots = rng.permutation(kh)[:m].astype(np.int32)
+    admit = (rng.random(m) < 0.5).astype(np.uint8)
+    rig.store(table, admit, slots)
+    rig.check()
+    # 2. full store, contiguous ids and slots (long copy-engine runs), reversed table
+    rig.store(np.arange(m, dtype=np.int32)[::-1].copy(), None, np.arange(m, dtype=np.int32))
+    rig.check()
+    # 3. load into shuffled fresh blocks
+    k = m // 2
+    src = rng.permutation(kh)[:k].astype(np.int32)
+    dst = rng.permutation(nb)[:k].astype(np.int32)
+    rig.load(src, dst)
+    rig.check()
+    # 4. round trip: load(store(x)) == x into other blocks
+    blocks = np.arange(0, 8, dtype=np.int32)
+    rig.store(blocks, None, np.arange(8, dtype=np.int32))
+    rig.load(np.arange(8, dtype=np.int32), np.arange(8, 16, dtype=np.int32))
+    rig.check()
+    for q in range(shape.pieces_per_block):
+        assert np.array_equal(rig.pool_np[q][0:8], rig.pool_np[q][8:16])
+    # 5. degenerate calls: empty, all-zero mask, single block
+    rig.store(np.zeros(0, np.int32), None, np.zeros(0, np.int32))
+    rig.load(np.zeros(0, np.int32), np.zeros(0, np.int32))
+    rig.store(table, np.zeros(m, np.uint8), slots)
+    rig.store(np.array([nb - 1], np.int32), None, np.array([kh - 1], np.int32))
+    rig.load(np.array([0], np.int32), np.array([nb - 2], np.int32))
+    rig.check()
+    rig.close()
+
+
+def test_llama_shape_multi_item_pieces():
+    e = eakv()
+    for kw in (dict(copy_path=e.COPY_VECTOR), dict(copy_path=e.COPY_BULK, tier_location=e.TIER_DEVICE),
+               dict(link_strategy=e.LINK_STAGED)):
+        rig = Rig(SHAPE_CASES["llama"], 12, 10, seed=12, **kw)
+        rig.store(np.array([3, 11, 0, 7], np.int32), np.array([1, 1, 0, 1], np.uint8),
+                  np.array([9, 0, 5, 4], np.int32))
+        rig.load(np.array([9, 4], np.int32), np.array([1, 2], np.int32))
+        rig.check()
+        rig.close()
+
+
+def test_nan_payloads_and_negative_zero_survive():
+    shape = SHAPES["tiny"]
+    rig = Rig(shape, 4, 4, seed=13)
+    words = np.array([0x7FC1, 0xFFFF, 0x8000, 0x7F80, 0xFF80, 0x0001] * (shape.piece_bytes // 12),
+                     dtype=np.uint16)
+    for q in range(shape.pieces_per_block):
+        rig.pool_np[q][0, :len(words) * 2] = words.view(np.uint8)
+        rig.pool_dev[q][0, :len(words)] = torch.from_numpy(words.view(np.int16)).cuda()
+    rig.store(np.array([0], np.int32), None, np.array([2], np.int32))
+    rig.load(np.array([2], np.int32), np.array([3], np.int32))
+    rig.check()
+    assert np.array_equal(rig.pool_np[0][3, :len(words) * 2].view(np.uint16), words)
+    rig.close()
+
+
+def test_validation_errors_change_nothing():
+    e = eakv()
+    shape = SHAPES["tiny"]
+    rig = Rig(shape, 8, 6, seed=14)
+    i32 = lambda *a: np.array(a, np.int32)
+    cases = [
+        (lambda: rig.ctx.eakv_store(i32(0, 8), None, i32(0, 1)), e.E_RANGE),     # block id == NB
+        (lambda: rig.ctx.eakv_store(i32(0, -1), None, i32(0, 1)), e.E_RANGE),
+        (lambda: rig.ctx.eakv_store(i32(0, 1), None, i32(0, 6)), e.E_RANGE),     # slot == K_H
+        (lambda: rig.ctx.eakv_store(i32(0, 1), None, i32(3, 3)), e.E_INVAL),     # duplicate slot
+        (lambda: rig.ctx.eakv_load(i32(0, 1), i32(5, 5)), e.E_INVAL),            # duplicate block
+        (lambda: rig.ctx.eakv_load(i32(0, 7), i32(1, 2)), e.E_RANGE),
+        (lambda: rig.ctx.eakv_load(i32(0, 1), i32(1, 9)), e.E_RANGE),
+    ]
+    for fn, code in cases:
+        with pytest.raises(e.EakvError) as ei:
+            fn()
+        assert ei.value.code == code
+    # masked-out entries are not validated, duplicates among them are fine
+    rig.store(i32(0, 99, 99), np.array([1, 0, 0], np.uint8), i32(2, 2, 2))
+    rig.check()
+    assert rig.ctx.eakv_get_stats()["blocks_stored"] == 1
+    rig.close()
+
+
+def test_bad_shapes_rejected_at_create():
+    e = eakv()
+    t = torch.zeros(64, dtype=torch.int16, device="cuda")
+    base = dict(num_layers=1, kv_heads=1, head_dim=8, block_size=16, gpu_blocks=1, host_blocks=1,
+                kv_base=[t.data_ptr(), t.data_ptr()])
+    for patch in (dict(head_dim=3, block_size=1),              # piece bytes not a multiple of 16
+                  dict(kv_base=[t.data_ptr() + 2, t.data_ptr()]),   # misaligned base
+                  dict(block_size=8192), dict(host_blocks=0), dict(policy=7)):
+        with pytest.raises(e.EakvError) as ei:
+            e.Context(**{**base, **patch})
+        assert ei.value.code == e.E_INVAL

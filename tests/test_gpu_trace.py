@@ -1,0 +1,148 @@
+"""GPU parity on whole agent traces: every per-request output (keys, G, H, hit/admit/slot
+sequences, evictions, GPU block assignment) and every byte of KV in both tiers must equal
+the oracle's, for config 0, its large-tier sibling, and both admission policies."""
+import numpy as np
+import pytest
+
+from eakv_workloads import CONFIGS, SHAPES, key_words_numpy, key_words_torch, make_trace, normal_bf16_words
+from oracle.trace import TraceOracle
+
+from gpu_util import require_gpu, torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _gpu():
+    require_gpu()
+
+
+def normal_payload(keys, q, n_words):
+    """Config 0's payload: bf16(N(0,1)) drawn per (block key, piece)."""
+    return np.stack([normal_bf16_words((0, int(k), q), n_words) for k in keys])
+
+
+def compare_records(got, want):
+    assert len(got) == len(want)
+    for g, w in zip(got, want):
+        assert [int(x) for x in g["keys"]] == w["keys"]
+        for f in ("n_tokens", "G", "H", "new_chunks", "pressure", "save", "loaded", "stored",
+                  "fresh_tokens", "filled"):
+            assert g[f] == w[f], f
+        for f in ("hit", "admit", "slot", "gpu_resident", "gpu_block"):
+            assert [int(x) for x in g[f]] == [int(x) for x in w[f]], f
+        assert [(int(k), int(s)) for k, s in g["evicted"]] == w["evicted"]
+
+
+def compare_bytes(server, oracle):
+    server.ctx.eakv_sync()
+    for q, t in enumerate(server.pool.pieces):
+        got = t.cpu().numpy().view(np.uint8)
+        # only key-indexed GPU blocks have defined content
+        for key, blk in oracle.gpu.order.items():
+            assert np.array_equal(got[blk], oracle.pool[q][blk]), (q, blk)
+    tier = server.ctx.tier_host_view()
+    for key, slot in oracle.host.order.items():
+        assert np.array_equal(tier[slot], oracle.tier[slot]), slot
+
+
+@pytest.mark.parametrize("cfg_name", ["c0", "c0_big_tier"])
+@pytest.mark.parametrize("link", [0, 1])
+def test_config0_bit_exact(cfg_name, link):
+    from paper_2609_33762_b200.harness import AgentServer
+    cfg = CONFIGS[cfg_name]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg)
+    payload = normal_payload if cfg_name == "c0" and link == 0 else key_words_numpy
+    oracle = TraceOracle(shape, cfg.gpu_blocks, cfg.host_blocks, payload=payload)
+    oracle.run(trace)
+    server = AgentServer(shape, cfg.gpu_blocks, cfg.host_blocks, payload, link_strategy=link,
+                         staging_bytes=7 * shape.block_bytes, incremental_hash=(link == 1))
+    server.run(trace)
+    compare_records(server.records, oracle.records)
+    assert server.totals == oracle.totals
+    compare_bytes(server, oracle)
+    st = server.ctx.eakv_get_stats()
+    for f in ("requests", "references", "hits", "admitted", "declined", "evicted",
+              "declined_requests", "pressure_requests"):
+        assert st[f] == oracle.host.stats[f], f
+    assert st["blocks_stored"] == oracle.totals["stored_blocks"]
+    assert st["blocks_loaded"] == oracle.totals["loaded_blocks"]
+    server.close()
+
+
+@pytest.mark.parametrize("policy,kappa", [(1, 8), (2, 8), (2, 2), (1, 40)])
+def test_admission_policies_bit_exact(policy, kappa):
+    """Tool-gap interleave (config 2's recipe) on the tiny KV shape with a tier far below
+    the working set, so the pressure signal engages; device payload generator."""
+    from dataclasses import replace
+    from paper_2609_33762_b200.harness import AgentServer
+    cfg = replace(CONFIGS["c2"], shape="tiny", agents=6, turns=14, first_prompt=300,
+                  append_median=120.0, context_cap=1800, tool_gap_mean_ms=20_000.0)
+    shape = SHAPES["tiny"]
+    trace = make_trace(cfg, seed=21)
+    kw = dict(policy=policy, kappa_blocks=kappa, window_ms=60_000, len_window=16)
+    oracle = TraceOracle(shape, 128, 160, payload=key_words_numpy, **kw)
+    oracle.run(trace)
+    dev_payload = lambda keys, q, n: key_words_torch(keys.astype(np.int64), q, n, "cuda")
+    server = AgentServer(shape, 128, 160, dev_payload, **kw)
+    server.run(trace)
+    compare_records(server.records, oracle.records)
+    compare_bytes(server, oracle)
+    assert oracle.host.stats["declined_requests"] > 0          # the filter did engage
+    if policy == 2:
+        assert 0 < oracle.host.stats["pressure_requests"] < len(trace.requests)
+    server.close()
+
+
+def test_telemetry_off_uses_estimate_alone():
+    from dataclasses import replace
+    from paper_2609_33762_b200.harness import AgentServer
+    cfg = replace(CONFIGS["c2"], shape="tiny", agents=5, turns=8, first_prompt=300,
+                  append_median=100.0, context_cap=1500)
+    shape = SHAPES["tiny"]
+    trace = make_trace(cfg, seed=22)
+    kw = dict(policy=2, kappa_blocks=4, telemetry=0)
+    oracle = TraceOracle(shape, 128, 100, **{**kw, "telemetry": False})
+    oracle.run(trace)
+    server = AgentServer(shape, 128, 100, None, data_plane=False, **kw)
+    server.run(trace)
+    compare_records(server.records, oracle.records)
+    server.close()
+
+
+def test_tier_step_capacity_error_changes_nothing():
+    from paper_2609_33762_b200 import eakv
+    from paper_2609_33762_b200.harness import AgentServer
+    shape = SHAPES["tiny"]
+    server = AgentServer(shape, 16, 4, None, data_plane=False)
+    keys = np.arange(1, 6, dtype=np.uint64)
+    server.ctx.eakv_tier_step(keys[:2], 0, 32, 0)
+    before = server.ctx.eakv_get_stats()
+    with pytest.raises(eakv.EakvError) as ei:
+        server.ctx.eakv_tier_step(keys, 0, 80, 1)
+    assert ei.value.code == eakv.E_CAPACITY
+    assert server.ctx.eakv_get_stats() == before
+    with pytest.raises(eakv.EakvError) as ei:
+        server.ctx.eakv_gpu_tier_step(np.arange(1, 18, dtype=np.uint64), False)
+    assert ei.value.code == eakv.E_CAPACITY
+    G, H, gids, slots = server.ctx.eakv_match(keys)
+    assert (G, H) == (0, 2) and slots.tolist() == [0, 1]
+    server.close()
+
+
+def test_config2_control_plane_prefix():
+    """Config 2's own trace and KV shape, bookkeeping only (keys, match, both tiers), on
+    the first 400 requests with the 32 GiB tier of config 3 under conditioned admission."""
+    from paper_2609_33762_b200.harness import AgentServer
+    cfg = CONFIGS["c3"]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg)
+    kw = dict(policy=2, kappa_blocks=cfg.kappa_blocks)
+    oracle = TraceOracle(shape, cfg.gpu_blocks, cfg.host_blocks, **kw)
+    oracle.run(trace, limit=400)
+    server = AgentServer(shape, cfg.gpu_blocks, cfg.host_blocks, None, data_plane=False,
+                         incremental_hash=True, **kw)
+    server.run(trace, limit=400)
+    compare_records(server.records, oracle.records)
+    server.close()
