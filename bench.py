@@ -39,7 +39,7 @@ WORKLOAD = "c1_store_load_microbench_qwen3_30b_a3b"
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="eakv", choices=["eakv", "reference"])
     ap.add_argument("--blocks", type=int, default=4096, help="blocks per request")
@@ -50,6 +50,8 @@ def parse_args():
     ap.add_argument("--copy-ctas", type=int, default=0)
     ap.add_argument("--host-ctas", type=int, default=0)
     ap.add_argument("--staging-mib", type=int, default=64)
+    ap.add_argument("--no-overlap", dest="overlap", action="store_false",
+                    help="e2e arm: restores and host writes on one stream instead of two")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
@@ -62,54 +64,70 @@ def parse_args():
 # clocks
 # ------------------------------------------------------------------------------------------
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Polls SM clock and throttle reasons through NVML (read-only) every few milliseconds
+    on a thread, so that even a short timed region gets samples under load."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap"}
 
     def __init__(self, index):
         self.index = index
-        self.proc = None
-        self.lines = []
+        self.samples = []          # (perf_counter, sm_mhz, reasons bitmask)
+        self.thread = None
+        self.stop_flag = False
+        self.max_mhz = None
+        self.err = None
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
-                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
-            self.thread.start()
-        except OSError:
-            self.proc = None
+            import pynvml
+            pynvml.nvmlInit()
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            idx = self.index
+            if vis:
+                ids = [v for v in vis.split(",") if v.strip()]
+                if idx < len(ids) and ids[idx].strip().isdigit():
+                    idx = int(ids[idx])
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+            self.nv = pynvml
+        except Exception as e:  # noqa: BLE001
+            self.err = repr(e)
+            return
+        self.thread = threading.Thread(target=self._poll, daemon=True)
+        self.thread.start()
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
-
-    def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
-            parts = [p.strip() for p in ln.split(",")]
-            if len(parts) < 8:
-                continue
+    def _poll(self):
+        nv = self.nv
+        while not self.stop_flag:
             try:
-                sm.append(float(parts[0])); mx.append(float(parts[1]))
-            except ValueError:
-                continue
-            for name, val in zip(names, parts[4:8]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": float(np.median(sm)) if sm else None,
-                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm),
-                "reasons": sorted(reasons)}
+                mhz = nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM)
+                rs = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle)
+                self.samples.append((time.perf_counter(), float(mhz), int(rs)))
+            except Exception as e:  # noqa: BLE001
+                self.err = repr(e)
+                return
+            time.sleep(0.002)
+
+    def mark(self):
+        return time.perf_counter()
+
+    def stop(self, t0=None, t1=None):
+        self.stop_flag = True
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "samples": 0,
+                    "reasons": ["no samples: " + str(self.err)]}
+        sel = [x for x in self.samples if (t0 is None or x[0] >= t0) and (t1 is None or x[0] <= t1)]
+        scope = "timed region"
+        if len(sel) < 3:                      # region shorter than the polling period
+            sel, scope = self.samples, "warm-up + timed region"
+        mask = 0
+        for _, _, r in sel:
+            mask |= r
+        return {"sm_mhz": float(np.median([x[1] for x in sel])), "sm_max_mhz": self.max_mhz,
+                "samples": len(sel), "scope": scope,
+                "reasons": sorted(n for bit, n in self.REASONS.items() if mask & bit)}
 
 
 # ------------------------------------------------------------------------------------------
@@ -144,64 +162,95 @@ class Arm:
                                 gpu_blocks=pool.gpu_blocks, host_blocks=2 * self.m,
                                 kv_base=pool.kv_base, **kw)
         self.block_bytes = self.ctx.block_bytes
-        self.stream = torch.cuda.current_stream(device)
+        # lookups (hash, key read-back) run on their own stream so the host control plane of
+        # the next request overlaps the transfers of the previous one; the e2e arm also gives
+        # restores and host writes a stream each (full-duplex link), ordered by events
+        self.hash_stream = torch.cuda.Stream(device)
+        self.load_stream = torch.cuda.Stream(device)
+        self.store_stream = torch.cuda.Stream(device) if (host_tier and args.overlap) else self.load_stream
+        self.load_done = [torch.cuda.Event(), torch.cuda.Event()]    # by step parity
+        self.store_done = torch.cuda.Event()
         self.seed = self.ctx.eakv_hash_seed()
         self.keys_dev = torch.empty(self.m, dtype=torch.int64, device=device)
         self.keys_host = torch.empty(self.m, dtype=torch.int64).pin_memory()
         self.tok_dev = torch.empty(self.n_tokens, dtype=torch.int32, device=device)
-        self.kernel_ms = []          # (bytes, ms) per timed store/load launch
         self.h2d = self.d2h = 0
 
-    def request(self, tokens, table, agent, now, timed_events=None):
+    def streams(self):
+        return {self.hash_stream, self.load_stream, self.store_stream}
+
+    def request(self, tokens, table, agent, now, timed_events=None, step=0):
         """tokens: device int32 tensor (device arm) or pinned host tensor (e2e arm)."""
         torch = self.torch
-        if tokens.device.type == "cpu":
-            self.tok_dev.copy_(tokens, non_blocking=True)
-            self.h2d += tokens.numel() * 4
-            tok = self.tok_dev
-        else:
-            tok = tokens
-        nblk = self.ctx.eakv_hash_blocks(tok.data_ptr(), self.n_tokens, self.seed,
-                                         self.keys_dev.data_ptr(), self.stream)
-        self.keys_host.copy_(self.keys_dev, non_blocking=True)
-        self.stream.synchronize()
+        hs = self.hash_stream
+        with torch.cuda.stream(hs):
+            if tokens.device.type == "cpu":
+                self.tok_dev.copy_(tokens, non_blocking=True)
+                self.h2d += tokens.numel() * 4
+                tok = self.tok_dev
+            else:
+                tok = tokens
+            nblk = self.ctx.eakv_hash_blocks(tok.data_ptr(), self.n_tokens, self.seed,
+                                             self.keys_dev.data_ptr(), hs)
+            self.keys_host.copy_(self.keys_dev, non_blocking=True)
+        hs.synchronize()
         self.d2h += nblk * 8
         keys = self.keys_host.numpy().view(np.uint64)
         G, H, _, slots = self.ctx.eakv_match(keys)
         step = self.ctx.eakv_tier_step(keys, agent, self.n_tokens, now)
-        ev = None
-        if timed_events is not None:
-            ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-            ev[0].record(self.stream)
         moved = 0
         if H > 0:
-            self.ctx.eakv_load(slots[:H], table[:H], self.stream)
+            ls = self.load_stream
+            ls.wait_event(self.store_done)      # the slots being read were written by a store
+            ev = self._timer(ls, timed_events)
+            self.ctx.eakv_load(slots[:H], table[:H], ls)
+            self._timer_end(ls, ev, H * self.block_bytes, timed_events)
+            self.load_done[step % 2].record(ls)
             moved += H * self.block_bytes
             self.h2d += H * self.block_bytes if self.host_tier else 0
         n_admit = int(step["admit"].sum())
         if n_admit:
-            self.ctx.eakv_store(table, step["admit"], step["slot"], self.stream)
+            ss = self.store_stream
+            # the slots this store overwrites held the prompt the previous step restored
+            ss.wait_event(self.load_done[(step - 1) % 2])
+            ev = self._timer(ss, timed_events)
+            self.ctx.eakv_store(table, step["admit"], step["slot"], ss)
+            self._timer_end(ss, ev, n_admit * self.block_bytes, timed_events)
+            self.store_done.record(ss)
             moved += n_admit * self.block_bytes
             self.d2h += n_admit * self.block_bytes if self.host_tier else 0
-        if ev is not None:
-            ev[1].record(self.stream)
-            timed_events.append((moved, ev))
         return moved, H, n_admit
 
+    def _timer(self, stream, timed_events):
+        if timed_events is None:
+            return None
+        ev = (self.torch.cuda.Event(enable_timing=True), self.torch.cuda.Event(enable_timing=True))
+        ev[0].record(stream)
+        return ev
+
+    def _timer_end(self, stream, ev, nbytes, timed_events):
+        if ev is not None:
+            ev[1].record(stream)
+            timed_events.append((nbytes, ev))
+
     def step(self, s, prompts, tables, timed_events=None):
-        """prompts[s-1] was stored by the previous step; prompts[s] is new."""
-        moved = 0
-        a, _, _ = self.request(prompts[s - 1], tables[2 * s], agent=(s - 1) % 2, now=s * 1000,
-                               timed_events=timed_events)
-        b, _, _ = self.request(prompts[s], tables[2 * s + 1], agent=s % 2, now=s * 1000 + 500,
-                               timed_events=timed_events)
+        """prompts[s-1] was stored by the previous step; prompts[s] is new.  The two requests
+        use disjoint, freshly drawn pool blocks."""
+        m = self.m
+        a, _, _ = self.request(prompts[s - 1], tables[s][:m], agent=(s - 1) % 2, now=s * 1000,
+                               timed_events=timed_events, step=s)
+        b, _, _ = self.request(prompts[s], tables[s][m:], agent=s % 2, now=s * 1000 + 500,
+                               timed_events=timed_events, step=s)
         return a + b
 
 
-def run_arm(arm, prompts, tables, steps, warmup, dist, clocks=None):
+def run_arm(arm, prompts, tables, steps, warmup, dist, clocks=None, time_kernels=True):
     torch = arm.torch
+    main = torch.cuda.current_stream(arm.device)
+    if clocks:
+        clocks.start()
     # prime: store prompt 0 so that step 1 has something to restore
-    arm.request(prompts[0], tables[0], agent=0, now=0)
+    arm.request(prompts[0], tables[0][arm.m:], agent=0, now=0)
     for s in range(1, warmup + 1):
         arm.step(s, prompts, tables)
     torch.cuda.synchronize()
@@ -209,22 +258,25 @@ def run_arm(arm, prompts, tables, steps, warmup, dist, clocks=None):
         dist.barrier()
     arm.h2d = arm.d2h = 0
     launches0 = arm.ctx.eakv_get_stats()["kernel_launches"]
-    timed = []
-    if clocks:
-        clocks.start()
+    timed = [] if time_kernels else None
+    t0 = time.perf_counter()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(arm.stream)
+    e0.record(main)                      # the device is idle: this is the start of the region
+    for st in arm.streams():
+        st.wait_stream(main)
     moved = 0
     for s in range(warmup + 1, warmup + 1 + steps):
         moved += arm.step(s, prompts, tables, timed_events=timed)
-    e1.record(arm.stream)
+    for st in arm.streams():
+        main.wait_stream(st)
+    e1.record(main)
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
-    clk = clocks.stop() if clocks else None
+    clk = clocks.stop(t0, time.perf_counter()) if clocks else None
     if dist is not None:
         dist.barrier()
     launches = arm.ctx.eakv_get_stats()["kernel_launches"] - launches0
-    kernel = [(b, ev[0].elapsed_time(ev[1])) for b, ev in timed if b > 0]
+    kernel = [(b, ev[0].elapsed_time(ev[1])) for b, ev in (timed or []) if b > 0]
     return dict(ms=ms, moved=moved, launches=launches, kernel=kernel, clocks=clk,
                 h2d=arm.h2d / steps, d2h=arm.d2h / steps)
 
@@ -371,7 +423,7 @@ def main():
     prompts_dev = [torch.from_numpy(tok_np[i]).to(device) for i in range(total_steps + 1)]
     prompts_host = [torch.from_numpy(tok_np[i]).pin_memory() for i in range(total_steps + 1)]
     # fresh uniform-random block ids per request, without replacement
-    tables = [rng.permutation(nb)[:m].astype(np.int32) for _ in range(2 * total_steps + 2)]
+    tables = [rng.permutation(nb)[:2 * m].astype(np.int32) for _ in range(total_steps + 1)]
 
     clocks = ClockSampler(local_rank) if rank == 0 else None
 
@@ -401,7 +453,8 @@ def main():
         link = pinned_link_peak(torch, device) if rank == 0 else None
         arm = Arm(args, pool, shape, torch, eakv, host_tier=True, device=device)
         e_steps = max(2, min(args.steps, 5))
-        re_ = run_arm(arm, prompts_host, tables, e_steps, min(args.warmup, 3), dist, None)
+        re_ = run_arm(arm, prompts_host, tables, e_steps, min(args.warmup, 3), dist, None,
+                      time_kernels=False)
         arm.ctx.close()
         del arm
         e_ms, e_moved = aggregate_over_ranks(dist, re_["ms"], re_["moved"], device)
@@ -410,9 +463,13 @@ def main():
                "d2h_bytes_per_step": int(re_["d2h"]), "steps": e_steps,
                "ms_per_step": e_ms / e_steps, "link_strategy": args.link}
         if link:
-            # load and store alternate, so the bound is the harmonic mean of the two directions
-            bound = 2.0 / (1.0 / link["h2d"] + 1.0 / link["d2h"])
-            e2e.update(host_link_peak_gbps=link, frac_of_link=e_val / bound / max(world, 1))
+            # one direction at a time: harmonic mean of the two; both at once: the measured
+            # bidirectional pinned-memcpy rate
+            serial = 2.0 / (1.0 / link["h2d"] + 1.0 / link["d2h"])
+            bound = link["bidir"] if args.overlap else serial
+            e2e.update(host_link_peak_gbps=link, overlap=bool(args.overlap),
+                       frac_of_link=e_val / bound / max(world, 1),
+                       frac_of_one_direction=e_val / serial / max(world, 1))
 
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:
@@ -451,7 +508,7 @@ def main():
 def self_check(torch, arm, pool, tables, args, shape):
     """After the timed region: the last stored prompt's slots must equal its pool blocks."""
     s = args.warmup + args.steps
-    table = tables[2 * s + 1]
+    table = tables[s][args.blocks:]
     keys = arm.keys_host.numpy().view(np.uint64)         # keys of the last request
     _, H, _, slots = arm.ctx.eakv_match(keys)
     if H != len(keys):

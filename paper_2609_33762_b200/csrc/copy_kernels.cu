@@ -27,7 +27,8 @@ copy_blocks_vector_kernel(CopyLaunch L) {
         const int sub = r - q * L.subs_per_piece;
         const int2 e = __ldg(L.entries + j);
         char* pool = reinterpret_cast<char*>(__ldg(reinterpret_cast<const unsigned long long*>(L.kv_base) + q)) + (int64_t)e.x * L.piece_bytes;
-        char* tier = L.tier_base + ((int64_t)e.y * L.pieces + q) * L.piece_bytes;
+        const int64_t slot = L.slot_from_index ? j : (int64_t)e.y;
+        char* tier = L.tier_base + (slot * L.pieces + q) * L.piece_bytes;
         const int4* src = reinterpret_cast<const int4*>(TO_TIER ? pool : tier);
         int4* dst = reinterpret_cast<int4*>(TO_TIER ? tier : pool);
         const int unit0 = sub * (kCopyThreads * kCopyUnroll) + threadIdx.x;
@@ -118,7 +119,8 @@ __device__ __forceinline__ BulkItem bulk_decode(const CopyLaunch& L, int64_t it)
     const int64_t off = (int64_t)sub * kBulkStageBytes;
     char* pool = reinterpret_cast<char*>(__ldg(reinterpret_cast<const unsigned long long*>(L.kv_base) + q)) +
                  (int64_t)e.x * L.piece_bytes + off;
-    char* tier = L.tier_base + ((int64_t)e.y * L.pieces + q) * L.piece_bytes + off;
+    const int64_t slot = L.slot_from_index ? j : (int64_t)e.y;
+    char* tier = L.tier_base + (slot * L.pieces + q) * L.piece_bytes + off;
     BulkItem b;
     b.src = TO_TIER ? pool : tier;
     b.dst = TO_TIER ? tier : pool;

@@ -165,7 +165,7 @@ int copy_ctas(const eakv_ctx* ctx, bool touches_host) {
 }
 
 int launch_copy(eakv_ctx* ctx, const int2* d_entries, int64_t n, char* tier_base, bool to_tier,
-                bool touches_host, cudaStream_t stream) {
+                bool touches_host, bool packed, cudaStream_t stream) {
     CopyLaunch L;
     L.entries = d_entries;
     L.n_entries = n;
@@ -173,6 +173,7 @@ int launch_copy(eakv_ctx* ctx, const int2* d_entries, int64_t n, char* tier_base
     L.tier_base = tier_base;
     L.pieces = ctx->pieces;
     L.piece_bytes = ctx->piece_bytes;
+    L.slot_from_index = packed ? 1 : 0;
     L.subs_per_piece = (int32_t)((ctx->piece_bytes + kCopySubBytes - 1) / kCopySubBytes);
     cudaError_t e;
     if (ctx->cfg.copy_path == EAKV_COPY_BULK)
@@ -184,18 +185,24 @@ int launch_copy(eakv_ctx* ctx, const int2* d_entries, int64_t n, char* tier_base
     return EAKV_OK;
 }
 
-// upload n entries through a ring slot, then run `body(device entries)`; records the slot's event
-template <class F>
-int with_entries(eakv_ctx* ctx, const int2* entries, int64_t n, cudaStream_t stream, F body) {
+// Upload n entries through a ring slot.  *dev_out is valid for work enqueued on `stream`
+// (and on streams ordered after it) until ring_release records the slot's event.
+int ring_upload(eakv_ctx* ctx, const int2* entries, int64_t n, cudaStream_t stream,
+                RingSlot** slot_out, const int2** dev_out) {
     RingSlot* s = nullptr;
     int rc = ring_acquire(ctx, &s);
     if (rc != EAKV_OK) return rc;
     std::memcpy(s->host, entries, (size_t)n * sizeof(int2));
     CU(cudaMemcpyAsync(s->dev, s->host, (size_t)n * sizeof(int2), cudaMemcpyHostToDevice, stream));
     ctx->stats.memcpy_calls += 1;
-    rc = body(static_cast<const int2*>(s->dev));
+    *slot_out = s;
+    *dev_out = static_cast<const int2*>(s->dev);
+    return EAKV_OK;
+}
+
+int ring_release(eakv_ctx* ctx, RingSlot* s, cudaStream_t stream) {
     CU(cudaEventRecord(s->done, stream));
-    return rc;
+    return EAKV_OK;
 }
 
 int next_epoch(eakv_ctx* ctx) {
@@ -671,43 +678,45 @@ int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_m
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const bool host_tier = ctx->cfg.tier_location == EAKV_TIER_PINNED_HOST;
 
-    if (ctx->cfg.link_strategy == EAKV_LINK_ZERO_COPY) {
-        for (int64_t i = 0; i < m; i += ctx->max_call_blocks) {
-            const int64_t cur = std::min(ctx->max_call_blocks, m - i);
-            int rc = with_entries(ctx, ent.data() + i, cur, stream, [&](const int2* d) {
-                return launch_copy(ctx, d, cur, ctx->tier, true, host_tier, stream);
-            });
+    // one argument upload per max_call_blocks entries; the staged strategy walks each upload
+    // in staging-buffer-sized chunks
+    for (int64_t base = 0; base < m; base += ctx->max_call_blocks) {
+        const int64_t n = std::min(ctx->max_call_blocks, m - base);
+        RingSlot* rs = nullptr;
+        const int2* d = nullptr;
+        int rc = ring_upload(ctx, ent.data() + base, n, stream, &rs, &d);
+        if (rc != EAKV_OK) return rc;
+        if (ctx->cfg.link_strategy == EAKV_LINK_ZERO_COPY) {
+            rc = launch_copy(ctx, d, n, ctx->tier, true, host_tier, false, stream);
             if (rc != EAKV_OK) return rc;
+        } else {
+            Staging& S = ctx->st_store;
+            for (int64_t i = 0; i < n; i += ctx->staging_blocks) {
+                const int64_t cur = std::min(ctx->staging_blocks, n - i);
+                const int sb = S.next;
+                S.next ^= 1;
+                CU(cudaStreamWaitEvent(stream, S.freed[sb], 0));
+                rc = launch_copy(ctx, d + i, cur, S.buf[sb], true, false, true, stream);
+                if (rc != EAKV_OK) return rc;
+                CU(cudaEventRecord(S.ready[sb], stream));
+                CU(cudaStreamWaitEvent(S.side, S.ready[sb], 0));
+                const int2* e = ent.data() + base + i;
+                rc = for_slot_runs(e, cur, [&](int64_t a, int64_t z) {
+                    CU(cudaMemcpyAsync(ctx->tier + (int64_t)e[a].y * ctx->block_bytes,
+                                       S.buf[sb] + a * ctx->block_bytes,
+                                       (size_t)(z - a) * ctx->block_bytes, cudaMemcpyDefault, S.side));
+                    ctx->stats.memcpy_calls += 1;
+                    return EAKV_OK;
+                });
+                if (rc != EAKV_OK) return rc;
+                CU(cudaEventRecord(S.freed[sb], S.side));
+            }
+            // the call's work is complete, in stream order, once both buffers are drained
+            CU(cudaStreamWaitEvent(stream, S.freed[0], 0));
+            CU(cudaStreamWaitEvent(stream, S.freed[1], 0));
         }
-    } else {
-        Staging& S = ctx->st_store;
-        std::vector<int2> local;
-        for (int64_t i = 0; i < m; i += ctx->staging_blocks) {
-            const int64_t cur = std::min(ctx->staging_blocks, m - i);
-            const int sb = S.next;
-            S.next ^= 1;
-            local.resize((size_t)cur);
-            for (int64_t k = 0; k < cur; ++k) local[k] = make_int2(ent[i + k].x, (int)k);
-            CU(cudaStreamWaitEvent(stream, S.freed[sb], 0));
-            int rc = with_entries(ctx, local.data(), cur, stream, [&](const int2* d) {
-                return launch_copy(ctx, d, cur, S.buf[sb], true, false, stream);
-            });
-            if (rc != EAKV_OK) return rc;
-            CU(cudaEventRecord(S.ready[sb], stream));
-            CU(cudaStreamWaitEvent(S.side, S.ready[sb], 0));
-            rc = for_slot_runs(ent.data() + i, cur, [&](int64_t a, int64_t z) {
-                CU(cudaMemcpyAsync(ctx->tier + (int64_t)ent[i + a].y * ctx->block_bytes,
-                                   S.buf[sb] + a * ctx->block_bytes,
-                                   (size_t)(z - a) * ctx->block_bytes, cudaMemcpyDefault, S.side));
-                ctx->stats.memcpy_calls += 1;
-                return EAKV_OK;
-            });
-            if (rc != EAKV_OK) return rc;
-            CU(cudaEventRecord(S.freed[sb], S.side));
-        }
-        // the call's work is complete, in stream order, once both buffers are drained
-        CU(cudaStreamWaitEvent(stream, S.freed[0], 0));
-        CU(cudaStreamWaitEvent(stream, S.freed[1], 0));
+        rc = ring_release(ctx, rs, stream);
+        if (rc != EAKV_OK) return rc;
     }
     ctx->stats.blocks_stored += m;
     ctx->stats.bytes_stored += m * ctx->block_bytes;
@@ -735,43 +744,45 @@ int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_tab
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const bool host_tier = ctx->cfg.tier_location == EAKV_TIER_PINNED_HOST;
 
-    if (ctx->cfg.link_strategy == EAKV_LINK_ZERO_COPY) {
-        for (int64_t i = 0; i < m; i += ctx->max_call_blocks) {
-            const int64_t cur = std::min(ctx->max_call_blocks, m - i);
-            int rc = with_entries(ctx, ent.data() + i, cur, stream, [&](const int2* d) {
-                return launch_copy(ctx, d, cur, ctx->tier, false, host_tier, stream);
-            });
-            if (rc != EAKV_OK) return rc;
-        }
-    } else {
-        Staging& S = ctx->st_load;
-        std::vector<int2> local;
+    if (ctx->cfg.link_strategy == EAKV_LINK_STAGED) {
         // the side stream may read the tier only after what precedes this call on `stream`
-        CU(cudaEventRecord(S.start, stream));
-        CU(cudaStreamWaitEvent(S.side, S.start, 0));
-        for (int64_t i = 0; i < m; i += ctx->staging_blocks) {
-            const int64_t cur = std::min(ctx->staging_blocks, m - i);
-            const int sb = S.next;
-            S.next ^= 1;
-            CU(cudaStreamWaitEvent(S.side, S.freed[sb], 0));
-            int rc = for_slot_runs(ent.data() + i, cur, [&](int64_t a, int64_t z) {
-                CU(cudaMemcpyAsync(S.buf[sb] + a * ctx->block_bytes,
-                                   ctx->tier + (int64_t)ent[i + a].y * ctx->block_bytes,
-                                   (size_t)(z - a) * ctx->block_bytes, cudaMemcpyDefault, S.side));
-                ctx->stats.memcpy_calls += 1;
-                return EAKV_OK;
-            });
+        CU(cudaEventRecord(ctx->st_load.start, stream));
+        CU(cudaStreamWaitEvent(ctx->st_load.side, ctx->st_load.start, 0));
+    }
+    for (int64_t base = 0; base < m; base += ctx->max_call_blocks) {
+        const int64_t n = std::min(ctx->max_call_blocks, m - base);
+        RingSlot* rs = nullptr;
+        const int2* d = nullptr;
+        int rc = ring_upload(ctx, ent.data() + base, n, stream, &rs, &d);
+        if (rc != EAKV_OK) return rc;
+        if (ctx->cfg.link_strategy == EAKV_LINK_ZERO_COPY) {
+            rc = launch_copy(ctx, d, n, ctx->tier, false, host_tier, false, stream);
             if (rc != EAKV_OK) return rc;
-            CU(cudaEventRecord(S.ready[sb], S.side));
-            CU(cudaStreamWaitEvent(stream, S.ready[sb], 0));
-            local.resize((size_t)cur);
-            for (int64_t k = 0; k < cur; ++k) local[k] = make_int2(ent[i + k].x, (int)k);
-            rc = with_entries(ctx, local.data(), cur, stream, [&](const int2* d) {
-                return launch_copy(ctx, d, cur, S.buf[sb], false, false, stream);
-            });
-            if (rc != EAKV_OK) return rc;
-            CU(cudaEventRecord(S.freed[sb], stream));
+        } else {
+            Staging& S = ctx->st_load;
+            for (int64_t i = 0; i < n; i += ctx->staging_blocks) {
+                const int64_t cur = std::min(ctx->staging_blocks, n - i);
+                const int sb = S.next;
+                S.next ^= 1;
+                CU(cudaStreamWaitEvent(S.side, S.freed[sb], 0));
+                const int2* e = ent.data() + base + i;
+                rc = for_slot_runs(e, cur, [&](int64_t a, int64_t z) {
+                    CU(cudaMemcpyAsync(S.buf[sb] + a * ctx->block_bytes,
+                                       ctx->tier + (int64_t)e[a].y * ctx->block_bytes,
+                                       (size_t)(z - a) * ctx->block_bytes, cudaMemcpyDefault, S.side));
+                    ctx->stats.memcpy_calls += 1;
+                    return EAKV_OK;
+                });
+                if (rc != EAKV_OK) return rc;
+                CU(cudaEventRecord(S.ready[sb], S.side));
+                CU(cudaStreamWaitEvent(stream, S.ready[sb], 0));
+                rc = launch_copy(ctx, d + i, cur, S.buf[sb], false, false, true, stream);
+                if (rc != EAKV_OK) return rc;
+                CU(cudaEventRecord(S.freed[sb], stream));
+            }
         }
+        rc = ring_release(ctx, rs, stream);
+        if (rc != EAKV_OK) return rc;
     }
     ctx->stats.blocks_loaded += m;
     ctx->stats.bytes_loaded += m * ctx->block_bytes;

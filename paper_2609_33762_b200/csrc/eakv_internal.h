@@ -50,6 +50,7 @@ struct CopyLaunch {
     char* tier_base;            // slot-major destination/source
     int32_t pieces;             // 2L
     int32_t subs_per_piece;     // ceil(piece_bytes / kCopySubBytes)
+    int32_t slot_from_index;    // 1: entry j uses slot j (packed staging buffer) instead of entries[j].y
     int64_t piece_bytes;
 };
 // to_tier: pool -> tier (store/gather); else tier -> pool (load/scatter)
