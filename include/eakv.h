@@ -210,6 +210,27 @@ int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_m
 int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_table,
               int64_t n_blocks, void* cuda_stream);
 
+/* Block keys without a context and without any allocation.  (The paper has no counterpart;
+ * this exists for callers that cannot request device memory: code living inside a serving
+ * process whose engine has already claimed the GPU's memory, where an allocation may fail or
+ * stall the device, and latency-critical sections that cannot afford an allocation's implicit
+ * synchronisation.)  Same keys as eakv_hash_blocks for the same tokens, block_size, hash_base
+ * (0 = library default) and parent_hash (pass the seed for a fresh prompt).
+ *   tokens_dev device int32[n_tokens]; hashes_dev device uint64[n_tokens / block_size];
+ *   n_blocks_out host or NULL; cuda_stream as elsewhere.
+ * The scratch is a fixed array inside the library (about 545 KiB per GPU, resident until the
+ * process exits) sized for at most EAKV_STATIC_MAX_BLOCKS keys per call: a longer prompt gets
+ * EAKV_E_CAPACITY and nothing is launched; hash it in pieces, passing the last key of one piece
+ * as parent_hash of the next.  The first call on each device looks up the array's device
+ * address (with that device current); make that first call outside any stream capture.
+ * Every call on a device shares the array: calls whose GPU work can overlap race, so order
+ * them (one stream, or events).  Calls no cudaMalloc/cudaFree or other allocating routine.
+ * Errors: EAKV_E_INVAL (bad sizes/pointers, block_size > 4096), EAKV_E_CAPACITY, EAKV_E_CUDA. */
+#define EAKV_STATIC_MAX_BLOCKS 65536
+int eakv_hash_blocks_static(const int32_t* tokens_dev, int64_t n_tokens, int32_t block_size,
+                            uint64_t hash_base, uint64_t parent_hash, uint64_t* hashes_dev,
+                            int64_t* n_blocks_out, void* cuda_stream);
+
 /* Block the host until everything the context enqueued (side streams included) is done. */
 int eakv_sync(eakv_ctx* ctx);
 

@@ -275,3 +275,114 @@ cudaError_t hash_kernels_init() {
 }
 
 }  // namespace eakv
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free block keys.
+//
+// Some users of this library run where device memory cannot be requested: inside a serving
+// process whose engine has already claimed the GPU's memory for its KV pool (an allocation
+// there can fail outright, or stall the whole device while the driver makes room), or in a
+// latency-critical section that may not take the implicit synchronisation of an allocation.
+// eakv_hash_blocks_static computes the same keys as eakv_hash_blocks without a context and
+// without allocating anything: its scratch (block partials, the power table B^0..B^b and
+// the ticket counter) lives in the file-scope array below, which every GPU that loads the
+// library keeps resident until the process exits.
+//
+// The array is shared by every call on a device and keeps the previous call's contents:
+// each call rewrites the power table, overwrites the partials it uses and zeroes the ticket
+// counter before its kernel runs.  Two calls whose GPU work overlaps (different streams
+// without an ordering between them) race on it.
+// ---------------------------------------------------------------------------------------
+#include "../../include/eakv.h"
+
+namespace eakv {
+
+constexpr int64_t kStaticMaxBlocks = EAKV_STATIC_MAX_BLOCKS;                 // 65,536 keys per call
+constexpr size_t kStaticPartialBytes = (size_t)kStaticMaxBlocks * 8;          // 512 KiB
+constexpr size_t kStaticPowBytes = ((size_t)(kHashMaxBlockSize + 1) * 8 + 255) / 256 * 256;
+constexpr size_t kStaticCounterBytes = 256;
+constexpr size_t kStaticBytes = kStaticPartialBytes + kStaticPowBytes + kStaticCounterBytes;
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never an address.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+static unsigned char* g_static_ptr[kMaxDevices];   // device address per device, set once
+
+// thread e writes B^e mod p
+__global__ void fill_pow_table_kernel(uint64_t* pw, uint64_t base, int n_entries) {
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < n_entries; e += gridDim.x * blockDim.x) {
+        uint64_t r = 1, sq = base;
+        for (int bits = e; bits; bits >>= 1) {
+            if (bits & 1) r = mulmod61(r, sq);
+            sq = mulmod61(sq, sq);
+        }
+        pw[e] = r;
+    }
+}
+
+}  // namespace eakv
+
+extern "C" int eakv_hash_blocks_static(const int32_t* tokens_dev, int64_t n_tokens,
+                                       int32_t block_size, uint64_t hash_base,
+                                       uint64_t parent_hash, uint64_t* hashes_dev,
+                                       int64_t* n_blocks_out, void* cuda_stream) {
+    using namespace eakv;
+    if (n_tokens < 0 || block_size <= 0 || block_size > kHashMaxBlockSize) return EAKV_E_INVAL;
+    const int64_t nblk = n_tokens / block_size;
+    if (n_blocks_out) *n_blocks_out = nblk;
+    if (nblk > kStaticMaxBlocks) return EAKV_E_CAPACITY;   // more keys than the static scratch holds
+    if (nblk == 0) return EAKV_OK;
+    if (!tokens_dev || !hashes_dev) return EAKV_E_INVAL;
+    if (((uintptr_t)tokens_dev & 3) || ((uintptr_t)hashes_dev & 7)) return EAKV_E_INVAL;
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return EAKV_E_CUDA;
+    if (g_static_ptr[dev] == nullptr) {
+        // once per device, with that device current: resolve the array's device address
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return EAKV_E_CUDA;
+        }
+        if (hash_kernels_init() != cudaSuccess) {
+            cudaGetLastError();
+            return EAKV_E_CUDA;
+        }
+        g_static_ptr[dev] = static_cast<unsigned char*>(p);
+    }
+    unsigned char* scratch = g_static_ptr[dev];
+    uint64_t* partial = reinterpret_cast<uint64_t*>(scratch);
+    uint64_t* pw = reinterpret_cast<uint64_t*>(scratch + kStaticPartialBytes);
+    int* counter = reinterpret_cast<int*>(scratch + kStaticPartialBytes + kStaticPowBytes);
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    constexpr uint64_t P = (1ull << 61) - 1;
+    const uint64_t base = hash_base ? hash_base % P : 6364136223846793005ull % P;
+    if (cudaMemsetAsync(counter, 0, kStaticCounterBytes, stream) != cudaSuccess) {
+        cudaGetLastError();
+        return EAKV_E_CUDA;
+    }
+    const int n_pow = block_size + 1;
+    fill_pow_table_kernel<<<(n_pow + 255) / 256, 256, 0, stream>>>(pw, base, n_pow);
+    if (cudaGetLastError() != cudaSuccess) return EAKV_E_CUDA;
+
+    const bool generic = (block_size % 4) != 0;
+    const bool vec = !generic && (((uintptr_t)tokens_dev & 15) == 0);
+    HashLaunch L;
+    L.tokens = tokens_dev;
+    L.keys = hashes_dev;
+    L.partial = partial;
+    L.counters = counter;
+    L.pow_table = pw;
+    L.tiles = nullptr;
+    L.prompts = nullptr;
+    L.single_nblk = nblk;
+    L.single_parent = parent_hash % P;
+    L.single_parent_ptr = nullptr;
+    L.block_size = block_size;
+    L.tile_blocks = generic ? kHashThreads : (kHashTileTokens / block_size > 1 ? kHashTileTokens / block_size : 1);
+    const int n_tiles = (int)((nblk + L.tile_blocks - 1) / L.tile_blocks);
+    if (launch_hash(L, n_tiles, generic, vec, stream) != cudaSuccess) return EAKV_E_CUDA;
+    return EAKV_OK;
+}

@@ -65,7 +65,9 @@ EXPORTS = [
     "eakv_hash_blocks_batched", "eakv_match", "eakv_tier_step", "eakv_gpu_tier_step",
     "eakv_gpu_tier_release", "eakv_store", "eakv_load", "eakv_sync", "eakv_get_stats",
     "eakv_tier_ptr", "eakv_hash_seed", "eakv_hash_base", "eakv_strerror", "eakv_last_cuda_error",
+    "eakv_hash_blocks_static",
 ]
+STATIC_MAX_BLOCKS = 65536
 
 
 def lib():
@@ -83,6 +85,7 @@ def lib():
     L.eakv_create.argtypes = [C.POINTER(Config), C.POINTER(vp)]
     L.eakv_destroy.argtypes = [vp]
     L.eakv_hash_blocks.argtypes = [vp, vp, i64, u64, vp, C.POINTER(i64), vp]
+    L.eakv_hash_blocks_static.argtypes = [vp, i64, i32, u64, u64, vp, C.POINTER(i64), vp]
     L.eakv_hash_blocks_batched.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp]
     L.eakv_match.argtypes = [vp, vp, i64, C.POINTER(i64), C.POINTER(i64), vp, vp]
     L.eakv_tier_step.argtypes = [vp, vp, i64, i64, i64, i64, vp, vp, vp, vp, vp,
@@ -116,6 +119,19 @@ def _stream(s):
     if s is None:
         return None
     return C.c_void_p(int(getattr(s, "cuda_stream", s)))
+
+
+def eakv_hash_blocks_static(tokens_dev, n_tokens, block_size, hash_base, parent_hash,
+                            hashes_dev, stream=None):
+    """Context-free, allocation-free block keys (scratch lives inside the library; at most
+    STATIC_MAX_BLOCKS keys per call; calls on one device must not overlap on the GPU)."""
+    n = C.c_int64(0)
+    rc = lib().eakv_hash_blocks_static(C.c_void_p(int(tokens_dev)), int(n_tokens), int(block_size),
+                                       C.c_uint64(int(hash_base)), C.c_uint64(int(parent_hash)),
+                                       C.c_void_p(int(hashes_dev)), C.byref(n), _stream(stream))
+    if rc != OK:
+        raise EakvError(rc, "eakv_hash_blocks_static")
+    return n.value
 
 
 class Context:
