@@ -46,7 +46,7 @@ def parse_args():
     ap.add_argument("--pool-blocks", type=int, default=65536)
     ap.add_argument("--link", default="staged", choices=["zero_copy", "staged"],
                     help="host-link strategy of the e2e arm")
-    ap.add_argument("--copy-path", default="vector", choices=["vector", "bulk"])
+    ap.add_argument("--copy-path", default="bulk", choices=["vector", "bulk"])
     ap.add_argument("--copy-ctas", type=int, default=0)
     ap.add_argument("--host-ctas", type=int, default=0)
     ap.add_argument("--staging-mib", type=int, default=64)
@@ -179,20 +179,18 @@ class Arm:
     def streams(self):
         return {self.hash_stream, self.load_stream, self.store_stream}
 
-    def request(self, tokens, table, agent, now, timed_events=None, step=0):
+    def request(self, tokens, table, agent, now, timed_events=None, step_idx=0):
         """tokens: device int32 tensor (device arm) or pinned host tensor (e2e arm)."""
         torch = self.torch
         hs = self.hash_stream
-        with torch.cuda.stream(hs):
-            if tokens.device.type == "cpu":
-                self.tok_dev.copy_(tokens, non_blocking=True)
-                self.h2d += tokens.numel() * 4
-                tok = self.tok_dev
-            else:
-                tok = tokens
-            nblk = self.ctx.eakv_hash_blocks(tok.data_ptr(), self.n_tokens, self.seed,
-                                             self.keys_dev.data_ptr(), hs)
-            self.keys_host.copy_(self.keys_dev, non_blocking=True)
+        # Lookups never touch a copy engine: queued behind the bulk transfers of other
+        # requests they would wait for all of them.  Host-resident tokens are read by the
+        # hash kernel straight from pinned memory and the keys are written straight into
+        # pinned memory (both mapped into the device's address space).
+        if tokens.device.type == "cpu":
+            self.h2d += tokens.numel() * 4
+        nblk = self.ctx.eakv_hash_blocks(tokens.data_ptr(), self.n_tokens, self.seed,
+                                         self.keys_host.data_ptr(), hs)
         hs.synchronize()
         self.d2h += nblk * 8
         keys = self.keys_host.numpy().view(np.uint64)
@@ -205,14 +203,14 @@ class Arm:
             ev = self._timer(ls, timed_events)
             self.ctx.eakv_load(slots[:H], table[:H], ls)
             self._timer_end(ls, ev, H * self.block_bytes, timed_events)
-            self.load_done[step % 2].record(ls)
+            self.load_done[step_idx % 2].record(ls)
             moved += H * self.block_bytes
             self.h2d += H * self.block_bytes if self.host_tier else 0
         n_admit = int(step["admit"].sum())
         if n_admit:
             ss = self.store_stream
             # the slots this store overwrites held the prompt the previous step restored
-            ss.wait_event(self.load_done[(step - 1) % 2])
+            ss.wait_event(self.load_done[(step_idx - 1) % 2])
             ev = self._timer(ss, timed_events)
             self.ctx.eakv_store(table, step["admit"], step["slot"], ss)
             self._timer_end(ss, ev, n_admit * self.block_bytes, timed_events)
@@ -238,9 +236,9 @@ class Arm:
         use disjoint, freshly drawn pool blocks."""
         m = self.m
         a, _, _ = self.request(prompts[s - 1], tables[s][:m], agent=(s - 1) % 2, now=s * 1000,
-                               timed_events=timed_events, step=s)
+                               timed_events=timed_events, step_idx=s)
         b, _, _ = self.request(prompts[s], tables[s][m:], agent=s % 2, now=s * 1000 + 500,
-                               timed_events=timed_events, step=s)
+                               timed_events=timed_events, step_idx=s)
         return a + b
 
 
@@ -444,7 +442,8 @@ def main():
     kb = sum(b for b, _ in r["kernel"])
     kms = sum(t for _, t in r["kernel"])
     achieved = 2 * kb / (kms * 1e-3) / 1e9 if kms > 0 else 0.0
-    traffic = read_profile_traffic(shape, m)
+    kernel_name = "copy_blocks_vector_kernel" if args.copy_path == "vector" else "copy_blocks_bulk_kernel"
+    traffic = read_profile_traffic(kernel_name, m)
 
     # ---- end-to-end arm (pinned host tier, host tokens) ----
     e2e = None
@@ -493,7 +492,7 @@ def main():
             "gpu_launches": r["launches"],
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
-                         "kernel": "copy_blocks_vector_kernel" if args.copy_path == "vector" else "copy_blocks_bulk_kernel",
+                         "kernel": kernel_name,
                          "launches_timed": len(r["kernel"]),
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "cpu_baseline": cpu,
@@ -520,10 +519,11 @@ def self_check(torch, arm, pool, tables, args, shape):
     return bool(ok)
 
 
-def read_profile_traffic(shape, m):
-    """DRAM bytes per launch of the copy kernel from the committed ncu summary, if present:
-    a line `dram_bytes_per_block = <float>` in profiles/copy_blocks_vector_kernel.txt."""
-    path = os.path.join(ROOT, "profiles", "copy_blocks_vector_kernel.txt")
+def read_profile_traffic(kernel, m):
+    """DRAM bytes per launch of the copy kernel, scaled from the committed ncu summary of a
+    smaller launch (traffic is proportional to blocks moved): the line
+    `dram_bytes_per_block = <float>` in profiles/<kernel>.txt."""
+    path = os.path.join(ROOT, "profiles", kernel + ".txt")
     try:
         for ln in open(path):
             if ln.startswith("dram_bytes_per_block"):

@@ -61,11 +61,14 @@ extern "C" {
 
 /* where the tier lives */
 #define EAKV_TIER_PINNED_HOST 0 /* the product configuration                                   */
-#define EAKV_TIER_DEVICE      1 /* tier in HBM: on-device gather/scatter, for the HBM roofline */
+#define EAKV_TIER_DEVICE      1 /* tier in HBM: on-device gather/scatter, for the HBM roofline;
+                                   always copied directly (link_strategy is ignored)           */
 
 /* which device code moves the bytes */
 #define EAKV_COPY_VECTOR 0      /* 16-byte vector loads/stores, coalesced                       */
-#define EAKV_COPY_BULK   1      /* 1-D bulk async copies through a shared-memory ring           */
+#define EAKV_COPY_BULK   1      /* 1-D bulk async copies through a shared-memory ring (default);
+                                   used for device-resident buffers only: a mapped host tier
+                                   under EAKV_LINK_ZERO_COPY is always moved by the vector kernel */
 
 typedef struct eakv_ctx eakv_ctx;
 
@@ -113,7 +116,8 @@ typedef struct eakv_step_info {
 } eakv_step_info;
 
 /* Fill *cfg with zeros and the paper's controller defaults (Appendix D, parameter table:
- * theta 0.95, 60 s windows, 256 lookups, kappa 8) and write-all policy. */
+ * theta 0.95, 60 s windows, 256 lookups, kappa 8), write-all policy, the staged host-link
+ * strategy and the bulk copy path. */
 int eakv_config_init(eakv_config* cfg);
 
 /* Create a context on the current CUDA device.  Allocates the tier (pinned + mapped, or

@@ -12,10 +12,12 @@
 // copy-engine strategy.
 #include "eakv_internal.h"
 
+#include <cstdlib>
+
 namespace eakv {
 
 template <bool TO_TIER>
-__global__ void __launch_bounds__(kCopyThreads)
+__global__ void __launch_bounds__(kCopyThreads, 8)
 copy_blocks_vector_kernel(CopyLaunch L) {
     const int64_t items_per_entry = (int64_t)L.pieces * L.subs_per_piece;
     const int64_t n_items = L.n_entries * items_per_entry;
@@ -84,8 +86,13 @@ cudaError_t launch_copy_vector(const CopyLaunch& L, bool to_tier, int ctas, cuda
 // ---------------------------------------------------------------------------------------
 namespace eakv {
 
-constexpr int kBulkStages = 4;
-constexpr int kBulkStageBytes = kCopySubBytes;
+constexpr int kBulkMaxStages = 8;
+// Measured on B200 (6 GiB calls, random block ids): 3 stages x 16 KiB with 2 CTAs per SM
+// (96 KiB in flight per SM, ~14 MB on the chip) streams at the HBM copy peak; deeper rings or
+// more CTAs per SM lose 5-6 %.  The EAKV_TUNE_* environment variables override for sweeps.
+static int g_bulk_stages = 3;
+static int g_bulk_stage_bytes = kCopySubBytes;
+static int g_bulk_ctas_per_sm_cap = 2;
 constexpr uint32_t kBulkSpinLimit = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -109,7 +116,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
 struct BulkItem { const char* src; char* dst; uint32_t bytes; };
 
 template <bool TO_TIER>
-__device__ __forceinline__ BulkItem bulk_decode(const CopyLaunch& L, int64_t it) {
+__device__ __forceinline__ BulkItem bulk_decode(const CopyLaunch& L, int64_t it, int kBulkStageBytes) {
     const int64_t items_per_entry = (int64_t)L.pieces * L.subs_per_piece;
     const int64_t j = it / items_per_entry;
     const int r = (int)(it - j * items_per_entry);
@@ -131,9 +138,9 @@ __device__ __forceinline__ BulkItem bulk_decode(const CopyLaunch& L, int64_t it)
 
 template <bool TO_TIER>
 __global__ void __launch_bounds__(32)
-copy_blocks_bulk_kernel(CopyLaunch L, int* error_flag) {
+copy_blocks_bulk_kernel(CopyLaunch L, int* error_flag, int kBulkStages, int kBulkStageBytes) {
     extern __shared__ __align__(128) unsigned char stage_mem[];
-    __shared__ __align__(8) uint64_t bars[kBulkStages];
+    __shared__ __align__(8) uint64_t bars[kBulkMaxStages];
     if (threadIdx.x != 0) return;
 
     const int64_t n_items = L.n_entries * L.pieces * L.subs_per_piece;
@@ -147,7 +154,7 @@ copy_blocks_bulk_kernel(CopyLaunch L, int* error_flag) {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 
     auto issue_load = [&](int64_t k) {
-        const BulkItem b = bulk_decode<TO_TIER>(L, first + k * stride);
+        const BulkItem b = bulk_decode<TO_TIER>(L, first + k * stride, kBulkStageBytes);
         const int s = (int)(k % kBulkStages);
         const uint32_t bar = smem_u32(&bars[s]);
         const uint32_t dst = smem_u32(stage_mem + (size_t)s * kBulkStageBytes);
@@ -168,7 +175,7 @@ copy_blocks_bulk_kernel(CopyLaunch L, int* error_flag) {
         const int s = (int)(k % kBulkStages);
         const uint32_t parity = (uint32_t)((k / kBulkStages) & 1);
         if (!mbar_wait_bounded(smem_u32(&bars[s]), parity)) { ok = false; break; }
-        const BulkItem b = bulk_decode<TO_TIER>(L, first + k * stride);
+        const BulkItem b = bulk_decode<TO_TIER>(L, first + k * stride, kBulkStageBytes);
         const uint32_t src = smem_u32(stage_mem + (size_t)s * kBulkStageBytes);
         asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                      :: "l"(b.dst), "r"(src), "r"(b.bytes) : "memory");
@@ -193,10 +200,17 @@ copy_blocks_bulk_kernel(CopyLaunch L, int* error_flag) {
 
 static int g_bulk_ctas_per_sm = 0;
 
-cudaError_t launch_copy_bulk(const CopyLaunch& L, bool to_tier, int ctas, int* error_flag,
+cudaError_t launch_copy_bulk(const CopyLaunch& L_in, bool to_tier, int ctas, int* error_flag,
                              cudaStream_t stream) {
-    if (L.n_entries <= 0) return cudaSuccess;
-    const size_t smem = (size_t)kBulkStages * kBulkStageBytes;
+    if (L_in.n_entries <= 0) return cudaSuccess;
+    if (g_bulk_ctas_per_sm == 0) {
+        if (const char* e = getenv("EAKV_TUNE_BULK_STAGES")) g_bulk_stages = atoi(e);
+        if (const char* e = getenv("EAKV_TUNE_BULK_STAGE_BYTES")) g_bulk_stage_bytes = atoi(e);
+        if (g_bulk_stages < 2) g_bulk_stages = 2;
+        if (g_bulk_stages > kBulkMaxStages) g_bulk_stages = kBulkMaxStages;
+        if (g_bulk_stage_bytes < 1024 || (g_bulk_stage_bytes & 15)) g_bulk_stage_bytes = kCopySubBytes;
+    }
+    const size_t smem = (size_t)g_bulk_stages * g_bulk_stage_bytes;
     if (g_bulk_ctas_per_sm == 0) {
         cudaError_t e = cudaFuncSetAttribute(copy_blocks_bulk_kernel<true>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -208,7 +222,12 @@ cudaError_t launch_copy_bulk(const CopyLaunch& L, bool to_tier, int ctas, int* e
                                                           copy_blocks_bulk_kernel<true>, 32, smem);
         if (e != cudaSuccess) return e;
         if (g_bulk_ctas_per_sm < 1) g_bulk_ctas_per_sm = 1;
+        if (const char* e2 = getenv("EAKV_TUNE_BULK_CTAS_PER_SM")) g_bulk_ctas_per_sm_cap = atoi(e2);
+        if (g_bulk_ctas_per_sm_cap >= 1 && g_bulk_ctas_per_sm_cap < g_bulk_ctas_per_sm)
+            g_bulk_ctas_per_sm = g_bulk_ctas_per_sm_cap;
     }
+    CopyLaunch L = L_in;
+    L.subs_per_piece = (int32_t)((L.piece_bytes + g_bulk_stage_bytes - 1) / g_bulk_stage_bytes);
     // the auto grid of the vector path assumes its occupancy; rescale to this kernel's
     const int per_sm_vec = copy_vector_ctas_per_sm();
     if (per_sm_vec > 0 && ctas % per_sm_vec == 0 && ctas / per_sm_vec >= 100)
@@ -216,8 +235,8 @@ cudaError_t launch_copy_bulk(const CopyLaunch& L, bool to_tier, int ctas, int* e
     const int64_t n_items = L.n_entries * L.pieces * L.subs_per_piece;
     if (ctas > n_items) ctas = (int)n_items;
     if (ctas < 1) ctas = 1;
-    if (to_tier) copy_blocks_bulk_kernel<true><<<ctas, 32, smem, stream>>>(L, error_flag);
-    else         copy_blocks_bulk_kernel<false><<<ctas, 32, smem, stream>>>(L, error_flag);
+    if (to_tier) copy_blocks_bulk_kernel<true><<<ctas, 32, smem, stream>>>(L, error_flag, g_bulk_stages, g_bulk_stage_bytes);
+    else         copy_blocks_bulk_kernel<false><<<ctas, 32, smem, stream>>>(L, error_flag, g_bulk_stages, g_bulk_stage_bytes);
     return cudaGetLastError();
 }
 

@@ -176,7 +176,9 @@ int launch_copy(eakv_ctx* ctx, const int2* d_entries, int64_t n, char* tier_base
     L.slot_from_index = packed ? 1 : 0;
     L.subs_per_piece = (int32_t)((ctx->piece_bytes + kCopySubBytes - 1) / kCopySubBytes);
     cudaError_t e;
-    if (ctx->cfg.copy_path == EAKV_COPY_BULK)
+    // bulk async copies serve device-resident buffers; a mapped host tier is always driven
+    // by the vector kernel (few CTAs, plain loads/stores over the link)
+    if (ctx->cfg.copy_path == EAKV_COPY_BULK && !touches_host)
         e = launch_copy_bulk(L, to_tier, copy_ctas(ctx, touches_host), ctx->d_error_flag, stream);
     else
         e = launch_copy_vector(L, to_tier, copy_ctas(ctx, touches_host), stream);
@@ -242,9 +244,9 @@ int eakv_config_init(eakv_config* cfg) {
     cfg->len_window = 256;
     cfg->window_ms = 60000;
     cfg->telemetry = 1;
-    cfg->link_strategy = EAKV_LINK_ZERO_COPY;
+    cfg->link_strategy = EAKV_LINK_STAGED;
     cfg->tier_location = EAKV_TIER_PINNED_HOST;
-    cfg->copy_path = EAKV_COPY_VECTOR;
+    cfg->copy_path = EAKV_COPY_BULK;
     return EAKV_OK;
 }
 
@@ -275,6 +277,8 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
     if (!ctx) return EAKV_E_NOMEM;
     ctx->cfg = *cfg;
     ctx->cfg.kv_base = nullptr;
+    // a tier in HBM is copied directly; staging only makes sense across the host link
+    if (cfg->tier_location == EAKV_TIER_DEVICE) ctx->cfg.link_strategy = EAKV_LINK_ZERO_COPY;
     std::memset(&ctx->stats, 0, sizeof(ctx->stats));
     ctx->pieces = pieces;
     ctx->piece_bytes = piece;
@@ -356,7 +360,7 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
     }
 
     // staged strategy
-    if (cfg->link_strategy == EAKV_LINK_STAGED) {
+    if (ctx->cfg.link_strategy == EAKV_LINK_STAGED) {
         int64_t sbytes = cfg->staging_bytes > 0 ? cfg->staging_bytes : (64ll << 20);
         ctx->staging_blocks = std::max<int64_t>(1, sbytes / ctx->block_bytes);
         ctx->staging_blocks = std::min(ctx->staging_blocks, ctx->max_call_blocks);

@@ -140,8 +140,8 @@ class Context:
     def __init__(self, *, num_layers, kv_heads, head_dim, block_size, gpu_blocks, host_blocks,
                  kv_base, elem_bytes=2, gpu_index_blocks=0, hash_base=0, hash_seed=0,
                  policy=POLICY_WRITE_ALL, kappa_blocks=8, theta_percent=95, len_window=256,
-                 window_ms=60_000, telemetry=1, link_strategy=LINK_ZERO_COPY,
-                 tier_location=TIER_PINNED_HOST, copy_path=COPY_VECTOR, copy_ctas=0,
+                 window_ms=60_000, telemetry=1, link_strategy=LINK_STAGED,
+                 tier_location=TIER_PINNED_HOST, copy_path=COPY_BULK, copy_ctas=0,
                  staging_bytes=0, max_call_blocks=0, hash_scratch_blocks=0, tier_memory=0):
         L = lib()
         cfg = Config()

@@ -71,6 +71,12 @@ class AgentServer:
     def close(self):
         self.ctx.close()
 
+    def _ensure_pinned(self, n_tokens):
+        if getattr(self, "_tok_pin", None) is None or self._tok_pin.numel() < n_tokens:
+            cap = 1 << max(12, int(n_tokens - 1).bit_length())
+            self._tok_pin = torch.empty(cap, dtype=torch.int32).pin_memory()
+            self._keys_pin = torch.empty(cap // self.b + 1, dtype=torch.int64).pin_memory()
+
     # -- block keys -------------------------------------------------------------------------
     def block_keys(self, tokens: np.ndarray, agent) -> np.ndarray:
         n = len(tokens)
@@ -81,14 +87,18 @@ class AgentServer:
         if start:
             out[:start] = prev[:start]
         if nblk > start:
-            seg = np.ascontiguousarray(tokens[start * self.b: nblk * self.b], dtype=np.int32)
-            tok_dev = torch.from_numpy(seg).to(self.device, non_blocking=False)
-            keys_dev = torch.empty(nblk - start, dtype=torch.int64, device=self.device)
+            # tokens are handed over in pinned host memory and keys come back into pinned host
+            # memory: the hash kernel reads and writes both directly (they are mapped into
+            # the device's address space), so a lookup never queues behind bulk KV copies
+            seg_len = (nblk - start) * self.b
+            self._ensure_pinned(seg_len)
+            self._tok_pin.numpy()[:seg_len] = tokens[start * self.b: nblk * self.b]
             parent = int(out[start - 1]) if start else self.seed
-            got = self.ctx.eakv_hash_blocks(tok_dev.data_ptr(), len(seg), parent,
-                                            keys_dev.data_ptr(), self.stream)
+            got = self.ctx.eakv_hash_blocks(self._tok_pin.data_ptr(), seg_len, parent,
+                                            self._keys_pin.data_ptr(), self.stream)
             assert got == nblk - start
-            out[start:] = keys_dev.cpu().numpy().view(np.uint64)
+            self.stream.synchronize()
+            out[start:] = self._keys_pin.numpy()[:got].view(np.uint64)
         if self.incremental:
             self._agent_keys[agent] = out
         return out

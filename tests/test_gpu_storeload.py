@@ -29,8 +29,6 @@ def variants():
     for link, loc, path in itertools.product((e.LINK_ZERO_COPY, e.LINK_STAGED),
                                              (e.TIER_PINNED_HOST, e.TIER_DEVICE),
                                              (e.COPY_VECTOR, e.COPY_BULK)):
-        if path == e.COPY_BULK and loc == e.TIER_PINNED_HOST and link == e.LINK_ZERO_COPY:
-            continue      # bulk copies are only used on device-resident buffers
         out.append(dict(link_strategy=link, tier_location=loc, copy_path=path))
     return out
 
