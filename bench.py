@@ -55,6 +55,9 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--hash-only", action="store_true",
+                    help="run only the prefix-hash throughput section and print its JSON")
+    ap.add_argument("--hash-prompts", type=int, default=512)
     ap.add_argument("--sweep", action="store_true",
                     help="also print the 1..4096-block curve (contiguous/random ids, masks)")
     return ap.parse_args()
@@ -279,6 +282,46 @@ def run_arm(arm, prompts, tables, steps, warmup, dist, clocks=None, time_kernels
                 h2d=arm.h2d / steps, d2h=arm.d2h / steps)
 
 
+def hash_throughput(torch, eakv, pool, shape, device, peak_gbs, prompts=512, tokens=65536, reps=10):
+    """Prefix-hash rate: a batch of long prompts in one launch (device-resident tokens, larger
+    than L2), and the latency of one 64k-token prompt."""
+    ctx = eakv.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+                       block_size=shape.block_size, gpu_blocks=pool.gpu_blocks, host_blocks=1,
+                       kv_base=pool.kv_base, tier_location=eakv.TIER_DEVICE,
+                       tier_memory=pool.pieces[0].data_ptr(),
+                       hash_scratch_blocks=prompts * tokens // shape.block_size)
+    toks = torch.randint(0, 151936, (prompts * tokens,), dtype=torch.int32, device=device)
+    keys = torch.empty(prompts * tokens // shape.block_size, dtype=torch.int64, device=device)
+    offsets = np.arange(prompts + 1, dtype=np.int64) * tokens
+    stream = torch.cuda.current_stream(device)
+    best = None
+    for i in range(reps + 3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        ctx.eakv_hash_blocks_batched(toks.data_ptr(), offsets, None, keys.data_ptr(), stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if i >= 3:
+            ms = e0.elapsed_time(e1)
+            best = ms if best is None else min(best, ms)
+    single = []
+    seed = ctx.eakv_hash_seed()
+    for i in range(reps + 3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        ctx.eakv_hash_blocks(toks.data_ptr() + 4 * tokens * (i % prompts), tokens, seed, keys.data_ptr(), stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if i >= 3:
+            single.append(e0.elapsed_time(e1) * 1e3)
+    ctx.close()
+    rate = prompts * tokens / (best * 1e-3)
+    return {"batched_tokens_per_s": rate, "batch": f"{prompts} prompts x {tokens} tokens, block {shape.block_size}",
+            "batched_ms": best, "frac_of_hbm_bound": rate * 4 / 1e9 / peak_gbs,
+            "hbm_bound_tokens_per_s": peak_gbs * 1e9 / 4,
+            "single_prompt_tokens": tokens, "single_prompt_us_median": float(np.median(single))}
+
+
 def pinned_link_peak(torch, device, gib=1, reps=5):
     n = gib << 30
     host = torch.empty(n, dtype=torch.uint8).pin_memory()
@@ -415,6 +458,16 @@ def main():
     pool = PagedPool(shape, nb, device, fill=lambda q, t: t.random_())
     torch.cuda.synchronize()
 
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    else:
+        peak, peak_src = 6650.0, "fallback"
+    if args.hash_only:
+        print(json.dumps({"hash": hash_throughput(torch, eakv, pool, shape, device, peak,
+                                                  prompts=args.hash_prompts)}))
+        return
+
     total_steps = args.steps + args.warmup + 1
     rng = np.random.default_rng(1 + rank)
     tok_np = rng.integers(0, 151936, size=(total_steps + 1, m * shape.block_size), dtype=np.int32)
@@ -434,11 +487,6 @@ def main():
     ms_max, moved_sum = aggregate_over_ranks(dist, r["ms"], r["moved"], device)
     value = moved_sum / (ms_max * 1e-3) / 1e9
 
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
-    else:
-        peak, peak_src = 6650.0, "fallback"
     kb = sum(b for b, _ in r["kernel"])
     kms = sum(t for _, t in r["kernel"])
     achieved = 2 * kb / (kms * 1e-3) / 1e9 if kms > 0 else 0.0
@@ -470,6 +518,8 @@ def main():
                        frac_of_link=e_val / bound / max(world, 1),
                        frac_of_one_direction=e_val / serial / max(world, 1))
 
+    hashing = hash_throughput(torch, eakv, pool, shape, device, peak) if rank == 0 else None
+
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:
         g, s, dt = oracle_step_rate(args.cpu_seconds)
@@ -496,6 +546,7 @@ def main():
                          "launches_timed": len(r["kernel"]),
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "cpu_baseline": cpu,
+            "hash": hashing,
         }
         print(json.dumps(line))
         if args.sweep:

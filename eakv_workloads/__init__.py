@@ -8,6 +8,6 @@ path can both consume it without sharing any of the code under test.
 from .shapes import KVShape, SHAPES, CONFIGS, TraceConfig  # noqa: F401
 from .traces import Trace, Request, make_trace  # noqa: F401
 from .kvfill import (  # noqa: F401
-    normal_bf16_words, counter_words_numpy, counter_words_torch, key_words_numpy,
-    key_words_torch,
+    normal_bf16_words, counter_words_numpy, counter_words_torch, counter_words_at_torch,
+    key_words_numpy, key_words_torch,
 )

@@ -47,6 +47,13 @@ def counter_words_torch(salt: int, start: int, n_words: int, device):
     return ((v >> 29) & 0xBFFF).to(torch.int16)
 
 
+def counter_words_at_torch(salt: int, idx):
+    """``counter_words_torch`` evaluated at arbitrary int64 element indices ``idx``."""
+    import torch
+    v = (idx.to(torch.int64) * _signed(_M1) + _signed(salt)) * _signed(_M2)
+    return ((v >> 29) & 0xBFFF).to(torch.int16)
+
+
 def key_words_numpy(keys, q: int, n_words: int) -> np.ndarray:
     """[len(keys), n_words] uint16: payload of piece ``q`` of the blocks with these keys."""
     keys = np.asarray(keys, dtype=np.uint64).reshape(-1, 1)

@@ -416,9 +416,9 @@ int eakv_hash_blocks(eakv_ctx* ctx, const int32_t* tokens_dev, int64_t n_tokens,
     if (((uintptr_t)tokens_dev & 3) || ((uintptr_t)hashes_dev & 7)) return EAKV_E_INVAL;
     DeviceGuard g(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const bool generic = (b % 4) != 0;
-    const bool vec = !generic && (((uintptr_t)tokens_dev & 15) == 0);
-    const int tile_blocks = generic ? kHashThreads : std::max(1, kHashTileTokens / b);
+    const bool generic = hash_thread_per_block(b);
+    const bool vec = (b % 4) == 0 && (((uintptr_t)tokens_dev & 15) == 0);
+    const int tile_blocks = hash_tile_blocks(b, nblk);
     // split at the scratch capacity; a later piece reads its parent from the previous key
     const int64_t cap = ctx->hash_scratch_blocks;
     int64_t done = 0;
@@ -474,9 +474,9 @@ int eakv_hash_blocks_batched(eakv_ctx* ctx, const int32_t* tokens_dev,
     if (((uintptr_t)tokens_dev & 3) || ((uintptr_t)hashes_dev & 7)) return EAKV_E_INVAL;
     DeviceGuard g(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const bool generic = (b % 4) != 0;
-    bool vec = !generic && (((uintptr_t)tokens_dev & 15) == 0);
-    const int tile_blocks = generic ? kHashThreads : std::max(1, kHashTileTokens / b);
+    const bool generic = hash_thread_per_block(b);
+    bool vec = (b % 4) == 0 && (((uintptr_t)tokens_dev & 15) == 0);
+    const int tile_blocks = hash_tile_blocks(b, total_blocks);
 
     int64_t n_tiles = 0;
     for (int64_t i = 0; i < n_prompts; ++i) {

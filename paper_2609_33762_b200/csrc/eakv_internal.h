@@ -10,7 +10,7 @@ constexpr int kHashThreads = 256;
 constexpr int kHashUnroll = 4;
 constexpr int kHashTileTokens = kHashThreads * kHashUnroll * 4;   // 4096 tokens per CTA tile
 constexpr int kHashMaxBlockSize = 4096;
-constexpr int kHashMaxSmem = 64 * 1024;
+constexpr int kHashMaxSmem = 80 * 1024;
 
 struct HashTile { int32_t prompt; int32_t first_block; };
 struct HashPrompt {
@@ -35,8 +35,21 @@ struct HashLaunch {
     int32_t block_size;
     int32_t tile_blocks;
 };
+// one thread per block for small or odd block sizes, a group of threads per block otherwise
+inline bool hash_thread_per_block(int block_size) { return (block_size % 4) != 0 || block_size <= 64; }
+// blocks per CTA tile; large batches get longer tiles so fewer CTAs take tickets
+inline int hash_tile_blocks(int block_size, int64_t total_blocks) {
+    if (hash_thread_per_block(block_size)) {
+        int t = kHashThreads;
+        while (t < 4 * kHashThreads && total_blocks / t > 1184) t *= 2;
+        return t;
+    }
+    const int t = kHashTileTokens / block_size;
+    return t > 1 ? t : 1;
+}
 cudaError_t hash_kernels_init();
-cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool generic, bool vec, cudaStream_t stream);
+cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool thread_per_block, bool vec,
+                        cudaStream_t stream);
 
 // ---- gather / scatter ---------------------------------------------------------------------
 constexpr int kCopyThreads = 256;

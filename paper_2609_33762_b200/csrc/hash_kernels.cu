@@ -69,18 +69,35 @@ __device__ __forceinline__ Pair compose(Pair first, Pair second) {
 
 // Scan of one prompt's block partials into keys, by one whole CTA.
 //   partial[0..nblk) -> keys[0..nblk),  keys[j] = keys[j-1] * A + partial[j], keys[-1] = parent
-__device__ void scan_prompt(const uint64_t* partial, uint64_t* keys, int64_t nblk, uint64_t parent,
+__device__ __noinline__ void scan_prompt(const uint64_t* partial, uint64_t* keys, int64_t nblk, uint64_t parent,
                             uint64_t A, Pair* warp_tot /* smem [32] */) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
     const int64_t per = (nblk + nthr - 1) / nthr;
     const int64_t lo = min((int64_t)tid * per, nblk), hi = min(lo + per, nblk);
-    // fold this thread's run
+    // fold this thread's run (kept in registers when short, so the loads overlap)
+    constexpr int kRegRun = 8;
+    uint64_t run[kRegRun];
+    const bool in_regs = per <= kRegRun;
+    if (in_regs) {
+#pragma unroll
+        for (int i = 0; i < kRegRun; ++i) run[i] = (lo + i < hi) ? __ldcg(partial + lo + i) : 0;
+    }
     Pair mine{1, 0};
-    for (int64_t j = lo; j < hi; ++j) {
-        const uint64_t c = __ldcg(partial + j);
-        mine.a = mulmod61(mine.a, A);
-        mine.c = addmod61(mulmod61(mine.c, A), c);
+    if (in_regs) {
+#pragma unroll
+        for (int i = 0; i < kRegRun; ++i) {
+            if (lo + i < hi) {
+                mine.a = mulmod61(mine.a, A);
+                mine.c = addmod61(mulmod61(mine.c, A), run[i]);
+            }
+        }
+    } else {
+        for (int64_t j = lo; j < hi; ++j) {
+            const uint64_t c = __ldcg(partial + j);
+            mine.a = mulmod61(mine.a, A);
+            mine.c = addmod61(mulmod61(mine.c, A), c);
+        }
     }
     // inclusive warp scan over threads (earlier lanes apply first)
     Pair inc = mine;
@@ -112,9 +129,19 @@ __device__ void scan_prompt(const uint64_t* partial, uint64_t* keys, int64_t nbl
     if (lane == 0) exc = Pair{1, 0};
     if (warp > 0) exc = compose(warp_tot[warp - 1], exc);
     uint64_t h = addmod61(mulmod61(parent, exc.a), exc.c);
-    for (int64_t j = lo; j < hi; ++j) {
-        h = addmod61(mulmod61(h, A), __ldcg(partial + j));
-        keys[j] = h;
+    if (in_regs) {
+#pragma unroll
+        for (int i = 0; i < kRegRun; ++i) {
+            if (lo + i < hi) {
+                h = addmod61(mulmod61(h, A), run[i]);
+                keys[lo + i] = h;
+            }
+        }
+    } else {
+        for (int64_t j = lo; j < hi; ++j) {
+            h = addmod61(mulmod61(h, A), __ldcg(partial + j));
+            keys[j] = h;
+        }
     }
     __syncthreads();
 }
@@ -201,15 +228,46 @@ hash_blocks_kernel(HashLaunch L) {
     if (tid == 0) L.counters[p] = 0;   // ready for the next launch
 }
 
-// Any block size (not a multiple of 4): one thread per block, same two steps.
+// Thread-per-block variant: used for small blocks (<= 64 tokens, where it needs the fewest
+// instructions per token) and for block sizes that are not a multiple of four.  Each power
+// B^e is split into three 21-bit limbs, so a token costs three 32x21-bit multiply-adds into
+// three 64-bit sums that cannot overflow for up to 2,048 tokens; the sums are folded mod p
+// once per block.  The limb table is read from shared memory (broadcast: all lanes use the
+// same power at the same time).  Lanes read 16 bytes at a 4*b-byte stride, so a warp's loads
+// together cover a contiguous span that L1 serves.
+__device__ __forceinline__ uint64_t fold_limb_sums(uint64_t s0, uint64_t s1, uint64_t s2) {
+    // s0 + s1 * 2^21 + s2 * 2^42 (mod p), with 2^61 == 1
+    const uint64_t r = (s0 & P61) + (s0 >> 61)
+                     + (s1 >> 40) + ((s1 & ((1ull << 40) - 1)) << 21)
+                     + (s2 >> 19) + ((s2 & ((1ull << 19) - 1)) << 42);   // < 2^63
+    return reduce_once(r);
+}
+
+constexpr int kLimbFoldTokens = 1024;   // 1024 * 2^32 * 2^21 = 2^63: no overflow in between
+
+#define EAKV_MAC3(tok, e)                                   \
+    do {                                                    \
+        const uint32_t x_ = (uint32_t)(tok) + 1u;           \
+        const uint4 w_ = pw3[(e)];                          \
+        s0 += (uint64_t)x_ * w_.x;                          \
+        s1 += (uint64_t)x_ * w_.y;                          \
+        s2 += (uint64_t)x_ * w_.z;                          \
+    } while (0)
+
+template <bool VEC>
 __global__ void __launch_bounds__(kHashThreads)
-hash_blocks_generic_kernel(HashLaunch L) {
+hash_blocks_tpb_kernel(HashLaunch L) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint64_t* pw = reinterpret_cast<uint64_t*>(smem_raw);
+    uint4* pw3 = reinterpret_cast<uint4*>(smem_raw);       // limbs of B^0 .. B^(b-1)
     __shared__ Pair warp_tot[32];
     __shared__ int is_last;
     const int tid = threadIdx.x;
-    for (int e = tid; e <= L.block_size; e += blockDim.x) pw[e] = L.pow_table[e];
+    const int b = L.block_size;
+    for (int e = tid; e < b; e += blockDim.x) {
+        const uint64_t w = L.pow_table[e];
+        pw3[e] = make_uint4((uint32_t)(w & 0x1FFFFF), (uint32_t)((w >> 21) & 0x1FFFFF),
+                            (uint32_t)(w >> 42), 0u);
+    }
     int32_t p = 0;
     int64_t first_blk = (int64_t)blockIdx.x * L.tile_blocks;
     int64_t tok0 = 0, blk0 = 0, nblk = L.single_nblk;
@@ -229,11 +287,25 @@ hash_blocks_generic_kernel(HashLaunch L) {
     __syncthreads();
     uint64_t* partial = L.partial + blk0;
     for (int64_t j = tid; j < nb_tile; j += blockDim.x) {
-        const int32_t* t = L.tokens + tok0 + (first_blk + j) * L.block_size;
-        uint64_t s = 0;
-        for (int k = 0; k < L.block_size; ++k)
-            s = addmod61(s, mulmod61((uint64_t)((uint32_t)t[k] + 1u), pw[L.block_size - 1 - k]));
-        __stcg(partial + first_blk + j, s);
+        const int32_t* t = L.tokens + tok0 + (first_blk + j) * b;
+        uint64_t acc = 0;
+        for (int k0 = 0; k0 < b; k0 += kLimbFoldTokens) {
+            const int k1 = min(b, k0 + kLimbFoldTokens);
+            uint64_t s0 = 0, s1 = 0, s2 = 0;
+            int k = k0;
+            if (VEC) {
+                const int4* t4 = reinterpret_cast<const int4*>(t);
+#pragma unroll 4
+                for (; k + 4 <= k1; k += 4) {
+                    const int4 u = __ldg(t4 + (k >> 2));
+                    const int e = b - 1 - k;
+                    EAKV_MAC3(u.x, e); EAKV_MAC3(u.y, e - 1); EAKV_MAC3(u.z, e - 2); EAKV_MAC3(u.w, e - 3);
+                }
+            }
+            for (; k < k1; ++k) EAKV_MAC3(__ldg(t + k), b - 1 - k);
+            acc = addmod61(acc, fold_limb_sums(s0, s1, s2));
+        }
+        __stcg(partial + first_blk + j, acc);
     }
     __threadfence();
     __syncthreads();
@@ -244,15 +316,19 @@ hash_blocks_generic_kernel(HashLaunch L) {
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    scan_prompt(partial, L.keys + blk0, nblk, parent, pw[L.block_size], warp_tot);
+    scan_prompt(partial, L.keys + blk0, nblk, parent, L.pow_table[b], warp_tot);
     if (tid == 0) L.counters[p] = 0;
 }
+#undef EAKV_MAC3
 
-cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool generic, bool vec, cudaStream_t stream) {
+// thread_per_block: see hash_thread_per_block(); vec: 16-byte token loads are allowed
+cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool thread_per_block, bool vec,
+                        cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
-    if (generic) {
-        const size_t smem = (size_t)(L.block_size + 1) * 8;
-        hash_blocks_generic_kernel<<<n_tiles, kHashThreads, smem, stream>>>(L);
+    if (thread_per_block) {
+        const size_t smem = (size_t)L.block_size * sizeof(uint4);
+        if (vec) hash_blocks_tpb_kernel<true><<<n_tiles, kHashThreads, smem, stream>>>(L);
+        else     hash_blocks_tpb_kernel<false><<<n_tiles, kHashThreads, smem, stream>>>(L);
     } else {
         const size_t smem = (size_t)(L.block_size + 1) * 8 +
                             (size_t)L.tile_blocks * (L.block_size / 4) * 8;
@@ -270,7 +346,10 @@ cudaError_t hash_kernels_init() {
     e = cudaFuncSetAttribute(hash_blocks_kernel<false>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, kHashMaxSmem);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(hash_blocks_generic_kernel,
+    e = cudaFuncSetAttribute(hash_blocks_tpb_kernel<true>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kHashMaxSmem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(hash_blocks_tpb_kernel<false>,
                                 cudaFuncAttributeMaxDynamicSharedMemorySize, kHashMaxSmem);
 }
 
@@ -367,8 +446,8 @@ extern "C" int eakv_hash_blocks_static(const int32_t* tokens_dev, int64_t n_toke
     fill_pow_table_kernel<<<(n_pow + 255) / 256, 256, 0, stream>>>(pw, base, n_pow);
     if (cudaGetLastError() != cudaSuccess) return EAKV_E_CUDA;
 
-    const bool generic = (block_size % 4) != 0;
-    const bool vec = !generic && (((uintptr_t)tokens_dev & 15) == 0);
+    const bool generic = hash_thread_per_block(block_size);
+    const bool vec = (block_size % 4) == 0 && (((uintptr_t)tokens_dev & 15) == 0);
     HashLaunch L;
     L.tokens = tokens_dev;
     L.keys = hashes_dev;
@@ -381,7 +460,7 @@ extern "C" int eakv_hash_blocks_static(const int32_t* tokens_dev, int64_t n_toke
     L.single_parent = parent_hash % P;
     L.single_parent_ptr = nullptr;
     L.block_size = block_size;
-    L.tile_blocks = generic ? kHashThreads : (kHashTileTokens / block_size > 1 ? kHashTileTokens / block_size : 1);
+    L.tile_blocks = hash_tile_blocks(block_size, nblk);
     const int n_tiles = (int)((nblk + L.tile_blocks - 1) / L.tile_blocks);
     if (launch_hash(L, n_tiles, generic, vec, stream) != cudaSuccess) return EAKV_E_CUDA;
     return EAKV_OK;

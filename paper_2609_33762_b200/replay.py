@@ -1,0 +1,125 @@
+"""Replay a synthetic agent trace through the eakv path and report what the paper reports
+for its replays: computed (fresh) prefill tokens, host writes and restores, hit tokens —
+plus the achieved store/load rates.
+
+    python -m paper_2609_33762_b200.replay --config c2              # tier sized by Eq. 5
+    python -m paper_2609_33762_b200.replay --config c3 --policy conditioned
+    python -m paper_2609_33762_b200.replay --config c4 --host-gib 64 --limit 2000
+
+Sizing follows the paper's rule: working-set scale (A - 1) * N_mean * beta (Eq. 5) for
+configurations that ask for a tier "sized to the working set", capped by the pinned memory
+the box can spare.  With --no-data-plane only keys, matching and both tiers' bookkeeping run.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import time
+
+import numpy as np
+
+from . import eakv
+
+POLICIES = {"write_all": eakv.POLICY_WRITE_ALL, "fixed": eakv.POLICY_FILTER_FIXED,
+            "conditioned": eakv.POLICY_FILTER_CONDITIONED}
+GIB = 1 << 30
+
+
+def working_set_blocks(trace, shape):
+    """Eq. 5 in blocks: (A - 1) * mean prompt length * beta / block bytes."""
+    n_mean = trace.total_prompt_tokens / len(trace.requests)
+    agents = len(trace.agent_tokens)
+    return int((agents - 1) * n_mean * shape.bytes_per_token // shape.block_bytes)
+
+
+def mem_available_bytes():
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable:"):
+                return int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    return 0
+
+
+def plan(cfg, trace, shape, host_gib=None, data_plane=True, ram_fraction=0.6):
+    """Tier capacity in blocks for a configuration and the reason for it."""
+    if host_gib is not None:
+        kh, why = int(host_gib * GIB // shape.block_bytes), f"{host_gib} GiB requested"
+    elif cfg.host_blocks:
+        kh, why = cfg.host_blocks, "fixed by the configuration"
+    else:
+        kh, why = working_set_blocks(trace, shape), "working-set scale (A-1)*N_mean*beta"
+    if data_plane:
+        cap = int(mem_available_bytes() * ram_fraction // shape.block_bytes)
+        if cap and kh > cap:
+            kh, why = cap, why + f", capped at {ram_fraction:.0%} of available host memory"
+    return kh, why
+
+
+def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=True,
+        incremental_hash=True, device="cuda:0", link_strategy=eakv.LINK_STAGED, agents=None,
+        turns=None, server_hook=None):
+    import torch
+    from eakv_workloads import CONFIGS, SHAPES, key_words_torch, make_trace
+    from .harness import AgentServer
+
+    cfg = CONFIGS[config]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg, agents=agents, turns=turns)
+    kh, why = plan(cfg, trace, shape, host_gib, data_plane)
+    payload = (lambda keys, q, n: key_words_torch(keys.astype(np.int64), q, n, device)) if data_plane else None
+    t0 = time.perf_counter()
+    server = AgentServer(shape, cfg.gpu_blocks, kh, payload, device=device, data_plane=data_plane,
+                         incremental_hash=incremental_hash, policy=POLICIES[policy],
+                         kappa_blocks=cfg.kappa_blocks, link_strategy=link_strategy)
+    t_setup = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    server.run(trace, limit=limit)
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    if server_hook is not None:
+        server_hook(server, trace)
+    st = server.ctx.eakv_get_stats()
+    tot = server.totals
+    n_req = len(server.records)
+    out = {
+        "config": config, "policy": policy, "requests": n_req, "kv_shape": cfg.shape,
+        "gpu_blocks": cfg.gpu_blocks, "host_blocks": kh, "host_gib": kh * shape.block_bytes / GIB,
+        "host_sizing": why, "data_plane": data_plane,
+        "working_set_blocks_eq5": working_set_blocks(trace, shape),
+        "prompt_tokens": tot["prompt_tokens"], "computed_prefill_tokens": tot["fresh_tokens"],
+        "gpu_hit_tokens": tot["gpu_hit_blocks"] * shape.block_size,
+        "host_hit_tokens": tot["host_hit_blocks"] * shape.block_size,
+        "restored_tokens": tot["loaded_blocks"] * shape.block_size,
+        "stored_tokens": tot["stored_blocks"] * shape.block_size,
+        "restored_gib": tot["loaded_blocks"] * shape.block_bytes / GIB,
+        "stored_gib": tot["stored_blocks"] * shape.block_bytes / GIB,
+        "declined_requests": st["declined_requests"], "pressure_requests": st["pressure_requests"],
+        "declined_blocks": st["declined"], "evicted_blocks": st["evicted"],
+        "tokens_hashed": st["tokens_hashed"], "kernel_launches": st["kernel_launches"],
+        "wall_s": wall, "setup_s": t_setup,
+        "moved_gb_per_s_wall": (tot["loaded_blocks"] + tot["stored_blocks"]) * shape.block_bytes / wall / 1e9
+        if data_plane else None,
+    }
+    server.close()
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", default="c2", choices=["c0", "c0_big_tier", "c2", "c3", "c4"])
+    ap.add_argument("--policy", default="write_all", choices=sorted(POLICIES))
+    ap.add_argument("--host-gib", type=float, default=None)
+    ap.add_argument("--limit", type=int, default=None, help="replay only the first N requests")
+    ap.add_argument("--no-data-plane", dest="data_plane", action="store_false")
+    ap.add_argument("--zero-copy", action="store_true", help="zero-copy host link instead of staged")
+    args = ap.parse_args()
+    out = run(args.config, policy=args.policy, host_gib=args.host_gib, limit=args.limit,
+              data_plane=args.data_plane,
+              link_strategy=eakv.LINK_ZERO_COPY if args.zero_copy else eakv.LINK_STAGED)
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

@@ -129,20 +129,3 @@ def test_tier_step_capacity_error_changes_nothing():
     G, H, gids, slots = server.ctx.eakv_match(keys)
     assert (G, H) == (0, 2) and slots.tolist() == [0, 1]
     server.close()
-
-
-def test_config2_control_plane_prefix():
-    """Config 2's own trace and KV shape, bookkeeping only (keys, match, both tiers), on
-    the first 400 requests with the 32 GiB tier of config 3 under conditioned admission."""
-    from paper_2609_33762_b200.harness import AgentServer
-    cfg = CONFIGS["c3"]
-    shape = SHAPES[cfg.shape]
-    trace = make_trace(cfg)
-    kw = dict(policy=2, kappa_blocks=cfg.kappa_blocks)
-    oracle = TraceOracle(shape, cfg.gpu_blocks, cfg.host_blocks, **kw)
-    oracle.run(trace, limit=400)
-    server = AgentServer(shape, cfg.gpu_blocks, cfg.host_blocks, None, data_plane=False,
-                         incremental_hash=True, **kw)
-    server.run(trace, limit=400)
-    compare_records(server.records, oracle.records)
-    server.close()
