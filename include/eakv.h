@@ -93,6 +93,10 @@ typedef struct eakv_config {
     int64_t staging_bytes;         /* per staging buffer (two per direction); 0 = 64 MiB         */
     int64_t max_call_blocks;       /* entries per argument-ring slot; 0 = 16384                  */
     int64_t hash_scratch_blocks;   /* block partials the hash scratch holds; 0 = 1 << 20        */
+    int64_t min_staged_run_bytes;  /* EAKV_LINK_STAGED: a call whose runs of consecutive slots
+                                      average fewer bytes than this goes zero-copy instead (the
+                                      copy engine's per-copy cost outweighs its edge on scattered
+                                      single blocks); 0 = 3 MiB, negative = always stage         */
     void*   tier_memory;           /* NULL: the context allocates the tier.  Else adopt this
                                       buffer of host_blocks * block bytes (pinned host memory
                                       for TIER_PINNED_HOST, device memory for TIER_DEVICE);

@@ -27,9 +27,13 @@ copy_blocks_vector_kernel(CopyLaunch L) {
         const int r = (int)(it - j * items_per_entry);
         const int q = r / L.subs_per_piece;
         const int sub = r - q * L.subs_per_piece;
-        const int2 e = __ldg(L.entries + j);
+        const int2 e = L.entries ? __ldg(L.entries + j) : L.inline_entries[j];
         char* pool = reinterpret_cast<char*>(__ldg(reinterpret_cast<const unsigned long long*>(L.kv_base) + q)) + (int64_t)e.x * L.piece_bytes;
         const int64_t slot = L.slot_from_index ? j : (int64_t)e.y;
+        if ((uint64_t)e.x >= (uint64_t)L.gpu_blocks || (uint64_t)slot >= (uint64_t)L.tier_slots) {
+            if (threadIdx.x == 0) atomicExch(L.error_flag, kErrCopyRange);
+            continue;
+        }
         char* tier = L.tier_base + (slot * L.pieces + q) * L.piece_bytes;
         const int4* src = reinterpret_cast<const int4*>(TO_TIER ? pool : tier);
         int4* dst = reinterpret_cast<int4*>(TO_TIER ? tier : pool);
@@ -122,13 +126,17 @@ __device__ __forceinline__ BulkItem bulk_decode(const CopyLaunch& L, int64_t it,
     const int r = (int)(it - j * items_per_entry);
     const int q = r / L.subs_per_piece;
     const int sub = r - q * L.subs_per_piece;
-    const int2 e = __ldg(L.entries + j);
+    const int2 e = L.entries ? __ldg(L.entries + j) : L.inline_entries[j];
     const int64_t off = (int64_t)sub * kBulkStageBytes;
     char* pool = reinterpret_cast<char*>(__ldg(reinterpret_cast<const unsigned long long*>(L.kv_base) + q)) +
                  (int64_t)e.x * L.piece_bytes + off;
     const int64_t slot = L.slot_from_index ? j : (int64_t)e.y;
-    char* tier = L.tier_base + (slot * L.pieces + q) * L.piece_bytes + off;
     BulkItem b;
+    if ((uint64_t)e.x >= (uint64_t)L.gpu_blocks || (uint64_t)slot >= (uint64_t)L.tier_slots) {
+        b.src = nullptr; b.dst = nullptr; b.bytes = 0;      // the caller flags and skips it
+        return b;
+    }
+    char* tier = L.tier_base + (slot * L.pieces + q) * L.piece_bytes + off;
     b.src = TO_TIER ? pool : tier;
     b.dst = TO_TIER ? tier : pool;
     const int64_t left = L.piece_bytes - off;
@@ -138,7 +146,8 @@ __device__ __forceinline__ BulkItem bulk_decode(const CopyLaunch& L, int64_t it,
 
 template <bool TO_TIER>
 __global__ void __launch_bounds__(32)
-copy_blocks_bulk_kernel(CopyLaunch L, int* error_flag, int kBulkStages, int kBulkStageBytes) {
+copy_blocks_bulk_kernel(CopyLaunch L, int kBulkStages, int kBulkStageBytes) {
+    int* const error_flag = L.error_flag;
     extern __shared__ __align__(128) unsigned char stage_mem[];
     __shared__ __align__(8) uint64_t bars[kBulkMaxStages];
     if (threadIdx.x != 0) return;
@@ -152,6 +161,14 @@ copy_blocks_bulk_kernel(CopyLaunch L, int* error_flag, int kBulkStages, int kBul
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&bars[s])) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+
+    // self-check: every item of this CTA must be in range before anything is issued
+    for (int64_t k = 0; k < n_my; ++k) {
+        if (bulk_decode<TO_TIER>(L, first + k * stride, kBulkStageBytes).bytes == 0) {
+            atomicExch(error_flag, kErrCopyRange);
+            return;
+        }
+    }
 
     auto issue_load = [&](int64_t k) {
         const BulkItem b = bulk_decode<TO_TIER>(L, first + k * stride, kBulkStageBytes);
@@ -188,7 +205,7 @@ copy_blocks_bulk_kernel(CopyLaunch L, int* error_flag, int kBulkStages, int kBul
         }
     }
     if (!ok) {
-        atomicExch(error_flag, 1);
+        atomicExch(error_flag, kErrBulkTimeout);
         // drain the loads still in flight (bounded) so shared memory is quiescent on exit
         for (int64_t d = k + 1; d < loads_issued; ++d) {
             const int s = (int)(d % kBulkStages);
@@ -200,8 +217,7 @@ copy_blocks_bulk_kernel(CopyLaunch L, int* error_flag, int kBulkStages, int kBul
 
 static int g_bulk_ctas_per_sm = 0;
 
-cudaError_t launch_copy_bulk(const CopyLaunch& L_in, bool to_tier, int ctas, int* error_flag,
-                             cudaStream_t stream) {
+cudaError_t launch_copy_bulk(const CopyLaunch& L_in, bool to_tier, int ctas, cudaStream_t stream) {
     if (L_in.n_entries <= 0) return cudaSuccess;
     if (g_bulk_ctas_per_sm == 0) {
         if (const char* e = getenv("EAKV_TUNE_BULK_STAGES")) g_bulk_stages = atoi(e);
@@ -235,8 +251,8 @@ cudaError_t launch_copy_bulk(const CopyLaunch& L_in, bool to_tier, int ctas, int
     const int64_t n_items = L.n_entries * L.pieces * L.subs_per_piece;
     if (ctas > n_items) ctas = (int)n_items;
     if (ctas < 1) ctas = 1;
-    if (to_tier) copy_blocks_bulk_kernel<true><<<ctas, 32, smem, stream>>>(L, error_flag, g_bulk_stages, g_bulk_stage_bytes);
-    else         copy_blocks_bulk_kernel<false><<<ctas, 32, smem, stream>>>(L, error_flag, g_bulk_stages, g_bulk_stage_bytes);
+    if (to_tier) copy_blocks_bulk_kernel<true><<<ctas, 32, smem, stream>>>(L, g_bulk_stages, g_bulk_stage_bytes);
+    else         copy_blocks_bulk_kernel<false><<<ctas, 32, smem, stream>>>(L, g_bulk_stages, g_bulk_stage_bytes);
     return cudaGetLastError();
 }
 

@@ -78,6 +78,7 @@ struct eakv_ctx {
     // staged strategy
     Staging st_store, st_load;
     int64_t staging_blocks = 0;
+    int64_t min_staged_run_bytes = 0;
 
     int* d_error_flag = nullptr;
 
@@ -164,22 +165,27 @@ int copy_ctas(const eakv_ctx* ctx, bool touches_host) {
     return ctx->sm_count * copy_vector_ctas_per_sm();
 }
 
-int launch_copy(eakv_ctx* ctx, const int2* d_entries, int64_t n, char* tier_base, bool to_tier,
-                bool touches_host, bool packed, cudaStream_t stream) {
+// d_entries == NULL: the n (<= kCopyInlineEntries) entries at h_inline ride in the parameters
+int launch_copy(eakv_ctx* ctx, const int2* d_entries, const int2* h_inline, int64_t n,
+                char* tier_base, bool to_tier, bool touches_host, bool packed, cudaStream_t stream) {
     CopyLaunch L;
     L.entries = d_entries;
+    if (!d_entries) std::memcpy(L.inline_entries, h_inline, (size_t)n * sizeof(int2));
     L.n_entries = n;
     L.kv_base = ctx->d_kv_base;
     L.tier_base = tier_base;
     L.pieces = ctx->pieces;
     L.piece_bytes = ctx->piece_bytes;
     L.slot_from_index = packed ? 1 : 0;
+    L.gpu_blocks = ctx->cfg.gpu_blocks;
+    L.tier_slots = packed ? ctx->staging_blocks : ctx->cfg.host_blocks;
+    L.error_flag = ctx->d_error_flag;
     L.subs_per_piece = (int32_t)((ctx->piece_bytes + kCopySubBytes - 1) / kCopySubBytes);
     cudaError_t e;
     // bulk async copies serve device-resident buffers; a mapped host tier is always driven
     // by the vector kernel (few CTAs, plain loads/stores over the link)
     if (ctx->cfg.copy_path == EAKV_COPY_BULK && !touches_host)
-        e = launch_copy_bulk(L, to_tier, copy_ctas(ctx, touches_host), ctx->d_error_flag, stream);
+        e = launch_copy_bulk(L, to_tier, copy_ctas(ctx, touches_host), stream);
     else
         e = launch_copy_vector(L, to_tier, copy_ctas(ctx, touches_host), stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "copy kernel launch");
@@ -226,6 +232,91 @@ int for_slot_runs(const int2* e, int64_t n, F f) {
         int rc = f(i0, i1);
         if (rc != EAKV_OK) return rc;
         i0 = i1;
+    }
+    return EAKV_OK;
+}
+
+
+// Move the m compacted entries {pool block, tier slot} between pool and tier.
+//   direct : the copy kernel addresses the tier itself (HBM tier, or mapped host tier)
+//   staged : HBM staging buffers + copy engine on the side stream, double-buffered
+// Under EAKV_LINK_STAGED a call whose slots are so scattered that the copy engine would get
+// mostly single-block copies goes direct instead (per-copy overhead outweighs the DMA's edge).
+int move_blocks(eakv_ctx* ctx, const std::vector<int2>& ent, bool to_tier, cudaStream_t stream) {
+    const int64_t m = (int64_t)ent.size();
+    const bool host_tier = ctx->cfg.tier_location == EAKV_TIER_PINNED_HOST;
+    bool direct = ctx->cfg.link_strategy == EAKV_LINK_ZERO_COPY;
+    if (!direct) {
+        int64_t runs = 0;
+        for_slot_runs(ent.data(), m, [&](int64_t, int64_t) { ++runs; return EAKV_OK; });
+        const int64_t avg_run_bytes = m * ctx->block_bytes / runs;
+        direct = avg_run_bytes < ctx->min_staged_run_bytes;
+    }
+    Staging& S = to_tier ? ctx->st_store : ctx->st_load;
+    if (!direct && !to_tier) {
+        // the side stream may read the tier only after what precedes this call on `stream`
+        CU(cudaEventRecord(S.start, stream));
+        CU(cudaStreamWaitEvent(S.side, S.start, 0));
+    }
+    for (int64_t base = 0; base < m; base += ctx->max_call_blocks) {
+        const int64_t n = std::min(ctx->max_call_blocks, m - base);
+        const int2* h = ent.data() + base;
+        // small calls carry their entries in the kernel parameters: no upload, no ring slot
+        const bool inline_args = n <= kCopyInlineEntries;
+        RingSlot* rs = nullptr;
+        const int2* d = nullptr;
+        int rc = EAKV_OK;
+        if (!inline_args) {
+            rc = ring_upload(ctx, h, n, stream, &rs, &d);
+            if (rc != EAKV_OK) return rc;
+        }
+        if (direct) {
+            rc = launch_copy(ctx, d, h, n, ctx->tier, to_tier, host_tier, false, stream);
+            if (rc != EAKV_OK) return rc;
+        } else {
+            for (int64_t i = 0; i < n; i += ctx->staging_blocks) {
+                const int64_t cur = std::min(ctx->staging_blocks, n - i);
+                const int sb = S.next;
+                S.next ^= 1;
+                const int2* e = h + i;
+                auto dma = [&](int64_t a, int64_t z) {
+                    char* tier_p = ctx->tier + (int64_t)e[a].y * ctx->block_bytes;
+                    char* stage_p = S.buf[sb] + a * ctx->block_bytes;
+                    CU(cudaMemcpyAsync(to_tier ? tier_p : stage_p, to_tier ? stage_p : tier_p,
+                                       (size_t)(z - a) * ctx->block_bytes, cudaMemcpyDefault, S.side));
+                    ctx->stats.memcpy_calls += 1;
+                    return EAKV_OK;
+                };
+                if (to_tier) {
+                    CU(cudaStreamWaitEvent(stream, S.freed[sb], 0));
+                    rc = launch_copy(ctx, d ? d + i : nullptr, e, cur, S.buf[sb], true, false, true, stream);
+                    if (rc != EAKV_OK) return rc;
+                    CU(cudaEventRecord(S.ready[sb], stream));
+                    CU(cudaStreamWaitEvent(S.side, S.ready[sb], 0));
+                    rc = for_slot_runs(e, cur, dma);
+                    if (rc != EAKV_OK) return rc;
+                    CU(cudaEventRecord(S.freed[sb], S.side));
+                } else {
+                    CU(cudaStreamWaitEvent(S.side, S.freed[sb], 0));
+                    rc = for_slot_runs(e, cur, dma);
+                    if (rc != EAKV_OK) return rc;
+                    CU(cudaEventRecord(S.ready[sb], S.side));
+                    CU(cudaStreamWaitEvent(stream, S.ready[sb], 0));
+                    rc = launch_copy(ctx, d ? d + i : nullptr, e, cur, S.buf[sb], false, false, true, stream);
+                    if (rc != EAKV_OK) return rc;
+                    CU(cudaEventRecord(S.freed[sb], stream));
+                }
+            }
+            if (to_tier) {
+                // the call's work is complete, in stream order, once both buffers are drained
+                CU(cudaStreamWaitEvent(stream, S.freed[0], 0));
+                CU(cudaStreamWaitEvent(stream, S.freed[1], 0));
+            }
+        }
+        if (rs) {
+            rc = ring_release(ctx, rs, stream);
+            if (rc != EAKV_OK) return rc;
+        }
     }
     return EAKV_OK;
 }
@@ -288,6 +379,8 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
     ctx->max_call_blocks = cfg->max_call_blocks > 0 ? cfg->max_call_blocks : 16384;
     ctx->hash_scratch_blocks = cfg->hash_scratch_blocks > 0 ? cfg->hash_scratch_blocks : (1 << 20);
     ctx->max_prompts = ctx->max_call_blocks;
+    ctx->min_staged_run_bytes = cfg->min_staged_run_bytes >= 0 ? cfg->min_staged_run_bytes : 0;
+    if (cfg->min_staged_run_bytes == 0) ctx->min_staged_run_bytes = 3ll << 20;
 
 #define CUC(call)                                             \
     do {                                                      \
@@ -386,9 +479,13 @@ int eakv_sync(eakv_ctx* ctx) {
     CU(cudaDeviceSynchronize());
     int flag = 0;
     CU(cudaMemcpy(&flag, ctx->d_error_flag, sizeof(int), cudaMemcpyDeviceToHost));
-    if (flag != 0) {   // a bounded wait in the bulk-copy kernel gave up
+    if (flag != 0) {   // a device-side self-check tripped since the last sync
         CU(cudaMemset(ctx->d_error_flag, 0, sizeof(int)));
-        return EAKV_E_TIMEOUT;
+        CU(cudaMemset(ctx->d_counters, 0, (size_t)ctx->max_prompts * sizeof(int)));
+        ctx->cuda_err = flag == kErrBulkTimeout ? "bulk-copy wait gave up"
+                      : flag == kErrCopyRange ? "copy kernel: entry out of range (skipped)"
+                      : "hash kernel: tile out of range (skipped)";
+        return flag == kErrBulkTimeout ? EAKV_E_TIMEOUT : EAKV_E_RANGE;
     }
     return EAKV_OK;
 }
@@ -437,6 +534,9 @@ int eakv_hash_blocks(eakv_ctx* ctx, const int32_t* tokens_dev, int64_t n_tokens,
         L.single_parent_ptr = done ? hashes_dev + done - 1 : nullptr;
         L.block_size = b;
         L.tile_blocks = tile_blocks;
+        L.tokens_limit = n_tokens - done * b;
+        L.blocks_limit = cur;
+        L.error_flag = ctx->d_error_flag;
         const int n_tiles = (int)((cur + tile_blocks - 1) / tile_blocks);
         const bool piece_vec = vec && (((done * b) & 3) == 0);
         cudaError_t e = launch_hash(L, n_tiles, generic, piece_vec, stream);
@@ -524,6 +624,9 @@ int eakv_hash_blocks_batched(eakv_ctx* ctx, const int32_t* tokens_dev,
     L.single_parent_ptr = nullptr;
     L.block_size = b;
     L.tile_blocks = tile_blocks;
+    L.tokens_limit = offsets_host[n_prompts];
+    L.blocks_limit = total_blocks;
+    L.error_flag = ctx->d_error_flag;
     cudaError_t e = launch_hash(L, (int)n_tiles, generic, vec, stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "hash kernel launch");
     ctx->stats.kernel_launches += 1;
@@ -680,48 +783,8 @@ int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_m
     if (m == 0) return EAKV_OK;
     DeviceGuard g(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const bool host_tier = ctx->cfg.tier_location == EAKV_TIER_PINNED_HOST;
-
-    // one argument upload per max_call_blocks entries; the staged strategy walks each upload
-    // in staging-buffer-sized chunks
-    for (int64_t base = 0; base < m; base += ctx->max_call_blocks) {
-        const int64_t n = std::min(ctx->max_call_blocks, m - base);
-        RingSlot* rs = nullptr;
-        const int2* d = nullptr;
-        int rc = ring_upload(ctx, ent.data() + base, n, stream, &rs, &d);
-        if (rc != EAKV_OK) return rc;
-        if (ctx->cfg.link_strategy == EAKV_LINK_ZERO_COPY) {
-            rc = launch_copy(ctx, d, n, ctx->tier, true, host_tier, false, stream);
-            if (rc != EAKV_OK) return rc;
-        } else {
-            Staging& S = ctx->st_store;
-            for (int64_t i = 0; i < n; i += ctx->staging_blocks) {
-                const int64_t cur = std::min(ctx->staging_blocks, n - i);
-                const int sb = S.next;
-                S.next ^= 1;
-                CU(cudaStreamWaitEvent(stream, S.freed[sb], 0));
-                rc = launch_copy(ctx, d + i, cur, S.buf[sb], true, false, true, stream);
-                if (rc != EAKV_OK) return rc;
-                CU(cudaEventRecord(S.ready[sb], stream));
-                CU(cudaStreamWaitEvent(S.side, S.ready[sb], 0));
-                const int2* e = ent.data() + base + i;
-                rc = for_slot_runs(e, cur, [&](int64_t a, int64_t z) {
-                    CU(cudaMemcpyAsync(ctx->tier + (int64_t)e[a].y * ctx->block_bytes,
-                                       S.buf[sb] + a * ctx->block_bytes,
-                                       (size_t)(z - a) * ctx->block_bytes, cudaMemcpyDefault, S.side));
-                    ctx->stats.memcpy_calls += 1;
-                    return EAKV_OK;
-                });
-                if (rc != EAKV_OK) return rc;
-                CU(cudaEventRecord(S.freed[sb], S.side));
-            }
-            // the call's work is complete, in stream order, once both buffers are drained
-            CU(cudaStreamWaitEvent(stream, S.freed[0], 0));
-            CU(cudaStreamWaitEvent(stream, S.freed[1], 0));
-        }
-        rc = ring_release(ctx, rs, stream);
-        if (rc != EAKV_OK) return rc;
-    }
+    int rc = move_blocks(ctx, ent, true, stream);
+    if (rc != EAKV_OK) return rc;
     ctx->stats.blocks_stored += m;
     ctx->stats.bytes_stored += m * ctx->block_bytes;
     return EAKV_OK;
@@ -746,48 +809,8 @@ int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_tab
     const int64_t m = n_blocks;
     DeviceGuard g(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const bool host_tier = ctx->cfg.tier_location == EAKV_TIER_PINNED_HOST;
-
-    if (ctx->cfg.link_strategy == EAKV_LINK_STAGED) {
-        // the side stream may read the tier only after what precedes this call on `stream`
-        CU(cudaEventRecord(ctx->st_load.start, stream));
-        CU(cudaStreamWaitEvent(ctx->st_load.side, ctx->st_load.start, 0));
-    }
-    for (int64_t base = 0; base < m; base += ctx->max_call_blocks) {
-        const int64_t n = std::min(ctx->max_call_blocks, m - base);
-        RingSlot* rs = nullptr;
-        const int2* d = nullptr;
-        int rc = ring_upload(ctx, ent.data() + base, n, stream, &rs, &d);
-        if (rc != EAKV_OK) return rc;
-        if (ctx->cfg.link_strategy == EAKV_LINK_ZERO_COPY) {
-            rc = launch_copy(ctx, d, n, ctx->tier, false, host_tier, false, stream);
-            if (rc != EAKV_OK) return rc;
-        } else {
-            Staging& S = ctx->st_load;
-            for (int64_t i = 0; i < n; i += ctx->staging_blocks) {
-                const int64_t cur = std::min(ctx->staging_blocks, n - i);
-                const int sb = S.next;
-                S.next ^= 1;
-                CU(cudaStreamWaitEvent(S.side, S.freed[sb], 0));
-                const int2* e = ent.data() + base + i;
-                rc = for_slot_runs(e, cur, [&](int64_t a, int64_t z) {
-                    CU(cudaMemcpyAsync(S.buf[sb] + a * ctx->block_bytes,
-                                       ctx->tier + (int64_t)e[a].y * ctx->block_bytes,
-                                       (size_t)(z - a) * ctx->block_bytes, cudaMemcpyDefault, S.side));
-                    ctx->stats.memcpy_calls += 1;
-                    return EAKV_OK;
-                });
-                if (rc != EAKV_OK) return rc;
-                CU(cudaEventRecord(S.ready[sb], S.side));
-                CU(cudaStreamWaitEvent(stream, S.ready[sb], 0));
-                rc = launch_copy(ctx, d + i, cur, S.buf[sb], false, false, true, stream);
-                if (rc != EAKV_OK) return rc;
-                CU(cudaEventRecord(S.freed[sb], stream));
-            }
-        }
-        rc = ring_release(ctx, rs, stream);
-        if (rc != EAKV_OK) return rc;
-    }
+    int rc = move_blocks(ctx, ent, false, stream);
+    if (rc != EAKV_OK) return rc;
     ctx->stats.blocks_loaded += m;
     ctx->stats.bytes_loaded += m * ctx->block_bytes;
     return EAKV_OK;

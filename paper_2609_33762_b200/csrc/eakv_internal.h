@@ -11,6 +11,8 @@ constexpr int kHashUnroll = 4;
 constexpr int kHashTileTokens = kHashThreads * kHashUnroll * 4;   // 4096 tokens per CTA tile
 constexpr int kHashMaxBlockSize = 4096;
 constexpr int kHashMaxSmem = 80 * 1024;
+// staged kernel: limb table + two stages of 256 padded rows at the largest thread-per-block size (64)
+constexpr int kHashStagedMaxSmem = 64 * 16 + 2 * kHashThreads * (4 * 64 + 16);
 
 struct HashTile { int32_t prompt; int32_t first_block; };
 struct HashPrompt {
@@ -34,6 +36,10 @@ struct HashLaunch {
     const uint64_t* single_parent_ptr;   // non-NULL: read the parent from device memory instead
     int32_t block_size;
     int32_t tile_blocks;
+    // self-check limits: a CTA whose tile would reach past them raises *error_flag and skips
+    int64_t tokens_limit;           // tokens readable at `tokens`
+    int64_t blocks_limit;           // entries writable at `keys` and `partial`
+    int* error_flag;
 };
 // one thread per block for small or odd block sizes, a group of threads per block otherwise
 inline bool hash_thread_per_block(int block_size) { return (block_size % 4) != 0 || block_size <= 64; }
@@ -56,8 +62,10 @@ constexpr int kCopyThreads = 256;
 constexpr int kCopyUnroll = 4;
 constexpr int kCopySubBytes = kCopyThreads * kCopyUnroll * 16;    // 16 KiB per CTA work item
 
+constexpr int kCopyInlineEntries = 32;   // small calls carry their entries in the kernel parameters
+
 struct CopyLaunch {
-    const int2* entries;        // {pool block id, tier slot (or staging index)}
+    const int2* entries;        // {pool block id, tier slot (or staging index)}; NULL: use inline_entries
     int64_t n_entries;
     void* const* kv_base;       // device array of 2L piece-array base pointers
     char* tier_base;            // slot-major destination/source
@@ -65,11 +73,17 @@ struct CopyLaunch {
     int32_t subs_per_piece;     // ceil(piece_bytes / kCopySubBytes)
     int32_t slot_from_index;    // 1: entry j uses slot j (packed staging buffer) instead of entries[j].y
     int64_t piece_bytes;
+    // self-check limits: an entry outside them raises *error_flag and is skipped
+    int64_t gpu_blocks;
+    int64_t tier_slots;
+    int* error_flag;
+    int2 inline_entries[kCopyInlineEntries];
 };
+// values written to the error flag
+constexpr int kErrBulkTimeout = 1, kErrCopyRange = 2, kErrHashRange = 3;
 // to_tier: pool -> tier (store/gather); else tier -> pool (load/scatter)
 cudaError_t launch_copy_vector(const CopyLaunch& L, bool to_tier, int ctas, cudaStream_t stream);
-cudaError_t launch_copy_bulk(const CopyLaunch& L, bool to_tier, int ctas, int* error_flag,
-                             cudaStream_t stream);
+cudaError_t launch_copy_bulk(const CopyLaunch& L, bool to_tier, int ctas, cudaStream_t stream);
 cudaError_t copy_kernels_init();
 int copy_vector_ctas_per_sm();
 

@@ -76,7 +76,7 @@ __device__ __noinline__ void scan_prompt(const uint64_t* partial, uint64_t* keys
     const int64_t per = (nblk + nthr - 1) / nthr;
     const int64_t lo = min((int64_t)tid * per, nblk), hi = min(lo + per, nblk);
     // fold this thread's run (kept in registers when short, so the loads overlap)
-    constexpr int kRegRun = 8;
+    constexpr int kRegRun = 16;
     uint64_t run[kRegRun];
     const bool in_regs = per <= kRegRun;
     if (in_regs) {
@@ -87,10 +87,13 @@ __device__ __noinline__ void scan_prompt(const uint64_t* partial, uint64_t* keys
     if (in_regs) {
 #pragma unroll
         for (int i = 0; i < kRegRun; ++i) {
-            if (lo + i < hi) {
-                mine.a = mulmod61(mine.a, A);
-                mine.c = addmod61(mulmod61(mine.c, A), run[i]);
-            }
+            if (lo + i < hi) mine.c = addmod61(mulmod61(mine.c, A), run[i]);
+        }
+        // the run's multiplier is A^(hi-lo): square-and-multiply instead of one product per block
+        uint64_t sq = A;
+        for (int64_t n = hi - lo; n; n >>= 1) {
+            if (n & 1) mine.a = mulmod61(mine.a, sq);
+            sq = mulmod61(sq, sq);
         }
     } else {
         for (int64_t j = lo; j < hi; ++j) {
@@ -176,6 +179,14 @@ hash_blocks_kernel(HashLaunch L) {
         parent = *L.single_parent_ptr;
     }
     const int64_t nb_tile = min((int64_t)L.tile_blocks, nblk - first_blk);
+    {   // self-check: the tile must lie inside the buffers the caller described
+        const int64_t last_blk = blk0 + first_blk + nb_tile;
+        const int64_t last_tok = tok0 + (first_blk + nb_tile) * (int64_t)L.block_size;
+        if (nb_tile <= 0 || last_blk > L.blocks_limit || last_tok > L.tokens_limit || p < 0) {
+            if (threadIdx.x == 0) atomicExch(L.error_flag, kErrHashRange);
+            return;
+        }
+    }
     const int cpb = L.block_size >> 2;                                // chunks per block
     const int n_chunks = (int)nb_tile * cpb;
     const int32_t* tok = L.tokens + tok0 + first_blk * L.block_size;
@@ -284,6 +295,14 @@ hash_blocks_tpb_kernel(HashLaunch L) {
         parent = *L.single_parent_ptr;
     }
     const int64_t nb_tile = min((int64_t)L.tile_blocks, nblk - first_blk);
+    {   // self-check: the tile must lie inside the buffers the caller described
+        const int64_t last_blk = blk0 + first_blk + nb_tile;
+        const int64_t last_tok = tok0 + (first_blk + nb_tile) * (int64_t)L.block_size;
+        if (nb_tile <= 0 || last_blk > L.blocks_limit || last_tok > L.tokens_limit || p < 0) {
+            if (threadIdx.x == 0) atomicExch(L.error_flag, kErrHashRange);
+            return;
+        }
+    }
     __syncthreads();
     uint64_t* partial = L.partial + blk0;
     for (int64_t j = tid; j < nb_tile; j += blockDim.x) {
@@ -321,13 +340,130 @@ hash_blocks_tpb_kernel(HashLaunch L) {
 }
 #undef EAKV_MAC3
 
+// Staged thread-per-block variant for 16-byte-aligned tokens and b % 4 == 0: the tile's
+// tokens are brought into shared memory with fully coalesced 16-byte async copies (two
+// sub-tiles of 256 blocks in flight), in rows padded by 16 bytes so that the per-thread row
+// reads are bank-conflict free; the arithmetic is the same three-limb multiply-add.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(d), "l"(gmem_src) : "memory");
+}
+
+#define EAKV_MAC3(tok, e)                                   \
+    do {                                                    \
+        const uint32_t x_ = (uint32_t)(tok) + 1u;           \
+        const uint4 w_ = pw3[(e)];                          \
+        s0 += (uint64_t)x_ * w_.x;                          \
+        s1 += (uint64_t)x_ * w_.y;                          \
+        s2 += (uint64_t)x_ * w_.z;                          \
+    } while (0)
+
+__global__ void __launch_bounds__(kHashThreads)
+hash_blocks_staged_kernel(HashLaunch L) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ Pair warp_tot[32];
+    __shared__ int is_last;
+    const int tid = threadIdx.x;
+    const int b = L.block_size, cpb = b >> 2;
+    const int row_bytes = 4 * b + 16;
+    uint4* pw3 = reinterpret_cast<uint4*>(smem_raw);
+    unsigned char* const stage0 = smem_raw + (size_t)b * 16;
+    const size_t stage_bytes = (size_t)kHashThreads * row_bytes;
+    int32_t p = 0;
+    int64_t first_blk = (int64_t)blockIdx.x * L.tile_blocks;
+    int64_t tok0 = 0, blk0 = 0, nblk = L.single_nblk;
+    uint64_t parent = L.single_parent;
+    int32_t tiles_in_prompt = gridDim.x;
+    if (L.tiles != nullptr) {
+        const HashTile t = L.tiles[blockIdx.x];
+        p = t.prompt;
+        first_blk = t.first_block;
+        const HashPrompt hp = L.prompts[p];
+        tok0 = hp.tok_off; blk0 = hp.blk_off; nblk = hp.nblk; parent = hp.parent;
+        tiles_in_prompt = hp.tiles;
+    } else if (L.single_parent_ptr != nullptr) {
+        parent = *L.single_parent_ptr;
+    }
+    const int nb_tile = (int)min((int64_t)L.tile_blocks, nblk - first_blk);
+    {   // self-check: the tile must lie inside the buffers the caller described
+        const int64_t last_blk = blk0 + first_blk + nb_tile;
+        const int64_t last_tok = tok0 + (first_blk + nb_tile) * (int64_t)L.block_size;
+        if (nb_tile <= 0 || last_blk > L.blocks_limit || last_tok > L.tokens_limit || p < 0) {
+            if (threadIdx.x == 0) atomicExch(L.error_flag, kErrHashRange);
+            return;
+        }
+    }
+    const int n_sub = (nb_tile + kHashThreads - 1) / kHashThreads;
+    const int4* tile_src = reinterpret_cast<const int4*>(L.tokens + tok0 + first_blk * b);
+
+    auto issue = [&](int r) {
+        const int nb = min(kHashThreads, nb_tile - r * kHashThreads);
+        const int chunks = nb * cpb;
+        const int4* src = tile_src + (size_t)r * kHashThreads * cpb;
+        unsigned char* st = stage0 + (r & 1) * stage_bytes;
+        for (int c = tid; c < chunks; c += kHashThreads) {
+            const int row = c / cpb, col = c - row * cpb;
+            cp_async16(st + (size_t)row * row_bytes + col * 16, src + c);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+
+    issue(0);
+    for (int e = tid; e < b; e += blockDim.x) {
+        const uint64_t w = L.pow_table[e];
+        pw3[e] = make_uint4((uint32_t)(w & 0x1FFFFF), (uint32_t)((w >> 21) & 0x1FFFFF),
+                            (uint32_t)(w >> 42), 0u);
+    }
+    uint64_t* partial = L.partial + blk0;
+    for (int r = 0; r < n_sub; ++r) {
+        if (r + 1 < n_sub) {
+            issue(r + 1);
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+        } else {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        }
+        __syncthreads();
+        const int j = r * kHashThreads + tid;
+        if (j < nb_tile) {
+            const int4* row = reinterpret_cast<const int4*>(stage0 + (r & 1) * stage_bytes + (size_t)tid * row_bytes);
+            uint64_t acc = 0;
+            for (int k0 = 0; k0 < b; k0 += kLimbFoldTokens) {
+                const int k1 = min(b, k0 + kLimbFoldTokens);
+                uint64_t s0 = 0, s1 = 0, s2 = 0;
+#pragma unroll 4
+                for (int k = k0; k < k1; k += 4) {
+                    const int4 u = row[k >> 2];
+                    const int e = b - 1 - k;
+                    EAKV_MAC3(u.x, e); EAKV_MAC3(u.y, e - 1); EAKV_MAC3(u.z, e - 2); EAKV_MAC3(u.w, e - 3);
+                }
+                acc = addmod61(acc, fold_limb_sums(s0, s1, s2));
+            }
+            __stcg(partial + first_blk + j, acc);
+        }
+        __syncthreads();     // the stage is refilled two iterations from now
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int ticket = atomicAdd(L.counters + p, 1);
+        is_last = (ticket == tiles_in_prompt - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    scan_prompt(partial, L.keys + blk0, nblk, parent, L.pow_table[b], warp_tot);
+    if (tid == 0) L.counters[p] = 0;
+}
+#undef EAKV_MAC3
+
 // thread_per_block: see hash_thread_per_block(); vec: 16-byte token loads are allowed
 cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool thread_per_block, bool vec,
                         cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
     if (thread_per_block) {
         const size_t smem = (size_t)L.block_size * sizeof(uint4);
-        if (vec) hash_blocks_tpb_kernel<true><<<n_tiles, kHashThreads, smem, stream>>>(L);
+        const size_t staged = smem + 2 * (size_t)kHashThreads * (4 * L.block_size + 16);
+        if (vec) hash_blocks_staged_kernel<<<n_tiles, kHashThreads, staged, stream>>>(L);
         else     hash_blocks_tpb_kernel<false><<<n_tiles, kHashThreads, smem, stream>>>(L);
     } else {
         const size_t smem = (size_t)(L.block_size + 1) * 8 +
@@ -346,8 +482,8 @@ cudaError_t hash_kernels_init() {
     e = cudaFuncSetAttribute(hash_blocks_kernel<false>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, kHashMaxSmem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(hash_blocks_tpb_kernel<true>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, kHashMaxSmem);
+    e = cudaFuncSetAttribute(hash_blocks_staged_kernel,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kHashStagedMaxSmem);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(hash_blocks_tpb_kernel<false>,
                                 cudaFuncAttributeMaxDynamicSharedMemorySize, kHashMaxSmem);
@@ -461,6 +597,9 @@ extern "C" int eakv_hash_blocks_static(const int32_t* tokens_dev, int64_t n_toke
     L.single_parent_ptr = nullptr;
     L.block_size = block_size;
     L.tile_blocks = hash_tile_blocks(block_size, nblk);
+    L.tokens_limit = n_tokens;
+    L.blocks_limit = nblk;
+    L.error_flag = reinterpret_cast<int*>(scratch + kStaticPartialBytes + kStaticPowBytes) + 1;
     const int n_tiles = (int)((nblk + L.tile_blocks - 1) / L.tile_blocks);
     if (launch_hash(L, n_tiles, generic, vec, stream) != cudaSuccess) return EAKV_E_CUDA;
     return EAKV_OK;

@@ -40,7 +40,8 @@ class Config(C.Structure):
         ("link_strategy", C.c_int32), ("tier_location", C.c_int32), ("copy_path", C.c_int32),
         ("copy_ctas", C.c_int32),
         ("staging_bytes", C.c_int64), ("max_call_blocks", C.c_int64),
-        ("hash_scratch_blocks", C.c_int64), ("tier_memory", C.c_void_p),
+        ("hash_scratch_blocks", C.c_int64), ("min_staged_run_bytes", C.c_int64),
+        ("tier_memory", C.c_void_p),
     ]
 
 
@@ -142,7 +143,8 @@ class Context:
                  policy=POLICY_WRITE_ALL, kappa_blocks=8, theta_percent=95, len_window=256,
                  window_ms=60_000, telemetry=1, link_strategy=LINK_STAGED,
                  tier_location=TIER_PINNED_HOST, copy_path=COPY_BULK, copy_ctas=0,
-                 staging_bytes=0, max_call_blocks=0, hash_scratch_blocks=0, tier_memory=0):
+                 staging_bytes=0, max_call_blocks=0, hash_scratch_blocks=0, min_staged_run_bytes=0,
+                 tier_memory=0):
         L = lib()
         cfg = Config()
         L.eakv_config_init(C.byref(cfg))
@@ -160,6 +162,7 @@ class Context:
         cfg.copy_path, cfg.copy_ctas = copy_path, copy_ctas
         cfg.staging_bytes, cfg.max_call_blocks = staging_bytes, max_call_blocks
         cfg.hash_scratch_blocks = hash_scratch_blocks
+        cfg.min_staged_run_bytes = min_staged_run_bytes
         cfg.tier_memory = int(tier_memory) if tier_memory else None
         self._h = C.c_void_p()
         rc = L.eakv_create(C.byref(cfg), C.byref(self._h))

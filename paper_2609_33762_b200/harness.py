@@ -64,12 +64,39 @@ class AgentServer:
         self.b = shape.block_size
         self.seed = self.ctx.eakv_hash_seed()
         self._agent_keys = {}          # agent -> np.uint64 keys of its previous prompt
+        self._timed = {"load": [], "store": []}     # (bytes, start event, end event)
         self.records = []
         self.totals = dict(prompt_tokens=0, fresh_tokens=0, loaded_blocks=0, stored_blocks=0,
                            gpu_hit_blocks=0, host_hit_blocks=0)
 
     def close(self):
         self.ctx.close()
+
+    def _time(self, kind, nbytes):
+        """Context manager bracketing one store/load call with CUDA events on its stream."""
+        server = self
+
+        class _T:
+            def __enter__(self_t):
+                self_t.e0 = torch.cuda.Event(enable_timing=True)
+                self_t.e1 = torch.cuda.Event(enable_timing=True)
+                self_t.e0.record(server.stream)
+
+            def __exit__(self_t, *exc):
+                self_t.e1.record(server.stream)
+                server._timed[kind].append((nbytes, self_t.e0, self_t.e1))
+        return _T()
+
+    def transfer_rates(self):
+        """GB/s of the store and load calls so far (device time between the events that
+        bracket each call); call after a synchronize."""
+        out = {}
+        for kind, items in self._timed.items():
+            nbytes = sum(b for b, _, _ in items)
+            ms = sum(e0.elapsed_time(e1) for _, e0, e1 in items)
+            out[kind] = {"calls": len(items), "gib": nbytes / (1 << 30),
+                         "gb_per_s": nbytes / (ms * 1e-3) / 1e9 if ms > 0 else None}
+        return out
 
     def _ensure_pinned(self, n_tokens):
         if getattr(self, "_tok_pin", None) is None or self._tok_pin.numel() < n_tokens:
@@ -115,7 +142,8 @@ class AgentServer:
         cover = max(G, H)
         lo, hi = (G, H) if H > G else (G, G)
         if hi > lo and self.data_plane:
-            self.ctx.eakv_load(host_slots[lo:hi], blocks[lo:hi], self.stream)
+            with self._time("load", (hi - lo) * self.ctx.block_bytes):
+                self.ctx.eakv_load(host_slots[lo:hi], blocks[lo:hi], self.stream)
         fill = [j for j in range(cover, nblk) if not resident[j]]
         if fill and self.data_plane:
             ids = torch.as_tensor(blocks[fill].astype(np.int64), device=self.device)
@@ -126,7 +154,8 @@ class AgentServer:
                     w = torch.from_numpy(w.view(np.int16)).to(self.device)
                 piece[ids] = w.view(torch.int16)
         if self.data_plane and step["admit"].any():
-            self.ctx.eakv_store(blocks, step["admit"], step["slot"], self.stream)
+            with self._time("store", int(step["admit"].sum()) * self.ctx.block_bytes):
+                self.ctx.eakv_store(blocks, step["admit"], step["slot"], self.stream)
         if tail >= 0:
             self.ctx.eakv_gpu_tier_release(tail)
         rec = dict(agent=agent, now_ms=now_ms, n_tokens=n, keys=keys, G=G, H=H,

@@ -78,6 +78,7 @@ def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=Tru
     server.run(trace, limit=limit)
     torch.cuda.synchronize()
     wall = time.perf_counter() - t0
+    rates = server.transfer_rates() if data_plane else None
     if server_hook is not None:
         server_hook(server, trace)
     st = server.ctx.eakv_get_stats()
@@ -98,7 +99,7 @@ def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=Tru
         "declined_requests": st["declined_requests"], "pressure_requests": st["pressure_requests"],
         "declined_blocks": st["declined"], "evicted_blocks": st["evicted"],
         "tokens_hashed": st["tokens_hashed"], "kernel_launches": st["kernel_launches"],
-        "wall_s": wall, "setup_s": t_setup,
+        "wall_s": wall, "setup_s": t_setup, "transfer_rates": rates,
         "moved_gb_per_s_wall": (tot["loaded_blocks"] + tot["stored_blocks"]) * shape.block_bytes / wall / 1e9
         if data_plane else None,
     }

@@ -75,6 +75,8 @@ def test_full_size_store_load(pool, where):
         kw = dict(tier_location=eakv.TIER_DEVICE, tier_memory=tier_t.data_ptr())
     elif where == "host_zero_copy":
         kw["link_strategy"] = eakv.LINK_ZERO_COPY
+    else:
+        kw["min_staged_run_bytes"] = -1               # random slots, yet through the staging path
     ctx = eakv.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
                        block_size=shape.block_size, gpu_blocks=nb, host_blocks=M,
                        kv_base=pool.kv_base, **kw)

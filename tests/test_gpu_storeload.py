@@ -29,7 +29,13 @@ def variants():
     for link, loc, path in itertools.product((e.LINK_ZERO_COPY, e.LINK_STAGED),
                                              (e.TIER_PINNED_HOST, e.TIER_DEVICE),
                                              (e.COPY_VECTOR, e.COPY_BULK)):
-        out.append(dict(link_strategy=link, tier_location=loc, copy_path=path))
+        kw = dict(link_strategy=link, tier_location=loc, copy_path=path)
+        if link == e.LINK_STAGED:
+            kw["min_staged_run_bytes"] = -1          # always through the staging buffers
+        out.append(kw)
+    # the default: staged, but scattered slots fall back to the direct kernel
+    out.append(dict(link_strategy=e.LINK_STAGED, tier_location=e.TIER_PINNED_HOST,
+                    copy_path=e.COPY_BULK, min_staged_run_bytes=0))
     return out
 
 
@@ -144,7 +150,7 @@ def test_store_load_parity(name, kw):
 def test_llama_shape_multi_item_pieces():
     e = eakv()
     for kw in (dict(copy_path=e.COPY_VECTOR), dict(copy_path=e.COPY_BULK, tier_location=e.TIER_DEVICE),
-               dict(link_strategy=e.LINK_STAGED)):
+               dict(link_strategy=e.LINK_STAGED, min_staged_run_bytes=-1)):
         rig = Rig(SHAPE_CASES["llama"], 12, 10, seed=12, **kw)
         rig.store(np.array([3, 11, 0, 7], np.int32), np.array([1, 1, 0, 1], np.uint8),
                   np.array([9, 0, 5, 4], np.int32))

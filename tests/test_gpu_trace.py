@@ -57,7 +57,8 @@ def test_config0_bit_exact(cfg_name, link):
     oracle = TraceOracle(shape, cfg.gpu_blocks, cfg.host_blocks, payload=payload)
     oracle.run(trace)
     server = AgentServer(shape, cfg.gpu_blocks, cfg.host_blocks, payload, link_strategy=link,
-                         staging_bytes=7 * shape.block_bytes, incremental_hash=(link == 1))
+                         staging_bytes=7 * shape.block_bytes, incremental_hash=(link == 1),
+                         min_staged_run_bytes=-1 if link == 1 else 0)
     server.run(trace)
     compare_records(server.records, oracle.records)
     assert server.totals == oracle.totals
