@@ -3,7 +3,7 @@
 Qwen3-30B-A3B-shaped KV: 48 layers, 4 KV heads, head_dim 128, bf16, block 16).
 
 One step = one pass of the whole path over one batch: two requests of `--blocks` blocks
-each.  Request 1 resubmits the previous step's prompt (its KV is host-resident and gone
+each.  Request 1 resubmits the prompt of two steps ago (its KV is host-resident and gone
 from the GPU): hash -> match -> tier step (all hits) -> load every block into freshly
 drawn, uniform-random pool blocks.  Request 2 is a new prompt: hash -> match (nothing) ->
 tier step (every block admitted, evicting the oldest prompt) -> store from uniform-random
@@ -31,6 +31,11 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+# The request that restores resubmits the prompt stored LAG steps earlier, and the tier holds
+# TIER_PROMPTS prompts, so restores and host writes of neighbouring steps are independent and
+# both directions of the link stay busy (each prompt is still written once and restored once).
+LAG = 2
+TIER_PROMPTS = 3
 METRIC = "kv_store_load_gbps"
 UNIT = "GB/s"
 WORKLOAD = "c1_store_load_microbench_qwen3_30b_a3b"
@@ -156,13 +161,13 @@ class Arm:
                 kw["copy_ctas"] = args.copy_ctas
         else:
             # the tier is a tensor of ours that the context adopts, so it can be inspected
-            self.tier_t = torch.empty((2 * self.m, shape.pieces_per_block, shape.piece_bytes // 2),
+            self.tier_t = torch.empty((TIER_PROMPTS * self.m, shape.pieces_per_block, shape.piece_bytes // 2),
                                       dtype=torch.int16, device=device)
             kw.update(tier_location=eakv.TIER_DEVICE, link_strategy=eakv.LINK_ZERO_COPY,
                       copy_ctas=args.copy_ctas, tier_memory=self.tier_t.data_ptr())
         self.ctx = eakv.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads,
                                 head_dim=shape.head_dim, block_size=shape.block_size,
-                                gpu_blocks=pool.gpu_blocks, host_blocks=2 * self.m,
+                                gpu_blocks=pool.gpu_blocks, host_blocks=TIER_PROMPTS * self.m,
                                 kv_base=pool.kv_base, **kw)
         self.block_bytes = self.ctx.block_bytes
         # lookups (hash, key read-back) run on their own stream so the host control plane of
@@ -171,8 +176,8 @@ class Arm:
         self.hash_stream = torch.cuda.Stream(device)
         self.load_stream = torch.cuda.Stream(device)
         self.store_stream = torch.cuda.Stream(device) if (host_tier and args.overlap) else self.load_stream
-        self.load_done = [torch.cuda.Event(), torch.cuda.Event()]    # by step parity
-        self.store_done = torch.cuda.Event()
+        self.load_done = [torch.cuda.Event() for _ in range(4)]     # by step modulo 4
+        self.store_done = [torch.cuda.Event() for _ in range(4)]
         self.seed = self.ctx.eakv_hash_seed()
         self.keys_dev = torch.empty(self.m, dtype=torch.int64, device=device)
         self.keys_host = torch.empty(self.m, dtype=torch.int64).pin_memory()
@@ -202,22 +207,23 @@ class Arm:
         moved = 0
         if H > 0:
             ls = self.load_stream
-            ls.wait_event(self.store_done)      # the slots being read were written by a store
+            # the slots being read were written by the store of LAG steps ago
+            ls.wait_event(self.store_done[(step_idx - LAG) % 4])
             ev = self._timer(ls, timed_events)
             self.ctx.eakv_load(slots[:H], table[:H], ls)
             self._timer_end(ls, ev, H * self.block_bytes, timed_events)
-            self.load_done[step_idx % 2].record(ls)
+            self.load_done[step_idx % 4].record(ls)
             moved += H * self.block_bytes
             self.h2d += H * self.block_bytes if self.host_tier else 0
         n_admit = int(step["admit"].sum())
         if n_admit:
             ss = self.store_stream
             # the slots this store overwrites held the prompt the previous step restored
-            ss.wait_event(self.load_done[(step_idx - 1) % 2])
+            ss.wait_event(self.load_done[(step_idx - 1) % 4])
             ev = self._timer(ss, timed_events)
             self.ctx.eakv_store(table, step["admit"], step["slot"], ss)
             self._timer_end(ss, ev, n_admit * self.block_bytes, timed_events)
-            self.store_done.record(ss)
+            self.store_done[step_idx % 4].record(ss)
             moved += n_admit * self.block_bytes
             self.d2h += n_admit * self.block_bytes if self.host_tier else 0
         return moved, H, n_admit
@@ -235,12 +241,12 @@ class Arm:
             timed_events.append((nbytes, ev))
 
     def step(self, s, prompts, tables, timed_events=None):
-        """prompts[s-1] was stored by the previous step; prompts[s] is new.  The two requests
-        use disjoint, freshly drawn pool blocks."""
+        """prompts[s-LAG] was stored LAG steps ago; prompts[s] is new.  The two requests use
+        disjoint, freshly drawn pool blocks."""
         m = self.m
-        a, _, _ = self.request(prompts[s - 1], tables[s][:m], agent=(s - 1) % 2, now=s * 1000,
+        a, _, _ = self.request(prompts[s - LAG], tables[s][:m], agent=(s - LAG) % 4, now=s * 1000,
                                timed_events=timed_events, step_idx=s)
-        b, _, _ = self.request(prompts[s], tables[s][m:], agent=s % 2, now=s * 1000 + 500,
+        b, _, _ = self.request(prompts[s], tables[s][m:], agent=s % 4, now=s * 1000 + 500,
                                timed_events=timed_events, step_idx=s)
         return a + b
 
@@ -250,9 +256,10 @@ def run_arm(arm, prompts, tables, steps, warmup, dist, clocks=None, time_kernels
     main = torch.cuda.current_stream(arm.device)
     if clocks:
         clocks.start()
-    # prime: store prompt 0 so that step 1 has something to restore
-    arm.request(prompts[0], tables[0][arm.m:], agent=0, now=0)
-    for s in range(1, warmup + 1):
+    # prime: store the first LAG prompts so that the first step has something to restore
+    for s in range(LAG):
+        arm.request(prompts[s], tables[s][arm.m:], agent=s % 4, now=0, step_idx=s)
+    for s in range(LAG, warmup + LAG):
         arm.step(s, prompts, tables)
     torch.cuda.synchronize()
     if dist is not None:
@@ -266,7 +273,7 @@ def run_arm(arm, prompts, tables, steps, warmup, dist, clocks=None, time_kernels
     for st in arm.streams():
         st.wait_stream(main)
     moved = 0
-    for s in range(warmup + 1, warmup + 1 + steps):
+    for s in range(warmup + LAG, warmup + LAG + steps):
         moved += arm.step(s, prompts, tables, timed_events=timed)
     for st in arm.streams():
         main.wait_stream(st)
@@ -452,7 +459,7 @@ def main():
 
     # paged pool, as large as fits (200k blocks = 293 GiB do not fit one GPU)
     free, _total = torch.cuda.mem_get_info(device)
-    reserve = 2 * m * shape.block_bytes + (4 << 30) + 2 * (args.staging_mib << 20) * 2
+    reserve = TIER_PROMPTS * m * shape.block_bytes + (4 << 30) + 2 * (args.staging_mib << 20) * 2
     nb = min(args.pool_blocks, int((free - reserve) // shape.block_bytes))
     nb = max(nb, 2 * m)
     pool = PagedPool(shape, nb, device, fill=lambda q, t: t.random_())
@@ -468,13 +475,17 @@ def main():
                                                   prompts=args.hash_prompts)}))
         return
 
-    total_steps = args.steps + args.warmup + 1
+    total_steps = args.steps + args.warmup + LAG
     rng = np.random.default_rng(1 + rank)
     tok_np = rng.integers(0, 151936, size=(total_steps + 1, m * shape.block_size), dtype=np.int32)
     prompts_dev = [torch.from_numpy(tok_np[i]).to(device) for i in range(total_steps + 1)]
     prompts_host = [torch.from_numpy(tok_np[i]).pin_memory() for i in range(total_steps + 1)]
     # fresh uniform-random block ids per request, without replacement
-    tables = [rng.permutation(nb)[:2 * m].astype(np.int32) for _ in range(total_steps + 1)]
+    # uniform-random block ids without replacement: consecutive steps take disjoint windows of
+    # one random permutation of the pool, so transfers of neighbouring steps never share a block
+    perm = rng.permutation(nb).astype(np.int32)
+    windows = nb // (2 * m)
+    tables = [perm[(i % windows) * 2 * m:(i % windows + 1) * 2 * m] for i in range(total_steps + 1)]
 
     clocks = ClockSampler(local_rank) if rank == 0 else None
 
@@ -557,7 +568,7 @@ def main():
 
 def self_check(torch, arm, pool, tables, args, shape):
     """After the timed region: the last stored prompt's slots must equal its pool blocks."""
-    s = args.warmup + args.steps
+    s = args.warmup + args.steps + LAG - 1
     table = tables[s][args.blocks:]
     keys = arm.keys_host.numpy().view(np.uint64)         # keys of the last request
     _, H, _, slots = arm.ctx.eakv_match(keys)

@@ -52,6 +52,27 @@ copy_blocks_vector_kernel(CopyLaunch L) {
     }
 }
 
+// Argument fetch: per-call arguments (block/slot pairs, hash descriptors) are written by the
+// host into mapped pinned memory and pulled into device memory by this kernel instead of a
+// copy-engine transfer.  A small host-to-device memcpy would queue on the same copy engine as
+// the bulk restores of other requests and wait for all of them (measured: a 32 KB argument
+// upload behind a 6 GiB staged restore delayed the store that needed it by the whole restore).
+__global__ void fetch_args_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int n16) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += gridDim.x * blockDim.x)
+        dst[i] = __ldcs(src + i);
+}
+
+cudaError_t launch_fetch_args(void* dst_dev, const void* src_host_mapped, size_t bytes,
+                              cudaStream_t stream) {
+    const int n16 = (int)((bytes + 15) / 16);
+    if (n16 <= 0) return cudaSuccess;
+    int ctas = (n16 + 255) / 256;
+    if (ctas > 64) ctas = 64;
+    fetch_args_kernel<<<ctas, 256, 0, stream>>>(static_cast<const uint4*>(src_host_mapped),
+                                                static_cast<uint4*>(dst_dev), n16);
+    return cudaGetLastError();
+}
+
 static int g_vector_ctas_per_sm = 0;
 
 cudaError_t copy_kernels_init() {
@@ -162,19 +183,16 @@ copy_blocks_bulk_kernel(CopyLaunch L, int kBulkStages, int kBulkStageBytes) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 
-    // self-check: every item of this CTA must be in range before anything is issued
-    for (int64_t k = 0; k < n_my; ++k) {
-        if (bulk_decode<TO_TIER>(L, first + k * stride, kBulkStageBytes).bytes == 0) {
-            atomicExch(error_flag, kErrCopyRange);
-            return;
-        }
-    }
-
     auto issue_load = [&](int64_t k) {
         const BulkItem b = bulk_decode<TO_TIER>(L, first + k * stride, kBulkStageBytes);
         const int s = (int)(k % kBulkStages);
         const uint32_t bar = smem_u32(&bars[s]);
         const uint32_t dst = smem_u32(stage_mem + (size_t)s * kBulkStageBytes);
+        if (b.bytes == 0) {   // self-check tripped: flag it, complete the phase without a copy
+            atomicExch(error_flag, kErrCopyRange);
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+            return;
+        }
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
                      :: "r"(bar), "r"(b.bytes) : "memory");
         asm volatile(
@@ -194,8 +212,10 @@ copy_blocks_bulk_kernel(CopyLaunch L, int kBulkStages, int kBulkStageBytes) {
         if (!mbar_wait_bounded(smem_u32(&bars[s]), parity)) { ok = false; break; }
         const BulkItem b = bulk_decode<TO_TIER>(L, first + k * stride, kBulkStageBytes);
         const uint32_t src = smem_u32(stage_mem + (size_t)s * kBulkStageBytes);
-        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                     :: "l"(b.dst), "r"(src), "r"(b.bytes) : "memory");
+        if (b.bytes != 0) {
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                         :: "l"(b.dst), "r"(src), "r"(b.bytes) : "memory");
+        }
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         if (k >= 1 && loads_issued < n_my) {
             // all but the newest group have finished reading shared memory: stage of item k-1 is free

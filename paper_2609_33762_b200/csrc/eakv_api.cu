@@ -201,8 +201,8 @@ int ring_upload(eakv_ctx* ctx, const int2* entries, int64_t n, cudaStream_t stre
     int rc = ring_acquire(ctx, &s);
     if (rc != EAKV_OK) return rc;
     std::memcpy(s->host, entries, (size_t)n * sizeof(int2));
-    CU(cudaMemcpyAsync(s->dev, s->host, (size_t)n * sizeof(int2), cudaMemcpyHostToDevice, stream));
-    ctx->stats.memcpy_calls += 1;
+    CU(launch_fetch_args(s->dev, s->host, (size_t)n * sizeof(int2), stream));
+    ctx->stats.kernel_launches += 1;
     *slot_out = s;
     *dev_out = static_cast<const int2*>(s->dev);
     return EAKV_OK;
@@ -447,7 +447,7 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
                                            (size_t)ctx->max_call_blocks * sizeof(HashTile),
                                        (size_t)1 << 16);
     for (auto& s : ctx->ring) {
-        CUC(cudaHostAlloc(&s.host, ctx->ring_bytes, cudaHostAllocDefault));
+        CUC(cudaHostAlloc(&s.host, ctx->ring_bytes, cudaHostAllocMapped | cudaHostAllocPortable));
         CUC(cudaMalloc(&s.dev, ctx->ring_bytes));
         CUC(cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming));
     }
@@ -609,8 +609,8 @@ int eakv_hash_blocks_batched(eakv_ctx* ctx, const int32_t* tokens_dev,
         }
         acc += nb;
     }
-    CU(cudaMemcpyAsync(s->dev, s->host, need, cudaMemcpyHostToDevice, stream));
-    ctx->stats.memcpy_calls += 1;
+    CU(launch_fetch_args(s->dev, s->host, need, stream));
+    ctx->stats.kernel_launches += 1;
     HashLaunch L;
     L.tokens = tokens_dev;
     L.keys = hashes_dev;

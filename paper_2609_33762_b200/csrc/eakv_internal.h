@@ -84,6 +84,9 @@ constexpr int kErrBulkTimeout = 1, kErrCopyRange = 2, kErrHashRange = 3;
 // to_tier: pool -> tier (store/gather); else tier -> pool (load/scatter)
 cudaError_t launch_copy_vector(const CopyLaunch& L, bool to_tier, int ctas, cudaStream_t stream);
 cudaError_t launch_copy_bulk(const CopyLaunch& L, bool to_tier, int ctas, cudaStream_t stream);
+// pull `bytes` (rounded up to 16) of per-call arguments from mapped pinned memory into device memory
+cudaError_t launch_fetch_args(void* dst_dev, const void* src_host_mapped, size_t bytes,
+                              cudaStream_t stream);
 cudaError_t copy_kernels_init();
 int copy_vector_ctas_per_sm();
 
