@@ -89,11 +89,21 @@ __device__ __noinline__ void scan_prompt(const uint64_t* partial, uint64_t* keys
         for (int i = 0; i < kRegRun; ++i) {
             if (lo + i < hi) mine.c = addmod61(mulmod61(mine.c, A), run[i]);
         }
-        // the run's multiplier is A^(hi-lo): square-and-multiply instead of one product per block
-        uint64_t sq = A;
-        for (int64_t n = hi - lo; n; n >>= 1) {
-            if (n & 1) mine.a = mulmod61(mine.a, sq);
+        // the run's multiplier is A^(hi-lo).  All full runs share A^per: one warp-uniform
+        // square-and-multiply; only the single ragged run at the end needs its own.
+        uint64_t sq = A, a_full = 1;
+        for (int64_t n = per; n; n >>= 1) {
+            if (n & 1) a_full = mulmod61(a_full, sq);
             sq = mulmod61(sq, sq);
+        }
+        if (hi - lo == per) {
+            mine.a = a_full;
+        } else {
+            sq = A;
+            for (int64_t n = hi - lo; n; n >>= 1) {
+                if (n & 1) mine.a = mulmod61(mine.a, sq);
+                sq = mulmod61(sq, sq);
+            }
         }
     } else {
         for (int64_t j = lo; j < hi; ++j) {
@@ -358,13 +368,16 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
         s2 += (uint64_t)x_ * w_.z;                          \
     } while (0)
 
+// B: the block size when known at compile time (16, 32, 64: loops unroll and every shared-memory
+// offset becomes an immediate), 0: read it from the launch descriptor.
+template <int B>
 __global__ void __launch_bounds__(kHashThreads)
 hash_blocks_staged_kernel(HashLaunch L) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ Pair warp_tot[32];
     __shared__ int is_last;
     const int tid = threadIdx.x;
-    const int b = L.block_size, cpb = b >> 2;
+    const int b = B ? B : L.block_size, cpb = b >> 2;
     const int row_bytes = 4 * b + 16;
     uint4* pw3 = reinterpret_cast<uint4*>(smem_raw);
     unsigned char* const stage0 = smem_raw + (size_t)b * 16;
@@ -427,16 +440,27 @@ hash_blocks_staged_kernel(HashLaunch L) {
         if (j < nb_tile) {
             const int4* row = reinterpret_cast<const int4*>(stage0 + (r & 1) * stage_bytes + (size_t)tid * row_bytes);
             uint64_t acc = 0;
-            for (int k0 = 0; k0 < b; k0 += kLimbFoldTokens) {
-                const int k1 = min(b, k0 + kLimbFoldTokens);
+            if (B) {   // b <= 64 < kLimbFoldTokens: one fold per block, fully unrolled
                 uint64_t s0 = 0, s1 = 0, s2 = 0;
-#pragma unroll 4
-                for (int k = k0; k < k1; k += 4) {
+#pragma unroll
+                for (int k = 0; k < (B ? B : 4); k += 4) {
                     const int4 u = row[k >> 2];
-                    const int e = b - 1 - k;
+                    const int e = (B ? B : 4) - 1 - k;
                     EAKV_MAC3(u.x, e); EAKV_MAC3(u.y, e - 1); EAKV_MAC3(u.z, e - 2); EAKV_MAC3(u.w, e - 3);
                 }
-                acc = addmod61(acc, fold_limb_sums(s0, s1, s2));
+                acc = fold_limb_sums(s0, s1, s2);
+            } else {
+                for (int k0 = 0; k0 < b; k0 += kLimbFoldTokens) {
+                    const int k1 = min(b, k0 + kLimbFoldTokens);
+                    uint64_t s0 = 0, s1 = 0, s2 = 0;
+#pragma unroll 4
+                    for (int k = k0; k < k1; k += 4) {
+                        const int4 u = row[k >> 2];
+                        const int e = b - 1 - k;
+                        EAKV_MAC3(u.x, e); EAKV_MAC3(u.y, e - 1); EAKV_MAC3(u.z, e - 2); EAKV_MAC3(u.w, e - 3);
+                    }
+                    acc = addmod61(acc, fold_limb_sums(s0, s1, s2));
+                }
             }
             __stcg(partial + first_blk + j, acc);
         }
@@ -463,8 +487,11 @@ cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool thread_per_block,
     if (thread_per_block) {
         const size_t smem = (size_t)L.block_size * sizeof(uint4);
         const size_t staged = smem + 2 * (size_t)kHashThreads * (4 * L.block_size + 16);
-        if (vec) hash_blocks_staged_kernel<<<n_tiles, kHashThreads, staged, stream>>>(L);
-        else     hash_blocks_tpb_kernel<false><<<n_tiles, kHashThreads, smem, stream>>>(L);
+        if (!vec)                    hash_blocks_tpb_kernel<false><<<n_tiles, kHashThreads, smem, stream>>>(L);
+        else if (L.block_size == 16) hash_blocks_staged_kernel<16><<<n_tiles, kHashThreads, staged, stream>>>(L);
+        else if (L.block_size == 32) hash_blocks_staged_kernel<32><<<n_tiles, kHashThreads, staged, stream>>>(L);
+        else if (L.block_size == 64) hash_blocks_staged_kernel<64><<<n_tiles, kHashThreads, staged, stream>>>(L);
+        else                         hash_blocks_staged_kernel<0><<<n_tiles, kHashThreads, staged, stream>>>(L);
     } else {
         const size_t smem = (size_t)(L.block_size + 1) * 8 +
                             (size_t)L.tile_blocks * (L.block_size / 4) * 8;
@@ -482,7 +509,16 @@ cudaError_t hash_kernels_init() {
     e = cudaFuncSetAttribute(hash_blocks_kernel<false>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, kHashMaxSmem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(hash_blocks_staged_kernel,
+    e = cudaFuncSetAttribute(hash_blocks_staged_kernel<0>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kHashStagedMaxSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(hash_blocks_staged_kernel<16>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kHashStagedMaxSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(hash_blocks_staged_kernel<32>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kHashStagedMaxSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(hash_blocks_staged_kernel<64>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, kHashStagedMaxSmem);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(hash_blocks_tpb_kernel<false>,
