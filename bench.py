@@ -329,6 +329,35 @@ def hash_throughput(torch, eakv, pool, shape, device, peak_gbs, prompts=512, tok
             "single_prompt_tokens": tokens, "single_prompt_us_median": float(np.median(single))}
 
 
+def control_plane_rate(eakv, pool, shape, device, requests=400, blocks=4096):
+    """Single-thread rate of the host control plane: block references per second through
+    eakv_match and eakv_tier_step on a thrashing tier (every second request re-references the
+    previous one's keys, the others insert and evict)."""
+    ctx = eakv.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+                       block_size=shape.block_size, gpu_blocks=pool.gpu_blocks, host_blocks=3 * blocks,
+                       kv_base=pool.kv_base, tier_location=eakv.TIER_DEVICE,
+                       tier_memory=pool.pieces[0].data_ptr())
+    rng = np.random.default_rng(3)
+    keys = [rng.integers(1, 1 << 60, size=blocks, dtype=np.uint64) for _ in range(requests // 2 + 1)]
+    t_match = t_step = 0.0
+    refs = 0
+    for i in range(requests):
+        k = keys[i // 2]
+        t0 = time.perf_counter()
+        ctx.eakv_match(k)
+        t1 = time.perf_counter()
+        ctx.eakv_tier_step(k, i % 7, blocks * shape.block_size, i * 100)
+        t2 = time.perf_counter()
+        t_match += t1 - t0
+        t_step += t2 - t1
+        refs += blocks
+    st = ctx.eakv_get_stats()
+    ctx.close()
+    return {"match_refs_per_s": refs / t_match, "tier_step_refs_per_s": refs / t_step,
+            "references": refs, "hits": st["hits"], "evicted": st["evicted"],
+            "note": "through the Python binding, one thread"}
+
+
 def pinned_link_peak(torch, device, gib=1, reps=5):
     n = gib << 30
     host = torch.empty(n, dtype=torch.uint8).pin_memory()
@@ -530,6 +559,7 @@ def main():
                        frac_of_one_direction=e_val / serial / max(world, 1))
 
     hashing = hash_throughput(torch, eakv, pool, shape, device, peak) if rank == 0 else None
+    control = control_plane_rate(eakv, pool, shape, device) if rank == 0 else None
 
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:
@@ -558,6 +588,7 @@ def main():
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "cpu_baseline": cpu,
             "hash": hashing,
+            "control_plane": control,
         }
         print(json.dumps(line))
         if args.sweep:
