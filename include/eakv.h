@@ -97,6 +97,10 @@ typedef struct eakv_config {
                                       average fewer bytes than this goes zero-copy instead (the
                                       copy engine's per-copy cost outweighs its edge on scattered
                                       single blocks); 0 = 3 MiB, negative = always stage         */
+    int32_t control_plane_only;    /* 1: bookkeeping only (match, tier step, GPU-tier step): no
+                                      CUDA call is made, kv_base may be NULL, no tier memory is
+                                      allocated; hash/store/load return EAKV_E_INVAL            */
+    int32_t reserved0;
     void*   tier_memory;           /* NULL: the context allocates the tier.  Else adopt this
                                       buffer of host_blocks * block bytes (pinned host memory
                                       for TIER_PINNED_HOST, device memory for TIER_DEVICE);

@@ -345,7 +345,8 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
     if (!cfg || !out) return EAKV_E_INVAL;
     *out = nullptr;
     if (cfg->num_layers <= 0 || cfg->kv_heads <= 0 || cfg->head_dim <= 0 || cfg->block_size <= 0 ||
-        cfg->elem_bytes <= 0 || cfg->gpu_blocks <= 0 || cfg->host_blocks <= 0 || !cfg->kv_base)
+        cfg->elem_bytes <= 0 || cfg->gpu_blocks <= 0 || cfg->host_blocks <= 0 ||
+        (!cfg->kv_base && !cfg->control_plane_only))
         return EAKV_E_INVAL;
     if (cfg->block_size > kHashMaxBlockSize) return EAKV_E_INVAL;
     if (cfg->gpu_blocks > INT32_MAX || cfg->host_blocks > INT32_MAX) return EAKV_E_INVAL;
@@ -356,13 +357,14 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
     const int64_t piece = (int64_t)cfg->block_size * cfg->kv_heads * cfg->head_dim * cfg->elem_bytes;
     if (piece % 16 != 0) return EAKV_E_INVAL;
     const int pieces = 2 * cfg->num_layers;
-    for (int q = 0; q < pieces; ++q) {
+    for (int q = 0; q < pieces && !cfg->control_plane_only; ++q) {
         if (!cfg->kv_base[q] || ((uintptr_t)cfg->kv_base[q] & 15)) return EAKV_E_INVAL;
     }
     if (cfg->tier_memory && ((uintptr_t)cfg->tier_memory & 15)) return EAKV_E_INVAL;
 
     int ndev = 0;
-    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) return EAKV_E_CUDA;
+    if (!cfg->control_plane_only && (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0))
+        return EAKV_E_CUDA;
 
     eakv_ctx* ctx = new (std::nothrow) eakv_ctx();
     if (!ctx) return EAKV_E_NOMEM;
@@ -394,10 +396,12 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
         }                                                     \
     } while (0)
 
-    CUC(cudaGetDevice(&ctx->device));
-    CUC(cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device));
-    CUC(hash_kernels_init());
-    CUC(copy_kernels_init());
+    if (!cfg->control_plane_only) {
+        CUC(cudaGetDevice(&ctx->device));
+        CUC(cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device));
+        CUC(hash_kernels_init());
+        CUC(copy_kernels_init());
+    }
 
     try {
         ctx->host_tier = new KeyedLru(cfg->host_blocks);
@@ -410,6 +414,12 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
     } catch (const std::bad_alloc&) {
         free_all(ctx);
         return EAKV_E_NOMEM;
+    }
+
+    if (cfg->control_plane_only) {   // bookkeeping only: nothing below is needed
+        ctx->device = -1;
+        *out = ctx;
+        return EAKV_OK;
     }
 
     // piece-array base pointers
@@ -475,6 +485,7 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
 
 int eakv_sync(eakv_ctx* ctx) {
     if (!ctx) return EAKV_E_INVAL;
+    if (ctx->device < 0) return EAKV_OK;
     DeviceGuard g(ctx->device);
     CU(cudaDeviceSynchronize());
     int flag = 0;
@@ -492,6 +503,10 @@ int eakv_sync(eakv_ctx* ctx) {
 
 int eakv_destroy(eakv_ctx* ctx) {
     if (!ctx) return EAKV_E_INVAL;
+    if (ctx->device < 0) {
+        free_all(ctx);
+        return EAKV_OK;
+    }
     DeviceGuard g(ctx->device);
     cudaDeviceSynchronize();
     free_all(ctx);
@@ -504,7 +519,7 @@ int eakv_destroy(eakv_ctx* ctx) {
 int eakv_hash_blocks(eakv_ctx* ctx, const int32_t* tokens_dev, int64_t n_tokens,
                      uint64_t parent_hash, uint64_t* hashes_dev, int64_t* n_blocks_out,
                      void* cuda_stream) {
-    if (!ctx || n_tokens < 0) return EAKV_E_INVAL;
+    if (!ctx || n_tokens < 0 || ctx->device < 0) return EAKV_E_INVAL;
     const int b = ctx->cfg.block_size;
     const int64_t nblk = n_tokens / b;
     if (n_blocks_out) *n_blocks_out = nblk;
@@ -552,7 +567,7 @@ int eakv_hash_blocks_batched(eakv_ctx* ctx, const int32_t* tokens_dev,
                              const int64_t* offsets_host, int64_t n_prompts,
                              const uint64_t* parents_host, uint64_t* hashes_dev,
                              int64_t* block_offsets_out, void* cuda_stream) {
-    if (!ctx || n_prompts < 0 || !offsets_host) return EAKV_E_INVAL;
+    if (!ctx || n_prompts < 0 || !offsets_host || ctx->device < 0) return EAKV_E_INVAL;
     const int b = ctx->cfg.block_size;
     int64_t total_blocks = 0;
     for (int64_t i = 0; i < n_prompts; ++i) {
@@ -763,7 +778,7 @@ int eakv_gpu_tier_release(eakv_ctx* ctx, int32_t block_id) {
 // ------------------------------------------------------------------------------------------
 int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_mask,
                const int32_t* host_slots, int64_t n_blocks, void* cuda_stream) {
-    if (!ctx || n_blocks < 0) return EAKV_E_INVAL;
+    if (!ctx || n_blocks < 0 || ctx->device < 0) return EAKV_E_INVAL;
     if (n_blocks == 0) return EAKV_OK;
     if (!block_table || !host_slots) return EAKV_E_INVAL;
     // validate and compact before anything is enqueued
@@ -792,7 +807,7 @@ int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_m
 
 int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_table,
               int64_t n_blocks, void* cuda_stream) {
-    if (!ctx || n_blocks < 0) return EAKV_E_INVAL;
+    if (!ctx || n_blocks < 0 || ctx->device < 0) return EAKV_E_INVAL;
     if (n_blocks == 0) return EAKV_OK;
     if (!block_table || !host_slots) return EAKV_E_INVAL;
     next_epoch(ctx);

@@ -41,6 +41,7 @@ class Config(C.Structure):
         ("copy_ctas", C.c_int32),
         ("staging_bytes", C.c_int64), ("max_call_blocks", C.c_int64),
         ("hash_scratch_blocks", C.c_int64), ("min_staged_run_bytes", C.c_int64),
+        ("control_plane_only", C.c_int32), ("reserved0", C.c_int32),
         ("tier_memory", C.c_void_p),
     ]
 
@@ -144,17 +145,19 @@ class Context:
                  window_ms=60_000, telemetry=1, link_strategy=LINK_STAGED,
                  tier_location=TIER_PINNED_HOST, copy_path=COPY_BULK, copy_ctas=0,
                  staging_bytes=0, max_call_blocks=0, hash_scratch_blocks=0, min_staged_run_bytes=0,
-                 tier_memory=0):
+                 tier_memory=0, control_plane_only=False):
         L = lib()
         cfg = Config()
         L.eakv_config_init(C.byref(cfg))
-        ptrs = (C.c_void_p * len(kv_base))(*[int(p) for p in kv_base])
-        if len(kv_base) != 2 * num_layers:
+        kv_base = list(kv_base) if kv_base is not None else []
+        if not control_plane_only and len(kv_base) != 2 * num_layers:
             raise ValueError("kv_base must hold 2 * num_layers device pointers")
+        ptrs = (C.c_void_p * max(len(kv_base), 1))(*[int(p) for p in kv_base])
         cfg.num_layers, cfg.kv_heads, cfg.head_dim = num_layers, kv_heads, head_dim
         cfg.block_size, cfg.elem_bytes = block_size, elem_bytes
         cfg.gpu_blocks, cfg.host_blocks, cfg.gpu_index_blocks = gpu_blocks, host_blocks, gpu_index_blocks
-        cfg.kv_base = C.cast(ptrs, C.POINTER(C.c_void_p))
+        cfg.kv_base = C.cast(ptrs, C.POINTER(C.c_void_p)) if kv_base else None
+        cfg.control_plane_only = int(bool(control_plane_only))
         cfg.hash_base, cfg.hash_seed = hash_base, hash_seed
         cfg.policy, cfg.kappa_blocks, cfg.theta_percent = policy, kappa_blocks, theta_percent
         cfg.len_window, cfg.window_ms, cfg.telemetry = len_window, window_ms, telemetry

@@ -1,0 +1,192 @@
+"""The C++ control plane (eakv_match, eakv_tier_step, eakv_gpu_tier_step) against the oracle,
+on the CPU: a control-plane-only context makes no CUDA call, so this runs without a GPU.
+Keys come from the oracle's hash here; the GPU tests check the hash kernel itself."""
+import random
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+from eakv_workloads import CONFIGS, SHAPES, make_trace
+from oracle import hash as ohash
+from oracle.tier import CapacityError, HostTier
+from oracle.trace import GpuTier, TraceOracle
+
+
+@pytest.fixture(scope="module")
+def eakv():
+    from paper_2609_33762_b200 import build, eakv as m
+    build.build()
+    return m
+
+
+def cp_ctx(eakv, block_size, gpu_blocks, host_blocks, **kw):
+    return eakv.Context(num_layers=1, kv_heads=1, head_dim=8, block_size=block_size,
+                        gpu_blocks=gpu_blocks, host_blocks=host_blocks, kv_base=None,
+                        control_plane_only=True, **kw)
+
+
+def as_keys(keys):
+    return np.asarray(keys, dtype=np.uint64)
+
+
+@pytest.mark.parametrize("policy", [0, 1, 2])
+@pytest.mark.parametrize("telemetry", [1, 0])
+def test_tier_step_random_requests(eakv, policy, telemetry):
+    rng = random.Random(100 + 10 * policy + telemetry)
+    for case in range(40):
+        K = rng.randrange(3, 40)
+        b = rng.choice([1, 4, 16])
+        kappa = rng.choice([0, 1, 2, 5, 100])
+        theta = rng.choice([50, 95, 100])
+        window = rng.choice([5, 50, 10_000])
+        lw = rng.choice([1, 3, 256])
+        ctx = cp_ctx(eakv, b, 8, K, policy=policy, kappa_blocks=kappa, theta_percent=theta,
+                     window_ms=window, len_window=lw, telemetry=telemetry)
+        tier = HostTier(K, b, policy, kappa, theta, window, lw, bool(telemetry))
+        now = 0
+        for _ in range(rng.randrange(5, 60)):
+            agent = rng.randrange(5)
+            n = rng.randrange(0, K + 1)
+            start = rng.randrange(0, 4)
+            keys = [1000 * agent + start + j for j in range(n)]
+            if n > 2 and rng.random() < 0.3:            # a foreign key in the middle: isolated hits after it
+                keys[rng.randrange(1, n)] = 999_000 + rng.randrange(50)
+            n_tokens = n * b + rng.randrange(0, b)
+            now += rng.choice([0, 1, 7, 100])
+            G, H, _, slots = ctx.eakv_match(as_keys(keys))
+            assert H == tier.leading_run(keys)
+            assert slots.tolist() == [tier.slot_of(k) for k in keys[:H]]
+            want = tier.step(keys, n_tokens, agent, now)
+            got = ctx.eakv_tier_step(as_keys(keys), agent, n_tokens, now)
+            assert got["hit"].tolist() == want.hit and got["admit"].tolist() == want.admit
+            assert got["slot"].tolist() == want.slot
+            assert list(zip(got["evicted_keys"].tolist(), got["evicted_slots"].tolist())) == want.evicted
+            assert (got["host_prefix_blocks"], got["new_chunks"], got["pressure"], got["save"]) == \
+                   (want.host_prefix_blocks, want.new_chunks, want.pressure, want.save)
+        st = ctx.eakv_get_stats()
+        for f in ("requests", "references", "hits", "admitted", "declined", "evicted",
+                  "declined_requests", "pressure_requests"):
+            assert st[f] == tier.stats[f], f
+        assert st["resident"] == len(tier.order)
+        ctx.close()
+
+
+def test_gpu_tier_random_requests(eakv):
+    rng = random.Random(7)
+    for case in range(60):
+        NB = rng.randrange(2, 30)
+        ctx = cp_ctx(eakv, 4, NB, 4)
+        g = GpuTier(NB)
+        for _ in range(rng.randrange(3, 40)):
+            agent = rng.randrange(4)
+            tail = rng.random() < 0.5
+            n = rng.randrange(0, NB - int(tail) + 1)
+            keys = [100 * agent + j for j in range(n)]
+            G, _, gids, _ = ctx.eakv_match(as_keys(keys))
+            lead = 0
+            for k in keys:
+                if k not in g:
+                    break
+                lead += 1
+            assert G == lead and gids.tolist() == [g.order[k] for k in keys[:G]]
+            want = g.step(keys, tail)
+            res, blk, t = ctx.eakv_gpu_tier_step(as_keys(keys), tail)
+            assert (res.tolist(), blk.tolist(), t) == want
+            if tail:
+                g.release(t)
+                ctx.eakv_gpu_tier_release(t)
+        ctx.close()
+
+
+def drive(ctx, trace, b, limit=None):
+    """The harness's control sequence with oracle keys instead of the hash kernel."""
+    recs = []
+    for i, req in enumerate(trace.requests):
+        if limit is not None and i >= limit:
+            break
+        toks = trace.prompt(req)
+        keys = as_keys(ohash.hash_blocks(toks.tolist(), b))
+        G, H, _, slots = ctx.eakv_match(keys)
+        step = ctx.eakv_tier_step(keys, req.agent, len(toks), req.time_ms)
+        res, blk, tail = ctx.eakv_gpu_tier_step(keys, len(toks) % b != 0)
+        if tail >= 0:
+            ctx.eakv_gpu_tier_release(tail)
+        recs.append((keys, G, H, step, res, blk))
+    return recs
+
+
+def compare(recs, oracle_records):
+    assert len(recs) == len(oracle_records)
+    for (keys, G, H, step, res, blk), w in zip(recs, oracle_records):
+        assert [int(k) for k in keys] == w["keys"]
+        assert (G, H, step["new_chunks"], step["pressure"], step["save"]) == \
+               (w["G"], w["H"], w["new_chunks"], w["pressure"], w["save"])
+        assert step["hit"].tolist() == w["hit"] and step["admit"].tolist() == w["admit"]
+        assert step["slot"].tolist() == w["slot"]
+        assert list(zip(step["evicted_keys"].tolist(), step["evicted_slots"].tolist())) == w["evicted"]
+        assert res.tolist() == w["gpu_resident"] and blk.tolist() == w["gpu_block"]
+
+
+@pytest.mark.parametrize("cfg_name", ["c0", "c0_big_tier"])
+def test_config0_control_plane_on_cpu(eakv, cfg_name):
+    cfg = CONFIGS[cfg_name]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg)
+    oracle = TraceOracle(shape, cfg.gpu_blocks, cfg.host_blocks)
+    oracle.run(trace)
+    ctx = cp_ctx(eakv, shape.block_size, cfg.gpu_blocks, cfg.host_blocks)
+    compare(drive(ctx, trace, shape.block_size), oracle.records)
+    ctx.close()
+
+
+@pytest.mark.parametrize("policy", [1, 2])
+def test_policies_on_a_scaled_down_config2_trace(eakv, policy):
+    cfg = replace(CONFIGS["c2"], shape="tiny", agents=8, turns=16, first_prompt=400,
+                  append_median=150.0, context_cap=3000, tool_gap_mean_ms=15_000.0)
+    shape = SHAPES["tiny"]
+    trace = make_trace(cfg, seed=31)
+    kw = dict(policy=policy, kappa_blocks=6, window_ms=60_000, len_window=32)
+    oracle = TraceOracle(shape, 256, 300, **kw)
+    oracle.run(trace)
+    ctx = cp_ctx(eakv, shape.block_size, 256, 300, **kw)
+    compare(drive(ctx, trace, shape.block_size), oracle.records)
+    assert oracle.host.stats["declined_requests"] > 0
+    ctx.close()
+
+
+def test_capacity_and_argument_errors(eakv):
+    ctx = cp_ctx(eakv, 4, 6, 3)
+    keys = as_keys([1, 2, 3, 4])
+    ctx.eakv_tier_step(keys[:2], 0, 8, 0)
+    before = ctx.eakv_get_stats()
+    with pytest.raises(eakv.EakvError) as ei:
+        ctx.eakv_tier_step(keys, 0, 16, 1)                 # 4 blocks > K_H = 3
+    assert ei.value.code == eakv.E_CAPACITY and ctx.eakv_get_stats() == before
+    with pytest.raises(eakv.EakvError) as ei:
+        ctx.eakv_gpu_tier_step(as_keys(range(1, 7)), True)  # 6 blocks + tail > 6
+    assert ei.value.code == eakv.E_CAPACITY
+    res, blk, tail = ctx.eakv_gpu_tier_step(as_keys([1, 2]), True)
+    assert tail == 2
+    with pytest.raises(eakv.EakvError) as ei:
+        ctx.eakv_gpu_tier_step(as_keys([1, 2, 3, 4, 5]), True)   # the outstanding tail counts
+    assert ei.value.code == eakv.E_CAPACITY
+    for bad, code in ((0, eakv.E_INVAL), (7, eakv.E_RANGE), (-1, eakv.E_RANGE)):
+        with pytest.raises(eakv.EakvError) as ei:
+            ctx.eakv_gpu_tier_release(bad)                 # 0 is a keyed block, 7/-1 out of range
+        assert ei.value.code == code
+    ctx.eakv_gpu_tier_release(tail)
+    # data-plane calls are refused on a control-plane-only context; sync and stats still work
+    for call in (lambda: ctx.eakv_store([0], None, [0]), lambda: ctx.eakv_load([0], [0]),
+                 lambda: ctx.eakv_hash_blocks(16, 64, 1, 16)):
+        with pytest.raises(eakv.EakvError) as ei:
+            call()
+        assert ei.value.code == eakv.E_INVAL
+    ctx.eakv_sync()
+    ctx.close()
+
+
+def test_oracle_capacity_error_matches(eakv):
+    t = HostTier(2, 4)
+    with pytest.raises(CapacityError):
+        t.step([1, 2, 3], 12, 0, 0)
