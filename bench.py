@@ -438,6 +438,26 @@ def oracle_step_rate(seconds, blocks=128, pool_blocks=512, steps_cap=10**9):
     return moved / dt / 1e9, s, dt
 
 
+def oracle_component_rates():
+    """The oracle's parts timed alone, as they stand: hashed tokens/s, tier references/s."""
+    from oracle import hash as ohash
+    from oracle.tier import HostTier
+    rng = np.random.default_rng(2)
+    toks = rng.integers(0, 151936, size=1 << 20, dtype=np.int32).tolist()
+    t0 = time.perf_counter()
+    keys = ohash.hash_blocks(toks, 16)
+    t_hash = time.perf_counter() - t0
+    tier = HostTier(3 * 4096, 16)
+    t0 = time.perf_counter()
+    refs = 0
+    for i in range(40):
+        k = keys[(i // 2) * 4096 % len(keys):][:4096]
+        tier.step(k, len(k) * 16, i % 5, i)
+        refs += len(k)
+    t_tier = time.perf_counter() - t0
+    return {"hash_tokens_per_s": len(toks) / t_hash, "tier_refs_per_s": refs / t_tier}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -566,6 +586,7 @@ def main():
         g, s, dt = oracle_step_rate(args.cpu_seconds)
         cpu = {"value": g, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"{s} steps x 2 requests x 128 blocks of 1.5 MiB in {dt:.1f} s"}
+        cpu.update(oracle_component_rates())
 
     if rank == 0:
         line = {

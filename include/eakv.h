@@ -28,7 +28,7 @@
  *   - Layouts: the paged pool is 2L separate arrays, kv_base[2*l] = layer l's K and
  *     kv_base[2*l+1] = its V, each [gpu_blocks][block_size][kv_heads][head_dim] of
  *     elem_bytes-sized elements; one such [block_size][kv_heads][head_dim] slab is a
- *     "piece".  The tier is slot-major: [host_blocks][L][2][block_size][kv_heads][head_dim].
+ *     "piece".  The tier is slot-major: [host_blocks * chunk_blocks][L][2][block_size][kv_heads][head_dim].
  *     piece bytes must be a multiple of 16 and all base pointers 16-byte aligned.
  */
 #ifndef EAKV_H
@@ -100,9 +100,16 @@ typedef struct eakv_config {
     int32_t control_plane_only;    /* 1: bookkeeping only (match, tier step, GPU-tier step): no
                                       CUDA call is made, kv_base may be NULL, no tier memory is
                                       allocated; hash/store/load return EAKV_E_INVAL            */
-    int32_t reserved0;
+    int32_t chunk_blocks;          /* two granularities (the paper's 1,024-token host chunks over
+                                      16-token GPU blocks): the host tier's unit is a chunk of
+                                      this many consecutive blocks.  host_blocks then counts
+                                      chunks, eakv_tier_step takes one key per chunk and counts
+                                      u in chunks, and the tier memory holds host_blocks *
+                                      chunk_blocks block-sized slots: chunk slot s covers block
+                                      slots s*chunk_blocks .. (s+1)*chunk_blocks-1 for
+                                      eakv_store / eakv_load.  0 or 1: one granularity           */
     void*   tier_memory;           /* NULL: the context allocates the tier.  Else adopt this
-                                      buffer of host_blocks * block bytes (pinned host memory
+                                      buffer of host_blocks * chunk_blocks * block bytes (pinned host memory
                                       for TIER_PINNED_HOST, device memory for TIER_DEVICE);
                                       it must outlive the context                               */
 } eakv_config;

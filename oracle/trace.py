@@ -11,6 +11,13 @@ admitted blocks to their host slots.
 
 The GPU tier is never specified by the paper (it belongs to the serving engine); the
 model above is this build's reading.  KV payloads are a function of (block key, piece).
+
+Two granularities (Section 5.1 and Appendix A: 1,024-token host chunks over the engine's
+16-token blocks; Appendix C: restoration is counted "after chunk and block alignment"):
+with ``chunk_blocks`` = R > 1 the host tier's unit is a chunk of R consecutive blocks, keyed
+by the prefix hash at the chunk's last token.  Only full chunks are looked up and stored;
+host coverage is H_chunks * R blocks; the restore run is blocks [G, H_chunks * R); chunk
+slot s occupies block slots s*R .. s*R + R - 1 of the tier.
 """
 from collections import OrderedDict
 
@@ -64,13 +71,15 @@ class GpuTier:
 class TraceOracle:
     def __init__(self, shape, gpu_blocks, host_blocks, policy=0, kappa_blocks=8,
                  theta_percent=95, window_ms=60_000, len_window=256, telemetry=True,
-                 payload=None, hash_base=ohash.HASH_BASE, hash_seed=ohash.HASH_SEED):
+                 payload=None, hash_base=ohash.HASH_BASE, hash_seed=ohash.HASH_SEED,
+                 chunk_blocks=1):
         """``payload(keys, q, n_words) -> uint16[len(keys), n_words]`` enables full-bytes
         mode (pool and tier held in numpy); None runs metadata only."""
         self.shape = shape
         self.b = shape.block_size
+        self.R = int(chunk_blocks)
         self.gpu = GpuTier(gpu_blocks)
-        self.host = HostTier(host_blocks, self.b, policy, kappa_blocks, theta_percent,
+        self.host = HostTier(host_blocks, self.b * self.R, policy, kappa_blocks, theta_percent,
                              window_ms, len_window, telemetry)
         self.payload = payload
         self.hash_base, self.hash_seed = hash_base, hash_seed
@@ -79,7 +88,7 @@ class TraceOracle:
             P = shape.piece_bytes
             self.pool = [np.zeros((gpu_blocks, P), dtype=np.uint8)
                          for _ in range(shape.pieces_per_block)]
-            self.tier = np.zeros((host_blocks, shape.pieces_per_block, P), dtype=np.uint8)
+            self.tier = np.zeros((host_blocks * self.R, shape.pieces_per_block, P), dtype=np.uint8)
         self.records = []
         self.totals = dict(prompt_tokens=0, fresh_tokens=0, loaded_blocks=0, stored_blocks=0,
                            gpu_hit_blocks=0, host_hit_blocks=0)
@@ -92,13 +101,24 @@ class TraceOracle:
             if k not in self.gpu:
                 break
             G += 1
-        H = self.host.leading_run(keys)
-        host_slots = [self.host.slot_of(k) for k in keys[:H]]
-        res = self.host.step(keys, n, agent, now_ms)
+        R = self.R
+        chunk_keys = keys[R - 1::R]                      # key at each full chunk's last block
+        Hc = self.host.leading_run(chunk_keys)
+        H = Hc * R
+        # block slots of the host-covered prefix, chunk by chunk
+        host_slots = [self.host.slot_of(k) * R + i for k in chunk_keys[:Hc] for i in range(R)]
+        res = self.host.step(chunk_keys, n, agent, now_ms)
         resident, gpu_ids, tail = self.gpu.step(keys, n % self.b != 0)
         cover = max(G, H)
         lo, hi = (G, H) if H > G else (G, G)
         fill = [j for j in range(cover, len(keys)) if not resident[j]]
+        # per-block view of the chunk decisions (blocks past the last full chunk: no host part)
+        admit_b = [0] * len(keys)
+        slot_b = [-1] * len(keys)
+        for c, (a, s) in enumerate(zip(res.admit, res.slot)):
+            for i in range(R):
+                admit_b[c * R + i] = a
+                slot_b[c * R + i] = s * R + i if s >= 0 else -1
         if self.payload is not None:
             storeload.load(self.pool, self.tier, host_slots[lo:hi], gpu_ids[lo:hi])
             if fill:
@@ -107,13 +127,13 @@ class TraceOracle:
                     words = self.payload([keys[j] for j in fill], q, W)
                     for r, j in enumerate(fill):
                         self.pool[q][gpu_ids[j], :] = words[r].view(np.uint8)
-            storeload.store(self.pool, self.tier, gpu_ids, res.admit, res.slot)
+            storeload.store(self.pool, self.tier, gpu_ids, admit_b, slot_b)
         self.gpu.release(tail)
         rec = dict(agent=agent, now_ms=now_ms, n_tokens=n, keys=keys, G=G, H=H,
                    new_chunks=res.new_chunks, pressure=res.pressure, save=res.save,
                    hit=res.hit, admit=res.admit, slot=res.slot, evicted=res.evicted,
                    gpu_resident=resident, gpu_block=gpu_ids, loaded=hi - lo,
-                   stored=sum(res.admit), fresh_tokens=n - cover * self.b, filled=len(fill))
+                   stored=sum(admit_b), fresh_tokens=n - cover * self.b, filled=len(fill))
         t = self.totals
         t["prompt_tokens"] += n
         t["fresh_tokens"] += rec["fresh_tokens"]

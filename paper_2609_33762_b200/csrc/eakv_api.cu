@@ -78,6 +78,8 @@ struct eakv_ctx {
     // staged strategy
     Staging st_store, st_load;
     int64_t staging_blocks = 0;
+    int64_t tier_slots = 0;        // block-sized slots in the tier = host_blocks * chunk_blocks
+    int64_t chunk_tokens = 0;      // tokens per tier unit = block_size * chunk_blocks
     int64_t min_staged_run_bytes = 0;
 
     int* d_error_flag = nullptr;
@@ -178,7 +180,7 @@ int launch_copy(eakv_ctx* ctx, const int2* d_entries, const int2* h_inline, int6
     L.piece_bytes = ctx->piece_bytes;
     L.slot_from_index = packed ? 1 : 0;
     L.gpu_blocks = ctx->cfg.gpu_blocks;
-    L.tier_slots = packed ? ctx->staging_blocks : ctx->cfg.host_blocks;
+    L.tier_slots = packed ? ctx->staging_blocks : ctx->tier_slots;
     L.error_flag = ctx->d_error_flag;
     L.subs_per_piece = (int32_t)((ctx->piece_bytes + kCopySubBytes - 1) / kCopySubBytes);
     cudaError_t e;
@@ -349,7 +351,8 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
         (!cfg->kv_base && !cfg->control_plane_only))
         return EAKV_E_INVAL;
     if (cfg->block_size > kHashMaxBlockSize) return EAKV_E_INVAL;
-    if (cfg->gpu_blocks > INT32_MAX || cfg->host_blocks > INT32_MAX) return EAKV_E_INVAL;
+    const int64_t chunk_blocks = cfg->chunk_blocks > 0 ? cfg->chunk_blocks : 1;
+    if (cfg->gpu_blocks > INT32_MAX || cfg->host_blocks * chunk_blocks > INT32_MAX) return EAKV_E_INVAL;
     if (cfg->policy < 0 || cfg->policy > 2 || cfg->link_strategy < 0 || cfg->link_strategy > 1 ||
         cfg->tier_location < 0 || cfg->tier_location > 1 || cfg->copy_path < 0 || cfg->copy_path > 1)
         return EAKV_E_INVAL;
@@ -381,6 +384,8 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
     ctx->max_call_blocks = cfg->max_call_blocks > 0 ? cfg->max_call_blocks : 16384;
     ctx->hash_scratch_blocks = cfg->hash_scratch_blocks > 0 ? cfg->hash_scratch_blocks : (1 << 20);
     ctx->max_prompts = ctx->max_call_blocks;
+    ctx->tier_slots = cfg->host_blocks * chunk_blocks;
+    ctx->chunk_tokens = (int64_t)cfg->block_size * chunk_blocks;
     ctx->min_staged_run_bytes = cfg->min_staged_run_bytes >= 0 ? cfg->min_staged_run_bytes : 0;
     if (cfg->min_staged_run_bytes == 0) ctx->min_staged_run_bytes = 3ll << 20;
 
@@ -408,8 +413,8 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
         ctx->gpu_tier = new KeyedLru(cfg->gpu_index_blocks ? cfg->gpu_index_blocks : cfg->gpu_blocks);
         ctx->adm = new Admission(cfg->policy, cfg->kappa_blocks, cfg->theta_percent, cfg->window_ms,
                                  cfg->len_window > 0 ? cfg->len_window : 256, cfg->telemetry,
-                                 cfg->host_blocks, cfg->block_size);
-        ctx->slot_stamp.assign((size_t)cfg->host_blocks, 0);
+                                 cfg->host_blocks, cfg->block_size * (int32_t)chunk_blocks);
+        ctx->slot_stamp.assign((size_t)ctx->tier_slots, 0);
         ctx->blk_stamp.assign((size_t)cfg->gpu_blocks, 0);
     } catch (const std::bad_alloc&) {
         free_all(ctx);
@@ -427,7 +432,7 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
     CUC(cudaMemcpy(ctx->d_kv_base, cfg->kv_base, sizeof(void*) * pieces, cudaMemcpyHostToDevice));
 
     // tier memory
-    const size_t tier_bytes = (size_t)cfg->host_blocks * (size_t)ctx->block_bytes;
+    const size_t tier_bytes = (size_t)ctx->tier_slots * (size_t)ctx->block_bytes;
     if (cfg->tier_memory) {
         ctx->tier = static_cast<char*>(cfg->tier_memory);
     } else if (cfg->tier_location == EAKV_TIER_DEVICE) {
@@ -688,8 +693,8 @@ int eakv_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
     int64_t H = 0;
     while (H < n_blocks && T.find(hashes_host[H]) >= 0) ++H;
     const bool p = ctx->adm->pressure(agent_id, n_tokens, now_ms, T.resident());
-    const int b = ctx->cfg.block_size;
-    const int64_t u = n_tokens / b - (H * b) / b;
+    const int64_t cb = ctx->chunk_tokens;                 // tokens per tier unit
+    const int64_t u = n_tokens / cb - (H * cb) / cb;
     const bool save = !(p && u > ctx->adm->kappa());
     eakv_stats& st = ctx->stats;
     st.requests += 1;
@@ -788,7 +793,7 @@ int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_m
     for (int64_t j = 0; j < n_blocks; ++j) {
         if (admit_mask && !admit_mask[j]) continue;
         const int32_t blk = block_table[j], slot = host_slots[j];
-        if (blk < 0 || blk >= ctx->cfg.gpu_blocks || slot < 0 || slot >= ctx->cfg.host_blocks)
+        if (blk < 0 || blk >= ctx->cfg.gpu_blocks || slot < 0 || slot >= ctx->tier_slots)
             return EAKV_E_RANGE;
         if (ctx->slot_stamp[slot] == ctx->epoch) return EAKV_E_INVAL;
         ctx->slot_stamp[slot] = ctx->epoch;
@@ -815,7 +820,7 @@ int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_tab
     ent.clear();
     for (int64_t j = 0; j < n_blocks; ++j) {
         const int32_t blk = block_table[j], slot = host_slots[j];
-        if (blk < 0 || blk >= ctx->cfg.gpu_blocks || slot < 0 || slot >= ctx->cfg.host_blocks)
+        if (blk < 0 || blk >= ctx->cfg.gpu_blocks || slot < 0 || slot >= ctx->tier_slots)
             return EAKV_E_RANGE;
         if (ctx->blk_stamp[blk] == ctx->epoch) return EAKV_E_INVAL;
         ctx->blk_stamp[blk] = ctx->epoch;

@@ -41,7 +41,7 @@ class Config(C.Structure):
         ("copy_ctas", C.c_int32),
         ("staging_bytes", C.c_int64), ("max_call_blocks", C.c_int64),
         ("hash_scratch_blocks", C.c_int64), ("min_staged_run_bytes", C.c_int64),
-        ("control_plane_only", C.c_int32), ("reserved0", C.c_int32),
+        ("control_plane_only", C.c_int32), ("chunk_blocks", C.c_int32),
         ("tier_memory", C.c_void_p),
     ]
 
@@ -145,7 +145,7 @@ class Context:
                  window_ms=60_000, telemetry=1, link_strategy=LINK_STAGED,
                  tier_location=TIER_PINNED_HOST, copy_path=COPY_BULK, copy_ctas=0,
                  staging_bytes=0, max_call_blocks=0, hash_scratch_blocks=0, min_staged_run_bytes=0,
-                 tier_memory=0, control_plane_only=False):
+                 tier_memory=0, control_plane_only=False, chunk_blocks=1):
         L = lib()
         cfg = Config()
         L.eakv_config_init(C.byref(cfg))
@@ -158,6 +158,7 @@ class Context:
         cfg.gpu_blocks, cfg.host_blocks, cfg.gpu_index_blocks = gpu_blocks, host_blocks, gpu_index_blocks
         cfg.kv_base = C.cast(ptrs, C.POINTER(C.c_void_p)) if kv_base else None
         cfg.control_plane_only = int(bool(control_plane_only))
+        cfg.chunk_blocks = int(chunk_blocks)
         cfg.hash_base, cfg.hash_seed = hash_base, hash_seed
         cfg.policy, cfg.kappa_blocks, cfg.theta_percent = policy, kappa_blocks, theta_percent
         cfg.len_window, cfg.window_ms, cfg.telemetry = len_window, window_ms, telemetry
@@ -174,6 +175,8 @@ class Context:
             raise EakvError(rc, "eakv_create")
         self.block_size = block_size
         self.host_blocks = host_blocks
+        self.chunk_blocks = max(1, int(chunk_blocks))
+        self.tier_slots = host_blocks * self.chunk_blocks
         self.piece_bytes = block_size * kv_heads * head_dim * elem_bytes
         self.block_bytes = 2 * num_layers * self.piece_bytes
         self.tier_location = tier_location
@@ -307,10 +310,10 @@ class Context:
         return lib().eakv_hash_base(self._h)
 
     def tier_host_view(self):
-        """numpy uint8 view [host_blocks, 2L, piece_bytes] of a pinned-host tier."""
+        """numpy uint8 view [block slots, 2L, piece_bytes] of a pinned-host tier."""
         if self.tier_location != TIER_PINNED_HOST:
             raise ValueError("tier is not in host memory")
-        n = self.host_blocks * self.block_bytes
+        n = self.tier_slots * self.block_bytes
         buf = (C.c_uint8 * n).from_address(self.eakv_tier_ptr())
         return np.frombuffer(buf, dtype=np.uint8).reshape(
-            self.host_blocks, self.block_bytes // self.piece_bytes, self.piece_bytes)
+            self.tier_slots, self.block_bytes // self.piece_bytes, self.piece_bytes)

@@ -38,9 +38,13 @@ class PagedPool:
 
 class AgentServer:
     def __init__(self, shape, gpu_blocks, host_blocks, payload, *, device="cuda:0",
-                 gpu_index_blocks=0, incremental_hash=False, data_plane=True, **ctx_kwargs):
+                 gpu_index_blocks=0, incremental_hash=False, data_plane=True, chunk_blocks=1,
+                 **ctx_kwargs):
         """``payload(keys, q, n_words)`` returns the int16/uint16 words of piece q for the
-        blocks with these keys, as a numpy array or a tensor on ``device``."""
+        blocks with these keys, as a numpy array or a tensor on ``device``.  With
+        ``chunk_blocks`` = R > 1 the host tier works in chunks of R blocks (``host_blocks``
+        then counts chunks): one key per full chunk goes to the tier step, and chunk slot s
+        maps to block slots s*R .. s*R+R-1 for store and load."""
         self.shape = shape
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
@@ -57,11 +61,12 @@ class AgentServer:
             num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
             block_size=shape.block_size, elem_bytes=shape.elem_bytes, gpu_blocks=gpu_blocks,
             host_blocks=host_blocks, gpu_index_blocks=gpu_index_blocks, kv_base=self.pool.kv_base,
-            **ctx_kwargs)
+            chunk_blocks=chunk_blocks, **ctx_kwargs)
         self.payload = payload
         self.incremental = incremental_hash
         self.stream = torch.cuda.current_stream(self.device)
         self.b = shape.block_size
+        self.R = max(1, int(chunk_blocks))
         self.seed = self.ctx.eakv_hash_seed()
         self._agent_keys = {}          # agent -> np.uint64 keys of its previous prompt
         self._timed = {"load": [], "store": []}     # (bytes, start event, end event)
@@ -136,8 +141,26 @@ class AgentServer:
         n = len(tokens)
         keys = self.block_keys(tokens, agent)
         nblk = len(keys)
-        G, H, _gids, host_slots = self.ctx.eakv_match(keys)
-        step = self.ctx.eakv_tier_step(keys, agent, n, now_ms)
+        R = self.R
+        if R == 1:
+            G, H, _gids, host_slots = self.ctx.eakv_match(keys)
+            step = self.ctx.eakv_tier_step(keys, agent, n, now_ms)
+            admit_b, slot_b = step["admit"], step["slot"]
+        else:
+            # block keys locate the GPU prefix, chunk keys (the key at each full chunk's last
+            # block) the host prefix; chunk decisions are then spread over their blocks
+            G = self.ctx.eakv_match(keys)[0]
+            chunk_keys = np.ascontiguousarray(keys[R - 1::R])
+            _, Hc, _, chunk_slots = self.ctx.eakv_match(chunk_keys)
+            H = Hc * R
+            host_slots = (chunk_slots.astype(np.int64)[:, None] * R + np.arange(R)).reshape(-1).astype(np.int32)
+            step = self.ctx.eakv_tier_step(chunk_keys, agent, n, now_ms)
+            admit_b = np.zeros(nblk, dtype=np.uint8)
+            slot_b = np.full(nblk, -1, dtype=np.int32)
+            nc = len(chunk_keys)
+            admit_b[:nc * R] = np.repeat(step["admit"], R)
+            base = np.repeat(step["slot"].astype(np.int64), R) * R + np.tile(np.arange(R), nc)
+            slot_b[:nc * R] = np.where(np.repeat(step["slot"], R) >= 0, base, -1).astype(np.int32)
         resident, blocks, tail = self.ctx.eakv_gpu_tier_step(keys, n % self.b != 0)
         cover = max(G, H)
         lo, hi = (G, H) if H > G else (G, G)
@@ -153,9 +176,9 @@ class AgentServer:
                 if isinstance(w, np.ndarray):
                     w = torch.from_numpy(w.view(np.int16)).to(self.device)
                 piece[ids] = w.view(torch.int16)
-        if self.data_plane and step["admit"].any():
-            with self._time("store", int(step["admit"].sum()) * self.ctx.block_bytes):
-                self.ctx.eakv_store(blocks, step["admit"], step["slot"], self.stream)
+        if self.data_plane and admit_b.any():
+            with self._time("store", int(admit_b.sum()) * self.ctx.block_bytes):
+                self.ctx.eakv_store(blocks, admit_b, slot_b, self.stream)
         if tail >= 0:
             self.ctx.eakv_gpu_tier_release(tail)
         rec = dict(agent=agent, now_ms=now_ms, n_tokens=n, keys=keys, G=G, H=H,
@@ -163,7 +186,7 @@ class AgentServer:
                    hit=step["hit"], admit=step["admit"], slot=step["slot"],
                    evicted=list(zip(step["evicted_keys"].tolist(), step["evicted_slots"].tolist())),
                    gpu_resident=resident, gpu_block=blocks, loaded=hi - lo,
-                   stored=int(step["admit"].sum()), fresh_tokens=n - cover * self.b,
+                   stored=int(admit_b.sum()), fresh_tokens=n - cover * self.b,
                    filled=len(fill))
         t = self.totals
         t["prompt_tokens"] += n

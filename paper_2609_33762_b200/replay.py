@@ -59,7 +59,7 @@ def plan(cfg, trace, shape, host_gib=None, data_plane=True, ram_fraction=0.6):
 
 def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=True,
         incremental_hash=True, device="cuda:0", link_strategy=eakv.LINK_STAGED, agents=None,
-        turns=None, server_hook=None):
+        turns=None, server_hook=None, chunk_blocks=1, kappa=None):
     import torch
     from eakv_workloads import CONFIGS, SHAPES, key_words_torch, make_trace
     from .harness import AgentServer
@@ -68,11 +68,13 @@ def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=Tru
     shape = SHAPES[cfg.shape]
     trace = make_trace(cfg, agents=agents, turns=turns)
     kh, why = plan(cfg, trace, shape, host_gib, data_plane)
+    kh = max(1, kh // chunk_blocks)                  # the tier counts chunks of chunk_blocks blocks
     payload = (lambda keys, q, n: key_words_torch(keys.astype(np.int64), q, n, device)) if data_plane else None
     t0 = time.perf_counter()
     server = AgentServer(shape, cfg.gpu_blocks, kh, payload, device=device, data_plane=data_plane,
                          incremental_hash=incremental_hash, policy=POLICIES[policy],
-                         kappa_blocks=cfg.kappa_blocks, link_strategy=link_strategy)
+                         kappa_blocks=cfg.kappa_blocks if kappa is None else kappa,
+                         link_strategy=link_strategy, chunk_blocks=chunk_blocks)
     t_setup = time.perf_counter() - t0
     t0 = time.perf_counter()
     server.run(trace, limit=limit)
@@ -86,7 +88,8 @@ def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=Tru
     n_req = len(server.records)
     out = {
         "config": config, "policy": policy, "requests": n_req, "kv_shape": cfg.shape,
-        "gpu_blocks": cfg.gpu_blocks, "host_blocks": kh, "host_gib": kh * shape.block_bytes / GIB,
+        "gpu_blocks": cfg.gpu_blocks, "host_chunks": kh, "chunk_blocks": chunk_blocks,
+        "host_gib": kh * chunk_blocks * shape.block_bytes / GIB,
         "host_sizing": why, "data_plane": data_plane,
         "working_set_blocks_eq5": working_set_blocks(trace, shape),
         "prompt_tokens": tot["prompt_tokens"], "computed_prefill_tokens": tot["fresh_tokens"],
@@ -115,9 +118,12 @@ def main():
     ap.add_argument("--limit", type=int, default=None, help="replay only the first N requests")
     ap.add_argument("--no-data-plane", dest="data_plane", action="store_false")
     ap.add_argument("--zero-copy", action="store_true", help="zero-copy host link instead of staged")
+    ap.add_argument("--chunk-blocks", type=int, default=1,
+                    help="host-tier chunk in GPU blocks (64 = the paper's 1,024-token chunks at block 16)")
+    ap.add_argument("--kappa", type=int, default=None, help="write threshold in tier units")
     args = ap.parse_args()
     out = run(args.config, policy=args.policy, host_gib=args.host_gib, limit=args.limit,
-              data_plane=args.data_plane,
+              data_plane=args.data_plane, chunk_blocks=args.chunk_blocks, kappa=args.kappa,
               link_strategy=eakv.LINK_ZERO_COPY if args.zero_copy else eakv.LINK_STAGED)
     print(json.dumps(out))
 

@@ -20,6 +20,23 @@ def eakv():
     return m
 
 
+def drive_chunked(ctx, trace, b, R):
+    """Two granularities: block keys for the GPU tier, one key per full chunk for the host."""
+    recs = []
+    for req in trace.requests:
+        toks = trace.prompt(req)
+        keys = as_keys(ohash.hash_blocks(toks.tolist(), b))
+        G = ctx.eakv_match(keys)[0]
+        chunk_keys = np.ascontiguousarray(keys[R - 1::R])
+        _, Hc, _, _ = ctx.eakv_match(chunk_keys)
+        step = ctx.eakv_tier_step(chunk_keys, req.agent, len(toks), req.time_ms)
+        res, blk, tail = ctx.eakv_gpu_tier_step(keys, len(toks) % b != 0)
+        if tail >= 0:
+            ctx.eakv_gpu_tier_release(tail)
+        recs.append((keys, G, Hc * R, step, res, blk))
+    return recs
+
+
 def cp_ctx(eakv, block_size, gpu_blocks, host_blocks, **kw):
     return eakv.Context(num_layers=1, kv_heads=1, head_dim=8, block_size=block_size,
                         gpu_blocks=gpu_blocks, host_blocks=host_blocks, kv_base=None,
@@ -152,6 +169,26 @@ def test_policies_on_a_scaled_down_config2_trace(eakv, policy):
     ctx = cp_ctx(eakv, shape.block_size, 256, 300, **kw)
     compare(drive(ctx, trace, shape.block_size), oracle.records)
     assert oracle.host.stats["declined_requests"] > 0
+    ctx.close()
+
+
+@pytest.mark.parametrize("policy,R", [(0, 4), (2, 4), (2, 8), (1, 2)])
+def test_two_granularities(eakv, policy, R):
+    """Host chunks of R blocks over single GPU blocks: u and kappa count chunks, the tier holds
+    chunks, coverage is chunk-aligned."""
+    cfg = replace(CONFIGS["c2"], shape="tiny", agents=6, turns=14, first_prompt=500,
+                  append_median=200.0, context_cap=3500, tool_gap_mean_ms=15_000.0)
+    shape = SHAPES["tiny"]
+    trace = make_trace(cfg, seed=41)
+    kw = dict(policy=policy, kappa_blocks=2, window_ms=60_000, len_window=32)
+    kh = 700 // R                                            # about 700 blocks of host tier
+    oracle = TraceOracle(shape, 256, kh, chunk_blocks=R, **kw)
+    oracle.run(trace)
+    ctx = cp_ctx(eakv, shape.block_size, 256, kh, chunk_blocks=R, **kw)
+    compare(drive_chunked(ctx, trace, shape.block_size, R), oracle.records)
+    assert all(r["H"] % R == 0 for r in oracle.records)
+    if policy != 1:                                             # the fixed filter declines it all
+        assert any(r["H"] > r["G"] for r in oracle.records)      # restores do happen
     ctx.close()
 
 

@@ -44,12 +44,14 @@ def eq5_blocks(trace, shape):
     return int(ws // (shape.block_size * beta))
 
 
-def run_both(cfg_name, *, policy, host_blocks, limit=None, data_plane=False, link=1):
+def run_both(cfg_name, *, policy, host_blocks, limit=None, data_plane=False, link=1, chunk_blocks=1):
     from paper_2609_33762_b200.harness import AgentServer
     cfg = CONFIGS[cfg_name]
     shape = SHAPES[cfg.shape]
     trace = make_trace(cfg)
     kw = dict(policy=policy, kappa_blocks=cfg.kappa_blocks)
+    if chunk_blocks > 1:
+        kw["chunk_blocks"] = chunk_blocks
     oracle = TraceOracle(shape, cfg.gpu_blocks, host_blocks, **kw)
     oracle.run(trace, limit=limit)
     payload = (lambda keys, q, n: key_words_torch(keys.astype(np.int64), q, n, "cuda")) if data_plane else None
@@ -137,4 +139,25 @@ def test_config4_data_plane_prefix():
     server, oracle, shape, _ = run_both("c4", policy=0, host_blocks=kh, limit=60, data_plane=True, link=0)
     assert oracle.totals["stored_blocks"] > 0
     check_sampled_bytes(server, oracle, shape)
+    server.close()
+
+
+def test_config3_paper_granularity_control_plane():
+    """The paper's own granularities on config 3's trace: 1,024-token host chunks (64 blocks of
+    16 tokens), a 32 GiB tier = 341 chunks of 96 MiB, kappa = 8 chunks, conditioned admission."""
+    from dataclasses import replace
+    cfg = CONFIGS["c3"]
+    shape = SHAPES[cfg.shape]
+    R = 64
+    kh = (32 << 30) // (R * shape.block_bytes)
+    assert kh == 341
+    import eakv_workloads
+    old = eakv_workloads.CONFIGS["c3"]
+    try:
+        CONFIGS["c3"] = replace(old, kappa_blocks=8)
+        server, oracle, *_ = run_both("c3", policy=2, host_blocks=kh, limit=600, chunk_blocks=R)
+    finally:
+        CONFIGS["c3"] = old
+    assert oracle.host.stats["declined_requests"] > 0
+    assert all(r["H"] % R == 0 for r in oracle.records)
     server.close()

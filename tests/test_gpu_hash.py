@@ -130,6 +130,31 @@ def test_batched_many_prompts_back_to_back():
     ctx.close()
 
 
+def test_modular_multiply_edge_operands():
+    """With block size 1 the first key is parent * B + x, so base and parent choose the
+    multiplier's operands directly: (p-1)^2, (p-1)*1, 2^60 * 2 == 1, 0 * x, 1 * 1."""
+    for base in (P - 1, 1 << 60, 1, 2, P - 2):
+        ctx = hash_ctx(1, hash_base=base, hash_seed=1)
+        assert ctx.eakv_hash_base() == base
+        for parent in (P - 1, 0, 1, 2, 1 << 60, P - 2):
+            for toks in ([0], [2**31 - 1], [5, 0, 151935, 7]):
+                assert gpu_keys(ctx, toks, parent) == oh.hash_blocks(toks, 1, parent, base), (base, parent)
+        ctx.close()
+    # by hand: (p-1)*(p-1) + 1 == 2 and 2^60*2 + 1 == 2 (mod p)
+    ctx = hash_ctx(1, hash_base=P - 1, hash_seed=1)
+    assert gpu_keys(ctx, [0], P - 1) == [2]
+    ctx.close()
+    ctx = hash_ctx(1, hash_base=1 << 60, hash_seed=1)
+    assert gpu_keys(ctx, [0], 2) == [2]
+    ctx.close()
+    # the same operands through the block scan of a multi-block prompt (A = B^b)
+    for b, base in ((16, P - 1), (4, 1 << 60)):
+        ctx = hash_ctx(b, hash_base=base, hash_seed=1)
+        toks = np.full(b * 600 + 3, 2**31 - 1, dtype=np.int32)
+        assert gpu_keys(ctx, toks, P - 1) == oh.hash_blocks(toks.tolist(), b, P - 1, base)
+        ctx.close()
+
+
 def test_custom_base_and_seed():
     ctx = hash_ctx(16, hash_base=1234567891011, hash_seed=42)
     assert ctx.eakv_hash_base() == 1234567891011 and ctx.eakv_hash_seed() == 42

@@ -130,3 +130,34 @@ def test_tier_step_capacity_error_changes_nothing():
     G, H, gids, slots = server.ctx.eakv_match(keys)
     assert (G, H) == (0, 2) and slots.tolist() == [0, 1]
     server.close()
+
+
+@pytest.mark.parametrize("R,policy,link", [(4, 0, 1), (4, 2, 0), (8, 0, 1)])
+def test_two_granularities_bit_exact(R, policy, link):
+    """Host chunks of R GPU blocks (the paper's 1,024-token chunks over 16-token blocks, scaled
+    down): records and every resident byte against the oracle."""
+    from dataclasses import replace
+    from paper_2609_33762_b200.harness import AgentServer
+    cfg = replace(CONFIGS["c2"], shape="tiny", agents=6, turns=12, first_prompt=500,
+                  append_median=200.0, context_cap=3500, tool_gap_mean_ms=15_000.0)
+    shape = SHAPES["tiny"]
+    trace = make_trace(cfg, seed=42)
+    kw = dict(policy=policy, kappa_blocks=2, window_ms=60_000, len_window=32)
+    kh = 700 // R
+    oracle = TraceOracle(shape, 256, kh, payload=key_words_numpy, chunk_blocks=R, **kw)
+    oracle.run(trace)
+    server = AgentServer(shape, 256, kh, key_words_numpy, chunk_blocks=R, link_strategy=link,
+                         staging_bytes=6 * shape.block_bytes, **kw)
+    server.run(trace)
+    compare_records(server.records, oracle.records)
+    assert server.totals == oracle.totals and oracle.totals["loaded_blocks"] > 0
+    server.ctx.eakv_sync()
+    tier = server.ctx.tier_host_view()
+    for key, slot in oracle.host.order.items():
+        for i in range(R):
+            assert np.array_equal(tier[slot * R + i], oracle.tier[slot * R + i]), (slot, i)
+    for q, t in enumerate(server.pool.pieces):
+        got = t.cpu().numpy().view(np.uint8)
+        for key, blk in oracle.gpu.order.items():
+            assert np.array_equal(got[blk], oracle.pool[q][blk])
+    server.close()
