@@ -358,6 +358,36 @@ def control_plane_rate(eakv, pool, shape, device, requests=400, blocks=4096):
             "note": "through the Python binding, one thread"}
 
 
+def layered_load_probe(torch, arm, tables, shape, layers_per_group=12):
+    """Restore 4,096 blocks from the pinned tier whole, and in layer groups: when the first
+    group's event fires a consumer could start on those layers."""
+    m = arm.m
+    slots = np.arange(m, dtype=np.int32)
+    table = tables[0][:m]
+    st = torch.cuda.Stream(arm.device)
+    groups = -(-shape.num_layers // layers_per_group)
+    out = {}
+    for mode in ("plain", "layered"):
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(groups)]
+        for ev in evs:
+            ev.record(st)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        if mode == "plain":
+            arm.ctx.eakv_load(slots, table, st)
+        else:
+            arm.ctx.eakv_load_layers(slots, table, layers_per_group, [ev.cuda_event for ev in evs], st)
+        e1.record(st)
+        torch.cuda.synchronize()
+        out[mode + "_ms"] = e0.elapsed_time(e1)
+        if mode == "layered":
+            out["group_ready_ms"] = [e0.elapsed_time(ev) for ev in evs]
+    out["layers_per_group"] = layers_per_group
+    out["blocks"] = m
+    return out
+
+
 def pinned_link_peak(torch, device, gib=1, reps=5):
     n = gib << 30
     host = torch.empty(n, dtype=torch.uint8).pin_memory()
@@ -562,6 +592,7 @@ def main():
         e_steps = max(2, min(args.steps, 5))
         re_ = run_arm(arm, prompts_host, tables, e_steps, min(args.warmup, 3), dist, None,
                       time_kernels=False)
+        layered = layered_load_probe(torch, arm, tables, shape) if rank == 0 else None
         arm.ctx.close()
         del arm
         e_ms, e_moved = aggregate_over_ranks(dist, re_["ms"], re_["moved"], device)
@@ -569,6 +600,7 @@ def main():
         e2e = {"value": e_val, "unit": UNIT, "h2d_bytes_per_step": int(re_["h2d"]),
                "d2h_bytes_per_step": int(re_["d2h"]), "steps": e_steps,
                "ms_per_step": e_ms / e_steps, "link_strategy": args.link}
+        e2e["layered_load"] = layered
         if link:
             # one direction at a time: harmonic mean of the two; both at once: the measured
             # bidirectional pinned-memcpy rate

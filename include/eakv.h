@@ -229,6 +229,19 @@ int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_m
 int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_table,
               int64_t n_blocks, void* cuda_stream);
 
+/* Layer-pipelined restore (Section 3.1, Eq. 2: the fixed restoration overhead tau_load is
+ * what a consumer waits for before it can start; moving layers in order lets it start on
+ * the first ones while the rest are in flight).  Same result as eakv_load, but the 2L
+ * pieces of every block are moved in ascending groups of layers_per_group layers, and
+ * events[g] is recorded on cuda_stream as soon as group g of all blocks has landed.
+ *   events    host array of n_events cudaEvent_t handles (as void*), created by the caller;
+ *             n_events must equal ceil(num_layers / layers_per_group)
+ * A consumer stream that waits on events[g] may read layers g*layers_per_group .. of the
+ * blocks in block_table.  Errors as eakv_load, plus EAKV_E_INVAL for a wrong n_events. */
+int eakv_load_layers(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_table,
+                     int64_t n_blocks, int32_t layers_per_group, void* const* events,
+                     int32_t n_events, void* cuda_stream);
+
 /* Block keys without a context and without any allocation.  (The paper has no counterpart;
  * this exists for callers that cannot request device memory: code living inside a serving
  * process whose engine has already claimed the GPU's memory, where an allocation may fail or

@@ -28,13 +28,13 @@ copy_blocks_vector_kernel(CopyLaunch L) {
         const int q = r / L.subs_per_piece;
         const int sub = r - q * L.subs_per_piece;
         const int2 e = L.entries ? __ldg(L.entries + j) : L.inline_entries[j];
-        char* pool = reinterpret_cast<char*>(__ldg(reinterpret_cast<const unsigned long long*>(L.kv_base) + q)) + (int64_t)e.x * L.piece_bytes;
+        char* pool = reinterpret_cast<char*>(__ldg(reinterpret_cast<const unsigned long long*>(L.kv_base) + L.q_first + q)) + (int64_t)e.x * L.piece_bytes;
         const int64_t slot = L.slot_from_index ? j : (int64_t)e.y;
         if ((uint64_t)e.x >= (uint64_t)L.gpu_blocks || (uint64_t)slot >= (uint64_t)L.tier_slots) {
             if (threadIdx.x == 0) atomicExch(L.error_flag, kErrCopyRange);
             continue;
         }
-        char* tier = L.tier_base + (slot * L.pieces + q) * L.piece_bytes;
+        char* tier = L.tier_base + (slot * L.slot_pieces + L.slot_q_first + q) * L.piece_bytes;
         const int4* src = reinterpret_cast<const int4*>(TO_TIER ? pool : tier);
         int4* dst = reinterpret_cast<int4*>(TO_TIER ? tier : pool);
         const int unit0 = sub * (kCopyThreads * kCopyUnroll) + threadIdx.x;
@@ -149,7 +149,7 @@ __device__ __forceinline__ BulkItem bulk_decode(const CopyLaunch& L, int64_t it,
     const int sub = r - q * L.subs_per_piece;
     const int2 e = L.entries ? __ldg(L.entries + j) : L.inline_entries[j];
     const int64_t off = (int64_t)sub * kBulkStageBytes;
-    char* pool = reinterpret_cast<char*>(__ldg(reinterpret_cast<const unsigned long long*>(L.kv_base) + q)) +
+    char* pool = reinterpret_cast<char*>(__ldg(reinterpret_cast<const unsigned long long*>(L.kv_base) + L.q_first + q)) +
                  (int64_t)e.x * L.piece_bytes + off;
     const int64_t slot = L.slot_from_index ? j : (int64_t)e.y;
     BulkItem b;
@@ -157,7 +157,7 @@ __device__ __forceinline__ BulkItem bulk_decode(const CopyLaunch& L, int64_t it,
         b.src = nullptr; b.dst = nullptr; b.bytes = 0;      // the caller flags and skips it
         return b;
     }
-    char* tier = L.tier_base + (slot * L.pieces + q) * L.piece_bytes + off;
+    char* tier = L.tier_base + (slot * L.slot_pieces + L.slot_q_first + q) * L.piece_bytes + off;
     b.src = TO_TIER ? pool : tier;
     b.dst = TO_TIER ? tier : pool;
     const int64_t left = L.piece_bytes - off;

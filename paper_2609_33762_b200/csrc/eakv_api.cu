@@ -168,19 +168,24 @@ int copy_ctas(const eakv_ctx* ctx, bool touches_host) {
 }
 
 // d_entries == NULL: the n (<= kCopyInlineEntries) entries at h_inline ride in the parameters
+// [q_first, q_first + q_count): the piece arrays moved (all 2L, or one layer group)
 int launch_copy(eakv_ctx* ctx, const int2* d_entries, const int2* h_inline, int64_t n,
-                char* tier_base, bool to_tier, bool touches_host, bool packed, cudaStream_t stream) {
+                char* tier_base, bool to_tier, bool touches_host, bool packed, cudaStream_t stream,
+                int q_first, int q_count, int64_t packed_capacity) {
     CopyLaunch L;
     L.entries = d_entries;
     if (!d_entries) std::memcpy(L.inline_entries, h_inline, (size_t)n * sizeof(int2));
     L.n_entries = n;
     L.kv_base = ctx->d_kv_base;
     L.tier_base = tier_base;
-    L.pieces = ctx->pieces;
+    L.pieces = q_count;
+    L.q_first = q_first;
+    L.slot_pieces = packed ? q_count : ctx->pieces;
+    L.slot_q_first = packed ? 0 : q_first;
     L.piece_bytes = ctx->piece_bytes;
     L.slot_from_index = packed ? 1 : 0;
     L.gpu_blocks = ctx->cfg.gpu_blocks;
-    L.tier_slots = packed ? ctx->staging_blocks : ctx->tier_slots;
+    L.tier_slots = packed ? packed_capacity : ctx->tier_slots;
     L.error_flag = ctx->d_error_flag;
     L.subs_per_piece = (int32_t)((ctx->piece_bytes + kCopySubBytes - 1) / kCopySubBytes);
     cudaError_t e;
@@ -244,14 +249,20 @@ int for_slot_runs(const int2* e, int64_t n, F f) {
 //   staged : HBM staging buffers + copy engine on the side stream, double-buffered
 // Under EAKV_LINK_STAGED a call whose slots are so scattered that the copy engine would get
 // mostly single-block copies goes direct instead (per-copy overhead outweighs the DMA's edge).
-int move_blocks(eakv_ctx* ctx, const std::vector<int2>& ent, bool to_tier, cudaStream_t stream) {
+int move_blocks(eakv_ctx* ctx, const std::vector<int2>& ent, bool to_tier, cudaStream_t stream,
+                int q_first, int q_count) {
     const int64_t m = (int64_t)ent.size();
+    const bool whole = q_count == ctx->pieces;
+    const int64_t range_bytes = (int64_t)q_count * ctx->piece_bytes;      // per block
+    // a staging buffer holds more blocks when only a layer group of each is moved
+    const int64_t stage_cap = whole ? ctx->staging_blocks
+        : std::min<int64_t>(ctx->max_call_blocks, ctx->staging_blocks * ctx->block_bytes / range_bytes);
     const bool host_tier = ctx->cfg.tier_location == EAKV_TIER_PINNED_HOST;
     bool direct = ctx->cfg.link_strategy == EAKV_LINK_ZERO_COPY;
     if (!direct) {
         int64_t runs = 0;
         for_slot_runs(ent.data(), m, [&](int64_t, int64_t) { ++runs; return EAKV_OK; });
-        const int64_t avg_run_bytes = m * ctx->block_bytes / runs;
+        const int64_t avg_run_bytes = m * range_bytes / runs;
         direct = avg_run_bytes < ctx->min_staged_run_bytes;
     }
     Staging& S = to_tier ? ctx->st_store : ctx->st_load;
@@ -273,25 +284,36 @@ int move_blocks(eakv_ctx* ctx, const std::vector<int2>& ent, bool to_tier, cudaS
             if (rc != EAKV_OK) return rc;
         }
         if (direct) {
-            rc = launch_copy(ctx, d, h, n, ctx->tier, to_tier, host_tier, false, stream);
+            rc = launch_copy(ctx, d, h, n, ctx->tier, to_tier, host_tier, false, stream,
+                             q_first, q_count, 0);
             if (rc != EAKV_OK) return rc;
         } else {
-            for (int64_t i = 0; i < n; i += ctx->staging_blocks) {
-                const int64_t cur = std::min(ctx->staging_blocks, n - i);
+            for (int64_t i = 0; i < n; i += stage_cap) {
+                const int64_t cur = std::min(stage_cap, n - i);
                 const int sb = S.next;
                 S.next ^= 1;
                 const int2* e = h + i;
                 auto dma = [&](int64_t a, int64_t z) {
-                    char* tier_p = ctx->tier + (int64_t)e[a].y * ctx->block_bytes;
-                    char* stage_p = S.buf[sb] + a * ctx->block_bytes;
-                    CU(cudaMemcpyAsync(to_tier ? tier_p : stage_p, to_tier ? stage_p : tier_p,
-                                       (size_t)(z - a) * ctx->block_bytes, cudaMemcpyDefault, S.side));
+                    char* tier_p = ctx->tier + (int64_t)e[a].y * ctx->block_bytes +
+                                   (int64_t)q_first * ctx->piece_bytes;
+                    char* stage_p = S.buf[sb] + a * range_bytes;
+                    if (whole) {
+                        CU(cudaMemcpyAsync(to_tier ? tier_p : stage_p, to_tier ? stage_p : tier_p,
+                                           (size_t)(z - a) * ctx->block_bytes, cudaMemcpyDefault, S.side));
+                    } else {   // one strip per slot: rows of range_bytes, slot pitch on the tier side
+                        CU(cudaMemcpy2DAsync(to_tier ? tier_p : stage_p,
+                                             to_tier ? (size_t)ctx->block_bytes : (size_t)range_bytes,
+                                             to_tier ? stage_p : tier_p,
+                                             to_tier ? (size_t)range_bytes : (size_t)ctx->block_bytes,
+                                             (size_t)range_bytes, (size_t)(z - a), cudaMemcpyDefault, S.side));
+                    }
                     ctx->stats.memcpy_calls += 1;
                     return EAKV_OK;
                 };
                 if (to_tier) {
                     CU(cudaStreamWaitEvent(stream, S.freed[sb], 0));
-                    rc = launch_copy(ctx, d ? d + i : nullptr, e, cur, S.buf[sb], true, false, true, stream);
+                    rc = launch_copy(ctx, d ? d + i : nullptr, e, cur, S.buf[sb], true, false, true, stream,
+                                     q_first, q_count, stage_cap);
                     if (rc != EAKV_OK) return rc;
                     CU(cudaEventRecord(S.ready[sb], stream));
                     CU(cudaStreamWaitEvent(S.side, S.ready[sb], 0));
@@ -304,7 +326,8 @@ int move_blocks(eakv_ctx* ctx, const std::vector<int2>& ent, bool to_tier, cudaS
                     if (rc != EAKV_OK) return rc;
                     CU(cudaEventRecord(S.ready[sb], S.side));
                     CU(cudaStreamWaitEvent(stream, S.ready[sb], 0));
-                    rc = launch_copy(ctx, d ? d + i : nullptr, e, cur, S.buf[sb], false, false, true, stream);
+                    rc = launch_copy(ctx, d ? d + i : nullptr, e, cur, S.buf[sb], false, false, true, stream,
+                                     q_first, q_count, stage_cap);
                     if (rc != EAKV_OK) return rc;
                     CU(cudaEventRecord(S.freed[sb], stream));
                 }
@@ -803,7 +826,7 @@ int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_m
     if (m == 0) return EAKV_OK;
     DeviceGuard g(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    int rc = move_blocks(ctx, ent, true, stream);
+    int rc = move_blocks(ctx, ent, true, stream, 0, ctx->pieces);
     if (rc != EAKV_OK) return rc;
     ctx->stats.blocks_stored += m;
     ctx->stats.bytes_stored += m * ctx->block_bytes;
@@ -829,10 +852,47 @@ int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_tab
     const int64_t m = n_blocks;
     DeviceGuard g(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    int rc = move_blocks(ctx, ent, false, stream);
+    int rc = move_blocks(ctx, ent, false, stream, 0, ctx->pieces);
     if (rc != EAKV_OK) return rc;
     ctx->stats.blocks_loaded += m;
     ctx->stats.bytes_loaded += m * ctx->block_bytes;
+    return EAKV_OK;
+}
+
+int eakv_load_layers(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_table,
+                     int64_t n_blocks, int32_t layers_per_group, void* const* events,
+                     int32_t n_events, void* cuda_stream) {
+    if (!ctx || n_blocks < 0 || ctx->device < 0 || layers_per_group <= 0) return EAKV_E_INVAL;
+    const int L = ctx->cfg.num_layers;
+    const int groups = (L + layers_per_group - 1) / layers_per_group;
+    if (n_events != groups || (groups > 0 && !events)) return EAKV_E_INVAL;
+    for (int g = 0; g < groups; ++g)
+        if (!events[g]) return EAKV_E_INVAL;
+    if (n_blocks > 0 && (!block_table || !host_slots)) return EAKV_E_INVAL;
+    next_epoch(ctx);
+    std::vector<int2>& ent = ctx->scratch_entries;
+    ent.clear();
+    for (int64_t j = 0; j < n_blocks; ++j) {
+        const int32_t blk = block_table[j], slot = host_slots[j];
+        if (blk < 0 || blk >= ctx->cfg.gpu_blocks || slot < 0 || slot >= ctx->tier_slots)
+            return EAKV_E_RANGE;
+        if (ctx->blk_stamp[blk] == ctx->epoch) return EAKV_E_INVAL;
+        ctx->blk_stamp[blk] = ctx->epoch;
+        ent.push_back(make_int2(blk, slot));
+    }
+    DeviceGuard g(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    for (int grp = 0; grp < groups; ++grp) {
+        const int l0 = grp * layers_per_group;
+        const int l1 = std::min(L, l0 + layers_per_group);
+        if (n_blocks > 0) {
+            int rc = move_blocks(ctx, ent, false, stream, 2 * l0, 2 * (l1 - l0));
+            if (rc != EAKV_OK) return rc;
+        }
+        CU(cudaEventRecord(static_cast<cudaEvent_t>(events[grp]), stream));
+    }
+    ctx->stats.blocks_loaded += n_blocks;
+    ctx->stats.bytes_loaded += n_blocks * ctx->block_bytes;
     return EAKV_OK;
 }
 

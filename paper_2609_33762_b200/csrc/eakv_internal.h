@@ -69,7 +69,10 @@ struct CopyLaunch {
     int64_t n_entries;
     void* const* kv_base;       // device array of 2L piece-array base pointers
     char* tier_base;            // slot-major destination/source
-    int32_t pieces;             // 2L
+    int32_t pieces;             // pieces moved per entry (2L, or a layer group's share)
+    int32_t q_first;            // first pool piece array of the range moved
+    int32_t slot_pieces;        // pieces per slot in the tier-side buffer (2L, or `pieces` for packed staging)
+    int32_t slot_q_first;       // where the range starts inside a slot (q_first, or 0 for packed staging)
     int32_t subs_per_piece;     // ceil(piece_bytes / kCopySubBytes)
     int32_t slot_from_index;    // 1: entry j uses slot j (packed staging buffer) instead of entries[j].y
     int64_t piece_bytes;

@@ -67,7 +67,7 @@ EXPORTS = [
     "eakv_hash_blocks_batched", "eakv_match", "eakv_tier_step", "eakv_gpu_tier_step",
     "eakv_gpu_tier_release", "eakv_store", "eakv_load", "eakv_sync", "eakv_get_stats",
     "eakv_tier_ptr", "eakv_hash_seed", "eakv_hash_base", "eakv_strerror", "eakv_last_cuda_error",
-    "eakv_hash_blocks_static",
+    "eakv_hash_blocks_static", "eakv_load_layers",
 ]
 STATIC_MAX_BLOCKS = 65536
 
@@ -96,6 +96,7 @@ def lib():
     L.eakv_gpu_tier_release.argtypes = [vp, i32]
     L.eakv_store.argtypes = [vp, vp, vp, vp, i64, vp]
     L.eakv_load.argtypes = [vp, vp, vp, i64, vp]
+    L.eakv_load_layers.argtypes = [vp, vp, vp, i64, i32, vp, i32, vp]
     L.eakv_sync.argtypes = [vp]
     L.eakv_get_stats.argtypes = [vp, C.POINTER(Stats)]
     L.eakv_tier_ptr.argtypes = [vp]
@@ -290,6 +291,15 @@ class Context:
         hs, hsp = _np(host_slots, np.int32)
         rc = lib().eakv_load(self._h, hsp, btp, len(bt), _stream(stream))
         self._check(rc, "eakv_load")
+
+    def eakv_load_layers(self, host_slots, block_table, layers_per_group, events, stream=None):
+        """``events``: sequence of cudaEvent_t handles as integers (torch.cuda.Event.cuda_event)."""
+        bt, btp = _np(block_table, np.int32)
+        hs, hsp = _np(host_slots, np.int32)
+        ev = (C.c_void_p * max(len(events), 1))(*[int(e) for e in events])
+        rc = lib().eakv_load_layers(self._h, hsp, btp, len(bt), int(layers_per_group),
+                                    C.cast(ev, C.c_void_p), len(events), _stream(stream))
+        self._check(rc, "eakv_load_layers")
 
     def eakv_sync(self):
         self._check(lib().eakv_sync(self._h), "eakv_sync")

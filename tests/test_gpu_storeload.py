@@ -210,3 +210,53 @@ def test_bad_shapes_rejected_at_create():
         with pytest.raises(e.EakvError) as ei:
             e.Context(**{**base, **patch})
         assert ei.value.code == e.E_INVAL
+
+
+@pytest.mark.parametrize("kw", [
+    dict(tier_location=1, copy_path=1), dict(tier_location=1, copy_path=0),
+    dict(tier_location=0, link_strategy=0),
+    dict(tier_location=0, link_strategy=1, min_staged_run_bytes=-1),
+    dict(tier_location=0, link_strategy=1),
+], ids=["hbm-bulk", "hbm-vector", "host-zero-copy", "host-staged", "host-default"])
+@pytest.mark.parametrize("name,group", [("qwen", 12), ("qwen", 5), ("tiny", 1), ("ragged", 2), ("tiny", 4)])
+def test_layer_pipelined_load(name, group, kw):
+    """eakv_load_layers moves the same bytes as eakv_load, in layer groups, and records one
+    event per group."""
+    e = eakv()
+    shape = SHAPE_CASES[name]
+    nb, kh = (64, 48) if shape.block_bytes <= (1 << 21) else (24, 20)
+    rig = Rig(shape, nb, kh, seed=21, staging_bytes=3 * shape.block_bytes, **kw)
+    rng = rig.rng
+    groups = -(-shape.num_layers // group)
+    events = [torch.cuda.Event() for _ in range(groups)]
+    for ev in events:
+        ev.record()                                   # materialise the handles
+    torch.cuda.synchronize()
+    m = min(nb, kh) - 5
+    src = rng.permutation(kh)[:m].astype(np.int32)
+    dst = rng.permutation(nb)[:m].astype(np.int32)
+    stream = torch.cuda.Stream()
+    rig.ctx.eakv_load_layers(src, dst, group, [ev.cuda_event for ev in events], stream)
+    osl.load(rig.pool_np, rig.tier_np, src, dst)
+    for ev in events:
+        ev.synchronize()
+        assert ev.query()
+    stream.synchronize()
+    rig.check()
+    # contiguous slots (long copy-engine strips), a small call, and an empty one
+    rig.ctx.eakv_load_layers(np.arange(8, dtype=np.int32), np.arange(8, dtype=np.int32)[::-1].copy(),
+                             group, [ev.cuda_event for ev in events], stream)
+    osl.load(rig.pool_np, rig.tier_np, list(range(8)), list(range(8))[::-1])
+    rig.ctx.eakv_load_layers(np.zeros(0, np.int32), np.zeros(0, np.int32), group,
+                             [ev.cuda_event for ev in events], stream)
+    stream.synchronize()
+    rig.check()
+    with pytest.raises(e.EakvError) as ei:            # wrong number of events
+        rig.ctx.eakv_load_layers(src, dst, group, [ev.cuda_event for ev in events] + [events[0].cuda_event], stream)
+    assert ei.value.code == e.E_INVAL
+    with pytest.raises(e.EakvError) as ei:
+        rig.ctx.eakv_load_layers(np.array([0, 1], np.int32), np.array([3, 3], np.int32), group,
+                                 [ev.cuda_event for ev in events], stream)
+    assert ei.value.code == e.E_INVAL
+    rig.check()
+    rig.close()
