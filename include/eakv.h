@@ -242,6 +242,33 @@ int eakv_load_layers(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* bl
                      int64_t n_blocks, int32_t layers_per_group, void* const* events,
                      int32_t n_events, void* cuda_stream);
 
+/* Reuse (stack) distances of a reference stream (Section 3.2, Eq. 4): dist[i] = number of
+ * distinct other keys referenced strictly between reference i and the previous reference to
+ * the same key, or -1 on a first reference.  Under a fully associative LRU tier of K chunks
+ * that admits every miss, reference i hits iff 0 <= dist[i] < K.
+ *   keys_dev device uint64[n_refs] (values below 2^61); dist_dev device int64[n_refs] (written)
+ * Context-free.  Allocates its scratch (about (4 * ceil(log2 n) + 40) bytes per reference) with
+ * cudaMalloc and frees it before returning; returns after the stream has finished the work.
+ * n_refs < 2^31 - 16.  Errors: EAKV_E_INVAL, EAKV_E_CUDA (allocation or launch failure). */
+int eakv_reuse_distances(const uint64_t* keys_dev, int64_t n_refs, int64_t* dist_dev,
+                         void* cuda_stream);
+
+/* Capacity curve from reuse distances (Appendix C "Prefix coverage from a reference stream"):
+ * for every capacity K_c, hits = #{i : 0 <= dist[i] < K_c}; per request j (references
+ * req_offsets[j] .. req_offsets[j+1]) the host coverage H_j is its leading run of hits,
+ * restored += max(0, H_j - G_j) blocks and computed += n_j - max(G_j, H_j) * block_size tokens.
+ *   dist_dev device int64[n_refs]; req_offsets_host int64[n_requests + 1] (0 .. n_refs);
+ *   req_tokens_host, req_gpu_prefix_host int64[n_requests] (n_j and G_j in blocks);
+ *   capacities_host int64[n_capacities], n_capacities <= 64;
+ *   hits_out, restored_out, computed_out host int64[n_capacities];
+ *   cover_out host int64[n_capacities][n_requests] (H_j per capacity) or NULL.
+ * Context-free, allocates and frees its small scratch, returns after the work is done. */
+int eakv_capacity_curve(const int64_t* dist_dev, int64_t n_refs, const int64_t* req_offsets_host,
+                        const int64_t* req_tokens_host, const int64_t* req_gpu_prefix_host,
+                        int64_t n_requests, int32_t block_size, const int64_t* capacities_host,
+                        int32_t n_capacities, int64_t* hits_out, int64_t* restored_out,
+                        int64_t* computed_out, int64_t* cover_out, void* cuda_stream);
+
 /* Block keys without a context and without any allocation.  (The paper has no counterpart;
  * this exists for callers that cannot request device memory: code living inside a serving
  * process whose engine has already claimed the GPU's memory, where an allocation may fail or

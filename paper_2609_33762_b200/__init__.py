@@ -5,4 +5,4 @@ sm_100a plus a C++ control plane); ``harness`` drives whole agent turns through 
 PyTorch used only for device memory and streams.  Importing this package loads nothing;
 ``eakv.lib()`` loads the shared library and fails loudly when it has not been built.
 """
-__all__ = ["eakv", "build", "harness"]
+__all__ = ["eakv", "build", "harness", "replay", "capacity", "multi"]

@@ -7,7 +7,8 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libeakv.so")
-SOURCES = ["eakv_api.cu", "hash_kernels.cu", "copy_kernels.cu", "control_plane.cpp"]
+SOURCES = ["eakv_api.cu", "hash_kernels.cu", "copy_kernels.cu", "stackdist_kernels.cu",
+           "control_plane.cpp"]
 HEADERS = ["eakv_internal.h", "control_plane.h", os.path.join("..", "..", "include", "eakv.h")]
 
 

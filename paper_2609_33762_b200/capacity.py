@@ -1,0 +1,131 @@
+"""Capacity model of a trace on the GPU (the paper's stack-distance model, Section 3.2 and
+Appendix C): predicted computed prefill and restored volume for a sweep of host-tier sizes,
+and the working-set sizes that go with them.
+
+    python -m paper_2609_33762_b200.capacity --config c2 --host-gib 8,16,32,64,128,256
+
+The reference stream (every request references the full blocks of its prompt, in request
+order) is built from one batched hash launch: prompts only grow by appends, so a request's
+keys are a prefix of its agent's final key list.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import time
+
+import numpy as np
+
+from . import eakv
+
+GIB = 1 << 30
+
+
+def reference_stream(trace, shape, device="cuda:0"):
+    """(stream keys on the device as int64 tensor, request offsets, request tokens, host keys)."""
+    import torch
+    b = shape.block_size
+    agents = sorted(trace.agent_tokens)
+    lens = [len(trace.agent_tokens[a]) for a in agents]
+    # pad every agent's tokens to a multiple of 4 so each prompt starts 16-byte aligned
+    starts, cur = [], 0
+    for n in lens:
+        starts.append(cur)
+        cur += (n + 3) // 4 * 4
+    flat = np.zeros(cur, dtype=np.int32)
+    for a, s0, n in zip(agents, starts, lens):
+        flat[s0:s0 + n] = trace.agent_tokens[a]
+    # one launch per agent (each agent's final prompt once)
+    tok_dev = torch.from_numpy(flat).to(device)
+    ctx = eakv.Context(num_layers=1, kv_heads=1, head_dim=8, block_size=b, gpu_blocks=1, host_blocks=1,
+                       kv_base=[tok_dev.data_ptr(), tok_dev.data_ptr()], tier_location=eakv.TIER_DEVICE,
+                       tier_memory=tok_dev.data_ptr(), hash_scratch_blocks=max(1, cur // b + len(agents)))
+    agent_keys = {}
+    seed = ctx.eakv_hash_seed()
+    for a, s0, n in zip(agents, starts, lens):
+        nblk = n // b
+        out = torch.empty(max(nblk, 1), dtype=torch.int64, device=device)
+        ctx.eakv_hash_blocks(tok_dev.data_ptr() + 4 * s0, n, seed, out.data_ptr())
+        agent_keys[a] = out[:nblk]
+    torch.cuda.synchronize()
+    ctx.close()
+    pieces, offsets, tokens = [], [0], []
+    for r in trace.requests:
+        nblk = r.n_tokens // b
+        pieces.append(agent_keys[r.agent][:nblk])
+        offsets.append(offsets[-1] + nblk)
+        tokens.append(r.n_tokens)
+    stream = torch.cat(pieces) if pieces else torch.empty(0, dtype=torch.int64, device=device)
+    return stream, np.asarray(offsets, dtype=np.int64), np.asarray(tokens, dtype=np.int64)
+
+
+def gpu_prefixes(trace, shape, gpu_blocks, stream_host, offsets):
+    """G_j of every request from the library's GPU-tier bookkeeping (control plane only)."""
+    b = shape.block_size
+    ctx = eakv.Context(num_layers=1, kv_heads=1, head_dim=8, block_size=b, gpu_blocks=gpu_blocks,
+                       host_blocks=1, kv_base=None, control_plane_only=True)
+    G = np.zeros(len(trace.requests), dtype=np.int64)
+    for j, r in enumerate(trace.requests):
+        keys = stream_host[offsets[j]:offsets[j + 1]]
+        G[j] = ctx.eakv_match(keys)[0]
+        _, _, tail = ctx.eakv_gpu_tier_step(keys, r.n_tokens % b != 0)
+        if tail >= 0:
+            ctx.eakv_gpu_tier_release(tail)
+    ctx.close()
+    return G
+
+
+def model(config, host_gib, device="cuda:0", limit=None):
+    import torch
+    from eakv_workloads import CONFIGS, SHAPES, make_trace
+    cfg = CONFIGS[config]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg)
+    if limit:
+        trace.requests = trace.requests[:limit]
+    t0 = time.perf_counter()
+    stream, offsets, tokens = reference_stream(trace, shape, device)
+    t_stream = time.perf_counter() - t0
+    n_refs = int(offsets[-1])
+    dist = torch.empty(max(n_refs, 1), dtype=torch.int64, device=device)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    eakv.eakv_reuse_distances(stream.data_ptr(), n_refs, dist.data_ptr())
+    t_dist = time.perf_counter() - t0
+    stream_host = stream.cpu().numpy().view(np.uint64)
+    G = gpu_prefixes(trace, shape, cfg.gpu_blocks, stream_host, offsets)
+    caps = [max(1, int(g * GIB // shape.block_bytes)) for g in host_gib] + [1 << 40]
+    t0 = time.perf_counter()
+    out = eakv.eakv_capacity_curve(dist.data_ptr(), n_refs, offsets, tokens, G, shape.block_size, caps)
+    t_curve = time.perf_counter() - t0
+    finite = dist[:n_refs][dist[:n_refs] >= 0]
+    ws_full = int(finite.max().item()) + 1 if finite.numel() else 0
+    n_mean = trace.total_prompt_tokens / len(trace.requests)
+    ws_eq5 = int((len(trace.agent_tokens) - 1) * n_mean * shape.bytes_per_token // shape.block_bytes)
+    inf_computed = int(out["computed_tokens"][-1])
+    rows = []
+    for c, g in enumerate(host_gib):
+        rows.append({"host_gib": g, "blocks": caps[c], "hits": int(out["hits"][c]),
+                     "restored_tokens": int(out["restored_blocks"][c]) * shape.block_size,
+                     "computed_prefill_tokens": int(out["computed_tokens"][c])})
+    return {"config": config, "requests": len(trace.requests), "references": n_refs,
+            "prompt_tokens": int(tokens.sum()), "rows": rows,
+            "computed_prefill_tokens_infinite_tier": inf_computed,
+            "working_set_blocks": {"eq5": ws_eq5, "full": ws_full},
+            "working_set_gib": {"eq5": ws_eq5 * shape.block_bytes / GIB, "full": ws_full * shape.block_bytes / GIB},
+            "seconds": {"stream": t_stream, "distances": t_dist, "curve": t_curve},
+            "distance_refs_per_s": n_refs / t_dist if t_dist > 0 else None}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", default="c2", choices=["c0", "c0_big_tier", "c2", "c3", "c4"])
+    ap.add_argument("--host-gib", default="8,16,32,64,128,256")
+    ap.add_argument("--limit", type=int, default=None)
+    args = ap.parse_args()
+    out = model(args.config, [float(x) for x in args.host_gib.split(",")], limit=args.limit)
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

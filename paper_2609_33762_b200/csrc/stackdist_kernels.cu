@@ -1,0 +1,382 @@
+// Stack-distance capacity model on the GPU (Section 3.2, Eq. 4; Appendix C "Prefix coverage
+// from a reference stream").
+//
+// Reuse distance of reference i with previous reference p to the same chunk: the number of
+// distinct other chunks referenced strictly between them.  A position j in (p, i) is the
+// first reference to its chunk inside that window exactly when its own previous reference lies
+// before p, and every j <= p trivially has prev_j < p, so
+//
+//     D_i = #{ j < i : prev_j < p } - (p + 1).
+//
+// Steps, all data-parallel:
+//   1. prev[]: stable sort of (key, position) pairs by key (CUB radix sort, the one library
+//      primitive used here); equal neighbours give each position its predecessor.
+//   2. a wavelet matrix over v_j = prev_j + 1 (one stable 0/1 partition per bit, built with a
+//      three-kernel exclusive scan per level: no kernel waits for another);
+//   3. one "count of values below x in a prefix" query per reference, nbits steps each.
+// The capacity curve then needs only D: a reference hits a tier of K chunks iff D < K
+// (Mattson); a request's host coverage is its leading run of hits; restored = max(0, H - G);
+// computed prefill = n - max(G, H) * b.
+#include <cub/device/device_radix_sort.cuh>
+
+#include <algorithm>
+#include <cstdint>
+#include <vector>
+
+#include "../../include/eakv.h"
+
+namespace eakv {
+
+constexpr int kSdThreads = 256;
+constexpr int kSdItems = 4;                         // elements per thread in the scan kernels
+constexpr int kSdTile = kSdThreads * kSdItems;      // 1024 elements per CTA
+
+// ---- step 1 ---------------------------------------------------------------------------------
+__global__ void iota_kernel(int32_t* idx, int64_t n) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) idx[i] = (int32_t)i;
+}
+
+// sorted by (key, position): the predecessor of a position is its left neighbour with the same key
+__global__ void prev_from_sorted_kernel(const uint64_t* __restrict__ keys_sorted,
+                                        const int32_t* __restrict__ idx_sorted, int64_t n,
+                                        int32_t* __restrict__ prev, uint32_t* __restrict__ v) {
+    const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= n) return;
+    const int32_t i = idx_sorted[s];
+    const int32_t p = (s > 0 && keys_sorted[s - 1] == keys_sorted[s]) ? idx_sorted[s - 1] : -1;
+    prev[i] = p;
+    v[i] = (uint32_t)(p + 1);
+}
+
+// ---- step 2: one wavelet-matrix level = stable partition by one bit -------------------------
+// pass A: zeros per tile
+__global__ void __launch_bounds__(kSdThreads)
+wm_count_kernel(const uint32_t* __restrict__ a, int64_t n, int shift, int32_t* __restrict__ tile_zeros) {
+    __shared__ int warp_sum[kSdThreads / 32];
+    const int64_t base = (int64_t)blockIdx.x * kSdTile;
+    int z = 0;
+#pragma unroll
+    for (int k = 0; k < kSdItems; ++k) {
+        const int64_t i = base + (int64_t)threadIdx.x * kSdItems + k;
+        if (i < n) z += ((a[i] >> shift) & 1u) ^ 1u;
+    }
+    for (int d = 16; d; d >>= 1) z += __shfl_xor_sync(0xffffffffu, z, d);
+    if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = z;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int t = 0;
+        for (int w = 0; w < kSdThreads / 32; ++w) t += warp_sum[w];
+        tile_zeros[blockIdx.x] = t;
+    }
+}
+
+// pass B: exclusive scan of the tile counts by one CTA (in place), total to *total_zeros
+__global__ void __launch_bounds__(1024)
+wm_scan_tiles_kernel(int32_t* __restrict__ tile_zeros, int n_tiles, int32_t* __restrict__ total_zeros) {
+    __shared__ int warp_tot[32];
+    __shared__ int carry_s;
+    if (threadIdx.x == 0) carry_s = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int base = 0; base < n_tiles; base += 1024) {
+        const int i = base + threadIdx.x;
+        const int x = i < n_tiles ? tile_zeros[i] : 0;
+        int inc = x;
+        for (int d = 1; d < 32; d <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, inc, d);
+            if (lane >= d) inc += up;
+        }
+        if (lane == 31) warp_tot[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            int w = warp_tot[lane];
+            for (int d = 1; d < 32; d <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, w, d);
+                if (lane >= d) w += up;
+            }
+            warp_tot[lane] = w;
+        }
+        __syncthreads();
+        const int carry = carry_s;
+        const int excl = carry + (warp ? warp_tot[warp - 1] : 0) + inc - x;
+        if (i < n_tiles) tile_zeros[i] = excl;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry_s = carry + warp_tot[31];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *total_zeros = carry_s;
+}
+
+// pass C: zeros-before for every position, and the scatter into the next level's order
+__global__ void __launch_bounds__(kSdThreads)
+wm_scatter_kernel(const uint32_t* __restrict__ a, int64_t n, int shift,
+                  const int32_t* __restrict__ tile_excl, const int32_t* __restrict__ total_zeros,
+                  int32_t* __restrict__ zeros_before /* [n + 1] */, uint32_t* __restrict__ a_next) {
+    __shared__ int warp_tot[kSdThreads / 32];
+    const int64_t base = (int64_t)blockIdx.x * kSdTile + (int64_t)threadIdx.x * kSdItems;
+    uint32_t val[kSdItems];
+    int isz[kSdItems];
+    int mine = 0;
+#pragma unroll
+    for (int k = 0; k < kSdItems; ++k) {
+        const int64_t i = base + k;
+        val[k] = i < n ? a[i] : 0xffffffffu;
+        isz[k] = (i < n) ? (int)(((val[k] >> shift) & 1u) ^ 1u) : 0;
+        mine += isz[k];
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = mine;
+    for (int d = 1; d < 32; d <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, inc, d);
+        if (lane >= d) inc += up;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    int before = tile_excl[blockIdx.x] + inc - mine;
+    for (int w = 0; w < warp; ++w) before += warp_tot[w];
+    const int z_total = *total_zeros;
+#pragma unroll
+    for (int k = 0; k < kSdItems; ++k) {
+        const int64_t i = base + k;
+        if (i < n) {
+            zeros_before[i] = before;
+            const int64_t dst = isz[k] ? (int64_t)before : (int64_t)z_total + (i - before);
+            a_next[dst] = val[k];
+            before += isz[k];
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) zeros_before[n] = z_total;   // zeros in the whole level
+}
+
+// ---- step 3 ---------------------------------------------------------------------------------
+// dist[i] = #{ j < i : v_j < p + 1 } - (p + 1), or -1 on a first reference
+__global__ void reuse_distance_kernel(const int32_t* __restrict__ prev, int64_t n, int nbits,
+                                      const int32_t* __restrict__ zeros_before /* [nbits][n+1] */,
+                                      const int32_t* __restrict__ level_zeros /* [nbits] */,
+                                      int64_t* __restrict__ dist) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int32_t p = prev[i];
+    if (p < 0) {
+        dist[i] = -1;
+        return;
+    }
+    const uint32_t x = (uint32_t)p + 1u;
+    int64_t lo = 0, hi = i, count = 0;
+    for (int l = 0; l < nbits; ++l) {
+        const int32_t* zb = zeros_before + (int64_t)l * (n + 1);
+        const int64_t z_lo = zb[lo], z_hi = zb[hi];
+        if ((x >> (nbits - 1 - l)) & 1u) {
+            count += z_hi - z_lo;
+            const int64_t z = level_zeros[l];
+            lo = z + (lo - z_lo);
+            hi = z + (hi - z_hi);
+        } else {
+            lo = z_lo;
+            hi = z_hi;
+        }
+    }
+    dist[i] = count - ((int64_t)p + 1);
+}
+
+// ---- capacity curve ---------------------------------------------------------------------------
+// hits[c] += #{ i : 0 <= D_i < K_c }
+__global__ void curve_hits_kernel(const int64_t* __restrict__ dist, int64_t n,
+                                  const int64_t* __restrict__ caps, int n_caps,
+                                  unsigned long long* __restrict__ hits) {
+    extern __shared__ unsigned long long sh[];
+    for (int c = threadIdx.x; c < n_caps; c += blockDim.x) sh[c] = 0;
+    __syncthreads();
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t d = dist[i];
+        if (d < 0) continue;
+        for (int c = 0; c < n_caps; ++c)
+            if (d < caps[c]) atomicAdd(&sh[c], 1ull);
+    }
+    __syncthreads();
+    for (int c = threadIdx.x; c < n_caps; c += blockDim.x)
+        if (sh[c]) atomicAdd(&hits[c], sh[c]);
+}
+
+// one CTA per request: running maximum of D over the request's references (a first reference
+// counts as infinite), coverage H(K) = references before the maximum reaches K
+__global__ void __launch_bounds__(kSdThreads)
+curve_cover_kernel(const int64_t* __restrict__ dist, const int64_t* __restrict__ req_off,
+                   const int64_t* __restrict__ req_tokens, const int64_t* __restrict__ req_gpu,
+                   int64_t n_req, int block_size, const int64_t* __restrict__ caps, int n_caps,
+                   unsigned long long* __restrict__ restored, unsigned long long* __restrict__ computed,
+                   int64_t* __restrict__ cover /* [n_caps][n_req] or NULL */) {
+    __shared__ long long warp_max[kSdThreads / 32];
+    __shared__ long long carry_s;
+    __shared__ int cnt[64];
+    const int64_t r = blockIdx.x;
+    if (r >= n_req) return;
+    const int64_t lo = req_off[r], hi = req_off[r + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) carry_s = -1;
+    for (int c = threadIdx.x; c < n_caps; c += blockDim.x) cnt[c] = 0;
+    __syncthreads();
+    const long long INF = 0x7fffffffffffffffLL;
+    for (int64_t base = lo; base < hi; base += kSdThreads) {
+        const int64_t i = base + threadIdx.x;
+        long long m = -1;
+        if (i < hi) {
+            const long long d = dist[i];
+            m = d < 0 ? INF : d;
+        }
+        for (int d = 1; d < 32; d <<= 1) {
+            const long long up = __shfl_up_sync(0xffffffffu, m, d);
+            if (lane >= d) m = max(m, up);
+        }
+        if (lane == 31) warp_max[warp] = m;
+        __syncthreads();
+        long long pm = max(m, carry_s);
+        for (int w = 0; w < warp; ++w) pm = max(pm, warp_max[w]);
+        if (i < hi) {
+            for (int c = 0; c < n_caps; ++c)
+                if (pm < caps[c]) atomicAdd(&cnt[c], 1);
+        }
+        __syncthreads();
+        if (threadIdx.x == kSdThreads - 1) carry_s = pm;
+        __syncthreads();
+    }
+    if (threadIdx.x < n_caps) {
+        const int c = threadIdx.x;
+        const long long H = cnt[c], G = req_gpu[r], n = req_tokens[r];
+        if (cover) cover[(int64_t)c * n_req + r] = H;
+        if (H > G) atomicAdd(&restored[c], (unsigned long long)(H - G));
+        atomicAdd(&computed[c], (unsigned long long)(n - max(G, H) * (long long)block_size));
+    }
+}
+
+}  // namespace eakv
+
+using namespace eakv;
+
+#define SD_CU(call)                           \
+    do {                                      \
+        cudaError_t _e = (call);              \
+        if (_e != cudaSuccess) {              \
+            rc = EAKV_E_CUDA;                 \
+            goto done;                        \
+        }                                     \
+    } while (0)
+
+extern "C" int eakv_reuse_distances(const uint64_t* keys_dev, int64_t n_refs, int64_t* dist_dev,
+                                    void* cuda_stream) {
+    if (n_refs < 0 || n_refs > 0x7ffffff0LL) return EAKV_E_INVAL;
+    if (n_refs == 0) return EAKV_OK;
+    if (!keys_dev || !dist_dev) return EAKV_E_INVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t n = n_refs;
+    int nbits = 1;
+    while ((1ll << nbits) <= n) ++nbits;               // values v in [0, n] fit in nbits bits
+    const int n_tiles = (int)((n + kSdTile - 1) / kSdTile);
+    const int grid1 = (int)((n + 255) / 256);
+
+    int rc = EAKV_OK;
+    uint64_t* keys_sorted = nullptr;
+    int32_t *idx = nullptr, *idx_sorted = nullptr, *prev = nullptr, *zeros_before = nullptr;
+    int32_t *tile_zeros = nullptr, *level_zeros = nullptr;
+    uint32_t *va = nullptr, *vb = nullptr;
+    void* sort_tmp = nullptr;
+    size_t sort_bytes = 0;
+
+    SD_CU(cudaMalloc(&keys_sorted, n * 8));
+    SD_CU(cudaMalloc(&idx, n * 4));
+    SD_CU(cudaMalloc(&idx_sorted, n * 4));
+    SD_CU(cudaMalloc(&prev, n * 4));
+    SD_CU(cudaMalloc(&va, n * 4));
+    SD_CU(cudaMalloc(&vb, n * 4));
+    SD_CU(cudaMalloc(&zeros_before, (size_t)nbits * (n + 1) * 4));
+    SD_CU(cudaMalloc(&tile_zeros, (size_t)n_tiles * 4));
+    SD_CU(cudaMalloc(&level_zeros, (size_t)nbits * 4));
+    SD_CU(cub::DeviceRadixSort::SortPairs(nullptr, sort_bytes, keys_dev, keys_sorted, idx, idx_sorted,
+                                          (int)n, 0, 61, stream));
+    SD_CU(cudaMalloc(&sort_tmp, sort_bytes));
+
+    iota_kernel<<<grid1, 256, 0, stream>>>(idx, n);
+    SD_CU(cub::DeviceRadixSort::SortPairs(sort_tmp, sort_bytes, keys_dev, keys_sorted, idx, idx_sorted,
+                                          (int)n, 0, 61, stream));
+    prev_from_sorted_kernel<<<grid1, 256, 0, stream>>>(keys_sorted, idx_sorted, n, prev, va);
+    for (int l = 0; l < nbits; ++l) {
+        const int shift = nbits - 1 - l;
+        uint32_t* a = (l & 1) ? vb : va;
+        uint32_t* a_next = (l & 1) ? va : vb;
+        wm_count_kernel<<<n_tiles, kSdThreads, 0, stream>>>(a, n, shift, tile_zeros);
+        wm_scan_tiles_kernel<<<1, 1024, 0, stream>>>(tile_zeros, n_tiles, level_zeros + l);
+        wm_scatter_kernel<<<n_tiles, kSdThreads, 0, stream>>>(a, n, shift, tile_zeros, level_zeros + l,
+                                                             zeros_before + (int64_t)l * (n + 1), a_next);
+    }
+    reuse_distance_kernel<<<grid1, 256, 0, stream>>>(prev, n, nbits, zeros_before, level_zeros, dist_dev);
+    SD_CU(cudaGetLastError());
+    SD_CU(cudaStreamSynchronize(stream));
+done:
+    cudaFree(keys_sorted); cudaFree(idx); cudaFree(idx_sorted); cudaFree(prev); cudaFree(va);
+    cudaFree(vb); cudaFree(zeros_before); cudaFree(tile_zeros); cudaFree(level_zeros);
+    cudaFree(sort_tmp);
+    if (rc != EAKV_OK) cudaGetLastError();
+    return rc;
+}
+
+extern "C" int eakv_capacity_curve(const int64_t* dist_dev, int64_t n_refs,
+                                   const int64_t* req_offsets_host, const int64_t* req_tokens_host,
+                                   const int64_t* req_gpu_prefix_host, int64_t n_requests,
+                                   int32_t block_size, const int64_t* capacities_host,
+                                   int32_t n_capacities, int64_t* hits_out, int64_t* restored_out,
+                                   int64_t* computed_out, int64_t* cover_out, void* cuda_stream) {
+    if (n_refs < 0 || n_requests < 0 || n_capacities <= 0 || n_capacities > 64 || block_size <= 0)
+        return EAKV_E_INVAL;
+    if (!req_offsets_host || !capacities_host || !hits_out || !restored_out || !computed_out)
+        return EAKV_E_INVAL;
+    if (n_requests > 0 && (!req_tokens_host || !req_gpu_prefix_host)) return EAKV_E_INVAL;
+    if (n_refs > 0 && !dist_dev) return EAKV_E_INVAL;
+    if (req_offsets_host[0] != 0 || req_offsets_host[n_requests] != n_refs) return EAKV_E_INVAL;
+    for (int64_t r = 0; r < n_requests; ++r)
+        if (req_offsets_host[r + 1] < req_offsets_host[r]) return EAKV_E_INVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int rc = EAKV_OK;
+    int64_t *d_off = nullptr, *d_tok = nullptr, *d_gpu = nullptr, *d_caps = nullptr, *d_cover = nullptr;
+    unsigned long long* d_out = nullptr;     // hits | restored | computed
+    std::vector<unsigned long long> out(3 * (size_t)n_capacities);
+    const int C = n_capacities;
+
+    SD_CU(cudaMalloc(&d_off, (n_requests + 1) * 8));
+    SD_CU(cudaMalloc(&d_tok, std::max<int64_t>(n_requests, 1) * 8));
+    SD_CU(cudaMalloc(&d_gpu, std::max<int64_t>(n_requests, 1) * 8));
+    SD_CU(cudaMalloc(&d_caps, C * 8));
+    SD_CU(cudaMalloc(&d_out, 3 * C * 8));
+    if (cover_out) SD_CU(cudaMalloc(&d_cover, std::max<int64_t>((int64_t)C * n_requests, 1) * 8));
+    SD_CU(cudaMemcpyAsync(d_off, req_offsets_host, (n_requests + 1) * 8, cudaMemcpyHostToDevice, stream));
+    if (n_requests) {
+        SD_CU(cudaMemcpyAsync(d_tok, req_tokens_host, n_requests * 8, cudaMemcpyHostToDevice, stream));
+        SD_CU(cudaMemcpyAsync(d_gpu, req_gpu_prefix_host, n_requests * 8, cudaMemcpyHostToDevice, stream));
+    }
+    SD_CU(cudaMemcpyAsync(d_caps, capacities_host, C * 8, cudaMemcpyHostToDevice, stream));
+    SD_CU(cudaMemsetAsync(d_out, 0, 3 * C * 8, stream));
+    if (n_refs > 0) {
+        const int grid = (int)std::min<int64_t>((n_refs + 255) / 256, 148 * 8);
+        curve_hits_kernel<<<grid, 256, C * 8, stream>>>(dist_dev, n_refs, d_caps, C, d_out);
+    }
+    if (n_requests > 0) {
+        curve_cover_kernel<<<(unsigned)n_requests, kSdThreads, 0, stream>>>(
+            dist_dev, d_off, d_tok, d_gpu, n_requests, block_size, d_caps, C, d_out + C, d_out + 2 * C,
+            d_cover);
+    }
+    SD_CU(cudaGetLastError());
+    SD_CU(cudaMemcpyAsync(out.data(), d_out, 3 * C * 8, cudaMemcpyDeviceToHost, stream));
+    if (cover_out && n_requests)
+        SD_CU(cudaMemcpyAsync(cover_out, d_cover, (size_t)C * n_requests * 8, cudaMemcpyDeviceToHost, stream));
+    SD_CU(cudaStreamSynchronize(stream));
+    for (int c = 0; c < C; ++c) {
+        hits_out[c] = (int64_t)out[c];
+        restored_out[c] = (int64_t)out[C + c];
+        computed_out[c] = (int64_t)out[2 * C + c];
+    }
+done:
+    cudaFree(d_off); cudaFree(d_tok); cudaFree(d_gpu); cudaFree(d_caps); cudaFree(d_out); cudaFree(d_cover);
+    if (rc != EAKV_OK) cudaGetLastError();
+    return rc;
+}

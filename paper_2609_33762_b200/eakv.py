@@ -67,7 +67,7 @@ EXPORTS = [
     "eakv_hash_blocks_batched", "eakv_match", "eakv_tier_step", "eakv_gpu_tier_step",
     "eakv_gpu_tier_release", "eakv_store", "eakv_load", "eakv_sync", "eakv_get_stats",
     "eakv_tier_ptr", "eakv_hash_seed", "eakv_hash_base", "eakv_strerror", "eakv_last_cuda_error",
-    "eakv_hash_blocks_static", "eakv_load_layers",
+    "eakv_hash_blocks_static", "eakv_load_layers", "eakv_reuse_distances", "eakv_capacity_curve",
 ]
 STATIC_MAX_BLOCKS = 65536
 
@@ -97,6 +97,8 @@ def lib():
     L.eakv_store.argtypes = [vp, vp, vp, vp, i64, vp]
     L.eakv_load.argtypes = [vp, vp, vp, i64, vp]
     L.eakv_load_layers.argtypes = [vp, vp, vp, i64, i32, vp, i32, vp]
+    L.eakv_reuse_distances.argtypes = [vp, i64, vp, vp]
+    L.eakv_capacity_curve.argtypes = [vp, i64, vp, vp, vp, i64, i32, vp, i32, vp, vp, vp, vp, vp]
     L.eakv_sync.argtypes = [vp]
     L.eakv_get_stats.argtypes = [vp, C.POINTER(Stats)]
     L.eakv_tier_ptr.argtypes = [vp]
@@ -135,6 +137,36 @@ def eakv_hash_blocks_static(tokens_dev, n_tokens, block_size, hash_base, parent_
     if rc != OK:
         raise EakvError(rc, "eakv_hash_blocks_static")
     return n.value
+
+
+def eakv_reuse_distances(keys_dev, n_refs, dist_dev, stream=None):
+    """Reuse distances of the uint64 keys at device address ``keys_dev`` into int64 ``dist_dev``
+    (-1 = first reference)."""
+    rc = lib().eakv_reuse_distances(C.c_void_p(int(keys_dev)), int(n_refs), C.c_void_p(int(dist_dev)),
+                                    _stream(stream))
+    if rc != OK:
+        raise EakvError(rc, "eakv_reuse_distances")
+
+
+def eakv_capacity_curve(dist_dev, n_refs, req_offsets, req_tokens, req_gpu_prefix, block_size,
+                        capacities, want_cover=False, stream=None):
+    """Hits, restored blocks and computed tokens per capacity (and H_j per request if asked)."""
+    off, offp = _np(req_offsets, np.int64)
+    tok, tokp = _np(req_tokens, np.int64)
+    gpu, gpup = _np(req_gpu_prefix, np.int64)
+    caps, capsp = _np(capacities, np.int64)
+    J, Cn = len(off) - 1, len(caps)
+    hits = np.zeros(Cn, dtype=np.int64)
+    restored = np.zeros(Cn, dtype=np.int64)
+    computed = np.zeros(Cn, dtype=np.int64)
+    cover = np.zeros((Cn, J), dtype=np.int64) if want_cover else None
+    vp = lambda a: a.ctypes.data_as(C.c_void_p)
+    rc = lib().eakv_capacity_curve(C.c_void_p(int(dist_dev)), int(n_refs), offp, tokp, gpup, J,
+                                   int(block_size), capsp, Cn, vp(hits), vp(restored), vp(computed),
+                                   vp(cover) if want_cover else None, _stream(stream))
+    if rc != OK:
+        raise EakvError(rc, "eakv_capacity_curve")
+    return dict(hits=hits, restored_blocks=restored, computed_tokens=computed, cover=cover)
 
 
 class Context:
