@@ -117,13 +117,81 @@ def model(config, host_gib, device="cuda:0", limit=None):
             "distance_refs_per_s": n_refs / t_dist if t_dist > 0 else None}
 
 
+def audit(config, policy, host_gib, kappa=None, chunk_blocks=1, device="cuda:0", limit=None):
+    """Declined-chunk audit (Appendix D): run the tier bookkeeping under an admission policy,
+    then ask of every declined chunk whether its next reference lies beyond the tier's reach
+    (reuse distance D >= K_H from the GPU model) or never comes."""
+    import torch
+    from eakv_workloads import CONFIGS, SHAPES, make_trace
+    from .replay import POLICIES
+    cfg = CONFIGS[config]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg)
+    if limit:
+        trace.requests = trace.requests[:limit]
+    R = max(1, chunk_blocks)
+    b = shape.block_size
+    stream, offsets, tokens = reference_stream(trace, shape, device)
+    keys_host = stream.cpu().numpy().view(np.uint64)
+    # the tier's own reference stream: one key per full chunk
+    chunk_keys, chunk_off = [], [0]
+    for j in range(len(trace.requests)):
+        k = keys_host[offsets[j]:offsets[j + 1]][R - 1::R]
+        chunk_keys.append(k)
+        chunk_off.append(chunk_off[-1] + len(k))
+    cstream = np.concatenate(chunk_keys) if chunk_keys else np.zeros(0, np.uint64)
+    kh = max(1, int(host_gib * GIB // (R * shape.block_bytes)))
+    kap = cfg.kappa_blocks if kappa is None else kappa
+    ctx = eakv.Context(num_layers=1, kv_heads=1, head_dim=8, block_size=b, gpu_blocks=1, host_blocks=kh,
+                       kv_base=None, control_plane_only=True, policy=POLICIES[policy],
+                       kappa_blocks=kap, chunk_blocks=R)
+    declined = np.zeros(len(cstream), dtype=bool)
+    for j, r in enumerate(trace.requests):
+        st = ctx.eakv_tier_step(chunk_keys[j], r.agent, r.n_tokens, r.time_ms)
+        declined[chunk_off[j]:chunk_off[j + 1]] = (st["hit"] == 0) & (st["admit"] == 0)
+    stats = ctx.eakv_get_stats()
+    ctx.close()
+    n = len(cstream)
+    cdev = torch.from_numpy(cstream.view(np.int64)).to(device)
+    dist = torch.empty(max(n, 1), dtype=torch.int64, device=device)
+    eakv.eakv_reuse_distances(cdev.data_ptr(), n, dist.data_ptr())
+    D = dist[:n].cpu().numpy()
+    # next reference of every position: stable sort by key, neighbours to the right
+    order = np.argsort(cstream, kind="stable")
+    nxt = np.full(n, -1, dtype=np.int64)
+    same = cstream[order][1:] == cstream[order][:-1]
+    nxt[order[:-1][same]] = order[1:][same]
+    idx = np.nonzero(declined)[0]
+    nx = nxt[idx]
+    never = int((nx < 0).sum())
+    d_next = D[nx[nx >= 0]]
+    meets = never + int((d_next >= kh).sum())
+    return {"config": config, "policy": policy, "host_gib": host_gib, "tier_units": kh, "chunk_blocks": R,
+            "kappa": kap, "declined_chunks": int(len(idx)), "meet_condition": meets,
+            "share_meeting_condition": meets / len(idx) if len(idx) else None,
+            "never_referenced_again": never,
+            "median_distance_over_capacity": float(np.median(d_next / kh)) if len(d_next) else None,
+            "declined_requests": stats["declined_requests"], "pressure_requests": stats["pressure_requests"],
+            "admitted_chunks": stats["admitted"]}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", default="c2", choices=["c0", "c0_big_tier", "c2", "c3", "c4"])
     ap.add_argument("--host-gib", default="8,16,32,64,128,256")
     ap.add_argument("--limit", type=int, default=None)
+    ap.add_argument("--audit", default=None, choices=["fixed", "conditioned"],
+                    help="declined-chunk audit under this policy instead of the capacity sweep")
+    ap.add_argument("--chunk-blocks", type=int, default=1)
+    ap.add_argument("--kappa", type=int, default=None)
     args = ap.parse_args()
-    out = model(args.config, [float(x) for x in args.host_gib.split(",")], limit=args.limit)
+    gib = [float(x) for x in args.host_gib.split(",")]
+    if args.audit:
+        for g in gib:
+            print(json.dumps(audit(args.config, args.audit, g, kappa=args.kappa,
+                                   chunk_blocks=args.chunk_blocks, limit=args.limit)))
+        return
+    out = model(args.config, gib, limit=args.limit)
     print(json.dumps(out))
 
 

@@ -123,3 +123,41 @@ def test_argument_errors():
         eakv.eakv_capacity_curve(d.data_ptr(), 4, [0, 3], [48], [0], 16, [4])
     with pytest.raises(eakv.EakvError):                      # too many capacities
         eakv.eakv_capacity_curve(d.data_ptr(), 4, [0, 4], [64], [0], 16, list(range(1, 70)))
+
+
+def test_declined_chunk_audit_matches_oracle():
+    """The audit of declined writes (next reuse distance >= K_H or never again) on a scaled
+    config-2 trace under both filters, against the oracle's definition-level audit."""
+    from dataclasses import replace
+    import eakv_workloads
+    from oracle import audit as oaudit
+    from oracle import hash as ohash
+    from oracle.tier import HostTier
+    from paper_2609_33762_b200 import capacity
+    small = replace(CONFIGS["c2"], shape="tiny", agents=6, turns=12, first_prompt=400,
+                    append_median=150.0, context_cap=3000, tool_gap_mean_ms=15_000.0, kappa_blocks=4)
+    eakv_workloads.CONFIGS["_audit"] = small
+    try:
+        shape = SHAPES["tiny"]
+        trace = make_trace(small)
+        kh = 300
+        gib = kh * shape.block_bytes / (1 << 30)
+        for policy, pol_id in (("fixed", 1), ("conditioned", 2)):
+            got = capacity.audit("_audit", policy, gib)
+            tier = HostTier(kh, shape.block_size, pol_id, small.kappa_blocks)
+            stream, declined = [], []
+            for r in trace.requests:
+                keys = ohash.hash_blocks(trace.prompt(r).tolist(), shape.block_size)
+                res = tier.step(keys, r.n_tokens, r.agent, r.time_ms)
+                for k, h, a in zip(keys, res.hit, res.admit):
+                    if not h and not a:
+                        declined.append(len(stream))
+                    stream.append(k)
+            want = oaudit.declined_audit(stream, declined, kh)
+            assert got["tier_units"] == kh
+            assert got["declined_chunks"] == want["declined"] > 0
+            assert got["meet_condition"] == want["meets"]
+            assert got["never_referenced_again"] == want["never_again"]
+            assert got["declined_requests"] == tier.stats["declined_requests"]
+    finally:
+        del eakv_workloads.CONFIGS["_audit"]

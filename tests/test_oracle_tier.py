@@ -267,3 +267,35 @@ def test_length_window_keeps_last_256():
     for i, n in enumerate([100, 200, 300, 400]):
         t.step([], n, 0, i)
     assert list(t.lengths) == [200, 300, 400]
+
+
+def test_declined_audit_hand_case_and_kappa_sensitivity():
+    from oracle import audit
+    # positions 1 (key 2) and 2 (key 3) declined, K = 2: key 2 returns after {3, 1} (D = 2 >= K),
+    # key 3 never returns: both meet Proposition 1's condition
+    a = audit.declined_audit([1, 2, 3, 1, 2, 4, 1], [1, 2], 2)
+    assert (a["declined"], a["meets"], a["never_again"], a["ratios"]) == (2, 2, 1, [1.0])
+    # with K = 3 the returning chunk is within reach: declining it costs a hit
+    a = audit.declined_audit([1, 2, 3, 1, 2, 4, 1], [1, 2], 3)
+    assert (a["meets"], a["never_again"]) == (1, 1)
+    # brute force on random streams: the condition is "next D >= K or no next reference"
+    rng = random.Random(12)
+    for _ in range(50):
+        s = rand_stream(rng, rng.randrange(2, 50), rng.randrange(2, 9))
+        K = rng.randrange(1, 6)
+        dec = sorted(rng.sample(range(len(s)), rng.randrange(0, len(s))))
+        a = audit.declined_audit(s, dec, K)
+        want = 0
+        for i in dec:
+            later = [j for j in range(i + 1, len(s)) if s[j] == s[i]]
+            if not later or len(set(s[i + 1:later[0]]) - {s[i]}) >= K:
+                want += 1
+        assert a["meets"] == want
+    # kappa sensitivity: filtered requests shrink as kappa grows; kappa = infinity filters none
+    reqs = [([(a_, j) for j in range(n)], n * 4, a_, t) for t, (a_, n) in
+            enumerate([(0, 3), (1, 9), (0, 5), (2, 20), (1, 12), (0, 30), (2, 21)])]
+    out = audit.kappa_sensitivity(reqs, 40, 4, [0, 2, 8, 10**9])
+    filt = [out[k]["filtered_requests"] for k in (0, 2, 8, 10**9)]
+    assert filt == sorted(filt, reverse=True) and filt[-1] == 0 and filt[0] > 0
+    assert out[10**9]["declined_chunks"] == 0
+    assert audit.median([3, 1, 2]) == 2 and audit.median([4, 1, 2, 3]) == 2.5
