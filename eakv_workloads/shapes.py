@@ -66,6 +66,7 @@ class TraceConfig:
     host_blocks: int = 0          # 0: sized at run time (working-set estimate / sweep)
     policy: str = "write_all"
     kappa_blocks: int = 8
+    shared_prefix_tokens: int = 0     # tokens of a system prompt that every agent starts with
     extra: dict = field(default_factory=dict)
 
 

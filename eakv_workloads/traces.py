@@ -77,10 +77,15 @@ def make_trace(cfg, seed=None, agents=None, turns=None) -> Trace:
             gaps[0] = 0.0
             times[a] = np.floor(start[a] + np.cumsum(gaps)).astype(np.int64)
 
-    # token ids: independent stream per agent
+    # token ids: independent stream per agent, after an optional prefix common to all agents
     agent_tokens = {}
     for a in range(A):
         agent_tokens[a] = rng.integers(0, cfg.vocab, size=int(lengths[a, -1]), dtype=np.int32)
+    if cfg.shared_prefix_tokens > 0:
+        common = rng.integers(0, cfg.vocab, size=cfg.shared_prefix_tokens, dtype=np.int32)
+        for a in range(A):
+            k = min(len(common), len(agent_tokens[a]))
+            agent_tokens[a][:k] = common[:k]
 
     reqs = [Request(int(times[a, t]), a, t, int(lengths[a, t])) for a in range(A) for t in range(T)]
     reqs.sort(key=lambda r: (r.time_ms, r.agent, r.turn))

@@ -75,12 +75,15 @@ def gpu_prefixes(trace, shape, gpu_blocks, stream_host, offsets):
     return G
 
 
-def model(config, host_gib, device="cuda:0", limit=None):
+def model(config, host_gib, device="cuda:0", limit=None, agents=None, shared_prefix=0):
     import torch
+    from dataclasses import replace
     from eakv_workloads import CONFIGS, SHAPES, make_trace
     cfg = CONFIGS[config]
+    if shared_prefix:
+        cfg = replace(cfg, shared_prefix_tokens=shared_prefix)
     shape = SHAPES[cfg.shape]
-    trace = make_trace(cfg)
+    trace = make_trace(cfg, agents=agents)
     if limit:
         trace.requests = trace.requests[:limit]
     t0 = time.perf_counter()
@@ -108,7 +111,8 @@ def model(config, host_gib, device="cuda:0", limit=None):
         rows.append({"host_gib": g, "blocks": caps[c], "hits": int(out["hits"][c]),
                      "restored_tokens": int(out["restored_blocks"][c]) * shape.block_size,
                      "computed_prefill_tokens": int(out["computed_tokens"][c])})
-    return {"config": config, "requests": len(trace.requests), "references": n_refs,
+    return {"config": config, "agents": len(trace.agent_tokens), "shared_prefix_tokens": shared_prefix,
+            "requests": len(trace.requests), "references": n_refs,
             "prompt_tokens": int(tokens.sum()), "rows": rows,
             "computed_prefill_tokens_infinite_tier": inf_computed,
             "working_set_blocks": {"eq5": ws_eq5, "full": ws_full},
@@ -175,6 +179,38 @@ def audit(config, policy, host_gib, kappa=None, chunk_blocks=1, device="cuda:0",
             "admitted_chunks": stats["admitted"]}
 
 
+def kappa_sweep(config, host_gib, kappas, chunk_blocks=1, limit=None, device="cuda:0"):
+    """Threshold sensitivity (Appendix D): under fixed admission, the requests each kappa filters
+    and the share of new-chunk writes it declines, relative to a write-all run."""
+    from eakv_workloads import CONFIGS, SHAPES, make_trace
+    cfg = CONFIGS[config]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg)
+    if limit:
+        trace.requests = trace.requests[:limit]
+    R = max(1, chunk_blocks)
+    stream, offsets, _ = reference_stream(trace, shape, device)
+    keys_host = stream.cpu().numpy().view(np.uint64)
+    chunk_keys = [np.ascontiguousarray(keys_host[offsets[j]:offsets[j + 1]][R - 1::R])
+                  for j in range(len(trace.requests))]
+    kh = max(1, int(host_gib * GIB // (R * shape.block_bytes)))
+    rows = []
+    for kappa in kappas:
+        ctx = eakv.Context(num_layers=1, kv_heads=1, head_dim=8, block_size=shape.block_size, gpu_blocks=1,
+                           host_blocks=kh, kv_base=None, control_plane_only=True,
+                           policy=eakv.POLICY_FILTER_FIXED, kappa_blocks=kappa, chunk_blocks=R)
+        for j, r in enumerate(trace.requests):
+            ctx.eakv_tier_step(chunk_keys[j], r.agent, r.n_tokens, r.time_ms)
+        st = ctx.eakv_get_stats()
+        ctx.close()
+        new_chunks = st["admitted"] + st["declined"]
+        rows.append({"kappa": kappa, "filtered_requests": st["declined_requests"],
+                     "declined_chunks": st["declined"], "admitted_chunks": st["admitted"],
+                     "share_of_new_chunk_writes_declined": st["declined"] / new_chunks if new_chunks else None,
+                     "hits": st["hits"]})
+    return {"config": config, "host_gib": host_gib, "tier_units": kh, "chunk_blocks": R, "rows": rows}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", default="c2", choices=["c0", "c0_big_tier", "c2", "c3", "c4"])
@@ -184,14 +220,22 @@ def main():
                     help="declined-chunk audit under this policy instead of the capacity sweep")
     ap.add_argument("--chunk-blocks", type=int, default=1)
     ap.add_argument("--kappa", type=int, default=None)
+    ap.add_argument("--kappa-sweep", default=None, help="comma-separated thresholds, fixed admission")
+    ap.add_argument("--agents", type=int, default=None, help="active pool size (default: the config's)")
+    ap.add_argument("--shared-prefix", type=int, default=0, help="system-prompt tokens shared by all agents")
     args = ap.parse_args()
     gib = [float(x) for x in args.host_gib.split(",")]
+    if args.kappa_sweep:
+        for g in gib:
+            print(json.dumps(kappa_sweep(args.config, g, [int(k) for k in args.kappa_sweep.split(",")],
+                                         chunk_blocks=args.chunk_blocks, limit=args.limit)))
+        return
     if args.audit:
         for g in gib:
             print(json.dumps(audit(args.config, args.audit, g, kappa=args.kappa,
                                    chunk_blocks=args.chunk_blocks, limit=args.limit)))
         return
-    out = model(args.config, gib, limit=args.limit)
+    out = model(args.config, gib, limit=args.limit, agents=args.agents, shared_prefix=args.shared_prefix)
     print(json.dumps(out))
 
 

@@ -227,3 +227,21 @@ def test_oracle_capacity_error_matches(eakv):
     t = HostTier(2, 4)
     with pytest.raises(CapacityError):
         t.step([1, 2, 3], 12, 0, 0)
+
+
+def test_shared_system_prompt_is_deduplicated_across_agents(eakv):
+    """A prefix common to all agents (a weakly shared pool): its chunks are stored once and hit
+    by every other agent; product and oracle agree request by request."""
+    cfg = replace(CONFIGS["c0_big_tier"], shared_prefix_tokens=256)
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg)
+    oracle = TraceOracle(shape, cfg.gpu_blocks, cfg.host_blocks)
+    oracle.run(trace)
+    ctx = cp_ctx(eakv, shape.block_size, cfg.gpu_blocks, cfg.host_blocks)
+    compare(drive(ctx, trace, shape.block_size), oracle.records)
+    ctx.close()
+    first_turns = [r for r in oracle.records[:8]]
+    assert first_turns[0]["H"] == 0 and all(r["H"] == 16 for r in first_turns[1:])   # 256 tokens = 16 blocks
+    plain = TraceOracle(shape, cfg.gpu_blocks, cfg.host_blocks)
+    plain.run(make_trace(CONFIGS["c0_big_tier"]))
+    assert oracle.totals["stored_blocks"] < plain.totals["stored_blocks"]
