@@ -161,3 +161,25 @@ def test_custom_base_and_seed():
     toks = np.arange(100, dtype=np.int32)
     assert gpu_keys(ctx, toks) == oh.hash_blocks(toks.tolist(), 16, 42, 1234567891011)
     ctx.close()
+
+
+def test_batched_capacity_errors_and_empty_batches():
+    from paper_2609_33762_b200 import eakv
+    ctx = hash_ctx(16, hash_scratch_blocks=64, max_call_blocks=8)
+    toks = torch.zeros(16 * 100, dtype=torch.int32, device="cuda")
+    out = torch.zeros(100, dtype=torch.int64, device="cuda")
+    with pytest.raises(eakv.EakvError) as ei:           # 100 blocks > 64 blocks of scratch
+        ctx.eakv_hash_blocks_batched(toks.data_ptr(), [0, 1600], None, out.data_ptr())
+    assert ei.value.code == eakv.E_CAPACITY
+    with pytest.raises(eakv.EakvError) as ei:           # 9 prompts > 8
+        ctx.eakv_hash_blocks_batched(toks.data_ptr(), list(range(0, 160, 16)), None, out.data_ptr())
+    assert ei.value.code == eakv.E_CAPACITY
+    with pytest.raises(eakv.EakvError) as ei:           # offsets must not decrease
+        ctx.eakv_hash_blocks_batched(toks.data_ptr(), [0, 64, 32], None, out.data_ptr())
+    assert ei.value.code == eakv.E_INVAL
+    assert ctx.eakv_hash_blocks_batched(toks.data_ptr(), [0], None, out.data_ptr()).tolist() == [0]
+    assert ctx.eakv_hash_blocks_batched(toks.data_ptr(), [0, 5, 9], None, out.data_ptr()).tolist() == [0, 0, 0]
+    # the single-prompt call still works afterwards, chained over the small scratch
+    t = np.arange(1600, dtype=np.int32)
+    assert gpu_keys(ctx, t) == oh.hash_blocks(t.tolist(), 16)
+    ctx.close()

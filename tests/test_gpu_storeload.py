@@ -260,3 +260,60 @@ def test_layer_pipelined_load(name, group, kw):
     assert ei.value.code == e.E_INVAL
     rig.check()
     rig.close()
+
+
+def test_calls_larger_than_the_argument_ring_slot_are_split():
+    """max_call_blocks smaller than the call: several argument uploads per call; also more
+    calls than ring slots back to back (slot reuse)."""
+    e = eakv()
+    shape = SHAPE_CASES["tiny"]
+    for kw in (dict(tier_location=e.TIER_DEVICE), dict(link_strategy=e.LINK_STAGED, min_staged_run_bytes=-1),
+               dict(link_strategy=e.LINK_ZERO_COPY)):
+        rig = Rig(shape, 300, 280, seed=31, max_call_blocks=40, staging_bytes=9 * shape.block_bytes, **kw)
+        rng = rig.rng
+        for rep in range(12):                      # 12 calls x up to 7 uploads each > 8 ring slots
+            m = int(rng.integers(33, 270))
+            rig.store(rng.permutation(300)[:m].astype(np.int32), (rng.random(m) < 0.8).astype(np.uint8),
+                      rng.permutation(280)[:m].astype(np.int32))
+            k = int(rng.integers(33, 270))
+            rig.load(rng.permutation(280)[:k].astype(np.int32), rng.permutation(300)[:k].astype(np.int32))
+        rig.check()
+        rig.close()
+
+
+def test_store_and_load_on_two_streams_concurrently():
+    """A store and a load that touch disjoint blocks and slots may overlap on two streams."""
+    e = eakv()
+    shape = SHAPE_CASES["qwen"]
+    for kw in (dict(link_strategy=e.LINK_STAGED, min_staged_run_bytes=-1), dict(link_strategy=e.LINK_ZERO_COPY),
+               dict(tier_location=e.TIER_DEVICE)):
+        rig = Rig(shape, 128, 128, seed=32, staging_bytes=4 * shape.block_bytes, **kw)
+        s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+        torch.cuda.synchronize()
+        for rep in range(4):
+            blocks = rig.rng.permutation(128).astype(np.int32)
+            slots = rig.rng.permutation(128).astype(np.int32)
+            st_b, ld_b = blocks[:60], blocks[60:120]
+            st_s, ld_s = slots[:60], slots[60:120]
+            rig.ctx.eakv_load(ld_s, ld_b, s1)
+            rig.ctx.eakv_store(st_b, None, st_s, s2)
+            osl.load(rig.pool_np, rig.tier_np, ld_s, ld_b)
+            osl.store(rig.pool_np, rig.tier_np, st_b, [1] * 60, st_s)
+            s1.synchronize(); s2.synchronize()
+        rig.check()
+        rig.close()
+
+
+def test_staging_smaller_than_two_blocks_and_stats():
+    e = eakv()
+    shape = SHAPE_CASES["ragged"]
+    rig = Rig(shape, 20, 20, seed=33, link_strategy=e.LINK_STAGED, min_staged_run_bytes=-1,
+              staging_bytes=shape.block_bytes + 1)          # one block per staging buffer
+    rig.store(np.arange(7, dtype=np.int32), None, np.arange(7, dtype=np.int32)[::-1].copy())
+    rig.load(np.array([6, 5, 4], np.int32), np.array([17, 18, 19], np.int32))
+    rig.check()
+    st = rig.ctx.eakv_get_stats()
+    assert (st["blocks_stored"], st["blocks_loaded"]) == (7, 3)
+    assert st["bytes_stored"] == 7 * shape.block_bytes and st["bytes_loaded"] == 3 * shape.block_bytes
+    assert st["kernel_launches"] >= 10 and st["memcpy_calls"] >= 10
+    rig.close()
