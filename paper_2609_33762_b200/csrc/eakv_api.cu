@@ -64,6 +64,7 @@ struct eakv_ctx {
 
     // hash
     uint64_t* d_pow = nullptr;
+    std::vector<uint64_t> h_pow;   // B^0 .. B^b on the host
     uint64_t* d_partial = nullptr;
     int* d_counters = nullptr;
     int64_t hash_scratch_blocks = 0;
@@ -471,6 +472,7 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
         std::vector<uint64_t> pw((size_t)cfg->block_size + 1);
         pw[0] = 1;
         for (int e = 1; e <= cfg->block_size; ++e) pw[e] = mulmod_host(pw[e - 1], ctx->base);
+        ctx->h_pow = pw;
         CUC(cudaMalloc(&ctx->d_pow, pw.size() * 8));
         CUC(cudaMemcpy(ctx->d_pow, pw.data(), pw.size() * 8, cudaMemcpyHostToDevice));
         CUC(cudaMalloc(&ctx->d_partial, (size_t)ctx->hash_scratch_blocks * 8));
@@ -570,6 +572,7 @@ int eakv_hash_blocks(eakv_ctx* ctx, const int32_t* tokens_dev, int64_t n_tokens,
         L.partial = ctx->d_partial;
         L.counters = ctx->d_counters;
         L.pow_table = ctx->d_pow;
+        if (b <= 64) hash_fill_limbs(L, ctx->h_pow.data(), b); else L.pow_block = ctx->h_pow[b];
         L.tiles = nullptr;
         L.prompts = nullptr;
         L.single_nblk = cur;
@@ -660,6 +663,7 @@ int eakv_hash_blocks_batched(eakv_ctx* ctx, const int32_t* tokens_dev,
     L.partial = ctx->d_partial;
     L.counters = ctx->d_counters;
     L.pow_table = ctx->d_pow;
+    if (b <= 64) hash_fill_limbs(L, ctx->h_pow.data(), b); else L.pow_block = ctx->h_pow[b];
     L.prompts = static_cast<const HashPrompt*>(s->dev);
     L.tiles = reinterpret_cast<const HashTile*>(L.prompts + n_prompts);
     L.single_nblk = 0;

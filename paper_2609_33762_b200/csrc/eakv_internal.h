@@ -37,6 +37,10 @@ struct HashLaunch {
     int32_t block_size;
     int32_t tile_blocks;
     // self-check limits: a CTA whose tile would reach past them raises *error_flag and skips
+    // B^e for e < 64 as three 21-bit limbs each, passed by value: with the block size known at
+    // compile time they become constant-bank operands of the multiply-adds (no load at all)
+    uint32_t pw_limbs[3 * 64];
+    uint64_t pow_block;             // A = B^b, the per-block multiplier of the scan
     int64_t tokens_limit;           // tokens readable at `tokens`
     int64_t blocks_limit;           // entries writable at `keys` and `partial`
     int* error_flag;
@@ -52,6 +56,16 @@ inline int hash_tile_blocks(int block_size, int64_t total_blocks) {
     }
     const int t = kHashTileTokens / block_size;
     return t > 1 ? t : 1;
+}
+// fill L.pw_limbs / L.pow_block from powers B^0 .. B^b held on the host
+inline void hash_fill_limbs(HashLaunch& L, const uint64_t* pow_host, int block_size) {
+    for (int e = 0; e < 64; ++e) {
+        const uint64_t w = e < block_size ? pow_host[e] : 0;
+        L.pw_limbs[3 * e + 0] = (uint32_t)(w & 0x1FFFFF);
+        L.pw_limbs[3 * e + 1] = (uint32_t)((w >> 21) & 0x1FFFFF);
+        L.pw_limbs[3 * e + 2] = (uint32_t)(w >> 42);
+    }
+    L.pow_block = pow_host[block_size];
 }
 cudaError_t hash_kernels_init();
 cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool thread_per_block, bool vec,

@@ -370,9 +370,18 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
 
 // B: the block size when known at compile time (16, 32, 64: loops unroll and every shared-memory
 // offset becomes an immediate), 0: read it from the launch descriptor.
+// multiply-add against limbs that sit in the kernel parameters (constant bank)
+#define EAKV_MACP(tok, e)                                          \
+    do {                                                           \
+        const uint32_t x_ = (uint32_t)(tok) + 1u;                  \
+        s0 += (uint64_t)x_ * L.pw_limbs[3 * (e) + 0];              \
+        s1 += (uint64_t)x_ * L.pw_limbs[3 * (e) + 1];              \
+        s2 += (uint64_t)x_ * L.pw_limbs[3 * (e) + 2];              \
+    } while (0)
+
 template <int B>
 __global__ void __launch_bounds__(kHashThreads)
-hash_blocks_staged_kernel(HashLaunch L) {
+hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ Pair warp_tot[32];
     __shared__ int is_last;
@@ -422,10 +431,12 @@ hash_blocks_staged_kernel(HashLaunch L) {
     };
 
     issue(0);
-    for (int e = tid; e < b; e += blockDim.x) {
-        const uint64_t w = L.pow_table[e];
-        pw3[e] = make_uint4((uint32_t)(w & 0x1FFFFF), (uint32_t)((w >> 21) & 0x1FFFFF),
-                            (uint32_t)(w >> 42), 0u);
+    if (!B) {
+        for (int e = tid; e < b; e += blockDim.x) {
+            const uint64_t w = L.pow_table[e];
+            pw3[e] = make_uint4((uint32_t)(w & 0x1FFFFF), (uint32_t)((w >> 21) & 0x1FFFFF),
+                                (uint32_t)(w >> 42), 0u);
+        }
     }
     uint64_t* partial = L.partial + blk0;
     for (int r = 0; r < n_sub; ++r) {
@@ -446,7 +457,7 @@ hash_blocks_staged_kernel(HashLaunch L) {
                 for (int k = 0; k < (B ? B : 4); k += 4) {
                     const int4 u = row[k >> 2];
                     const int e = (B ? B : 4) - 1 - k;
-                    EAKV_MAC3(u.x, e); EAKV_MAC3(u.y, e - 1); EAKV_MAC3(u.z, e - 2); EAKV_MAC3(u.w, e - 3);
+                    EAKV_MACP(u.x, e); EAKV_MACP(u.y, e - 1); EAKV_MACP(u.z, e - 2); EAKV_MACP(u.w, e - 3);
                 }
                 acc = fold_limb_sums(s0, s1, s2);
             } else {
@@ -475,10 +486,11 @@ hash_blocks_staged_kernel(HashLaunch L) {
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    scan_prompt(partial, L.keys + blk0, nblk, parent, L.pow_table[b], warp_tot);
+    scan_prompt(partial, L.keys + blk0, nblk, parent, L.pow_block, warp_tot);
     if (tid == 0) L.counters[p] = 0;
 }
 #undef EAKV_MAC3
+#undef EAKV_MACP
 
 // thread_per_block: see hash_thread_per_block(); vec: 16-byte token loads are allowed
 cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool thread_per_block, bool vec,
@@ -633,6 +645,15 @@ extern "C" int eakv_hash_blocks_static(const int32_t* tokens_dev, int64_t n_toke
     L.single_parent_ptr = nullptr;
     L.block_size = block_size;
     L.tile_blocks = hash_tile_blocks(block_size, nblk);
+    {   // powers B^0 .. B^b on the host (at most 4,097 modular products) for the by-value limbs
+        uint64_t pw_host[65];
+        const int lim = block_size < 64 ? block_size : 64;
+        pw_host[0] = 1;
+        for (int e = 1; e <= lim; ++e)
+            pw_host[e] = (uint64_t)(((unsigned __int128)pw_host[e - 1] * base) % P);
+        if (block_size <= 64) hash_fill_limbs(L, pw_host, block_size);
+        else L.pow_block = 0;   // not used by the kernels chosen for larger blocks
+    }
     L.tokens_limit = n_tokens;
     L.blocks_limit = nblk;
     L.error_flag = reinterpret_cast<int*>(scratch + kStaticPartialBytes + kStaticPowBytes) + 1;
