@@ -605,7 +605,7 @@ def main():
     if not args.no_e2e:
         link = pinned_link_peak(torch, device) if rank == 0 else None
         arm = Arm(args, pool, shape, torch, eakv, host_tier=True, device=device)
-        e_steps = max(2, min(args.steps, 5))
+        e_steps = max(2, min(args.steps, 8))
         re_ = run_arm(arm, prompts_host, tables, e_steps, min(args.warmup, 3), dist, None,
                       time_kernels=False)
         layered = layered_load_probe(torch, arm, tables, shape) if rank == 0 else None
