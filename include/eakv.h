@@ -229,6 +229,48 @@ int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_m
 int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_table,
               int64_t n_blocks, void* cuda_stream);
 
+/* One agent turn in two calls (the order of Section 4 and Appendix D: lookup when the request is
+ * scheduled, restore before compute, store after compute).
+ *
+ * eakv_turn_begin: keys of the prompt's full blocks (eakv_hash_blocks on an internal lookup
+ * stream, so it never waits behind transfers; blocks whose keys the caller already knows from
+ * the previous turn are not hashed again), eakv_match, eakv_tier_step, eakv_gpu_tier_step, then
+ * eakv_load of the host-covered blocks [G, H) on cuda_stream.  With chunk_blocks = R > 1 the
+ * host tier sees one key per full chunk.  *view describes the turn; its arrays live in the
+ * context and stay valid until the next eakv_turn_begin.
+ *   tokens        device-accessible int32[n_tokens] (pinned host memory is fine), readable now
+ *   known_keys    host uint64[n_known] keys of the first n_known blocks, or NULL / 0
+ * The engine then produces the KV of every block with needs_fill[j] = 1 into gpu_block[j]
+ * (ordered after cuda_stream's load) and calls
+ * eakv_turn_end: eakv_store of the admitted blocks on cuda_stream, and release of the partial
+ * tail's temporary block.  One turn per context at a time.
+ * Errors: those of the calls above; EAKV_E_INVAL when a turn is already open (begin) or none
+ * is (end).  On an error in begin no turn is opened; bookkeeping done by then is kept. */
+typedef struct eakv_turn_view {
+    int64_t n_blocks;             /* full blocks of the prompt                              */
+    int64_t n_units;              /* tier units (= n_blocks / chunk_blocks)                 */
+    int64_t gpu_prefix_blocks;    /* G                                                      */
+    int64_t host_prefix_blocks;   /* H in blocks (host-covered units * chunk_blocks)        */
+    int64_t restore_lo, restore_hi; /* blocks [lo, hi) restored from the host               */
+    int64_t fresh_tokens;         /* n_tokens - max(G, H) * block_size                      */
+    int64_t new_chunks;           /* u of the write rule                                    */
+    int64_t n_fill, n_stored_blocks, n_evicted;
+    int32_t pressure, save, tail_block, reserved;
+    const uint64_t* keys;         /* [n_blocks]                                             */
+    const int32_t*  gpu_block;    /* [n_blocks] pool block of every prompt block            */
+    const uint8_t*  gpu_resident; /* [n_blocks] was resident when referenced                */
+    const uint8_t*  needs_fill;   /* [n_blocks] the engine must compute this block's KV     */
+    const uint8_t*  hit;          /* [n_units]                                              */
+    const uint8_t*  admit;        /* [n_units]                                              */
+    const int32_t*  slot;         /* [n_units] tier unit slot, -1 = declined                */
+    const uint64_t* evicted_keys; /* [n_evicted]                                            */
+    const int32_t*  evicted_slots;/* [n_evicted]                                            */
+} eakv_turn_view;
+int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
+                    const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
+                    void* cuda_stream, eakv_turn_view* view);
+int eakv_turn_end(eakv_ctx* ctx, void* cuda_stream);
+
 /* Layer-pipelined restore (Section 3.1, Eq. 2: the fixed restoration overhead tau_load is
  * what a consumer waits for before it can start; moving layers in order lets it start on
  * the first ones while the rest are in flight).  Same result as eakv_load, but the 2L

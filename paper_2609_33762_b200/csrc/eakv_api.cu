@@ -90,6 +90,16 @@ struct eakv_ctx {
     uint32_t epoch = 0;
     std::vector<int2> scratch_entries;
 
+    // two-call turn engine
+    cudaStream_t lookup_stream = nullptr;
+    uint64_t* turn_keys = nullptr;            // pinned + mapped; the hash kernel writes it directly
+    int64_t turn_keys_cap = 0;
+    bool turn_open = false;
+    int32_t turn_tail = -1;
+    std::vector<int32_t> t_block, t_slot_u, t_slot_b, t_evicted_slots, t_host_slots;
+    std::vector<uint8_t> t_resident, t_fill, t_hit, t_admit_u, t_admit_b;
+    std::vector<uint64_t> t_unit_keys, t_evicted_keys;
+
     std::string cuda_err;
 };
 
@@ -152,6 +162,8 @@ void free_all(eakv_ctx* c) {
     if (c->d_partial) cudaFree(c->d_partial);
     if (c->d_counters) cudaFree(c->d_counters);
     if (c->d_error_flag) cudaFree(c->d_error_flag);
+    if (c->turn_keys) cudaFreeHost(c->turn_keys);
+    if (c->lookup_stream) cudaStreamDestroy(c->lookup_stream);
     if (c->tier && c->tier_owned) {
         if (c->cfg.tier_location == EAKV_TIER_DEVICE) cudaFree(c->tier);
         else cudaFreeHost(c->tier);
@@ -898,6 +910,139 @@ int eakv_load_layers(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* bl
     ctx->stats.blocks_loaded += n_blocks;
     ctx->stats.bytes_loaded += n_blocks * ctx->block_bytes;
     return EAKV_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// one turn in two calls
+// ------------------------------------------------------------------------------------------
+int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
+                    const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
+                    void* cuda_stream, eakv_turn_view* view) {
+    if (!ctx || !view || n_tokens < 0 || n_known < 0 || ctx->device < 0) return EAKV_E_INVAL;
+    if (ctx->turn_open) return EAKV_E_INVAL;
+    if (n_known > 0 && !known_keys) return EAKV_E_INVAL;
+    const int b = ctx->cfg.block_size;
+    const int64_t R = ctx->chunk_tokens / b;
+    const int64_t nblk = n_tokens / b;
+    if (n_known > nblk) n_known = nblk;
+    DeviceGuard g(ctx->device);
+    // key buffer in mapped pinned memory, grown in powers of two
+    if (nblk > ctx->turn_keys_cap) {
+        int64_t cap = 4096;
+        while (cap < nblk) cap <<= 1;
+        if (ctx->turn_keys) {
+            CU(cudaStreamSynchronize(ctx->lookup_stream));
+            CU(cudaFreeHost(ctx->turn_keys));
+            ctx->turn_keys = nullptr;
+            ctx->turn_keys_cap = 0;
+        }
+        cudaError_t e = cudaHostAlloc(&ctx->turn_keys, (size_t)cap * 8,
+                                      cudaHostAllocMapped | cudaHostAllocPortable);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return EAKV_E_NOMEM;
+        }
+        ctx->turn_keys_cap = cap;
+    }
+    if (!ctx->lookup_stream) CU(cudaStreamCreateWithFlags(&ctx->lookup_stream, cudaStreamNonBlocking));
+    uint64_t* keys = ctx->turn_keys;
+    if (n_known > 0) std::memcpy(keys, known_keys, (size_t)n_known * 8);
+    if (nblk > n_known) {
+        if (!tokens) return EAKV_E_INVAL;
+        const uint64_t parent = n_known ? keys[n_known - 1] : ctx->seed;
+        int rc = eakv_hash_blocks(ctx, tokens + n_known * b, (nblk - n_known) * (int64_t)b, parent,
+                                  keys + n_known, nullptr, ctx->lookup_stream);
+        if (rc != EAKV_OK) return rc;
+        CU(cudaStreamSynchronize(ctx->lookup_stream));
+    }
+    // tier units: one key per full chunk (the key at the chunk's last block)
+    const int64_t nu = nblk / R;
+    const uint64_t* ukeys = keys;
+    if (R > 1) {
+        ctx->t_unit_keys.resize((size_t)nu);
+        for (int64_t c = 0; c < nu; ++c) ctx->t_unit_keys[c] = keys[c * R + R - 1];
+        ukeys = ctx->t_unit_keys.data();
+    }
+    ctx->t_block.resize((size_t)nblk); ctx->t_resident.resize((size_t)nblk);
+    ctx->t_fill.assign((size_t)nblk, 0);
+    ctx->t_hit.resize((size_t)nu); ctx->t_admit_u.resize((size_t)nu); ctx->t_slot_u.resize((size_t)nu);
+    ctx->t_evicted_keys.resize((size_t)nu); ctx->t_evicted_slots.resize((size_t)nu);
+    ctx->t_host_slots.resize((size_t)nu);
+    int64_t G = 0, G_unused = 0, Hu = 0;
+    int rc = eakv_match(ctx, keys, nblk, &G, nullptr, nullptr, nullptr);
+    if (rc != EAKV_OK) return rc;
+    rc = eakv_match(ctx, ukeys, nu, &G_unused, &Hu, nullptr, ctx->t_host_slots.data());
+    if (rc != EAKV_OK) return rc;
+    int64_t n_ev = nu;
+    eakv_step_info info;
+    rc = eakv_tier_step(ctx, ukeys, nu, agent_id, n_tokens, now_ms, ctx->t_hit.data(),
+                        ctx->t_admit_u.data(), ctx->t_slot_u.data(), ctx->t_evicted_keys.data(),
+                        ctx->t_evicted_slots.data(), &n_ev, &info);
+    if (rc != EAKV_OK) return rc;
+    int32_t tail = -1;
+    rc = eakv_gpu_tier_step(ctx, keys, nblk, (n_tokens % b) != 0, ctx->t_resident.data(),
+                            ctx->t_block.data(), &tail);
+    if (rc != EAKV_OK) return rc;
+    const int64_t H = Hu * R;
+    const int64_t cover = std::max(G, H);
+    const int64_t lo = G, hi = H > G ? H : G;
+    if (hi > lo) {
+        // block slots of the restored blocks: chunk slot * R + position inside the chunk
+        std::vector<int32_t> slots((size_t)(hi - lo));
+        for (int64_t j = lo; j < hi; ++j)
+            slots[j - lo] = (int32_t)((int64_t)ctx->t_host_slots[j / R] * R + j % R);
+        rc = eakv_load(ctx, slots.data(), ctx->t_block.data() + lo, hi - lo, cuda_stream);
+        if (rc != EAKV_OK) {
+            if (tail >= 0) eakv_gpu_tier_release(ctx, tail);
+            return rc;
+        }
+    }
+    int64_t n_fill = 0;
+    for (int64_t j = cover; j < nblk; ++j)
+        if (!ctx->t_resident[j]) { ctx->t_fill[j] = 1; ++n_fill; }
+    // per-block view of the unit decisions, for the store at the end of the turn
+    ctx->t_admit_b.assign((size_t)nblk, 0);
+    ctx->t_slot_b.assign((size_t)nblk, -1);
+    int64_t n_store = 0;
+    for (int64_t c = 0; c < nu; ++c) {
+        if (!ctx->t_admit_u[c]) continue;
+        for (int64_t i = 0; i < R; ++i) {
+            ctx->t_admit_b[c * R + i] = 1;
+            ctx->t_slot_b[c * R + i] = (int32_t)((int64_t)ctx->t_slot_u[c] * R + i);
+            ++n_store;
+        }
+    }
+    ctx->turn_open = true;
+    ctx->turn_tail = tail;
+    view->n_blocks = nblk; view->n_units = nu;
+    view->gpu_prefix_blocks = G; view->host_prefix_blocks = H;
+    view->restore_lo = lo; view->restore_hi = hi;
+    view->fresh_tokens = n_tokens - cover * b;
+    view->new_chunks = info.new_chunks;
+    view->n_fill = n_fill; view->n_stored_blocks = n_store; view->n_evicted = n_ev;
+    view->pressure = info.pressure; view->save = info.save; view->tail_block = tail; view->reserved = 0;
+    view->keys = keys;
+    view->gpu_block = ctx->t_block.data(); view->gpu_resident = ctx->t_resident.data();
+    view->needs_fill = ctx->t_fill.data();
+    view->hit = ctx->t_hit.data(); view->admit = ctx->t_admit_u.data(); view->slot = ctx->t_slot_u.data();
+    view->evicted_keys = ctx->t_evicted_keys.data(); view->evicted_slots = ctx->t_evicted_slots.data();
+    return EAKV_OK;
+}
+
+int eakv_turn_end(eakv_ctx* ctx, void* cuda_stream) {
+    if (!ctx || ctx->device < 0 || !ctx->turn_open) return EAKV_E_INVAL;
+    ctx->turn_open = false;
+    int rc = EAKV_OK;
+    const int64_t nblk = (int64_t)ctx->t_block.size();
+    if (nblk > 0)
+        rc = eakv_store(ctx, ctx->t_block.data(), ctx->t_admit_b.data(), ctx->t_slot_b.data(), nblk,
+                        cuda_stream);
+    if (ctx->turn_tail >= 0) {
+        const int rc2 = eakv_gpu_tier_release(ctx, ctx->turn_tail);
+        ctx->turn_tail = -1;
+        if (rc == EAKV_OK) rc = rc2;
+    }
+    return rc;
 }
 
 // ------------------------------------------------------------------------------------------

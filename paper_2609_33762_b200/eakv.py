@@ -62,12 +62,32 @@ class StepInfo(C.Structure):
                 ("pressure", C.c_int32), ("save", C.c_int32)]
 
 
+class TurnView(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in (
+        "n_blocks", "n_units", "gpu_prefix_blocks", "host_prefix_blocks", "restore_lo", "restore_hi",
+        "fresh_tokens", "new_chunks", "n_fill", "n_stored_blocks", "n_evicted")] + [
+        ("pressure", C.c_int32), ("save", C.c_int32), ("tail_block", C.c_int32), ("reserved", C.c_int32),
+        ("keys", C.c_void_p), ("gpu_block", C.c_void_p), ("gpu_resident", C.c_void_p),
+        ("needs_fill", C.c_void_p), ("hit", C.c_void_p), ("admit", C.c_void_p), ("slot", C.c_void_p),
+        ("evicted_keys", C.c_void_p), ("evicted_slots", C.c_void_p)]
+
+
+def _view_array(ptr, n, dtype):
+    """Copy n items of a context-owned host array (valid until the next turn) into numpy."""
+    if n <= 0 or not ptr:
+        return np.zeros(0, dtype=dtype)
+    nbytes = n * np.dtype(dtype).itemsize
+    buf = (C.c_uint8 * nbytes).from_address(ptr)
+    return np.frombuffer(buf, dtype=dtype).copy()
+
+
 EXPORTS = [
     "eakv_config_init", "eakv_create", "eakv_destroy", "eakv_hash_blocks",
     "eakv_hash_blocks_batched", "eakv_match", "eakv_tier_step", "eakv_gpu_tier_step",
     "eakv_gpu_tier_release", "eakv_store", "eakv_load", "eakv_sync", "eakv_get_stats",
     "eakv_tier_ptr", "eakv_hash_seed", "eakv_hash_base", "eakv_strerror", "eakv_last_cuda_error",
     "eakv_hash_blocks_static", "eakv_load_layers", "eakv_reuse_distances", "eakv_capacity_curve",
+    "eakv_turn_begin", "eakv_turn_end",
 ]
 STATIC_MAX_BLOCKS = 65536
 
@@ -99,6 +119,8 @@ def lib():
     L.eakv_load_layers.argtypes = [vp, vp, vp, i64, i32, vp, i32, vp]
     L.eakv_reuse_distances.argtypes = [vp, i64, vp, vp]
     L.eakv_capacity_curve.argtypes = [vp, i64, vp, vp, vp, i64, i32, vp, i32, vp, vp, vp, vp, vp]
+    L.eakv_turn_begin.argtypes = [vp, vp, i64, vp, i64, i64, i64, vp, C.POINTER(TurnView)]
+    L.eakv_turn_end.argtypes = [vp, vp]
     L.eakv_sync.argtypes = [vp]
     L.eakv_get_stats.argtypes = [vp, C.POINTER(Stats)]
     L.eakv_tier_ptr.argtypes = [vp]
@@ -332,6 +354,30 @@ class Context:
         rc = lib().eakv_load_layers(self._h, hsp, btp, len(bt), int(layers_per_group),
                                     C.cast(ev, C.c_void_p), len(events), _stream(stream))
         self._check(rc, "eakv_load_layers")
+
+    def eakv_turn_begin(self, tokens_ptr, n_tokens, known_keys, agent_id, now_ms, stream=None):
+        """First half of a turn; returns a dict of the view's scalars and (copied) arrays."""
+        kp, nk = None, 0
+        if known_keys is not None and len(known_keys):
+            kk, kp = _np(known_keys, np.uint64)
+            nk = len(kk)
+        v = TurnView()
+        rc = lib().eakv_turn_begin(self._h, C.c_void_p(int(tokens_ptr)), int(n_tokens), kp, nk,
+                                   int(agent_id), int(now_ms), _stream(stream), C.byref(v))
+        self._check(rc, "eakv_turn_begin")
+        nb, nu, ne = v.n_blocks, v.n_units, v.n_evicted
+        out = {n: getattr(v, n) for n, _ in TurnView._fields_[:15] if n != "reserved"}
+        out.update(keys=_view_array(v.keys, nb, np.uint64), gpu_block=_view_array(v.gpu_block, nb, np.int32),
+                   gpu_resident=_view_array(v.gpu_resident, nb, np.uint8),
+                   needs_fill=_view_array(v.needs_fill, nb, np.uint8),
+                   hit=_view_array(v.hit, nu, np.uint8), admit=_view_array(v.admit, nu, np.uint8),
+                   slot=_view_array(v.slot, nu, np.int32),
+                   evicted_keys=_view_array(v.evicted_keys, ne, np.uint64),
+                   evicted_slots=_view_array(v.evicted_slots, ne, np.int32))
+        return out
+
+    def eakv_turn_end(self, stream=None):
+        self._check(lib().eakv_turn_end(self._h, _stream(stream)), "eakv_turn_end")
 
     def eakv_sync(self):
         self._check(lib().eakv_sync(self._h), "eakv_sync")

@@ -39,7 +39,7 @@ class PagedPool:
 class AgentServer:
     def __init__(self, shape, gpu_blocks, host_blocks, payload, *, device="cuda:0",
                  gpu_index_blocks=0, incremental_hash=False, data_plane=True, chunk_blocks=1,
-                 **ctx_kwargs):
+                 native_turn=False, **ctx_kwargs):
         """``payload(keys, q, n_words)`` returns the int16/uint16 words of piece q for the
         blocks with these keys, as a numpy array or a tensor on ``device``.  With
         ``chunk_blocks`` = R > 1 the host tier works in chunks of R blocks (``host_blocks``
@@ -67,6 +67,9 @@ class AgentServer:
         self.stream = torch.cuda.current_stream(self.device)
         self.b = shape.block_size
         self.R = max(1, int(chunk_blocks))
+        self.native_turn = native_turn     # drive turns through eakv_turn_begin / eakv_turn_end
+        if native_turn and not data_plane:
+            raise ValueError("the two-call turn engine always moves KV bytes: it needs the data plane")
         self.seed = self.ctx.eakv_hash_seed()
         self._agent_keys = {}          # agent -> np.uint64 keys of its previous prompt
         self._timed = {"load": [], "store": []}     # (bytes, start event, end event)
@@ -136,8 +139,41 @@ class AgentServer:
         return out
 
     # -- one request ------------------------------------------------------------------------
+    def _turn_native(self, tokens, agent, now_ms):
+        """The same turn through the library's two-call engine: lookup, bookkeeping and the
+        restore happen inside eakv_turn_begin, the store inside eakv_turn_end."""
+        n = len(tokens)
+        self._ensure_pinned(max(n, 1))
+        self._tok_pin.numpy()[:n] = tokens
+        known = self._agent_keys.get(agent) if self.incremental else None
+        v = self.ctx.eakv_turn_begin(self._tok_pin.data_ptr(), n, known, agent, now_ms, self.stream)
+        keys, blocks = v["keys"], v["gpu_block"]
+        if self.incremental:
+            self._agent_keys[agent] = keys
+        fill = np.nonzero(v["needs_fill"])[0]
+        if len(fill) and self.data_plane:
+            ids = torch.as_tensor(blocks[fill].astype(np.int64), device=self.device)
+            for q, piece in enumerate(self.pool.pieces):
+                w = self.payload(keys[fill], q, self.pool.words)
+                if isinstance(w, np.ndarray):
+                    w = torch.from_numpy(w.view(np.int16)).to(self.device)
+                piece[ids] = w.view(torch.int16)
+        self.ctx.eakv_turn_end(self.stream)
+        G, H = v["gpu_prefix_blocks"], v["host_prefix_blocks"]
+        rec = dict(agent=agent, now_ms=now_ms, n_tokens=n, keys=keys, G=G, H=H,
+                   new_chunks=v["new_chunks"], pressure=bool(v["pressure"]), save=bool(v["save"]),
+                   hit=v["hit"], admit=v["admit"], slot=v["slot"],
+                   evicted=list(zip(v["evicted_keys"].tolist(), v["evicted_slots"].tolist())),
+                   gpu_resident=v["gpu_resident"], gpu_block=blocks,
+                   loaded=v["restore_hi"] - v["restore_lo"], stored=v["n_stored_blocks"],
+                   fresh_tokens=v["fresh_tokens"], filled=int(v["n_fill"]))
+        return rec, G, H
+
     def turn(self, tokens, agent, now_ms):
         tokens = np.asarray(tokens, dtype=np.int32)
+        if self.native_turn:
+            rec, G, H = self._turn_native(tokens, agent, now_ms)
+            return self._account(rec, G, H)
         n = len(tokens)
         keys = self.block_keys(tokens, agent)
         nblk = len(keys)
@@ -188,8 +224,11 @@ class AgentServer:
                    gpu_resident=resident, gpu_block=blocks, loaded=hi - lo,
                    stored=int(admit_b.sum()), fresh_tokens=n - cover * self.b,
                    filled=len(fill))
+        return self._account(rec, G, H)
+
+    def _account(self, rec, G, H):
         t = self.totals
-        t["prompt_tokens"] += n
+        t["prompt_tokens"] += rec["n_tokens"]
         t["fresh_tokens"] += rec["fresh_tokens"]
         t["loaded_blocks"] += rec["loaded"]
         t["stored_blocks"] += rec["stored"]

@@ -59,7 +59,7 @@ def plan(cfg, trace, shape, host_gib=None, data_plane=True, ram_fraction=0.6):
 
 def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=True,
         incremental_hash=True, device="cuda:0", link_strategy=eakv.LINK_STAGED, agents=None,
-        turns=None, server_hook=None, chunk_blocks=1, kappa=None):
+        turns=None, server_hook=None, chunk_blocks=1, kappa=None, native_turn=False):
     import torch
     from eakv_workloads import CONFIGS, SHAPES, key_words_torch, make_trace
     from .harness import AgentServer
@@ -74,7 +74,8 @@ def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=Tru
     server = AgentServer(shape, cfg.gpu_blocks, kh, payload, device=device, data_plane=data_plane,
                          incremental_hash=incremental_hash, policy=POLICIES[policy],
                          kappa_blocks=cfg.kappa_blocks if kappa is None else kappa,
-                         link_strategy=link_strategy, chunk_blocks=chunk_blocks)
+                         link_strategy=link_strategy, chunk_blocks=chunk_blocks,
+                         native_turn=native_turn and data_plane)
     t_setup = time.perf_counter() - t0
     t0 = time.perf_counter()
     server.run(trace, limit=limit)
@@ -90,7 +91,7 @@ def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=Tru
         "config": config, "policy": policy, "requests": n_req, "kv_shape": cfg.shape,
         "gpu_blocks": cfg.gpu_blocks, "host_chunks": kh, "chunk_blocks": chunk_blocks,
         "host_gib": kh * chunk_blocks * shape.block_bytes / GIB,
-        "host_sizing": why, "data_plane": data_plane,
+        "host_sizing": why, "data_plane": data_plane, "native_turn": bool(native_turn and data_plane),
         "working_set_blocks_eq5": working_set_blocks(trace, shape),
         "prompt_tokens": tot["prompt_tokens"], "computed_prefill_tokens": tot["fresh_tokens"],
         "gpu_hit_tokens": tot["gpu_hit_blocks"] * shape.block_size,
@@ -121,9 +122,12 @@ def main():
     ap.add_argument("--chunk-blocks", type=int, default=1,
                     help="host-tier chunk in GPU blocks (64 = the paper's 1,024-token chunks at block 16)")
     ap.add_argument("--kappa", type=int, default=None, help="write threshold in tier units")
+    ap.add_argument("--native-turn", action="store_true",
+                    help="drive turns through eakv_turn_begin / eakv_turn_end")
     args = ap.parse_args()
     out = run(args.config, policy=args.policy, host_gib=args.host_gib, limit=args.limit,
               data_plane=args.data_plane, chunk_blocks=args.chunk_blocks, kappa=args.kappa,
+              native_turn=args.native_turn,
               link_strategy=eakv.LINK_ZERO_COPY if args.zero_copy else eakv.LINK_STAGED)
     print(json.dumps(out))
 

@@ -161,3 +161,45 @@ def test_two_granularities_bit_exact(R, policy, link):
         for key, blk in oracle.gpu.order.items():
             assert np.array_equal(got[blk], oracle.pool[q][blk])
     server.close()
+
+
+@pytest.mark.parametrize("cfg_name,R,policy,incremental", [
+    ("c0", 1, 0, False), ("c0_big_tier", 1, 0, True), ("c0_big_tier", 4, 0, True),
+    ("c0", 1, 2, True), ("c0", 2, 1, False)])
+def test_native_turn_engine_bit_exact(cfg_name, R, policy, incremental):
+    """eakv_turn_begin / eakv_turn_end (lookup, bookkeeping, restore and store inside the
+    library) against the oracle: every record and every resident byte."""
+    from paper_2609_33762_b200 import eakv
+    from paper_2609_33762_b200.harness import AgentServer
+    cfg = CONFIGS[cfg_name]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg)
+    kh = cfg.host_blocks // R
+    kw = dict(policy=policy, kappa_blocks=20, window_ms=40, len_window=16)
+    oracle = TraceOracle(shape, cfg.gpu_blocks, kh, payload=key_words_numpy, chunk_blocks=R, **kw)
+    oracle.run(trace)
+    server = AgentServer(shape, cfg.gpu_blocks, kh, key_words_numpy, chunk_blocks=R, native_turn=True,
+                         incremental_hash=incremental, **kw)
+    server.run(trace)
+    compare_records(server.records, oracle.records)
+    assert server.totals == oracle.totals
+    server.ctx.eakv_sync()
+    tier = server.ctx.tier_host_view()
+    for key, slot in oracle.host.order.items():
+        for i in range(R):
+            assert np.array_equal(tier[slot * R + i], oracle.tier[slot * R + i])
+    for q, t in enumerate(server.pool.pieces):
+        got = t.cpu().numpy().view(np.uint8)
+        for key, blk in oracle.gpu.order.items():
+            assert np.array_equal(got[blk], oracle.pool[q][blk])
+    # protocol errors: end without begin, begin twice
+    with pytest.raises(eakv.EakvError) as ei:
+        server.ctx.eakv_turn_end()
+    assert ei.value.code == eakv.E_INVAL
+    toks = torch.zeros(64, dtype=torch.int32).pin_memory()
+    server.ctx.eakv_turn_begin(toks.data_ptr(), 40, None, 99, 10**6)
+    with pytest.raises(eakv.EakvError) as ei:
+        server.ctx.eakv_turn_begin(toks.data_ptr(), 40, None, 99, 10**6)
+    assert ei.value.code == eakv.E_INVAL
+    server.ctx.eakv_turn_end()
+    server.close()
