@@ -371,12 +371,12 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
 // B: the block size when known at compile time (16, 32, 64: loops unroll and every shared-memory
 // offset becomes an immediate), 0: read it from the launch descriptor.
 // multiply-add against limbs that sit in the kernel parameters (constant bank)
-#define EAKV_MACP(tok, e)                                          \
+#define EAKV_MACP(tok, e, A0, A1, A2)                              \
     do {                                                           \
         const uint32_t x_ = (uint32_t)(tok) + 1u;                  \
-        s0 += (uint64_t)x_ * L.pw_limbs[3 * (e) + 0];              \
-        s1 += (uint64_t)x_ * L.pw_limbs[3 * (e) + 1];              \
-        s2 += (uint64_t)x_ * L.pw_limbs[3 * (e) + 2];              \
+        A0 += (uint64_t)x_ * L.pw_limbs[3 * (e) + 0];              \
+        A1 += (uint64_t)x_ * L.pw_limbs[3 * (e) + 1];              \
+        A2 += (uint64_t)x_ * L.pw_limbs[3 * (e) + 2];              \
     } while (0)
 
 template <int B>
@@ -418,14 +418,20 @@ hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
     const int n_sub = (nb_tile + kHashThreads - 1) / kHashThreads;
     const int4* tile_src = reinterpret_cast<const int4*>(L.tokens + tok0 + first_blk * b);
 
+    // Every warp stages and consumes its own 32 rows, so the main loop needs no block-wide
+    // barrier: a warp waits for its own async copies and synchronises only with itself.
+    const int lane = tid & 31, warp = tid >> 5;
     auto issue = [&](int r) {
         const int nb = min(kHashThreads, nb_tile - r * kHashThreads);
-        const int chunks = nb * cpb;
+        const int nb_w = max(0, min(32, nb - warp * 32));
+        const int chunks_w = nb_w * cpb;
+        const int first_chunk = warp * 32 * cpb;
         const int4* src = tile_src + (size_t)r * kHashThreads * cpb;
         unsigned char* st = stage0 + (r & 1) * stage_bytes;
-        for (int c = tid; c < chunks; c += kHashThreads) {
-            const int row = c / cpb, col = c - row * cpb;
-            cp_async16(st + (size_t)row * row_bytes + col * 16, src + c);
+        for (int c = lane; c < chunks_w; c += 32) {
+            const int cg = first_chunk + c;
+            const int row = cg / cpb, col = cg - row * cpb;
+            cp_async16(st + (size_t)row * row_bytes + col * 16, src + cg);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
@@ -437,6 +443,7 @@ hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
             pw3[e] = make_uint4((uint32_t)(w & 0x1FFFFF), (uint32_t)((w >> 21) & 0x1FFFFF),
                                 (uint32_t)(w >> 42), 0u);
         }
+        __syncthreads();     // the limb table is shared by the whole CTA
     }
     uint64_t* partial = L.partial + blk0;
     for (int r = 0; r < n_sub; ++r) {
@@ -446,20 +453,22 @@ hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
         } else {
             asm volatile("cp.async.wait_group 0;" ::: "memory");
         }
-        __syncthreads();
+        __syncwarp();
         const int j = r * kHashThreads + tid;
         if (j < nb_tile) {
             const int4* row = reinterpret_cast<const int4*>(stage0 + (r & 1) * stage_bytes + (size_t)tid * row_bytes);
             uint64_t acc = 0;
             if (B) {   // b <= 64 < kLimbFoldTokens: one fold per block, fully unrolled
-                uint64_t s0 = 0, s1 = 0, s2 = 0;
+                // two independent accumulator sets: six multiply-add chains in flight
+                uint64_t s0 = 0, s1 = 0, s2 = 0, t0 = 0, t1 = 0, t2 = 0;
 #pragma unroll
                 for (int k = 0; k < (B ? B : 4); k += 4) {
                     const int4 u = row[k >> 2];
                     const int e = (B ? B : 4) - 1 - k;
-                    EAKV_MACP(u.x, e); EAKV_MACP(u.y, e - 1); EAKV_MACP(u.z, e - 2); EAKV_MACP(u.w, e - 3);
+                    EAKV_MACP(u.x, e, s0, s1, s2); EAKV_MACP(u.y, e - 1, t0, t1, t2);
+                    EAKV_MACP(u.z, e - 2, s0, s1, s2); EAKV_MACP(u.w, e - 3, t0, t1, t2);
                 }
-                acc = fold_limb_sums(s0, s1, s2);
+                acc = fold_limb_sums(s0 + t0, s1 + t1, s2 + t2);
             } else {
                 for (int k0 = 0; k0 < b; k0 += kLimbFoldTokens) {
                     const int k1 = min(b, k0 + kLimbFoldTokens);
@@ -475,7 +484,7 @@ hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
             }
             __stcg(partial + first_blk + j, acc);
         }
-        __syncthreads();     // the stage is refilled two iterations from now
+        __syncwarp();        // this warp refills the stage two iterations from now
     }
     __threadfence();
     __syncthreads();
