@@ -13,6 +13,10 @@
 // scan.  No CTA ever waits for another, so there is no spin loop anywhere.
 #include "eakv_internal.h"
 
+#ifndef EAKV_HASH_MIN_CTAS
+#define EAKV_HASH_MIN_CTAS 1
+#endif
+
 namespace eakv {
 
 static constexpr uint64_t P61 = (1ull << 61) - 1;
@@ -380,7 +384,7 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
     } while (0)
 
 template <int B>
-__global__ void __launch_bounds__(kHashThreads)
+__global__ void __launch_bounds__(kHashThreads, EAKV_HASH_MIN_CTAS)
 hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ Pair warp_tot[32];
