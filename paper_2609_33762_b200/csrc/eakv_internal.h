@@ -51,7 +51,10 @@ inline bool hash_thread_per_block(int block_size) { return (block_size % 4) != 0
 // blocks per CTA tile; large batches get longer tiles so fewer CTAs take tickets
 inline int hash_tile_blocks(int block_size, int64_t total_blocks) {
     if (hash_thread_per_block(block_size)) {
-        if (const char* e = getenv("EAKV_TUNE_HASH_TILE")) return atoi(e);
+        if (const char* e = getenv("EAKV_TUNE_HASH_TILE")) {   // developer override for sweeps
+            const int v = atoi(e);
+            if (v >= 1) return v;
+        }
         int t = kHashThreads;
         while (t < 16 * kHashThreads && total_blocks / t > 1184) t *= 2;   // up to a whole 64k-token prompt per CTA
         return t;
