@@ -56,7 +56,7 @@ extern "C" {
 
 /* how bytes cross the host link */
 #define EAKV_LINK_ZERO_COPY 0   /* kernels read/write the mapped pinned tier directly          */
-#define EAKV_LINK_STAGED    1   /* gather to HBM staging + copy engine on a side stream,
+#define EAKV_LINK_STAGED    1   /* (default) gather to HBM staging + copy engine on a side stream,
                                    double-buffered against the next gather (and the mirror) */
 
 /* where the tier lives */
@@ -75,13 +75,14 @@ typedef struct eakv_ctx eakv_ctx;
 typedef struct eakv_config {
     int32_t num_layers, kv_heads, head_dim, block_size, elem_bytes;
     int64_t gpu_blocks;            /* NB: blocks in each of the 2L paged arrays                 */
-    int64_t host_blocks;           /* K_H = floor(C_H / (b * beta)): tier capacity in blocks    */
+    int64_t host_blocks;           /* K_H = floor(C_H / (b * beta)): tier capacity in blocks
+                                      (in chunks when chunk_blocks > 1)                          */
     int64_t gpu_index_blocks;      /* K_G: blocks the GPU-tier LRU hands out (<= gpu_blocks);
                                       0 = gpu_blocks                                             */
     void* const* kv_base;          /* host array of 2L device pointers (copied at create)       */
     uint64_t hash_base, hash_seed; /* B and S of the prefix hash; 0 = library defaults          */
     int32_t policy;                /* EAKV_POLICY_*                                              */
-    int32_t kappa_blocks;          /* write threshold kappa, in blocks                           */
+    int32_t kappa_blocks;          /* write threshold kappa, in tier units (blocks, or chunks)   */
     int32_t theta_percent;         /* occupancy threshold theta, in percent (paper: 95)          */
     int32_t len_window;            /* prompt-length window, in requests (paper: 256)             */
     int64_t window_ms;             /* activity / eviction window (paper: 60 s)                   */
@@ -245,7 +246,9 @@ int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_tab
  * eakv_turn_end: eakv_store of the admitted blocks on cuda_stream, and release of the partial
  * tail's temporary block.  One turn per context at a time.
  * Errors: those of the calls above; EAKV_E_INVAL when a turn is already open (begin) or none
- * is (end).  On an error in begin no turn is opened; bookkeeping done by then is kept. */
+ * is (end).  On an error in begin no turn is opened; bookkeeping done by then is kept.
+ * eakv_turn_begin hashes on the context's own stream with the context's hash scratch: do not
+ * run eakv_hash_blocks of the same context concurrently with it. */
 typedef struct eakv_turn_view {
     int64_t n_blocks;             /* full blocks of the prompt                              */
     int64_t n_units;              /* tier units (= n_blocks / chunk_blocks)                 */
