@@ -93,9 +93,12 @@ class TraceOracle:
         self.totals = dict(prompt_tokens=0, fresh_tokens=0, loaded_blocks=0, stored_blocks=0,
                            gpu_hit_blocks=0, host_hit_blocks=0)
 
-    def turn(self, tokens, agent, now_ms):
+    def turn(self, tokens, agent, now_ms, keys=None):
+        """``keys``: the prompt's block keys if the caller already has them (prompts that only
+        grow by appends share their prefix keys with the previous turn); else they are hashed."""
         n = len(tokens)
-        keys = ohash.hash_blocks(tokens, self.b, self.hash_seed, self.hash_base)
+        if keys is None:
+            keys = ohash.hash_blocks(tokens, self.b, self.hash_seed, self.hash_base)
         G = 0
         for k in keys:
             if k not in self.gpu:

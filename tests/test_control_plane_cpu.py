@@ -245,3 +245,36 @@ def test_shared_system_prompt_is_deduplicated_across_agents(eakv):
     plain = TraceOracle(shape, cfg.gpu_blocks, cfg.host_blocks)
     plain.run(make_trace(CONFIGS["c0_big_tier"]))
     assert oracle.totals["stored_blocks"] < plain.totals["stored_blocks"]
+
+
+def test_config3_full_trace_control_plane_on_cpu(eakv):
+    """All 1,280 requests (3.88 M references) of the config 2/3 trace at the 32 GiB tier under
+    capacity-conditioned admission, through the C++ control plane and the oracle."""
+    cfg = CONFIGS["c3"]
+    shape = SHAPES[cfg.shape]
+    b = shape.block_size
+    trace = make_trace(cfg)
+    agent_keys = {a: ohash.hash_blocks(t.tolist(), b) for a, t in trace.agent_tokens.items()}
+    kw = dict(policy=2, kappa_blocks=cfg.kappa_blocks)
+    oracle = TraceOracle(shape, cfg.gpu_blocks, cfg.host_blocks, **kw)
+    ctx = cp_ctx(eakv, b, cfg.gpu_blocks, cfg.host_blocks, **kw)
+    for r in trace.requests:
+        keys = agent_keys[r.agent][: r.n_tokens // b]
+        w = oracle.turn(range(r.n_tokens), r.agent, r.time_ms, keys=keys)
+        k = as_keys(keys)
+        G, H, _, _ = ctx.eakv_match(k)
+        st = ctx.eakv_tier_step(k, r.agent, r.n_tokens, r.time_ms)
+        res, blk, tail = ctx.eakv_gpu_tier_step(k, r.n_tokens % b != 0)
+        if tail >= 0:
+            ctx.eakv_gpu_tier_release(tail)
+        assert (G, H, st["pressure"], st["save"]) == (w["G"], w["H"], w["pressure"], w["save"])
+        assert np.array_equal(st["admit"], np.asarray(w["admit"], dtype=np.uint8))
+        assert np.array_equal(st["slot"], np.asarray(w["slot"], dtype=np.int32))
+        assert np.array_equal(blk, np.asarray(w["gpu_block"], dtype=np.int32))
+        oracle.records.clear()
+    st = ctx.eakv_get_stats()
+    for f in ("requests", "references", "hits", "admitted", "declined", "evicted", "declined_requests",
+              "pressure_requests"):
+        assert st[f] == oracle.host.stats[f], f
+    assert 0 < st["declined_requests"] < st["requests"]
+    ctx.close()
