@@ -592,6 +592,8 @@ int eakv_hash_blocks(eakv_ctx* ctx, const int32_t* tokens_dev, int64_t n_tokens,
         L.single_parent_ptr = done ? hashes_dev + done - 1 : nullptr;
         L.block_size = b;
         L.tile_blocks = tile_blocks;
+        L.stages = hash_stages(b);
+        L.pad0 = 0;
         L.tokens_limit = n_tokens - done * b;
         L.blocks_limit = cur;
         L.error_flag = ctx->d_error_flag;
@@ -683,6 +685,8 @@ int eakv_hash_blocks_batched(eakv_ctx* ctx, const int32_t* tokens_dev,
     L.single_parent_ptr = nullptr;
     L.block_size = b;
     L.tile_blocks = tile_blocks;
+    L.stages = hash_stages(b);
+    L.pad0 = 0;
     L.tokens_limit = offsets_host[n_prompts];
     L.blocks_limit = total_blocks;
     L.error_flag = ctx->d_error_flag;

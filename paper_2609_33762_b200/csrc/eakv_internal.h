@@ -37,11 +37,13 @@ struct HashLaunch {
     const uint64_t* single_parent_ptr;   // non-NULL: read the parent from device memory instead
     int32_t block_size;
     int32_t tile_blocks;
-    // self-check limits: a CTA whose tile would reach past them raises *error_flag and skips
+    int32_t stages;                 // staged kernel: sub-tiles in flight per warp (2..4)
+    int32_t pad0;
     // B^e for e < 64 as three 21-bit limbs each, passed by value: with the block size known at
     // compile time they become constant-bank operands of the multiply-adds (no load at all)
     uint32_t pw_limbs[3 * 64];
     uint64_t pow_block;             // A = B^b, the per-block multiplier of the scan
+    // self-check limits: a CTA whose tile would reach past them raises *error_flag and skips
     int64_t tokens_limit;           // tokens readable at `tokens`
     int64_t blocks_limit;           // entries writable at `keys` and `partial`
     int* error_flag;
@@ -71,6 +73,15 @@ inline void hash_fill_limbs(HashLaunch& L, const uint64_t* pow_host, int block_s
         L.pw_limbs[3 * e + 2] = (uint32_t)(w >> 42);
     }
     L.pow_block = pow_host[block_size];
+}
+// Sub-tiles in flight per warp in the staged kernel.  Two is the measured optimum: three and
+// four (more shared memory, fewer CTAs per SM) were 3-10 % slower.
+inline int hash_stages(int block_size) {
+    if (const char* e = getenv("EAKV_TUNE_HASH_STAGES")) {      // developer override for sweeps
+        const int v = atoi(e);
+        if (v >= 2 && v <= 4 && (size_t)v * kHashThreads * (4 * block_size + 16) <= 136 * 1024) return v;
+    }
+    return 2;
 }
 cudaError_t hash_kernels_init();
 cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool thread_per_block, bool vec,

@@ -395,6 +395,7 @@ hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
     uint4* pw3 = reinterpret_cast<uint4*>(smem_raw);
     unsigned char* const stage0 = smem_raw + (size_t)b * 16;
     const size_t stage_bytes = (size_t)kHashThreads * row_bytes;
+    const int S = L.stages;
     int32_t p = 0;
     int64_t first_blk = (int64_t)blockIdx.x * L.tile_blocks;
     int64_t tok0 = 0, blk0 = 0, nblk = L.single_nblk;
@@ -431,7 +432,7 @@ hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
         const int chunks_w = nb_w * cpb;
         const int first_chunk = warp * 32 * cpb;
         const int4* src = tile_src + (size_t)r * kHashThreads * cpb;
-        unsigned char* st = stage0 + (r & 1) * stage_bytes;
+        unsigned char* st = stage0 + (r % S) * stage_bytes;
         for (int c = lane; c < chunks_w; c += 32) {
             const int cg = first_chunk + c;
             const int row = cg / cpb, col = cg - row * cpb;
@@ -440,7 +441,12 @@ hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
 
-    issue(0);
+    // exactly one group is committed per sub-tile slot (empty past the end), so "all but the
+    // newest S-1 groups are complete" always means that sub-tile r has landed
+    for (int r = 0; r < S - 1; ++r) {
+        if (r < n_sub) issue(r);
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+    }
     if (!B) {
         for (int e = tid; e < b; e += blockDim.x) {
             const uint64_t w = L.pow_table[e];
@@ -451,16 +457,15 @@ hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
     }
     uint64_t* partial = L.partial + blk0;
     for (int r = 0; r < n_sub; ++r) {
-        if (r + 1 < n_sub) {
-            issue(r + 1);
-            asm volatile("cp.async.wait_group 1;" ::: "memory");
-        } else {
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-        }
+        if (r + S - 1 < n_sub) issue(r + S - 1);
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+        if (S == 2)      asm volatile("cp.async.wait_group 1;" ::: "memory");
+        else if (S == 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
+        else             asm volatile("cp.async.wait_group 3;" ::: "memory");
         __syncwarp();
         const int j = r * kHashThreads + tid;
         if (j < nb_tile) {
-            const int4* row = reinterpret_cast<const int4*>(stage0 + (r & 1) * stage_bytes + (size_t)tid * row_bytes);
+            const int4* row = reinterpret_cast<const int4*>(stage0 + (r % S) * stage_bytes + (size_t)tid * row_bytes);
             uint64_t acc = 0;
             if (B) {   // b <= 64 < kLimbFoldTokens: one fold per block, fully unrolled
                 // two independent accumulator sets: six multiply-add chains in flight
@@ -488,7 +493,7 @@ hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
             }
             __stcg(partial + first_blk + j, acc);
         }
-        __syncwarp();        // this warp refills the stage two iterations from now
+        __syncwarp();        // this warp refills the stage S-1 iterations from now
     }
     __threadfence();
     __syncthreads();
@@ -511,7 +516,7 @@ cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool thread_per_block,
     if (n_tiles <= 0) return cudaSuccess;
     if (thread_per_block) {
         const size_t smem = (size_t)L.block_size * sizeof(uint4);
-        const size_t staged = smem + 2 * (size_t)kHashThreads * (4 * L.block_size + 16);
+        const size_t staged = smem + (size_t)L.stages * kHashThreads * (4 * L.block_size + 16);
         if (!vec)                    hash_blocks_tpb_kernel<false><<<n_tiles, kHashThreads, smem, stream>>>(L);
         else if (L.block_size == 16) hash_blocks_staged_kernel<16><<<n_tiles, kHashThreads, staged, stream>>>(L);
         else if (L.block_size == 32) hash_blocks_staged_kernel<32><<<n_tiles, kHashThreads, staged, stream>>>(L);
@@ -658,6 +663,8 @@ extern "C" int eakv_hash_blocks_static(const int32_t* tokens_dev, int64_t n_toke
     L.single_parent_ptr = nullptr;
     L.block_size = block_size;
     L.tile_blocks = hash_tile_blocks(block_size, nblk);
+    L.stages = hash_stages(block_size);
+    L.pad0 = 0;
     {   // powers B^0 .. B^b on the host (at most 4,097 modular products) for the by-value limbs
         uint64_t pw_host[65];
         const int lim = block_size < 64 ? block_size : 64;
