@@ -337,11 +337,19 @@ def hash_throughput(torch, eakv, pool, shape, device, peak_gbs, prompts=512, tok
     ctx.close()
     rate = prompts * tokens / (best * 1e-3)
     srate = prompts * tokens / (sustained * 1e-3)
+    # multiply-pipe ceiling from stand-alone measurements on this GPU type: 31.5 wide (32x32->64)
+    # multiply-adds and 2.3 modular 61-bit products per SM per clock; 3 of the former per token
+    # and 2.7 of the latter per block
+    props = torch.cuda.get_device_properties(device)
+    clk_hz = 1.965e9
+    alu_bound = props.multi_processor_count * clk_hz / (3 / 31.5 + 2.7 / shape.block_size / 2.3)
     return {"sustained_tokens_per_s": srate, "sustained_ms_per_launch": sustained,
             "sustained_frac_of_hbm_bound": srate * 4 / 1e9 / peak_gbs,
             "batched_tokens_per_s": rate, "batch": f"{prompts} prompts x {tokens} tokens, block {shape.block_size}",
             "batched_ms": best, "frac_of_hbm_bound": rate * 4 / 1e9 / peak_gbs,
             "hbm_bound_tokens_per_s": peak_gbs * 1e9 / 4,
+            "multiply_pipe_bound_tokens_per_s": alu_bound,
+            "sustained_frac_of_multiply_pipe_bound": srate / alu_bound,
             "single_prompt_tokens": tokens, "single_prompt_us_median": float(np.median(single))}
 
 
