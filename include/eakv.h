@@ -70,6 +70,13 @@ extern "C" {
                                    used for device-resident buffers only: a mapped host tier
                                    under EAKV_LINK_ZERO_COPY is always moved by the vector kernel */
 
+/* GPU-tier recency order of one request's blocks after eakv_gpu_tier_step (the GPU tier belongs
+ * to the serving engine in the paper, Section 2; both orders are this library's model of it) */
+#define EAKV_FREE_ASCENDING 0   /* as referenced: the prompt's first block is the request's least
+                                   recent, so it is the first of them to be evicted              */
+#define EAKV_FREE_REVERSE   1   /* tail first, the way a paged engine frees a sequence: the last
+                                   block is evicted first and what survives is still a prefix     */
+
 typedef struct eakv_ctx eakv_ctx;
 
 typedef struct eakv_config {
@@ -113,6 +120,9 @@ typedef struct eakv_config {
                                       buffer of host_blocks * chunk_blocks * block bytes (pinned host memory
                                       for TIER_PINNED_HOST, device memory for TIER_DEVICE);
                                       it must outlive the context                               */
+    int32_t gpu_free_order;        /* EAKV_FREE_*: recency order a request leaves its blocks in
+                                      within the GPU tier                                        */
+    int32_t reserved0;
 } eakv_config;
 
 typedef struct eakv_stats {

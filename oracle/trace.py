@@ -29,10 +29,16 @@ from .tier import HostTier
 
 
 class GpuTier:
-    """LRU of keyed GPU blocks with a free stack that first yields 0, 1, 2, ..."""
+    """LRU of keyed GPU blocks with a free stack that first yields 0, 1, 2, ...
 
-    def __init__(self, num_blocks):
+    ``free_order``: how a finished request leaves its blocks in the recency order.  0: as
+    referenced (the prompt's first block is the least recent of the request).  1: reversed,
+    the way a paged engine returns a sequence's blocks tail first, so that the tail is
+    evicted before the head and what survives of a sequence is still a prefix."""
+
+    def __init__(self, num_blocks, free_order=0):
         self.NB = int(num_blocks)
+        self.free_order = int(free_order)
         self.order = OrderedDict()                 # key -> block id, least recent first
         self.free = list(range(self.NB - 1, -1, -1))
 
@@ -61,6 +67,9 @@ class GpuTier:
                 resident.append(0)
                 ids.append(blk)
         tail = self._alloc() if need_tail else -1
+        if self.free_order == 1:
+            for k in reversed(keys):
+                self.order.move_to_end(k)
         return resident, ids, tail
 
     def release(self, block_id):
@@ -72,13 +81,13 @@ class TraceOracle:
     def __init__(self, shape, gpu_blocks, host_blocks, policy=0, kappa_blocks=8,
                  theta_percent=95, window_ms=60_000, len_window=256, telemetry=True,
                  payload=None, hash_base=ohash.HASH_BASE, hash_seed=ohash.HASH_SEED,
-                 chunk_blocks=1):
+                 chunk_blocks=1, gpu_free_order=0):
         """``payload(keys, q, n_words) -> uint16[len(keys), n_words]`` enables full-bytes
         mode (pool and tier held in numpy); None runs metadata only."""
         self.shape = shape
         self.b = shape.block_size
         self.R = int(chunk_blocks)
-        self.gpu = GpuTier(gpu_blocks)
+        self.gpu = GpuTier(gpu_blocks, gpu_free_order)
         self.host = HostTier(host_blocks, self.b * self.R, policy, kappa_blocks, theta_percent,
                              window_ms, len_window, telemetry)
         self.payload = payload

@@ -59,11 +59,11 @@ def reference_stream(trace, shape, device="cuda:0"):
     return stream, np.asarray(offsets, dtype=np.int64), np.asarray(tokens, dtype=np.int64)
 
 
-def gpu_prefixes(trace, shape, gpu_blocks, stream_host, offsets):
+def gpu_prefixes(trace, shape, gpu_blocks, stream_host, offsets, gpu_free_order=eakv.FREE_ASCENDING):
     """G_j of every request from the library's GPU-tier bookkeeping (control plane only)."""
     b = shape.block_size
     ctx = eakv.Context(num_layers=1, kv_heads=1, head_dim=8, block_size=b, gpu_blocks=gpu_blocks,
-                       host_blocks=1, kv_base=None, control_plane_only=True)
+                       host_blocks=1, kv_base=None, control_plane_only=True, gpu_free_order=gpu_free_order)
     G = np.zeros(len(trace.requests), dtype=np.int64)
     for j, r in enumerate(trace.requests):
         keys = stream_host[offsets[j]:offsets[j + 1]]
@@ -75,7 +75,8 @@ def gpu_prefixes(trace, shape, gpu_blocks, stream_host, offsets):
     return G
 
 
-def model(config, host_gib, device="cuda:0", limit=None, agents=None, shared_prefix=0):
+def model(config, host_gib, device="cuda:0", limit=None, agents=None, shared_prefix=0,
+          gpu_free_order=eakv.FREE_ASCENDING):
     import torch
     from dataclasses import replace
     from eakv_workloads import CONFIGS, SHAPES, make_trace
@@ -96,7 +97,7 @@ def model(config, host_gib, device="cuda:0", limit=None, agents=None, shared_pre
     eakv.eakv_reuse_distances(stream.data_ptr(), n_refs, dist.data_ptr())
     t_dist = time.perf_counter() - t0
     stream_host = stream.cpu().numpy().view(np.uint64)
-    G = gpu_prefixes(trace, shape, cfg.gpu_blocks, stream_host, offsets)
+    G = gpu_prefixes(trace, shape, cfg.gpu_blocks, stream_host, offsets, gpu_free_order)
     caps = [max(1, int(g * GIB // shape.block_bytes)) for g in host_gib] + [1 << 40]
     t0 = time.perf_counter()
     out = eakv.eakv_capacity_curve(dist.data_ptr(), n_refs, offsets, tokens, G, shape.block_size, caps)
@@ -112,6 +113,8 @@ def model(config, host_gib, device="cuda:0", limit=None, agents=None, shared_pre
                      "restored_tokens": int(out["restored_blocks"][c]) * shape.block_size,
                      "computed_prefill_tokens": int(out["computed_tokens"][c])})
     return {"config": config, "agents": len(trace.agent_tokens), "shared_prefix_tokens": shared_prefix,
+            "gpu_free_order": "reverse" if gpu_free_order == eakv.FREE_REVERSE else "ascending",
+            "gpu_hit_tokens": int(G.sum()) * shape.block_size,
             "requests": len(trace.requests), "references": n_refs,
             "prompt_tokens": int(tokens.sum()), "rows": rows,
             "computed_prefill_tokens_infinite_tier": inf_computed,
@@ -223,6 +226,8 @@ def main():
     ap.add_argument("--kappa-sweep", default=None, help="comma-separated thresholds, fixed admission")
     ap.add_argument("--agents", type=int, default=None, help="active pool size (default: the config's)")
     ap.add_argument("--shared-prefix", type=int, default=0, help="system-prompt tokens shared by all agents")
+    ap.add_argument("--reverse-free", action="store_true",
+                    help="GPU tier keeps a request's blocks tail-first in its recency order")
     args = ap.parse_args()
     gib = [float(x) for x in args.host_gib.split(",")]
     if args.kappa_sweep:
@@ -235,7 +240,8 @@ def main():
             print(json.dumps(audit(args.config, args.audit, g, kappa=args.kappa,
                                    chunk_blocks=args.chunk_blocks, limit=args.limit)))
         return
-    out = model(args.config, gib, limit=args.limit, agents=args.agents, shared_prefix=args.shared_prefix)
+    out = model(args.config, gib, limit=args.limit, agents=args.agents, shared_prefix=args.shared_prefix,
+                gpu_free_order=eakv.FREE_REVERSE if args.reverse_free else eakv.FREE_ASCENDING)
     print(json.dumps(out))
 
 

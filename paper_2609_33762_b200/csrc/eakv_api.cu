@@ -390,7 +390,8 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
     const int64_t chunk_blocks = cfg->chunk_blocks > 0 ? cfg->chunk_blocks : 1;
     if (cfg->gpu_blocks > INT32_MAX || cfg->host_blocks * chunk_blocks > INT32_MAX) return EAKV_E_INVAL;
     if (cfg->policy < 0 || cfg->policy > 2 || cfg->link_strategy < 0 || cfg->link_strategy > 1 ||
-        cfg->tier_location < 0 || cfg->tier_location > 1 || cfg->copy_path < 0 || cfg->copy_path > 1)
+        cfg->tier_location < 0 || cfg->tier_location > 1 || cfg->copy_path < 0 || cfg->copy_path > 1 ||
+        cfg->gpu_free_order < 0 || cfg->gpu_free_order > 1)
         return EAKV_E_INVAL;
     if (cfg->gpu_index_blocks < 0 || cfg->gpu_index_blocks > cfg->gpu_blocks) return EAKV_E_INVAL;
     const int64_t piece = (int64_t)cfg->block_size * cfg->kv_heads * cfg->head_dim * cfg->elem_bytes;
@@ -809,6 +810,8 @@ int eakv_gpu_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blo
         *tail_block_out = T.take_unkeyed(&ev, &vkey, &vslot);
         ctx->gpu_unkeyed += 1;
     }
+    if (ctx->cfg.gpu_free_order == EAKV_FREE_REVERSE)
+        for (int64_t j = n_blocks - 1; j >= 0; --j) T.promote(block_out[j]);
     return EAKV_OK;
 }
 

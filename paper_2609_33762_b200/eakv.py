@@ -13,6 +13,7 @@ OK, E_INVAL, E_RANGE, E_CAPACITY, E_NOMEM, E_CUDA, E_TIMEOUT = 0, -1, -2, -3, -4
 POLICY_WRITE_ALL, POLICY_FILTER_FIXED, POLICY_FILTER_CONDITIONED = 0, 1, 2
 LINK_ZERO_COPY, LINK_STAGED = 0, 1
 TIER_PINNED_HOST, TIER_DEVICE = 0, 1
+FREE_ASCENDING, FREE_REVERSE = 0, 1
 COPY_VECTOR, COPY_BULK = 0, 1
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libeakv.so")
@@ -43,6 +44,7 @@ class Config(C.Structure):
         ("hash_scratch_blocks", C.c_int64), ("min_staged_run_bytes", C.c_int64),
         ("control_plane_only", C.c_int32), ("chunk_blocks", C.c_int32),
         ("tier_memory", C.c_void_p),
+        ("gpu_free_order", C.c_int32), ("reserved0", C.c_int32),
     ]
 
 
@@ -200,7 +202,8 @@ class Context:
                  window_ms=60_000, telemetry=1, link_strategy=LINK_STAGED,
                  tier_location=TIER_PINNED_HOST, copy_path=COPY_BULK, copy_ctas=0,
                  staging_bytes=0, max_call_blocks=0, hash_scratch_blocks=0, min_staged_run_bytes=0,
-                 tier_memory=0, control_plane_only=False, chunk_blocks=1):
+                 tier_memory=0, control_plane_only=False, chunk_blocks=1,
+                 gpu_free_order=FREE_ASCENDING):
         L = lib()
         cfg = Config()
         L.eakv_config_init(C.byref(cfg))
@@ -214,6 +217,7 @@ class Context:
         cfg.kv_base = C.cast(ptrs, C.POINTER(C.c_void_p)) if kv_base else None
         cfg.control_plane_only = int(bool(control_plane_only))
         cfg.chunk_blocks = int(chunk_blocks)
+        cfg.gpu_free_order = int(gpu_free_order)
         cfg.hash_base, cfg.hash_seed = hash_base, hash_seed
         cfg.policy, cfg.kappa_blocks, cfg.theta_percent = policy, kappa_blocks, theta_percent
         cfg.len_window, cfg.window_ms, cfg.telemetry = len_window, window_ms, telemetry

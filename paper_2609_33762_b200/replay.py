@@ -59,7 +59,8 @@ def plan(cfg, trace, shape, host_gib=None, data_plane=True, ram_fraction=0.6):
 
 def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=True,
         incremental_hash=True, device="cuda:0", link_strategy=eakv.LINK_STAGED, agents=None,
-        turns=None, server_hook=None, chunk_blocks=1, kappa=None, native_turn=False):
+        turns=None, server_hook=None, chunk_blocks=1, kappa=None, native_turn=False,
+        gpu_free_order=eakv.FREE_ASCENDING):
     import torch
     from eakv_workloads import CONFIGS, SHAPES, key_words_torch, make_trace
     from .harness import AgentServer
@@ -75,7 +76,7 @@ def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=Tru
                          incremental_hash=incremental_hash, policy=POLICIES[policy],
                          kappa_blocks=cfg.kappa_blocks if kappa is None else kappa,
                          link_strategy=link_strategy, chunk_blocks=chunk_blocks,
-                         native_turn=native_turn and data_plane)
+                         native_turn=native_turn and data_plane, gpu_free_order=gpu_free_order)
     t_setup = time.perf_counter() - t0
     t0 = time.perf_counter()
     server.run(trace, limit=limit)
@@ -90,6 +91,7 @@ def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=Tru
     out = {
         "config": config, "policy": policy, "requests": n_req, "kv_shape": cfg.shape,
         "gpu_blocks": cfg.gpu_blocks, "host_chunks": kh, "chunk_blocks": chunk_blocks,
+        "gpu_free_order": "reverse" if gpu_free_order == eakv.FREE_REVERSE else "ascending",
         "host_gib": kh * chunk_blocks * shape.block_bytes / GIB,
         "host_sizing": why, "data_plane": data_plane, "native_turn": bool(native_turn and data_plane),
         "working_set_blocks_eq5": working_set_blocks(trace, shape),
@@ -124,10 +126,13 @@ def main():
     ap.add_argument("--kappa", type=int, default=None, help="write threshold in tier units")
     ap.add_argument("--native-turn", action="store_true",
                     help="drive turns through eakv_turn_begin / eakv_turn_end")
+    ap.add_argument("--reverse-free", action="store_true",
+                    help="GPU tier keeps a request's blocks tail-first in its recency order")
     args = ap.parse_args()
     out = run(args.config, policy=args.policy, host_gib=args.host_gib, limit=args.limit,
               data_plane=args.data_plane, chunk_blocks=args.chunk_blocks, kappa=args.kappa,
               native_turn=args.native_turn,
+              gpu_free_order=eakv.FREE_REVERSE if args.reverse_free else eakv.FREE_ASCENDING,
               link_strategy=eakv.LINK_ZERO_COPY if args.zero_copy else eakv.LINK_STAGED)
     print(json.dumps(out))
 

@@ -39,7 +39,7 @@ def test_config_defaults_and_layout(lib):
     assert (cfg.theta_percent, cfg.window_ms, cfg.len_window, cfg.kappa_blocks) == (95, 60000, 256, 8)
     assert cfg.policy == eakv.POLICY_WRITE_ALL and cfg.elem_bytes == 2
     assert cfg.link_strategy == eakv.LINK_STAGED and cfg.copy_path == eakv.COPY_BULK
-    assert C.sizeof(eakv.Config) == 168 and C.sizeof(eakv.Stats) == 128
+    assert C.sizeof(eakv.Config) == 176 and C.sizeof(eakv.Stats) == 128
     assert lib.eakv_config_init(None) == eakv.E_INVAL
 
 

@@ -89,12 +89,13 @@ def test_tier_step_random_requests(eakv, policy, telemetry):
         ctx.close()
 
 
-def test_gpu_tier_random_requests(eakv):
-    rng = random.Random(7)
+@pytest.mark.parametrize("free_order", [0, 1])
+def test_gpu_tier_random_requests(eakv, free_order):
+    rng = random.Random(7 + free_order)
     for case in range(60):
         NB = rng.randrange(2, 30)
-        ctx = cp_ctx(eakv, 4, NB, 4)
-        g = GpuTier(NB)
+        ctx = cp_ctx(eakv, 4, NB, 4, gpu_free_order=free_order)
+        g = GpuTier(NB, free_order)
         for _ in range(rng.randrange(3, 40)):
             agent = rng.randrange(4)
             tail = rng.random() < 0.5
@@ -278,3 +279,25 @@ def test_config3_full_trace_control_plane_on_cpu(eakv):
         assert st[f] == oracle.host.stats[f], f
     assert 0 < st["declined_requests"] < st["requests"]
     ctx.close()
+
+
+def test_reverse_free_order_whole_trace(eakv):
+    """C0 with the tail-first GPU recency order: every record equals the oracle's, and the GPU
+    tier keeps more prefix blocks than with the ascending order."""
+    cfg = CONFIGS["c0_big_tier"]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg, agents=3)      # three agents: the pool holds a part of each prompt
+    totals = {}
+    for order in (0, 1):
+        orc = TraceOracle(shape, cfg.gpu_blocks, cfg.host_blocks, gpu_free_order=order)
+        orc.run(trace)
+        ctx = cp_ctx(eakv, shape.block_size, cfg.gpu_blocks, cfg.host_blocks, gpu_free_order=order)
+        compare(drive(ctx, trace, shape.block_size), orc.records)
+        ctx.close()
+        totals[order] = orc.totals["gpu_hit_blocks"]
+    assert totals[1] > totals[0]
+
+
+def test_free_order_argument_is_checked(eakv):
+    with pytest.raises(eakv.EakvError):
+        cp_ctx(eakv, 4, 8, 8, gpu_free_order=2)

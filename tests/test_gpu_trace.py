@@ -203,3 +203,24 @@ def test_native_turn_engine_bit_exact(cfg_name, R, policy, incremental):
     assert ei.value.code == eakv.E_INVAL
     server.ctx.eakv_turn_end()
     server.close()
+
+
+@pytest.mark.parametrize("native", [False, True])
+def test_reverse_free_order_bit_exact(native):
+    """Tail-first GPU recency order (a request's last block is its least recent): records and
+    resident bytes equal the oracle's, with the step-by-step harness and the turn engine."""
+    from paper_2609_33762_b200 import eakv
+    from paper_2609_33762_b200.harness import AgentServer
+    cfg = CONFIGS["c0_big_tier"]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg, agents=3)
+    oracle = TraceOracle(shape, cfg.gpu_blocks, cfg.host_blocks, payload=key_words_numpy, gpu_free_order=1)
+    oracle.run(trace)
+    assert oracle.totals["gpu_hit_blocks"] > 0 and oracle.totals["loaded_blocks"] > 0
+    server = AgentServer(shape, cfg.gpu_blocks, cfg.host_blocks, key_words_numpy, native_turn=native,
+                         incremental_hash=True, gpu_free_order=eakv.FREE_REVERSE)
+    server.run(trace)
+    compare_records(server.records, oracle.records)
+    assert server.totals == oracle.totals
+    compare_bytes(server, oracle)
+    server.close()

@@ -299,3 +299,44 @@ def test_declined_audit_hand_case_and_kappa_sensitivity():
     assert filt == sorted(filt, reverse=True) and filt[-1] == 0 and filt[0] > 0
     assert out[10**9]["declined_chunks"] == 0
     assert audit.median([3, 1, 2]) == 2 and audit.median([4, 1, 2, 3]) == 2.5
+
+
+def test_gpu_tier_free_order_closed_cases():
+    """Pool of 10 blocks, request A = 6 blocks, then request B = 5 blocks: one block of A has to
+    go.  Ascending order loses A's first block (nothing of A is a resident prefix any more);
+    tail-first order loses A's last block (five of six stay a prefix)."""
+    from oracle.trace import GpuTier
+    A = [("a", j) for j in range(6)]
+    B = [("b", j) for j in range(5)]
+    lead = lambda g, ks: next((i for i, k in enumerate(ks) if k not in g), len(ks))
+    for order, want in ((0, 0), (1, 5)):
+        g = GpuTier(10, order)
+        g.step(A, False)
+        g.step(B, False)
+        assert lead(g, A) == want and lead(g, B) == 5
+        assert len(g.order) == 10
+
+
+def test_gpu_tier_free_order_against_timestamp_brute_force():
+    """Brute force with explicit time stamps: a request's block j gets stamp (t, j) in ascending
+    order and (t, -j) in tail-first order; the victim is always the smallest stamp."""
+    import random
+    from oracle.trace import GpuTier
+    rng = random.Random(3)
+    for order in (0, 1):
+        for case in range(40):
+            NB = rng.randrange(3, 16)
+            g = GpuTier(NB, order)
+            stamp = {}
+            for t in range(30):
+                agent = rng.randrange(3)
+                n = rng.randrange(1, NB + 1)
+                keys = [(agent, j) for j in range(n)]
+                # brute force: residents after the request = its keys plus the newest others
+                for j, k in enumerate(keys):
+                    stamp[k] = (t, -j if order else j)
+                while len(stamp) > NB:
+                    del stamp[min(stamp, key=stamp.get)]
+                g.step(keys, False)
+                assert set(g.order) == set(stamp)
+                assert list(g.order) == sorted(stamp, key=stamp.get)
