@@ -28,6 +28,11 @@ class Trace:
     config: TraceConfig
     requests: List[Request]
     agent_tokens: Dict[int, np.ndarray]  # agent -> int32[max prompt length of that agent]
+    # agent -> int64[turns]: tool/agent time in ms between the end of turn t-1 and turn t
+    # (entry 0 is 0).  ``requests`` is the open-loop order these gaps give with zero service
+    # time; a closed-loop replay takes the gaps and lengths and orders the calls itself.
+    agent_gaps_ms: Dict[int, np.ndarray] = None
+    agent_lengths: Dict[int, np.ndarray] = None   # agent -> int64[turns] prompt lengths
 
     def prompt(self, req: Request) -> np.ndarray:
         return self.agent_tokens[req.agent][: req.n_tokens]
@@ -64,6 +69,7 @@ def make_trace(cfg, seed=None, agents=None, turns=None) -> Trace:
 
     # request times
     times = np.zeros((A, T), dtype=np.int64)
+    gaps_ms = np.zeros((A, T), dtype=np.int64)
     if cfg.interleave == "round_robin":
         for t in range(T):
             for a in range(A):
@@ -76,6 +82,7 @@ def make_trace(cfg, seed=None, agents=None, turns=None) -> Trace:
             gaps = rng.exponential(cfg.tool_gap_mean_ms, size=T)
             gaps[0] = 0.0
             times[a] = np.floor(start[a] + np.cumsum(gaps)).astype(np.int64)
+            gaps_ms[a] = np.floor(gaps).astype(np.int64)
 
     # token ids: independent stream per agent, after an optional prefix common to all agents
     agent_tokens = {}
@@ -89,4 +96,6 @@ def make_trace(cfg, seed=None, agents=None, turns=None) -> Trace:
 
     reqs = [Request(int(times[a, t]), a, t, int(lengths[a, t])) for a in range(A) for t in range(T)]
     reqs.sort(key=lambda r: (r.time_ms, r.agent, r.turn))
-    return Trace(cfg, reqs, agent_tokens)
+    return Trace(cfg, reqs, agent_tokens,
+                 agent_gaps_ms={a: gaps_ms[a].copy() for a in range(A)},
+                 agent_lengths={a: lengths[a].copy() for a in range(A)})

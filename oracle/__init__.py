@@ -13,6 +13,8 @@ Modules
   stackdist   reuse (stack) distances, Mattson hit prediction, coverage prediction
   sizing      KV footprint, working-set scale, pressure ratios, offload benefit ratio
   trace       whole-trace driver: one agent turn = hash, match, tier step, load, store
+  audit       declined-chunk audit and threshold sensitivity
+  closedloop  closed-loop replay: active pool, first-come-first-served engine, Eq. 2 service times
 
 Parity unpinned: the paper's trace-level results (its prediction tables, replay table
 and declined-chunk shares) need the authors' recorded trajectories, which are not
