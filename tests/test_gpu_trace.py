@@ -224,3 +224,29 @@ def test_reverse_free_order_bit_exact(native):
     assert server.totals == oracle.totals
     compare_bytes(server, oracle)
     server.close()
+
+
+@pytest.mark.parametrize("policy,kh,pool,native", [(0, 1024, 3, False), (2, 200, 4, True), (0, 160, 8, False)])
+def test_closed_loop_replay_bit_exact(policy, kh, pool, native):
+    """Closed-loop replay on the GPU path: the call order that the service times produce, the
+    makespan, every record and every resident byte equal the oracle's closed-loop replay."""
+    from oracle import closedloop as ocl
+    from paper_2609_33762_b200 import closedloop
+    from paper_2609_33762_b200.harness import AgentServer
+    cfg = CONFIGS["c0_big_tier"]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg, agents=8, turns=8)
+    kw = dict(policy=policy, kappa_blocks=10, window_ms=50, len_window=16)
+    rates = dict(t_pf_ns=40_000, h2d_bytes_per_us=9_000, d2h_bytes_per_us=7_000, tau_load_us=120,
+                 call_overhead_us=33)
+    oracle = TraceOracle(shape, cfg.gpu_blocks, kh, payload=key_words_numpy, **kw)
+    want = ocl.replay(trace, oracle, ocl.ServiceModel(**rates), pool, shape.bytes_per_token)
+    server = AgentServer(shape, cfg.gpu_blocks, kh, key_words_numpy, incremental_hash=True,
+                         native_turn=native, **kw)
+    order, makespan, _ = closedloop.replay_trace(trace, server.turn, closedloop.ServiceModel(**rates), pool,
+                                                 shape.bytes_per_token, shape.block_size)
+    assert order == want["order"] and makespan == want["makespan_us"]
+    compare_records(server.records, oracle.records)
+    assert server.totals == oracle.totals
+    compare_bytes(server, oracle)
+    server.close()
