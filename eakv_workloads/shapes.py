@@ -34,6 +34,11 @@ class KVShape:
     def bytes_per_token(self) -> int:
         return self.block_bytes // self.block_size
 
+    def tp_shard(self, tp: int) -> "KVShape":
+        """One tensor-parallel rank's share: max(1, ceil(H_kv / TP)) KV heads of every layer."""
+        heads = max(1, -(-self.kv_heads // tp))
+        return KVShape(self.num_layers, heads, self.head_dim, self.block_size, self.elem_bytes)
+
 
 SHAPES = {
     # 4 layers, 2 KV heads, head_dim 64, block 16: piece 4 KiB, block 32 KiB

@@ -148,7 +148,7 @@ def audit(config, policy, host_gib, kappa=None, chunk_blocks=1, device="cuda:0",
         chunk_off.append(chunk_off[-1] + len(k))
     cstream = np.concatenate(chunk_keys) if chunk_keys else np.zeros(0, np.uint64)
     kh = max(1, int(host_gib * GIB // (R * shape.block_bytes)))
-    kap = cfg.kappa_blocks if kappa is None else kappa
+    kap = max(1, cfg.kappa_blocks // R) if kappa is None else kappa     # the config's threshold, in tier units
     ctx = eakv.Context(num_layers=1, kv_heads=1, head_dim=8, block_size=b, gpu_blocks=1, host_blocks=kh,
                        kv_base=None, control_plane_only=True, policy=POLICIES[policy],
                        kappa_blocks=kap, chunk_blocks=R)

@@ -141,7 +141,7 @@ def run(config, *, policy="write_all", host_gib=None, active_pool=None, model=Se
     payload = (lambda keys, q, n: key_words_torch(keys.astype(np.int64), q, n, device)) if data_plane else None
     server = AgentServer(shape, cfg.gpu_blocks, kh, payload, device=device, data_plane=data_plane,
                          incremental_hash=True, policy=POLICIES[policy],
-                         kappa_blocks=cfg.kappa_blocks if kappa is None else kappa,
+                         kappa_blocks=max(1, cfg.kappa_blocks // chunk_blocks) if kappa is None else kappa,
                          theta_percent=theta, chunk_blocks=chunk_blocks, gpu_free_order=gpu_free_order)
     seen = {"load": 0, "store": 0}
 

@@ -43,3 +43,26 @@ def aggregate_over_ranks(dist, elapsed_ms: float, units: float, device=None):
 def shard_agents(n_agents: int, rank: int, world: int):
     """Agents served by this rank when a trace is split across replicas (round-robin)."""
     return [a for a in range(n_agents) if a % world == rank]
+
+
+def tp_rank_plan(shape, tp: int, host_bytes_per_rank: int):
+    """Tensor-parallel serving (Eq. 1 and Section 2 of the paper: every rank holds its head shard
+    of each token's KV and its own host tier, so sizes are stated per rank).  Returns the rank's
+    KV shape and K_H = floor(C_H / (b * beta_rank)).  Every rank sees the same keys and the same
+    K_H, hence takes the same decisions; only the bytes per block differ from the unsharded
+    shape.  No exchange step exists between the ranks' tiers."""
+    shard = shape.tp_shard(tp)
+    return shard, int(host_bytes_per_rank) // shard.block_bytes
+
+
+def decisions_digest(records) -> str:
+    """Order-sensitive digest of the per-request decisions (hit / admit / slot / evictions), to
+    compare ranks without shipping the records."""
+    import hashlib
+    h = hashlib.sha256()
+    for r in records:
+        for f in ("hit", "admit", "slot"):
+            h.update(bytes(memoryview(r[f]).cast("B")))
+        for k, s in r["evicted"]:
+            h.update(int(k).to_bytes(8, "little") + int(s).to_bytes(4, "little", signed=True))
+    return h.hexdigest()

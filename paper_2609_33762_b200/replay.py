@@ -74,7 +74,7 @@ def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=Tru
     t0 = time.perf_counter()
     server = AgentServer(shape, cfg.gpu_blocks, kh, payload, device=device, data_plane=data_plane,
                          incremental_hash=incremental_hash, policy=POLICIES[policy],
-                         kappa_blocks=cfg.kappa_blocks if kappa is None else kappa,
+                         kappa_blocks=max(1, cfg.kappa_blocks // chunk_blocks) if kappa is None else kappa,
                          link_strategy=link_strategy, chunk_blocks=chunk_blocks,
                          native_turn=native_turn and data_plane, gpu_free_order=gpu_free_order)
     t_setup = time.perf_counter() - t0

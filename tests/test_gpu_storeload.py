@@ -103,11 +103,12 @@ SHAPE_CASES = {
     "llama": SHAPES["llama3_8b"],                 # piece 64 KiB (4 items per piece)
     "ragged": KVShape(3, 5, 128, 16),             # piece 20 KiB (16 KiB + 4 KiB tail)
     "small": KVShape(2, 3, 40, 2),                # piece 480 B
+    "qwen_tp8": SHAPES["qwen3_30b_a3b"].tp_shard(8),   # one rank of TP8: 96 pieces of 4 KiB per block
 }
 
 
 @pytest.mark.parametrize("kw", variants(), ids=lambda k: "-".join(f"{v}" for v in k.values()))
-@pytest.mark.parametrize("name", ["tiny", "qwen", "ragged", "small"])
+@pytest.mark.parametrize("name", ["tiny", "qwen", "ragged", "small", "qwen_tp8"])
 def test_store_load_parity(name, kw):
     shape = SHAPE_CASES[name]
     nb, kh = (96, 80) if shape.block_bytes <= (1 << 21) else (24, 20)

@@ -55,3 +55,69 @@ def test_single_process_is_identity():
         for k, v in env.items():
             if v is not None:
                 os.environ[k] = v
+
+
+TP_WORKER = textwrap.dedent("""
+    import json, os, sys
+    import numpy as np
+    sys.path.insert(0, %r)
+    from eakv_workloads import CONFIGS, SHAPES, make_trace
+    from oracle import hash as ohash
+    from paper_2609_33762_b200 import eakv
+    from paper_2609_33762_b200.multi import decisions_digest, init_distributed, tp_rank_plan
+    rank, world, local_rank, dist = init_distributed(2, backend="gloo")
+    cfg = CONFIGS["c0"]
+    full = SHAPES[cfg.shape]
+    shard, kh = tp_rank_plan(full, world, 4 << 20)          # 4 MiB of host memory per rank
+    trace = make_trace(cfg)
+    ctx = eakv.Context(num_layers=shard.num_layers, kv_heads=shard.kv_heads, head_dim=shard.head_dim,
+                       block_size=shard.block_size, gpu_blocks=cfg.gpu_blocks, host_blocks=kh,
+                       kv_base=None, control_plane_only=True, policy=eakv.POLICY_FILTER_CONDITIONED)
+    recs, stored_bytes = [], 0
+    for req in trace.requests:
+        toks = trace.prompt(req)
+        keys = np.asarray(ohash.hash_blocks(toks.tolist(), shard.block_size), dtype=np.uint64)
+        st = ctx.eakv_tier_step(keys, req.agent, len(toks), req.time_ms)
+        recs.append(dict(hit=st["hit"], admit=st["admit"], slot=st["slot"],
+                         evicted=list(zip(st["evicted_keys"].tolist(), st["evicted_slots"].tolist()))))
+        stored_bytes += int(st["admit"].sum()) * ctx.block_bytes
+    ctx.close()
+    mine = dict(rank=rank, digest=decisions_digest(recs), kh=kh, stored_bytes=stored_bytes,
+                heads=shard.kv_heads, block_bytes=shard.block_bytes)
+    gathered = [None] * world
+    dist.all_gather_object(gathered, mine)
+    dist.barrier()
+    if rank == 0:
+        print(json.dumps(gathered))
+    dist.destroy_process_group()
+""") % ROOT
+
+
+def test_tensor_parallel_ranks_take_the_same_decisions(tmp_path):
+    """Two TP ranks, each with its head shard and its own tier of the same byte budget: identical
+    K_H and decisions, half the bytes per block of the unsharded shape (Eq. 1)."""
+    import json
+    from eakv_workloads import CONFIGS, SHAPES
+    from oracle import sizing
+    script = tmp_path / "tp_worker.py"
+    script.write_text(TP_WORKER)
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE="2",
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env,
+                                      stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True))
+    outs = [p.communicate(timeout=180) for p in procs]
+    for p, (out, err) in zip(procs, outs):
+        assert p.returncode == 0, err
+    got = json.loads(outs[0][0].strip().splitlines()[-1])
+    full = SHAPES[CONFIGS["c0"].shape]
+    beta = sizing.beta_rank(full.num_layers, full.head_dim, full.elem_bytes, full.kv_heads, tp=2)
+    assert got[0]["digest"] == got[1]["digest"]
+    assert got[0]["stored_bytes"] == got[1]["stored_bytes"] > 0
+    for g in got:
+        assert g["heads"] == 1 and g["block_bytes"] == full.block_size * beta == full.block_bytes // 2
+        assert g["kh"] == sizing.tier_chunks(4 << 20, full.block_size, beta)
