@@ -165,6 +165,34 @@ __device__ __forceinline__ BulkItem bulk_decode(const CopyLaunch& L, int64_t it,
     return b;
 }
 
+// Small pieces (at most half a stage): an item is a group of up to L.group_pieces consecutive
+// pieces of one block.  They are contiguous on the tier side (one bulk copy) and live in
+// separate arrays on the pool side (one bulk copy each), so a stage still carries about
+// 16 KiB and the bytes in flight per SM do not shrink with the piece size.
+struct BulkGroup { char* tier; int64_t pool_off; int q0; int cnt; };
+
+__device__ __forceinline__ BulkGroup bulk_decode_group(const CopyLaunch& L, int64_t it) {
+    const int groups_per_entry = (L.pieces + L.group_pieces - 1) / L.group_pieces;
+    const int64_t j = it / groups_per_entry;
+    const int g = (int)(it - j * groups_per_entry);
+    const int2 e = L.entries ? __ldg(L.entries + j) : L.inline_entries[j];
+    const int64_t slot = L.slot_from_index ? j : (int64_t)e.y;
+    BulkGroup b;
+    b.q0 = g * L.group_pieces;
+    b.cnt = L.pieces - b.q0 < L.group_pieces ? L.pieces - b.q0 : L.group_pieces;
+    if ((uint64_t)e.x >= (uint64_t)L.gpu_blocks || (uint64_t)slot >= (uint64_t)L.tier_slots) {
+        b.tier = nullptr; b.pool_off = 0; b.cnt = 0;        // the caller flags and skips it
+        return b;
+    }
+    b.tier = L.tier_base + (slot * L.slot_pieces + L.slot_q_first + b.q0) * L.piece_bytes;
+    b.pool_off = (int64_t)e.x * L.piece_bytes;
+    return b;
+}
+
+__device__ __forceinline__ char* bulk_pool_piece(const CopyLaunch& L, int q, int64_t pool_off) {
+    return reinterpret_cast<char*>(__ldg(reinterpret_cast<const unsigned long long*>(L.kv_base) + L.q_first + q)) + pool_off;
+}
+
 template <bool TO_TIER>
 __global__ void __launch_bounds__(32)
 copy_blocks_bulk_kernel(CopyLaunch L, int kBulkStages, int kBulkStageBytes) {
@@ -173,7 +201,9 @@ copy_blocks_bulk_kernel(CopyLaunch L, int kBulkStages, int kBulkStageBytes) {
     __shared__ __align__(8) uint64_t bars[kBulkMaxStages];
     if (threadIdx.x != 0) return;
 
-    const int64_t n_items = L.n_entries * L.pieces * L.subs_per_piece;
+    const bool grouped = L.group_pieces > 1;
+    const int64_t n_items = grouped ? L.n_entries * ((L.pieces + L.group_pieces - 1) / L.group_pieces)
+                                    : L.n_entries * L.pieces * L.subs_per_piece;
     const int64_t first = blockIdx.x, stride = gridDim.x;
     if (first >= n_items) return;
     const int64_t n_my = (n_items - first + stride - 1) / stride;
@@ -184,10 +214,33 @@ copy_blocks_bulk_kernel(CopyLaunch L, int kBulkStages, int kBulkStageBytes) {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 
     auto issue_load = [&](int64_t k) {
-        const BulkItem b = bulk_decode<TO_TIER>(L, first + k * stride, kBulkStageBytes);
         const int s = (int)(k % kBulkStages);
         const uint32_t bar = smem_u32(&bars[s]);
         const uint32_t dst = smem_u32(stage_mem + (size_t)s * kBulkStageBytes);
+        if (grouped) {
+            const BulkGroup g = bulk_decode_group(L, first + k * stride);
+            if (g.cnt == 0) {
+                atomicExch(error_flag, kErrCopyRange);
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+                return;
+            }
+            const uint32_t pb = (uint32_t)L.piece_bytes;
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                         :: "r"(bar), "r"(pb * g.cnt) : "memory");
+            if (TO_TIER) {
+                for (int i = 0; i < g.cnt; ++i)
+                    asm volatile(
+                        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                        :: "r"(dst + i * pb), "l"(bulk_pool_piece(L, g.q0 + i, g.pool_off)), "r"(pb), "r"(bar)
+                        : "memory");
+            } else {
+                asm volatile(
+                    "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                    :: "r"(dst), "l"(g.tier), "r"(pb * g.cnt), "r"(bar) : "memory");
+            }
+            return;
+        }
+        const BulkItem b = bulk_decode<TO_TIER>(L, first + k * stride, kBulkStageBytes);
         if (b.bytes == 0) {   // self-check tripped: flag it, complete the phase without a copy
             atomicExch(error_flag, kErrCopyRange);
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
@@ -210,11 +263,26 @@ copy_blocks_bulk_kernel(CopyLaunch L, int kBulkStages, int kBulkStageBytes) {
         const int s = (int)(k % kBulkStages);
         const uint32_t parity = (uint32_t)((k / kBulkStages) & 1);
         if (!mbar_wait_bounded(smem_u32(&bars[s]), parity)) { ok = false; break; }
-        const BulkItem b = bulk_decode<TO_TIER>(L, first + k * stride, kBulkStageBytes);
         const uint32_t src = smem_u32(stage_mem + (size_t)s * kBulkStageBytes);
-        if (b.bytes != 0) {
-            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                         :: "l"(b.dst), "r"(src), "r"(b.bytes) : "memory");
+        if (grouped) {
+            const BulkGroup g = bulk_decode_group(L, first + k * stride);
+            const uint32_t pb = (uint32_t)L.piece_bytes;
+            if (TO_TIER) {
+                if (g.cnt != 0)
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                                 :: "l"(g.tier), "r"(src), "r"(pb * g.cnt) : "memory");
+            } else {
+                for (int i = 0; i < g.cnt; ++i)
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                                 :: "l"(bulk_pool_piece(L, g.q0 + i, g.pool_off)), "r"(src + i * pb), "r"(pb)
+                                 : "memory");
+            }
+        } else {
+            const BulkItem b = bulk_decode<TO_TIER>(L, first + k * stride, kBulkStageBytes);
+            if (b.bytes != 0) {
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                             :: "l"(b.dst), "r"(src), "r"(b.bytes) : "memory");
+            }
         }
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         if (k >= 1 && loads_issued < n_my) {
@@ -264,11 +332,21 @@ cudaError_t launch_copy_bulk(const CopyLaunch& L_in, bool to_tier, int ctas, cud
     }
     CopyLaunch L = L_in;
     L.subs_per_piece = (int32_t)((L.piece_bytes + g_bulk_stage_bytes - 1) / g_bulk_stage_bytes);
+    // pieces of at most half a stage travel in groups that fill the stage (at most 32 per group)
+    L.group_pieces = 1;
+    if (L.piece_bytes * 2 <= g_bulk_stage_bytes) {
+        int64_t g = g_bulk_stage_bytes / L.piece_bytes;
+        if (g > 32) g = 32;
+        if (g > L.pieces) g = L.pieces;
+        L.group_pieces = (int32_t)g;
+    }
     // the auto grid of the vector path assumes its occupancy; rescale to this kernel's
     const int per_sm_vec = copy_vector_ctas_per_sm();
     if (per_sm_vec > 0 && ctas % per_sm_vec == 0 && ctas / per_sm_vec >= 100)
         ctas = ctas / per_sm_vec * g_bulk_ctas_per_sm;
-    const int64_t n_items = L.n_entries * L.pieces * L.subs_per_piece;
+    const int64_t n_items = L.group_pieces > 1
+        ? L.n_entries * ((L.pieces + L.group_pieces - 1) / L.group_pieces)
+        : L.n_entries * L.pieces * L.subs_per_piece;
     if (ctas > n_items) ctas = (int)n_items;
     if (ctas < 1) ctas = 1;
     if (to_tier) copy_blocks_bulk_kernel<true><<<ctas, 32, smem, stream>>>(L, g_bulk_stages, g_bulk_stage_bytes);

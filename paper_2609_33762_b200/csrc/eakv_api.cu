@@ -201,6 +201,8 @@ int launch_copy(eakv_ctx* ctx, const int2* d_entries, const int2* h_inline, int6
     L.tier_slots = packed ? packed_capacity : ctx->tier_slots;
     L.error_flag = ctx->d_error_flag;
     L.subs_per_piece = (int32_t)((ctx->piece_bytes + kCopySubBytes - 1) / kCopySubBytes);
+    L.group_pieces = 1;          // the bulk launcher raises it for small pieces
+    L.pad0 = 0;
     cudaError_t e;
     // bulk async copies serve device-resident buffers; a mapped host tier is always driven
     // by the vector kernel (few CTAs, plain loads/stores over the link)

@@ -105,6 +105,8 @@ struct CopyLaunch {
     int32_t slot_q_first;       // where the range starts inside a slot (q_first, or 0 for packed staging)
     int32_t subs_per_piece;     // ceil(piece_bytes / kCopySubBytes)
     int32_t slot_from_index;    // 1: entry j uses slot j (packed staging buffer) instead of entries[j].y
+    int32_t group_pieces;       // bulk kernel: consecutive pieces of a block per work item (1: piece by piece)
+    int32_t pad0;
     int64_t piece_bytes;
     // self-check limits: an entry outside them raises *error_flag and is skipped
     int64_t gpu_blocks;
