@@ -63,6 +63,9 @@ def parse_args():
     ap.add_argument("--hash-only", action="store_true",
                     help="run only the prefix-hash throughput section and print its JSON")
     ap.add_argument("--hash-prompts", type=int, default=512)
+    ap.add_argument("--tp-shard", type=int, default=1,
+                    help="run the microbench on one tensor-parallel rank's KV shape (heads / TP) instead "
+                         "of the unsharded one; not the headline workload")
     ap.add_argument("--sweep", action="store_true",
                     help="also print the 1..4096-block curve (contiguous/random ids, masks)")
     return ap.parse_args()
@@ -558,6 +561,10 @@ def main():
     device = torch.device(f"cuda:{local_rank}")
     torch.cuda.set_device(device)
     shape = SHAPES["qwen3_30b_a3b"]
+    workload = WORKLOAD
+    if args.tp_shard > 1:
+        shape = shape.tp_shard(args.tp_shard)
+        workload = f"{WORKLOAD}_tp{args.tp_shard}_rank"
     m = args.blocks
 
     # paged pool, as large as fits (200k blocks = 293 GiB do not fit one GPU)
@@ -605,7 +612,8 @@ def main():
     kms = sum(t for _, t in r["kernel"])
     achieved = 2 * kb / (kms * 1e-3) / 1e9 if kms > 0 else 0.0
     kernel_name = "copy_blocks_vector_kernel" if args.copy_path == "vector" else "copy_blocks_bulk_kernel"
-    traffic = read_profile_traffic(kernel_name, m)
+    # the profile's per-block DRAM traffic was captured on the unsharded shape
+    traffic = read_profile_traffic(kernel_name, m) if args.tp_shard == 1 else None
 
     # ---- end-to-end arm (pinned host tier, host tokens) ----
     e2e = None
@@ -649,10 +657,10 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "blocks_per_request": m, "requests_per_step": 2,
+            "config": {"workload": workload, "blocks_per_request": m, "requests_per_step": 2,
                        "pool_blocks": nb, "block_bytes": shape.block_bytes,
                        "block_ids": "uniform-random without replacement", "admit_mask": "from tier step (all admitted)",
-                       "l2": "inputs larger than L2 (12 GiB moved per step)",
+                       "l2": f"inputs larger than L2 ({4 * m * shape.block_bytes / 2**30:.1f} GiB moved per step)",
                        "tokens_hashed_per_step": 2 * m * shape.block_size,
                        "copy_path": args.copy_path, "self_check": check_ok},
             "clocks": r["clocks"],
@@ -750,6 +758,46 @@ def sweep(args, torch, eakv, pool, shape, device):
         ctx.close()
     for row in rows:
         print(json.dumps({"sweep": row}), file=sys.stderr)
+    shape_sweep(torch, eakv, shape, device)
+
+
+def shape_sweep(torch, eakv, shape, device, call_bytes=3 << 29):
+    """Copy rate at tensor-parallel rank shapes (the paper states sizes per TP rank: a rank holds
+    max(1, ceil(H_kv / TP)) heads, so pieces shrink with TP): 1.5 GiB per call between a device
+    pool and a device tier, random block ids, both copy paths."""
+    rng = np.random.default_rng(9)
+    for tp in (1, 2, 8):
+        sh = shape.tp_shard(tp)
+        n = call_bytes // sh.block_bytes
+        words = sh.piece_bytes // 2
+        pieces = [torch.empty((2 * n, words), dtype=torch.int16, device=device) for _ in range(sh.pieces_per_block)]
+        tier = torch.empty(n * sh.block_bytes, dtype=torch.uint8, device=device)
+        for path, pname in ((eakv.COPY_BULK, "bulk"), (eakv.COPY_VECTOR, "vector")):
+            ctx = eakv.Context(num_layers=sh.num_layers, kv_heads=sh.kv_heads, head_dim=sh.head_dim,
+                               block_size=sh.block_size, gpu_blocks=2 * n, host_blocks=n,
+                               kv_base=[t.data_ptr() for t in pieces], tier_location=eakv.TIER_DEVICE,
+                               tier_memory=tier.data_ptr(), copy_path=path, max_call_blocks=n)
+            table = rng.permutation(2 * n)[:n].astype(np.int32)
+            slots = rng.permutation(n).astype(np.int32)
+            stream = torch.cuda.current_stream(device)
+            row = dict(tp=tp, kv_heads=sh.kv_heads, piece_bytes=sh.piece_bytes, blocks=int(n), path=pname)
+            for op in ("store", "load"):
+                ts = []
+                for i in range(8):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    if op == "store":
+                        ctx.eakv_store(table, None, slots, stream)
+                    else:
+                        ctx.eakv_load(slots, table, stream)
+                    e1.record(stream)
+                    torch.cuda.synchronize()
+                    if i >= 3:
+                        ts.append(e0.elapsed_time(e1))
+                row[op + "_gbps_read_plus_write"] = 2 * n * sh.block_bytes / (float(np.median(ts)) * 1e-3) / 1e9
+            ctx.close()
+            print(json.dumps({"shape_sweep": row}), file=sys.stderr)
+        del pieces, tier
 
 
 if __name__ == "__main__":
