@@ -115,9 +115,6 @@ constexpr int kBulkMaxStages = 8;
 // Measured on B200 (6 GiB calls, random block ids): 3 stages x 16 KiB with 2 CTAs per SM
 // (96 KiB in flight per SM, ~14 MB on the chip) streams at the HBM copy peak; deeper rings or
 // more CTAs per SM lose 5-6 %.  The EAKV_TUNE_* environment variables override for sweeps.
-static int g_bulk_stages = 3;
-static int g_bulk_stage_bytes = kCopySubBytes;
-static int g_bulk_ctas_per_sm_cap = 2;
 constexpr uint32_t kBulkSpinLimit = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -303,39 +300,59 @@ copy_blocks_bulk_kernel(CopyLaunch L, int kBulkStages, int kBulkStageBytes) {
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
-static int g_bulk_ctas_per_sm = 0;
+// Ring geometry by piece size.  Measured on B200 at full size (6 GiB calls over a 96 GiB pool,
+// read+write GB/s): pieces of 16 KiB and more want 3 stages x 16 KiB x 2 CTAs per SM (6,616;
+// the small-piece geometry gives 6,379); pieces of 8 KiB and less want more issuing threads
+// and about 128 KiB in flight per SM: 2 stages x 8 KiB x 8 CTAs per SM (8 KiB pieces 6,378
+// against 6,175; 4 KiB pieces 6,213 against 5,730).
+struct BulkGeometry { int stages, stage_bytes, ctas_per_sm_cap, ctas_per_sm; };
+static BulkGeometry g_bulk_geo[2] = {{3, kCopySubBytes, 2, 0}, {2, 8192, 8, 0}};
+static bool g_bulk_ready = false;
+
+static cudaError_t bulk_setup() {
+    for (BulkGeometry& g : g_bulk_geo) {
+        if (const char* e = getenv("EAKV_TUNE_BULK_STAGES")) g.stages = atoi(e);
+        if (const char* e = getenv("EAKV_TUNE_BULK_STAGE_BYTES")) g.stage_bytes = atoi(e);
+        if (const char* e = getenv("EAKV_TUNE_BULK_CTAS_PER_SM")) g.ctas_per_sm_cap = atoi(e);
+        if (g.stages < 2) g.stages = 2;
+        if (g.stages > kBulkMaxStages) g.stages = kBulkMaxStages;
+        if (g.stage_bytes < 1024 || (g.stage_bytes & 15)) g.stage_bytes = kCopySubBytes;
+    }
+    size_t smem_max = 0;
+    for (const BulkGeometry& g : g_bulk_geo)
+        if ((size_t)g.stages * g.stage_bytes > smem_max) smem_max = (size_t)g.stages * g.stage_bytes;
+    cudaError_t e = cudaFuncSetAttribute(copy_blocks_bulk_kernel<true>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(copy_blocks_bulk_kernel<false>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
+    if (e != cudaSuccess) return e;
+    for (BulkGeometry& g : g_bulk_geo) {
+        int fit = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, copy_blocks_bulk_kernel<true>, 32,
+                                                          (size_t)g.stages * g.stage_bytes);
+        if (e != cudaSuccess) return e;
+        if (fit < 1) fit = 1;
+        g.ctas_per_sm = (g.ctas_per_sm_cap >= 1 && g.ctas_per_sm_cap < fit) ? g.ctas_per_sm_cap : fit;
+    }
+    g_bulk_ready = true;
+    return cudaSuccess;
+}
 
 cudaError_t launch_copy_bulk(const CopyLaunch& L_in, bool to_tier, int ctas, cudaStream_t stream) {
     if (L_in.n_entries <= 0) return cudaSuccess;
-    if (g_bulk_ctas_per_sm == 0) {
-        if (const char* e = getenv("EAKV_TUNE_BULK_STAGES")) g_bulk_stages = atoi(e);
-        if (const char* e = getenv("EAKV_TUNE_BULK_STAGE_BYTES")) g_bulk_stage_bytes = atoi(e);
-        if (g_bulk_stages < 2) g_bulk_stages = 2;
-        if (g_bulk_stages > kBulkMaxStages) g_bulk_stages = kBulkMaxStages;
-        if (g_bulk_stage_bytes < 1024 || (g_bulk_stage_bytes & 15)) g_bulk_stage_bytes = kCopySubBytes;
+    if (!g_bulk_ready) {
+        cudaError_t e = bulk_setup();
+        if (e != cudaSuccess) return e;
     }
-    const size_t smem = (size_t)g_bulk_stages * g_bulk_stage_bytes;
-    if (g_bulk_ctas_per_sm == 0) {
-        cudaError_t e = cudaFuncSetAttribute(copy_blocks_bulk_kernel<true>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(copy_blocks_bulk_kernel<false>,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&g_bulk_ctas_per_sm,
-                                                          copy_blocks_bulk_kernel<true>, 32, smem);
-        if (e != cudaSuccess) return e;
-        if (g_bulk_ctas_per_sm < 1) g_bulk_ctas_per_sm = 1;
-        if (const char* e2 = getenv("EAKV_TUNE_BULK_CTAS_PER_SM")) g_bulk_ctas_per_sm_cap = atoi(e2);
-        if (g_bulk_ctas_per_sm_cap >= 1 && g_bulk_ctas_per_sm_cap < g_bulk_ctas_per_sm)
-            g_bulk_ctas_per_sm = g_bulk_ctas_per_sm_cap;
-    }
+    const BulkGeometry& geo = g_bulk_geo[L_in.piece_bytes <= 8192 ? 1 : 0];
+    const size_t smem = (size_t)geo.stages * geo.stage_bytes;
     CopyLaunch L = L_in;
-    L.subs_per_piece = (int32_t)((L.piece_bytes + g_bulk_stage_bytes - 1) / g_bulk_stage_bytes);
+    L.subs_per_piece = (int32_t)((L.piece_bytes + geo.stage_bytes - 1) / geo.stage_bytes);
     // pieces of at most half a stage travel in groups that fill the stage (at most 32 per group)
     L.group_pieces = 1;
-    if (L.piece_bytes * 2 <= g_bulk_stage_bytes) {
-        int64_t g = g_bulk_stage_bytes / L.piece_bytes;
+    if (L.piece_bytes * 2 <= geo.stage_bytes) {
+        int64_t g = geo.stage_bytes / L.piece_bytes;
         if (g > 32) g = 32;
         if (g > L.pieces) g = L.pieces;
         L.group_pieces = (int32_t)g;
@@ -343,14 +360,14 @@ cudaError_t launch_copy_bulk(const CopyLaunch& L_in, bool to_tier, int ctas, cud
     // the auto grid of the vector path assumes its occupancy; rescale to this kernel's
     const int per_sm_vec = copy_vector_ctas_per_sm();
     if (per_sm_vec > 0 && ctas % per_sm_vec == 0 && ctas / per_sm_vec >= 100)
-        ctas = ctas / per_sm_vec * g_bulk_ctas_per_sm;
+        ctas = ctas / per_sm_vec * geo.ctas_per_sm;
     const int64_t n_items = L.group_pieces > 1
         ? L.n_entries * ((L.pieces + L.group_pieces - 1) / L.group_pieces)
         : L.n_entries * L.pieces * L.subs_per_piece;
     if (ctas > n_items) ctas = (int)n_items;
     if (ctas < 1) ctas = 1;
-    if (to_tier) copy_blocks_bulk_kernel<true><<<ctas, 32, smem, stream>>>(L, g_bulk_stages, g_bulk_stage_bytes);
-    else         copy_blocks_bulk_kernel<false><<<ctas, 32, smem, stream>>>(L, g_bulk_stages, g_bulk_stage_bytes);
+    if (to_tier) copy_blocks_bulk_kernel<true><<<ctas, 32, smem, stream>>>(L, geo.stages, geo.stage_bytes);
+    else         copy_blocks_bulk_kernel<false><<<ctas, 32, smem, stream>>>(L, geo.stages, geo.stage_bytes);
     return cudaGetLastError();
 }
 
