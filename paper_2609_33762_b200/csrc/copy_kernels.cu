@@ -112,9 +112,6 @@ cudaError_t launch_copy_vector(const CopyLaunch& L, bool to_tier, int ctas, cuda
 namespace eakv {
 
 constexpr int kBulkMaxStages = 8;
-// Measured on B200 (6 GiB calls, random block ids): 3 stages x 16 KiB with 2 CTAs per SM
-// (96 KiB in flight per SM, ~14 MB on the chip) streams at the HBM copy peak; deeper rings or
-// more CTAs per SM lose 5-6 %.  The EAKV_TUNE_* environment variables override for sweeps.
 constexpr uint32_t kBulkSpinLimit = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -304,7 +301,8 @@ copy_blocks_bulk_kernel(CopyLaunch L, int kBulkStages, int kBulkStageBytes) {
 // read+write GB/s): pieces of 16 KiB and more want 3 stages x 16 KiB x 2 CTAs per SM (6,616;
 // the small-piece geometry gives 6,379); pieces of 8 KiB and less want more issuing threads
 // and about 128 KiB in flight per SM: 2 stages x 8 KiB x 8 CTAs per SM (8 KiB pieces 6,378
-// against 6,175; 4 KiB pieces 6,213 against 5,730).
+// against 6,175; 4 KiB pieces 6,213 against 5,730).  For the large pieces deeper rings or more
+// CTAs per SM lose 5-6 %.  The EAKV_TUNE_BULK_* environment variables override both for sweeps.
 struct BulkGeometry { int stages, stage_bytes, ctas_per_sm_cap, ctas_per_sm; };
 static BulkGeometry g_bulk_geo[2] = {{3, kCopySubBytes, 2, 0}, {2, 8192, 8, 0}};
 static bool g_bulk_ready = false;
