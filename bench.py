@@ -758,7 +758,8 @@ def sweep(args, torch, eakv, pool, shape, device):
         ctx.close()
     for row in rows:
         print(json.dumps({"sweep": row}), file=sys.stderr)
-    shape_sweep(torch, eakv, shape, device)
+    from eakv_workloads import SHAPES
+    shape_sweep(torch, eakv, SHAPES["qwen3_30b_a3b"], device)     # always from the unsharded shape
 
 
 def shape_sweep(torch, eakv, shape, device, call_bytes=3 << 29):
