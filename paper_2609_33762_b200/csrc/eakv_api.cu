@@ -596,7 +596,7 @@ int eakv_hash_blocks(eakv_ctx* ctx, const int32_t* tokens_dev, int64_t n_tokens,
         L.block_size = b;
         L.tile_blocks = tile_blocks;
         L.stages = hash_stages(b);
-        L.pad0 = 0;
+        L.n_prompts = 0;
         L.tokens_limit = n_tokens - done * b;
         L.blocks_limit = cur;
         L.error_flag = ctx->d_error_flag;
@@ -689,13 +689,14 @@ int eakv_hash_blocks_batched(eakv_ctx* ctx, const int32_t* tokens_dev,
     L.block_size = b;
     L.tile_blocks = tile_blocks;
     L.stages = hash_stages(b);
-    L.pad0 = 0;
+    L.n_prompts = (int32_t)n_prompts;
     L.tokens_limit = offsets_host[n_prompts];
     L.blocks_limit = total_blocks;
     L.error_flag = ctx->d_error_flag;
-    cudaError_t e = launch_hash(L, (int)n_tiles, generic, vec, stream);
+    int launched = 0;
+    cudaError_t e = launch_hash(L, (int)n_tiles, generic, vec, stream, &launched);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "hash kernel launch");
-    ctx->stats.kernel_launches += 1;
+    ctx->stats.kernel_launches += launched;
     CU(cudaEventRecord(s->done, stream));
     ctx->stats.tokens_hashed += total_blocks * b;
     return EAKV_OK;

@@ -37,8 +37,8 @@ struct HashLaunch {
     const uint64_t* single_parent_ptr;   // non-NULL: read the parent from device memory instead
     int32_t block_size;
     int32_t tile_blocks;
-    int32_t stages;                 // staged kernel: sub-tiles in flight per warp (2..4)
-    int32_t pad0;
+    int32_t stages;                 // sub-tiles in flight per warp (staged kernel 2..4, run kernel 1..2)
+    int32_t n_prompts;              // batched launches: prompts described at `prompts`; 0 otherwise
     // B^e for e < 64 as three 21-bit limbs each, passed by value: with the block size known at
     // compile time they become constant-bank operands of the multiply-adds (no load at all)
     uint32_t pw_limbs[3 * 64];
@@ -79,13 +79,14 @@ inline void hash_fill_limbs(HashLaunch& L, const uint64_t* pow_host, int block_s
 inline int hash_stages(int block_size) {
     if (const char* e = getenv("EAKV_TUNE_HASH_STAGES")) {      // developer override for sweeps
         const int v = atoi(e);
-        if (v >= 2 && v <= 4 && (size_t)v * kHashThreads * (4 * block_size + 16) <= 136 * 1024) return v;
+        if (v >= 1 && v <= 4 && (size_t)v * kHashThreads * (4 * block_size + 16) <= 136 * 1024) return v;
     }
     return 2;
 }
 cudaError_t hash_kernels_init();
+// *launches_out (optional) receives the number of kernels launched: one, or two for large batches
 cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool thread_per_block, bool vec,
-                        cudaStream_t stream);
+                        cudaStream_t stream, int* launches_out = nullptr);
 
 // ---- gather / scatter ---------------------------------------------------------------------
 constexpr int kCopyThreads = 256;

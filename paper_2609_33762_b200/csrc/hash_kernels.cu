@@ -508,14 +508,285 @@ hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
     if (tid == 0) L.counters[p] = 0;
 }
 #undef EAKV_MAC3
-#undef EAKV_MACP
 
 // thread_per_block: see hash_thread_per_block(); vec: 16-byte token loads are allowed
-cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool thread_per_block, bool vec,
-                        cudaStream_t stream) {
+// ---------------------------------------------------------------------------------------
+// Run variant for b in {16, 32, 64} and 16-byte-aligned tokens.
+//
+// A lane owns RUN = 64 / b consecutive blocks (64 tokens, 256 bytes) of a warp tile, so that
+// the per-block chain h' = h * A + c over those blocks runs inside the lane, interleaved with
+// the next block's multiply-adds, and what the lane publishes per block is already the prefix
+// inside its run.  Every warp stages its own tiles (32 lanes x 256 bytes, coalesced 16-byte
+// async copies at immediate offsets into rows padded by 16 bytes) in a ring of one or two
+// stages and synchronises only with itself; this launch has no fence, ticket or block-wide
+// barrier.  A second launch, one CTA per prompt, then needs one modular product per block: it
+// scans the run totals (constant multiplier A^RUN), leaves every run's incoming hash in shared
+// memory and finishes all blocks with coalesced accesses.  Used for batches of many prompts;
+// single prompts keep the one-launch kernels above (a second launch would cost them latency).
+//
+// Measured on B200, 512 prompts x 65,536 tokens, block 16 (device time of the launches): token
+// launch 32 us, of which the loads alone are 29 us and the arithmetic is hidden; scan launch
+// 20 us; the one-launch staged kernel takes 64 us for the same work.  Variants that were slower:
+// the scan fused behind a ticket (its registers cut the token phase's occupancy: 55-61 us), 512
+// threads per scan CTA (22 us), a third launch that applies the incoming hashes (12 + 11 us).
+// ---------------------------------------------------------------------------------------
+constexpr int kRunThreads = 128;
+constexpr int kRunRowBytes = 256 + 16;
+constexpr int kRunWarpStage = 32 * kRunRowBytes;                      // 8,704 bytes
+constexpr int kRunSmem = 2 * (kRunThreads / 32) * kRunWarpStage;      // 69,632 bytes
+constexpr int kRunChunkRuns = 2048;      // runs scanned per pass: their incoming hashes take 16 KiB
+
+template <int RUN>
+__device__ __forceinline__ uint64_t pick_pow(const uint64_t (&apow)[5], int m) {
+    uint64_t r = apow[RUN];
+#pragma unroll
+    for (int q = 1; q < RUN; ++q)
+        if (m == q) r = apow[q];
+    return r;
+}
+
+template <int RUN, int NTHR>
+__device__ __forceinline__ void scan_runs(const uint64_t* partial, uint64_t* keys, int64_t nblk, uint64_t parent,
+                                       uint64_t A, Pair* warp_tot, uint64_t* h_in, uint64_t* carry_slot) {
+    constexpr int kPer = kRunChunkRuns / NTHR;             // runs per thread and pass
+    const int tid = threadIdx.x, nthr = NTHR;
+    const int lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
+    uint64_t apow[5] = {1, A, 0, 0, 0};
+#pragma unroll
+    for (int q = 2; q <= RUN; ++q) apow[q] = mulmod61(apow[q - 1], A);
+    // M = A^RUN is the multiplier of every full run; M^(2^k) for the per-thread products
+    uint64_t mpow[5];
+    mpow[0] = apow[RUN];
+#pragma unroll
+    for (int k = 1; k < 5; ++k) mpow[k] = mulmod61(mpow[k - 1], mpow[k - 1]);
+    uint64_t carry = parent;
+    for (int64_t base = 0; base < nblk; base += (int64_t)kRunChunkRuns * RUN) {
+        const int64_t cblk = min((int64_t)kRunChunkRuns * RUN, nblk - base);
+        const int n_runs = (int)((cblk + RUN - 1) / RUN);
+        const int m_last = (int)(cblk - (int64_t)(n_runs - 1) * RUN);   // blocks in the pass's last run
+        const int per = (n_runs + nthr - 1) / nthr;                       // <= kPer
+        const int lo = min(tid * per, n_runs), hi = min(lo + per, n_runs);
+        // all of this thread's run totals at once (a run's total sits at its last block)
+        uint64_t tot[kPer];
+#pragma unroll
+        for (int q = 0; q < kPer; ++q) {
+            const int jq = lo + q;
+            tot[q] = jq < hi ? __ldcg(partial + base + min((int64_t)(jq + 1) * RUN, cblk) - 1) : 0;
+        }
+        // the thread's runs as one affine map: c by Horner, a = M^(full runs) * A^(ragged run)
+        const bool has_ragged = (hi == n_runs) && (hi > lo) && (m_last != RUN);
+        const int full = hi - lo - (has_ragged ? 1 : 0);
+        Pair mine{1, 0};
+#pragma unroll
+        for (int k = 0; k < 5; ++k)
+            if (full & (1 << k)) mine.a = mulmod61(mine.a, mpow[k]);
+        if (has_ragged) mine.a = mulmod61(mine.a, pick_pow<RUN>(apow, m_last));
+#pragma unroll
+        for (int q = 0; q < kPer; ++q) {
+            if (lo + q < hi) {
+                const uint64_t mult = (has_ragged && lo + q == hi - 1) ? pick_pow<RUN>(apow, m_last) : mpow[0];
+                mine.c = addmod61(mulmod61(mine.c, mult), tot[q]);
+            }
+        }
+        Pair inc = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            Pair up;
+            up.a = __shfl_up_sync(0xffffffffu, inc.a, d);
+            up.c = __shfl_up_sync(0xffffffffu, inc.c, d);
+            if (lane >= d) inc = compose(up, inc);
+        }
+        if (lane == 31) warp_tot[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            Pair w = lane < nwarp ? warp_tot[lane] : Pair{1, 0};
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                Pair up;
+                up.a = __shfl_up_sync(0xffffffffu, w.a, d);
+                up.c = __shfl_up_sync(0xffffffffu, w.c, d);
+                if (lane >= d) w = compose(up, w);
+            }
+            warp_tot[lane] = w;
+        }
+        __syncthreads();
+        Pair exc;
+        exc.a = __shfl_up_sync(0xffffffffu, inc.a, 1);
+        exc.c = __shfl_up_sync(0xffffffffu, inc.c, 1);
+        if (lane == 0) exc = Pair{1, 0};
+        if (warp > 0) exc = compose(warp_tot[warp - 1], exc);
+        uint64_t h = addmod61(mulmod61(carry, exc.a), exc.c);
+        // incoming hash of each of this thread's runs
+#pragma unroll
+        for (int q = 0; q < kPer; ++q) {
+            if (lo + q < hi) {
+                h_in[lo + q] = h;
+                const uint64_t mult = (has_ragged && lo + q == hi - 1) ? pick_pow<RUN>(apow, m_last) : mpow[0];
+                h = addmod61(mulmod61(h, mult), tot[q]);
+            }
+        }
+        if (lo < hi && hi == n_runs) *carry_slot = h;     // hash at the end of this pass
+        __syncthreads();
+        carry = *carry_slot;
+        // key of block i = (incoming hash of its run) * A^(position in run + 1) + prefix inside the run;
+        // eight independent blocks per thread and step keep the loads in flight together
+        constexpr int kU = NTHR >= 512 ? 4 : 8;
+        for (int64_t i0 = tid; i0 < cblk; i0 += (int64_t)nthr * kU) {
+            uint64_t pv[kU];
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+                const int64_t i = i0 + (int64_t)u * nthr;
+                pv[u] = i < cblk ? __ldcg(partial + base + i) : 0;
+            }
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+                const int64_t i = i0 + (int64_t)u * nthr;
+                if (i < cblk) {
+                    const uint64_t mult = pick_pow<RUN>(apow, (int)(i % RUN) + 1);
+                    keys[base + i] = addmod61(mulmod61(h_in[i / RUN], mult), pv[u]);
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+template <int B>
+__global__ void __launch_bounds__(kRunThreads)
+hash_blocks_run_kernel(const __grid_constant__ HashLaunch L) {
+    constexpr int RUN = 64 / B;
+    constexpr int WT = 32 * RUN;                 // blocks per warp tile
+    constexpr int CPB = B / 4;                   // 16-byte chunks per block
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const HashTile tile = L.tiles[blockIdx.x];
+    const HashPrompt hp = L.prompts[tile.prompt];
+    const int64_t first_blk = tile.first_block;
+    const int64_t tok0 = hp.tok_off, blk0 = hp.blk_off, nblk = hp.nblk;
+    const int nb_tile = (int)min((int64_t)L.tile_blocks, nblk - first_blk);
+    {   // self-check: the tile must lie inside the buffers the caller described
+        const int64_t last_blk = blk0 + first_blk + nb_tile;
+        const int64_t last_tok = tok0 + (first_blk + nb_tile) * (int64_t)B;
+        if (nb_tile <= 0 || last_blk > L.blocks_limit || last_tok > L.tokens_limit || tile.prompt < 0 ||
+            (L.tile_blocks % WT) != 0) {
+            if (threadIdx.x == 0) atomicExch(L.error_flag, kErrHashRange);
+            return;
+        }
+    }
+    const int n_wt = (nb_tile + WT - 1) / WT;
+    const int4* tile_src = reinterpret_cast<const int4*>(L.tokens + tok0 + first_blk * B);
+    const int S = L.stages;                      // 1: no prefetch (more CTAs per SM), 2: two-stage ring
+    unsigned char* const ring = smem_raw + (size_t)warp * S * kRunWarpStage;
+    const int dst_lane = (lane >> 4) * kRunRowBytes + (lane & 15) * 16;
+
+    auto issue = [&](int t, int stage) {
+        const int nb = min(WT, nb_tile - t * WT);
+        const int chunks = nb * CPB;                          // valid 16-byte chunks, 512 when full
+        const int4* src = tile_src + (size_t)t * (WT * CPB) + lane;
+        unsigned char* dst = ring + stage * kRunWarpStage + dst_lane;
+        if (chunks == 512) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) cp_async16(dst + i * 2 * kRunRowBytes, src + 32 * i);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                if (lane + 32 * i < chunks) cp_async16(dst + i * 2 * kRunRowBytes, src + 32 * i);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+
+    const uint64_t A = L.pow_block;
+    uint64_t* partial = L.partial + blk0 + first_blk;
+    if (S == 2) {
+        if (warp < n_wt) issue(warp, 0);
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    int it = 0;
+    for (int t = warp; t < n_wt; t += kRunThreads / 32, ++it) {
+        if (S == 2) {
+            // one group per iteration (empty past the end): "all but the newest" = this tile has landed
+            if (t + kRunThreads / 32 < n_wt) issue(t + kRunThreads / 32, (it + 1) & 1);
+            else asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+        } else {
+            issue(t, 0);
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        }
+        __syncwarp();
+        const unsigned char* row = ring + (S == 2 ? (it & 1) : 0) * kRunWarpStage + lane * kRunRowBytes;
+        const int nb = min(WT, nb_tile - t * WT);
+        uint64_t chain = 0;
+#pragma unroll
+        for (int r = 0; r < RUN; ++r) {
+            if (lane * RUN + r < nb) {
+                const int4* blk = reinterpret_cast<const int4*>(row + r * B * 4);
+                uint64_t s0 = 0, s1 = 0, s2 = 0, t0 = 0, t1 = 0, t2 = 0;
+#pragma unroll
+                for (int k = 0; k < B; k += 4) {
+                    const int4 u = blk[k >> 2];
+                    const int e = B - 1 - k;
+                    EAKV_MACP(u.x, e, s0, s1, s2); EAKV_MACP(u.y, e - 1, t0, t1, t2);
+                    EAKV_MACP(u.z, e - 2, s0, s1, s2); EAKV_MACP(u.w, e - 3, t0, t1, t2);
+                }
+                const uint64_t c = fold_limb_sums(s0 + t0, s1 + t1, s2 + t2);
+                chain = r == 0 ? c : addmod61(mulmod61(chain, A), c);
+                __stcg(partial + (int64_t)t * WT + lane * RUN + r, chain);
+            }
+        }
+        __syncwarp();        // this warp refills the stage two iterations from now
+    }
+}
+
+// Second launch: one CTA per prompt turns the run prefixes into keys.
+template <int RUN>
+__global__ void __launch_bounds__(kRunThreads)
+hash_scan_runs_kernel(const __grid_constant__ HashLaunch L) {
+    __shared__ Pair warp_tot[32];
+    __shared__ uint64_t carry_slot;
+    __shared__ __align__(16) uint64_t h_in[kRunChunkRuns];
+    const HashPrompt hp = L.prompts[blockIdx.x];
+    if (hp.nblk <= 0) return;
+    if (hp.blk_off < 0 || hp.blk_off + hp.nblk > L.blocks_limit) {
+        if (threadIdx.x == 0) atomicExch(L.error_flag, kErrHashRange);
+        return;
+    }
+    scan_runs<RUN, kRunThreads>(L.partial + hp.blk_off, L.keys + hp.blk_off, hp.nblk, hp.parent, L.pow_block,
+                                warp_tot, h_in, &carry_slot);
+}
+
+#undef EAKV_MACP
+
+cudaError_t launch_hash(const HashLaunch& L_in, int n_tiles, bool thread_per_block, bool vec,
+                        cudaStream_t stream, int* launches_out) {
+    if (launches_out) *launches_out = n_tiles > 0 ? 1 : 0;
     if (n_tiles <= 0) return cudaSuccess;
+    HashLaunch L = L_in;
+    const bool run_shape = vec && (L.block_size == 16 || L.block_size == 32 || L.block_size == 64);
+    if (run_shape && L.stages > 2) L.stages = 2;             // the run kernel has one or two stages
     if (thread_per_block) {
         const size_t smem = (size_t)L.block_size * sizeof(uint4);
+        // Many prompts of a block size known at compile time: two launches, the token phase
+        // (a lane per run of consecutive blocks) and the per-prompt scan.  Neither needs a fence
+        // or a ticket, and the scan's registers do not limit the token phase's occupancy.
+        // (EAKV_TUNE_HASH_KERNEL=staged keeps the single-launch kernel, for A/B runs.)
+        static const bool use_run = [] {
+            const char* e = getenv("EAKV_TUNE_HASH_KERNEL");
+            return !(e && e[0] == 's');
+        }();
+        if (run_shape && use_run && L.tiles != nullptr && L.n_prompts > 0 && n_tiles >= 2 * 148) {
+            const size_t rs = L.stages == 2 ? kRunSmem : kRunSmem / 2;
+            if (L.block_size == 16)      hash_blocks_run_kernel<16><<<n_tiles, kRunThreads, rs, stream>>>(L);
+            else if (L.block_size == 32) hash_blocks_run_kernel<32><<<n_tiles, kRunThreads, rs, stream>>>(L);
+            else                         hash_blocks_run_kernel<64><<<n_tiles, kRunThreads, rs, stream>>>(L);
+            cudaError_t e = cudaGetLastError();
+            if (e != cudaSuccess) return e;
+            if (L.block_size == 16)      hash_scan_runs_kernel<4><<<L.n_prompts, kRunThreads, 0, stream>>>(L);
+            else if (L.block_size == 32) hash_scan_runs_kernel<2><<<L.n_prompts, kRunThreads, 0, stream>>>(L);
+            else                         hash_scan_runs_kernel<1><<<L.n_prompts, kRunThreads, 0, stream>>>(L);
+            if (launches_out) *launches_out = 2;
+            return cudaGetLastError();
+        }
+        if (L.stages < 2) L.stages = 2;          // the staged kernel keeps two to four sub-tiles in flight
         const size_t staged = smem + (size_t)L.stages * kHashThreads * (4 * L.block_size + 16);
         if (!vec)                    hash_blocks_tpb_kernel<false><<<n_tiles, kHashThreads, smem, stream>>>(L);
         else if (L.block_size == 16) hash_blocks_staged_kernel<16><<<n_tiles, kHashThreads, staged, stream>>>(L);
@@ -550,6 +821,12 @@ cudaError_t hash_kernels_init() {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(hash_blocks_staged_kernel<64>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, kHashStagedMaxSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(hash_blocks_run_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRunSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(hash_blocks_run_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRunSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(hash_blocks_run_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRunSmem);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(hash_blocks_tpb_kernel<false>,
                                 cudaFuncAttributeMaxDynamicSharedMemorySize, kHashMaxSmem);
@@ -664,7 +941,7 @@ extern "C" int eakv_hash_blocks_static(const int32_t* tokens_dev, int64_t n_toke
     L.block_size = block_size;
     L.tile_blocks = hash_tile_blocks(block_size, nblk);
     L.stages = hash_stages(block_size);
-    L.pad0 = 0;
+    L.n_prompts = 0;
     {   // powers B^0 .. B^b on the host (at most 4,097 modular products) for the by-value limbs
         uint64_t pw_host[65];
         const int lim = block_size < 64 ? block_size : 64;

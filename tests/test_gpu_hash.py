@@ -183,3 +183,37 @@ def test_batched_capacity_errors_and_empty_batches():
     t = np.arange(1600, dtype=np.int32)
     assert gpu_keys(ctx, t) == oh.hash_blocks(t.tolist(), 16)
     ctx.close()
+
+
+@pytest.mark.parametrize("b", [16, 32, 64])
+def test_large_batch_two_launch_path(b):
+    """Batches of many prompts take the two-launch form (token phase, then one scan CTA per prompt):
+    ragged lengths, empty prompts, parents, a prompt longer than one scan pass, three calls in a row."""
+    ctx = hash_ctx(b, hash_scratch_blocks=1 << 18)
+    rng = np.random.default_rng(60 + b)
+    lens = [int(x) for x in rng.integers(0, 9000, size=420)]
+    lens[3], lens[17], lens[100], lens[200] = 0, b - 1, 70000, 64 * 2048 + 5 * b + 3   # > 2,048 runs of 64 tokens
+    lens = [x - x % 4 for x in lens]                       # every prompt starts 16-byte aligned
+    offsets = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    toks = rng.integers(0, 151936, size=int(offsets[-1]), dtype=np.int32)
+    parents = [int(x) for x in rng.integers(0, P, size=len(lens), dtype=np.uint64)]
+    dev = torch.from_numpy(toks).cuda()
+    total = sum(x // b for x in lens)
+    expect = {}
+    for par in (None, parents):
+        for i, n in enumerate(lens):
+            p0 = oh.HASH_SEED if par is None else par[i]
+            expect[(par is None, i)] = oh.hash_blocks(toks[offsets[i]:offsets[i + 1]].tolist(), b, p0)
+    for rep in range(3):
+        par = None if rep != 1 else parents
+        out = torch.full((total + 1,), -1, dtype=torch.int64, device="cuda")
+        before = ctx.eakv_get_stats()["kernel_launches"]
+        boff = ctx.eakv_hash_blocks_batched(dev.data_ptr(), offsets, par, out.data_ptr())
+        ctx.eakv_sync()
+        assert ctx.eakv_get_stats()["kernel_launches"] - before == 3      # arguments, token phase, scan
+        res = out.cpu().numpy()
+        assert res[total] == -1
+        for i in range(len(lens)):
+            got = [int(x) for x in res[boff[i]:boff[i + 1]].view(np.uint64)]
+            assert got == expect[(par is None, i)], (b, rep, i, lens[i])
+    ctx.close()
