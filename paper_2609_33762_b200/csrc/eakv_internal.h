@@ -43,6 +43,7 @@ struct HashLaunch {
     // compile time they become constant-bank operands of the multiply-adds (no load at all)
     uint32_t pw_limbs[3 * 64];
     uint64_t pow_block;             // A = B^b, the per-block multiplier of the scan
+    uint64_t apow[5];               // A^0 .. A^4 (the scan launch of the two-launch form)
     // self-check limits: a CTA whose tile would reach past them raises *error_flag and skips
     int64_t tokens_limit;           // tokens readable at `tokens`
     int64_t blocks_limit;           // entries writable at `keys` and `partial`
@@ -73,6 +74,10 @@ inline void hash_fill_limbs(HashLaunch& L, const uint64_t* pow_host, int block_s
         L.pw_limbs[3 * e + 2] = (uint32_t)(w >> 42);
     }
     L.pow_block = pow_host[block_size];
+    constexpr uint64_t kP61 = (1ull << 61) - 1;
+    L.apow[0] = 1;
+    for (int q = 1; q < 5; ++q)
+        L.apow[q] = (uint64_t)(((unsigned __int128)L.apow[q - 1] * L.pow_block) % kP61);
 }
 // Sub-tiles in flight per warp in the staged kernel.  Two is the measured optimum: three and
 // four (more shared memory, fewer CTAs per SM) were 3-10 % slower.

@@ -545,106 +545,116 @@ __device__ __forceinline__ uint64_t pick_pow(const uint64_t (&apow)[5], int m) {
     return r;
 }
 
+// Shared state of one scan pass.  All full runs have the multiplier M = A^RUN and every thread but
+// the last non-empty one holds exactly `per` of them, so the scan over threads needs one modular
+// product per step against multipliers that are the same for the whole CTA.
+struct ScanShared {
+    uint64_t step_pow[5];      // (M^per)^(2^k)
+    uint64_t lane_pow[32];     // (M^per)^lane
+    uint64_t warp_mult;        // (M^per)^32
+    uint64_t warp_tot[32];     // inclusive total of each warp
+    uint64_t warp_in[32];      // hash entering each warp
+    uint64_t carry;            // hash entering the next pass
+};
+
 template <int RUN, int NTHR>
 __device__ __forceinline__ void scan_runs(const uint64_t* partial, uint64_t* keys, int64_t nblk, uint64_t parent,
-                                       uint64_t A, Pair* warp_tot, uint64_t* h_in, uint64_t* carry_slot) {
+                                          const uint64_t (&apow)[5], uint64_t* h_in, ScanShared* sh) {
     constexpr int kPer = kRunChunkRuns / NTHR;             // runs per thread and pass
-    const int tid = threadIdx.x, nthr = NTHR;
-    const int lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
-    uint64_t apow[5] = {1, A, 0, 0, 0};
-#pragma unroll
-    for (int q = 2; q <= RUN; ++q) apow[q] = mulmod61(apow[q - 1], A);
-    // M = A^RUN is the multiplier of every full run; M^(2^k) for the per-thread products
-    uint64_t mpow[5];
-    mpow[0] = apow[RUN];
-#pragma unroll
-    for (int k = 1; k < 5; ++k) mpow[k] = mulmod61(mpow[k - 1], mpow[k - 1]);
+    const int tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5;
+    constexpr int nwarp = NTHR / 32;
+    const uint64_t M = apow[RUN];
+    // every block a thread finishes has the same position in its run (NTHR is a multiple of RUN)
+    const uint64_t my_mult = pick_pow<RUN>(apow, tid % RUN + 1);
     uint64_t carry = parent;
     for (int64_t base = 0; base < nblk; base += (int64_t)kRunChunkRuns * RUN) {
-        const int64_t cblk = min((int64_t)kRunChunkRuns * RUN, nblk - base);
-        const int n_runs = (int)((cblk + RUN - 1) / RUN);
-        const int m_last = (int)(cblk - (int64_t)(n_runs - 1) * RUN);   // blocks in the pass's last run
-        const int per = (n_runs + nthr - 1) / nthr;                       // <= kPer
+        const int cblk = (int)min((int64_t)kRunChunkRuns * RUN, nblk - base);
+        const int n_runs = (cblk + RUN - 1) / RUN;
+        const int m_last = cblk - (n_runs - 1) * RUN;                    // blocks in the pass's last run
+        const int per = (n_runs + NTHR - 1) / NTHR;                      // <= kPer
         const int lo = min(tid * per, n_runs), hi = min(lo + per, n_runs);
-        // all of this thread's run totals at once (a run's total sits at its last block)
+        if (warp == 0) {          // this pass's uniform multipliers
+            uint64_t mper = 1, sq = M;
+            for (int n = per; n; n >>= 1) {
+                if (n & 1) mper = mulmod61(mper, sq);
+                sq = mulmod61(sq, sq);
+            }
+            uint64_t sp = mper, lp = 1;
+#pragma unroll
+            for (int k = 0; k < 5; ++k) {
+                if (lane == 0) sh->step_pow[k] = sp;
+                if ((lane >> k) & 1) lp = mulmod61(lp, sp);
+                sp = mulmod61(sp, sp);
+            }
+            sh->lane_pow[lane] = lp;
+            if (lane == 0) sh->warp_mult = sp;
+        }
+        // all of this thread's run totals at once (a run's total sits at its last block), then Horner
         uint64_t tot[kPer];
 #pragma unroll
         for (int q = 0; q < kPer; ++q) {
             const int jq = lo + q;
-            tot[q] = jq < hi ? __ldcg(partial + base + min((int64_t)(jq + 1) * RUN, cblk) - 1) : 0;
+            tot[q] = jq < hi ? __ldcg(partial + base + min((jq + 1) * RUN, cblk) - 1) : 0;
         }
-        // the thread's runs as one affine map: c by Horner, a = M^(full runs) * A^(ragged run)
         const bool has_ragged = (hi == n_runs) && (hi > lo) && (m_last != RUN);
-        const int full = hi - lo - (has_ragged ? 1 : 0);
-        Pair mine{1, 0};
-#pragma unroll
-        for (int k = 0; k < 5; ++k)
-            if (full & (1 << k)) mine.a = mulmod61(mine.a, mpow[k]);
-        if (has_ragged) mine.a = mulmod61(mine.a, pick_pow<RUN>(apow, m_last));
+        const uint64_t ragged_mult = pick_pow<RUN>(apow, m_last);
+        uint64_t c = 0;
 #pragma unroll
         for (int q = 0; q < kPer; ++q) {
             if (lo + q < hi) {
-                const uint64_t mult = (has_ragged && lo + q == hi - 1) ? pick_pow<RUN>(apow, m_last) : mpow[0];
-                mine.c = addmod61(mulmod61(mine.c, mult), tot[q]);
+                const uint64_t mult = (has_ragged && lo + q == hi - 1) ? ragged_mult : M;
+                c = addmod61(mulmod61(c, mult), tot[q]);
             }
         }
-        Pair inc = mine;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            Pair up;
-            up.a = __shfl_up_sync(0xffffffffu, inc.a, d);
-            up.c = __shfl_up_sync(0xffffffffu, inc.c, d);
-            if (lane >= d) inc = compose(up, inc);
-        }
-        if (lane == 31) warp_tot[warp] = inc;
         __syncthreads();
-        if (warp == 0) {
-            Pair w = lane < nwarp ? warp_tot[lane] : Pair{1, 0};
+        uint64_t inc = c;
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                Pair up;
-                up.a = __shfl_up_sync(0xffffffffu, w.a, d);
-                up.c = __shfl_up_sync(0xffffffffu, w.c, d);
-                if (lane >= d) w = compose(up, w);
+        for (int k = 0; k < 5; ++k) {
+            const uint64_t up = __shfl_up_sync(0xffffffffu, inc, 1 << k);
+            if (lane >= (1 << k)) inc = addmod61(mulmod61(up, sh->step_pow[k]), inc);
+        }
+        uint64_t exc = __shfl_up_sync(0xffffffffu, inc, 1);
+        if (lane == 0) exc = 0;
+        if (lane == 31) sh->warp_tot[warp] = inc;
+        __syncthreads();
+        if (tid == 0) {
+            uint64_t h = carry;
+            for (int w = 0; w < nwarp; ++w) {
+                sh->warp_in[w] = h;
+                h = addmod61(mulmod61(h, sh->warp_mult), sh->warp_tot[w]);
             }
-            warp_tot[lane] = w;
         }
         __syncthreads();
-        Pair exc;
-        exc.a = __shfl_up_sync(0xffffffffu, inc.a, 1);
-        exc.c = __shfl_up_sync(0xffffffffu, inc.c, 1);
-        if (lane == 0) exc = Pair{1, 0};
-        if (warp > 0) exc = compose(warp_tot[warp - 1], exc);
-        uint64_t h = addmod61(mulmod61(carry, exc.a), exc.c);
+        uint64_t h = addmod61(mulmod61(sh->warp_in[warp], sh->lane_pow[lane]), exc);
         // incoming hash of each of this thread's runs
 #pragma unroll
         for (int q = 0; q < kPer; ++q) {
             if (lo + q < hi) {
                 h_in[lo + q] = h;
-                const uint64_t mult = (has_ragged && lo + q == hi - 1) ? pick_pow<RUN>(apow, m_last) : mpow[0];
+                const uint64_t mult = (has_ragged && lo + q == hi - 1) ? ragged_mult : M;
                 h = addmod61(mulmod61(h, mult), tot[q]);
             }
         }
-        if (lo < hi && hi == n_runs) *carry_slot = h;     // hash at the end of this pass
+        if (lo < hi && hi == n_runs) sh->carry = h;       // hash at the end of this pass
         __syncthreads();
-        carry = *carry_slot;
+        carry = sh->carry;
         // key of block i = (incoming hash of its run) * A^(position in run + 1) + prefix inside the run;
         // eight independent blocks per thread and step keep the loads in flight together
-        constexpr int kU = NTHR >= 512 ? 4 : 8;
-        for (int64_t i0 = tid; i0 < cblk; i0 += (int64_t)nthr * kU) {
+        constexpr int kU = 8;
+        const uint64_t* pin = partial + base;
+        uint64_t* kout = keys + base;
+        for (int i0 = tid; i0 < cblk; i0 += NTHR * kU) {
             uint64_t pv[kU];
 #pragma unroll
             for (int u = 0; u < kU; ++u) {
-                const int64_t i = i0 + (int64_t)u * nthr;
-                pv[u] = i < cblk ? __ldcg(partial + base + i) : 0;
+                const int i = i0 + u * NTHR;
+                pv[u] = i < cblk ? __ldcg(pin + i) : 0;
             }
 #pragma unroll
             for (int u = 0; u < kU; ++u) {
-                const int64_t i = i0 + (int64_t)u * nthr;
-                if (i < cblk) {
-                    const uint64_t mult = pick_pow<RUN>(apow, (int)(i % RUN) + 1);
-                    keys[base + i] = addmod61(mulmod61(h_in[i / RUN], mult), pv[u]);
-                }
+                const int i = i0 + u * NTHR;
+                if (i < cblk) kout[i] = addmod61(mulmod61(h_in[i / RUN], my_mult), pv[u]);
             }
         }
         __syncthreads();
@@ -741,8 +751,7 @@ hash_blocks_run_kernel(const __grid_constant__ HashLaunch L) {
 template <int RUN>
 __global__ void __launch_bounds__(kRunThreads)
 hash_scan_runs_kernel(const __grid_constant__ HashLaunch L) {
-    __shared__ Pair warp_tot[32];
-    __shared__ uint64_t carry_slot;
+    __shared__ ScanShared sh;
     __shared__ __align__(16) uint64_t h_in[kRunChunkRuns];
     const HashPrompt hp = L.prompts[blockIdx.x];
     if (hp.nblk <= 0) return;
@@ -750,8 +759,7 @@ hash_scan_runs_kernel(const __grid_constant__ HashLaunch L) {
         if (threadIdx.x == 0) atomicExch(L.error_flag, kErrHashRange);
         return;
     }
-    scan_runs<RUN, kRunThreads>(L.partial + hp.blk_off, L.keys + hp.blk_off, hp.nblk, hp.parent, L.pow_block,
-                                warp_tot, h_in, &carry_slot);
+    scan_runs<RUN, kRunThreads>(L.partial + hp.blk_off, L.keys + hp.blk_off, hp.nblk, hp.parent, L.apow, h_in, &sh);
 }
 
 #undef EAKV_MACP
