@@ -211,6 +211,22 @@ int eakv_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
                    uint64_t* evicted_keys_out, int32_t* evicted_slots_out,
                    int64_t* n_evicted_inout, eakv_step_info* info_out);
 
+/* Tier index export / import: carry a host tier across a restart of the process that owns the
+ * context (no counterpart in the paper, whose replays start from a cold cache; Section 5.1).
+ * eakv_tier_export writes the keys and slots of the resident units in recency order, least
+ * recent first, into host arrays of `capacity` entries (either may be NULL) and the number of
+ * residents into *n_out; E_CAPACITY if capacity is too small (nothing but *n_out is written).
+ * eakv_tier_import fills the EMPTY host tier of a fresh context with such a list; together with
+ * eakv_config.tier_memory pointing at the memory the old context used, the new context then
+ * serves the same restores.  Slots handed out afterwards are the unused ones in ascending order,
+ * as in a run that never evicted.  Not carried over: the GPU tier (the engine's blocks are gone
+ * with the process), the admission windows (activity, prompt lengths, evictions restart empty,
+ * so capacity-conditioned admission may decide differently until they refill) and the counters.
+ * E_INVAL: tier not empty, a repeated key or slot, a slot outside the tier; nothing changes. */
+int eakv_tier_export(const eakv_ctx* ctx, uint64_t* keys_host_out, int32_t* slots_host_out,
+                     int64_t capacity, int64_t* n_out);
+int eakv_tier_import(eakv_ctx* ctx, const uint64_t* keys_host, const int32_t* slots_host, int64_t n);
+
 /* The GPU tier's bookkeeping, which the paper leaves to the serving engine (Section 2):
  * an LRU of gpu_index_blocks keyed blocks referenced in order; a non-resident key takes
  * a block from a free stack (0, 1, 2, ... first; an evicted block is reused next).  With

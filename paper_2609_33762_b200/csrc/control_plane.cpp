@@ -128,6 +128,46 @@ void KeyedLru::release_unkeyed(int32_t s) {
     free_.push_back(s);
 }
 
+int64_t KeyedLru::export_order(uint64_t* keys, int32_t* slots, int64_t capacity) const {
+    int64_t n = 0;
+    for (int32_t s = lru_; s >= 0; s = next_[s], ++n) {
+        if (n < capacity) {
+            if (keys) keys[n] = key_[s];
+            if (slots) slots[n] = s;
+        }
+    }
+    return n;
+}
+
+bool KeyedLru::import_order(const uint64_t* keys, const int32_t* slots, int64_t n) {
+    if (resident_ != 0 || (int64_t)free_.size() != cap_ || n < 0 || n > cap_) return false;
+    int64_t done = 0;
+    bool ok = true;
+    for (; done < n; ++done) {
+        const int32_t s = slots[done];
+        if (s < 0 || s >= cap_ || state_[s] != 0 || find(keys[done]) >= 0) { ok = false; break; }
+        key_[s] = keys[done];
+        state_[s] = 1;
+        table_put(keys[done], s);
+        push_mru(s);
+        ++resident_;
+    }
+    if (!ok) {                     // undo: back to the empty tier
+        for (int64_t i = 0; i < done; ++i) {
+            const int32_t s = slots[i];
+            table_erase(key_[s]);
+            unlink(s);
+            state_[s] = 0;
+        }
+        resident_ = 0;
+        return false;
+    }
+    free_.clear();
+    for (int64_t s = cap_ - 1; s >= 0; --s)
+        if (state_[s] == 0) free_.push_back((int32_t)s);
+    return true;
+}
+
 Admission::Admission(int32_t policy, int32_t kappa_blocks, int32_t theta_percent,
                      int64_t window_ms, int32_t len_window, int32_t telemetry,
                      int64_t host_blocks, int32_t block_size)

@@ -33,6 +33,14 @@ public:
     // give an unkeyed slot back to the free stack
     void release_unkeyed(int32_t slot);
     bool is_unkeyed_taken(int32_t slot) const { return state_[slot] == 2; }
+    // Residents in recency order, least recent first, into keys[]/slots[] (either may be NULL);
+    // returns how many there are (at most `capacity` are written).
+    int64_t export_order(uint64_t* keys, int32_t* slots, int64_t capacity) const;
+    // Fill an EMPTY tier: entry i becomes resident at slots[i], later entries more recent.  The
+    // free stack afterwards yields the unused slots in ascending order, exactly as if the entries
+    // had been inserted by a run that never evicted.  False (and nothing changes) when the tier
+    // is not empty or the input repeats a key or slot or leaves the range.
+    bool import_order(const uint64_t* keys, const int32_t* slots, int64_t n);
 
 private:
     void table_put(uint64_t key, int32_t slot);

@@ -786,6 +786,22 @@ int eakv_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
     return EAKV_OK;
 }
 
+int eakv_tier_export(const eakv_ctx* ctx, uint64_t* keys_host_out, int32_t* slots_host_out,
+                     int64_t capacity, int64_t* n_out) {
+    if (!ctx || !n_out || capacity < 0) return EAKV_E_INVAL;
+    *n_out = ctx->host_tier->resident();
+    if ((keys_host_out || slots_host_out) && capacity < *n_out) return EAKV_E_CAPACITY;
+    ctx->host_tier->export_order(keys_host_out, slots_host_out, capacity);
+    return EAKV_OK;
+}
+
+int eakv_tier_import(eakv_ctx* ctx, const uint64_t* keys_host, const int32_t* slots_host, int64_t n) {
+    if (!ctx || n < 0 || (n > 0 && (!keys_host || !slots_host))) return EAKV_E_INVAL;
+    if (!ctx->host_tier->import_order(keys_host, slots_host, n)) return EAKV_E_INVAL;
+    ctx->stats.resident = ctx->host_tier->resident();
+    return EAKV_OK;
+}
+
 int eakv_gpu_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
                        int32_t need_tail, uint8_t* resident_out, int32_t* block_out,
                        int32_t* tail_block_out) {

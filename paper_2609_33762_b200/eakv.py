@@ -89,7 +89,7 @@ EXPORTS = [
     "eakv_gpu_tier_release", "eakv_store", "eakv_load", "eakv_sync", "eakv_get_stats",
     "eakv_tier_ptr", "eakv_hash_seed", "eakv_hash_base", "eakv_strerror", "eakv_last_cuda_error",
     "eakv_hash_blocks_static", "eakv_load_layers", "eakv_reuse_distances", "eakv_capacity_curve",
-    "eakv_turn_begin", "eakv_turn_end",
+    "eakv_turn_begin", "eakv_turn_end", "eakv_tier_export", "eakv_tier_import",
 ]
 STATIC_MAX_BLOCKS = 65536
 
@@ -123,6 +123,8 @@ def lib():
     L.eakv_capacity_curve.argtypes = [vp, i64, vp, vp, vp, i64, i32, vp, i32, vp, vp, vp, vp, vp]
     L.eakv_turn_begin.argtypes = [vp, vp, i64, vp, i64, i64, i64, vp, C.POINTER(TurnView)]
     L.eakv_turn_end.argtypes = [vp, vp]
+    L.eakv_tier_export.argtypes = [vp, vp, vp, i64, C.POINTER(i64)]
+    L.eakv_tier_import.argtypes = [vp, vp, vp, i64]
     L.eakv_sync.argtypes = [vp]
     L.eakv_get_stats.argtypes = [vp, C.POINTER(Stats)]
     L.eakv_tier_ptr.argtypes = [vp]
@@ -298,6 +300,24 @@ class Context:
                               gids.ctypes.data_as(C.c_void_p), slots.ctypes.data_as(C.c_void_p))
         self._check(rc, "eakv_match")
         return G.value, H.value, gids[:G.value], slots[:H.value]
+
+    def eakv_tier_export(self):
+        """(keys, slots) of the host tier's residents, least recent first."""
+        n = C.c_int64(0)
+        self._check(lib().eakv_tier_export(self._h, None, None, 0, C.byref(n)), "eakv_tier_export")
+        keys = np.zeros(n.value, dtype=np.uint64)
+        slots = np.zeros(n.value, dtype=np.int32)
+        rc = lib().eakv_tier_export(self._h, keys.ctypes.data_as(C.c_void_p), slots.ctypes.data_as(C.c_void_p),
+                                    n.value, C.byref(n))
+        self._check(rc, "eakv_tier_export")
+        return keys, slots
+
+    def eakv_tier_import(self, keys, slots):
+        k, kp = _np(keys, np.uint64)
+        s_, sp = _np(slots, np.int32)
+        if len(k) != len(s_):
+            raise ValueError("keys and slots differ in length")
+        self._check(lib().eakv_tier_import(self._h, kp, sp, len(k)), "eakv_tier_import")
 
     def eakv_tier_step(self, hashes, agent_id, n_tokens, now_ms):
         h, hp = _np(hashes, np.uint64)

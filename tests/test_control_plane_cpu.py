@@ -301,3 +301,59 @@ def test_reverse_free_order_whole_trace(eakv):
 def test_free_order_argument_is_checked(eakv):
     with pytest.raises(eakv.EakvError):
         cp_ctx(eakv, 4, 8, 8, gpu_free_order=2)
+
+
+@pytest.mark.parametrize("policy", [0, 1])
+def test_tier_export_import_restart(eakv, policy):
+    """Stop after half of the trace, export the host tier's index, import it into a fresh context
+    and go on: every later decision equals the uninterrupted oracle run whose GPU tier was emptied
+    at the same point (write-all and fixed admission keep no window state)."""
+    cfg = CONFIGS["c0_big_tier"]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg, agents=5)
+    kw = dict(policy=policy, kappa_blocks=40)          # first prompts (32 blocks) pass the filter
+    half = len(trace.requests) // 2
+    orc = TraceOracle(shape, cfg.gpu_blocks, 300, **kw)
+    for i, req in enumerate(trace.requests):
+        if i == half:
+            orc.gpu = GpuTier(cfg.gpu_blocks)                # the engine's blocks do not survive
+        orc.turn(trace.prompt(req), req.agent, req.time_ms)
+    first, second = replace_requests(trace, 0, half), replace_requests(trace, half, None)
+    ctx = cp_ctx(eakv, shape.block_size, cfg.gpu_blocks, 300, **kw)
+    recs = drive(ctx, first, shape.block_size)
+    keys, slots = ctx.eakv_tier_export()
+    assert list(zip(keys.tolist(), slots.tolist())) == list(orc_order_at(trace, shape, cfg, half, kw))
+    ctx.close()
+    ctx = cp_ctx(eakv, shape.block_size, cfg.gpu_blocks, 300, **kw)
+    ctx.eakv_tier_import(keys, slots)
+    assert ctx.eakv_get_stats()["resident"] == len(keys)
+    recs += drive(ctx, second, shape.block_size)
+    compare(recs, orc.records)
+    # import is refused into a tier that is not empty, and for repeated slots or keys
+    with pytest.raises(eakv.EakvError):
+        ctx.eakv_tier_import(keys[:1], slots[:1])
+    ctx.close()
+    ctx = cp_ctx(eakv, shape.block_size, cfg.gpu_blocks, 300, **kw)
+    for bad_k, bad_s in (([1, 2], [0, 0]), ([1, 1], [0, 1]), ([1], [300]), ([1], [-1])):
+        with pytest.raises(eakv.EakvError):
+            ctx.eakv_tier_import(np.array(bad_k, np.uint64), np.array(bad_s, np.int32))
+        assert ctx.eakv_get_stats()["resident"] == 0 and len(ctx.eakv_tier_export()[0]) == 0
+    ctx.eakv_tier_import(np.array([7, 9], np.uint64), np.array([5, 0], np.int32))
+    st = ctx.eakv_tier_step(as_keys([11, 12, 13]), 0, 12, 0)          # unused slots, ascending
+    assert st["slot"].tolist() == [1, 2, 3]
+    ctx.close()
+
+
+def replace_requests(trace, lo, hi):
+    from copy import copy
+    t = copy(trace)
+    t.requests = trace.requests[lo:hi]
+    return t
+
+
+def orc_order_at(trace, shape, cfg, n, kw):
+    """Host tier order (key, slot), least recent first, after the first n requests."""
+    o = TraceOracle(shape, cfg.gpu_blocks, 300, **kw)
+    for req in trace.requests[:n]:
+        o.turn(trace.prompt(req), req.agent, req.time_ms)
+    return o.host.order.items()

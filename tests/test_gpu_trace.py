@@ -250,3 +250,41 @@ def test_closed_loop_replay_bit_exact(policy, kh, pool, native):
     assert server.totals == oracle.totals
     compare_bytes(server, oracle)
     server.close()
+
+
+def test_warm_restart_with_adopted_tier_memory():
+    """Half of the trace, then the process 'restarts': the host tier's index is exported, the
+    context destroyed, a new one adopts the same pinned tier memory and imports the index.  The
+    rest of the trace restores the old bytes: records and resident bytes equal the oracle run
+    whose GPU tier was emptied at the same point."""
+    from oracle.trace import GpuTier
+    from paper_2609_33762_b200.harness import AgentServer
+    cfg = CONFIGS["c0_big_tier"]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg, agents=5)
+    kh = cfg.host_blocks                                  # large enough that prefixes survive
+    half = len(trace.requests) // 2
+    oracle = TraceOracle(shape, cfg.gpu_blocks, kh, payload=key_words_numpy)
+    for i, req in enumerate(trace.requests):
+        if i == half:
+            oracle.gpu = GpuTier(cfg.gpu_blocks)
+        oracle.turn(trace.prompt(req), req.agent, req.time_ms)
+    tier_mem = torch.zeros(kh * shape.block_bytes, dtype=torch.uint8).pin_memory()
+    server = AgentServer(shape, cfg.gpu_blocks, kh, key_words_numpy, tier_memory=tier_mem.data_ptr())
+    for req in trace.requests[:half]:
+        server.turn(trace.prompt(req), req.agent, req.time_ms)
+    server.ctx.eakv_sync()
+    recs = list(server.records)
+    keys, slots = server.ctx.eakv_tier_export()
+    assert len(keys) > 0
+    server.close()
+    del server
+    server = AgentServer(shape, cfg.gpu_blocks, kh, key_words_numpy, tier_memory=tier_mem.data_ptr())
+    server.ctx.eakv_tier_import(keys, slots)
+    for req in trace.requests[half:]:
+        server.turn(trace.prompt(req), req.agent, req.time_ms)
+    recs += server.records
+    compare_records(recs, oracle.records)
+    assert sum(r["loaded"] for r in server.records) > 0          # restores came from the old bytes
+    compare_bytes(server, oracle)
+    server.close()
