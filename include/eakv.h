@@ -168,7 +168,8 @@ int eakv_hash_blocks(eakv_ctx* ctx, const int32_t* tokens_dev, int64_t n_tokens,
                      uint64_t parent_hash, uint64_t* hashes_dev, int64_t* n_blocks_out,
                      void* cuda_stream);
 
-/* The same for many prompts in one launch.  Prompt i is tokens_dev[offsets[i] ..
+/* The same for many prompts in one call (one kernel launch; large batches with block size 16,
+ * 32 or 64 take two: the token phase, then one scan CTA per prompt).  Prompt i is tokens_dev[offsets[i] ..
  * offsets[i+1]) and starts from parents[i] (NULL: the seed for all).  Keys are packed:
  * prompt i's keys start at block_offsets_out[i] = sum_{k<i} len_k / block_size.
  *   offsets_host       host, int64[n_prompts + 1], non-decreasing
