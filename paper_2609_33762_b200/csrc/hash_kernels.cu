@@ -34,6 +34,19 @@ __device__ __forceinline__ uint64_t mulmod61(uint64_t a, uint64_t b) {   // a, b
     return reduce_once((lo & P61) + ((hi << 3) | (lo >> 61)));
 }
 
+// (x * m + add) mod p for a multiplier split once into m0 = low 32 bits, m1 = high 29 bits:
+// four 32x32->64 products, no 64-bit high multiply.  x, add < 2^61.
+__device__ __forceinline__ uint64_t mulmod61_split_add(uint64_t x, uint32_t m0, uint32_t m1, uint64_t add) {
+    const uint32_t x0 = (uint32_t)x, x1 = (uint32_t)(x >> 32);
+    const uint64_t p00 = (uint64_t)x0 * m0;                        // < 2^64
+    const uint64_t mid = (uint64_t)x0 * m1 + (uint64_t)x1 * m0;    // < 2^62
+    const uint64_t p11 = (uint64_t)x1 * m1;                        // < 2^58
+    // x*m = p00 + mid * 2^32 + p11 * 2^64, with 2^61 == 1 and 2^64 == 8 (mod p)
+    const uint64_t r = (p00 & P61) + (p00 >> 61) + (mid >> 29) + ((mid & ((1ull << 29) - 1)) << 32) +
+                       (p11 << 3) + add;                           // < 2^64
+    return reduce_once(r);
+}
+
 __device__ __forceinline__ uint64_t addmod61(uint64_t a, uint64_t b) {
     uint64_t r = a + b;
     if (r >= P61) r -= P61;
@@ -567,6 +580,8 @@ __device__ __forceinline__ void scan_runs(const uint64_t* partial, uint64_t* key
     const uint64_t M = apow[RUN];
     // every block a thread finishes has the same position in its run (NTHR is a multiple of RUN)
     const uint64_t my_mult = pick_pow<RUN>(apow, tid % RUN + 1);
+    const uint32_t my_m0 = (uint32_t)my_mult, my_m1 = (uint32_t)(my_mult >> 32);
+    const uint32_t M0 = (uint32_t)M, M1 = (uint32_t)(M >> 32);
     uint64_t carry = parent;
     for (int64_t base = 0; base < nblk; base += (int64_t)kRunChunkRuns * RUN) {
         const int cblk = (int)min((int64_t)kRunChunkRuns * RUN, nblk - base);
@@ -599,12 +614,13 @@ __device__ __forceinline__ void scan_runs(const uint64_t* partial, uint64_t* key
         }
         const bool has_ragged = (hi == n_runs) && (hi > lo) && (m_last != RUN);
         const uint64_t ragged_mult = pick_pow<RUN>(apow, m_last);
+        const uint32_t R0 = (uint32_t)ragged_mult, R1 = (uint32_t)(ragged_mult >> 32);
         uint64_t c = 0;
 #pragma unroll
         for (int q = 0; q < kPer; ++q) {
             if (lo + q < hi) {
-                const uint64_t mult = (has_ragged && lo + q == hi - 1) ? ragged_mult : M;
-                c = addmod61(mulmod61(c, mult), tot[q]);
+                const bool rg = has_ragged && lo + q == hi - 1;
+                c = mulmod61_split_add(c, rg ? R0 : M0, rg ? R1 : M1, tot[q]);
             }
         }
         __syncthreads();
@@ -632,8 +648,8 @@ __device__ __forceinline__ void scan_runs(const uint64_t* partial, uint64_t* key
         for (int q = 0; q < kPer; ++q) {
             if (lo + q < hi) {
                 h_in[lo + q] = h;
-                const uint64_t mult = (has_ragged && lo + q == hi - 1) ? ragged_mult : M;
-                h = addmod61(mulmod61(h, mult), tot[q]);
+                const bool rg = has_ragged && lo + q == hi - 1;
+                h = mulmod61_split_add(h, rg ? R0 : M0, rg ? R1 : M1, tot[q]);
             }
         }
         if (lo < hi && hi == n_runs) sh->carry = h;       // hash at the end of this pass
@@ -654,7 +670,7 @@ __device__ __forceinline__ void scan_runs(const uint64_t* partial, uint64_t* key
 #pragma unroll
             for (int u = 0; u < kU; ++u) {
                 const int i = i0 + u * NTHR;
-                if (i < cblk) kout[i] = addmod61(mulmod61(h_in[i / RUN], my_mult), pv[u]);
+                if (i < cblk) kout[i] = mulmod61_split_add(h_in[i / RUN], my_m0, my_m1, pv[u]);
             }
         }
         __syncthreads();
