@@ -219,7 +219,8 @@ def test_bad_shapes_rejected_at_create():
     dict(tier_location=0, link_strategy=1, min_staged_run_bytes=-1),
     dict(tier_location=0, link_strategy=1),
 ], ids=["hbm-bulk", "hbm-vector", "host-zero-copy", "host-staged", "host-default"])
-@pytest.mark.parametrize("name,group", [("qwen", 12), ("qwen", 5), ("tiny", 1), ("ragged", 2), ("tiny", 4)])
+@pytest.mark.parametrize("name,group", [("qwen", 12), ("qwen", 5), ("tiny", 1), ("ragged", 2), ("tiny", 4),
+                                        ("qwen_tp8", 12), ("qwen_tp8", 5), ("small", 1)])
 def test_layer_pipelined_load(name, group, kw):
     """eakv_load_layers moves the same bytes as eakv_load, in layer groups, and records one
     event per group."""
