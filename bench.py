@@ -49,7 +49,7 @@ def parse_args():
     ap.add_argument("--impl", default="eakv", choices=["eakv", "reference"])
     ap.add_argument("--blocks", type=int, default=4096, help="blocks per request")
     ap.add_argument("--pool-blocks", type=int, default=65536)
-    ap.add_argument("--link", default="staged", choices=["zero_copy", "staged"],
+    ap.add_argument("--link", default="staged", choices=["zero_copy", "staged", "copy_engine"],
                     help="host-link strategy of the e2e arm")
     ap.add_argument("--copy-path", default="bulk", choices=["vector", "bulk"])
     ap.add_argument("--copy-ctas", type=int, default=0)
@@ -161,7 +161,8 @@ class Arm:
                   max_call_blocks=max(16384, self.m))
         if host_tier:
             kw.update(tier_location=eakv.TIER_PINNED_HOST,
-                      link_strategy=eakv.LINK_STAGED if args.link == "staged" else eakv.LINK_ZERO_COPY,
+                      link_strategy={"staged": eakv.LINK_STAGED, "zero_copy": eakv.LINK_ZERO_COPY,
+                                     "copy_engine": eakv.LINK_COPY_ENGINE}[args.link],
                       staging_bytes=args.staging_mib << 20, copy_ctas=args.host_ctas)
             if args.link == "staged":
                 kw["copy_ctas"] = args.copy_ctas
@@ -651,7 +652,7 @@ def main():
     reserve = TIER_PROMPTS * m * shape.block_bytes + (4 << 30) + 2 * (args.staging_mib << 20) * 2
     nb = min(args.pool_blocks, int((free - reserve) // shape.block_bytes))
     nb = max(nb, 2 * m)
-    pool = PagedPool(shape, nb, device, fill=lambda q, t: t.random_())
+    pool = PagedPool(shape, nb, device, fill=lambda q, t: t.random_(), contiguous=True)
     torch.cuda.synchronize()
 
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -810,7 +811,8 @@ def sweep(args, torch, eakv, pool, shape, device):
     arms = [("hbm", dict(tier_location=eakv.TIER_DEVICE)),
             ("host_zero_copy", dict(tier_location=eakv.TIER_PINNED_HOST, link_strategy=eakv.LINK_ZERO_COPY)),
             ("host_staged", dict(tier_location=eakv.TIER_PINNED_HOST, link_strategy=eakv.LINK_STAGED,
-                                 staging_bytes=args.staging_mib << 20))]
+                                 staging_bytes=args.staging_mib << 20)),
+            ("host_copy_engine", dict(tier_location=eakv.TIER_PINNED_HOST, link_strategy=eakv.LINK_COPY_ENGINE))]
     for name, kw in arms:
         ctx = eakv.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
                            block_size=shape.block_size, gpu_blocks=nb, host_blocks=kh,

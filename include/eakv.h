@@ -58,6 +58,11 @@ extern "C" {
 #define EAKV_LINK_ZERO_COPY 0   /* kernels read/write the mapped pinned tier directly          */
 #define EAKV_LINK_STAGED    1   /* (default) gather to HBM staging + copy engine on a side stream,
                                    double-buffered against the next gather (and the mirror) */
+#define EAKV_LINK_COPY_ENGINE 2 /* no kernel at all: one strided copy-engine transfer per block (rows =
+                                   the block's pieces, pitch = the distance between piece arrays), issued on
+                                   the caller's stream.  Needs the 2L piece arrays to sit at one constant
+                                   pitch (one [2L][gpu_blocks][piece] allocation); eakv_create returns
+                                   EAKV_E_INVAL otherwise.  Uses no SM while the engine's own kernels run */
 
 /* where the tier lives */
 #define EAKV_TIER_PINNED_HOST 0 /* the product configuration                                   */

@@ -53,6 +53,8 @@ struct eakv_ctx {
     uint64_t base = 0, seed = 0;
 
     void** d_kv_base = nullptr;
+    char* pool_base = nullptr;     // kv_base[0]
+    int64_t pool_pitch = 0;        // bytes between consecutive piece arrays when constant, else 0
     char* tier = nullptr;
     bool tier_owned = false;
 
@@ -273,6 +275,18 @@ int move_blocks(eakv_ctx* ctx, const std::vector<int2>& ent, bool to_tier, cudaS
     const int64_t stage_cap = whole ? ctx->staging_blocks
         : std::min<int64_t>(ctx->max_call_blocks, ctx->staging_blocks * ctx->block_bytes / range_bytes);
     const bool host_tier = ctx->cfg.tier_location == EAKV_TIER_PINNED_HOST;
+    if (ctx->cfg.link_strategy == EAKV_LINK_COPY_ENGINE) {
+        // one strided transfer per block: q_count rows of one piece, pool pitch against slot pitch
+        for (int64_t i = 0; i < m; ++i) {
+            char* pool_p = ctx->pool_base + (int64_t)q_first * ctx->pool_pitch + (int64_t)ent[i].x * ctx->piece_bytes;
+            char* tier_p = ctx->tier + (int64_t)ent[i].y * ctx->block_bytes + (int64_t)q_first * ctx->piece_bytes;
+            CU(cudaMemcpy2DAsync(to_tier ? tier_p : pool_p, to_tier ? (size_t)ctx->piece_bytes : (size_t)ctx->pool_pitch,
+                                 to_tier ? pool_p : tier_p, to_tier ? (size_t)ctx->pool_pitch : (size_t)ctx->piece_bytes,
+                                 (size_t)ctx->piece_bytes, (size_t)q_count, cudaMemcpyDefault, stream));
+            ctx->stats.memcpy_calls += 1;
+        }
+        return EAKV_OK;
+    }
     bool direct = ctx->cfg.link_strategy == EAKV_LINK_ZERO_COPY;
     if (!direct) {
         int64_t runs = 0;
@@ -391,7 +405,7 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
     if (cfg->block_size > kHashMaxBlockSize) return EAKV_E_INVAL;
     const int64_t chunk_blocks = cfg->chunk_blocks > 0 ? cfg->chunk_blocks : 1;
     if (cfg->gpu_blocks > INT32_MAX || cfg->host_blocks * chunk_blocks > INT32_MAX) return EAKV_E_INVAL;
-    if (cfg->policy < 0 || cfg->policy > 2 || cfg->link_strategy < 0 || cfg->link_strategy > 1 ||
+    if (cfg->policy < 0 || cfg->policy > 2 || cfg->link_strategy < 0 || cfg->link_strategy > 2 ||
         cfg->tier_location < 0 || cfg->tier_location > 1 || cfg->copy_path < 0 || cfg->copy_path > 1 ||
         cfg->gpu_free_order < 0 || cfg->gpu_free_order > 1)
         return EAKV_E_INVAL;
@@ -413,7 +427,20 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
     ctx->cfg = *cfg;
     ctx->cfg.kv_base = nullptr;
     // a tier in HBM is copied directly; staging only makes sense across the host link
-    if (cfg->tier_location == EAKV_TIER_DEVICE) ctx->cfg.link_strategy = EAKV_LINK_ZERO_COPY;
+    if (cfg->tier_location == EAKV_TIER_DEVICE && cfg->link_strategy == EAKV_LINK_STAGED)
+        ctx->cfg.link_strategy = EAKV_LINK_ZERO_COPY;
+    if (!cfg->control_plane_only) {
+        ctx->pool_base = static_cast<char*>(cfg->kv_base[0]);
+        int64_t pitch = pieces > 1 ? static_cast<char*>(cfg->kv_base[1]) - static_cast<char*>(cfg->kv_base[0]) : piece * cfg->gpu_blocks;
+        for (int q = 1; q < pieces && pitch > 0; ++q)
+            if (static_cast<char*>(cfg->kv_base[q]) - static_cast<char*>(cfg->kv_base[q - 1]) != pitch) pitch = 0;
+        if (pitch < piece * cfg->gpu_blocks) pitch = 0;
+        ctx->pool_pitch = pitch;
+    }
+    if (cfg->link_strategy == EAKV_LINK_COPY_ENGINE && (cfg->control_plane_only || ctx->pool_pitch == 0)) {
+        delete ctx;
+        return EAKV_E_INVAL;
+    }
     std::memset(&ctx->stats, 0, sizeof(ctx->stats));
     ctx->pieces = pieces;
     ctx->piece_bytes = piece;

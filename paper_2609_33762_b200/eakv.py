@@ -11,7 +11,7 @@ import numpy as np
 
 OK, E_INVAL, E_RANGE, E_CAPACITY, E_NOMEM, E_CUDA, E_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
 POLICY_WRITE_ALL, POLICY_FILTER_FIXED, POLICY_FILTER_CONDITIONED = 0, 1, 2
-LINK_ZERO_COPY, LINK_STAGED = 0, 1
+LINK_ZERO_COPY, LINK_STAGED, LINK_COPY_ENGINE = 0, 1, 2
 TIER_PINNED_HOST, TIER_DEVICE = 0, 1
 FREE_ASCENDING, FREE_REVERSE = 0, 1
 COPY_VECTOR, COPY_BULK = 0, 1

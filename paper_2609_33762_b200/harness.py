@@ -16,17 +16,23 @@ from . import eakv
 
 
 class PagedPool:
-    """2L paged arrays [gpu_blocks, piece_bytes] as int16 tensors on one CUDA device."""
+    """2L paged arrays [gpu_blocks, piece_bytes] as int16 tensors on one CUDA device.  With
+    ``contiguous`` they are the slices of one [2L, gpu_blocks, piece] allocation, i.e. they sit
+    at one constant pitch (what the copy-engine-only link strategy needs)."""
 
-    def __init__(self, shape, gpu_blocks, device="cuda:0", fill=None):
+    def __init__(self, shape, gpu_blocks, device="cuda:0", fill=None, contiguous=False):
         self.shape = shape
         self.gpu_blocks = int(gpu_blocks)
         self.device = torch.device(device)
         W = shape.piece_bytes // 2
         self.words = W
         alloc = torch.zeros if fill is None else torch.empty
-        self.pieces = [alloc((self.gpu_blocks, W), dtype=torch.int16, device=self.device)
-                       for _ in range(shape.pieces_per_block)]
+        if contiguous:
+            self.whole = alloc((shape.pieces_per_block, self.gpu_blocks, W), dtype=torch.int16, device=self.device)
+            self.pieces = [self.whole[q] for q in range(shape.pieces_per_block)]
+        else:
+            self.pieces = [alloc((self.gpu_blocks, W), dtype=torch.int16, device=self.device)
+                           for _ in range(shape.pieces_per_block)]
         if fill is not None:
             for q, t in enumerate(self.pieces):
                 fill(q, t)

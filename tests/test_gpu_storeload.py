@@ -36,6 +36,9 @@ def variants():
     # the default: staged, but scattered slots fall back to the direct kernel
     out.append(dict(link_strategy=e.LINK_STAGED, tier_location=e.TIER_PINNED_HOST,
                     copy_path=e.COPY_BULK, min_staged_run_bytes=0))
+    # copy engine only: needs the piece arrays at one pitch, i.e. one allocation for the whole pool
+    for loc in (e.TIER_PINNED_HOST, e.TIER_DEVICE):
+        out.append(dict(link_strategy=e.LINK_COPY_ENGINE, tier_location=loc, contiguous_pool=True))
     return out
 
 
@@ -44,7 +47,10 @@ def random_pool(rng, shape, nb):
             for _ in range(shape.pieces_per_block)]
 
 
-def to_device(pool_np):
+def to_device(pool_np, contiguous=False):
+    if contiguous:      # one [2L][blocks][words] allocation; the piece arrays are its slices
+        whole = torch.from_numpy(np.stack([a.view(np.int16) for a in pool_np])).cuda()
+        return [whole[q] for q in range(len(pool_np))]
     return [torch.from_numpy(a.view(np.int16).copy()).cuda() for a in pool_np]
 
 
@@ -61,7 +67,7 @@ class Rig:
         rng = np.random.default_rng(seed)
         self.rng = rng
         self.pool_np = random_pool(rng, shape, nb)
-        self.pool_dev = to_device(self.pool_np)
+        self.pool_dev = to_device(self.pool_np, kw.pop("contiguous_pool", False))
         self.tier_np = rng.integers(0, 256, size=(kh, shape.pieces_per_block, shape.piece_bytes),
                                     dtype=np.uint8)
         self.loc = kw.get("tier_location", e.TIER_PINNED_HOST)
@@ -207,7 +213,9 @@ def test_bad_shapes_rejected_at_create():
                 kv_base=[t.data_ptr(), t.data_ptr()])
     for patch in (dict(head_dim=3, block_size=1),              # piece bytes not a multiple of 16
                   dict(kv_base=[t.data_ptr() + 2, t.data_ptr()]),   # misaligned base
-                  dict(block_size=8192), dict(host_blocks=0), dict(policy=7)):
+                  dict(block_size=8192), dict(host_blocks=0), dict(policy=7),
+                  dict(link_strategy=e.LINK_COPY_ENGINE),       # piece arrays not at one positive pitch
+                  dict(link_strategy=3)):
         with pytest.raises(e.EakvError) as ei:
             e.Context(**{**base, **patch})
         assert ei.value.code == e.E_INVAL
@@ -218,7 +226,8 @@ def test_bad_shapes_rejected_at_create():
     dict(tier_location=0, link_strategy=0),
     dict(tier_location=0, link_strategy=1, min_staged_run_bytes=-1),
     dict(tier_location=0, link_strategy=1),
-], ids=["hbm-bulk", "hbm-vector", "host-zero-copy", "host-staged", "host-default"])
+    dict(tier_location=0, link_strategy=2, contiguous_pool=True),
+], ids=["hbm-bulk", "hbm-vector", "host-zero-copy", "host-staged", "host-default", "host-copy-engine"])
 @pytest.mark.parametrize("name,group", [("qwen", 12), ("qwen", 5), ("tiny", 1), ("ragged", 2), ("tiny", 4),
                                         ("qwen_tp8", 12), ("qwen_tp8", 5), ("small", 1)])
 def test_layer_pipelined_load(name, group, kw):
