@@ -127,7 +127,13 @@ typedef struct eakv_config {
                                       it must outlive the context                               */
     int32_t gpu_free_order;        /* EAKV_FREE_*: recency order a request leaves its blocks in
                                       within the GPU tier                                        */
-    int32_t reserved0;
+    int32_t write_behind;          /* 1: eakv_turn_end enqueues the turn's host write on a stream of the
+                                      context, after what precedes it on the caller's stream, and returns
+                                      with the caller's stream free.  The library orders what must wait
+                                      for that write: every later store and load, and a later turn whose
+                                      new blocks reuse a GPU block the write still reads (the caller's
+                                      stream is then made to wait at eakv_turn_begin).  Call eakv_sync
+                                      before reading the tier on the host                              */
 } eakv_config;
 
 typedef struct eakv_stats {

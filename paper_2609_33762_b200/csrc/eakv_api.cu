@@ -94,6 +94,12 @@ struct eakv_ctx {
 
     // two-call turn engine
     cudaStream_t lookup_stream = nullptr;
+    // write-behind: the host write of a finished turn runs on wb_stream
+    cudaStream_t wb_stream = nullptr;
+    cudaEvent_t wb_fence = nullptr, wb_done = nullptr;
+    bool wb_pending = false;
+    std::vector<uint8_t> wb_blocks;     // by GPU block: a pending write still reads it
+    std::vector<uint8_t> wb_slots;      // by tier slot: a pending write still fills it
     uint64_t* turn_keys = nullptr;            // pinned + mapped; the hash kernel writes it directly
     int64_t turn_keys_cap = 0;
     bool turn_open = false;
@@ -166,6 +172,9 @@ void free_all(eakv_ctx* c) {
     if (c->d_error_flag) cudaFree(c->d_error_flag);
     if (c->turn_keys) cudaFreeHost(c->turn_keys);
     if (c->lookup_stream) cudaStreamDestroy(c->lookup_stream);
+    if (c->wb_stream) cudaStreamDestroy(c->wb_stream);
+    if (c->wb_fence) cudaEventDestroy(c->wb_fence);
+    if (c->wb_done) cudaEventDestroy(c->wb_done);
     if (c->tier && c->tier_owned) {
         if (c->cfg.tier_location == EAKV_TIER_DEVICE) cudaFree(c->tier);
         else cudaFreeHost(c->tier);
@@ -269,6 +278,21 @@ int for_slot_runs(const int2* e, int64_t n, F f) {
 //   staged : HBM staging buffers + copy engine on the side stream, double-buffered
 // Under EAKV_LINK_STAGED a call whose slots are so scattered that the copy engine would get
 // mostly single-block copies goes direct instead (per-copy overhead outweighs the DMA's edge).
+// Order `stream` after a pending write-behind store (no-op when none is pending, when it has
+// completed, or for the write-behind stream itself).
+int wait_write_behind(eakv_ctx* ctx, cudaStream_t stream) {
+    if (!ctx->wb_pending || stream == ctx->wb_stream) return EAKV_OK;
+    if (cudaEventQuery(ctx->wb_done) == cudaSuccess) {
+        ctx->wb_pending = false;
+        std::fill(ctx->wb_blocks.begin(), ctx->wb_blocks.end(), (uint8_t)0);
+        std::fill(ctx->wb_slots.begin(), ctx->wb_slots.end(), (uint8_t)0);
+        return EAKV_OK;
+    }
+    cudaGetLastError();            // cudaErrorNotReady is not an error here
+    CU(cudaStreamWaitEvent(stream, ctx->wb_done, 0));
+    return EAKV_OK;
+}
+
 int move_blocks(eakv_ctx* ctx, const std::vector<int2>& ent, bool to_tier, cudaStream_t stream,
                 int q_first, int q_count) {
     const int64_t m = (int64_t)ent.size();
@@ -898,7 +922,9 @@ int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_m
     if (m == 0) return EAKV_OK;
     DeviceGuard g(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    int rc = move_blocks(ctx, ent, true, stream, 0, ctx->pieces);
+    int rc = wait_write_behind(ctx, stream);
+    if (rc != EAKV_OK) return rc;
+    rc = move_blocks(ctx, ent, true, stream, 0, ctx->pieces);
     if (rc != EAKV_OK) return rc;
     ctx->stats.blocks_stored += m;
     ctx->stats.bytes_stored += m * ctx->block_bytes;
@@ -924,7 +950,14 @@ int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_tab
     const int64_t m = n_blocks;
     DeviceGuard g(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    int rc = move_blocks(ctx, ent, false, stream, 0, ctx->pieces);
+    int rc = EAKV_OK;
+    if (ctx->wb_pending) {                        // a slot may still be receiving a deferred write
+        bool touches = false;
+        for (int64_t j = 0; j < m && !touches; ++j) touches = ctx->wb_slots[ent[j].y] != 0;
+        if (touches) rc = wait_write_behind(ctx, stream);
+        if (rc != EAKV_OK) return rc;
+    }
+    rc = move_blocks(ctx, ent, false, stream, 0, ctx->pieces);
     if (rc != EAKV_OK) return rc;
     ctx->stats.blocks_loaded += m;
     ctx->stats.bytes_loaded += m * ctx->block_bytes;
@@ -954,6 +987,14 @@ int eakv_load_layers(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* bl
     }
     DeviceGuard g(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (ctx->wb_pending) {
+        bool touches = false;
+        for (size_t j = 0; j < ent.size() && !touches; ++j) touches = ctx->wb_slots[ent[j].y] != 0;
+        if (touches) {
+            const int rcw = wait_write_behind(ctx, stream);
+            if (rcw != EAKV_OK) return rcw;
+        }
+    }
     for (int grp = 0; grp < groups; ++grp) {
         const int l0 = grp * layers_per_group;
         const int l1 = std::min(L, l0 + layers_per_group);
@@ -1039,6 +1080,21 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
     rc = eakv_gpu_tier_step(ctx, keys, nblk, (n_tokens % b) != 0, ctx->t_resident.data(),
                             ctx->t_block.data(), &tail);
     if (rc != EAKV_OK) return rc;
+    if (ctx->wb_pending) {
+        bool reused = tail >= 0 && ctx->wb_blocks[tail];
+        for (int64_t j = 0; j < nblk && !reused; ++j)
+            reused = !ctx->t_resident[j] && ctx->wb_blocks[ctx->t_block[j]];
+        if (reused) {
+            // the caller is about to overwrite a block the deferred write still reads
+            DeviceGuard gw(ctx->device);
+            rc = wait_write_behind(ctx, static_cast<cudaStream_t>(cuda_stream));
+            if (rc != EAKV_OK) {
+                if (tail >= 0) eakv_gpu_tier_release(ctx, tail);
+                return rc;
+            }
+            // (the marks stay until the write is seen complete: another stream may come next)
+        }
+    }
     const int64_t H = Hu * R;
     const int64_t cover = std::max(G, H);
     const int64_t lo = G, hi = H > G ? H : G;
@@ -1090,9 +1146,36 @@ int eakv_turn_end(eakv_ctx* ctx, void* cuda_stream) {
     ctx->turn_open = false;
     int rc = EAKV_OK;
     const int64_t nblk = (int64_t)ctx->t_block.size();
-    if (nblk > 0)
+    bool any_store = false;
+    for (int64_t j = 0; j < nblk && !any_store; ++j) any_store = ctx->t_admit_b[j] != 0;
+    if (any_store && ctx->cfg.write_behind) {
+        // deferred write: on the context's stream, after what precedes it on the caller's stream
+        DeviceGuard g(ctx->device);
+        cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+        if (!ctx->wb_stream) {
+            CU(cudaStreamCreateWithFlags(&ctx->wb_stream, cudaStreamNonBlocking));
+            CU(cudaEventCreateWithFlags(&ctx->wb_fence, cudaEventDisableTiming));
+            CU(cudaEventCreateWithFlags(&ctx->wb_done, cudaEventDisableTiming));
+            ctx->wb_blocks.assign((size_t)ctx->cfg.gpu_blocks, 0);
+            ctx->wb_slots.assign((size_t)ctx->tier_slots, 0);
+        }
+        CU(cudaEventRecord(ctx->wb_fence, stream));
+        CU(cudaStreamWaitEvent(ctx->wb_stream, ctx->wb_fence, 0));
+        rc = eakv_store(ctx, ctx->t_block.data(), ctx->t_admit_b.data(), ctx->t_slot_b.data(), nblk,
+                        ctx->wb_stream);
+        if (rc == EAKV_OK) {
+            CU(cudaEventRecord(ctx->wb_done, ctx->wb_stream));
+            for (int64_t j = 0; j < nblk; ++j)
+                if (ctx->t_admit_b[j]) {
+                    ctx->wb_blocks[ctx->t_block[j]] = 1;
+                    ctx->wb_slots[ctx->t_slot_b[j]] = 1;
+                }
+            ctx->wb_pending = true;
+        }
+    } else if (nblk > 0) {
         rc = eakv_store(ctx, ctx->t_block.data(), ctx->t_admit_b.data(), ctx->t_slot_b.data(), nblk,
                         cuda_stream);
+    }
     if (ctx->turn_tail >= 0) {
         const int rc2 = eakv_gpu_tier_release(ctx, ctx->turn_tail);
         ctx->turn_tail = -1;

@@ -60,7 +60,7 @@ def plan(cfg, trace, shape, host_gib=None, data_plane=True, ram_fraction=0.6):
 def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=True,
         incremental_hash=True, device="cuda:0", link_strategy=eakv.LINK_STAGED, agents=None,
         turns=None, server_hook=None, chunk_blocks=1, kappa=None, native_turn=False,
-        gpu_free_order=eakv.FREE_ASCENDING):
+        gpu_free_order=eakv.FREE_ASCENDING, write_behind=False):
     import torch
     from eakv_workloads import CONFIGS, SHAPES, key_words_torch, make_trace
     from .harness import AgentServer
@@ -76,7 +76,8 @@ def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=Tru
                          incremental_hash=incremental_hash, policy=POLICIES[policy],
                          kappa_blocks=max(1, cfg.kappa_blocks // chunk_blocks) if kappa is None else kappa,
                          link_strategy=link_strategy, chunk_blocks=chunk_blocks,
-                         native_turn=native_turn and data_plane, gpu_free_order=gpu_free_order)
+                         native_turn=native_turn and data_plane, gpu_free_order=gpu_free_order,
+                         write_behind=write_behind)
     t_setup = time.perf_counter() - t0
     t0 = time.perf_counter()
     server.run(trace, limit=limit)
@@ -92,6 +93,7 @@ def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=Tru
         "config": config, "policy": policy, "requests": n_req, "kv_shape": cfg.shape,
         "gpu_blocks": cfg.gpu_blocks, "host_chunks": kh, "chunk_blocks": chunk_blocks,
         "gpu_free_order": "reverse" if gpu_free_order == eakv.FREE_REVERSE else "ascending",
+        "write_behind": bool(write_behind),
         "host_gib": kh * chunk_blocks * shape.block_bytes / GIB,
         "host_sizing": why, "data_plane": data_plane, "native_turn": bool(native_turn and data_plane),
         "working_set_blocks_eq5": working_set_blocks(trace, shape),
@@ -126,12 +128,14 @@ def main():
     ap.add_argument("--kappa", type=int, default=None, help="write threshold in tier units")
     ap.add_argument("--native-turn", action="store_true",
                     help="drive turns through eakv_turn_begin / eakv_turn_end")
+    ap.add_argument("--write-behind", action="store_true",
+                    help="with --native-turn: host writes are deferred to a stream of the context")
     ap.add_argument("--reverse-free", action="store_true",
                     help="GPU tier keeps a request's blocks tail-first in its recency order")
     args = ap.parse_args()
     out = run(args.config, policy=args.policy, host_gib=args.host_gib, limit=args.limit,
               data_plane=args.data_plane, chunk_blocks=args.chunk_blocks, kappa=args.kappa,
-              native_turn=args.native_turn,
+              native_turn=args.native_turn, write_behind=args.write_behind,
               gpu_free_order=eakv.FREE_REVERSE if args.reverse_free else eakv.FREE_ASCENDING,
               link_strategy=eakv.LINK_ZERO_COPY if args.zero_copy else eakv.LINK_STAGED)
     print(json.dumps(out))

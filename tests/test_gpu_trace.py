@@ -288,3 +288,34 @@ def test_warm_restart_with_adopted_tier_memory():
     assert sum(r["loaded"] for r in server.records) > 0          # restores came from the old bytes
     compare_bytes(server, oracle)
     server.close()
+
+
+@pytest.mark.parametrize("cfg_name,R,policy", [("c0", 1, 0), ("c0_big_tier", 1, 0), ("c0_big_tier", 4, 2)])
+def test_write_behind_turn_engine_bit_exact(cfg_name, R, policy):
+    """Deferred host writes (eakv_turn_end returns with the caller's stream free): records and every
+    resident byte still equal the oracle's.  Config 0's GPU tier turns over completely every turn, so
+    blocks are handed to new keys while their write is still pending and the library has to make the
+    caller's stream wait; the large-tier sibling also restores from slots written by deferred stores."""
+    from paper_2609_33762_b200.harness import AgentServer
+    cfg = CONFIGS[cfg_name]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg)
+    kh = cfg.host_blocks // R
+    kw = dict(policy=policy, kappa_blocks=20, window_ms=40, len_window=16)
+    oracle = TraceOracle(shape, cfg.gpu_blocks, kh, payload=key_words_numpy, chunk_blocks=R, **kw)
+    oracle.run(trace)
+    server = AgentServer(shape, cfg.gpu_blocks, kh, key_words_numpy, chunk_blocks=R, native_turn=True,
+                         incremental_hash=True, write_behind=True, **kw)
+    server.run(trace)
+    compare_records(server.records, oracle.records)
+    assert server.totals == oracle.totals
+    server.ctx.eakv_sync()
+    tier = server.ctx.tier_host_view()
+    for key, slot in oracle.host.order.items():
+        for i in range(R):
+            assert np.array_equal(tier[slot * R + i], oracle.tier[slot * R + i])
+    for q, t in enumerate(server.pool.pieces):
+        got = t.cpu().numpy().view(np.uint8)
+        for key, blk in oracle.gpu.order.items():
+            assert np.array_equal(got[blk], oracle.pool[q][blk])
+    server.close()
