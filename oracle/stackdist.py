@@ -104,3 +104,17 @@ def working_set_full(distances):
     """Smallest capacity (in chunks) at which every re-reference hits: max finite D + 1."""
     finite = [d for d in distances if d != INF]
     return (max(finite) + 1) if finite else 0
+
+
+def working_set_within(request_keys, request_tokens, gpu_prefix_blocks, block_size, percent=1):
+    """Smallest capacity K (in chunks) whose predicted computed tokens are within ``percent`` % of
+    the prediction for an unbounded tier: computed(K) * 100 <= computed(inf) * (100 + percent).
+    Plain scan over K = 0, 1, 2, ... (computed(K) never grows with K, by inclusion)."""
+    stream = [k for keys in request_keys for k in keys]
+    top = working_set_full(reuse_distances(stream))
+    floor_tokens = predict_trace(request_keys, request_tokens, gpu_prefix_blocks, top, block_size)["computed_tokens"]
+    for K in range(0, top + 1):
+        c = predict_trace(request_keys, request_tokens, gpu_prefix_blocks, K, block_size)["computed_tokens"]
+        if c * 100 <= floor_tokens * (100 + percent):
+            return K
+    return top

@@ -75,6 +75,29 @@ def gpu_prefixes(trace, shape, gpu_blocks, stream_host, offsets, gpu_free_order=
     return G
 
 
+def working_set_within(dist_ptr, n_refs, offsets, tokens, G, block_size, ws_full, percent=1):
+    """Smallest tier (in blocks) whose predicted computed prefill is within ``percent`` % of the
+    unbounded tier's: 64 capacities per curve launch, narrowed until the bracket is one block wide
+    (computed prefill never grows with capacity, so the condition is monotone)."""
+    floor_tokens = int(eakv.eakv_capacity_curve(dist_ptr, n_refs, offsets, tokens, G, block_size,
+                                                [max(ws_full, 1)])["computed_tokens"][0])
+    ok = lambda c: int(c) * 100 <= floor_tokens * (100 + percent)
+    lo, hi = -1, max(ws_full, 0)            # lo fails (or is below 0), hi passes
+    while hi - lo > 1:
+        span = hi - lo
+        cand = sorted({lo + max(1, (span * i) // 65) for i in range(1, 65) if lo + max(1, (span * i) // 65) < hi})
+        if not cand:
+            break
+        out = eakv.eakv_capacity_curve(dist_ptr, n_refs, offsets, tokens, G, block_size, [max(c, 0) for c in cand])
+        passed = [c for c, v in zip(cand, out["computed_tokens"]) if ok(v)]
+        failed = [c for c, v in zip(cand, out["computed_tokens"]) if not ok(v)]
+        if passed:
+            hi = min(passed)
+        if failed:
+            lo = max([c for c in failed if c < hi] or [lo])
+    return hi
+
+
 def model(config, host_gib, device="cuda:0", limit=None, agents=None, shared_prefix=0,
           gpu_free_order=eakv.FREE_ASCENDING):
     import torch
@@ -104,6 +127,7 @@ def model(config, host_gib, device="cuda:0", limit=None, agents=None, shared_pre
     t_curve = time.perf_counter() - t0
     finite = dist[:n_refs][dist[:n_refs] >= 0]
     ws_full = int(finite.max().item()) + 1 if finite.numel() else 0
+    ws_99 = working_set_within(dist.data_ptr(), n_refs, offsets, tokens, G, shape.block_size, ws_full)
     n_mean = trace.total_prompt_tokens / len(trace.requests)
     ws_eq5 = int((len(trace.agent_tokens) - 1) * n_mean * shape.bytes_per_token // shape.block_bytes)
     inf_computed = int(out["computed_tokens"][-1])
@@ -118,8 +142,9 @@ def model(config, host_gib, device="cuda:0", limit=None, agents=None, shared_pre
             "requests": len(trace.requests), "references": n_refs,
             "prompt_tokens": int(tokens.sum()), "rows": rows,
             "computed_prefill_tokens_infinite_tier": inf_computed,
-            "working_set_blocks": {"eq5": ws_eq5, "full": ws_full},
-            "working_set_gib": {"eq5": ws_eq5 * shape.block_bytes / GIB, "full": ws_full * shape.block_bytes / GIB},
+            "working_set_blocks": {"eq5": ws_eq5, "full": ws_full, "within_1_percent": ws_99},
+            "working_set_gib": {"eq5": ws_eq5 * shape.block_bytes / GIB, "full": ws_full * shape.block_bytes / GIB,
+                                "within_1_percent": ws_99 * shape.block_bytes / GIB},
             "seconds": {"stream": t_stream, "distances": t_dist, "curve": t_curve},
             "distance_refs_per_s": n_refs / t_dist if t_dist > 0 else None}
 

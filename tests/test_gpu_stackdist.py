@@ -85,6 +85,14 @@ def test_capacity_curve_on_config0():
     assert out["restored_blocks"][c] == oracle.totals["loaded_blocks"]
     assert out["computed_tokens"][c] == oracle.totals["fresh_tokens"]
     assert np.all(np.diff(out["hits"]) >= 0)             # hits are monotone in capacity
+    # smallest tier within 1 % (and 10 %) of the unbounded tier's computed prefill: GPU narrowing
+    # against the oracle's plain scan over every capacity
+    from paper_2609_33762_b200 import capacity
+    ws_full = sd.working_set_full(sd.reuse_distances(stream))
+    for pct in (1, 10):
+        got = capacity.working_set_within(dist_dev.data_ptr(), len(stream), offsets, n_tok, G,
+                                          shape.block_size, ws_full, percent=pct)
+        assert got == sd.working_set_within(req_keys, n_tok, G, shape.block_size, percent=pct)
 
 
 def test_config3_prefix_distances_and_product_tier_agree():

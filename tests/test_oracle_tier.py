@@ -340,3 +340,19 @@ def test_gpu_tier_free_order_against_timestamp_brute_force():
                 g.step(keys, False)
                 assert set(g.order) == set(stamp)
                 assert list(g.order) == sorted(stamp, key=stamp.get)
+
+
+def test_working_set_within_hand_case():
+    """Two requests of 4 keys each, alternating: between two references of a key lie the other 7
+    keys, so every reuse distance is 7; a tier of 8 recovers everything and smaller tiers nothing:
+    both the full working set and the 1 % size are 8; with a GPU prefix covering all of it, nothing
+    is left to recover and the size is 0."""
+    from oracle import stackdist as sd
+    a, b = [1, 2, 3, 4], [5, 6, 7, 8]
+    reqs = [a, b, a, b]
+    toks = [16, 16, 16, 16]
+    assert sd.working_set_full(sd.reuse_distances([k for r in reqs for k in r])) == 8
+    assert sd.working_set_within(reqs, toks, [0, 0, 0, 0], 4, percent=1) == 8
+    assert sd.working_set_within(reqs, toks, [4, 4, 4, 4], 4, percent=1) == 0
+    # half of the benefit is not within 1 % but is within 100 %
+    assert sd.working_set_within(reqs, toks, [0, 0, 0, 0], 4, percent=10**6) == 0
