@@ -591,7 +591,16 @@ def oracle_component_rates():
         tier.step(k, len(k) * 16, i % 5, i)
         refs += len(k)
     t_tier = time.perf_counter() - t0
-    return {"hash_tokens_per_s": len(toks) / t_hash, "tier_refs_per_s": refs / t_tier}
+    # the whole of config 0 (96 requests, every byte held in numpy) through the trace oracle
+    from eakv_workloads import CONFIGS, SHAPES, key_words_numpy, make_trace
+    from oracle.trace import TraceOracle
+    cfg = CONFIGS["c0"]
+    trace = make_trace(cfg)
+    t0 = time.perf_counter()
+    TraceOracle(SHAPES[cfg.shape], cfg.gpu_blocks, cfg.host_blocks, payload=key_words_numpy).run(trace)
+    t_c0 = time.perf_counter() - t0
+    return {"hash_tokens_per_s": len(toks) / t_hash, "tier_refs_per_s": refs / t_tier,
+            "config0_trace_seconds": t_c0}
 
 
 def run_reference(args):
