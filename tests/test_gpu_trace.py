@@ -319,3 +319,47 @@ def test_write_behind_turn_engine_bit_exact(cfg_name, R, policy):
         for key, blk in oracle.gpu.order.items():
             assert np.array_equal(got[blk], oracle.pool[q][blk])
     server.close()
+
+
+def test_write_behind_orders_block_reuse_and_slot_reads():
+    """A deferred write of ~0.9 GiB is still on the link when the next turn is handed the same GPU
+    blocks and fills them at once, and when a third turn restores from the slots being written:
+    the tier must receive the first turn's bytes and the restore must return them."""
+    from paper_2609_33762_b200 import eakv
+    from paper_2609_33762_b200.harness import PagedPool
+    shape = SHAPES["qwen3_30b_a3b"]
+    nb, kh, m = 700, 1400, 640                       # the second prompt has to take 580 of the first's blocks
+    pool = PagedPool(shape, nb, "cuda:0")
+    ctx = eakv.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+                       block_size=shape.block_size, gpu_blocks=nb, host_blocks=kh, kv_base=pool.kv_base,
+                       write_behind=True)
+    stream = torch.cuda.current_stream()
+    rng = np.random.default_rng(77)
+    n = m * shape.block_size
+    prompts = [torch.from_numpy(rng.integers(0, 151936, size=n, dtype=np.int32)).pin_memory() for _ in range(2)]
+
+    def turn(p, value, fill=True):
+        v = ctx.eakv_turn_begin(prompts[p].data_ptr(), n, None, p, 0, stream)
+        ids = torch.as_tensor(v["gpu_block"][v["needs_fill"] != 0].astype(np.int64), device="cuda")
+        if fill and len(ids):
+            for piece in pool.pieces:
+                piece[ids] = value                   # the engine's prefill, on the same stream, at once
+        ctx.eakv_turn_end(stream)
+        return v
+
+    a = turn(0, 0x1111)
+    assert a["n_stored_blocks"] == m and a["n_fill"] == m
+    b = turn(1, 0x2222)                              # reuses most of a's GPU blocks while a's write is pending
+    assert len(set(a["gpu_block"].tolist()) & set(b["gpu_block"][b["needs_fill"] != 0].tolist())) >= 500
+    c = turn(0, 0x3333, fill=False)                  # a's prompt again: restored from the slots just written
+    assert c["restore_hi"] - c["restore_lo"] == m and c["n_fill"] == 0
+    ctx.eakv_sync()
+    tier = ctx.tier_host_view().view(np.uint16)
+    for slot in a["slot"].tolist():
+        assert (tier[slot] == 0x1111).all(), slot
+    for slot in b["slot"].tolist():
+        assert (tier[slot] == 0x2222).all(), slot
+    ids = torch.as_tensor(c["gpu_block"].astype(np.int64), device="cuda")
+    for piece in pool.pieces[::17]:
+        assert bool((piece[ids].view(torch.int16) == 0x1111).all())
+    ctx.close()
