@@ -363,3 +363,33 @@ def test_write_behind_orders_block_reuse_and_slot_reads():
     for piece in pool.pieces[::17]:
         assert bool((piece[ids].view(torch.int16) == 0x1111).all())
     ctx.close()
+
+
+def test_write_behind_orders_a_direct_load_of_pending_slots():
+    """eakv_load of slots that a deferred write is still filling, into GPU blocks the write does
+    not touch: only the slot marks can make it wait, and it must return the written bytes."""
+    from paper_2609_33762_b200 import eakv
+    from paper_2609_33762_b200.harness import PagedPool
+    shape = SHAPES["qwen3_30b_a3b"]
+    nb, kh, m = 1400, 700, 640
+    pool = PagedPool(shape, nb, "cuda:0")
+    ctx = eakv.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+                       block_size=shape.block_size, gpu_blocks=nb, host_blocks=kh, kv_base=pool.kv_base,
+                       write_behind=True)
+    stream = torch.cuda.current_stream()
+    n = m * shape.block_size
+    toks = torch.from_numpy(np.random.default_rng(78).integers(0, 151936, size=n, dtype=np.int32)).pin_memory()
+    v = ctx.eakv_turn_begin(toks.data_ptr(), n, None, 0, 0, stream)
+    ids = torch.as_tensor(v["gpu_block"].astype(np.int64), device="cuda")
+    for piece in pool.pieces:
+        piece[ids] = 0x4444
+    ctx.eakv_turn_end(stream)                        # ~0.9 GiB now on its way to the tier
+    used = set(v["gpu_block"].tolist())
+    spare = np.array([b for b in range(nb) if b not in used][:m], dtype=np.int32)
+    # at once, into blocks the write never touches, last-written slots first
+    ctx.eakv_load(np.ascontiguousarray(v["slot"][::-1]), spare, stream)
+    ctx.eakv_sync()
+    dst = torch.as_tensor(spare.astype(np.int64), device="cuda")
+    for piece in pool.pieces[::13]:
+        assert bool((piece[dst].view(torch.int16) == 0x4444).all())
+    ctx.close()
