@@ -134,6 +134,8 @@ def model(config, host_gib, device="cuda:0", limit=None, agents=None, shared_pre
     rows = []
     for c, g in enumerate(host_gib):
         rows.append({"host_gib": g, "blocks": caps[c], "hits": int(out["hits"][c]),
+                     # gamma_H = C_reuse / C_H (Section 3.2), with C_reuse the Eq. 5 scale
+                     "gamma_h": ws_eq5 / caps[c],
                      "restored_tokens": int(out["restored_blocks"][c]) * shape.block_size,
                      "computed_prefill_tokens": int(out["computed_tokens"][c])})
     return {"config": config, "agents": len(trace.agent_tokens), "shared_prefix_tokens": shared_prefix,
@@ -142,6 +144,8 @@ def model(config, host_gib, device="cuda:0", limit=None, agents=None, shared_pre
             "requests": len(trace.requests), "references": n_refs,
             "prompt_tokens": int(tokens.sum()), "rows": rows,
             "computed_prefill_tokens_infinite_tier": inf_computed,
+            # gamma_G = A * N_bar / K_G (Section 3.2), K_G in tokens
+            "gamma_g": len(trace.agent_tokens) * n_mean / (cfg.gpu_blocks * shape.block_size),
             "working_set_blocks": {"eq5": ws_eq5, "full": ws_full, "within_1_percent": ws_99},
             "working_set_gib": {"eq5": ws_eq5 * shape.block_bytes / GIB, "full": ws_full * shape.block_bytes / GIB,
                                 "within_1_percent": ws_99 * shape.block_bytes / GIB},
