@@ -536,11 +536,53 @@ def oracle_step_rate(seconds, blocks=128, pool_blocks=512, steps_cap=10**9):
     return moved / dt / 1e9, s, dt
 
 
+def oracle_step_rate_c(seconds, blocks=128, pool_blocks=512, steps_cap=10**9):
+    """The same step through the plain C oracle (oracle/eakv_oracle.c: Horner hash with 128-bit
+    products, linear-scan LRU tier, per-piece memcpy), as it stands; (GB/s, steps, seconds)."""
+    from eakv_workloads import SHAPES
+    from oracle import c_oracle
+    from oracle import hash as ohash
+    shape = SHAPES["qwen3_30b_a3b"]
+    rng = np.random.default_rng(1)
+    b, P, Q = shape.block_size, shape.piece_bytes, shape.pieces_per_block
+    pool = [rng.integers(0, 256, size=(pool_blocks, P), dtype=np.uint8) for _ in range(Q)]
+    tier_mem = np.zeros((2 * blocks, Q, P), dtype=np.uint8)
+    tier = c_oracle.Tier(2 * blocks, 0, 8)
+    prompts = {}
+
+    def prompt(s):
+        if s not in prompts:
+            prompts[s] = rng.integers(0, 151936, size=blocks * b, dtype=np.int32)
+        return prompts[s]
+
+    def request(tokens, table):
+        keys = c_oracle.hash_blocks(tokens, b, ohash.HASH_SEED, ohash.HASH_BASE)
+        H, slots = tier.leading_run(keys)
+        _save, _hit, admit, slot = tier.step(keys)
+        c_oracle.load(pool, tier_mem, slots, table[:H])
+        c_oracle.store(pool, tier_mem, table, admit, slot)
+        return (H + int(admit.sum())) * shape.block_bytes
+
+    request(prompt(0), rng.permutation(pool_blocks)[:blocks].astype(np.int32))
+    t0 = time.perf_counter()
+    moved, s = 0, 0
+    while True:
+        s += 1
+        moved += request(prompt(s - 1), rng.permutation(pool_blocks)[:blocks].astype(np.int32))
+        moved += request(prompt(s), rng.permutation(pool_blocks)[:blocks].astype(np.int32))
+        prompts.pop(s - 1, None)
+        dt = time.perf_counter() - t0
+        if dt >= seconds or s >= steps_cap:
+            break
+    tier.close()
+    return moved / dt / 1e9, s, dt
+
+
 def oracle_all_cores(seconds):
     """The same oracle step on every host core at once (one independent process per core, as it
     stands); returns (summed GB/s, processes) or None if the children could not be run."""
     n = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
-    code = f"import bench; print(bench.oracle_step_rate({float(seconds)!r})[0])"
+    code = f"import bench; print(bench.oracle_step_rate_c({float(seconds)!r})[0])"
     env = dict(os.environ, CUDA_VISIBLE_DEVICES="", OMP_NUM_THREADS="1")
     procs = [subprocess.Popen([sys.executable, "-c", code], cwd=ROOT, env=env, stdout=subprocess.PIPE,
                               stderr=subprocess.DEVNULL, text=True) for _ in range(n)]
@@ -616,8 +658,13 @@ def oracle_component_rates():
     t0 = time.perf_counter()
     TraceOracle(SHAPES[cfg.shape], cfg.gpu_blocks, cfg.host_blocks, payload=key_words_numpy).run(trace)
     t_c0 = time.perf_counter() - t0
-    return {"hash_tokens_per_s": len(toks) / t_hash, "tier_refs_per_s": refs / t_tier,
-            "config0_trace_seconds": t_c0}
+    from oracle import c_oracle
+    big = rng.integers(0, 151936, size=1 << 24, dtype=np.int32)
+    t0 = time.perf_counter()
+    c_oracle.hash_blocks(big, 16, ohash.HASH_SEED, ohash.HASH_BASE)
+    t_chash = time.perf_counter() - t0
+    return {"python_hash_tokens_per_s": len(toks) / t_hash, "python_tier_refs_per_s": refs / t_tier,
+            "python_config0_trace_seconds": t_c0, "c_hash_tokens_per_s": len(big) / t_chash}
 
 
 def run_reference(args):
@@ -626,15 +673,15 @@ def run_reference(args):
         return
     blocks = 128
     # warm-up steps, then K timed steps of the bounded sample
-    oracle_step_rate(0.0, blocks=blocks, steps_cap=max(1, min(args.warmup, 2)))
-    gbps, steps, dt = oracle_step_rate(1e9, blocks=blocks, steps_cap=args.steps)
+    oracle_step_rate_c(0.0, blocks=blocks, steps_cap=max(1, min(args.warmup, 2)))
+    gbps, steps, dt = oracle_step_rate_c(1e9, blocks=blocks, steps_cap=args.steps)
     line = {
         "impl": "reference", "metric": METRIC, "value": gbps, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
         "data": "synthetic", "gpu_launches": 0,
         "config": {"workload": WORKLOAD, "blocks_per_request": blocks,
-                   "note": "CPU oracle on a bounded sample of the step (128 blocks per request)"},
+                   "note": "plain C oracle on a bounded sample of the step (128 blocks per request)"},
         "cpu_baseline": {"value": gbps, "unit": UNIT, "cores": 1, "kind": "oracle",
                          "sample": f"{steps} steps x 2 requests x {blocks} blocks (1.5 MiB each)"},
         "e2e": {"value": gbps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -759,9 +806,11 @@ def main():
 
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:
-        g, s, dt = oracle_step_rate(args.cpu_seconds)
+        g, s, dt = oracle_step_rate_c(args.cpu_seconds)
+        gp, sp, dtp = oracle_step_rate(min(args.cpu_seconds, 4.0))
         cpu = {"value": g, "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": f"{s} steps x 2 requests x 128 blocks of 1.5 MiB in {dt:.1f} s"}
+               "sample": f"plain C oracle: {s} steps x 2 requests x 128 blocks of 1.5 MiB in {dt:.1f} s",
+               "python_oracle_value": gp}
         cpu.update(oracle_component_rates())
         allc = oracle_all_cores(min(args.cpu_seconds, 6.0))
         cpu["all_cores"] = ({"value": allc[0], "unit": UNIT, "cores": allc[1],

@@ -15,6 +15,8 @@ Modules
   trace       whole-trace driver: one agent turn = hash, match, tier step, load, store
   audit       declined-chunk audit and threshold sensitivity
   closedloop  closed-loop replay: active pool, first-come-first-served engine, Eq. 2 service times
+  eakv_oracle.c / c_oracle   the same hash, store/load and LRU tier (write-all, fixed admission) in plain C,
+              checked against the modules above; the timed CPU baseline
 
 Parity unpinned: the paper's trace-level results (its prediction tables, replay table
 and declined-chunk shares) need the authors' recorded trajectories, which are not
