@@ -796,9 +796,7 @@ def main():
     traffic = read_profile_traffic(kernel_name, m) if args.tp_shard == 1 else None
 
     # ---- end-to-end arm (pinned host tier, host tokens) ----
-    e2e = None
-    link = None
-    if not args.no_e2e:
+    def e2e_section():
         link = pinned_link_peak(torch, device) if rank == 0 else None
         arm = Arm(args, pool, shape, torch, eakv, host_tier=True, device=device)
         e_steps = max(2, min(args.steps, 8))
@@ -827,21 +825,37 @@ def main():
             e2e.update(host_link_peak_gbps=link, overlap=bool(args.overlap),
                        frac_of_link=e_val / bound / max(world, 1),
                        frac_of_one_direction=e_val / serial / max(world, 1))
+        return e2e
 
-    hashing = hash_throughput(torch, eakv, pool, shape, device, peak) if rank == 0 else None
-    control = control_plane_rate(eakv, pool, shape, device) if rank == 0 else None
+    # side measurements never take the main line down with them
+    def guarded(fn, *a, **k):
+        try:
+            return fn(*a, **k)
+        except Exception as exc:  # noqa: BLE001
+            return {"error": f"{type(exc).__name__}: {exc}"}
+
+    e2e = None
+    if not args.no_e2e:
+        # with one rank a failure here (say, no pinned memory left) must not lose the main line;
+        # with several ranks the section holds collectives, so it runs unguarded
+        e2e = guarded(e2e_section) if dist is None else e2e_section()
+        if "error" in e2e:
+            e2e.update(value=None, unit=UNIT)
+    hashing = guarded(hash_throughput, torch, eakv, pool, shape, device, peak) if rank == 0 else None
+    control = guarded(control_plane_rate, eakv, pool, shape, device) if rank == 0 else None
 
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:
         g, s, dt = oracle_step_rate_c(args.cpu_seconds)
-        gp, sp, dtp = oracle_step_rate(min(args.cpu_seconds, 4.0))
         cpu = {"value": g, "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": f"plain C oracle: {s} steps x 2 requests x 128 blocks of 1.5 MiB in {dt:.1f} s",
-               "python_oracle_value": gp}
-        cpu.update(oracle_component_rates())
-        allc = oracle_all_cores(min(args.cpu_seconds, 6.0))
+               "sample": f"plain C oracle: {s} steps x 2 requests x 128 blocks of 1.5 MiB in {dt:.1f} s"}
+        py = guarded(oracle_step_rate, min(args.cpu_seconds, 4.0))
+        cpu["python_oracle_value"] = py[0] if isinstance(py, tuple) else py
+        cpu.update(guarded(oracle_component_rates))
+        allc = guarded(oracle_all_cores, min(args.cpu_seconds, 6.0))
         cpu["all_cores"] = ({"value": allc[0], "unit": UNIT, "cores": allc[1],
-                             "note": "one independent oracle process per core"} if allc else None)
+                             "note": "one independent oracle process per core"}
+                            if isinstance(allc, tuple) else allc)
 
     if rank == 0:
         line = {
