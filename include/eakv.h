@@ -232,12 +232,21 @@ int eakv_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
  * eakv_config.tier_memory pointing at the memory the old context used, the new context then
  * serves the same restores.  Slots handed out afterwards are the unused ones in ascending order,
  * as in a run that never evicted.  Not carried over: the GPU tier (the engine's blocks are gone
- * with the process), the admission windows (activity, prompt lengths, evictions restart empty,
- * so capacity-conditioned admission may decide differently until they refill) and the counters.
+ * with the process), the counters, and the admission windows, which have a pair of calls of their
+ * own below (without them they restart empty and capacity-conditioned admission may decide
+ * differently until they refill).
  * E_INVAL: tier not empty, a repeated key or slot, a slot outside the tier; nothing changes. */
 int eakv_tier_export(const eakv_ctx* ctx, uint64_t* keys_host_out, int32_t* slots_host_out,
                      int64_t capacity, int64_t* n_out);
 int eakv_tier_import(eakv_ctx* ctx, const uint64_t* keys_host, const int32_t* slots_host, int64_t n);
+
+/* The admission windows (activity per agent, the last prompt lengths, eviction times: the inputs of
+ * the pressure signal, Eq. 10) as an opaque list of int64 values, so that a restarted context decides
+ * exactly as the old one would have.  Export: *n_out = number of values; values_host_out (may be
+ * NULL) receives them if capacity suffices, else E_CAPACITY.  Import replaces the windows of a
+ * context created with the same window settings; E_INVAL (nothing changes) on a malformed list. */
+int eakv_admission_export(const eakv_ctx* ctx, int64_t* values_host_out, int64_t capacity, int64_t* n_out);
+int eakv_admission_import(eakv_ctx* ctx, const int64_t* values_host, int64_t n);
 
 /* The GPU tier's bookkeeping, which the paper leaves to the serving engine (Section 2):
  * an LRU of gpu_index_blocks keyed blocks referenced in order; a non-resident key takes

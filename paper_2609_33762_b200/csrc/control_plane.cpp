@@ -199,4 +199,50 @@ bool Admission::pressure(int64_t agent, int64_t n_tokens, int64_t now_ms, int64_
     return estimate && full && evicting;
 }
 
+int64_t Admission::export_state(int64_t* out, int64_t capacity) const {
+    std::vector<int64_t> v;
+    std::map<int64_t, int64_t> ordered(agent_last_.begin(), agent_last_.end());
+    v.push_back((int64_t)ordered.size());
+    for (const auto& kv : ordered) { v.push_back(kv.first); v.push_back(kv.second); }
+    v.push_back((int64_t)lengths_.size());
+    for (int64_t x : lengths_) v.push_back(x);
+    v.push_back((int64_t)evict_times_.size());
+    for (int64_t x : evict_times_) v.push_back(x);
+    for (size_t i = 0; i < v.size() && (int64_t)i < capacity; ++i) out[i] = v[i];
+    return (int64_t)v.size();
+}
+
+bool Admission::import_state(const int64_t* in, int64_t n) {
+    int64_t i = 0;
+    auto take = [&](int64_t* x) { if (i >= n) return false; *x = in[i++]; return true; };
+    int64_t na = 0, nl = 0, ne = 0;
+    std::unordered_map<int64_t, int64_t> agents;
+    std::deque<int64_t> lengths, evs;
+    int64_t sum = 0;
+    if (!take(&na) || na < 0 || na > (n - i) / 2) return false;
+    for (int64_t k = 0; k < na; ++k) {
+        int64_t a = 0, t = 0;
+        if (!take(&a) || !take(&t)) return false;
+        agents[a] = t;
+    }
+    if (!take(&nl) || nl < 0 || nl > len_window_ || nl > n - i) return false;
+    for (int64_t k = 0; k < nl; ++k) {
+        int64_t x = 0;
+        if (!take(&x) || x < 0) return false;
+        lengths.push_back(x);
+        sum += x;
+    }
+    if (!take(&ne) || ne < 0 || ne != n - i) return false;
+    for (int64_t k = 0; k < ne; ++k) {
+        int64_t x = 0;
+        if (!take(&x)) return false;
+        evs.push_back(x);
+    }
+    agent_last_.swap(agents);
+    lengths_.swap(lengths);
+    length_sum_ = sum;
+    evict_times_.swap(evs);
+    return true;
+}
+
 }  // namespace eakv

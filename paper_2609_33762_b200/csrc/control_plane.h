@@ -8,6 +8,7 @@
 #pragma once
 #include <cstdint>
 #include <deque>
+#include <map>
 #include <unordered_map>
 #include <vector>
 
@@ -73,6 +74,12 @@ public:
     bool pressure(int64_t agent, int64_t n_tokens, int64_t now_ms, int64_t resident_now);
     void note_eviction(int64_t now_ms) { evict_times_.push_back(now_ms); }
     int32_t kappa() const { return kappa_; }
+    // The windows as a flat list of int64: n_agents, (agent, last time) pairs in ascending agent
+    // order, n_lengths, the prompt lengths oldest first, n_evictions, the eviction times oldest
+    // first.  export_state returns the number of values (at most `capacity` are written);
+    // import_state replaces the windows and returns false (nothing changed) on a malformed list.
+    int64_t export_state(int64_t* out, int64_t capacity) const;
+    bool import_state(const int64_t* in, int64_t n);
 
 private:
     int32_t policy_, kappa_, theta_percent_, telemetry_;

@@ -856,6 +856,20 @@ int eakv_tier_import(eakv_ctx* ctx, const uint64_t* keys_host, const int32_t* sl
     return EAKV_OK;
 }
 
+int eakv_admission_export(const eakv_ctx* ctx, int64_t* values_host_out, int64_t capacity, int64_t* n_out) {
+    if (!ctx || !n_out || capacity < 0) return EAKV_E_INVAL;
+    *n_out = ctx->adm->export_state(nullptr, 0);
+    if (!values_host_out) return EAKV_OK;
+    if (capacity < *n_out) return EAKV_E_CAPACITY;
+    ctx->adm->export_state(values_host_out, capacity);
+    return EAKV_OK;
+}
+
+int eakv_admission_import(eakv_ctx* ctx, const int64_t* values_host, int64_t n) {
+    if (!ctx || n <= 0 || !values_host) return EAKV_E_INVAL;
+    return ctx->adm->import_state(values_host, n) ? EAKV_OK : EAKV_E_INVAL;
+}
+
 int eakv_gpu_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
                        int32_t need_tail, uint8_t* resident_out, int32_t* block_out,
                        int32_t* tail_block_out) {

@@ -90,6 +90,7 @@ EXPORTS = [
     "eakv_tier_ptr", "eakv_hash_seed", "eakv_hash_base", "eakv_strerror", "eakv_last_cuda_error",
     "eakv_hash_blocks_static", "eakv_load_layers", "eakv_reuse_distances", "eakv_capacity_curve",
     "eakv_turn_begin", "eakv_turn_end", "eakv_tier_export", "eakv_tier_import",
+    "eakv_admission_export", "eakv_admission_import",
 ]
 STATIC_MAX_BLOCKS = 65536
 
@@ -125,6 +126,8 @@ def lib():
     L.eakv_turn_end.argtypes = [vp, vp]
     L.eakv_tier_export.argtypes = [vp, vp, vp, i64, C.POINTER(i64)]
     L.eakv_tier_import.argtypes = [vp, vp, vp, i64]
+    L.eakv_admission_export.argtypes = [vp, vp, i64, C.POINTER(i64)]
+    L.eakv_admission_import.argtypes = [vp, vp, i64]
     L.eakv_sync.argtypes = [vp]
     L.eakv_get_stats.argtypes = [vp, C.POINTER(Stats)]
     L.eakv_tier_ptr.argtypes = [vp]
@@ -319,6 +322,19 @@ class Context:
         if len(k) != len(s_):
             raise ValueError("keys and slots differ in length")
         self._check(lib().eakv_tier_import(self._h, kp, sp, len(k)), "eakv_tier_import")
+
+    def eakv_admission_export(self):
+        """The admission windows as an opaque int64 array (see eakv_admission_import)."""
+        n = C.c_int64(0)
+        self._check(lib().eakv_admission_export(self._h, None, 0, C.byref(n)), "eakv_admission_export")
+        vals = np.zeros(n.value, dtype=np.int64)
+        self._check(lib().eakv_admission_export(self._h, vals.ctypes.data_as(C.c_void_p), n.value, C.byref(n)),
+                    "eakv_admission_export")
+        return vals
+
+    def eakv_admission_import(self, values):
+        v, vp_ = _np(values, np.int64)
+        self._check(lib().eakv_admission_import(self._h, vp_, len(v)), "eakv_admission_import")
 
     def eakv_tier_step(self, hashes, agent_id, n_tokens, now_ms):
         h, hp = _np(hashes, np.uint64)

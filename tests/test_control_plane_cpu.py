@@ -303,15 +303,16 @@ def test_free_order_argument_is_checked(eakv):
         cp_ctx(eakv, 4, 8, 8, gpu_free_order=2)
 
 
-@pytest.mark.parametrize("policy", [0, 1])
+@pytest.mark.parametrize("policy", [0, 1, 2])
 def test_tier_export_import_restart(eakv, policy):
-    """Stop after half of the trace, export the host tier's index, import it into a fresh context
-    and go on: every later decision equals the uninterrupted oracle run whose GPU tier was emptied
-    at the same point (write-all and fixed admission keep no window state)."""
+    """Stop after half of the trace, export the host tier's index and the admission windows, import
+    them into a fresh context and go on: every later decision equals the uninterrupted oracle run
+    whose GPU tier was emptied at the same point."""
     cfg = CONFIGS["c0_big_tier"]
     shape = SHAPES[cfg.shape]
     trace = make_trace(cfg, agents=5)
-    kw = dict(policy=policy, kappa_blocks=40)          # first prompts (32 blocks) pass the filter
+    # first prompts (32 blocks) pass the filter; short windows so that the pressure signal moves
+    kw = dict(policy=policy, kappa_blocks=40, window_ms=30, len_window=8)
     half = len(trace.requests) // 2
     orc = TraceOracle(shape, cfg.gpu_blocks, 300, **kw)
     for i, req in enumerate(trace.requests):
@@ -322,13 +323,28 @@ def test_tier_export_import_restart(eakv, policy):
     ctx = cp_ctx(eakv, shape.block_size, cfg.gpu_blocks, 300, **kw)
     recs = drive(ctx, first, shape.block_size)
     keys, slots = ctx.eakv_tier_export()
+    windows = ctx.eakv_admission_export()
     assert list(zip(keys.tolist(), slots.tolist())) == list(orc_order_at(trace, shape, cfg, half, kw))
     ctx.close()
     ctx = cp_ctx(eakv, shape.block_size, cfg.gpu_blocks, 300, **kw)
     ctx.eakv_tier_import(keys, slots)
+    ctx.eakv_admission_import(windows)
+    assert ctx.eakv_admission_export().tolist() == windows.tolist()
+    for bad in ([], [5], [1, 3], [0, 2, 7], [0, 0, 3, 1], [0, 9, 1, 2, 3, 4, 5, 6, 7, 8, 9, 0]):
+        with pytest.raises(eakv.EakvError):
+            ctx.eakv_admission_import(np.array(bad, dtype=np.int64))
+    assert ctx.eakv_admission_export().tolist() == windows.tolist()
     assert ctx.eakv_get_stats()["resident"] == len(keys)
     recs += drive(ctx, second, shape.block_size)
     compare(recs, orc.records)
+    if policy == 2:
+        # the windows matter: with the index alone the restarted context decides differently
+        assert sum(int(r["pressure"]) for r in orc.records[half:]) > 0
+        cold = cp_ctx(eakv, shape.block_size, cfg.gpu_blocks, 300, **kw)
+        cold.eakv_tier_import(keys, slots)
+        cold_recs = drive(cold, second, shape.block_size)
+        cold.close()
+        assert [int(r[3]["save"]) for r in cold_recs] != [int(w["save"]) for w in orc.records[half:]]
     # import is refused into a tier that is not empty, and for repeated slots or keys
     with pytest.raises(eakv.EakvError):
         ctx.eakv_tier_import(keys[:1], slots[:1])
