@@ -373,3 +373,29 @@ def orc_order_at(trace, shape, cfg, n, kw):
     for req in trace.requests[:n]:
         o.turn(trace.prompt(req), req.agent, req.time_ms)
     return o.host.order.items()
+
+
+def test_random_traces_across_every_option(eakv):
+    """Small random traces through every combination of policy, chunking, telemetry and GPU free
+    order: the C++ control plane and the oracle must agree on every record."""
+    rng = random.Random(2024)
+    cfg0 = CONFIGS["c0_big_tier"]
+    shape = SHAPES[cfg0.shape]
+    for case in range(24):
+        policy = case % 3
+        R = (1, 2, 4)[(case // 3) % 3]
+        telemetry = (case // 9) % 2
+        order = rng.randrange(2)
+        agents = rng.randrange(2, 7)
+        cfg = replace(cfg0, seed=100 + case, append_median=float(rng.choice([60, 200, 500])),
+                      first_prompt=rng.choice([96, 256, 512]))
+        trace = make_trace(cfg, agents=agents, turns=rng.randrange(3, 8))
+        kh = max(trace.config.context_cap // (shape.block_size * R) + 1, rng.randrange(40, 400) // R)
+        kw = dict(policy=policy, kappa_blocks=rng.choice([0, 2, 8, 30]), theta_percent=rng.choice([50, 95, 100]),
+                  window_ms=rng.choice([5, 40, 60000]), len_window=rng.choice([4, 256]), telemetry=telemetry)
+        orc = TraceOracle(shape, cfg.gpu_blocks, kh, chunk_blocks=R, gpu_free_order=order, **kw)
+        orc.run(trace)
+        ctx = cp_ctx(eakv, shape.block_size, cfg.gpu_blocks, kh, chunk_blocks=R, gpu_free_order=order, **kw)
+        recs = drive_chunked(ctx, trace, shape.block_size, R) if R > 1 else drive(ctx, trace, shape.block_size)
+        compare(recs, orc.records)
+        ctx.close()
