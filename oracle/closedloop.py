@@ -70,16 +70,19 @@ def simulate(n_tasks, turns_of, gap_us_of, active_pool, serve):
     return order, makespan
 
 
-def replay(trace, oracle, model, active_pool, bytes_per_token):
+def replay(trace, oracle, model, active_pool, bytes_per_token, agent_keys=None):
     """Closed-loop replay of ``trace`` against a TraceOracle.  Returns dict(order, makespan_us,
-    totals) where totals are the oracle's token/block counters."""
+    totals) where totals are the oracle's token/block counters.  ``agent_keys`` (agent -> block
+    keys of its final prompt) spares re-hashing: prompts only grow by appends, so a call's keys are
+    a prefix of that list."""
     tasks = sorted(trace.agent_tokens)
     b = oracle.b
 
     def serve(i, turn, start_us):
         a = tasks[i]
         n = int(trace.agent_lengths[a][turn])
-        rec = oracle.turn(trace.agent_tokens[a][:n], a, start_us // 1000)
+        keys = None if agent_keys is None else agent_keys[a][: n // b]
+        rec = oracle.turn(trace.agent_tokens[a][:n], a, start_us // 1000, keys=keys)
         return service_us(model, rec["fresh_tokens"], rec["loaded"] * b * bytes_per_token,
                           rec["stored"] * b * bytes_per_token)
 

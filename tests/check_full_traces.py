@@ -2,6 +2,7 @@
 
     python tests/check_full_traces.py --config c4 --host-gib 64,512
     python tests/check_full_traces.py --config c3 --policy 2
+    python tests/check_full_traces.py --config c3 --policy 2 --host-gib 32 --closed-loop 16
 
 Runs every request of a configuration's trace through the library's control plane
 (control-plane-only context: no GPU needed) and through the oracle, and compares every output
@@ -24,12 +25,47 @@ from oracle.trace import TraceOracle  # noqa: E402
 from paper_2609_33762_b200 import build, eakv  # noqa: E402
 
 
+def closed_loop(args, cfg, shape, trace, agent_keys, kh, kw, gib):
+    """The library's scheduler and control plane against the oracle's closed-loop replay."""
+    from oracle import closedloop as ocl
+    from paper_2609_33762_b200 import closedloop
+    b = shape.block_size
+    t0 = time.time()
+    want = ocl.replay(trace, TraceOracle(shape, cfg.gpu_blocks, kh, **kw), ocl.ServiceModel(), args.closed_loop,
+                      shape.bytes_per_token, agent_keys=agent_keys)
+    ctx = eakv.Context(num_layers=1, kv_heads=1, head_dim=8, block_size=b, gpu_blocks=cfg.gpu_blocks,
+                       host_blocks=kh, kv_base=None, control_plane_only=True, **kw)
+    np_keys = {a: np.asarray(k, dtype=np.uint64) for a, k in agent_keys.items()}
+
+    def turn(tokens, agent, now_ms):
+        n = len(tokens)
+        k = np_keys[agent][: n // b]
+        G, H, _, _ = ctx.eakv_match(k)
+        st = ctx.eakv_tier_step(k, agent, n, now_ms)
+        _, _, tail = ctx.eakv_gpu_tier_step(k, n % b != 0)
+        if tail >= 0:
+            ctx.eakv_gpu_tier_release(tail)
+        return dict(fresh_tokens=n - max(G, H) * b, loaded=max(H - G, 0), stored=int(st["admit"].sum()))
+
+    order, makespan, _ = closedloop.replay_trace(trace, turn, closedloop.ServiceModel(), args.closed_loop,
+                                                 shape.bytes_per_token, b)
+    stats = ctx.eakv_get_stats()
+    ctx.close()
+    assert order == want["order"], "call order differs"
+    assert makespan == want["makespan_us"]
+    print(f"{args.config} policy {args.policy} tier {gib} GiB closed loop A={args.closed_loop}: {len(order)} calls "
+          f"in identical order, makespan {makespan / 1e6:.1f} s, computed prefill {want['totals']['fresh_tokens']}, "
+          f"hits {stats['hits']} ({time.time() - t0:.0f} s)", flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", default="c4")
     ap.add_argument("--host-gib", default="64")
     ap.add_argument("--policy", type=int, default=0)
     ap.add_argument("--limit", type=int, default=None)
+    ap.add_argument("--closed-loop", type=int, default=0, metavar="A",
+                    help="closed-loop replay with an active pool of A tasks: call order, makespan and totals")
     args = ap.parse_args()
     build.build()
     cfg = CONFIGS[args.config]
@@ -42,6 +78,9 @@ def main():
     for gib in [float(x) for x in args.host_gib.split(",")]:
         kh = int(gib * (1 << 30) // shape.block_bytes)
         kw = dict(policy=args.policy, kappa_blocks=cfg.kappa_blocks)
+        if args.closed_loop:
+            closed_loop(args, cfg, shape, trace, agent_keys, kh, kw, gib)
+            continue
         oracle = TraceOracle(shape, cfg.gpu_blocks, kh, **kw)
         ctx = eakv.Context(num_layers=1, kv_heads=1, head_dim=8, block_size=b, gpu_blocks=cfg.gpu_blocks,
                            host_blocks=kh, kv_base=None, control_plane_only=True, **kw)

@@ -94,3 +94,19 @@ def test_smaller_pool_shrinks_the_working_set(mods):
         ctx.close()
         fresh[pool] = tot["fresh"]
     assert fresh[2] < fresh[8]
+
+
+def test_config3_full_closed_loop_parity():
+    """All 1,280 calls of config 3 under conditioned admission, active pool 16, 32 GiB tier: the
+    library's scheduler and control plane give the oracle's call order and makespan (a few seconds;
+    keys come from the oracle's hash, once per agent)."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, os.path.join(root, "tests", "check_full_traces.py"), "--config", "c3",
+                          "--policy", "2", "--host-gib", "32", "--closed-loop", "16"],
+                         capture_output=True, text=True, timeout=600, cwd=root)
+    assert out.returncode == 0, out.stderr[-2000:]
+    assert "1280 calls in identical order" in out.stdout
+    assert "makespan 595.6 s" in out.stdout and "computed prefill 44250953" in out.stdout

@@ -393,3 +393,48 @@ def test_write_behind_orders_a_direct_load_of_pending_slots():
     for piece in pool.pieces[::13]:
         assert bool((piece[dst].view(torch.int16) == 0x4444).all())
     ctx.close()
+
+
+def test_random_traces_with_bytes_across_options():
+    """Small random traces with KV bytes through combinations of policy, chunking, link strategy,
+    copy path, GPU free order, the turn engine and deferred writes: records and resident bytes
+    equal the oracle's in every case."""
+    import random
+    from dataclasses import replace
+    from paper_2609_33762_b200.harness import AgentServer
+    rng = random.Random(77)
+    cfg0 = CONFIGS["c0_big_tier"]
+    shape = SHAPES[cfg0.shape]
+    for case in range(12):
+        policy = case % 3
+        R = (1, 2, 4)[(case // 3) % 3]
+        native = case % 2 == 1
+        wb = native and case % 4 == 3
+        link = rng.randrange(2)
+        order = rng.randrange(2)
+        cfg = replace(cfg0, seed=300 + case, append_median=float(rng.choice([60, 200, 500])),
+                      first_prompt=rng.choice([96, 256, 512]))
+        trace = make_trace(cfg, agents=rng.randrange(2, 6), turns=rng.randrange(3, 7))
+        kh = max(cfg.context_cap // (shape.block_size * R) + 1, rng.randrange(60, 500) // R)
+        kw = dict(policy=policy, kappa_blocks=rng.choice([0, 2, 8, 30]), window_ms=rng.choice([5, 40, 60000]),
+                  len_window=rng.choice([4, 256]))
+        oracle = TraceOracle(shape, cfg.gpu_blocks, kh, payload=key_words_numpy, chunk_blocks=R,
+                             gpu_free_order=order, **kw)
+        oracle.run(trace)
+        server = AgentServer(shape, cfg.gpu_blocks, kh, key_words_numpy, chunk_blocks=R, native_turn=native,
+                             incremental_hash=bool(case & 1), link_strategy=link, copy_path=rng.randrange(2),
+                             gpu_free_order=order, write_behind=wb,
+                             staging_bytes=rng.choice([3, 9]) * shape.block_bytes, **kw)
+        server.run(trace)
+        compare_records(server.records, oracle.records)
+        assert server.totals == oracle.totals, case
+        server.ctx.eakv_sync()
+        tier = server.ctx.tier_host_view()
+        for key, slot in oracle.host.order.items():
+            for i in range(R):
+                assert np.array_equal(tier[slot * R + i], oracle.tier[slot * R + i]), (case, slot)
+        for q, t in enumerate(server.pool.pieces):
+            got = t.cpu().numpy().view(np.uint8)
+            for key, blk in oracle.gpu.order.items():
+                assert np.array_equal(got[blk], oracle.pool[q][blk]), (case, q, blk)
+        server.close()
