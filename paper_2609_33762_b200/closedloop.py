@@ -168,6 +168,8 @@ def run(config, *, policy="write_all", host_gib=None, active_pool=None, model=Se
         "host_sizing": why, "chunk_blocks": chunk_blocks, "theta_percent": theta,
         "data_plane": data_plane, "measured_transfers": measured_transfers,
         "service_model": model.__dict__,
+        # Eq. 2 for long prefixes: OBR -> 1 - beta / (B_H2D * t_pf)
+        "obr_long_prefix": 1.0 - shape.bytes_per_token / model.h2d_bytes_per_us / (model.t_pf_ns / 1000.0),
         "makespan_s": makespan / 1e6, "mean_queue_delay_ms": queue_us / max(1, len(order)) / 1e3,
         "engine_busy_s": {k[:-3]: v / 1e6 for k, v in busy.items()},
         "prompt_tokens": tot["prompt_tokens"], "computed_prefill_tokens": tot["fresh_tokens"],
