@@ -130,9 +130,10 @@ typedef struct eakv_config {
     int32_t write_behind;          /* 1: eakv_turn_end enqueues the turn's host write on a stream of the
                                       context, after what precedes it on the caller's stream, and returns
                                       with the caller's stream free.  The library orders what must wait
-                                      for that write: every later store and load, and a later turn whose
-                                      new blocks reuse a GPU block the write still reads (the caller's
-                                      stream is then made to wait at eakv_turn_begin).  Call eakv_sync
+                                      for that write: every later store, a load that reads a slot the
+                                      write still fills, and a later turn whose new blocks reuse a GPU
+                                      block the write still reads (the caller's stream is then made to
+                                      wait at eakv_turn_begin).  Call eakv_sync
                                       before reading the tier on the host                              */
 } eakv_config;
 
@@ -290,7 +291,8 @@ int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_tab
  *   known_keys    host uint64[n_known] keys of the first n_known blocks, or NULL / 0
  * The engine then produces the KV of every block with needs_fill[j] = 1 into gpu_block[j]
  * (ordered after cuda_stream's load) and calls
- * eakv_turn_end: eakv_store of the admitted blocks on cuda_stream, and release of the partial
+ * eakv_turn_end: eakv_store of the admitted blocks on cuda_stream (with eakv_config.write_behind:
+ * on a stream of the context, behind what cuda_stream holds so far), and release of the partial
  * tail's temporary block.  One turn per context at a time.
  * Errors: those of the calls above; EAKV_E_INVAL when a turn is already open (begin) or none
  * is (end).  On an error in begin no turn is opened; bookkeeping done by then is kept.
