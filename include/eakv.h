@@ -98,7 +98,8 @@ typedef struct eakv_config {
     int32_t theta_percent;         /* occupancy threshold theta, in percent (paper: 95)          */
     int32_t len_window;            /* prompt-length window, in requests (paper: 256)             */
     int64_t window_ms;             /* activity / eviction window (paper: 60 s)                   */
-    int32_t telemetry;             /* 1: tier report available; 0: the estimate alone decides    */
+    int32_t telemetry;             /* 1: the tier's report (occupancy, evictions) is read; 0: no
+                                      report, p_t is the working-set test of Eq. 10 alone        */
     int32_t link_strategy;         /* EAKV_LINK_*                                                */
     int32_t tier_location;         /* EAKV_TIER_*                                                */
     int32_t copy_path;             /* EAKV_COPY_*                                                */
@@ -295,7 +296,18 @@ int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_tab
  * on a stream of the context, behind what cuda_stream holds so far), and release of the partial
  * tail's temporary block.  One turn per context at a time.
  * Errors: those of the calls above; EAKV_E_INVAL when a turn is already open (begin) or none
- * is (end).  On an error in begin no turn is opened; bookkeeping done by then is kept.
+ * is (end, abort).  eakv_turn_begin refuses what it can refuse (a prompt with more units than the
+ * host tier, or more blocks than the GPU tier can hand out: EAKV_E_CAPACITY) before either tier
+ * changes.  If a CUDA call fails after the bookkeeping (the restore in begin, the store in end),
+ * no turn stays open and what the turn registered without producing it is taken back: the units
+ * it admitted leave the host index and, in begin, the GPU blocks it newly keyed leave the GPU
+ * index, so that no later lookup is answered from memory that was never written.  Promotions
+ * and evictions the turn caused stand.
+ * eakv_turn_abort closes an open turn whose KV the engine will not produce (a cancelled or
+ * preempted request): admitted units and the blocks flagged needs_fill are taken back in the same
+ * way, restored blocks stay, the tail block is released; nothing is stored.
+ * A context created with control_plane_only runs the same two calls as pure bookkeeping (no
+ * restore, no store) provided the caller passes all of the prompt's keys in known_keys.
  * eakv_turn_begin hashes on the context's own stream with the context's hash scratch: do not
  * run eakv_hash_blocks of the same context concurrently with it. */
 typedef struct eakv_turn_view {
@@ -322,6 +334,7 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
                     const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
                     void* cuda_stream, eakv_turn_view* view);
 int eakv_turn_end(eakv_ctx* ctx, void* cuda_stream);
+int eakv_turn_abort(eakv_ctx* ctx);
 
 /* Layer-pipelined restore (Section 3.1, Eq. 2: the fixed restoration overhead tau_load is
  * what a consumer waits for before it can start; moving layers in order lets it start on
@@ -371,21 +384,50 @@ int eakv_capacity_curve(const int64_t* dist_dev, int64_t n_refs, const int64_t* 
  * (0 = library default) and parent_hash (pass the seed for a fresh prompt).
  *   tokens_dev device int32[n_tokens]; hashes_dev device uint64[n_tokens / block_size];
  *   n_blocks_out host or NULL; cuda_stream as elsewhere.
- * The scratch is a fixed array inside the library (about 545 KiB per GPU, resident until the
- * process exits) sized for at most EAKV_STATIC_MAX_BLOCKS keys per call: a longer prompt gets
- * EAKV_E_CAPACITY and nothing is launched; hash it in pieces, passing the last key of one piece
- * as parent_hash of the next.  The first call on each device looks up the array's device
- * address (with that device current); make that first call outside any stream capture.
+ * The scratch is a fixed array inside the library (about 545 KiB per GPU, held from the moment
+ * the GPU loads the library's device code until the process exits) sized for at most
+ * EAKV_STATIC_MAX_BLOCKS keys per call: a longer prompt gets EAKV_E_CAPACITY and nothing is
+ * launched; hash it in pieces, passing the last key of one piece as parent_hash of the next.
+ * The first call on each device looks up the array's device address (with that device
+ * current).  Under the CUDA runtime's lazy loading that first call may also be what loads the
+ * device code, array included, so make it once per device at start-up -- before the engine
+ * claims the memory, outside any stream capture; a zero-length warm-up is not enough, pass at
+ * least one block.  Concurrent first calls from several host threads are safe.
  * Every call on a device shares the array: calls whose GPU work can overlap race, so order
  * them (one stream, or events).  Calls no cudaMalloc/cudaFree or other allocating routine.
- * Errors: EAKV_E_INVAL (bad sizes/pointers, block_size > 4096), EAKV_E_CAPACITY, EAKV_E_CUDA. */
+ * Errors: EAKV_E_INVAL (bad sizes/pointers, block_size > 4096), EAKV_E_CAPACITY, EAKV_E_CUDA.
+ *
+ * eakv_hash_blocks_static_status: the kernels behind the call above check every tile against the
+ * sizes they were given and, instead of touching memory outside them, skip the tile and raise a
+ * word in the same fixed array (the context-bound calls report this through eakv_sync).  This
+ * call waits for cuda_stream, reads that word and returns EAKV_OK, or EAKV_E_RANGE after clearing
+ * it: then keys of some call since the last query are missing.  Allocates nothing either. */
 #define EAKV_STATIC_MAX_BLOCKS 65536
 int eakv_hash_blocks_static(const int32_t* tokens_dev, int64_t n_tokens, int32_t block_size,
                             uint64_t hash_base, uint64_t parent_hash, uint64_t* hashes_dev,
                             int64_t* n_blocks_out, void* cuda_stream);
+int eakv_hash_blocks_static_status(void* cuda_stream);
 
 /* Block the host until everything the context enqueued (side streams included) is done. */
 int eakv_sync(eakv_ctx* ctx);
+
+/* Self-tests of the device-side checks (no counterpart in the paper).  Every kernel of the
+ * library compares each entry / tile with the sizes of the buffers it was given and, instead of
+ * touching memory outside them, skips it and raises an error word that the next eakv_sync
+ * reports (EAKV_E_RANGE, or EAKV_E_TIMEOUT for a bounded wait that gave up) and clears.  The host
+ * validates every id first, so in normal use these checks never trip; the two calls below make
+ * them trip on purpose without any access out of bounds and without any unbounded wait.
+ * eakv_selfcheck_limits: the kernels check against these NARROWER limits (pool blocks, tier
+ * slots, keys per hash launch) until called again with zeros; values above the real sizes are
+ * refused (EAKV_E_INVAL).  An entry between the narrowed and the real limit is then skipped on the
+ * device: its bytes do not move, the rest of the call does (one exception: a store under
+ * EAKV_LINK_STAGED gathers into a staging buffer that the copy engine moves as a whole, so the
+ * slot of a skipped entry receives whatever that part of the staging buffer held).
+ * eakv_selfcheck_wait_probe: enqueues a one-thread kernel that waits, with a short poll limit, on a
+ * barrier nothing arrives at, gives up and raises the word: the next eakv_sync returns
+ * EAKV_E_TIMEOUT and the context stays usable. */
+int eakv_selfcheck_limits(eakv_ctx* ctx, int64_t gpu_blocks, int64_t tier_slots, int64_t hash_blocks);
+int eakv_selfcheck_wait_probe(eakv_ctx* ctx, void* cuda_stream);
 
 int eakv_get_stats(const eakv_ctx* ctx, eakv_stats* out);
 /* Base address of the tier (host pointer for TIER_PINNED_HOST, device pointer otherwise). */

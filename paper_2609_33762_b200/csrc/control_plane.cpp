@@ -111,6 +111,17 @@ int32_t KeyedLru::insert(uint64_t key, bool* evicted, uint64_t* victim_key, int3
     return s;
 }
 
+int32_t KeyedLru::erase(uint64_t key) {
+    const int32_t s = find(key);
+    if (s < 0) return -1;
+    table_erase(key);
+    unlink(s);
+    state_[s] = 0;
+    --resident_;
+    free_.push_back(s);
+    return s;
+}
+
 int32_t KeyedLru::take_unkeyed(bool* evicted, uint64_t* victim_key, int32_t* victim_slot) {
     *evicted = false;
     if (free_.empty()) {

@@ -29,6 +29,9 @@ public:
     // least-recent resident and reports it through (*victim_key, *victim_slot).
     // Returns the slot given to key.  *evicted is set to whether an eviction happened.
     int32_t insert(uint64_t key, bool* evicted, uint64_t* victim_key, int32_t* victim_slot);
+    // Remove a resident key: its slot goes back on the free stack (it is the next one handed
+    // out).  Returns the slot, or -1 when the key is not resident.
+    int32_t erase(uint64_t key);
     // take an unkeyed slot (evicting the least-recent resident when none is free)
     int32_t take_unkeyed(bool* evicted, uint64_t* victim_key, int32_t* victim_slot);
     // give an unkeyed slot back to the free stack

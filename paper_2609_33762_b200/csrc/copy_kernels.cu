@@ -118,8 +118,9 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kBulkSpinLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
+                                                  uint32_t limit = kBulkSpinLimit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -295,6 +296,22 @@ copy_blocks_bulk_kernel(CopyLaunch L, int kBulkStages, int kBulkStageBytes) {
         }
     }
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+// Self-test of the bounded wait: one thread waits on a barrier that nothing ever arrives at, with
+// a short poll limit, gives up, raises the error word exactly as the copy kernel would and
+// returns.  Nothing is in flight, so there is nothing to drain.
+__global__ void wait_probe_kernel(int* error_flag, uint32_t limit) {
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x != 0) return;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&bar)) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait_bounded(smem_u32(&bar), 0, limit)) atomicExch(error_flag, kErrBulkTimeout);
+}
+
+cudaError_t launch_wait_probe(int* error_flag, cudaStream_t stream) {
+    wait_probe_kernel<<<1, 32, 0, stream>>>(error_flag, 1u << 12);
+    return cudaGetLastError();
 }
 
 // Ring geometry by piece size.  Measured on B200 at full size (6 GiB calls over a 96 GiB pool,

@@ -86,6 +86,9 @@ struct eakv_ctx {
     int64_t min_staged_run_bytes = 0;
 
     int* d_error_flag = nullptr;
+    // limits the kernels check their entries / tiles against; narrower than the real sizes only
+    // while eakv_selfcheck_limits is in force
+    int64_t check_gpu_blocks = 0, check_tier_slots = 0, check_hash_blocks = 0;
 
     // duplicate-destination checks
     std::vector<uint32_t> slot_stamp, blk_stamp;
@@ -106,7 +109,9 @@ struct eakv_ctx {
     int32_t turn_tail = -1;
     std::vector<int32_t> t_block, t_slot_u, t_slot_b, t_evicted_slots, t_host_slots;
     std::vector<uint8_t> t_resident, t_fill, t_hit, t_admit_u, t_admit_b;
-    std::vector<uint64_t> t_unit_keys, t_evicted_keys;
+    std::vector<uint64_t> t_unit_keys, t_evicted_keys, t_keys_host;
+    const uint64_t* t_keys = nullptr;         // the open turn's block keys and tier-unit keys
+    const uint64_t* t_ukeys = nullptr;
 
     std::string cuda_err;
 };
@@ -130,7 +135,7 @@ struct DeviceGuard {
     int prev = -1;
     bool switched = false;
     explicit DeviceGuard(int dev) {
-        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) {
+        if (dev >= 0 && cudaGetDevice(&prev) == cudaSuccess && prev != dev) {
             switched = cudaSetDevice(dev) == cudaSuccess;
         }
     }
@@ -211,8 +216,8 @@ int launch_copy(eakv_ctx* ctx, const int2* d_entries, const int2* h_inline, int6
     L.slot_q_first = packed ? 0 : q_first;
     L.piece_bytes = ctx->piece_bytes;
     L.slot_from_index = packed ? 1 : 0;
-    L.gpu_blocks = ctx->cfg.gpu_blocks;
-    L.tier_slots = packed ? packed_capacity : ctx->tier_slots;
+    L.gpu_blocks = ctx->check_gpu_blocks;
+    L.tier_slots = packed ? packed_capacity : ctx->check_tier_slots;
     L.error_flag = ctx->d_error_flag;
     L.subs_per_piece = (int32_t)((ctx->piece_bytes + kCopySubBytes - 1) / kCopySubBytes);
     L.group_pieces = 1;          // the bulk launcher raises it for small pieces
@@ -478,6 +483,8 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
     ctx->hash_scratch_blocks = cfg->hash_scratch_blocks > 0 ? cfg->hash_scratch_blocks : (1 << 20);
     ctx->max_prompts = ctx->max_call_blocks;
     ctx->tier_slots = cfg->host_blocks * chunk_blocks;
+    ctx->check_gpu_blocks = cfg->gpu_blocks;
+    ctx->check_tier_slots = ctx->tier_slots;
     ctx->chunk_tokens = (int64_t)cfg->block_size * chunk_blocks;
     ctx->min_staged_run_bytes = cfg->min_staged_run_bytes >= 0 ? cfg->min_staged_run_bytes : 0;
     if (cfg->min_staged_run_bytes == 0) ctx->min_staged_run_bytes = 3ll << 20;
@@ -600,6 +607,25 @@ int eakv_sync(eakv_ctx* ctx) {
     return EAKV_OK;
 }
 
+int eakv_selfcheck_limits(eakv_ctx* ctx, int64_t gpu_blocks, int64_t tier_slots, int64_t hash_blocks) {
+    if (!ctx || ctx->device < 0) return EAKV_E_INVAL;
+    if (gpu_blocks < 0 || gpu_blocks > ctx->cfg.gpu_blocks || tier_slots < 0 || tier_slots > ctx->tier_slots ||
+        hash_blocks < 0)
+        return EAKV_E_INVAL;
+    ctx->check_gpu_blocks = gpu_blocks ? gpu_blocks : ctx->cfg.gpu_blocks;
+    ctx->check_tier_slots = tier_slots ? tier_slots : ctx->tier_slots;
+    ctx->check_hash_blocks = hash_blocks;
+    return EAKV_OK;
+}
+
+int eakv_selfcheck_wait_probe(eakv_ctx* ctx, void* cuda_stream) {
+    if (!ctx || ctx->device < 0) return EAKV_E_INVAL;
+    DeviceGuard g(ctx->device);
+    CU(launch_wait_probe(ctx->d_error_flag, static_cast<cudaStream_t>(cuda_stream)));
+    ctx->stats.kernel_launches += 1;
+    return EAKV_OK;
+}
+
 int eakv_destroy(eakv_ctx* ctx) {
     if (!ctx) return EAKV_E_INVAL;
     if (ctx->device < 0) {
@@ -652,7 +678,7 @@ int eakv_hash_blocks(eakv_ctx* ctx, const int32_t* tokens_dev, int64_t n_tokens,
         L.stages = hash_stages(b);
         L.n_prompts = 0;
         L.tokens_limit = n_tokens - done * b;
-        L.blocks_limit = cur;
+        L.blocks_limit = ctx->check_hash_blocks > 0 ? std::min(cur, ctx->check_hash_blocks) : cur;
         L.error_flag = ctx->d_error_flag;
         const int n_tiles = (int)((cur + tile_blocks - 1) / tile_blocks);
         const bool piece_vec = vec && (((done * b) & 3) == 0);
@@ -745,7 +771,7 @@ int eakv_hash_blocks_batched(eakv_ctx* ctx, const int32_t* tokens_dev,
     L.stages = hash_stages(b);
     L.n_prompts = (int32_t)n_prompts;
     L.tokens_limit = offsets_host[n_prompts];
-    L.blocks_limit = total_blocks;
+    L.blocks_limit = ctx->check_hash_blocks > 0 ? std::min(total_blocks, ctx->check_hash_blocks) : total_blocks;
     L.error_flag = ctx->d_error_flag;
     int launched = 0;
     cudaError_t e = launch_hash(L, (int)n_tiles, generic, vec, stream, &launched);
@@ -1026,48 +1052,92 @@ int eakv_load_layers(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* bl
 // ------------------------------------------------------------------------------------------
 // one turn in two calls
 // ------------------------------------------------------------------------------------------
+namespace {
+
+// Take back what an open turn registered but will never produce.  host_units: the tier units the
+// turn admitted leave the host index (their slots were never written).  gpu_mode 1: every GPU
+// block the turn newly keyed leaves the GPU index (nothing was restored or computed); 2: only
+// those the engine was to fill (the restored ones hold their bytes).  Promotions and evictions
+// the turn caused stand.  Releases the tail block and closes the turn.
+void withdraw_turn(eakv_ctx* ctx, bool host_units, int gpu_mode) {
+    if (host_units) {
+        int64_t n = 0;
+        // last admitted first, so that the free stack hands the slots out again in the same order
+        for (size_t c = ctx->t_admit_u.size(); c-- > 0;)
+            if (ctx->t_admit_u[c] && ctx->host_tier->erase(ctx->t_ukeys[c]) >= 0) ++n;
+        ctx->stats.admitted -= n;
+        ctx->stats.resident = ctx->host_tier->resident();
+    }
+    if (gpu_mode) {
+        for (size_t j = ctx->t_block.size(); j-- > 0;) {
+            const bool drop = gpu_mode == 1 ? !ctx->t_resident[j] : ctx->t_fill[j] != 0;
+            if (drop) ctx->gpu_tier->erase(ctx->t_keys[j]);
+        }
+    }
+    if (ctx->turn_tail >= 0) {
+        eakv_gpu_tier_release(ctx, ctx->turn_tail);
+        ctx->turn_tail = -1;
+    }
+    ctx->turn_open = false;
+}
+
+}  // namespace
+
 int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
                     const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
                     void* cuda_stream, eakv_turn_view* view) {
-    if (!ctx || !view || n_tokens < 0 || n_known < 0 || ctx->device < 0) return EAKV_E_INVAL;
+    if (!ctx || !view || n_tokens < 0 || n_known < 0) return EAKV_E_INVAL;
     if (ctx->turn_open) return EAKV_E_INVAL;
     if (n_known > 0 && !known_keys) return EAKV_E_INVAL;
+    const bool bookkeeping_only = ctx->device < 0;
     const int b = ctx->cfg.block_size;
     const int64_t R = ctx->chunk_tokens / b;
     const int64_t nblk = n_tokens / b;
+    const int64_t nu = nblk / R;
+    const bool need_tail = (n_tokens % b) != 0;
     if (n_known > nblk) n_known = nblk;
-    DeviceGuard g(ctx->device);
-    // key buffer in mapped pinned memory, grown in powers of two
-    if (nblk > ctx->turn_keys_cap) {
-        int64_t cap = 4096;
-        while (cap < nblk) cap <<= 1;
-        if (ctx->turn_keys) {
+    // a context without a device cannot hash: the caller supplies every key
+    if (bookkeeping_only && n_known < nblk) return EAKV_E_INVAL;
+    if (nblk > n_known && !tokens) return EAKV_E_INVAL;
+    // everything that can be refused without a CUDA error is refused here, before either tier changes
+    if (nu > ctx->host_tier->capacity()) return EAKV_E_CAPACITY;
+    if (nblk + (need_tail ? 1 : 0) + ctx->gpu_unkeyed > ctx->gpu_tier->capacity()) return EAKV_E_CAPACITY;
+    DeviceGuard g(bookkeeping_only ? -1 : ctx->device);
+    uint64_t* keys = nullptr;
+    if (bookkeeping_only) {
+        ctx->t_keys_host.assign(known_keys, known_keys + nblk);
+        keys = ctx->t_keys_host.data();
+    } else {
+        // key buffer in mapped pinned memory, grown in powers of two
+        if (nblk > ctx->turn_keys_cap) {
+            int64_t cap = 4096;
+            while (cap < nblk) cap <<= 1;
+            if (ctx->turn_keys) {
+                CU(cudaStreamSynchronize(ctx->lookup_stream));
+                CU(cudaFreeHost(ctx->turn_keys));
+                ctx->turn_keys = nullptr;
+                ctx->turn_keys_cap = 0;
+            }
+            cudaError_t e = cudaHostAlloc(&ctx->turn_keys, (size_t)cap * 8,
+                                          cudaHostAllocMapped | cudaHostAllocPortable);
+            if (e != cudaSuccess) {
+                cudaGetLastError();
+                return EAKV_E_NOMEM;
+            }
+            ctx->turn_keys_cap = cap;
+        }
+        if (!ctx->lookup_stream) CU(cudaStreamCreateWithFlags(&ctx->lookup_stream, cudaStreamNonBlocking));
+        keys = ctx->turn_keys;
+        if (n_known > 0) std::memcpy(keys, known_keys, (size_t)n_known * 8);
+        if (nblk > n_known) {
+            const uint64_t parent = n_known ? keys[n_known - 1] : ctx->seed;
+            int rc = eakv_hash_blocks(ctx, tokens + n_known * b, (nblk - n_known) * (int64_t)b, parent,
+                                      keys + n_known, nullptr, ctx->lookup_stream);
+            if (rc != EAKV_OK) return rc;
             CU(cudaStreamSynchronize(ctx->lookup_stream));
-            CU(cudaFreeHost(ctx->turn_keys));
-            ctx->turn_keys = nullptr;
-            ctx->turn_keys_cap = 0;
         }
-        cudaError_t e = cudaHostAlloc(&ctx->turn_keys, (size_t)cap * 8,
-                                      cudaHostAllocMapped | cudaHostAllocPortable);
-        if (e != cudaSuccess) {
-            cudaGetLastError();
-            return EAKV_E_NOMEM;
-        }
-        ctx->turn_keys_cap = cap;
-    }
-    if (!ctx->lookup_stream) CU(cudaStreamCreateWithFlags(&ctx->lookup_stream, cudaStreamNonBlocking));
-    uint64_t* keys = ctx->turn_keys;
-    if (n_known > 0) std::memcpy(keys, known_keys, (size_t)n_known * 8);
-    if (nblk > n_known) {
-        if (!tokens) return EAKV_E_INVAL;
-        const uint64_t parent = n_known ? keys[n_known - 1] : ctx->seed;
-        int rc = eakv_hash_blocks(ctx, tokens + n_known * b, (nblk - n_known) * (int64_t)b, parent,
-                                  keys + n_known, nullptr, ctx->lookup_stream);
-        if (rc != EAKV_OK) return rc;
-        CU(cudaStreamSynchronize(ctx->lookup_stream));
     }
     // tier units: one key per full chunk (the key at the chunk's last block)
-    const int64_t nu = nblk / R;
     const uint64_t* ukeys = keys;
     if (R > 1) {
         ctx->t_unit_keys.resize((size_t)nu);
@@ -1076,7 +1146,7 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
     }
     ctx->t_block.resize((size_t)nblk); ctx->t_resident.resize((size_t)nblk);
     ctx->t_fill.assign((size_t)nblk, 0);
-    ctx->t_hit.resize((size_t)nu); ctx->t_admit_u.resize((size_t)nu); ctx->t_slot_u.resize((size_t)nu);
+    ctx->t_hit.resize((size_t)nu); ctx->t_admit_u.assign((size_t)nu, 0); ctx->t_slot_u.resize((size_t)nu);
     ctx->t_evicted_keys.resize((size_t)nu); ctx->t_evicted_slots.resize((size_t)nu);
     ctx->t_host_slots.resize((size_t)nu);
     int64_t G = 0, G_unused = 0, Hu = 0;
@@ -1089,21 +1159,27 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
     rc = eakv_tier_step(ctx, ukeys, nu, agent_id, n_tokens, now_ms, ctx->t_hit.data(),
                         ctx->t_admit_u.data(), ctx->t_slot_u.data(), ctx->t_evicted_keys.data(),
                         ctx->t_evicted_slots.data(), &n_ev, &info);
-    if (rc != EAKV_OK) return rc;
+    if (rc != EAKV_OK) return rc;                // refused requests change nothing
+    ctx->t_keys = keys;
+    ctx->t_ukeys = ukeys;
     int32_t tail = -1;
-    rc = eakv_gpu_tier_step(ctx, keys, nblk, (n_tokens % b) != 0, ctx->t_resident.data(),
-                            ctx->t_block.data(), &tail);
-    if (rc != EAKV_OK) return rc;
+    rc = eakv_gpu_tier_step(ctx, keys, nblk, need_tail, ctx->t_resident.data(), ctx->t_block.data(), &tail);
+    if (rc != EAKV_OK) {                          // (capacity was checked above)
+        ctx->t_block.clear();
+        withdraw_turn(ctx, true, 0);
+        return rc;
+    }
+    ctx->turn_open = true;
+    ctx->turn_tail = tail;
     if (ctx->wb_pending) {
         bool reused = tail >= 0 && ctx->wb_blocks[tail];
         for (int64_t j = 0; j < nblk && !reused; ++j)
             reused = !ctx->t_resident[j] && ctx->wb_blocks[ctx->t_block[j]];
         if (reused) {
             // the caller is about to overwrite a block the deferred write still reads
-            DeviceGuard gw(ctx->device);
             rc = wait_write_behind(ctx, static_cast<cudaStream_t>(cuda_stream));
             if (rc != EAKV_OK) {
-                if (tail >= 0) eakv_gpu_tier_release(ctx, tail);
+                withdraw_turn(ctx, true, 1);
                 return rc;
             }
             // (the marks stay until the write is seen complete: another stream may come next)
@@ -1112,14 +1188,15 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
     const int64_t H = Hu * R;
     const int64_t cover = std::max(G, H);
     const int64_t lo = G, hi = H > G ? H : G;
-    if (hi > lo) {
+    if (hi > lo && !bookkeeping_only) {
         // block slots of the restored blocks: chunk slot * R + position inside the chunk
         std::vector<int32_t> slots((size_t)(hi - lo));
         for (int64_t j = lo; j < hi; ++j)
             slots[j - lo] = (int32_t)((int64_t)ctx->t_host_slots[j / R] * R + j % R);
         rc = eakv_load(ctx, slots.data(), ctx->t_block.data() + lo, hi - lo, cuda_stream);
         if (rc != EAKV_OK) {
-            if (tail >= 0) eakv_gpu_tier_release(ctx, tail);
+            // nothing of this turn was restored or will be computed: neither tier may list it
+            withdraw_turn(ctx, true, 1);
             return rc;
         }
     }
@@ -1138,8 +1215,6 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
             ++n_store;
         }
     }
-    ctx->turn_open = true;
-    ctx->turn_tail = tail;
     view->n_blocks = nblk; view->n_units = nu;
     view->gpu_prefix_blocks = G; view->host_prefix_blocks = H;
     view->restore_lo = lo; view->restore_hi = hi;
@@ -1156,28 +1231,30 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
 }
 
 int eakv_turn_end(eakv_ctx* ctx, void* cuda_stream) {
-    if (!ctx || ctx->device < 0 || !ctx->turn_open) return EAKV_E_INVAL;
-    ctx->turn_open = false;
+    if (!ctx || !ctx->turn_open) return EAKV_E_INVAL;
     int rc = EAKV_OK;
     const int64_t nblk = (int64_t)ctx->t_block.size();
     bool any_store = false;
     for (int64_t j = 0; j < nblk && !any_store; ++j) any_store = ctx->t_admit_b[j] != 0;
-    if (any_store && ctx->cfg.write_behind) {
+    if (ctx->device < 0) {
+        // bookkeeping only: nothing to copy
+    } else if (any_store && ctx->cfg.write_behind) {
         // deferred write: on the context's stream, after what precedes it on the caller's stream
         DeviceGuard g(ctx->device);
         cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-        if (!ctx->wb_stream) {
-            CU(cudaStreamCreateWithFlags(&ctx->wb_stream, cudaStreamNonBlocking));
-            CU(cudaEventCreateWithFlags(&ctx->wb_fence, cudaEventDisableTiming));
-            CU(cudaEventCreateWithFlags(&ctx->wb_done, cudaEventDisableTiming));
-            ctx->wb_blocks.assign((size_t)ctx->cfg.gpu_blocks, 0);
-            ctx->wb_slots.assign((size_t)ctx->tier_slots, 0);
-        }
-        CU(cudaEventRecord(ctx->wb_fence, stream));
-        CU(cudaStreamWaitEvent(ctx->wb_stream, ctx->wb_fence, 0));
-        rc = eakv_store(ctx, ctx->t_block.data(), ctx->t_admit_b.data(), ctx->t_slot_b.data(), nblk,
-                        ctx->wb_stream);
-        if (rc == EAKV_OK) {
+        rc = [&]() -> int {
+            if (!ctx->wb_stream) {
+                CU(cudaStreamCreateWithFlags(&ctx->wb_stream, cudaStreamNonBlocking));
+                CU(cudaEventCreateWithFlags(&ctx->wb_fence, cudaEventDisableTiming));
+                CU(cudaEventCreateWithFlags(&ctx->wb_done, cudaEventDisableTiming));
+                ctx->wb_blocks.assign((size_t)ctx->cfg.gpu_blocks, 0);
+                ctx->wb_slots.assign((size_t)ctx->tier_slots, 0);
+            }
+            CU(cudaEventRecord(ctx->wb_fence, stream));
+            CU(cudaStreamWaitEvent(ctx->wb_stream, ctx->wb_fence, 0));
+            int r = eakv_store(ctx, ctx->t_block.data(), ctx->t_admit_b.data(), ctx->t_slot_b.data(), nblk,
+                               ctx->wb_stream);
+            if (r != EAKV_OK) return r;
             CU(cudaEventRecord(ctx->wb_done, ctx->wb_stream));
             for (int64_t j = 0; j < nblk; ++j)
                 if (ctx->t_admit_b[j]) {
@@ -1185,17 +1262,21 @@ int eakv_turn_end(eakv_ctx* ctx, void* cuda_stream) {
                     ctx->wb_slots[ctx->t_slot_b[j]] = 1;
                 }
             ctx->wb_pending = true;
-        }
-    } else if (nblk > 0) {
+            return EAKV_OK;
+        }();
+    } else if (any_store) {
         rc = eakv_store(ctx, ctx->t_block.data(), ctx->t_admit_b.data(), ctx->t_slot_b.data(), nblk,
                         cuda_stream);
     }
-    if (ctx->turn_tail >= 0) {
-        const int rc2 = eakv_gpu_tier_release(ctx, ctx->turn_tail);
-        ctx->turn_tail = -1;
-        if (rc == EAKV_OK) rc = rc2;
-    }
+    // a store that could not be enqueued leaves slots unwritten: their keys must not stay listed
+    withdraw_turn(ctx, rc != EAKV_OK, 0);
     return rc;
+}
+
+int eakv_turn_abort(eakv_ctx* ctx) {
+    if (!ctx || !ctx->turn_open) return EAKV_E_INVAL;
+    withdraw_turn(ctx, true, 2);
+    return EAKV_OK;
 }
 
 // ------------------------------------------------------------------------------------------

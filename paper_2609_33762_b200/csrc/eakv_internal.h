@@ -128,6 +128,8 @@ cudaError_t launch_copy_bulk(const CopyLaunch& L, bool to_tier, int ctas, cudaSt
 // pull `bytes` (rounded up to 16) of per-call arguments from mapped pinned memory into device memory
 cudaError_t launch_fetch_args(void* dst_dev, const void* src_host_mapped, size_t bytes,
                               cudaStream_t stream);
+// bounded-wait self-test: a wait that nothing satisfies gives up and raises kErrBulkTimeout
+cudaError_t launch_wait_probe(int* error_flag, cudaStream_t stream);
 cudaError_t copy_kernels_init();
 int copy_vector_ctas_per_sm();
 

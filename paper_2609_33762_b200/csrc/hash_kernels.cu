@@ -866,30 +866,37 @@ cudaError_t hash_kernels_init() {
 // there can fail outright, or stall the whole device while the driver makes room), or in a
 // latency-critical section that may not take the implicit synchronisation of an allocation.
 // eakv_hash_blocks_static computes the same keys as eakv_hash_blocks without a context and
-// without allocating anything: its scratch (block partials, the power table B^0..B^b and
-// the ticket counter) lives in the file-scope array below, which every GPU that loads the
-// library keeps resident until the process exits.
+// without allocating anything: its scratch (block partials, the power table B^0..B^b, the
+// ticket counter and a self-check word) lives in the file-scope array below, which every GPU
+// that loads the library keeps resident until the process exits.
 //
 // The array is shared by every call on a device and keeps the previous call's contents:
 // each call rewrites the power table, overwrites the partials it uses and zeroes the ticket
 // counter before its kernel runs.  Two calls whose GPU work overlaps (different streams
-// without an ordering between them) race on it.
+// without an ordering between them) race on it.  The self-check word is the one thing a call
+// does not clear: it stays raised until eakv_hash_blocks_static_status reads it.
 // ---------------------------------------------------------------------------------------
 #include "../../include/eakv.h"
+
+#include <atomic>
+#include <mutex>
 
 namespace eakv {
 
 constexpr int64_t kStaticMaxBlocks = EAKV_STATIC_MAX_BLOCKS;                 // 65,536 keys per call
 constexpr size_t kStaticPartialBytes = (size_t)kStaticMaxBlocks * 8;          // 512 KiB
 constexpr size_t kStaticPowBytes = ((size_t)(kHashMaxBlockSize + 1) * 8 + 255) / 256 * 256;
-constexpr size_t kStaticCounterBytes = 256;
-constexpr size_t kStaticBytes = kStaticPartialBytes + kStaticPowBytes + kStaticCounterBytes;
+constexpr size_t kStaticCounterBytes = 256;      // ticket counter (cleared per call)
+constexpr size_t kStaticFlagBytes = 256;         // self-check word (cleared only when read)
+constexpr size_t kStaticBytes = kStaticPartialBytes + kStaticPowBytes + kStaticCounterBytes + kStaticFlagBytes;
 
 // In host code this name is only a handle for cudaGetSymbolAddress, never an address.
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
 
 constexpr int kMaxDevices = 64;
-static unsigned char* g_static_ptr[kMaxDevices];   // device address per device, set once
+// device address per device; published once, under g_static_mutex, after the set-up succeeded
+static std::atomic<unsigned char*> g_static_ptr[kMaxDevices];
+static std::mutex g_static_mutex;
 
 // thread e writes B^e mod p
 __global__ void fill_pow_table_kernel(uint64_t* pw, uint64_t base, int n_entries) {
@@ -901,6 +908,30 @@ __global__ void fill_pow_table_kernel(uint64_t* pw, uint64_t base, int n_entries
         }
         pw[e] = r;
     }
+}
+
+// The array's device address on the current device (set-up on first use), or NULL.
+static unsigned char* static_scratch(int* dev_out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    if (dev_out) *dev_out = dev;
+    unsigned char* p = g_static_ptr[dev].load(std::memory_order_acquire);
+    if (p) return p;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    p = g_static_ptr[dev].load(std::memory_order_acquire);
+    if (p) return p;
+    // once per device, with that device current: resolve the array's device address
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || addr == nullptr) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    if (hash_kernels_init() != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    g_static_ptr[dev].store(static_cast<unsigned char*>(addr), std::memory_order_release);
+    return static_cast<unsigned char*>(addr);
 }
 
 }  // namespace eakv
@@ -918,25 +949,12 @@ extern "C" int eakv_hash_blocks_static(const int32_t* tokens_dev, int64_t n_toke
     if (!tokens_dev || !hashes_dev) return EAKV_E_INVAL;
     if (((uintptr_t)tokens_dev & 3) || ((uintptr_t)hashes_dev & 7)) return EAKV_E_INVAL;
 
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return EAKV_E_CUDA;
-    if (g_static_ptr[dev] == nullptr) {
-        // once per device, with that device current: resolve the array's device address
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
-            cudaGetLastError();
-            return EAKV_E_CUDA;
-        }
-        if (hash_kernels_init() != cudaSuccess) {
-            cudaGetLastError();
-            return EAKV_E_CUDA;
-        }
-        g_static_ptr[dev] = static_cast<unsigned char*>(p);
-    }
-    unsigned char* scratch = g_static_ptr[dev];
+    unsigned char* scratch = static_scratch(nullptr);
+    if (!scratch) return EAKV_E_CUDA;
     uint64_t* partial = reinterpret_cast<uint64_t*>(scratch);
     uint64_t* pw = reinterpret_cast<uint64_t*>(scratch + kStaticPartialBytes);
     int* counter = reinterpret_cast<int*>(scratch + kStaticPartialBytes + kStaticPowBytes);
+    int* flag = reinterpret_cast<int*>(scratch + kStaticPartialBytes + kStaticPowBytes + kStaticCounterBytes);
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     constexpr uint64_t P = (1ull << 61) - 1;
@@ -966,19 +984,40 @@ extern "C" int eakv_hash_blocks_static(const int32_t* tokens_dev, int64_t n_toke
     L.tile_blocks = hash_tile_blocks(block_size, nblk);
     L.stages = hash_stages(block_size);
     L.n_prompts = 0;
-    {   // powers B^0 .. B^b on the host (at most 4,097 modular products) for the by-value limbs
+    {   // powers B^0 .. B^min(b, 64) on the host for the by-value limbs of the small-block kernels
         uint64_t pw_host[65];
         const int lim = block_size < 64 ? block_size : 64;
         pw_host[0] = 1;
         for (int e = 1; e <= lim; ++e)
             pw_host[e] = (uint64_t)(((unsigned __int128)pw_host[e - 1] * base) % P);
         if (block_size <= 64) hash_fill_limbs(L, pw_host, block_size);
-        else L.pow_block = 0;   // not used by the kernels chosen for larger blocks
+        else L.pow_block = 0;   // larger blocks read B^b from the device power table
     }
     L.tokens_limit = n_tokens;
     L.blocks_limit = nblk;
-    L.error_flag = reinterpret_cast<int*>(scratch + kStaticPartialBytes + kStaticPowBytes) + 1;
+    L.error_flag = flag;
     const int n_tiles = (int)((nblk + L.tile_blocks - 1) / L.tile_blocks);
     if (launch_hash(L, n_tiles, generic, vec, stream) != cudaSuccess) return EAKV_E_CUDA;
     return EAKV_OK;
+}
+
+extern "C" int eakv_hash_blocks_static_status(void* cuda_stream) {
+    using namespace eakv;
+    unsigned char* scratch = static_scratch(nullptr);
+    if (!scratch) return EAKV_E_CUDA;
+    int* flag = reinterpret_cast<int*>(scratch + kStaticPartialBytes + kStaticPowBytes + kStaticCounterBytes);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int value = 0;
+    if (cudaMemcpyAsync(&value, flag, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess) {
+        cudaGetLastError();
+        return EAKV_E_CUDA;
+    }
+    if (value == 0) return EAKV_OK;
+    if (cudaMemsetAsync(flag, 0, sizeof(int), stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess) {
+        cudaGetLastError();
+        return EAKV_E_CUDA;
+    }
+    return EAKV_E_RANGE;
 }

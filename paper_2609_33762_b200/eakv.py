@@ -88,9 +88,10 @@ EXPORTS = [
     "eakv_hash_blocks_batched", "eakv_match", "eakv_tier_step", "eakv_gpu_tier_step",
     "eakv_gpu_tier_release", "eakv_store", "eakv_load", "eakv_sync", "eakv_get_stats",
     "eakv_tier_ptr", "eakv_hash_seed", "eakv_hash_base", "eakv_strerror", "eakv_last_cuda_error",
-    "eakv_hash_blocks_static", "eakv_load_layers", "eakv_reuse_distances", "eakv_capacity_curve",
-    "eakv_turn_begin", "eakv_turn_end", "eakv_tier_export", "eakv_tier_import",
+    "eakv_hash_blocks_static", "eakv_hash_blocks_static_status", "eakv_load_layers", "eakv_reuse_distances", "eakv_capacity_curve",
+    "eakv_turn_begin", "eakv_turn_end", "eakv_turn_abort", "eakv_tier_export", "eakv_tier_import",
     "eakv_admission_export", "eakv_admission_import",
+    "eakv_selfcheck_limits", "eakv_selfcheck_wait_probe",
 ]
 STATIC_MAX_BLOCKS = 65536
 
@@ -111,6 +112,7 @@ def lib():
     L.eakv_destroy.argtypes = [vp]
     L.eakv_hash_blocks.argtypes = [vp, vp, i64, u64, vp, C.POINTER(i64), vp]
     L.eakv_hash_blocks_static.argtypes = [vp, i64, i32, u64, u64, vp, C.POINTER(i64), vp]
+    L.eakv_hash_blocks_static_status.argtypes = [vp]
     L.eakv_hash_blocks_batched.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp]
     L.eakv_match.argtypes = [vp, vp, i64, C.POINTER(i64), C.POINTER(i64), vp, vp]
     L.eakv_tier_step.argtypes = [vp, vp, i64, i64, i64, i64, vp, vp, vp, vp, vp,
@@ -124,11 +126,14 @@ def lib():
     L.eakv_capacity_curve.argtypes = [vp, i64, vp, vp, vp, i64, i32, vp, i32, vp, vp, vp, vp, vp]
     L.eakv_turn_begin.argtypes = [vp, vp, i64, vp, i64, i64, i64, vp, C.POINTER(TurnView)]
     L.eakv_turn_end.argtypes = [vp, vp]
+    L.eakv_turn_abort.argtypes = [vp]
     L.eakv_tier_export.argtypes = [vp, vp, vp, i64, C.POINTER(i64)]
     L.eakv_tier_import.argtypes = [vp, vp, vp, i64]
     L.eakv_admission_export.argtypes = [vp, vp, i64, C.POINTER(i64)]
     L.eakv_admission_import.argtypes = [vp, vp, i64]
     L.eakv_sync.argtypes = [vp]
+    L.eakv_selfcheck_limits.argtypes = [vp, i64, i64, i64]
+    L.eakv_selfcheck_wait_probe.argtypes = [vp, vp]
     L.eakv_get_stats.argtypes = [vp, C.POINTER(Stats)]
     L.eakv_tier_ptr.argtypes = [vp]
     L.eakv_tier_ptr.restype = vp
@@ -166,6 +171,14 @@ def eakv_hash_blocks_static(tokens_dev, n_tokens, block_size, hash_base, parent_
     if rc != OK:
         raise EakvError(rc, "eakv_hash_blocks_static")
     return n.value
+
+
+def eakv_hash_blocks_static_status(stream=None):
+    """Raise EakvError(E_RANGE) if a self-check of the allocation-free hash tripped since the
+    last query (the word is cleared by the query); waits for ``stream``."""
+    rc = lib().eakv_hash_blocks_static_status(_stream(stream))
+    if rc != OK:
+        raise EakvError(rc, "eakv_hash_blocks_static_status")
 
 
 def eakv_reuse_distances(keys_dev, n_refs, dist_dev, stream=None):
@@ -420,8 +433,18 @@ class Context:
     def eakv_turn_end(self, stream=None):
         self._check(lib().eakv_turn_end(self._h, _stream(stream)), "eakv_turn_end")
 
+    def eakv_turn_abort(self):
+        self._check(lib().eakv_turn_abort(self._h), "eakv_turn_abort")
+
     def eakv_sync(self):
         self._check(lib().eakv_sync(self._h), "eakv_sync")
+
+    def eakv_selfcheck_limits(self, gpu_blocks=0, tier_slots=0, hash_blocks=0):
+        self._check(lib().eakv_selfcheck_limits(self._h, int(gpu_blocks), int(tier_slots), int(hash_blocks)),
+                    "eakv_selfcheck_limits")
+
+    def eakv_selfcheck_wait_probe(self, stream=None):
+        self._check(lib().eakv_selfcheck_wait_probe(self._h, _stream(stream)), "eakv_selfcheck_wait_probe")
 
     # -- introspection ----------------------------------------------------------------------
     def eakv_get_stats(self):

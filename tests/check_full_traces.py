@@ -1,4 +1,5 @@
-"""Whole-trace control-plane parity on the CPU (not collected by pytest: it takes minutes).
+"""Whole-trace control-plane parity on the CPU from the command line, for tier sizes and policies
+beyond the ones tests/test_full_traces_cpu.py runs.
 
     python tests/check_full_traces.py --config c4 --host-gib 64,512
     python tests/check_full_traces.py --config c3 --policy 2
@@ -18,6 +19,7 @@ import numpy as np
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 sys.path.insert(0, ROOT)
+sys.path.insert(0, os.path.join(ROOT, "tests"))
 
 from eakv_workloads import CONFIGS, SHAPES, make_trace  # noqa: E402
 from oracle import hash as ohash  # noqa: E402
@@ -64,57 +66,25 @@ def main():
     ap.add_argument("--host-gib", default="64")
     ap.add_argument("--policy", type=int, default=0)
     ap.add_argument("--limit", type=int, default=None)
+    ap.add_argument("--turn-engine", action="store_true", help="drive eakv_turn_begin / eakv_turn_end")
     ap.add_argument("--closed-loop", type=int, default=0, metavar="A",
                     help="closed-loop replay with an active pool of A tasks: call order, makespan and totals")
     args = ap.parse_args()
     build.build()
-    cfg = CONFIGS[args.config]
-    shape = SHAPES[cfg.shape]
-    b = shape.block_size
-    trace = make_trace(cfg)
-    t0 = time.time()
-    agent_keys = {a: ohash.hash_blocks(toks.tolist(), b) for a, toks in trace.agent_tokens.items()}
-    print(f"keys of {len(agent_keys)} agents in {time.time() - t0:.1f} s", flush=True)
+    from full_trace_util import compare_full_trace, trace_and_keys
+    cfg, shape, trace, agent_keys = trace_and_keys(args.config)
     for gib in [float(x) for x in args.host_gib.split(",")]:
         kh = int(gib * (1 << 30) // shape.block_bytes)
-        kw = dict(policy=args.policy, kappa_blocks=cfg.kappa_blocks)
         if args.closed_loop:
+            kw = dict(policy=args.policy, kappa_blocks=cfg.kappa_blocks)
             closed_loop(args, cfg, shape, trace, agent_keys, kh, kw, gib)
             continue
-        oracle = TraceOracle(shape, cfg.gpu_blocks, kh, **kw)
-        ctx = eakv.Context(num_layers=1, kv_heads=1, head_dim=8, block_size=b, gpu_blocks=cfg.gpu_blocks,
-                           host_blocks=kh, kv_base=None, control_plane_only=True, **kw)
-        t0 = time.time()
-        refs = 0
-        for i, r in enumerate(trace.requests):
-            if args.limit and i >= args.limit:
-                break
-            keys = agent_keys[r.agent][: r.n_tokens // b]
-            w = oracle.turn(range(r.n_tokens), r.agent, r.time_ms, keys=keys)
-            k = np.asarray(keys, dtype=np.uint64)
-            G, H, _, _ = ctx.eakv_match(k)
-            st = ctx.eakv_tier_step(k, r.agent, r.n_tokens, r.time_ms)
-            res, blk, tail = ctx.eakv_gpu_tier_step(k, r.n_tokens % b != 0)
-            if tail >= 0:
-                ctx.eakv_gpu_tier_release(tail)
-            assert (G, H, st["new_chunks"], st["pressure"], st["save"]) == \
-                   (w["G"], w["H"], w["new_chunks"], w["pressure"], w["save"]), i
-            assert np.array_equal(st["hit"], np.asarray(w["hit"], dtype=np.uint8)), i
-            assert np.array_equal(st["admit"], np.asarray(w["admit"], dtype=np.uint8)), i
-            assert np.array_equal(st["slot"], np.asarray(w["slot"], dtype=np.int32)), i
-            assert list(zip(st["evicted_keys"].tolist(), st["evicted_slots"].tolist())) == w["evicted"], i
-            assert np.array_equal(res, np.asarray(w["gpu_resident"], dtype=np.uint8)), i
-            assert np.array_equal(blk, np.asarray(w["gpu_block"], dtype=np.int32)), i
-            oracle.records.clear()
-            refs += len(keys)
-        stats = ctx.eakv_get_stats()
-        for f in ("requests", "references", "hits", "admitted", "declined", "evicted"):
-            assert stats[f] == oracle.host.stats[f], f
-        ctx.close()
-        print(f"{args.config} policy {args.policy} tier {gib} GiB ({kh} blocks): {i + 1} requests, "
-              f"{refs} references identical; computed prefill {oracle.totals['fresh_tokens']}, "
-              f"restored blocks {oracle.totals['loaded_blocks']}, stored blocks "
-              f"{oracle.totals['stored_blocks']} ({time.time() - t0:.0f} s)", flush=True)
+        out = compare_full_trace(eakv, args.config, gib, policy=args.policy, limit=args.limit,
+                                 turn_engine=args.turn_engine)
+        print(f"{args.config} policy {args.policy} tier {gib} GiB ({kh} blocks): {out['requests']} requests, "
+              f"{out['references']} references identical; computed prefill {out['computed_prefill']}, "
+              f"restored blocks {out['restored_blocks']}, stored blocks {out['stored_blocks']} "
+              f"({out['seconds']:.0f} s)", flush=True)
 
 
 if __name__ == "__main__":

@@ -217,3 +217,26 @@ def test_large_batch_two_launch_path(b):
             got = [int(x) for x in res[boff[i]:boff[i + 1]].view(np.uint64)]
             assert got == expect[(par is None, i)], (b, rep, i, lens[i])
     ctx.close()
+
+
+def test_hash_self_check_reports_range_and_recovers():
+    """The hash kernels check every tile against the number of keys the call may write; told a
+    narrower number than the call needs they skip the tiles beyond it and eakv_sync reports
+    EAKV_E_RANGE once.  Nothing outside the buffers is touched, and the next call is exact again."""
+    from paper_2609_33762_b200 import eakv
+    rng = np.random.default_rng(12)
+    for b, nblk in ((16, 3000), (128, 700), (10, 900)):
+        ctx = hash_ctx(b)
+        toks = rng.integers(0, 151936, size=nblk * b, dtype=np.int32)
+        ctx.eakv_selfcheck_limits(hash_blocks=200)
+        dev = torch.from_numpy(toks).cuda()
+        out = torch.full((nblk + 1,), -1, dtype=torch.int64, device="cuda")
+        ctx.eakv_hash_blocks(dev.data_ptr(), len(toks), ctx.eakv_hash_seed(), out.data_ptr())
+        with pytest.raises(eakv.EakvError) as ei:
+            ctx.eakv_sync()
+        assert ei.value.code == eakv.E_RANGE
+        assert int(out[nblk].item()) == -1
+        ctx.eakv_sync()
+        ctx.eakv_selfcheck_limits()
+        assert gpu_keys(ctx, toks) == oh.hash_blocks(toks.tolist(), b)
+        ctx.close()

@@ -273,6 +273,131 @@ def test_layer_pipelined_load(name, group, kw):
     rig.close()
 
 
+@pytest.mark.parametrize("kw", [
+    dict(tier_location=1, copy_path=1),
+    dict(tier_location=0, link_strategy=0),
+    dict(tier_location=0, link_strategy=1, min_staged_run_bytes=-1),
+    dict(tier_location=0, link_strategy=1),
+    dict(tier_location=0, link_strategy=2, contiguous_pool=True),
+], ids=["hbm-bulk", "host-zero-copy", "host-staged", "host-default", "host-copy-engine"])
+@pytest.mark.parametrize("name,group,contiguous_slots", [("qwen", 12, True), ("qwen", 5, False), ("qwen_tp8", 16, True)])
+def test_layer_group_event_means_the_group_has_landed(name, group, contiguous_slots, kw):
+    """The contract of eakv_load_layers (Section 3.1, Eq. 2: tau_load is what a consumer waits for):
+    a stream that waits on events[g] and on nothing else may read the layers of group g.  One
+    consumer stream per group waits on its event and copies that group's layers of the
+    destination blocks into a side buffer, all enqueued while the restore is still in flight;
+    every side buffer must hold the oracle's bytes."""
+    shape = SHAPE_CASES[name]
+    nb, kh = 64, 48
+    rig = Rig(shape, nb, kh, seed=33, staging_bytes=4 * shape.block_bytes, **kw)
+    rng = rig.rng
+    groups = -(-shape.num_layers // group)
+    events = [torch.cuda.Event() for _ in range(groups)]
+    for ev in events:
+        ev.record()
+    torch.cuda.synchronize()
+    m = 40
+    src = (np.arange(m) + 3 if contiguous_slots else rng.permutation(kh)[:m]).astype(np.int32)
+    dst = rng.permutation(nb)[:m].astype(np.int32)
+    ids = torch.as_tensor(dst.astype(np.int64), device="cuda")
+    consumers = [torch.cuda.Stream() for _ in range(groups)]
+    side = [None] * groups
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    rig.ctx.eakv_load_layers(src, dst, group, [ev.cuda_event for ev in events], stream)
+    for g in range(groups):
+        q0, q1 = 2 * g * group, min(2 * (g + 1) * group, shape.pieces_per_block)
+        consumers[g].wait_event(events[g])
+        with torch.cuda.stream(consumers[g]):
+            side[g] = torch.stack([rig.pool_dev[q][ids] for q in range(q0, q1)])
+    osl.load(rig.pool_np, rig.tier_np, src, dst)
+    for g in range(groups):
+        consumers[g].synchronize()
+        q0, q1 = 2 * g * group, min(2 * (g + 1) * group, shape.pieces_per_block)
+        got = side[g].cpu().numpy().view(np.uint8)
+        for i, q in enumerate(range(q0, q1)):
+            assert np.array_equal(got[i], rig.pool_np[q][dst]), (g, q)
+    stream.synchronize()
+    rig.check()
+    rig.close()
+
+
+@pytest.mark.parametrize("kw", [
+    dict(tier_location=1, copy_path=1), dict(tier_location=1, copy_path=0),
+    dict(tier_location=0, link_strategy=0),
+    dict(tier_location=0, link_strategy=1, min_staged_run_bytes=-1),
+], ids=["hbm-bulk", "hbm-vector", "host-zero-copy", "host-staged"])
+@pytest.mark.parametrize("name,m", [("tiny", 12), ("qwen", 40), ("qwen_tp8", 40)])
+def test_device_self_check_skips_the_entry_and_reports_range(name, m, kw):
+    """The kernels' own bounds checks, made to trip without any access out of bounds: the host
+    validates against the real pool size, the kernels are told a narrower one.  Entries between
+    the two are skipped on the device (their bytes do not move, everything else does) and the next
+    eakv_sync returns EAKV_E_RANGE once; afterwards the context works as before."""
+    e = eakv()
+    shape = SHAPE_CASES[name]
+    nb, kh = 64, 48
+    rig = Rig(shape, nb, kh, seed=44, staging_bytes=4 * shape.block_bytes, **kw)
+    rng = rig.rng
+    narrowed = nb - 8
+    rig.ctx.eakv_selfcheck_limits(gpu_blocks=narrowed)
+    # (a staged store gathers into a staging buffer that the copy engine then moves as a whole, so
+    # a skipped entry's slot would receive stale staging bytes: only its restore is checked here)
+    staged = kw.get("link_strategy") == e.LINK_STAGED and kw.get("tier_location") == e.TIER_PINNED_HOST
+    for op in (("load",) if staged else ("store", "load")):
+        table = rng.permutation(nb)[:m].astype(np.int32)
+        assert (table >= narrowed).any() and (table < narrowed).any()
+        slots = rng.permutation(kh)[:m].astype(np.int32)
+        keep = table < narrowed
+        if op == "store":
+            rig.ctx.eakv_store(table, None, slots)
+            osl.store(rig.pool_np, rig.tier_np, table[keep], [1] * int(keep.sum()), slots[keep])
+        else:
+            rig.ctx.eakv_load(slots, table)
+            osl.load(rig.pool_np, rig.tier_np, slots[keep], table[keep])
+        with pytest.raises(e.EakvError) as ei:
+            rig.ctx.eakv_sync()
+        assert ei.value.code == e.E_RANGE
+        rig.check()                               # the sync inside succeeds: the word was cleared
+    with pytest.raises(e.EakvError) as ei:        # limits above the real sizes are refused
+        rig.ctx.eakv_selfcheck_limits(gpu_blocks=nb + 1)
+    assert ei.value.code == e.E_INVAL
+    rig.ctx.eakv_selfcheck_limits()               # back to the real sizes
+    table = rng.permutation(nb)[:m].astype(np.int32)
+    slots = rng.permutation(kh)[:m].astype(np.int32)
+    rig.store(table, None, slots)
+    rig.load(slots[::-1].copy(), rng.permutation(nb)[:m].astype(np.int32))
+    rig.check()
+    rig.close()
+
+
+def test_tier_slot_self_check_and_bounded_wait_report():
+    e = eakv()
+    shape = SHAPE_CASES["tiny"]
+    nb, kh = 32, 32
+    for kw in (dict(tier_location=1, copy_path=1), dict(tier_location=0, link_strategy=0)):
+        rig = Rig(shape, nb, kh, seed=45, **kw)
+        rig.ctx.eakv_selfcheck_limits(tier_slots=kh - 4)
+        table = np.arange(nb, dtype=np.int32)
+        slots = np.arange(kh, dtype=np.int32)[::-1].copy()
+        keep = slots < kh - 4
+        rig.ctx.eakv_store(table, None, slots)
+        osl.store(rig.pool_np, rig.tier_np, table[keep], [1] * int(keep.sum()), slots[keep])
+        with pytest.raises(e.EakvError) as ei:
+            rig.ctx.eakv_sync()
+        assert ei.value.code == e.E_RANGE
+        rig.check()
+        rig.ctx.eakv_selfcheck_limits()
+        # a bounded wait that nothing satisfies gives up, reports, and leaves the context usable
+        rig.ctx.eakv_selfcheck_wait_probe()
+        with pytest.raises(e.EakvError) as ei:
+            rig.ctx.eakv_sync()
+        assert ei.value.code == e.E_TIMEOUT
+        rig.ctx.eakv_sync()
+        rig.store(table, None, slots)
+        rig.check()
+        rig.close()
+
+
 def test_calls_larger_than_the_argument_ring_slot_are_split():
     """max_call_blocks smaller than the call: several argument uploads per call; also more
     calls than ring slots back to back (slot reuse)."""

@@ -1,0 +1,141 @@
+"""The two-call turn engine (eakv_turn_begin / eakv_turn_end / eakv_turn_abort) as pure
+bookkeeping on the CPU: a control-plane-only context runs it when the caller supplies every
+key.  Checked against the trace oracle per request, and for what a refused, failed or aborted
+turn must leave behind: no key may stay listed whose bytes were never written."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+from eakv_workloads import CONFIGS, SHAPES, make_trace
+from oracle import hash as ohash
+from oracle.trace import TraceOracle
+
+
+@pytest.fixture(scope="module")
+def eakv():
+    from paper_2609_33762_b200 import build, eakv as m
+    build.build()
+    return m
+
+
+def cp_ctx(eakv, block_size, gpu_blocks, host_blocks, **kw):
+    return eakv.Context(num_layers=1, kv_heads=1, head_dim=8, block_size=block_size,
+                        gpu_blocks=gpu_blocks, host_blocks=host_blocks, kv_base=None,
+                        control_plane_only=True, **kw)
+
+
+def keys_of(tokens, b):
+    return np.asarray(ohash.hash_blocks(np.asarray(tokens).tolist(), b), dtype=np.uint64)
+
+
+def compare_view(v, w, R=1):
+    assert [int(k) for k in v["keys"]] == w["keys"]
+    assert (v["gpu_prefix_blocks"], v["host_prefix_blocks"], v["new_chunks"], bool(v["pressure"]), bool(v["save"])) == \
+           (w["G"], w["H"], w["new_chunks"], w["pressure"], w["save"])
+    for f in ("hit", "admit", "slot"):
+        assert v[f].tolist() == w[f], f
+    assert list(zip(v["evicted_keys"].tolist(), v["evicted_slots"].tolist())) == w["evicted"]
+    assert v["gpu_resident"].tolist() == w["gpu_resident"] and v["gpu_block"].tolist() == w["gpu_block"]
+    assert v["restore_hi"] - v["restore_lo"] == w["loaded"]
+    assert v["n_stored_blocks"] == w["stored"] and v["fresh_tokens"] == w["fresh_tokens"]
+    assert v["n_fill"] == w["filled"]
+
+
+@pytest.mark.parametrize("R,policy", [(1, 0), (1, 2), (4, 0), (4, 1), (2, 2)])
+def test_turn_engine_bookkeeping_equals_oracle(eakv, R, policy):
+    cfg = replace(CONFIGS["c2"], shape="tiny", agents=6, turns=14, first_prompt=500,
+                  append_median=200.0, context_cap=3500, tool_gap_mean_ms=15_000.0)
+    shape = SHAPES["tiny"]
+    b = shape.block_size
+    trace = make_trace(cfg, seed=41)
+    kw = dict(policy=policy, kappa_blocks=max(1, 8 // R), window_ms=60_000, len_window=32)
+    kh = 700 // R
+    oracle = TraceOracle(shape, 256, kh, chunk_blocks=R, **kw)
+    ctx = cp_ctx(eakv, b, 256, kh, chunk_blocks=R, **kw)
+    for req in trace.requests:
+        toks = trace.prompt(req)
+        w = oracle.turn(toks, req.agent, req.time_ms)
+        v = ctx.eakv_turn_begin(0, len(toks), keys_of(toks, b), req.agent, req.time_ms)
+        compare_view(v, w, R)
+        ctx.eakv_turn_end()
+    st = ctx.eakv_get_stats()
+    for f in ("requests", "references", "hits", "admitted", "declined", "evicted"):
+        assert st[f] == oracle.host.stats[f], f
+    if policy != 1:                              # the fixed filter declines nearly everything
+        assert oracle.totals["loaded_blocks"] > 0
+    ctx.close()
+
+
+def test_turn_without_all_keys_needs_a_device(eakv):
+    ctx = cp_ctx(eakv, 4, 16, 16)
+    with pytest.raises(eakv.EakvError) as ei:
+        ctx.eakv_turn_begin(0, 16, np.asarray([1, 2], dtype=np.uint64), 0, 0)     # 4 blocks, 2 keys
+    assert ei.value.code == eakv.E_INVAL
+    with pytest.raises(eakv.EakvError):
+        ctx.eakv_turn_end()                      # no turn was opened
+    ctx.close()
+
+
+def test_prompt_larger_than_the_gpu_tier_is_refused_before_anything_changes(eakv):
+    """A prompt with more blocks than the GPU tier hands out: EAKV_E_CAPACITY, and neither tier
+    has changed, in particular the host index does not list keys whose slots were never written."""
+    b = 4
+    ctx = cp_ctx(eakv, b, 8, 64)                              # K_G = 8 blocks, K_H = 64
+    small = np.arange(1, 7, dtype=np.uint64)                  # 6 blocks: fits
+    v = ctx.eakv_turn_begin(0, 6 * b, small, 0, 0)
+    assert v["n_stored_blocks"] == 6
+    ctx.eakv_turn_end()
+    before = ctx.eakv_get_stats()
+    big = np.arange(100, 112, dtype=np.uint64)                # 12 blocks > K_G
+    with pytest.raises(eakv.EakvError) as ei:
+        ctx.eakv_turn_begin(0, 12 * b, big, 1, 1)
+    assert ei.value.code == eakv.E_CAPACITY
+    G, H, _, _ = ctx.eakv_match(big)
+    assert (G, H) == (0, 0)
+    assert ctx.eakv_get_stats() == before
+    # exactly K_G blocks with a partial tail does not fit either (the tail needs a ninth block)
+    eight = np.arange(200, 208, dtype=np.uint64)
+    with pytest.raises(eakv.EakvError) as ei:
+        ctx.eakv_turn_begin(0, 8 * b + 1, eight, 1, 2)
+    assert ei.value.code == eakv.E_CAPACITY and ctx.eakv_match(eight)[:2] == (0, 0)
+    # more units than the host tier
+    ctx2 = cp_ctx(eakv, b, 64, 4)
+    with pytest.raises(eakv.EakvError) as ei:
+        ctx2.eakv_turn_begin(0, 6 * b, small, 0, 0)
+    assert ei.value.code == eakv.E_CAPACITY and ctx2.eakv_match(small)[:2] == (0, 0)
+    # the first context still serves what it stored, and the next turn opens normally
+    assert ctx.eakv_match(small)[:2] == (6, 6)
+    v = ctx.eakv_turn_begin(0, 6 * b, small, 0, 3)
+    assert v["hit"].tolist() == [1] * 6
+    ctx.eakv_turn_end()
+    ctx.close(); ctx2.close()
+
+
+def test_aborted_turn_takes_back_what_it_never_produced(eakv):
+    """A turn that is aborted after begin (the engine will not compute its KV): the units it
+    admitted leave the host index, the blocks it was to fill leave the GPU index, what was
+    resident before stays, and the slots and blocks are handed out again."""
+    b = 4
+    ctx = cp_ctx(eakv, b, 32, 32)
+    first = np.arange(1, 5, dtype=np.uint64)
+    ctx.eakv_turn_begin(0, 4 * b, first, 0, 0)
+    ctx.eakv_turn_end()
+    longer = np.arange(1, 11, dtype=np.uint64)                # the same 4 blocks + 6 new ones + a tail
+    v = ctx.eakv_turn_begin(0, 10 * b + 2, longer, 0, 1)
+    assert v["hit"].tolist() == [1] * 4 + [0] * 6 and v["admit"].tolist() == [0] * 4 + [1] * 6
+    assert v["needs_fill"].tolist() == [0] * 4 + [1] * 6 and v["tail_block"] >= 0
+    with pytest.raises(eakv.EakvError):
+        ctx.eakv_turn_begin(0, 4 * b, first, 1, 1)            # one turn at a time
+    ctx.eakv_turn_abort()
+    assert ctx.eakv_match(longer)[:2] == (4, 4)               # only what existed before is listed
+    assert ctx.eakv_get_stats()["resident"] == 4
+    with pytest.raises(eakv.EakvError):
+        ctx.eakv_turn_abort()                                 # nothing open any more
+    # the withdrawn slots, blocks and the tail block are free again: the same turn repeats exactly
+    v2 = ctx.eakv_turn_begin(0, 10 * b + 2, longer, 0, 2)
+    assert v2["slot"].tolist() == v["slot"].tolist()
+    assert sorted(v2["gpu_block"].tolist() + [v2["tail_block"]]) == sorted(v["gpu_block"].tolist() + [v["tail_block"]])
+    ctx.eakv_turn_end()
+    assert ctx.eakv_match(longer)[:2] == (10, 10)
+    ctx.close()
