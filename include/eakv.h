@@ -61,8 +61,11 @@ extern "C" {
 #define EAKV_LINK_COPY_ENGINE 2 /* no kernel at all: one strided copy-engine transfer per block (rows =
                                    the block's pieces, pitch = the distance between piece arrays), issued on
                                    the caller's stream.  Needs the 2L piece arrays to sit at one constant
-                                   pitch (one [2L][gpu_blocks][piece] allocation); eakv_create returns
-                                   EAKV_E_INVAL otherwise.  Uses no SM while the engine's own kernels run */
+                                   pitch (one [2L][gpu_blocks][piece] allocation) that, like the bytes of
+                                   one block, does not exceed the device's largest copy pitch
+                                   (cudaDevAttrMaxPitch, 2 GiB - 1 on current parts: for instance at most
+                                   131,071 blocks of 16-KiB pieces); eakv_create returns EAKV_E_INVAL
+                                   otherwise.  Uses no SM while the engine's own kernels run */
 
 /* where the tier lives */
 #define EAKV_TIER_PINNED_HOST 0 /* the product configuration                                   */

@@ -319,16 +319,18 @@ cudaError_t launch_wait_probe(int* error_flag, cudaStream_t stream) {
 // the small-piece geometry gives 6,379); pieces of 8 KiB and less want more issuing threads
 // and about 128 KiB in flight per SM: 2 stages x 8 KiB x 8 CTAs per SM (8 KiB pieces 6,378
 // against 6,175; 4 KiB pieces 6,213 against 5,730).  For the large pieces deeper rings or more
-// CTAs per SM lose 5-6 %.  The EAKV_TUNE_BULK_* environment variables override both for sweeps.
+// CTAs per SM lose 5-6 %.  (A build with -DEAKV_TUNING reads EAKV_TUNE_BULK_* from the environment for sweeps.)
 struct BulkGeometry { int stages, stage_bytes, ctas_per_sm_cap, ctas_per_sm; };
 static BulkGeometry g_bulk_geo[2] = {{3, kCopySubBytes, 2, 0}, {2, 8192, 8, 0}};
 static bool g_bulk_ready = false;
 
 static cudaError_t bulk_setup() {
     for (BulkGeometry& g : g_bulk_geo) {
+#ifdef EAKV_TUNING   // sweep builds only: the shipped library's geometry does not depend on the environment
         if (const char* e = getenv("EAKV_TUNE_BULK_STAGES")) g.stages = atoi(e);
         if (const char* e = getenv("EAKV_TUNE_BULK_STAGE_BYTES")) g.stage_bytes = atoi(e);
         if (const char* e = getenv("EAKV_TUNE_BULK_CTAS_PER_SM")) g.ctas_per_sm_cap = atoi(e);
+#endif
         if (g.stages < 2) g.stages = 2;
         if (g.stages > kBulkMaxStages) g.stages = kBulkMaxStages;
         if (g.stage_bytes < 1024 || (g.stage_bytes & 15)) g.stage_bytes = kCopySubBytes;
@@ -354,7 +356,8 @@ static cudaError_t bulk_setup() {
     return cudaSuccess;
 }
 
-cudaError_t launch_copy_bulk(const CopyLaunch& L_in, bool to_tier, int ctas, cudaStream_t stream) {
+// ctas > 0: the caller's explicit grid, used as given; 0: sm_count x this geometry's CTAs per SM
+cudaError_t launch_copy_bulk(const CopyLaunch& L_in, bool to_tier, int ctas, int sm_count, cudaStream_t stream) {
     if (L_in.n_entries <= 0) return cudaSuccess;
     if (!g_bulk_ready) {
         cudaError_t e = bulk_setup();
@@ -372,10 +375,7 @@ cudaError_t launch_copy_bulk(const CopyLaunch& L_in, bool to_tier, int ctas, cud
         if (g > L.pieces) g = L.pieces;
         L.group_pieces = (int32_t)g;
     }
-    // the auto grid of the vector path assumes its occupancy; rescale to this kernel's
-    const int per_sm_vec = copy_vector_ctas_per_sm();
-    if (per_sm_vec > 0 && ctas % per_sm_vec == 0 && ctas / per_sm_vec >= 100)
-        ctas = ctas / per_sm_vec * geo.ctas_per_sm;
+    if (ctas <= 0) ctas = sm_count * geo.ctas_per_sm;
     const int64_t n_items = L.group_pieces > 1
         ? L.n_entries * ((L.pieces + L.group_pieces - 1) / L.group_pieces)
         : L.n_entries * L.pieces * L.subs_per_piece;

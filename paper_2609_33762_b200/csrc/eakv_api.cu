@@ -190,7 +190,8 @@ void free_all(eakv_ctx* c) {
     delete c;
 }
 
-int copy_ctas(const eakv_ctx* ctx, bool touches_host) {
+// grid of the vector kernel: the configured one, else sized here
+int vector_ctas(const eakv_ctx* ctx, bool touches_host) {
     if (ctx->cfg.copy_ctas > 0) return ctx->cfg.copy_ctas;
     // A few SMs saturate the host link and the rest stay with the engine.  Measured with restores
     // and writes running at once (zero-copy, 6 GiB each way): 16 CTAs 49.5 GB/s, 32: 63.7, 64: 74.1,
@@ -226,9 +227,9 @@ int launch_copy(eakv_ctx* ctx, const int2* d_entries, const int2* h_inline, int6
     // bulk async copies serve device-resident buffers; a mapped host tier is always driven
     // by the vector kernel (few CTAs, plain loads/stores over the link)
     if (ctx->cfg.copy_path == EAKV_COPY_BULK && !touches_host)
-        e = launch_copy_bulk(L, to_tier, copy_ctas(ctx, touches_host), stream);
+        e = launch_copy_bulk(L, to_tier, ctx->cfg.copy_ctas > 0 ? ctx->cfg.copy_ctas : 0, ctx->sm_count, stream);
     else
-        e = launch_copy_vector(L, to_tier, copy_ctas(ctx, touches_host), stream);
+        e = launch_copy_vector(L, to_tier, vector_ctas(ctx, touches_host), stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "copy kernel launch");
     ctx->stats.kernel_launches += 1;
     return EAKV_OK;
@@ -472,6 +473,20 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
     if (cfg->link_strategy == EAKV_LINK_COPY_ENGINE && (cfg->control_plane_only || ctx->pool_pitch == 0)) {
         delete ctx;
         return EAKV_E_INVAL;
+    }
+    if (cfg->link_strategy == EAKV_LINK_COPY_ENGINE) {
+        // a strided copy-engine transfer takes no pitch above the device's limit (cudaDevAttrMaxPitch)
+        int dev = 0, max_pitch = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&max_pitch, cudaDevAttrMaxPitch, dev) != cudaSuccess) {
+            cudaGetLastError();
+            delete ctx;
+            return EAKV_E_CUDA;
+        }
+        if (ctx->pool_pitch > (int64_t)max_pitch || piece * pieces > (int64_t)max_pitch) {
+            delete ctx;
+            return EAKV_E_INVAL;
+        }
     }
     std::memset(&ctx->stats, 0, sizeof(ctx->stats));
     ctx->pieces = pieces;

@@ -54,10 +54,12 @@ inline bool hash_thread_per_block(int block_size) { return (block_size % 4) != 0
 // blocks per CTA tile; large batches get longer tiles so fewer CTAs take tickets
 inline int hash_tile_blocks(int block_size, int64_t total_blocks) {
     if (hash_thread_per_block(block_size)) {
-        if (const char* e = getenv("EAKV_TUNE_HASH_TILE")) {   // developer override for sweeps
+#ifdef EAKV_TUNING
+        if (const char* e = getenv("EAKV_TUNE_HASH_TILE")) {   // sweep builds only
             const int v = atoi(e);
             if (v >= 1) return v;
         }
+#endif
         int t = kHashThreads;
         while (t < 16 * kHashThreads && total_blocks / t > 1184) t *= 2;   // up to a whole 64k-token prompt per CTA
         return t;
@@ -82,12 +84,16 @@ inline void hash_fill_limbs(HashLaunch& L, const uint64_t* pow_host, int block_s
 // Sub-tiles in flight per warp in the staged kernel.  Two is the measured optimum: three and
 // four (more shared memory, fewer CTAs per SM) were 3-10 % slower.
 inline int hash_stages(int block_size) {
-    if (const char* e = getenv("EAKV_TUNE_HASH_STAGES")) {      // developer override for sweeps
+#ifdef EAKV_TUNING
+    if (const char* e = getenv("EAKV_TUNE_HASH_STAGES")) {      // sweep builds only
         const int v = atoi(e);
         if (v >= 1 && v <= 4 && (size_t)v * kHashThreads * (4 * block_size + 16) <= 136 * 1024) return v;
     }
+#endif
+    (void)block_size;
     return 2;
 }
+// also records the current device's SM count for the launch heuristics
 cudaError_t hash_kernels_init();
 // *launches_out (optional) receives the number of kernels launched: one, or two for large batches
 cudaError_t launch_hash(const HashLaunch& L, int n_tiles, bool thread_per_block, bool vec,
@@ -124,7 +130,7 @@ struct CopyLaunch {
 constexpr int kErrBulkTimeout = 1, kErrCopyRange = 2, kErrHashRange = 3;
 // to_tier: pool -> tier (store/gather); else tier -> pool (load/scatter)
 cudaError_t launch_copy_vector(const CopyLaunch& L, bool to_tier, int ctas, cudaStream_t stream);
-cudaError_t launch_copy_bulk(const CopyLaunch& L, bool to_tier, int ctas, cudaStream_t stream);
+cudaError_t launch_copy_bulk(const CopyLaunch& L, bool to_tier, int ctas, int sm_count, cudaStream_t stream);
 // pull `bytes` (rounded up to 16) of per-call arguments from mapped pinned memory into device memory
 cudaError_t launch_fetch_args(void* dst_dev, const void* src_host_mapped, size_t bytes,
                               cudaStream_t stream);

@@ -780,6 +780,8 @@ hash_scan_runs_kernel(const __grid_constant__ HashLaunch L) {
 
 #undef EAKV_MACP
 
+static int g_hash_sm_count = 148;      // replaced by the device's own count in hash_kernels_init
+
 cudaError_t launch_hash(const HashLaunch& L_in, int n_tiles, bool thread_per_block, bool vec,
                         cudaStream_t stream, int* launches_out) {
     if (launches_out) *launches_out = n_tiles > 0 ? 1 : 0;
@@ -792,12 +794,15 @@ cudaError_t launch_hash(const HashLaunch& L_in, int n_tiles, bool thread_per_blo
         // Many prompts of a block size known at compile time: two launches, the token phase
         // (a lane per run of consecutive blocks) and the per-prompt scan.  Neither needs a fence
         // or a ticket, and the scan's registers do not limit the token phase's occupancy.
-        // (EAKV_TUNE_HASH_KERNEL=staged keeps the single-launch kernel, for A/B runs.)
+#ifdef EAKV_TUNING   // EAKV_TUNE_HASH_KERNEL=staged keeps the single-launch kernel, for A/B runs
         static const bool use_run = [] {
             const char* e = getenv("EAKV_TUNE_HASH_KERNEL");
             return !(e && e[0] == 's');
         }();
-        if (run_shape && use_run && L.tiles != nullptr && L.n_prompts > 0 && n_tiles >= 2 * 148) {
+#else
+        constexpr bool use_run = true;
+#endif
+        if (run_shape && use_run && L.tiles != nullptr && L.n_prompts > 0 && n_tiles >= 2 * g_hash_sm_count) {
             const size_t rs = L.stages == 2 ? kRunSmem : kRunSmem / 2;
             if (L.block_size == 16)      hash_blocks_run_kernel<16><<<n_tiles, kRunThreads, rs, stream>>>(L);
             else if (L.block_size == 32) hash_blocks_run_kernel<32><<<n_tiles, kRunThreads, rs, stream>>>(L);
@@ -827,8 +832,14 @@ cudaError_t launch_hash(const HashLaunch& L_in, int n_tiles, bool thread_per_blo
 }
 
 cudaError_t hash_kernels_init() {
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    if (sms > 0) g_hash_sm_count = sms;
     // allow tiles whose chunk sums plus a large power table exceed the 48 KB default
-    cudaError_t e = cudaFuncSetAttribute(hash_blocks_kernel<true>,
+    e = cudaFuncSetAttribute(hash_blocks_kernel<true>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kHashMaxSmem);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(hash_blocks_kernel<false>,

@@ -357,7 +357,9 @@ extern "C" int eakv_capacity_curve(const int64_t* dist_dev, int64_t n_refs,
     SD_CU(cudaMemcpyAsync(d_caps, capacities_host, C * 8, cudaMemcpyHostToDevice, stream));
     SD_CU(cudaMemsetAsync(d_out, 0, 3 * C * 8, stream));
     if (n_refs > 0) {
-        const int grid = (int)std::min<int64_t>((n_refs + 255) / 256, 148 * 8);
+        int dev = 0, sms = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const int grid = (int)std::min<int64_t>((n_refs + 255) / 256, (int64_t)sms * 8);
         curve_hits_kernel<<<grid, 256, C * 8, stream>>>(dist_dev, n_refs, d_caps, C, d_out);
     }
     if (n_requests > 0) {

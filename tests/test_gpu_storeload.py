@@ -219,6 +219,17 @@ def test_bad_shapes_rejected_at_create():
         with pytest.raises(e.EakvError) as ei:
             e.Context(**{**base, **patch})
         assert ei.value.code == e.E_INVAL
+    # Copy engine alone: the pitch between piece arrays (2 GiB here: 131,072 blocks of 16 KiB) is
+    # above what a strided copy-engine transfer accepts, so the configuration is refused at create
+    # rather than failing on every later call.  The pool addresses are only compared, never
+    # dereferenced: create returns before anything is allocated or copied.
+    piece = 16 * 4 * 128 * 2
+    pitch = 131072 * piece
+    fake = [t.data_ptr() + q * pitch for q in range(4)]
+    with pytest.raises(e.EakvError) as ei:
+        e.Context(num_layers=2, kv_heads=4, head_dim=128, block_size=16, gpu_blocks=131072, host_blocks=1,
+                  kv_base=fake, link_strategy=e.LINK_COPY_ENGINE)
+    assert ei.value.code == e.E_INVAL
 
 
 @pytest.mark.parametrize("kw", [
