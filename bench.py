@@ -150,22 +150,27 @@ class ClockSampler:
 class Arm:
     """One configuration of the path (device tier or pinned-host tier) over a shared pool."""
 
-    def __init__(self, args, pool, shape, torch, eakv, *, host_tier, device):
+    def __init__(self, args, pool, shape, torch, eakv, *, host_tier, device, link=None, copy_path=None,
+                 tier_memory=None):
         self.torch, self.eakv = torch, eakv
+        link = link or args.link
+        copy_path = copy_path or args.copy_path
         self.m = args.blocks
         self.b = shape.block_size
         self.n_tokens = self.m * self.b
         self.host_tier = host_tier
         self.device = device
-        kw = dict(copy_path=eakv.COPY_BULK if args.copy_path == "bulk" else eakv.COPY_VECTOR,
+        kw = dict(copy_path=eakv.COPY_BULK if copy_path == "bulk" else eakv.COPY_VECTOR,
                   max_call_blocks=max(16384, self.m))
         if host_tier:
             kw.update(tier_location=eakv.TIER_PINNED_HOST,
                       link_strategy={"staged": eakv.LINK_STAGED, "zero_copy": eakv.LINK_ZERO_COPY,
-                                     "copy_engine": eakv.LINK_COPY_ENGINE}[args.link],
+                                     "copy_engine": eakv.LINK_COPY_ENGINE}[link],
                       staging_bytes=args.staging_mib << 20, copy_ctas=args.host_ctas)
-            if args.link == "staged":
+            if link == "staged":
                 kw["copy_ctas"] = args.copy_ctas
+            if tier_memory is not None:
+                kw["tier_memory"] = tier_memory
         else:
             # the tier is a tensor of ours that the context adopts, so it can be inspected
             self.tier_t = torch.empty((TIER_PROMPTS * self.m, shape.pieces_per_block, shape.piece_bytes // 2),
@@ -399,12 +404,6 @@ def hash_throughput(torch, eakv, pool, shape, device, peak_gbs, prompts=512, tok
     ctx.close()
     rate = prompts * tokens / (best * 1e-3)
     srate = prompts * tokens / (sustained * 1e-3)
-    # multiply-pipe ceiling from stand-alone measurements on this GPU type: 31.5 wide (32x32->64)
-    # multiply-adds and 2.3 modular 61-bit products per SM per clock; 3 of the former per token
-    # and 2.7 of the latter per block
-    props = torch.cuda.get_device_properties(device)
-    clk_hz = 1.965e9
-    alu_bound = props.multi_processor_count * clk_hz / (3 / 31.5 + 2.7 / shape.block_size / 2.3)
     return {"sustained_tokens_per_s": srate, "sustained_ms_per_launch": sustained,
             "sustained_frac_of_hbm_bound": srate * 4 / 1e9 / peak_gbs,
             "two_streams_tokens_per_s": prompts * tokens / (two_stream * 1e-3),
@@ -412,8 +411,6 @@ def hash_throughput(torch, eakv, pool, shape, device, peak_gbs, prompts=512, tok
             "batched_tokens_per_s": rate, "batch": f"{prompts} prompts x {tokens} tokens, block {shape.block_size}",
             "batched_ms": best, "frac_of_hbm_bound": rate * 4 / 1e9 / peak_gbs,
             "hbm_bound_tokens_per_s": peak_gbs * 1e9 / 4,
-            "multiply_pipe_bound_tokens_per_s": alu_bound,
-            "sustained_frac_of_multiply_pipe_bound": srate / alu_bound,
             "single_prompt_tokens": tokens, "single_prompt_us_median": float(np.median(single)),
             "single_call_us_by_tokens": latency,
             "host_resident_prompt": {"tokens": n_host, "us": host_us, "tokens_per_s": n_host / (host_us * 1e-6),
@@ -481,6 +478,62 @@ def layered_load_probe(torch, arm, tables, shape, layers_per_group=12):
     out["layers_per_group"] = layers_per_group
     out["blocks"] = m
     return out
+
+
+def store_load_curve(torch, eakv, pool, shape, device, args, h2d_peak, d2h_peak, tier_ptr=None,
+                     tier_blocks=4096, reps=5):
+    """The microbench's curve: 1 to 4,096 blocks per call, block ids contiguous or uniform-random
+    over the pool (host slots alike), admit mask all-ones or Bernoulli(0.5); GB/s of the admitted
+    bytes, median of ``reps`` calls timed with CUDA events on the launching stream.  Host tier
+    under the default strategy (staged, scattered calls go direct) and a tier in HBM."""
+    rng = np.random.default_rng(7)
+    nb, kh = pool.gpu_blocks, int(min(4096, tier_blocks))
+    rows = []
+    tier_dev = torch.empty(kh * shape.block_bytes, dtype=torch.uint8, device=device)
+    arms = [("host", dict(tier_location=eakv.TIER_PINNED_HOST, link_strategy=eakv.LINK_STAGED,
+                          staging_bytes=args.staging_mib << 20,
+                          **({"tier_memory": tier_ptr} if tier_ptr else {}))),
+            ("hbm", dict(tier_location=eakv.TIER_DEVICE, tier_memory=tier_dev.data_ptr()))]
+    stream = torch.cuda.current_stream(device)
+    for name, kw in arms:
+        ctx = eakv.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+                           block_size=shape.block_size, gpu_blocks=nb, host_blocks=kh,
+                           kv_base=pool.kv_base, **kw)
+        for m in (1, 16, 256, 4096):
+            if m > kh or m > nb:
+                continue
+            for ids in ("contiguous", "random"):
+                for mask in ("ones", "bernoulli"):
+                    for op in ("store", "load"):
+                        if op == "load" and mask != "ones":
+                            continue                      # a restore has no mask
+                        rates = []
+                        for i in range(reps + 1):
+                            start = int(rng.integers(0, nb - m + 1))
+                            table = (np.arange(start, start + m) if ids == "contiguous"
+                                     else rng.permutation(nb)[:m]).astype(np.int32)
+                            slots = (np.arange(m) if ids == "contiguous" else rng.permutation(kh)[:m]).astype(np.int32)
+                            adm = None if mask == "ones" else (rng.random(m) < 0.5).astype(np.uint8)
+                            nbytes = (m if adm is None else int(adm.sum())) * shape.block_bytes
+                            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                            e0.record(stream)
+                            if op == "store":
+                                ctx.eakv_store(table, adm, slots, stream)
+                            else:
+                                ctx.eakv_load(slots, table, stream)
+                            e1.record(stream)
+                            torch.cuda.synchronize()
+                            if nbytes and i > 0:          # the first call of a kind warms up
+                                rates.append(nbytes / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+                        if rates:
+                            row = dict(tier=name, op=op, blocks=m, ids=ids, mask=mask,
+                                       gbps=round(float(np.median(rates)), 2))
+                            if name == "host":
+                                pk = d2h_peak if op == "store" else h2d_peak
+                                row["frac_of_link"] = round(row["gbps"] / pk, 3) if pk else None
+                            rows.append(row)
+        ctx.close()
+    return {"unit": "GB/s of admitted bytes, median of %d calls" % reps, "rows": rows}
 
 
 def pinned_link_peak(torch, device, gib=1, reps=5):
@@ -788,17 +841,37 @@ def main():
     ms_max, moved_sum = aggregate_over_ranks(dist, r["ms"], r["moved"], device)
     value = moved_sum / (ms_max * 1e-3) / 1e9
 
-    kb = sum(b for b, _ in r["kernel"])
-    kms = sum(t for _, t in r["kernel"])
-    achieved = 2 * kb / (kms * 1e-3) / 1e9 if kms > 0 else 0.0
+    def kernel_rate(res):
+        kb = sum(b for b, _ in res["kernel"])
+        kms = sum(t for _, t in res["kernel"])
+        return 2 * kb / (kms * 1e-3) / 1e9 if kms > 0 else 0.0
+
+    achieved = kernel_rate(r)
     kernel_name = "copy_blocks_vector_kernel" if args.copy_path == "vector" else "copy_blocks_bulk_kernel"
+    # the other device copy path on the same step (fewer steps), so both appear side by side
+    other = "vector" if args.copy_path == "bulk" else "bulk"
+    arm_o = Arm(args, pool, shape, torch, eakv, host_tier=False, device=device, copy_path=other)
+    r_o = run_arm(arm_o, prompts_dev, tables, max(2, min(args.steps, 10)), min(args.warmup, 3), dist, None)
+    arm_o.ctx.close()
+    del arm_o
+    by_copy_path = {args.copy_path: {"achieved": achieved, "frac": achieved / peak,
+                                     "launches_timed": len(r["kernel"])},
+                    other: {"achieved": kernel_rate(r_o), "frac": kernel_rate(r_o) / peak,
+                            "launches_timed": len(r_o["kernel"])}}
     # the profile's per-block DRAM traffic was captured on the unsharded shape
     traffic = read_profile_traffic(kernel_name, m) if args.tp_shard == 1 else None
 
     # ---- end-to-end arm (pinned host tier, host tokens) ----
     def e2e_section():
         link = pinned_link_peak(torch, device) if rank == 0 else None
-        arm = Arm(args, pool, shape, torch, eakv, host_tier=True, device=device)
+        # one pinned tier shared by every strategy's context (allocating 18 GiB of pinned memory
+        # takes seconds; the contexts adopt it one after the other)
+        try:
+            tier_pin = torch.empty(TIER_PROMPTS * m * shape.block_bytes, dtype=torch.uint8, pin_memory=True)
+            tier_ptr = tier_pin.data_ptr()
+        except RuntimeError:
+            tier_pin, tier_ptr = None, None
+        arm = Arm(args, pool, shape, torch, eakv, host_tier=True, device=device, tier_memory=tier_ptr)
         e_steps = max(2, min(args.steps, 8))
         # measured twice on the same arm, the faster pass reported and both listed: the first
         # pass on a freshly started machine has been seen to run its two directions one after
@@ -817,6 +890,7 @@ def main():
                "ms_per_step": e_ms / e_steps, "link_strategy": args.link,
                "passes_gbps": [mv / (ms_ * 1e-3) / 1e9 for ms_, mv in pass_ms]}
         e2e["layered_load"] = layered
+        serial = bound = None
         if link:
             # one direction at a time: harmonic mean of the two; both at once: the measured
             # bidirectional pinned-memcpy rate
@@ -825,6 +899,24 @@ def main():
             e2e.update(host_link_peak_gbps=link, overlap=bool(args.overlap),
                        frac_of_link=e_val / bound / max(world, 1),
                        frac_of_one_direction=e_val / serial / max(world, 1))
+        # the same step under every host-link strategy, side by side (fewer steps each)
+        by = {args.link: {"value": e_val, "frac_of_link": e2e.get("frac_of_link"), "steps": e_steps}}
+        for name in ("staged", "zero_copy", "copy_engine"):
+            if name in by:
+                continue
+            a2 = Arm(args, pool, shape, torch, eakv, host_tier=True, device=device, link=name,
+                     tier_memory=tier_ptr)
+            r2 = run_arm(a2, prompts_host, tables, 3, 2, dist, None, time_kernels=False)
+            a2.ctx.close()
+            del a2
+            ms2, mv2 = aggregate_over_ranks(dist, r2["ms"], r2["moved"], device)
+            v2 = mv2 / (ms2 * 1e-3) / 1e9
+            by[name] = {"value": v2, "frac_of_link": v2 / bound / max(world, 1) if bound else None, "steps": 3}
+        e2e["by_strategy"] = by
+        if rank == 0:
+            e2e["curve"] = guarded(store_load_curve, torch, eakv, pool, shape, device, args,
+                                   link.get("h2d"), link.get("d2h"), tier_ptr, TIER_PROMPTS * m)
+        del tier_pin
         return e2e
 
     # side measurements never take the main line down with them
@@ -875,6 +967,7 @@ def main():
                          "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                          "kernel": kernel_name,
                          "launches_timed": len(r["kernel"]),
+                         "by_copy_path": by_copy_path,
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "cpu_baseline": cpu,
             "hash": hashing,

@@ -35,6 +35,14 @@ def test_bench_line_on_a_small_case():
     e = d["e2e"]
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0
     assert len(e["passes_gbps"]) == 2 and e["value"] == max(e["passes_gbps"])
+    # every host-link strategy and both device copy paths side by side, and the microbench's curve
+    assert set(e["by_strategy"]) == {"staged", "zero_copy", "copy_engine"}
+    assert all(v["value"] > 0 for v in e["by_strategy"].values())
+    assert set(r["by_copy_path"]) == {"bulk", "vector"} and all(v["achieved"] > 0 for v in r["by_copy_path"].values())
+    rows = e["curve"]["rows"]
+    assert {(x["tier"], x["op"], x["ids"], x["mask"]) for x in rows} >= {
+        ("host", "store", "random", "bernoulli"), ("host", "load", "contiguous", "ones"), ("hbm", "store", "random", "ones")}
+    assert {x["blocks"] for x in rows} == {1, 16, 256} and all(x["gbps"] > 0 for x in rows)
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["value"] > 0 and c["cores"] == 1
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}

@@ -355,8 +355,10 @@ def test_device_self_check_skips_the_entry_and_reports_range(name, m, kw):
     # a skipped entry's slot would receive stale staging bytes: only its restore is checked here)
     staged = kw.get("link_strategy") == e.LINK_STAGED and kw.get("tier_location") == e.TIER_PINNED_HOST
     for op in (("load",) if staged else ("store", "load")):
-        table = rng.permutation(nb)[:m].astype(np.int32)
-        assert (table >= narrowed).any() and (table < narrowed).any()
+        # m - 3 blocks below the narrowed limit and 3 between it and the real one, shuffled
+        table = np.concatenate([rng.permutation(narrowed)[:m - 3],
+                                narrowed + rng.permutation(nb - narrowed)[:3]]).astype(np.int32)
+        rng.shuffle(table)
         slots = rng.permutation(kh)[:m].astype(np.int32)
         keep = table < narrowed
         if op == "store":
