@@ -102,19 +102,27 @@ class HostTier:
         return estimate_exceeds and full and evicting
 
     # ---- one request ----------------------------------------------------------------------
-    def step(self, keys, n_tokens, agent, now_ms):
+    def step(self, keys, n_tokens, agent, now_ms, decided=None):
+        """``decided``: None for the request's first lookup.  A later lookup of the same request
+        (after a preemption; Appendix D: the store/skip choice is kept for later lookups of the
+        same request) passes the choice made then: the walk is the same, but the request is not
+        registered again in the activity and prompt-length windows, which count first lookups."""
         if len(keys) > self.K:
             raise CapacityError("request references more blocks than the tier holds")
         res = StepResult()
         H = self.leading_run(keys)
         res.host_prefix_blocks = H
-        res.pressure = self._pressure(agent, n_tokens, now_ms)
         res.new_chunks = n_tokens // self.b - (H * self.b) // self.b
-        res.save = not (res.pressure and res.new_chunks > self.kappa)
         st = self.stats
-        st["requests"] += 1
-        st["pressure_requests"] += int(res.pressure)
-        st["declined_requests"] += int(not res.save)
+        if decided is None:
+            res.pressure = self._pressure(agent, n_tokens, now_ms)
+            res.save = not (res.pressure and res.new_chunks > self.kappa)
+            st["requests"] += 1
+            st["pressure_requests"] += int(res.pressure)
+            st["declined_requests"] += int(not res.save)
+        else:
+            res.pressure = False
+            res.save = bool(decided)
         for k in keys:
             st["references"] += 1
             if k in self.order:

@@ -39,11 +39,13 @@ class GpuTier:
     def __init__(self, num_blocks, free_order=0):
         self.NB = int(num_blocks)
         self.free_order = int(free_order)
-        self.order = OrderedDict()                 # key -> block id, least recent first
+        self.order = OrderedDict()                 # key -> block id, least recent first (evictable)
         self.free = list(range(self.NB - 1, -1, -1))
+        self.pinned = {}                           # key -> [block id, holders]: out of the recency order
+        self.held = {}                             # request id -> (keys in prompt order, tail block)
 
     def __contains__(self, key):
-        return key in self.order
+        return key in self.order or key in self.pinned
 
     def _alloc(self):
         if not self.free:
@@ -75,6 +77,58 @@ class GpuTier:
     def release(self, block_id):
         if block_id >= 0:
             self.free.append(block_id)
+
+    # ---- several requests at once: a running request's blocks cannot be evicted -------------
+    # (Section 2: the engine runs several requests at once and suspends one when GPU KV memory
+    # runs out.)  A pinned block is out of the recency order; when its last holder lets go it
+    # re-enters at the most-recent end.  acquire() followed at once by release_request() leaves
+    # the tier exactly as step() does.
+    def fits(self, keys, need_tail):
+        """Can ``keys`` (+ a tail block) be acquired without touching a pinned block?  Every key
+        whose block nobody holds yet takes one block out of the free and the evictable ones."""
+        pinned = self.pinned
+        cost = int(need_tail) + sum(1 for k in dict.fromkeys(keys) if k not in pinned)
+        return cost <= len(self.free) + len(self.order)
+
+    def acquire(self, request_id, keys, need_tail):
+        """Reference ``keys`` in order and pin their blocks for ``request_id``.  Returns
+        (was_resident[], block_id[], tail_block) or None, with nothing changed, if they do not fit."""
+        pinned = self.pinned
+        if request_id in self.held:
+            raise ValueError("request already holds blocks")
+        if not self.fits(keys, need_tail):
+            return None
+        resident, ids = [], []
+        for k in keys:
+            if k in pinned:                       # held by a running request (maybe this one)
+                pinned[k][1] += 1
+                resident.append(1)
+                ids.append(pinned[k][0])
+            elif k in self.order:
+                blk = self.order.pop(k)
+                pinned[k] = [blk, 1]
+                resident.append(1)
+                ids.append(blk)
+            else:
+                blk = self._alloc()
+                pinned[k] = [blk, 1]
+                resident.append(0)
+                ids.append(blk)
+        tail = self._alloc() if need_tail else -1
+        self.held[request_id] = (list(keys), tail)
+        return resident, ids, tail
+
+    def release_request(self, request_id):
+        """The request finished or was suspended: its blocks become evictable again, entering
+        the recency order in prompt order (or tail first, see ``free_order``)."""
+        keys, tail = self.held.pop(request_id)
+        for k in (reversed(keys) if self.free_order == 1 else keys):
+            ent = self.pinned[k]
+            ent[1] -= 1
+            if ent[1] == 0:
+                del self.pinned[k]
+                self.order[k] = ent[0]
+        self.release(tail)
 
 
 class TraceOracle:
@@ -155,6 +209,71 @@ class TraceOracle:
         t["host_hit_blocks"] += H
         self.records.append(rec)
         return rec
+
+    # ---- requests that overlap: begin pins the GPU blocks, finish lets them go ---------------
+    def begin(self, request_id, tokens, agent, now_ms, keys=None, decided=None):
+        """The same turn as ``turn`` up to and including the store, with the request's GPU blocks
+        pinned until ``finish``.  Returns None, with nothing changed, if the GPU tier cannot hold
+        the request beside the running ones.  ``decided``: the save decision of the request's
+        first lookup when this is a later one (a resumed request), else None."""
+        n = len(tokens)
+        if keys is None:
+            keys = ohash.hash_blocks(tokens, self.b, self.hash_seed, self.hash_base)
+        need_tail = n % self.b != 0
+        if not self.gpu.fits(keys, need_tail):
+            return None
+        G = 0
+        for k in keys:
+            if k not in self.gpu:
+                break
+            G += 1
+        R = self.R
+        chunk_keys = keys[R - 1::R]
+        Hc = self.host.leading_run(chunk_keys)
+        H = Hc * R
+        host_slots = [self.host.slot_of(k) * R + i for k in chunk_keys[:Hc] for i in range(R)]
+        res = self.host.step(chunk_keys, n, agent, now_ms, decided=decided)
+        resident, gpu_ids, tail = self.gpu.acquire(request_id, keys, need_tail)
+        cover = max(G, H)
+        lo, hi = (G, H) if H > G else (G, G)
+        fill = [j for j in range(cover, len(keys)) if not resident[j]]
+        admit_b = [0] * len(keys)
+        slot_b = [-1] * len(keys)
+        for c, (a, s) in enumerate(zip(res.admit, res.slot)):
+            for i in range(R):
+                admit_b[c * R + i] = a
+                slot_b[c * R + i] = s * R + i if s >= 0 else -1
+        if self.payload is not None:
+            storeload.load(self.pool, self.tier, host_slots[lo:hi], gpu_ids[lo:hi])
+            if fill:
+                W = self.shape.piece_bytes // 2
+                for q in range(self.shape.pieces_per_block):
+                    words = self.payload([keys[j] for j in fill], q, W)
+                    for r, j in enumerate(fill):
+                        self.pool[q][gpu_ids[j], :] = words[r].view(np.uint8)
+            storeload.store(self.pool, self.tier, gpu_ids, admit_b, slot_b)
+        rec = dict(agent=agent, now_ms=now_ms, n_tokens=n, keys=keys, G=G, H=H,
+                   new_chunks=res.new_chunks, pressure=res.pressure, save=res.save,
+                   hit=res.hit, admit=res.admit, slot=res.slot, evicted=res.evicted,
+                   gpu_resident=resident, gpu_block=gpu_ids, loaded=hi - lo,
+                   stored=sum(admit_b), fresh_tokens=n - cover * self.b, filled=len(fill),
+                   request_id=request_id, resumed=decided is not None, tail_block=tail)
+        t = self.totals
+        if decided is None:
+            t["prompt_tokens"] += n
+            t["fresh_tokens"] += rec["fresh_tokens"]
+            t["gpu_hit_blocks"] += G
+            t["host_hit_blocks"] += H
+        else:       # Appendix C: tokens recomputed after a preemption add to computed prefill (J)
+            t["preempt_recomputed_tokens"] = t.get("preempt_recomputed_tokens", 0) + rec["fresh_tokens"]
+        t["loaded_blocks"] += rec["loaded"]
+        t["stored_blocks"] += rec["stored"]
+        self.records.append(rec)
+        return rec
+
+    def finish(self, request_id):
+        """The request finished, or the engine suspended it: its blocks become evictable."""
+        self.gpu.release_request(request_id)
 
     def run(self, trace, limit=None):
         for i, req in enumerate(trace.requests):
