@@ -228,6 +228,17 @@ int eakv_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
                    uint64_t* evicted_keys_out, int32_t* evicted_slots_out,
                    int64_t* n_evicted_inout, eakv_step_info* info_out);
 
+/* A later lookup of a request whose write admission is already decided (Appendix D: the store or
+ * skip choice of a request's first prefix lookup is kept for its later lookups, including those
+ * after a preemption).  The walk, promotions, insertions and evictions are those of
+ * eakv_tier_step with save(r) = `save`; the request is not registered again in the activity and
+ * prompt-length windows of Eq. 10, which count first lookups, and it does not count as a request
+ * in the statistics.  info_out->pressure is 0. */
+int eakv_tier_step_again(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks, int64_t n_tokens,
+                         int64_t now_ms, int32_t save, uint8_t* hit_out, uint8_t* admit_out,
+                         int32_t* slot_out, uint64_t* evicted_keys_out, int32_t* evicted_slots_out,
+                         int64_t* n_evicted_inout, eakv_step_info* info_out);
+
 /* Tier index export / import: carry a host tier across a restart of the process that owns the
  * context (no counterpart in the paper, whose replays start from a cold cache; Section 5.1).
  * eakv_tier_export writes the keys and slots of the resident units in recency order, least
@@ -264,6 +275,25 @@ int eakv_gpu_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blo
                        int32_t need_tail, uint8_t* resident_out, int32_t* block_out,
                        int32_t* tail_block_out);
 int eakv_gpu_tier_release(eakv_ctx* ctx, int32_t block_id);
+
+/* Several requests at once (Section 2: the engine runs up to a cap of requests at the same time
+ * and suspends one when GPU KV memory runs out; Appendix A: cap 16).  eakv_gpu_tier_acquire is
+ * eakv_gpu_tier_step for a request that stays running: it references the keys in order in the same
+ * way and then keeps every block of the prompt (and the tail block) pinned under request_id, out
+ * of the recency order, so that no other request can take them.  A block already pinned by
+ * another running request (a shared prefix) is shared.  EAKV_E_CAPACITY, nothing changed, when the
+ * blocks nobody holds do not suffice: the caller waits, or suspends a running request with
+ * eakv_gpu_tier_release_request and tries again.  eakv_gpu_tier_release_request lets a finished
+ * or suspended request's blocks go: those no other request holds re-enter the recency order at
+ * the most-recent end in prompt order (tail first under EAKV_FREE_REVERSE) and keep their keys, so a
+ * resumed request finds what has not been evicted meanwhile; the tail block is freed.  With one
+ * request at a time acquire + release leaves the tier exactly as eakv_gpu_tier_step does.  While
+ * any request holds blocks, eakv_gpu_tier_step and eakv_turn_begin return EAKV_E_INVAL.
+ * Errors: EAKV_E_INVAL (request_id already holds blocks / holds none). */
+int eakv_gpu_tier_acquire(eakv_ctx* ctx, int64_t request_id, const uint64_t* hashes_host, int64_t n_blocks,
+                          int32_t need_tail, uint8_t* resident_out, int32_t* block_out,
+                          int32_t* tail_block_out);
+int eakv_gpu_tier_release_request(eakv_ctx* ctx, int64_t request_id);
 
 /* Store (Section 2 host writes; Appendix D: copy only absent chunks, from their original
  * GPU KV locations): for every j with admit_mask[j] != 0 copy all 2L pieces of pool block

@@ -13,7 +13,7 @@ static inline uint64_t mix64(uint64_t x) {
 
 KeyedLru::KeyedLru(int64_t capacity)
     : cap_(capacity), resident_(0), key_(capacity), prev_(capacity, -1), next_(capacity, -1),
-      state_(capacity, 0), lru_(-1), mru_(-1) {
+      state_(capacity, 0), pin_count_(capacity, 0), lru_(-1), mru_(-1) {
     free_.reserve(capacity);
     for (int64_t s = capacity - 1; s >= 0; --s) free_.push_back((int32_t)s);
     size_t n = 16;
@@ -111,9 +111,23 @@ int32_t KeyedLru::insert(uint64_t key, bool* evicted, uint64_t* victim_key, int3
     return s;
 }
 
+void KeyedLru::pin(int32_t s) {
+    if (pin_count_[s]++ == 0) {
+        unlink(s);
+        ++pinned_;
+    }
+}
+
+void KeyedLru::unpin(int32_t s) {
+    if (--pin_count_[s] == 0) {
+        push_mru(s);
+        --pinned_;
+    }
+}
+
 int32_t KeyedLru::erase(uint64_t key) {
     const int32_t s = find(key);
-    if (s < 0) return -1;
+    if (s < 0 || pin_count_[s] > 0) return -1;
     table_erase(key);
     unlink(s);
     state_[s] = 0;

@@ -37,6 +37,15 @@ public:
     // give an unkeyed slot back to the free stack
     void release_unkeyed(int32_t slot);
     bool is_unkeyed_taken(int32_t slot) const { return state_[slot] == 2; }
+    // Pinning (a running request holds the slot): a pinned resident leaves the recency order, so
+    // it can be neither evicted nor promoted; when its last holder unpins it, it re-enters at the
+    // most-recent end.  insert / take_unkeyed must not be called when nothing is free and every
+    // resident is pinned (callers check evictable() + free_slots() first).
+    void pin(int32_t slot);
+    void unpin(int32_t slot);
+    bool is_pinned(int32_t slot) const { return pin_count_[slot] > 0; }
+    int64_t evictable() const { return resident_ - pinned_; }
+    int64_t free_slots() const { return (int64_t)free_.size(); }
     // Residents in recency order, least recent first, into keys[]/slots[] (either may be NULL);
     // returns how many there are (at most `capacity` are written).
     int64_t export_order(uint64_t* keys, int32_t* slots, int64_t capacity) const;
@@ -58,6 +67,8 @@ private:
     std::vector<uint64_t> key_;        // by slot
     std::vector<int32_t> prev_, next_; // by slot; -1 ends
     std::vector<uint8_t> state_;       // 0 free, 1 keyed resident, 2 unkeyed taken
+    std::vector<int32_t> pin_count_;   // holders per slot
+    int64_t pinned_ = 0;               // residents with at least one holder
     int32_t lru_, mru_;
     std::vector<int32_t> free_;        // stack
     std::vector<int32_t> table_;       // slot + 1, 0 = empty

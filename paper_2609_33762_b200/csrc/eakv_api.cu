@@ -9,6 +9,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <unordered_map>
 #include <vector>
 
 #include "control_plane.h"
@@ -62,6 +63,8 @@ struct eakv_ctx {
     KeyedLru* gpu_tier = nullptr;
     Admission* adm = nullptr;
     int64_t gpu_unkeyed = 0;
+    struct HeldRequest { std::vector<int32_t> blocks; int32_t tail = -1; };
+    std::unordered_map<int64_t, HeldRequest> held;     // running requests and the GPU blocks they pin
     eakv_stats stats;
 
     // hash
@@ -820,11 +823,13 @@ int eakv_match(const eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_block
     return EAKV_OK;
 }
 
-int eakv_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
-                   int64_t agent_id, int64_t n_tokens, int64_t now_ms,
-                   uint8_t* hit_out, uint8_t* admit_out, int32_t* slot_out,
-                   uint64_t* evicted_keys_out, int32_t* evicted_slots_out,
-                   int64_t* n_evicted_inout, eakv_step_info* info_out) {
+// decided < 0: the request's first lookup (admission is decided here and the request enters the
+// activity and prompt-length windows); 0 / 1: a later lookup of a request whose choice was skip / store
+static int tier_step_impl(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
+                          int64_t agent_id, int64_t n_tokens, int64_t now_ms, int decided,
+                          uint8_t* hit_out, uint8_t* admit_out, int32_t* slot_out,
+                          uint64_t* evicted_keys_out, int32_t* evicted_slots_out,
+                          int64_t* n_evicted_inout, eakv_step_info* info_out) {
     if (!ctx || n_blocks < 0 || n_tokens < 0) return EAKV_E_INVAL;
     if (n_blocks > 0 && (!hashes_host || !hit_out || !admit_out || !slot_out)) return EAKV_E_INVAL;
     if (n_blocks > ctx->host_tier->capacity()) return EAKV_E_CAPACITY;
@@ -834,14 +839,17 @@ int eakv_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
     KeyedLru& T = *ctx->host_tier;
     int64_t H = 0;
     while (H < n_blocks && T.find(hashes_host[H]) >= 0) ++H;
-    const bool p = ctx->adm->pressure(agent_id, n_tokens, now_ms, T.resident());
+    const bool first = decided < 0;
+    const bool p = first ? ctx->adm->pressure(agent_id, n_tokens, now_ms, T.resident()) : false;
     const int64_t cb = ctx->chunk_tokens;                 // tokens per tier unit
     const int64_t u = n_tokens / cb - (H * cb) / cb;
-    const bool save = !(p && u > ctx->adm->kappa());
+    const bool save = first ? !(p && u > ctx->adm->kappa()) : decided != 0;
     eakv_stats& st = ctx->stats;
-    st.requests += 1;
-    st.pressure_requests += p;
-    st.declined_requests += !save;
+    if (first) {
+        st.requests += 1;
+        st.pressure_requests += p;
+        st.declined_requests += !save;
+    }
     int64_t n_ev = 0;
     for (int64_t j = 0; j < n_blocks; ++j) {
         const uint64_t key = hashes_host[j];
@@ -881,6 +889,23 @@ int eakv_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
     return EAKV_OK;
 }
 
+int eakv_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks,
+                   int64_t agent_id, int64_t n_tokens, int64_t now_ms,
+                   uint8_t* hit_out, uint8_t* admit_out, int32_t* slot_out,
+                   uint64_t* evicted_keys_out, int32_t* evicted_slots_out,
+                   int64_t* n_evicted_inout, eakv_step_info* info_out) {
+    return tier_step_impl(ctx, hashes_host, n_blocks, agent_id, n_tokens, now_ms, -1, hit_out, admit_out,
+                          slot_out, evicted_keys_out, evicted_slots_out, n_evicted_inout, info_out);
+}
+
+int eakv_tier_step_again(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blocks, int64_t n_tokens,
+                         int64_t now_ms, int32_t save, uint8_t* hit_out, uint8_t* admit_out,
+                         int32_t* slot_out, uint64_t* evicted_keys_out, int32_t* evicted_slots_out,
+                         int64_t* n_evicted_inout, eakv_step_info* info_out) {
+    return tier_step_impl(ctx, hashes_host, n_blocks, 0, n_tokens, now_ms, save ? 1 : 0, hit_out, admit_out,
+                          slot_out, evicted_keys_out, evicted_slots_out, n_evicted_inout, info_out);
+}
+
 int eakv_tier_export(const eakv_ctx* ctx, uint64_t* keys_host_out, int32_t* slots_host_out,
                      int64_t capacity, int64_t* n_out) {
     if (!ctx || !n_out || capacity < 0) return EAKV_E_INVAL;
@@ -918,6 +943,7 @@ int eakv_gpu_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blo
     if (n_blocks > 0 && (!hashes_host || !resident_out || !block_out)) return EAKV_E_INVAL;
     if (need_tail && !tail_block_out) return EAKV_E_INVAL;
     KeyedLru& T = *ctx->gpu_tier;
+    if (!ctx->held.empty()) return EAKV_E_INVAL;    // running requests hold blocks: use acquire / release
     if (n_blocks + (need_tail ? 1 : 0) + ctx->gpu_unkeyed > T.capacity()) return EAKV_E_CAPACITY;
     bool ev;
     uint64_t vkey;
@@ -940,6 +966,62 @@ int eakv_gpu_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blo
     }
     if (ctx->cfg.gpu_free_order == EAKV_FREE_REVERSE)
         for (int64_t j = n_blocks - 1; j >= 0; --j) T.promote(block_out[j]);
+    return EAKV_OK;
+}
+
+int eakv_gpu_tier_acquire(eakv_ctx* ctx, int64_t request_id, const uint64_t* hashes_host, int64_t n_blocks,
+                          int32_t need_tail, uint8_t* resident_out, int32_t* block_out,
+                          int32_t* tail_block_out) {
+    if (!ctx || n_blocks < 0) return EAKV_E_INVAL;
+    if (n_blocks > 0 && (!hashes_host || !resident_out || !block_out)) return EAKV_E_INVAL;
+    if (need_tail && !tail_block_out) return EAKV_E_INVAL;
+    if (ctx->held.count(request_id)) return EAKV_E_INVAL;
+    KeyedLru& T = *ctx->gpu_tier;
+    // every key whose block nobody holds yet takes one block out of the free and the evictable
+    // ones (a resident one takes itself); blocks held by running requests are out of reach
+    int64_t cost = need_tail ? 1 : 0;
+    for (int64_t j = 0; j < n_blocks; ++j) {
+        const int32_t s = T.find(hashes_host[j]);
+        if (s < 0 || !T.is_pinned(s)) ++cost;
+    }
+    if (cost > T.free_slots() + T.evictable()) return EAKV_E_CAPACITY;
+    eakv_ctx::HeldRequest& h = ctx->held[request_id];
+    h.blocks.resize((size_t)n_blocks);
+    bool ev;
+    uint64_t vkey;
+    int32_t vslot;
+    for (int64_t j = 0; j < n_blocks; ++j) {
+        int32_t s = T.find(hashes_host[j]);
+        resident_out[j] = s >= 0;
+        if (s < 0) s = T.insert(hashes_host[j], &ev, &vkey, &vslot);
+        T.pin(s);
+        block_out[j] = s;
+        h.blocks[(size_t)j] = s;
+    }
+    if (tail_block_out) *tail_block_out = -1;
+    if (need_tail) {
+        h.tail = T.take_unkeyed(&ev, &vkey, &vslot);
+        *tail_block_out = h.tail;
+        ctx->gpu_unkeyed += 1;
+    }
+    return EAKV_OK;
+}
+
+int eakv_gpu_tier_release_request(eakv_ctx* ctx, int64_t request_id) {
+    if (!ctx) return EAKV_E_INVAL;
+    auto it = ctx->held.find(request_id);
+    if (it == ctx->held.end()) return EAKV_E_INVAL;
+    KeyedLru& T = *ctx->gpu_tier;
+    const std::vector<int32_t>& b = it->second.blocks;
+    if (ctx->cfg.gpu_free_order == EAKV_FREE_REVERSE)
+        for (size_t j = b.size(); j-- > 0;) T.unpin(b[j]);
+    else
+        for (size_t j = 0; j < b.size(); ++j) T.unpin(b[j]);
+    if (it->second.tail >= 0) {
+        T.release_unkeyed(it->second.tail);
+        ctx->gpu_unkeyed -= 1;
+    }
+    ctx->held.erase(it);
     return EAKV_OK;
 }
 
@@ -1102,7 +1184,7 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
                     const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
                     void* cuda_stream, eakv_turn_view* view) {
     if (!ctx || !view || n_tokens < 0 || n_known < 0) return EAKV_E_INVAL;
-    if (ctx->turn_open) return EAKV_E_INVAL;
+    if (ctx->turn_open || !ctx->held.empty()) return EAKV_E_INVAL;
     if (n_known > 0 && !known_keys) return EAKV_E_INVAL;
     const bool bookkeeping_only = ctx->device < 0;
     const int b = ctx->cfg.block_size;

@@ -92,6 +92,7 @@ EXPORTS = [
     "eakv_turn_begin", "eakv_turn_end", "eakv_turn_abort", "eakv_tier_export", "eakv_tier_import",
     "eakv_admission_export", "eakv_admission_import",
     "eakv_selfcheck_limits", "eakv_selfcheck_wait_probe",
+    "eakv_gpu_tier_acquire", "eakv_gpu_tier_release_request", "eakv_tier_step_again",
 ]
 STATIC_MAX_BLOCKS = 65536
 
@@ -119,6 +120,10 @@ def lib():
                                  C.POINTER(i64), C.POINTER(StepInfo)]
     L.eakv_gpu_tier_step.argtypes = [vp, vp, i64, i32, vp, vp, C.POINTER(i32)]
     L.eakv_gpu_tier_release.argtypes = [vp, i32]
+    L.eakv_gpu_tier_acquire.argtypes = [vp, i64, vp, i64, i32, vp, vp, C.POINTER(i32)]
+    L.eakv_gpu_tier_release_request.argtypes = [vp, i64]
+    L.eakv_tier_step_again.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp,
+                                       C.POINTER(i64), C.POINTER(StepInfo)]
     L.eakv_store.argtypes = [vp, vp, vp, vp, i64, vp]
     L.eakv_load.argtypes = [vp, vp, vp, i64, vp]
     L.eakv_load_layers.argtypes = [vp, vp, vp, i64, i32, vp, i32, vp]
@@ -349,7 +354,9 @@ class Context:
         v, vp_ = _np(values, np.int64)
         self._check(lib().eakv_admission_import(self._h, vp_, len(v)), "eakv_admission_import")
 
-    def eakv_tier_step(self, hashes, agent_id, n_tokens, now_ms):
+    def eakv_tier_step(self, hashes, agent_id, n_tokens, now_ms, decided=None):
+        """``decided``: None for a request's first lookup; True / False = the store / skip choice
+        of that first lookup when this is a later one (eakv_tier_step_again)."""
         h, hp = _np(hashes, np.uint64)
         n = len(h)
         hit = np.zeros(n, dtype=np.uint8)
@@ -360,9 +367,14 @@ class Context:
         nev = C.c_int64(n)
         info = StepInfo()
         vp = lambda a: a.ctypes.data_as(C.c_void_p)
-        rc = lib().eakv_tier_step(self._h, hp, n, int(agent_id), int(n_tokens), int(now_ms),
-                                  vp(hit), vp(admit), vp(slot), vp(ek), vp(es), C.byref(nev),
-                                  C.byref(info))
+        if decided is None:
+            rc = lib().eakv_tier_step(self._h, hp, n, int(agent_id), int(n_tokens), int(now_ms),
+                                      vp(hit), vp(admit), vp(slot), vp(ek), vp(es), C.byref(nev),
+                                      C.byref(info))
+        else:
+            rc = lib().eakv_tier_step_again(self._h, hp, n, int(n_tokens), int(now_ms), int(bool(decided)),
+                                            vp(hit), vp(admit), vp(slot), vp(ek), vp(es), C.byref(nev),
+                                            C.byref(info))
         self._check(rc, "eakv_tier_step")
         k = nev.value
         return dict(hit=hit, admit=admit, slot=slot, evicted_keys=ek[:k], evicted_slots=es[:k],
@@ -380,6 +392,26 @@ class Context:
                                       blk.ctypes.data_as(C.c_void_p), C.byref(tail))
         self._check(rc, "eakv_gpu_tier_step")
         return res, blk, tail.value
+
+    def eakv_gpu_tier_acquire(self, request_id, hashes, need_tail):
+        """(resident, blocks, tail) with the blocks pinned under ``request_id``, or None when they
+        do not fit beside the running requests (nothing changed)."""
+        h, hp = _np(hashes, np.uint64)
+        n = len(h)
+        res = np.zeros(n, dtype=np.uint8)
+        blk = np.zeros(n, dtype=np.int32)
+        tail = C.c_int32(-1)
+        rc = lib().eakv_gpu_tier_acquire(self._h, int(request_id), hp, n, int(bool(need_tail)),
+                                         res.ctypes.data_as(C.c_void_p), blk.ctypes.data_as(C.c_void_p),
+                                         C.byref(tail))
+        if rc == E_CAPACITY:
+            return None
+        self._check(rc, "eakv_gpu_tier_acquire")
+        return res, blk, tail.value
+
+    def eakv_gpu_tier_release_request(self, request_id):
+        self._check(lib().eakv_gpu_tier_release_request(self._h, int(request_id)),
+                    "eakv_gpu_tier_release_request")
 
     def eakv_gpu_tier_release(self, block_id):
         self._check(lib().eakv_gpu_tier_release(self._h, int(block_id)), "eakv_gpu_tier_release")

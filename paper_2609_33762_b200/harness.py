@@ -175,6 +175,83 @@ class AgentServer:
                    fresh_tokens=v["fresh_tokens"], filled=int(v["n_fill"]))
         return rec, G, H
 
+    def begin(self, request_id, tokens, agent, now_ms, decided=None):
+        """A turn of a request that stays running: the same steps as ``turn`` up to and including
+        the store, with the request's GPU blocks pinned under ``request_id`` until ``finish``
+        (eakv_gpu_tier_acquire).  Returns None, with nothing changed, when the blocks do not fit
+        beside the running requests.  ``decided``: None for the request's first lookup, else the
+        store/skip choice made then (a resumed request: eakv_tier_step_again)."""
+        tokens = np.asarray(tokens, dtype=np.int32)
+        n = len(tokens)
+        keys = self.block_keys(tokens, agent)
+        nblk = len(keys)
+        R = self.R
+        # lookups first (they change nothing), then the GPU side: if the blocks cannot be had,
+        # neither tier may change
+        if R == 1:
+            G, H, _, host_slots = self.ctx.eakv_match(keys)
+            unit_keys = keys
+        else:
+            G = self.ctx.eakv_match(keys)[0]
+            unit_keys = np.ascontiguousarray(keys[R - 1::R])
+            _, Hc, _, chunk_slots = self.ctx.eakv_match(unit_keys)
+            H = Hc * R
+            host_slots = (chunk_slots.astype(np.int64)[:, None] * R + np.arange(R)).reshape(-1).astype(np.int32)
+        got = self.ctx.eakv_gpu_tier_acquire(request_id, keys, n % self.b != 0)
+        if got is None:
+            return None
+        resident, blocks, tail = got
+        step = self.ctx.eakv_tier_step(unit_keys, agent, n, now_ms, decided=decided)
+        if R == 1:
+            admit_b, slot_b = step["admit"], step["slot"]
+        else:
+            admit_b = np.zeros(nblk, dtype=np.uint8)
+            slot_b = np.full(nblk, -1, dtype=np.int32)
+            nc = len(unit_keys)
+            admit_b[:nc * R] = np.repeat(step["admit"], R)
+            base = np.repeat(step["slot"].astype(np.int64), R) * R + np.tile(np.arange(R), nc)
+            slot_b[:nc * R] = np.where(np.repeat(step["slot"], R) >= 0, base, -1).astype(np.int32)
+        cover = max(G, H)
+        lo, hi = (G, H) if H > G else (G, G)
+        if hi > lo and self.data_plane:
+            with self._time("load", (hi - lo) * self.ctx.block_bytes):
+                self.ctx.eakv_load(host_slots[lo:hi], blocks[lo:hi], self.stream)
+        fill = [j for j in range(cover, nblk) if not resident[j]]
+        if fill and self.data_plane:
+            ids = torch.as_tensor(blocks[fill].astype(np.int64), device=self.device)
+            fkeys = keys[fill]
+            for q, piece in enumerate(self.pool.pieces):
+                w = self.payload(fkeys, q, self.pool.words)
+                if isinstance(w, np.ndarray):
+                    w = torch.from_numpy(w.view(np.int16)).to(self.device)
+                piece[ids] = w.view(torch.int16)
+        if self.data_plane and admit_b.any():
+            with self._time("store", int(admit_b.sum()) * self.ctx.block_bytes):
+                self.ctx.eakv_store(blocks, admit_b, slot_b, self.stream)
+        rec = dict(agent=agent, now_ms=now_ms, n_tokens=n, keys=keys, G=G, H=H,
+                   new_chunks=step["new_chunks"], pressure=step["pressure"], save=step["save"],
+                   hit=step["hit"], admit=step["admit"], slot=step["slot"],
+                   evicted=list(zip(step["evicted_keys"].tolist(), step["evicted_slots"].tolist())),
+                   gpu_resident=resident, gpu_block=blocks, loaded=hi - lo,
+                   stored=int(admit_b.sum()), fresh_tokens=n - cover * self.b,
+                   filled=len(fill), request_id=request_id, resumed=decided is not None, tail_block=tail)
+        t = self.totals
+        if decided is None:
+            t["prompt_tokens"] += n
+            t["fresh_tokens"] += rec["fresh_tokens"]
+            t["gpu_hit_blocks"] += G
+            t["host_hit_blocks"] += H
+        else:
+            t["preempt_recomputed_tokens"] = t.get("preempt_recomputed_tokens", 0) + rec["fresh_tokens"]
+        t["loaded_blocks"] += rec["loaded"]
+        t["stored_blocks"] += rec["stored"]
+        self.records.append(rec)
+        return rec
+
+    def finish(self, request_id):
+        """The request finished, or the engine suspended it: its GPU blocks become evictable."""
+        self.ctx.eakv_gpu_tier_release_request(request_id)
+
     def turn(self, tokens, agent, now_ms):
         tokens = np.asarray(tokens, dtype=np.int32)
         if self.native_turn:

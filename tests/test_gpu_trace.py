@@ -252,6 +252,44 @@ def test_closed_loop_replay_bit_exact(policy, kh, pool, native):
     server.close()
 
 
+@pytest.mark.parametrize("policy,kh,gpu_blocks,S,decode_us,R,link", [
+    (0, 1024, 130, 4, 20_000, 1, 1), (0, 160, 140, 3, 60_000, 1, 0), (2, 200, 200, 6, 40_000, 1, 1),
+    (0, 64, 136, 4, 50_000, 4, 1)])
+def test_engine_replay_with_preemption_bit_exact(policy, kh, gpu_blocks, S, decode_us, R, link):
+    """The engine model (several running requests with pinned GPU blocks, suspension when GPU KV
+    memory runs out, resumption by restoring and recomputing) on the GPU path with bytes: every
+    scheduler event, every record of every first and resumed lookup, J, and every resident byte of
+    both tiers equal the oracle's."""
+    from oracle import closedloop as ocl
+    from oracle import engine as oen
+    from paper_2609_33762_b200 import closedloop
+    from paper_2609_33762_b200.harness import AgentServer
+    cfg = CONFIGS["c0_big_tier"]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg, agents=8, turns=8)
+    kw = dict(policy=policy, kappa_blocks=10 if R == 1 else 2, window_ms=50, len_window=16)
+    rates = dict(t_pf_ns=40_000, h2d_bytes_per_us=9_000, d2h_bytes_per_us=7_000, tau_load_us=120)
+    oracle = TraceOracle(shape, gpu_blocks, kh, payload=key_words_numpy, chunk_blocks=R, **kw)
+    want = oen.replay(trace, oracle, ocl.ServiceModel(**rates), 8, S, decode_us, shape.bytes_per_token)
+    server = AgentServer(shape, gpu_blocks, kh, key_words_numpy, incremental_hash=True, chunk_blocks=R,
+                         link_strategy=link, **kw)
+    got = closedloop.replay_engine(trace, server.begin, server.finish, closedloop.ServiceModel(**rates), 8, S,
+                                   decode_us, shape.bytes_per_token, shape.block_size)
+    assert got["events"] == want["events"] and got["order"] == want["order"]
+    assert got["makespan_us"] == want["makespan_us"] and got["preemptions"] == want["preemptions"] > 0
+    assert got["recomputed_after_preemption"] == want["totals"]["preempt_recomputed_tokens"]
+    compare_records(server.records, oracle.records)
+    assert [r["resumed"] for r in server.records] == [r["resumed"] for r in oracle.records]
+    want_totals = dict(oracle.totals)
+    want_totals.setdefault("preempt_recomputed_tokens", 0)
+    got_totals = dict(server.totals)
+    got_totals.setdefault("preempt_recomputed_tokens", 0)
+    assert got_totals == want_totals
+    assert any(r["resumed"] and r["loaded"] > 0 for r in oracle.records) or policy == 2 or kh <= 160
+    compare_bytes(server, oracle)
+    server.close()
+
+
 def test_warm_restart_with_adopted_tier_memory():
     """Half of the trace, then the process 'restarts': the host tier's index is exported, the
     context destroyed, a new one adopts the same pinned tier memory and imports the index.  The
