@@ -22,6 +22,18 @@ Readings taken where the paper is silent (integers only, virtual time in ms):
   * slots come from a free stack that first yields 0, 1, 2, ...; an evicted chunk's slot
     is the next one handed out;
   * a request with more full chunks than K_H is refused and changes nothing.
+
+Tier reports (Appendix D, "Pressure signal" and the parameter table: the tier publishes the number
+of registered chunks, K_H and e_t every second; a report older than 5 seconds is not fresh; when
+no fresh report exists, before the first publication for instance, the first factor alone
+decides).  With ``telemetry_period_ms`` = P > 0 the second factor is read from the latest report
+instead of from the tier itself: reports are published at the virtual times P, 2P, 3P, ...; the
+report of time t describes the tier as the requests before t left it (registered chunks, and the
+evictions with a time in (t - W, t)); a request at time ``now`` reads the report of time
+floor(now / P) * P, which exists from P on; it is fresh while now - t <= ``telemetry_max_age_ms``
+(0: any age).  The paper's scheduler reads reports every 0.5 s; since that divides its 1 s report
+interval, a read always sees the latest report, so the read interval is no parameter here.
+P = 0 is the synchronous reading above.
 """
 from collections import OrderedDict, deque
 
@@ -51,8 +63,12 @@ class StepResult:
 
 class HostTier:
     def __init__(self, capacity_blocks, block_size, policy=WRITE_ALL, kappa_blocks=8,
-                 theta_percent=95, window_ms=60_000, len_window=256, telemetry=True):
+                 theta_percent=95, window_ms=60_000, len_window=256, telemetry=True,
+                 telemetry_period_ms=0, telemetry_max_age_ms=0):
         self.K = int(capacity_blocks)
+        self.period = int(telemetry_period_ms)
+        self.max_age = int(telemetry_max_age_ms)
+        self.report = None                            # (time, registered chunks, e_t) of the latest report
         self.b = int(block_size)
         self.policy = policy
         self.kappa = int(kappa_blocks)
@@ -82,6 +98,18 @@ class HostTier:
             n += 1
         return n
 
+    # ---- published reports ----------------------------------------------------------------
+    def _publish(self, now_ms):
+        """Bring the latest report up to date before a request at ``now_ms`` changes anything:
+        if a publication time has passed since the last report, the tier as it stands is what
+        that publication saw (every earlier request came before it)."""
+        if self.period <= 0:
+            return
+        t = (now_ms // self.period) * self.period
+        if t >= self.period and (self.report is None or self.report[0] < t):
+            e = sum(1 for x in self.evict_times if t - self.window_ms < x < t)
+            self.report = (t, len(self.order), e)
+
     # ---- Eq. 10 ---------------------------------------------------------------------------
     def _pressure(self, agent, n_tokens, now_ms):
         self.agent_last[agent] = now_ms
@@ -97,6 +125,12 @@ class HostTier:
         estimate_exceeds = (active - 1) * sum(self.lengths) > self.K * self.b * len(self.lengths)
         if not self.telemetry:
             return estimate_exceeds
+        if self.period > 0:
+            fresh = self.report is not None and (self.max_age <= 0 or now_ms - self.report[0] <= self.max_age)
+            if not fresh:
+                return estimate_exceeds
+            _, registered, evicted = self.report
+            return estimate_exceeds and 100 * registered >= self.theta_percent * self.K and evicted > 0
         full = 100 * len(self.order) >= self.theta_percent * self.K
         evicting = len(self.evict_times) > 0
         return estimate_exceeds and full and evicting
@@ -109,6 +143,7 @@ class HostTier:
         registered again in the activity and prompt-length windows, which count first lookups."""
         if len(keys) > self.K:
             raise CapacityError("request references more blocks than the tier holds")
+        self._publish(now_ms)
         res = StepResult()
         H = self.leading_run(keys)
         res.host_prefix_blocks = H

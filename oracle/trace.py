@@ -135,7 +135,7 @@ class TraceOracle:
     def __init__(self, shape, gpu_blocks, host_blocks, policy=0, kappa_blocks=8,
                  theta_percent=95, window_ms=60_000, len_window=256, telemetry=True,
                  payload=None, hash_base=ohash.HASH_BASE, hash_seed=ohash.HASH_SEED,
-                 chunk_blocks=1, gpu_free_order=0):
+                 chunk_blocks=1, gpu_free_order=0, telemetry_period_ms=0, telemetry_max_age_ms=0):
         """``payload(keys, q, n_words) -> uint16[len(keys), n_words]`` enables full-bytes
         mode (pool and tier held in numpy); None runs metadata only."""
         self.shape = shape
@@ -143,7 +143,7 @@ class TraceOracle:
         self.R = int(chunk_blocks)
         self.gpu = GpuTier(gpu_blocks, gpu_free_order)
         self.host = HostTier(host_blocks, self.b * self.R, policy, kappa_blocks, theta_percent,
-                             window_ms, len_window, telemetry)
+                             window_ms, len_window, telemetry, telemetry_period_ms, telemetry_max_age_ms)
         self.payload = payload
         self.hash_base, self.hash_seed = hash_base, hash_seed
         self.pool = self.tier = None

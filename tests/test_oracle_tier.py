@@ -356,3 +356,102 @@ def test_working_set_within_hand_case():
     assert sd.working_set_within(reqs, toks, [4, 4, 4, 4], 4, percent=1) == 0
     # half of the benefit is not within 1 % but is within 100 %
     assert sd.working_set_within(reqs, toks, [0, 0, 0, 0], 4, percent=10**6) == 0
+
+
+# ---- tier reports published at intervals (Appendix D: 1 s report interval, 5 s maximum age) --------
+def test_published_reports_hand_case():
+    """K_H = 4 chunks of 4 tokens, theta 50 %, kappa 0, reports every 1,000 ms, fresh for 5,000 ms.
+    Two agents with 40-token prompts make the estimate (A-1) * sum(len) > K_H * b * count true
+    from the second request on."""
+    from oracle.tier import FILTER_CONDITIONED, HostTier
+    kw = dict(policy=FILTER_CONDITIONED, kappa_blocks=0, theta_percent=50, window_ms=60_000)
+    t = HostTier(4, 4, telemetry_period_ms=1000, telemetry_max_age_ms=5000, **kw)
+    sync = HostTier(4, 4, **kw)
+    # 100 ms: first request; one agent, estimate false -> saved, the tier is full afterwards
+    for x in (t, sync):
+        r = x.step([1, 2, 3, 4], 40, agent=0, now_ms=100)
+        assert r.save and not r.pressure
+    # 200 ms: no report has been published yet (the first one comes at 1,000 ms): the estimate
+    # alone decides, and it says pressure.  Read synchronously, the tier is full but has not
+    # evicted anything, so there is no pressure.
+    r = t.step([5, 6], 40, agent=1, now_ms=200)
+    assert r.pressure and not r.save and r.admit == [0, 0] and t.report is None
+    assert not sync.step([5, 6], 40, agent=1, now_ms=200).pressure          # (it stores 5, 6, evicting 1, 2)
+    # 1,500 ms: the report of 1,000 ms says 4 registered chunks, no evictions -> no pressure
+    r = t.step([5, 6], 40, agent=1, now_ms=1500)
+    assert t.report == (1000, 4, 0) and not r.pressure and r.save
+    assert r.evicted == [(1, 0), (2, 1)]                                     # evictions at 1,500 ms
+    # 1,900 ms: 0.4 s after those evictions the latest report is still the one of 1,000 ms
+    r = t.step([1, 2], 40, agent=0, now_ms=1900)
+    assert t.report == (1000, 4, 0) and not r.pressure and r.save and len(r.evicted) == 2
+    # 2,100 ms: the report of 2,000 ms counts the four evictions -> full and evicting -> pressure
+    r = t.step([7], 40, agent=1, now_ms=2100)
+    assert t.report == (2000, 4, 4) and r.pressure and not r.save
+    # a request exactly at a publication time reads that report, which does not yet see what the
+    # request itself (or another request of the same millisecond) does
+    r = t.step([8], 4, agent=1, now_ms=3000)
+    assert t.report == (3000, 4, 4)
+    # the eviction window of a report is (t - 60 s, t): the report of 61,000 ms still counts the
+    # evictions of 1,500 and 1,900 ms, the report of 62,000 ms none of them
+    t.step([1], 4, agent=0, now_ms=61_400)
+    assert t.report == (61_000, 4, 4)
+    t.step([1], 4, agent=0, now_ms=62_000)
+    assert t.report == (62_000, 4, 0)
+
+
+def test_stale_report_falls_back_to_the_estimate():
+    """Reports every 10 s, fresh for 5 s; K_H * b = 16 tokens.  The report of 10,000 ms says
+    "3 of 4 chunks, no evictions", i.e. no pressure whatever the estimate says."""
+    from oracle.tier import FILTER_CONDITIONED, HostTier
+    kw = dict(policy=FILTER_CONDITIONED, kappa_blocks=0, theta_percent=50, window_ms=600_000)
+    t = HostTier(4, 4, telemetry_period_ms=10_000, telemetry_max_age_ms=5_000, **kw)
+    assert t.step([1, 2, 3], 12, agent=0, now_ms=100).save              # one agent: estimate false
+    # 12,000 ms: the report is 2 s old, fresh.  Estimate (2-1) * (12+100) = 112 > 16 * 2 is true,
+    # the tier is full (75 % >= 50 %) but the report shows no eviction: no pressure, saved
+    r = t.step([4], 100, agent=1, now_ms=12_000)
+    assert t.report == (10_000, 3, 0) and not r.pressure and r.save
+    # 16,500 ms: the same report is 6.5 s old and no newer one exists (the next comes at 20,000 ms):
+    # not fresh, so the estimate alone decides: (2-1) * 212 > 16 * 3 -> pressure, declined
+    r = t.step([5], 100, agent=0, now_ms=16_500)
+    assert t.report == (10_000, 3, 0) and r.pressure and not r.save and r.new_chunks == 25
+    # with no age limit the old report is still used: no pressure
+    t3 = HostTier(4, 4, telemetry_period_ms=10_000, telemetry_max_age_ms=0, **kw)
+    t3.step([1, 2, 3], 12, agent=0, now_ms=100)
+    t3.step([4], 100, agent=1, now_ms=12_000)
+    assert not t3.step([5], 100, agent=0, now_ms=16_500).pressure
+    # a stale report and an estimate that says no: no pressure (window of one prompt length)
+    t2 = HostTier(4, 4, telemetry_period_ms=10_000, telemetry_max_age_ms=5_000, len_window=1, **kw)
+    t2.step([1, 2, 3], 12, agent=0, now_ms=100)
+    assert not t2.step([4], 100, agent=1, now_ms=12_000).pressure       # fresh report without evictions
+    assert not t2.step([5], 4, agent=0, now_ms=16_500).pressure         # stale; (2-1) * 4 <= 16
+    assert t2.step([6], 100, agent=0, now_ms=16_600).pressure           # stale; (2-1) * 100 > 16
+    # at 20,000 ms the next report appears and is read again
+    t2.step([7], 100, agent=1, now_ms=20_000)
+    assert t2.report[0] == 20_000
+
+
+def test_reports_every_millisecond_equal_the_synchronous_reading():
+    """With a report every millisecond and requests at distinct times the latest report is the tier
+    as the request finds it, so the decisions must be those of the synchronous reading (which has
+    its own hand-computed pins above)."""
+    import random as _random
+    from oracle.tier import FILTER_CONDITIONED, HostTier
+    rng = _random.Random(17)
+    for case in range(20):
+        kw = dict(policy=FILTER_CONDITIONED, kappa_blocks=rng.randrange(0, 4), theta_percent=rng.choice([50, 95]),
+                  window_ms=rng.choice([30, 200]), len_window=rng.choice([4, 64]))
+        a = HostTier(12, 4, **kw)
+        c = HostTier(12, 4, telemetry_period_ms=1, telemetry_max_age_ms=5, **kw)
+        now = 0
+        engaged = 0
+        for i in range(300):
+            now += rng.randrange(1, 9)
+            start = rng.randrange(6) * 20
+            keys = [start + j for j in range(rng.randrange(0, 10))]
+            n_tok = 4 * len(keys) + rng.randrange(4)
+            agent = rng.randrange(4)
+            ra, rc = a.step(keys, n_tok, agent, now), c.step(keys, n_tok, agent, now)
+            assert (ra.pressure, ra.save, ra.hit, ra.admit, ra.slot, ra.evicted) == \
+                   (rc.pressure, rc.save, rc.hit, rc.admit, rc.slot, rc.evicted)
+            engaged += ra.pressure
+        assert engaged > 0
