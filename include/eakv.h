@@ -139,6 +139,18 @@ typedef struct eakv_config {
                                       block the write still reads (the caller's stream is then made to
                                       wait at eakv_turn_begin).  Call eakv_sync
                                       before reading the tier on the host                              */
+    int64_t telemetry_period_ms;   /* Appendix D, pressure signal and parameter table (report interval 1 s,
+                                      maximum age of a fresh report 5 s).  0: the occupancy and eviction
+                                      terms of Eq. 10 are read from the tier itself at every request.
+                                      P > 0: they are read from the latest published report.  Reports are
+                                      published at the virtual times P, 2P, ... (now_ms of eakv_tier_step);
+                                      the report of time t describes the tier as the requests before t
+                                      left it: resident units, and the evictions with a time in
+                                      (t - window_ms, t).  A request at now_ms reads the report of
+                                      floor(now_ms / P) * P                                               */
+    int64_t telemetry_max_age_ms;  /* a report older than this is not fresh (0: any age is).  Without a
+                                      fresh report -- before the first publication, too -- p_t is the
+                                      working-set test of Eq. 10 alone                                    */
 } eakv_config;
 
 typedef struct eakv_stats {

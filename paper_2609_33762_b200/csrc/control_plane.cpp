@@ -195,10 +195,24 @@ bool KeyedLru::import_order(const uint64_t* keys, const int32_t* slots, int64_t 
 
 Admission::Admission(int32_t policy, int32_t kappa_blocks, int32_t theta_percent,
                      int64_t window_ms, int32_t len_window, int32_t telemetry,
-                     int64_t host_blocks, int32_t block_size)
+                     int64_t host_blocks, int32_t block_size, int64_t report_period_ms,
+                     int64_t report_max_age_ms)
     : policy_(policy), kappa_(kappa_blocks), theta_percent_(theta_percent),
       telemetry_(telemetry), window_ms_(window_ms), host_blocks_(host_blocks),
+      period_ms_(report_period_ms), max_age_ms_(report_max_age_ms),
       len_window_(len_window), block_size_(block_size), length_sum_(0) {}
+
+void Admission::publish(int64_t now_ms, int64_t resident_now) {
+    if (period_ms_ <= 0) return;
+    const int64_t t = now_ms / period_ms_ * period_ms_;
+    if (t < period_ms_ || t <= report_time_) return;
+    // every earlier request came before t, so the tier as it stands is what that publication saw
+    int64_t e = 0;
+    for (int64_t x : evict_times_) e += (x > t - window_ms_ && x < t);
+    report_time_ = t;
+    report_resident_ = resident_now;
+    report_evicted_ = e;
+}
 
 bool Admission::pressure(int64_t agent, int64_t n_tokens, int64_t now_ms, int64_t resident_now) {
     agent_last_[agent] = now_ms;
@@ -219,6 +233,12 @@ bool Admission::pressure(int64_t agent, int64_t n_tokens, int64_t now_ms, int64_
     const __int128 rhs = (__int128)host_blocks_ * block_size_ * (__int128)lengths_.size();
     const bool estimate = lhs > rhs;
     if (!telemetry_) return estimate;
+    if (period_ms_ > 0) {
+        const bool fresh = report_time_ >= 0 && (max_age_ms_ <= 0 || now_ms - report_time_ <= max_age_ms_);
+        if (!fresh) return estimate;
+        return estimate && (__int128)100 * report_resident_ >= (__int128)theta_percent_ * host_blocks_ &&
+               report_evicted_ > 0;
+    }
     const bool full = (__int128)100 * resident_now >= (__int128)theta_percent_ * host_blocks_;
     const bool evicting = !evict_times_.empty();
     return estimate && full && evicting;
@@ -233,6 +253,9 @@ int64_t Admission::export_state(int64_t* out, int64_t capacity) const {
     for (int64_t x : lengths_) v.push_back(x);
     v.push_back((int64_t)evict_times_.size());
     for (int64_t x : evict_times_) v.push_back(x);
+    v.push_back(report_time_);
+    v.push_back(report_resident_);
+    v.push_back(report_evicted_);
     for (size_t i = 0; i < v.size() && (int64_t)i < capacity; ++i) out[i] = v[i];
     return (int64_t)v.size();
 }
@@ -257,12 +280,17 @@ bool Admission::import_state(const int64_t* in, int64_t n) {
         lengths.push_back(x);
         sum += x;
     }
-    if (!take(&ne) || ne < 0 || ne != n - i) return false;
+    if (!take(&ne) || ne < 0 || ne != n - i - 3) return false;
     for (int64_t k = 0; k < ne; ++k) {
         int64_t x = 0;
         if (!take(&x)) return false;
         evs.push_back(x);
     }
+    int64_t rt = -1, rr = 0, re = 0;
+    if (!take(&rt) || !take(&rr) || !take(&re) || rt < -1 || rr < 0 || re < 0) return false;
+    report_time_ = rt;
+    report_resident_ = rr;
+    report_evicted_ = re;
     agent_last_.swap(agents);
     lengths_.swap(lengths);
     length_sum_ = sum;

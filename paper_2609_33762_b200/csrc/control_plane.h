@@ -79,10 +79,18 @@ private:
 //   estimate  (A_t - 1) * sum(len) > K_H * b * count     (beta cancels, C_H = K_H b beta)
 //   full      100 * resident >= theta_percent * K_H
 //   evicting  evictions in (now - window, now] > 0
+// With a report period the last two are read from the latest published report instead, if one
+// exists and is not older than the maximum age; otherwise the estimate alone decides.
 class Admission {
 public:
     Admission(int32_t policy, int32_t kappa_blocks, int32_t theta_percent, int64_t window_ms,
-              int32_t len_window, int32_t telemetry, int64_t host_blocks, int32_t block_size);
+              int32_t len_window, int32_t telemetry, int64_t host_blocks, int32_t block_size,
+              int64_t report_period_ms = 0, int64_t report_max_age_ms = 0);
+    // Published tier reports (report_period_ms = P > 0): call before a request at now_ms changes
+    // the tier.  If a publication time P, 2P, ... has passed since the latest report, the tier as
+    // it stands (resident_now chunks, evictions inside the window before that time) becomes the
+    // report of floor(now / P) * P.
+    void publish(int64_t now_ms, int64_t resident_now);
     // registers the request (agent activity, prompt length), expires old evictions and
     // returns p_t; call once per request before the walk
     bool pressure(int64_t agent, int64_t n_tokens, int64_t now_ms, int64_t resident_now);
@@ -90,7 +98,7 @@ public:
     int32_t kappa() const { return kappa_; }
     // The windows as a flat list of int64: n_agents, (agent, last time) pairs in ascending agent
     // order, n_lengths, the prompt lengths oldest first, n_evictions, the eviction times oldest
-    // first.  export_state returns the number of values (at most `capacity` are written);
+    // first, then the latest published report (time or -1, resident chunks, evictions).  export_state returns the number of values (at most `capacity` are written);
     // import_state replaces the windows and returns false (nothing changed) on a malformed list.
     int64_t export_state(int64_t* out, int64_t capacity) const;
     bool import_state(const int64_t* in, int64_t n);
@@ -98,6 +106,8 @@ public:
 private:
     int32_t policy_, kappa_, theta_percent_, telemetry_;
     int64_t window_ms_, host_blocks_;
+    int64_t period_ms_, max_age_ms_;
+    int64_t report_time_ = -1, report_resident_ = 0, report_evicted_ = 0;   // latest report; time -1: none yet
     int32_t len_window_, block_size_;
     std::unordered_map<int64_t, int64_t> agent_last_;
     std::deque<int64_t> lengths_;

@@ -446,6 +446,7 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
         cfg->gpu_free_order < 0 || cfg->gpu_free_order > 1)
         return EAKV_E_INVAL;
     if (cfg->gpu_index_blocks < 0 || cfg->gpu_index_blocks > cfg->gpu_blocks) return EAKV_E_INVAL;
+    if (cfg->telemetry_period_ms < 0 || cfg->telemetry_max_age_ms < 0) return EAKV_E_INVAL;
     const int64_t piece = (int64_t)cfg->block_size * cfg->kv_heads * cfg->head_dim * cfg->elem_bytes;
     if (piece % 16 != 0) return EAKV_E_INVAL;
     const int pieces = 2 * cfg->num_layers;
@@ -531,7 +532,8 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
         ctx->gpu_tier = new KeyedLru(cfg->gpu_index_blocks ? cfg->gpu_index_blocks : cfg->gpu_blocks);
         ctx->adm = new Admission(cfg->policy, cfg->kappa_blocks, cfg->theta_percent, cfg->window_ms,
                                  cfg->len_window > 0 ? cfg->len_window : 256, cfg->telemetry,
-                                 cfg->host_blocks, cfg->block_size * (int32_t)chunk_blocks);
+                                 cfg->host_blocks, cfg->block_size * (int32_t)chunk_blocks,
+                                 cfg->telemetry_period_ms, cfg->telemetry_max_age_ms);
         ctx->slot_stamp.assign((size_t)ctx->tier_slots, 0);
         ctx->blk_stamp.assign((size_t)cfg->gpu_blocks, 0);
     } catch (const std::bad_alloc&) {
@@ -837,6 +839,7 @@ static int tier_step_impl(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_
     if (want_evicted && (!n_evicted_inout || *n_evicted_inout < n_blocks)) return EAKV_E_CAPACITY;
 
     KeyedLru& T = *ctx->host_tier;
+    ctx->adm->publish(now_ms, T.resident());
     int64_t H = 0;
     while (H < n_blocks && T.find(hashes_host[H]) >= 0) ++H;
     const bool first = decided < 0;

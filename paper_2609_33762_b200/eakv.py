@@ -45,6 +45,7 @@ class Config(C.Structure):
         ("control_plane_only", C.c_int32), ("chunk_blocks", C.c_int32),
         ("tier_memory", C.c_void_p),
         ("gpu_free_order", C.c_int32), ("write_behind", C.c_int32),
+        ("telemetry_period_ms", C.c_int64), ("telemetry_max_age_ms", C.c_int64),
     ]
 
 
@@ -226,7 +227,8 @@ class Context:
                  tier_location=TIER_PINNED_HOST, copy_path=COPY_BULK, copy_ctas=0,
                  staging_bytes=0, max_call_blocks=0, hash_scratch_blocks=0, min_staged_run_bytes=0,
                  tier_memory=0, control_plane_only=False, chunk_blocks=1,
-                 gpu_free_order=FREE_ASCENDING, write_behind=False):
+                 gpu_free_order=FREE_ASCENDING, write_behind=False, telemetry_period_ms=0,
+                 telemetry_max_age_ms=0):
         L = lib()
         cfg = Config()
         L.eakv_config_init(C.byref(cfg))
@@ -242,6 +244,7 @@ class Context:
         cfg.chunk_blocks = int(chunk_blocks)
         cfg.gpu_free_order = int(gpu_free_order)
         cfg.write_behind = int(bool(write_behind))
+        cfg.telemetry_period_ms, cfg.telemetry_max_age_ms = int(telemetry_period_ms), int(telemetry_max_age_ms)
         cfg.hash_base, cfg.hash_seed = hash_base, hash_seed
         cfg.policy, cfg.kappa_blocks, cfg.theta_percent = policy, kappa_blocks, theta_percent
         cfg.len_window, cfg.window_ms, cfg.telemetry = len_window, window_ms, telemetry

@@ -39,8 +39,31 @@ def test_config_defaults_and_layout(lib):
     assert (cfg.theta_percent, cfg.window_ms, cfg.len_window, cfg.kappa_blocks) == (95, 60000, 256, 8)
     assert cfg.policy == eakv.POLICY_WRITE_ALL and cfg.elem_bytes == 2
     assert cfg.link_strategy == eakv.LINK_STAGED and cfg.copy_path == eakv.COPY_BULK
-    assert C.sizeof(eakv.Config) == 176 and C.sizeof(eakv.Stats) == 128
     assert lib.eakv_config_init(None) == eakv.E_INVAL
+
+
+def test_binding_structs_have_the_layout_of_the_header(tmp_path):
+    """include/eakv.h compiles as plain C, and the ctypes mirrors of its structs have the same
+    sizes and field offsets as a C compiler gives them."""
+    import subprocess
+    from paper_2609_33762_b200 import eakv
+    src = tmp_path / "layout.c"
+    src.write_text(
+        '#include <stdio.h>\n#include <stddef.h>\n#include "eakv.h"\n'
+        'int main(void) {\n'
+        '  printf("%zu %zu %zu %zu\\n", sizeof(eakv_config), sizeof(eakv_stats), sizeof(eakv_step_info), sizeof(eakv_turn_view));\n'
+        '  printf("%zu %zu %zu %zu %zu\\n", offsetof(eakv_config, kv_base), offsetof(eakv_config, window_ms),\n'
+        '         offsetof(eakv_config, tier_memory), offsetof(eakv_config, telemetry_period_ms),\n'
+        '         offsetof(eakv_turn_view, keys));\n'
+        '  return 0;\n}\n')
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)],
+                   check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split()
+    sizes, offsets = [int(x) for x in out[:4]], [int(x) for x in out[4:]]
+    assert sizes == [C.sizeof(eakv.Config), C.sizeof(eakv.Stats), C.sizeof(eakv.StepInfo), C.sizeof(eakv.TurnView)]
+    assert offsets == [eakv.Config.kv_base.offset, eakv.Config.window_ms.offset, eakv.Config.tier_memory.offset,
+                       eakv.Config.telemetry_period_ms.offset, eakv.TurnView.keys.offset]
 
 
 def test_strerror(lib):

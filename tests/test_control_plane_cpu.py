@@ -399,3 +399,83 @@ def test_random_traces_across_every_option(eakv):
         recs = drive_chunked(ctx, trace, shape.block_size, R) if R > 1 else drive(ctx, trace, shape.block_size)
         compare(recs, orc.records)
         ctx.close()
+
+
+@pytest.mark.parametrize("period,max_age", [(1, 5), (10, 0), (10, 25), (100, 50), (1000, 5000)])
+def test_published_reports_random_requests(eakv, period, max_age):
+    """Tier reports published at intervals (Appendix D): capacity-conditioned admission that reads
+    the latest report, fresh or stale, against the oracle on random request streams."""
+    rng = random.Random(300 + period + max_age)
+    engaged = stale = 0
+    for case in range(40):
+        K = rng.randrange(3, 40)
+        b = rng.choice([1, 4, 16])
+        kw = dict(policy=2, kappa_blocks=rng.choice([0, 1, 2, 5]), theta_percent=rng.choice([50, 95, 100]),
+                  window_ms=rng.choice([50, 400, 10_000]), len_window=rng.choice([1, 3, 256]),
+                  telemetry_period_ms=period, telemetry_max_age_ms=max_age)
+        ctx = cp_ctx(eakv, b, 8, K, **kw)
+        tier = HostTier(K, b, **kw)
+        now = 0
+        for _ in range(rng.randrange(5, 80)):
+            agent = rng.randrange(5)
+            n = rng.randrange(0, K + 1)
+            keys = [1000 * agent + rng.randrange(0, 4) + j for j in range(n)]
+            n_tokens = n * b + rng.randrange(0, b)
+            now += rng.choice([0, 1, 7, 100, 3 * period])
+            decided = None if rng.random() < 0.85 else (rng.random() < 0.5)
+            want = tier.step(keys, n_tokens, agent, now, decided=decided)
+            got = ctx.eakv_tier_step(as_keys(keys), agent, n_tokens, now, decided=decided)
+            assert got["hit"].tolist() == want.hit and got["admit"].tolist() == want.admit
+            assert got["slot"].tolist() == want.slot
+            assert (got["pressure"], got["save"]) == (want.pressure, want.save)
+            engaged += want.pressure
+            stale += tier.report is not None and max_age > 0 and now - tier.report[0] > max_age
+        ctx.close()
+    assert engaged > 0
+    if 0 < max_age < period:
+        assert stale > 0
+
+
+def test_scaled_config2_trace_with_the_papers_report_interval(eakv):
+    """Config 2's generator scaled down, capacity-conditioned admission reading reports published
+    every second that stay fresh for five (the paper's parameter table), whole trace against the
+    oracle; and the decisions differ from the synchronous reading somewhere, so the reports matter."""
+    cfg = replace(CONFIGS["c2"], shape="tiny", agents=8, turns=16, first_prompt=400,
+                  append_median=150.0, context_cap=3000, tool_gap_mean_ms=5_000.0)
+    shape = SHAPES["tiny"]
+    trace = make_trace(cfg, seed=31)
+    base = dict(policy=2, kappa_blocks=6, window_ms=60_000, len_window=32)
+    kw = dict(base, telemetry_period_ms=1000, telemetry_max_age_ms=5000)
+    oracle = TraceOracle(shape, 256, 300, **kw)
+    oracle.run(trace)
+    ctx = cp_ctx(eakv, shape.block_size, 256, 300, **kw)
+    compare(drive(ctx, trace, shape.block_size), oracle.records)
+    ctx.close()
+    sync = TraceOracle(shape, 256, 300, **base)
+    sync.run(trace)
+    assert [r["pressure"] for r in sync.records] != [r["pressure"] for r in oracle.records]
+    assert oracle.host.stats["declined_requests"] > 0
+
+
+def test_admission_export_carries_the_latest_report(eakv):
+    kw = dict(policy=2, kappa_blocks=0, theta_percent=50, window_ms=60_000, telemetry_period_ms=1000,
+              telemetry_max_age_ms=5000)
+    ctx = cp_ctx(eakv, 4, 8, 4, **kw)
+    tier = HostTier(4, 4, **kw)
+    steps = [([1, 2, 3, 4], 40, 0, 100), ([5, 6], 40, 1, 1500), ([1, 2], 40, 0, 1900), ([7], 40, 1, 2100)]
+    for keys, n, agent, now in steps:
+        tier.step(keys, n, agent, now)
+        ctx.eakv_tier_step(as_keys(keys), agent, n, now)
+    assert tier.report == (2000, 4, 4)
+    state = ctx.eakv_admission_export()
+    assert state[-3:].tolist() == [2000, 4, 4]
+    k, s = ctx.eakv_tier_export()
+    ctx.close()
+    ctx = cp_ctx(eakv, 4, 8, 4, **kw)
+    ctx.eakv_tier_import(k, s)
+    ctx.eakv_admission_import(state)
+    # 2,900 ms: still the report of 2,000 ms, which the restarted context can only know from the import
+    want = tier.step([8], 40, 0, 2900)
+    got = ctx.eakv_tier_step(as_keys([8]), 0, 40, 2900)
+    assert want.pressure and got["pressure"] and not got["save"]
+    ctx.close()
