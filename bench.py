@@ -775,8 +775,19 @@ def main():
     if args.impl == "reference":
         run_reference(args)
         return
+    if args.gpus < 1:
+        raise SystemExit("--gpus must be at least 1")
 
     import torch
+    from paper_2609_33762_b200.multi import launched, spawn_local_ranks
+    if args.gpus > 1 and not launched():
+        # no launcher: start the N replicas here, one process per GPU; rank 0 prints the line
+        have = torch.cuda.device_count() if torch.cuda.is_available() else 0
+        if have < args.gpus:
+            raise SystemExit(f"bench.py --gpus {args.gpus}: this machine has {have} CUDA device(s); "
+                             "the eakv path has no CPU fallback")
+        sys.exit(spawn_local_ranks([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], args.gpus))
+
     from eakv_workloads import SHAPES
     from paper_2609_33762_b200 import eakv
     from paper_2609_33762_b200.harness import PagedPool

@@ -8,10 +8,14 @@ import os
 
 
 def init_distributed(expected_world: int, backend: str | None = None):
-    """Join the process group torchrun set up; returns (rank, world, local_rank, dist|None)."""
+    """Join the process group the launcher set up (torchrun, or spawn_local_ranks below); returns
+    (rank, world, local_rank, dist|None).  The launcher's WORLD_SIZE must be the number of
+    replicas the caller asked for: a mismatch raises instead of silently running another count."""
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if expected_world and expected_world != world:
+        raise RuntimeError(f"{expected_world} replicas were asked for but the launcher set WORLD_SIZE={world}")
     if world <= 1:
         return 0, 1, local_rank, None
     import torch
@@ -22,9 +26,45 @@ def init_distributed(expected_world: int, backend: str | None = None):
     if backend == "nccl":
         torch.cuda.set_device(local_rank)
     dist.init_process_group(backend=backend, rank=rank, world_size=world)
-    if expected_world and expected_world != world:
-        raise RuntimeError(f"--gpus {expected_world} but WORLD_SIZE={world}")
     return rank, world, local_rank, dist
+
+
+def launched() -> bool:
+    """Did a launcher (torchrun or spawn_local_ranks) start this process as one rank of several?"""
+    return "WORLD_SIZE" in os.environ and "RANK" in os.environ
+
+
+def spawn_local_ranks(argv, n_ranks: int, timeout_s: float | None = None) -> int:
+    """Run ``argv`` (a command line) as ``n_ranks`` local processes, one replica each, with the
+    rendezvous variables a launcher would set (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR =
+    127.0.0.1, a free MASTER_PORT).  Rank 0 inherits this process's stdout, so its single result
+    line is this command's; the other ranks' stdout is dropped, every rank's stderr passes through.
+    Returns the largest exit code (a rank that had to be killed counts as 1).  No data-path
+    collective is involved anywhere: the replicas only meet at barriers and at the final max/sum."""
+    import socket
+    import subprocess
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs = []
+    for rank in range(n_ranks):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n_ranks),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen(list(argv), env=env, stdout=None if rank == 0 else subprocess.DEVNULL))
+    worst = 0
+    try:
+        for p in procs:
+            rc = p.wait(timeout=timeout_s)
+            worst = max(worst, rc if rc >= 0 else 1)
+    except subprocess.TimeoutExpired:
+        worst = 1
+    finally:
+        for p in procs:                 # exactly the processes started here, by handle
+            if p.poll() is None:
+                p.kill()
+                p.wait()
+                worst = max(worst, 1)
+    return worst
 
 
 def aggregate_over_ranks(dist, elapsed_ms: float, units: float, device=None):

@@ -121,3 +121,81 @@ def test_tensor_parallel_ranks_take_the_same_decisions(tmp_path):
     for g in got:
         assert g["heads"] == 1 and g["block_bytes"] == full.block_size * beta == full.block_bytes // 2
         assert g["kh"] == sizing.tier_chunks(4 << 20, full.block_size, beta)
+
+
+SPAWNED = textwrap.dedent("""
+    import json, os, sys
+    sys.path.insert(0, %r)
+    from paper_2609_33762_b200.multi import aggregate_over_ranks, init_distributed, launched
+    assert launched()
+    rank, world, local_rank, dist = init_distributed(int(sys.argv[1]), backend="gloo")
+    dist.barrier()
+    ms, units = aggregate_over_ranks(dist, 1.0 + rank, 10.0)
+    dist.barrier()
+    if rank == 0:
+        print(json.dumps(dict(world=world, ms=ms, units=units, local_rank=local_rank)))
+    else:
+        print("a line from another rank that must not reach the caller's stdout")
+    dist.destroy_process_group()
+    sys.exit(int(sys.argv[2]) if rank == 1 else 0)
+""") % ROOT
+
+SPAWNER = textwrap.dedent("""
+    import sys
+    sys.path.insert(0, %r)
+    from paper_2609_33762_b200.multi import spawn_local_ranks
+    sys.exit(spawn_local_ranks([sys.executable, sys.argv[1], sys.argv[2], sys.argv[3]], int(sys.argv[2])))
+""") % ROOT
+
+
+def test_spawned_local_ranks_rendezvous_and_only_rank0_prints(tmp_path):
+    """The path `bench.py --gpus N` takes without a launcher, with a stub in place of the arm: N
+    local ranks meet over gloo, rank 0's line is the only output, the worst exit code comes back."""
+    import json
+    worker, spawner = tmp_path / "spawned.py", tmp_path / "spawner.py"
+    worker.write_text(SPAWNED)
+    spawner.write_text(SPAWNER)
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, str(spawner), str(worker), "3", "0"], env=env, capture_output=True,
+                         text=True, timeout=180)
+    assert out.returncode == 0, out.stderr
+    lines = [ln for ln in out.stdout.splitlines() if ln.strip()]
+    assert len(lines) == 1
+    assert json.loads(lines[0]) == dict(world=3, ms=3.0, units=30.0, local_rank=0)
+    # a failing rank makes the whole command fail
+    out = subprocess.run([sys.executable, str(spawner), str(worker), "2", "7"], env=env, capture_output=True,
+                         text=True, timeout=180)
+    assert out.returncode == 7
+
+
+def test_world_size_mismatch_is_an_error():
+    from paper_2609_33762_b200.multi import init_distributed
+    import pytest
+    saved = {k: os.environ.get(k) for k in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    try:
+        os.environ.update(WORLD_SIZE="1", RANK="0", LOCAL_RANK="0")
+        with pytest.raises(RuntimeError, match="WORLD_SIZE=1"):
+            init_distributed(8)                      # asked for 8, launched as 1: used to run one replica silently
+        for k in saved:
+            os.environ.pop(k, None)
+        with pytest.raises(RuntimeError, match="WORLD_SIZE=1"):
+            init_distributed(2)                      # no launcher at all
+    finally:
+        for k, v in saved.items():
+            if v is None:
+                os.environ.pop(k, None)
+            else:
+                os.environ[k] = v
+
+
+def test_bench_gpus_2_without_devices_fails_loudly():
+    """On a machine without CUDA devices `bench.py --gpus 2` must not print a one-replica line."""
+    import torch
+    if torch.cuda.is_available() and torch.cuda.device_count() >= 2:
+        import pytest
+        pytest.skip("this machine has the devices")
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1"],
+                         env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode != 0
+    assert "CUDA device" in out.stderr and not out.stdout.strip()
