@@ -381,6 +381,29 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
 int eakv_turn_end(eakv_ctx* ctx, void* cuda_stream);
 int eakv_turn_abort(eakv_ctx* ctx);
 
+/* The same turn for an engine that runs several requests at once (Section 2: the engine's cap on
+ * running requests; Appendix A: 16) and suspends one when GPU KV memory runs out.  Any number of
+ * requests may be open, each under a request_id of the caller's choosing.
+ * eakv_request_begin: as eakv_turn_begin, but the prompt's GPU blocks are taken with
+ * eakv_gpu_tier_acquire and stay pinned under request_id.  EAKV_E_CAPACITY, with neither tier
+ * changed, when they do not fit beside the running requests: wait, or suspend a running request
+ * (eakv_request_release) and try again.  decided: -1 for the request's first lookup; 0 / 1 for a
+ * later lookup of a resumed request, carrying the skip / store choice of its first one (Appendix D;
+ * see eakv_tier_step_again).  *view's arrays stay valid until the request is released.
+ * eakv_request_store: after the engine has produced the blocks flagged needs_fill, eakv_store of
+ * the admitted blocks on cuda_stream (deferred under eakv_config.write_behind); once per begin.
+ * eakv_request_release: the request finished or is suspended: its blocks become evictable
+ * (eakv_gpu_tier_release_request) and its tail block is freed.  Released before its store -- the
+ * engine never produced the KV -- it is taken back like an aborted turn.
+ * Errors: EAKV_E_INVAL for a request_id that is already open (begin) or not open (store, release),
+ * for a second store, and while a single turn (eakv_turn_begin) is open; failures after the
+ * bookkeeping are handled as in eakv_turn_begin / eakv_turn_end and close the request. */
+int eakv_request_begin(eakv_ctx* ctx, int64_t request_id, const int32_t* tokens, int64_t n_tokens,
+                       const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
+                       int32_t decided, void* cuda_stream, eakv_turn_view* view);
+int eakv_request_store(eakv_ctx* ctx, int64_t request_id, void* cuda_stream);
+int eakv_request_release(eakv_ctx* ctx, int64_t request_id);
+
 /* Layer-pipelined restore (Section 3.1, Eq. 2: the fixed restoration overhead tau_load is
  * what a consumer waits for before it can start; moving layers in order lets it start on
  * the first ones while the rest are in flight).  Same result as eakv_load, but the 2L
@@ -420,6 +443,46 @@ int eakv_capacity_curve(const int64_t* dist_dev, int64_t n_refs, const int64_t* 
                         int64_t n_requests, int32_t block_size, const int64_t* capacities_host,
                         int32_t n_capacities, int64_t* hits_out, int64_t* restored_out,
                         int64_t* computed_out, int64_t* cover_out, void* cuda_stream);
+
+/* Declined-chunk audit (Appendix D, "Reuse distance of declined chunks"; Proposition 1): of the
+ * references whose miss an admission policy declined, how many could be declined at no cost --
+ * their chunk is referenced next at reuse distance D >= capacity, or never again.
+ *   keys_dev      device uint64[n_refs], the tier's reference stream (values below 2^61)
+ *   declined_dev  device uint8[n_refs], non-zero where the miss was declined
+ *   capacity      K_H in tier units
+ *   declined_out, meets_out, never_out  host: declined references, those meeting the condition,
+ *                 those never referenced again (counted in meets_out too)
+ *   next_dist_dev device int64[n_refs] or NULL: per reference, D of the next reference to its
+ *                 chunk if it was declined (-1: never referenced again), -2 if it was not declined
+ * Context-free; allocates its scratch (as eakv_reuse_distances, plus 12 bytes per reference) and
+ * frees it before returning; returns after the stream has finished.  Errors as eakv_reuse_distances. */
+int eakv_declined_audit(const uint64_t* keys_dev, const uint8_t* declined_dev, int64_t n_refs,
+                        int64_t capacity, int64_t* declined_out, int64_t* meets_out, int64_t* never_out,
+                        int64_t* next_dist_dev, void* cuda_stream);
+
+/* Sizing arithmetic of Section 2 and Section 3.2 in integers (host only, no CUDA call):
+ * beta_rank = 2 L d s max(1, ceil(H_kv / TP)) (Eq. 1); the working-set scale
+ * C_reuse = (A - 1) * N_bar * beta_rank (Eq. 5) with N_bar = total_prompt_tokens / n_requests kept
+ * as a fraction until the final floor; the pressure ratios gamma_G = A * N_bar / K_G with
+ * K_G = gpu_blocks * block_size tokens and gamma_H = C_reuse / C_H with
+ * C_H = host_blocks * block_size * beta_rank.  The two flags compare the fractions exactly
+ * (gamma > 1); the doubles are for display.  A zero gpu_blocks / host_blocks leaves its ratio 0. */
+typedef struct eakv_working_set_in {
+    int32_t num_layers, kv_heads, head_dim, elem_bytes, tensor_parallel, block_size;
+    int64_t active_pool;             /* A                                         */
+    int64_t total_prompt_tokens;     /* sum of the prompt lengths of n_requests   */
+    int64_t n_requests;
+    int64_t gpu_blocks, host_blocks; /* K_G and K_H in blocks of block_size       */
+} eakv_working_set_in;
+typedef struct eakv_working_set_out {
+    int64_t beta_rank_bytes;         /* Eq. 1                                     */
+    int64_t working_set_bytes;       /* Eq. 5, floor                              */
+    int64_t working_set_blocks;      /* floor(C_reuse / (block_size * beta_rank)) */
+    double gamma_g, gamma_h;
+    int32_t pool_exceeds_gpu;        /* gamma_G > 1                               */
+    int32_t working_set_exceeds_host;/* gamma_H > 1                               */
+} eakv_working_set_out;
+int eakv_working_set(const eakv_working_set_in* in, eakv_working_set_out* out);
 
 /* Block keys without a context and without any allocation.  (The paper has no counterpart;
  * this exists for callers that cannot request device memory: code living inside a serving

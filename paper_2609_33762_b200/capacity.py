@@ -128,14 +128,23 @@ def model(config, host_gib, device="cuda:0", limit=None, agents=None, shared_pre
     finite = dist[:n_refs][dist[:n_refs] >= 0]
     ws_full = int(finite.max().item()) + 1 if finite.numel() else 0
     ws_99 = working_set_within(dist.data_ptr(), n_refs, offsets, tokens, G, shape.block_size, ws_full)
-    n_mean = trace.total_prompt_tokens / len(trace.requests)
-    ws_eq5 = int((len(trace.agent_tokens) - 1) * n_mean * shape.bytes_per_token // shape.block_bytes)
+    # Eq. 5 and the pressure ratios of Section 3.2, integer arithmetic in the library
+    sizing = eakv.eakv_working_set(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+                                   elem_bytes=shape.elem_bytes, block_size=shape.block_size,
+                                   active_pool=len(trace.agent_tokens),
+                                   total_prompt_tokens=trace.total_prompt_tokens, n_requests=len(trace.requests),
+                                   gpu_blocks=cfg.gpu_blocks, host_blocks=0)
+    ws_eq5 = sizing["working_set_blocks"]
     inf_computed = int(out["computed_tokens"][-1])
     rows = []
     for c, g in enumerate(host_gib):
         rows.append({"host_gib": g, "blocks": caps[c], "hits": int(out["hits"][c]),
                      # gamma_H = C_reuse / C_H (Section 3.2), with C_reuse the Eq. 5 scale
-                     "gamma_h": ws_eq5 / caps[c],
+                     "gamma_h": eakv.eakv_working_set(
+                         num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+                         elem_bytes=shape.elem_bytes, block_size=shape.block_size,
+                         active_pool=len(trace.agent_tokens), total_prompt_tokens=trace.total_prompt_tokens,
+                         n_requests=len(trace.requests), host_blocks=caps[c])["gamma_h"],
                      "restored_tokens": int(out["restored_blocks"][c]) * shape.block_size,
                      "computed_prefill_tokens": int(out["computed_tokens"][c])})
     return {"config": config, "agents": len(trace.agent_tokens), "shared_prefix_tokens": shared_prefix,
@@ -145,7 +154,7 @@ def model(config, host_gib, device="cuda:0", limit=None, agents=None, shared_pre
             "prompt_tokens": int(tokens.sum()), "rows": rows,
             "computed_prefill_tokens_infinite_tier": inf_computed,
             # gamma_G = A * N_bar / K_G (Section 3.2), K_G in tokens
-            "gamma_g": len(trace.agent_tokens) * n_mean / (cfg.gpu_blocks * shape.block_size),
+            "gamma_g": sizing["gamma_g"],
             "working_set_blocks": {"eq5": ws_eq5, "full": ws_full, "within_1_percent": ws_99},
             "working_set_gib": {"eq5": ws_eq5 * shape.block_bytes / GIB, "full": ws_full * shape.block_bytes / GIB,
                                 "within_1_percent": ws_99 * shape.block_bytes / GIB},
@@ -189,19 +198,14 @@ def audit(config, policy, host_gib, kappa=None, chunk_blocks=1, device="cuda:0",
     ctx.close()
     n = len(cstream)
     cdev = torch.from_numpy(cstream.view(np.int64)).to(device)
-    dist = torch.empty(max(n, 1), dtype=torch.int64, device=device)
-    eakv.eakv_reuse_distances(cdev.data_ptr(), n, dist.data_ptr())
-    D = dist[:n].cpu().numpy()
-    # next reference of every position: stable sort by key, neighbours to the right
-    order = np.argsort(cstream, kind="stable")
-    nxt = np.full(n, -1, dtype=np.int64)
-    same = cstream[order][1:] == cstream[order][:-1]
-    nxt[order[:-1][same]] = order[1:][same]
-    idx = np.nonzero(declined)[0]
-    nx = nxt[idx]
-    never = int((nx < 0).sum())
-    d_next = D[nx[nx >= 0]]
-    meets = never + int((d_next >= kh).sum())
+    ddev = torch.from_numpy(declined.astype(np.uint8)).to(device)
+    next_dist = torch.empty(max(n, 1), dtype=torch.int64, device=device)
+    # the audit itself (reuse distances, next references, the condition of Proposition 1) runs in the library
+    n_declined, meets, never = eakv.eakv_declined_audit(cdev.data_ptr(), ddev.data_ptr(), n, kh,
+                                                        next_dist.data_ptr())
+    nd = next_dist[:n]
+    d_next = nd[nd >= 0].cpu().numpy()             # declined chunks that are referenced again: their D
+    idx = range(n_declined)
     return {"config": config, "policy": policy, "host_gib": host_gib, "tier_units": kh, "chunk_blocks": R,
             "kappa": kap, "declined_chunks": int(len(idx)), "meet_condition": meets,
             "share_meeting_condition": meets / len(idx) if len(idx) else None,

@@ -45,6 +45,20 @@ struct Staging {
 
 }  // namespace
 
+namespace {
+constexpr int64_t kNoRequest = INT64_MIN;       // the single-turn calls are not bound to a request id
+
+// what one open turn registered: its keys, both tiers' decisions, the per-block store plan
+struct TurnState {
+    std::vector<uint64_t> keys, unit_keys, evicted_keys;
+    std::vector<int32_t> block, slot_u, slot_b, evicted_slots, host_slots;
+    std::vector<uint8_t> resident, fill, hit, admit_u, admit_b;
+    int64_t request_id = kNoRequest;
+    int32_t tail = -1;
+    bool open = false, stored = false;
+};
+}  // namespace
+
 struct eakv_ctx {
     eakv_config cfg;
     int device = 0;
@@ -108,13 +122,8 @@ struct eakv_ctx {
     std::vector<uint8_t> wb_slots;      // by tier slot: a pending write still fills it
     uint64_t* turn_keys = nullptr;            // pinned + mapped; the hash kernel writes it directly
     int64_t turn_keys_cap = 0;
-    bool turn_open = false;
-    int32_t turn_tail = -1;
-    std::vector<int32_t> t_block, t_slot_u, t_slot_b, t_evicted_slots, t_host_slots;
-    std::vector<uint8_t> t_resident, t_fill, t_hit, t_admit_u, t_admit_b;
-    std::vector<uint64_t> t_unit_keys, t_evicted_keys, t_keys_host;
-    const uint64_t* t_keys = nullptr;         // the open turn's block keys and tier-unit keys
-    const uint64_t* t_ukeys = nullptr;
+    TurnState turn;                            // the one open turn of eakv_turn_begin / eakv_turn_end
+    std::unordered_map<int64_t, TurnState> requests;   // open turns of running requests (eakv_request_*)
 
     std::string cuda_err;
 };
@@ -1150,45 +1159,50 @@ int eakv_load_layers(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* bl
 }
 
 // ------------------------------------------------------------------------------------------
-// one turn in two calls
+// turns: one at a time (eakv_turn_*), or several running requests at once (eakv_request_*)
 // ------------------------------------------------------------------------------------------
 namespace {
 
 // Take back what an open turn registered but will never produce.  host_units: the tier units the
 // turn admitted leave the host index (their slots were never written).  gpu_mode 1: every GPU
 // block the turn newly keyed leaves the GPU index (nothing was restored or computed); 2: only
-// those the engine was to fill (the restored ones hold their bytes).  Promotions and evictions
-// the turn caused stand.  Releases the tail block and closes the turn.
-void withdraw_turn(eakv_ctx* ctx, bool host_units, int gpu_mode) {
+// those the engine was to fill (the restored ones hold their bytes).  A block another running
+// request shares stays.  Promotions and evictions the turn caused stand.  Lets the turn's GPU
+// blocks go (pins, tail block).
+void withdraw_turn(eakv_ctx* ctx, TurnState& T, bool host_units, int gpu_mode) {
     if (host_units) {
         int64_t n = 0;
+        const uint64_t* ukeys = T.unit_keys.empty() ? T.keys.data() : T.unit_keys.data();
         // last admitted first, so that the free stack hands the slots out again in the same order
-        for (size_t c = ctx->t_admit_u.size(); c-- > 0;)
-            if (ctx->t_admit_u[c] && ctx->host_tier->erase(ctx->t_ukeys[c]) >= 0) ++n;
+        for (size_t c = T.admit_u.size(); c-- > 0;)
+            if (T.admit_u[c] && ctx->host_tier->erase(ukeys[c]) >= 0) ++n;
         ctx->stats.admitted -= n;
         ctx->stats.resident = ctx->host_tier->resident();
     }
+    if (T.request_id != kNoRequest && ctx->held.count(T.request_id)) {
+        // the pins go first (without the tail: it is released below)
+        auto it = ctx->held.find(T.request_id);
+        it->second.tail = -1;
+        eakv_gpu_tier_release_request(ctx, T.request_id);
+    }
     if (gpu_mode) {
-        for (size_t j = ctx->t_block.size(); j-- > 0;) {
-            const bool drop = gpu_mode == 1 ? !ctx->t_resident[j] : ctx->t_fill[j] != 0;
-            if (drop) ctx->gpu_tier->erase(ctx->t_keys[j]);
+        for (size_t j = T.block.size(); j-- > 0;) {
+            const bool drop = gpu_mode == 1 ? !T.resident[j] : T.fill[j] != 0;
+            if (drop) ctx->gpu_tier->erase(T.keys[j]);
         }
     }
-    if (ctx->turn_tail >= 0) {
-        eakv_gpu_tier_release(ctx, ctx->turn_tail);
-        ctx->turn_tail = -1;
+    if (T.tail >= 0) {
+        eakv_gpu_tier_release(ctx, T.tail);
+        T.tail = -1;
     }
-    ctx->turn_open = false;
+    T.open = false;
 }
 
-}  // namespace
-
-int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
-                    const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
+// decided < 0: the request's first lookup; 0 / 1: a later lookup with that store/skip choice
+int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32_t* tokens, int64_t n_tokens,
+                    const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms, int decided,
                     void* cuda_stream, eakv_turn_view* view) {
-    if (!ctx || !view || n_tokens < 0 || n_known < 0) return EAKV_E_INVAL;
-    if (ctx->turn_open || !ctx->held.empty()) return EAKV_E_INVAL;
-    if (n_known > 0 && !known_keys) return EAKV_E_INVAL;
+    const bool as_request = request_id != kNoRequest;
     const bool bookkeeping_only = ctx->device < 0;
     const int b = ctx->cfg.block_size;
     const int64_t R = ctx->chunk_tokens / b;
@@ -1201,17 +1215,18 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
     if (nblk > n_known && !tokens) return EAKV_E_INVAL;
     // everything that can be refused without a CUDA error is refused here, before either tier changes
     if (nu > ctx->host_tier->capacity()) return EAKV_E_CAPACITY;
-    if (nblk + (need_tail ? 1 : 0) + ctx->gpu_unkeyed > ctx->gpu_tier->capacity()) return EAKV_E_CAPACITY;
+    if (!as_request && nblk + (need_tail ? 1 : 0) + ctx->gpu_unkeyed > ctx->gpu_tier->capacity())
+        return EAKV_E_CAPACITY;
     DeviceGuard g(bookkeeping_only ? -1 : ctx->device);
-    uint64_t* keys = nullptr;
-    if (bookkeeping_only) {
-        ctx->t_keys_host.assign(known_keys, known_keys + nblk);
-        keys = ctx->t_keys_host.data();
-    } else {
-        // key buffer in mapped pinned memory, grown in powers of two
-        if (nblk > ctx->turn_keys_cap) {
+    T.keys.resize((size_t)nblk);
+    uint64_t* keys = T.keys.data();
+    if (n_known > 0) std::memcpy(keys, known_keys, (size_t)n_known * 8);
+    if (nblk > n_known) {
+        // hash into mapped pinned memory (grown in powers of two), then keep a copy with the turn
+        const int64_t need = nblk - n_known;
+        if (need > ctx->turn_keys_cap) {
             int64_t cap = 4096;
-            while (cap < nblk) cap <<= 1;
+            while (cap < need) cap <<= 1;
             if (ctx->turn_keys) {
                 CU(cudaStreamSynchronize(ctx->lookup_stream));
                 CU(cudaFreeHost(ctx->turn_keys));
@@ -1227,59 +1242,61 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
             ctx->turn_keys_cap = cap;
         }
         if (!ctx->lookup_stream) CU(cudaStreamCreateWithFlags(&ctx->lookup_stream, cudaStreamNonBlocking));
-        keys = ctx->turn_keys;
-        if (n_known > 0) std::memcpy(keys, known_keys, (size_t)n_known * 8);
-        if (nblk > n_known) {
-            const uint64_t parent = n_known ? keys[n_known - 1] : ctx->seed;
-            int rc = eakv_hash_blocks(ctx, tokens + n_known * b, (nblk - n_known) * (int64_t)b, parent,
-                                      keys + n_known, nullptr, ctx->lookup_stream);
-            if (rc != EAKV_OK) return rc;
-            CU(cudaStreamSynchronize(ctx->lookup_stream));
-        }
+        const uint64_t parent = n_known ? keys[n_known - 1] : ctx->seed;
+        int rc = eakv_hash_blocks(ctx, tokens + n_known * b, need * (int64_t)b, parent, ctx->turn_keys, nullptr,
+                                  ctx->lookup_stream);
+        if (rc != EAKV_OK) return rc;
+        CU(cudaStreamSynchronize(ctx->lookup_stream));
+        std::memcpy(keys + n_known, ctx->turn_keys, (size_t)need * 8);
     }
     // tier units: one key per full chunk (the key at the chunk's last block)
     const uint64_t* ukeys = keys;
+    T.unit_keys.clear();
     if (R > 1) {
-        ctx->t_unit_keys.resize((size_t)nu);
-        for (int64_t c = 0; c < nu; ++c) ctx->t_unit_keys[c] = keys[c * R + R - 1];
-        ukeys = ctx->t_unit_keys.data();
+        T.unit_keys.resize((size_t)nu);
+        for (int64_t c = 0; c < nu; ++c) T.unit_keys[c] = keys[c * R + R - 1];
+        ukeys = T.unit_keys.data();
     }
-    ctx->t_block.resize((size_t)nblk); ctx->t_resident.resize((size_t)nblk);
-    ctx->t_fill.assign((size_t)nblk, 0);
-    ctx->t_hit.resize((size_t)nu); ctx->t_admit_u.assign((size_t)nu, 0); ctx->t_slot_u.resize((size_t)nu);
-    ctx->t_evicted_keys.resize((size_t)nu); ctx->t_evicted_slots.resize((size_t)nu);
-    ctx->t_host_slots.resize((size_t)nu);
+    T.block.resize((size_t)nblk); T.resident.resize((size_t)nblk);
+    T.fill.assign((size_t)nblk, 0);
+    T.hit.resize((size_t)nu); T.admit_u.assign((size_t)nu, 0); T.slot_u.resize((size_t)nu);
+    T.evicted_keys.resize((size_t)nu); T.evicted_slots.resize((size_t)nu);
+    T.host_slots.resize((size_t)nu);
+    T.request_id = request_id;
+    T.tail = -1;
+    T.stored = false;
+    // lookups (they change nothing), then the GPU side -- a running request whose blocks do not fit
+    // beside the others is refused here with both tiers untouched -- then the host tier
     int64_t G = 0, G_unused = 0, Hu = 0;
     int rc = eakv_match(ctx, keys, nblk, &G, nullptr, nullptr, nullptr);
     if (rc != EAKV_OK) return rc;
-    rc = eakv_match(ctx, ukeys, nu, &G_unused, &Hu, nullptr, ctx->t_host_slots.data());
+    rc = eakv_match(ctx, ukeys, nu, &G_unused, &Hu, nullptr, T.host_slots.data());
     if (rc != EAKV_OK) return rc;
+    int32_t tail = -1;
+    if (as_request)
+        rc = eakv_gpu_tier_acquire(ctx, request_id, keys, nblk, need_tail, T.resident.data(), T.block.data(), &tail);
+    else
+        rc = eakv_gpu_tier_step(ctx, keys, nblk, need_tail, T.resident.data(), T.block.data(), &tail);
+    if (rc != EAKV_OK) return rc;
+    T.tail = tail;
+    T.open = true;
     int64_t n_ev = nu;
     eakv_step_info info;
-    rc = eakv_tier_step(ctx, ukeys, nu, agent_id, n_tokens, now_ms, ctx->t_hit.data(),
-                        ctx->t_admit_u.data(), ctx->t_slot_u.data(), ctx->t_evicted_keys.data(),
-                        ctx->t_evicted_slots.data(), &n_ev, &info);
-    if (rc != EAKV_OK) return rc;                // refused requests change nothing
-    ctx->t_keys = keys;
-    ctx->t_ukeys = ukeys;
-    int32_t tail = -1;
-    rc = eakv_gpu_tier_step(ctx, keys, nblk, need_tail, ctx->t_resident.data(), ctx->t_block.data(), &tail);
-    if (rc != EAKV_OK) {                          // (capacity was checked above)
-        ctx->t_block.clear();
-        withdraw_turn(ctx, true, 0);
+    rc = tier_step_impl(ctx, ukeys, nu, agent_id, n_tokens, now_ms, decided, T.hit.data(), T.admit_u.data(),
+                        T.slot_u.data(), T.evicted_keys.data(), T.evicted_slots.data(), &n_ev, &info);
+    if (rc != EAKV_OK) {                          // (its capacity was checked above)
+        withdraw_turn(ctx, T, false, 1);
         return rc;
     }
-    ctx->turn_open = true;
-    ctx->turn_tail = tail;
     if (ctx->wb_pending) {
         bool reused = tail >= 0 && ctx->wb_blocks[tail];
         for (int64_t j = 0; j < nblk && !reused; ++j)
-            reused = !ctx->t_resident[j] && ctx->wb_blocks[ctx->t_block[j]];
+            reused = !T.resident[j] && ctx->wb_blocks[T.block[j]];
         if (reused) {
             // the caller is about to overwrite a block the deferred write still reads
             rc = wait_write_behind(ctx, static_cast<cudaStream_t>(cuda_stream));
             if (rc != EAKV_OK) {
-                withdraw_turn(ctx, true, 1);
+                withdraw_turn(ctx, T, true, 1);
                 return rc;
             }
             // (the marks stay until the write is seen complete: another stream may come next)
@@ -1292,26 +1309,26 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
         // block slots of the restored blocks: chunk slot * R + position inside the chunk
         std::vector<int32_t> slots((size_t)(hi - lo));
         for (int64_t j = lo; j < hi; ++j)
-            slots[j - lo] = (int32_t)((int64_t)ctx->t_host_slots[j / R] * R + j % R);
-        rc = eakv_load(ctx, slots.data(), ctx->t_block.data() + lo, hi - lo, cuda_stream);
+            slots[j - lo] = (int32_t)((int64_t)T.host_slots[j / R] * R + j % R);
+        rc = eakv_load(ctx, slots.data(), T.block.data() + lo, hi - lo, cuda_stream);
         if (rc != EAKV_OK) {
             // nothing of this turn was restored or will be computed: neither tier may list it
-            withdraw_turn(ctx, true, 1);
+            withdraw_turn(ctx, T, true, 1);
             return rc;
         }
     }
     int64_t n_fill = 0;
     for (int64_t j = cover; j < nblk; ++j)
-        if (!ctx->t_resident[j]) { ctx->t_fill[j] = 1; ++n_fill; }
-    // per-block view of the unit decisions, for the store at the end of the turn
-    ctx->t_admit_b.assign((size_t)nblk, 0);
-    ctx->t_slot_b.assign((size_t)nblk, -1);
+        if (!T.resident[j]) { T.fill[j] = 1; ++n_fill; }
+    // per-block view of the unit decisions, for the store
+    T.admit_b.assign((size_t)nblk, 0);
+    T.slot_b.assign((size_t)nblk, -1);
     int64_t n_store = 0;
     for (int64_t c = 0; c < nu; ++c) {
-        if (!ctx->t_admit_u[c]) continue;
+        if (!T.admit_u[c]) continue;
         for (int64_t i = 0; i < R; ++i) {
-            ctx->t_admit_b[c * R + i] = 1;
-            ctx->t_slot_b[c * R + i] = (int32_t)((int64_t)ctx->t_slot_u[c] * R + i);
+            T.admit_b[c * R + i] = 1;
+            T.slot_b[c * R + i] = (int32_t)((int64_t)T.slot_u[c] * R + i);
             ++n_store;
         }
     }
@@ -1323,59 +1340,105 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
     view->n_fill = n_fill; view->n_stored_blocks = n_store; view->n_evicted = n_ev;
     view->pressure = info.pressure; view->save = info.save; view->tail_block = tail; view->reserved = 0;
     view->keys = keys;
-    view->gpu_block = ctx->t_block.data(); view->gpu_resident = ctx->t_resident.data();
-    view->needs_fill = ctx->t_fill.data();
-    view->hit = ctx->t_hit.data(); view->admit = ctx->t_admit_u.data(); view->slot = ctx->t_slot_u.data();
-    view->evicted_keys = ctx->t_evicted_keys.data(); view->evicted_slots = ctx->t_evicted_slots.data();
+    view->gpu_block = T.block.data(); view->gpu_resident = T.resident.data();
+    view->needs_fill = T.fill.data();
+    view->hit = T.hit.data(); view->admit = T.admit_u.data(); view->slot = T.slot_u.data();
+    view->evicted_keys = T.evicted_keys.data(); view->evicted_slots = T.evicted_slots.data();
     return EAKV_OK;
 }
 
-int eakv_turn_end(eakv_ctx* ctx, void* cuda_stream) {
-    if (!ctx || !ctx->turn_open) return EAKV_E_INVAL;
-    int rc = EAKV_OK;
-    const int64_t nblk = (int64_t)ctx->t_block.size();
+// the store of an open turn's admitted blocks (directly, or deferred on the context's stream)
+int turn_store_impl(eakv_ctx* ctx, TurnState& T, void* cuda_stream) {
+    const int64_t nblk = (int64_t)T.block.size();
     bool any_store = false;
-    for (int64_t j = 0; j < nblk && !any_store; ++j) any_store = ctx->t_admit_b[j] != 0;
-    if (ctx->device < 0) {
-        // bookkeeping only: nothing to copy
-    } else if (any_store && ctx->cfg.write_behind) {
-        // deferred write: on the context's stream, after what precedes it on the caller's stream
-        DeviceGuard g(ctx->device);
-        cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-        rc = [&]() -> int {
-            if (!ctx->wb_stream) {
-                CU(cudaStreamCreateWithFlags(&ctx->wb_stream, cudaStreamNonBlocking));
-                CU(cudaEventCreateWithFlags(&ctx->wb_fence, cudaEventDisableTiming));
-                CU(cudaEventCreateWithFlags(&ctx->wb_done, cudaEventDisableTiming));
-                ctx->wb_blocks.assign((size_t)ctx->cfg.gpu_blocks, 0);
-                ctx->wb_slots.assign((size_t)ctx->tier_slots, 0);
-            }
-            CU(cudaEventRecord(ctx->wb_fence, stream));
-            CU(cudaStreamWaitEvent(ctx->wb_stream, ctx->wb_fence, 0));
-            int r = eakv_store(ctx, ctx->t_block.data(), ctx->t_admit_b.data(), ctx->t_slot_b.data(), nblk,
-                               ctx->wb_stream);
-            if (r != EAKV_OK) return r;
-            CU(cudaEventRecord(ctx->wb_done, ctx->wb_stream));
-            for (int64_t j = 0; j < nblk; ++j)
-                if (ctx->t_admit_b[j]) {
-                    ctx->wb_blocks[ctx->t_block[j]] = 1;
-                    ctx->wb_slots[ctx->t_slot_b[j]] = 1;
-                }
-            ctx->wb_pending = true;
-            return EAKV_OK;
-        }();
-    } else if (any_store) {
-        rc = eakv_store(ctx, ctx->t_block.data(), ctx->t_admit_b.data(), ctx->t_slot_b.data(), nblk,
-                        cuda_stream);
+    for (int64_t j = 0; j < nblk && !any_store; ++j) any_store = T.admit_b[j] != 0;
+    T.stored = true;
+    if (ctx->device < 0 || !any_store) return EAKV_OK;       // bookkeeping only, or nothing admitted
+    if (!ctx->cfg.write_behind)
+        return eakv_store(ctx, T.block.data(), T.admit_b.data(), T.slot_b.data(), nblk, cuda_stream);
+    // deferred write: on the context's stream, after what precedes it on the caller's stream
+    DeviceGuard g(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (!ctx->wb_stream) {
+        CU(cudaStreamCreateWithFlags(&ctx->wb_stream, cudaStreamNonBlocking));
+        CU(cudaEventCreateWithFlags(&ctx->wb_fence, cudaEventDisableTiming));
+        CU(cudaEventCreateWithFlags(&ctx->wb_done, cudaEventDisableTiming));
+        ctx->wb_blocks.assign((size_t)ctx->cfg.gpu_blocks, 0);
+        ctx->wb_slots.assign((size_t)ctx->tier_slots, 0);
     }
+    CU(cudaEventRecord(ctx->wb_fence, stream));
+    CU(cudaStreamWaitEvent(ctx->wb_stream, ctx->wb_fence, 0));
+    int r = eakv_store(ctx, T.block.data(), T.admit_b.data(), T.slot_b.data(), nblk, ctx->wb_stream);
+    if (r != EAKV_OK) return r;
+    CU(cudaEventRecord(ctx->wb_done, ctx->wb_stream));
+    for (int64_t j = 0; j < nblk; ++j)
+        if (T.admit_b[j]) {
+            ctx->wb_blocks[T.block[j]] = 1;
+            ctx->wb_slots[T.slot_b[j]] = 1;
+        }
+    ctx->wb_pending = true;
+    return EAKV_OK;
+}
+
+}  // namespace
+
+int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
+                    const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
+                    void* cuda_stream, eakv_turn_view* view) {
+    if (!ctx || !view || n_tokens < 0 || n_known < 0) return EAKV_E_INVAL;
+    if (ctx->turn.open || !ctx->held.empty()) return EAKV_E_INVAL;
+    if (n_known > 0 && !known_keys) return EAKV_E_INVAL;
+    return turn_begin_impl(ctx, ctx->turn, kNoRequest, tokens, n_tokens, known_keys, n_known, agent_id, now_ms,
+                           -1, cuda_stream, view);
+}
+
+int eakv_turn_end(eakv_ctx* ctx, void* cuda_stream) {
+    if (!ctx || !ctx->turn.open) return EAKV_E_INVAL;
+    const int rc = turn_store_impl(ctx, ctx->turn, cuda_stream);
     // a store that could not be enqueued leaves slots unwritten: their keys must not stay listed
-    withdraw_turn(ctx, rc != EAKV_OK, 0);
+    withdraw_turn(ctx, ctx->turn, rc != EAKV_OK, 0);
     return rc;
 }
 
 int eakv_turn_abort(eakv_ctx* ctx) {
-    if (!ctx || !ctx->turn_open) return EAKV_E_INVAL;
-    withdraw_turn(ctx, true, 2);
+    if (!ctx || !ctx->turn.open) return EAKV_E_INVAL;
+    withdraw_turn(ctx, ctx->turn, true, 2);
+    return EAKV_OK;
+}
+
+int eakv_request_begin(eakv_ctx* ctx, int64_t request_id, const int32_t* tokens, int64_t n_tokens,
+                       const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
+                       int32_t decided, void* cuda_stream, eakv_turn_view* view) {
+    if (!ctx || !view || n_tokens < 0 || n_known < 0 || request_id == kNoRequest) return EAKV_E_INVAL;
+    if (ctx->turn.open || ctx->requests.count(request_id) || ctx->held.count(request_id)) return EAKV_E_INVAL;
+    if (n_known > 0 && !known_keys) return EAKV_E_INVAL;
+    TurnState& T = ctx->requests[request_id];
+    const int rc = turn_begin_impl(ctx, T, request_id, tokens, n_tokens, known_keys, n_known, agent_id, now_ms,
+                                   decided < 0 ? -1 : (decided ? 1 : 0), cuda_stream, view);
+    if (rc != EAKV_OK) ctx->requests.erase(request_id);
+    return rc;
+}
+
+int eakv_request_store(eakv_ctx* ctx, int64_t request_id, void* cuda_stream) {
+    if (!ctx) return EAKV_E_INVAL;
+    auto it = ctx->requests.find(request_id);
+    if (it == ctx->requests.end() || it->second.stored) return EAKV_E_INVAL;
+    const int rc = turn_store_impl(ctx, it->second, cuda_stream);
+    if (rc != EAKV_OK) {
+        withdraw_turn(ctx, it->second, true, 0);
+        ctx->requests.erase(it);
+    }
+    return rc;
+}
+
+int eakv_request_release(eakv_ctx* ctx, int64_t request_id) {
+    if (!ctx) return EAKV_E_INVAL;
+    auto it = ctx->requests.find(request_id);
+    if (it == ctx->requests.end()) return EAKV_E_INVAL;
+    // released before its store: the engine never produced the KV, so what was registered is taken back
+    if (!it->second.stored) withdraw_turn(ctx, it->second, true, 2);
+    else withdraw_turn(ctx, it->second, false, 0);
+    ctx->requests.erase(it);
     return EAKV_OK;
 }
 

@@ -38,15 +38,55 @@ __global__ void iota_kernel(int32_t* idx, int64_t n) {
 }
 
 // sorted by (key, position): the predecessor of a position is its left neighbour with the same key
+// (and its successor, when asked for, the right neighbour with the same key)
 __global__ void prev_from_sorted_kernel(const uint64_t* __restrict__ keys_sorted,
                                         const int32_t* __restrict__ idx_sorted, int64_t n,
-                                        int32_t* __restrict__ prev, uint32_t* __restrict__ v) {
+                                        int32_t* __restrict__ prev, uint32_t* __restrict__ v,
+                                        int32_t* __restrict__ next /* or NULL */) {
     const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= n) return;
     const int32_t i = idx_sorted[s];
     const int32_t p = (s > 0 && keys_sorted[s - 1] == keys_sorted[s]) ? idx_sorted[s - 1] : -1;
     prev[i] = p;
     v[i] = (uint32_t)(p + 1);
+    if (next) next[i] = (s + 1 < n && keys_sorted[s + 1] == keys_sorted[s]) ? idx_sorted[s + 1] : -1;
+}
+
+// Declined-chunk audit (Appendix D, "Reuse distance of declined chunks"): for every declined
+// position, the reuse distance at which its chunk is referenced next.  counts[0] = declined
+// positions, counts[1] = those whose next reference lies at D >= capacity or never comes (the
+// condition of Proposition 1), counts[2] = those never referenced again.
+__global__ void declined_audit_kernel(const uint8_t* __restrict__ declined, const int32_t* __restrict__ next,
+                                      const int64_t* __restrict__ dist, int64_t n, int64_t capacity,
+                                      int64_t* __restrict__ next_dist /* or NULL */,
+                                      unsigned long long* __restrict__ counts) {
+    unsigned long long c0 = 0, c1 = 0, c2 = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        int64_t out = -2;                       // not declined
+        if (declined[i]) {
+            const int32_t j = next[i];
+            ++c0;
+            if (j < 0) {
+                ++c1; ++c2;
+                out = -1;                       // never referenced again
+            } else {
+                out = dist[j];
+                if (out >= capacity) ++c1;
+            }
+        }
+        if (next_dist) next_dist[i] = out;
+    }
+    for (int d = 16; d; d >>= 1) {
+        c0 += __shfl_xor_sync(0xffffffffu, c0, d);
+        c1 += __shfl_xor_sync(0xffffffffu, c1, d);
+        c2 += __shfl_xor_sync(0xffffffffu, c2, d);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (c0) atomicAdd(&counts[0], c0);
+        if (c1) atomicAdd(&counts[1], c1);
+        if (c2) atomicAdd(&counts[2], c2);
+    }
 }
 
 // ---- step 2: one wavelet-matrix level = stable partition by one bit -------------------------
@@ -264,12 +304,10 @@ using namespace eakv;
         }                                     \
     } while (0)
 
-extern "C" int eakv_reuse_distances(const uint64_t* keys_dev, int64_t n_refs, int64_t* dist_dev,
-                                    void* cuda_stream) {
-    if (n_refs < 0 || n_refs > 0x7ffffff0LL) return EAKV_E_INVAL;
-    if (n_refs == 0) return EAKV_OK;
-    if (!keys_dev || !dist_dev) return EAKV_E_INVAL;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+// dist_dev[i] for all references; next_dev (optional, int32[n]) receives the position of the next
+// reference to the same key or -1.  Returns after the stream has finished the work.
+static int reuse_distances_impl(const uint64_t* keys_dev, int64_t n_refs, int64_t* dist_dev,
+                                int32_t* next_dev, cudaStream_t stream) {
     const int64_t n = n_refs;
     int nbits = 1;
     while ((1ll << nbits) <= n) ++nbits;               // values v in [0, n] fit in nbits bits
@@ -300,7 +338,7 @@ extern "C" int eakv_reuse_distances(const uint64_t* keys_dev, int64_t n_refs, in
     iota_kernel<<<grid1, 256, 0, stream>>>(idx, n);
     SD_CU(cub::DeviceRadixSort::SortPairs(sort_tmp, sort_bytes, keys_dev, keys_sorted, idx, idx_sorted,
                                           (int)n, 0, 61, stream));
-    prev_from_sorted_kernel<<<grid1, 256, 0, stream>>>(keys_sorted, idx_sorted, n, prev, va);
+    prev_from_sorted_kernel<<<grid1, 256, 0, stream>>>(keys_sorted, idx_sorted, n, prev, va, next_dev);
     for (int l = 0; l < nbits; ++l) {
         const int shift = nbits - 1 - l;
         uint32_t* a = (l & 1) ? vb : va;
@@ -319,6 +357,77 @@ done:
     cudaFree(sort_tmp);
     if (rc != EAKV_OK) cudaGetLastError();
     return rc;
+}
+
+extern "C" int eakv_reuse_distances(const uint64_t* keys_dev, int64_t n_refs, int64_t* dist_dev,
+                                    void* cuda_stream) {
+    if (n_refs < 0 || n_refs > 0x7ffffff0LL) return EAKV_E_INVAL;
+    if (n_refs == 0) return EAKV_OK;
+    if (!keys_dev || !dist_dev) return EAKV_E_INVAL;
+    return reuse_distances_impl(keys_dev, n_refs, dist_dev, nullptr, static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" int eakv_declined_audit(const uint64_t* keys_dev, const uint8_t* declined_dev, int64_t n_refs,
+                                   int64_t capacity, int64_t* declined_out, int64_t* meets_out,
+                                   int64_t* never_out, int64_t* next_dist_dev, void* cuda_stream) {
+    if (n_refs < 0 || n_refs > 0x7ffffff0LL || capacity < 0) return EAKV_E_INVAL;
+    if (!declined_out || !meets_out || !never_out) return EAKV_E_INVAL;
+    *declined_out = *meets_out = *never_out = 0;
+    if (n_refs == 0) return EAKV_OK;
+    if (!keys_dev || !declined_dev) return EAKV_E_INVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int rc = EAKV_OK;
+    int64_t* dist = nullptr;
+    int32_t* next = nullptr;
+    unsigned long long* counts = nullptr;
+    unsigned long long host_counts[3] = {0, 0, 0};
+    int dev = 0, sms = 148;
+    SD_CU(cudaMalloc(&dist, n_refs * 8));
+    SD_CU(cudaMalloc(&next, n_refs * 4));
+    SD_CU(cudaMalloc(&counts, 3 * 8));
+    SD_CU(cudaMemsetAsync(counts, 0, 3 * 8, stream));
+    rc = reuse_distances_impl(keys_dev, n_refs, dist, next, stream);
+    if (rc != EAKV_OK) goto done;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    declined_audit_kernel<<<(int)std::min<int64_t>((n_refs + 255) / 256, (int64_t)sms * 8), 256, 0, stream>>>(
+        declined_dev, next, dist, n_refs, capacity, next_dist_dev, counts);
+    SD_CU(cudaGetLastError());
+    SD_CU(cudaMemcpyAsync(host_counts, counts, 3 * 8, cudaMemcpyDeviceToHost, stream));
+    SD_CU(cudaStreamSynchronize(stream));
+    *declined_out = (int64_t)host_counts[0];
+    *meets_out = (int64_t)host_counts[1];
+    *never_out = (int64_t)host_counts[2];
+done:
+    cudaFree(dist); cudaFree(next); cudaFree(counts);
+    if (rc != EAKV_OK) cudaGetLastError();
+    return rc;
+}
+
+extern "C" int eakv_working_set(const eakv_working_set_in* in, eakv_working_set_out* out) {
+    if (!in || !out) return EAKV_E_INVAL;
+    if (in->num_layers <= 0 || in->kv_heads <= 0 || in->head_dim <= 0 || in->elem_bytes <= 0 ||
+        in->tensor_parallel <= 0 || in->block_size <= 0 || in->active_pool <= 0 || in->n_requests <= 0 ||
+        in->total_prompt_tokens < 0 || in->gpu_blocks < 0 || in->host_blocks < 0)
+        return EAKV_E_INVAL;
+    typedef __int128 wide;
+    // Eq. 1: beta_rank = 2 L d s max(1, ceil(H_kv / TP))
+    const int64_t heads = std::max<int64_t>(1, (in->kv_heads + in->tensor_parallel - 1) / in->tensor_parallel);
+    const int64_t beta = 2ll * in->num_layers * in->head_dim * in->elem_bytes * heads;
+    // Eq. 5 with N_bar = total / requests kept as a fraction: (A - 1) * total * beta / requests
+    const wide num = (wide)(in->active_pool - 1) * in->total_prompt_tokens;
+    out->beta_rank_bytes = beta;
+    out->working_set_bytes = (int64_t)(num * beta / in->n_requests);
+    out->working_set_blocks = (int64_t)(num / ((wide)in->n_requests * in->block_size));
+    // gamma_G = A * N_bar / K_G with K_G = gpu_blocks * b tokens; gamma_H = C_reuse / C_H with
+    // C_H = host_blocks * b * beta (beta cancels)
+    const wide g_num = (wide)in->active_pool * in->total_prompt_tokens;
+    const wide g_den = (wide)in->n_requests * in->gpu_blocks * in->block_size;
+    const wide h_den = (wide)in->n_requests * in->host_blocks * in->block_size;
+    out->gamma_g = g_den ? (double)g_num / (double)g_den : 0.0;
+    out->gamma_h = h_den ? (double)num / (double)h_den : 0.0;
+    out->pool_exceeds_gpu = g_den ? (g_num > g_den) : 0;
+    out->working_set_exceeds_host = h_den ? (num > h_den) : 0;
+    return EAKV_OK;
 }
 
 extern "C" int eakv_capacity_curve(const int64_t* dist_dev, int64_t n_refs,

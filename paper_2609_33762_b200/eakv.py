@@ -65,6 +65,19 @@ class StepInfo(C.Structure):
                 ("pressure", C.c_int32), ("save", C.c_int32)]
 
 
+class WorkingSetIn(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("num_layers", "kv_heads", "head_dim", "elem_bytes", "tensor_parallel",
+                                         "block_size")] + \
+               [(n, C.c_int64) for n in ("active_pool", "total_prompt_tokens", "n_requests", "gpu_blocks",
+                                         "host_blocks")]
+
+
+class WorkingSetOut(C.Structure):
+    _fields_ = [("beta_rank_bytes", C.c_int64), ("working_set_bytes", C.c_int64),
+                ("working_set_blocks", C.c_int64), ("gamma_g", C.c_double), ("gamma_h", C.c_double),
+                ("pool_exceeds_gpu", C.c_int32), ("working_set_exceeds_host", C.c_int32)]
+
+
 class TurnView(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
         "n_blocks", "n_units", "gpu_prefix_blocks", "host_prefix_blocks", "restore_lo", "restore_hi",
@@ -94,6 +107,8 @@ EXPORTS = [
     "eakv_admission_export", "eakv_admission_import",
     "eakv_selfcheck_limits", "eakv_selfcheck_wait_probe",
     "eakv_gpu_tier_acquire", "eakv_gpu_tier_release_request", "eakv_tier_step_again",
+    "eakv_declined_audit", "eakv_working_set",
+    "eakv_request_begin", "eakv_request_store", "eakv_request_release",
 ]
 STATIC_MAX_BLOCKS = 65536
 
@@ -130,9 +145,14 @@ def lib():
     L.eakv_load_layers.argtypes = [vp, vp, vp, i64, i32, vp, i32, vp]
     L.eakv_reuse_distances.argtypes = [vp, i64, vp, vp]
     L.eakv_capacity_curve.argtypes = [vp, i64, vp, vp, vp, i64, i32, vp, i32, vp, vp, vp, vp, vp]
+    L.eakv_declined_audit.argtypes = [vp, vp, i64, i64, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), vp, vp]
+    L.eakv_working_set.argtypes = [C.POINTER(WorkingSetIn), C.POINTER(WorkingSetOut)]
     L.eakv_turn_begin.argtypes = [vp, vp, i64, vp, i64, i64, i64, vp, C.POINTER(TurnView)]
     L.eakv_turn_end.argtypes = [vp, vp]
     L.eakv_turn_abort.argtypes = [vp]
+    L.eakv_request_begin.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i32, vp, C.POINTER(TurnView)]
+    L.eakv_request_store.argtypes = [vp, i64, vp]
+    L.eakv_request_release.argtypes = [vp, i64]
     L.eakv_tier_export.argtypes = [vp, vp, vp, i64, C.POINTER(i64)]
     L.eakv_tier_import.argtypes = [vp, vp, vp, i64]
     L.eakv_admission_export.argtypes = [vp, vp, i64, C.POINTER(i64)]
@@ -194,6 +214,29 @@ def eakv_reuse_distances(keys_dev, n_refs, dist_dev, stream=None):
                                     _stream(stream))
     if rc != OK:
         raise EakvError(rc, "eakv_reuse_distances")
+
+
+def eakv_declined_audit(keys_dev, declined_dev, n_refs, capacity, next_dist_dev=0, stream=None):
+    """(declined, meets, never) of the declined references at device address ``declined_dev`` (uint8)."""
+    d, m, nv = C.c_int64(0), C.c_int64(0), C.c_int64(0)
+    rc = lib().eakv_declined_audit(C.c_void_p(int(keys_dev)), C.c_void_p(int(declined_dev)), int(n_refs),
+                                   int(capacity), C.byref(d), C.byref(m), C.byref(nv),
+                                   C.c_void_p(int(next_dist_dev)) if next_dist_dev else None, _stream(stream))
+    if rc != OK:
+        raise EakvError(rc, "eakv_declined_audit")
+    return d.value, m.value, nv.value
+
+
+def eakv_working_set(*, num_layers, kv_heads, head_dim, block_size, active_pool, total_prompt_tokens,
+                     n_requests, gpu_blocks=0, host_blocks=0, elem_bytes=2, tensor_parallel=1):
+    """Eq. 1, Eq. 5 and the pressure ratios of Section 3.2 as a dict (integer arithmetic in the library)."""
+    i = WorkingSetIn(num_layers, kv_heads, head_dim, elem_bytes, tensor_parallel, block_size, active_pool,
+                     total_prompt_tokens, n_requests, gpu_blocks, host_blocks)
+    o = WorkingSetOut()
+    rc = lib().eakv_working_set(C.byref(i), C.byref(o))
+    if rc != OK:
+        raise EakvError(rc, "eakv_working_set")
+    return {n: getattr(o, n) for n, _ in WorkingSetOut._fields_}
 
 
 def eakv_capacity_curve(dist_dev, n_refs, req_offsets, req_tokens, req_gpu_prefix, block_size,
@@ -454,6 +497,34 @@ class Context:
         rc = lib().eakv_turn_begin(self._h, C.c_void_p(int(tokens_ptr)), int(n_tokens), kp, nk,
                                    int(agent_id), int(now_ms), _stream(stream), C.byref(v))
         self._check(rc, "eakv_turn_begin")
+        return self._view_dict(v)
+
+    def eakv_request_begin(self, request_id, tokens_ptr, n_tokens, known_keys, agent_id, now_ms,
+                           decided=None, stream=None):
+        """First half of a running request's turn (its GPU blocks stay pinned until
+        eakv_request_release); None when the blocks do not fit beside the running requests.
+        ``decided``: None for the first lookup, else the store/skip choice made then."""
+        kp, nk = None, 0
+        if known_keys is not None and len(known_keys):
+            kk, kp = _np(known_keys, np.uint64)
+            nk = len(kk)
+        v = TurnView()
+        rc = lib().eakv_request_begin(self._h, int(request_id), C.c_void_p(int(tokens_ptr)), int(n_tokens), kp, nk,
+                                      int(agent_id), int(now_ms), -1 if decided is None else int(bool(decided)),
+                                      _stream(stream), C.byref(v))
+        if rc == E_CAPACITY:
+            return None
+        self._check(rc, "eakv_request_begin")
+        return self._view_dict(v)
+
+    def eakv_request_store(self, request_id, stream=None):
+        self._check(lib().eakv_request_store(self._h, int(request_id), _stream(stream)), "eakv_request_store")
+
+    def eakv_request_release(self, request_id):
+        self._check(lib().eakv_request_release(self._h, int(request_id)), "eakv_request_release")
+
+    @staticmethod
+    def _view_dict(v):
         nb, nu, ne = v.n_blocks, v.n_units, v.n_evicted
         out = {n: getattr(v, n) for n, _ in TurnView._fields_[:15] if n != "reserved"}
         out.update(keys=_view_array(v.keys, nb, np.uint64), gpu_block=_view_array(v.gpu_block, nb, np.int32),

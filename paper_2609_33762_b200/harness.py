@@ -4,8 +4,16 @@ runs inside libeakv.  The "prefill" of a real serving engine is replaced by writ
 fresh block's synthetic payload into the paged pool.
 
 One turn (the order follows the paper: lookup at scheduling time, restore before compute,
-store after): hash -> match -> host tier step -> GPU tier step -> load blocks [G, H) ->
+store after): hash -> match -> GPU tier step -> host tier step -> load blocks [G, H) ->
 fill fresh blocks -> store admitted blocks.
+
+By default the server drives the library's turn engine (eakv_turn_begin / eakv_turn_end, and
+eakv_request_begin / _store / _release for requests that overlap): the whole turn, including
+what to restore, what the engine must compute and what to store, is decided inside the
+library.  ``native_turn=False`` drives the single calls (eakv_hash_blocks, eakv_match,
+eakv_tier_step, eakv_gpu_tier_step, eakv_load, eakv_store) one by one instead; that path exists
+to test those calls and to run bookkeeping-only replays, and is the only place where this module
+combines their results itself.
 """
 from __future__ import annotations
 
@@ -45,7 +53,7 @@ class PagedPool:
 class AgentServer:
     def __init__(self, shape, gpu_blocks, host_blocks, payload, *, device="cuda:0",
                  gpu_index_blocks=0, incremental_hash=False, data_plane=True, chunk_blocks=1,
-                 native_turn=False, **ctx_kwargs):
+                 native_turn=None, **ctx_kwargs):
         """``payload(keys, q, n_words)`` returns the int16/uint16 words of piece q for the
         blocks with these keys, as a numpy array or a tensor on ``device``.  With
         ``chunk_blocks`` = R > 1 the host tier works in chunks of R blocks (``host_blocks``
@@ -73,7 +81,9 @@ class AgentServer:
         self.stream = torch.cuda.current_stream(self.device)
         self.b = shape.block_size
         self.R = max(1, int(chunk_blocks))
-        self.native_turn = native_turn     # drive turns through eakv_turn_begin / eakv_turn_end
+        if native_turn is None:
+            native_turn = bool(data_plane)
+        self.native_turn = native_turn     # drive turns through the library's turn engine
         if native_turn and not data_plane:
             raise ValueError("the two-call turn engine always moves KV bytes: it needs the data plane")
         self.seed = self.ctx.eakv_hash_seed()
@@ -156,23 +166,10 @@ class AgentServer:
         keys, blocks = v["keys"], v["gpu_block"]
         if self.incremental:
             self._agent_keys[agent] = keys
-        fill = np.nonzero(v["needs_fill"])[0]
-        if len(fill) and self.data_plane:
-            ids = torch.as_tensor(blocks[fill].astype(np.int64), device=self.device)
-            for q, piece in enumerate(self.pool.pieces):
-                w = self.payload(keys[fill], q, self.pool.words)
-                if isinstance(w, np.ndarray):
-                    w = torch.from_numpy(w.view(np.int16)).to(self.device)
-                piece[ids] = w.view(torch.int16)
+        self._fill(keys, blocks, np.nonzero(v["needs_fill"])[0])
         self.ctx.eakv_turn_end(self.stream)
-        G, H = v["gpu_prefix_blocks"], v["host_prefix_blocks"]
-        rec = dict(agent=agent, now_ms=now_ms, n_tokens=n, keys=keys, G=G, H=H,
-                   new_chunks=v["new_chunks"], pressure=bool(v["pressure"]), save=bool(v["save"]),
-                   hit=v["hit"], admit=v["admit"], slot=v["slot"],
-                   evicted=list(zip(v["evicted_keys"].tolist(), v["evicted_slots"].tolist())),
-                   gpu_resident=v["gpu_resident"], gpu_block=blocks,
-                   loaded=v["restore_hi"] - v["restore_lo"], stored=v["n_stored_blocks"],
-                   fresh_tokens=v["fresh_tokens"], filled=int(v["n_fill"]))
+        rec = self._record_from_view(v, agent, now_ms, n)
+        G, H = rec["G"], rec["H"]
         return rec, G, H
 
     def begin(self, request_id, tokens, agent, now_ms, decided=None):
@@ -183,6 +180,8 @@ class AgentServer:
         store/skip choice made then (a resumed request: eakv_tier_step_again)."""
         tokens = np.asarray(tokens, dtype=np.int32)
         n = len(tokens)
+        if self.native_turn:
+            return self._begin_native(request_id, tokens, agent, now_ms, decided)
         keys = self.block_keys(tokens, agent)
         nblk = len(keys)
         R = self.R
@@ -248,9 +247,64 @@ class AgentServer:
         self.records.append(rec)
         return rec
 
+    def _begin_native(self, request_id, tokens, agent, now_ms, decided):
+        """The same through eakv_request_begin / eakv_request_store."""
+        n = len(tokens)
+        self._ensure_pinned(max(n, 1))
+        self._tok_pin.numpy()[:n] = tokens
+        known = self._agent_keys.get(agent) if self.incremental else None
+        v = self.ctx.eakv_request_begin(request_id, self._tok_pin.data_ptr(), n, known, agent, now_ms,
+                                        decided=decided, stream=self.stream)
+        if v is None:
+            return None
+        keys, blocks = v["keys"], v["gpu_block"]
+        if self.incremental:
+            prev = self._agent_keys.get(agent)
+            if prev is None or len(keys) >= len(prev):
+                self._agent_keys[agent] = keys
+        self._fill(keys, blocks, np.nonzero(v["needs_fill"])[0])
+        self.ctx.eakv_request_store(request_id, self.stream)
+        rec = self._record_from_view(v, agent, now_ms, n)
+        rec.update(request_id=request_id, resumed=decided is not None)
+        t = self.totals
+        if decided is None:
+            t["prompt_tokens"] += n
+            t["fresh_tokens"] += rec["fresh_tokens"]
+            t["gpu_hit_blocks"] += rec["G"]
+            t["host_hit_blocks"] += rec["H"]
+        else:
+            t["preempt_recomputed_tokens"] = t.get("preempt_recomputed_tokens", 0) + rec["fresh_tokens"]
+        t["loaded_blocks"] += rec["loaded"]
+        t["stored_blocks"] += rec["stored"]
+        self.records.append(rec)
+        return rec
+
+    def _fill(self, keys, blocks, fill):
+        """The engine's part: produce the KV of the blocks the library flagged (synthetic payload)."""
+        if len(fill) and self.data_plane:
+            ids = torch.as_tensor(blocks[fill].astype(np.int64), device=self.device)
+            for q, piece in enumerate(self.pool.pieces):
+                w = self.payload(keys[fill], q, self.pool.words)
+                if isinstance(w, np.ndarray):
+                    w = torch.from_numpy(w.view(np.int16)).to(self.device)
+                piece[ids] = w.view(torch.int16)
+
+    @staticmethod
+    def _record_from_view(v, agent, now_ms, n):
+        return dict(agent=agent, now_ms=now_ms, n_tokens=n, keys=v["keys"], G=v["gpu_prefix_blocks"],
+                    H=v["host_prefix_blocks"], new_chunks=v["new_chunks"], pressure=bool(v["pressure"]),
+                    save=bool(v["save"]), hit=v["hit"], admit=v["admit"], slot=v["slot"],
+                    evicted=list(zip(v["evicted_keys"].tolist(), v["evicted_slots"].tolist())),
+                    gpu_resident=v["gpu_resident"], gpu_block=v["gpu_block"],
+                    loaded=v["restore_hi"] - v["restore_lo"], stored=v["n_stored_blocks"],
+                    fresh_tokens=v["fresh_tokens"], filled=int(v["n_fill"]), tail_block=v["tail_block"])
+
     def finish(self, request_id):
         """The request finished, or the engine suspended it: its GPU blocks become evictable."""
-        self.ctx.eakv_gpu_tier_release_request(request_id)
+        if self.native_turn:
+            self.ctx.eakv_request_release(request_id)
+        else:
+            self.ctx.eakv_gpu_tier_release_request(request_id)
 
     def turn(self, tokens, agent, now_ms):
         tokens = np.asarray(tokens, dtype=np.int32)

@@ -26,10 +26,12 @@ GIB = 1 << 30
 
 
 def working_set_blocks(trace, shape):
-    """Eq. 5 in blocks: (A - 1) * mean prompt length * beta / block bytes."""
-    n_mean = trace.total_prompt_tokens / len(trace.requests)
-    agents = len(trace.agent_tokens)
-    return int((agents - 1) * n_mean * shape.bytes_per_token // shape.block_bytes)
+    """Eq. 5 in blocks: (A - 1) * mean prompt length * beta / block bytes (eakv_working_set)."""
+    return eakv.eakv_working_set(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+                                 elem_bytes=shape.elem_bytes, block_size=shape.block_size,
+                                 active_pool=len(trace.agent_tokens),
+                                 total_prompt_tokens=trace.total_prompt_tokens,
+                                 n_requests=len(trace.requests))["working_set_blocks"]
 
 
 def mem_available_bytes():

@@ -145,10 +145,27 @@ def engine_begin(ctx, b, keys_of):
     return begin
 
 
+def request_begin(ctx, b, keys_of):
+    """The same through the library's request calls (bookkeeping only: every key is supplied)."""
+    def begin(request_id, tokens, agent, now_ms, decided):
+        v = ctx.eakv_request_begin(request_id, 0, len(tokens), keys_of(tokens), agent, now_ms, decided=decided)
+        if v is None:
+            return None
+        ctx.eakv_request_store(request_id)
+        return dict(fresh_tokens=v["fresh_tokens"], loaded=v["restore_hi"] - v["restore_lo"],
+                    stored=v["n_stored_blocks"], save=bool(v["save"]), G=v["gpu_prefix_blocks"],
+                    H=v["host_prefix_blocks"], gpu_block=v["gpu_block"].tolist(),
+                    gpu_resident=v["gpu_resident"].tolist(), hit=v["hit"].tolist(), admit=v["admit"].tolist(),
+                    slot=v["slot"].tolist(),
+                    evicted=list(zip(v["evicted_keys"].tolist(), v["evicted_slots"].tolist())))
+    return begin
+
+
+@pytest.mark.parametrize("api", ["single-calls", "request-calls"])
 @pytest.mark.parametrize("policy,kh,gpu_blocks,A,S,decode_us", [
     (0, 1024, 130, 8, 4, 20_000), (0, 160, 140, 8, 3, 60_000), (2, 200, 200, 6, 6, 40_000),
     (1, 300, 300, 8, 2, 10_000), (2, 160, 135, 8, 8, 100_000), (0, 1024, 130, 5, 1, 700)])
-def test_engine_replay_matches_oracle(mods, policy, kh, gpu_blocks, A, S, decode_us):
+def test_engine_replay_matches_oracle(mods, policy, kh, gpu_blocks, A, S, decode_us, api):
     eakv, closedloop = mods
     cfg = CONFIGS["c0_big_tier"]
     shape = SHAPES[cfg.shape]
@@ -161,7 +178,9 @@ def test_engine_replay_matches_oracle(mods, policy, kh, gpu_blocks, A, S, decode
     pm = closedloop.ServiceModel(t_pf_ns=40_000, h2d_bytes_per_us=9_000, d2h_bytes_per_us=7_000, tau_load_us=120)
     ctx = cp_ctx(eakv, b, gpu_blocks, kh, **kw)
     recs = []
-    begin = engine_begin(ctx, b, lambda t: as_keys(ohash.hash_blocks(t.tolist(), b)))
+    keys_of = lambda t: as_keys(ohash.hash_blocks(t.tolist(), b))
+    begin = engine_begin(ctx, b, keys_of) if api == "single-calls" else request_begin(ctx, b, keys_of)
+    release = ctx.eakv_gpu_tier_release_request if api == "single-calls" else ctx.eakv_request_release
 
     def logged_begin(*a):
         r = begin(*a)
@@ -169,8 +188,7 @@ def test_engine_replay_matches_oracle(mods, policy, kh, gpu_blocks, A, S, decode
             recs.append(r)
         return r
 
-    got = closedloop.replay_engine(trace, logged_begin, ctx.eakv_gpu_tier_release_request, pm, A, S, decode_us,
-                                   shape.bytes_per_token, b)
+    got = closedloop.replay_engine(trace, logged_begin, release, pm, A, S, decode_us, shape.bytes_per_token, b)
     st = ctx.eakv_get_stats()
     ctx.close()
     assert got["events"] == want["events"]
@@ -212,7 +230,7 @@ def test_config3_full_trace_engine_parity(mods):
 
     for a in tasks:
         by_len[id(trace.agent_tokens[a])] = np_keys[a]
-    got = closedloop.replay_engine(trace, engine_begin(ctx, b, keys_of), ctx.eakv_gpu_tier_release_request,
+    got = closedloop.replay_engine(trace, request_begin(ctx, b, keys_of), ctx.eakv_request_release,
                                    closedloop.ServiceModel(), 16, 16, 2_000_000, shape.bytes_per_token, b)
     ctx.close()
     assert got["events"] == want["events"] and got["makespan_us"] == want["makespan_us"]

@@ -55,7 +55,7 @@ def run_both(cfg_name, *, policy, host_blocks, limit=None, data_plane=False, lin
     oracle = TraceOracle(shape, cfg.gpu_blocks, host_blocks, **kw)
     oracle.run(trace, limit=limit)
     payload = (lambda keys, q, n: key_words_torch(keys.astype(np.int64), q, n, "cuda")) if data_plane else None
-    server = AgentServer(shape, cfg.gpu_blocks, host_blocks, payload, data_plane=data_plane,
+    server = AgentServer(shape, cfg.gpu_blocks, host_blocks, payload, data_plane=data_plane, native_turn=False,
                          incremental_hash=True, link_strategy=link, **kw)
     server.run(trace, limit=limit)
     compare_records_fast(server.records, oracle.records)

@@ -133,6 +133,34 @@ def test_argument_errors():
         eakv.eakv_capacity_curve(d.data_ptr(), 4, [0, 4], [64], [0], 16, list(range(1, 70)))
 
 
+@pytest.mark.parametrize("T,U,K", [(1, 1, 1), (50, 5, 3), (3000, 200, 64), (40_000, 3000, 500), (20_000, 50, 10)])
+def test_declined_audit_entry_point_on_random_streams(T, U, K):
+    """eakv_declined_audit against the oracle's definition-level audit: random reference streams,
+    random sets of declined positions; the three counts and, per declined position, the reuse
+    distance of the chunk's next reference."""
+    from oracle import audit as oaudit
+    from paper_2609_33762_b200 import eakv
+    rng = np.random.default_rng(T + U)
+    stream = rng.integers(1, U + 1, size=T, dtype=np.int64)
+    mask = (rng.random(T) < 0.3).astype(np.uint8)
+    declined = np.nonzero(mask)[0].tolist()
+    want = oaudit.declined_audit(stream.tolist(), declined, K)
+    kd = torch.from_numpy(stream).cuda()
+    md = torch.from_numpy(mask).cuda()
+    nd = torch.full((T + 1,), 7, dtype=torch.int64, device="cuda")
+    got = eakv.eakv_declined_audit(kd.data_ptr(), md.data_ptr(), T, K, nd.data_ptr())
+    assert got == (want["declined"], want["meets"], want["never_again"])
+    nd = nd.cpu().numpy()
+    assert nd[T] == 7                                                  # nothing written past the end
+    assert ((nd[:T] == -2) == (mask == 0)).all()
+    assert int((nd[:T] == -1).sum()) == want["never_again"]
+    again = nd[:T][nd[:T] >= 0]
+    assert sorted((again / K).tolist()) == sorted(want["ratios"])
+    # without the per-reference output, and an empty stream
+    assert eakv.eakv_declined_audit(kd.data_ptr(), md.data_ptr(), T, K) == got
+    assert eakv.eakv_declined_audit(0, 0, 0, K) == (0, 0, 0)
+
+
 def test_declined_chunk_audit_matches_oracle():
     """The audit of declined writes (next reuse distance >= K_H or never again) on a scaled
     config-2 trace under both filters, against the oracle's definition-level audit."""

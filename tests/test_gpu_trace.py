@@ -56,7 +56,7 @@ def test_config0_bit_exact(cfg_name, link):
     payload = normal_payload if cfg_name == "c0" and link == 0 else key_words_numpy
     oracle = TraceOracle(shape, cfg.gpu_blocks, cfg.host_blocks, payload=payload)
     oracle.run(trace)
-    server = AgentServer(shape, cfg.gpu_blocks, cfg.host_blocks, payload, link_strategy=link,
+    server = AgentServer(shape, cfg.gpu_blocks, cfg.host_blocks, payload, native_turn=False, link_strategy=link,
                          staging_bytes=7 * shape.block_bytes, incremental_hash=(link == 1),
                          min_staged_run_bytes=-1 if link == 1 else 0)
     server.run(trace)
@@ -86,7 +86,7 @@ def test_admission_policies_bit_exact(policy, kappa):
     oracle = TraceOracle(shape, 128, 160, payload=key_words_numpy, **kw)
     oracle.run(trace)
     dev_payload = lambda keys, q, n: key_words_torch(keys.astype(np.int64), q, n, "cuda")
-    server = AgentServer(shape, 128, 160, dev_payload, **kw)
+    server = AgentServer(shape, 128, 160, dev_payload, native_turn=False, **kw)
     server.run(trace)
     compare_records(server.records, oracle.records)
     compare_bytes(server, oracle)
@@ -146,7 +146,7 @@ def test_two_granularities_bit_exact(R, policy, link):
     kh = 700 // R
     oracle = TraceOracle(shape, 256, kh, payload=key_words_numpy, chunk_blocks=R, **kw)
     oracle.run(trace)
-    server = AgentServer(shape, 256, kh, key_words_numpy, chunk_blocks=R, link_strategy=link,
+    server = AgentServer(shape, 256, kh, key_words_numpy, chunk_blocks=R, native_turn=False, link_strategy=link,
                          staging_bytes=6 * shape.block_bytes, **kw)
     server.run(trace)
     compare_records(server.records, oracle.records)
@@ -252,10 +252,11 @@ def test_closed_loop_replay_bit_exact(policy, kh, pool, native):
     server.close()
 
 
+@pytest.mark.parametrize("native", [True, False], ids=["request-calls", "single-calls"])
 @pytest.mark.parametrize("policy,kh,gpu_blocks,S,decode_us,R,link", [
     (0, 1024, 130, 4, 20_000, 1, 1), (0, 160, 140, 3, 60_000, 1, 0), (2, 200, 200, 6, 40_000, 1, 1),
     (0, 64, 136, 4, 50_000, 4, 1)])
-def test_engine_replay_with_preemption_bit_exact(policy, kh, gpu_blocks, S, decode_us, R, link):
+def test_engine_replay_with_preemption_bit_exact(policy, kh, gpu_blocks, S, decode_us, R, link, native):
     """The engine model (several running requests with pinned GPU blocks, suspension when GPU KV
     memory runs out, resumption by restoring and recomputing) on the GPU path with bytes: every
     scheduler event, every record of every first and resumed lookup, J, and every resident byte of
@@ -272,7 +273,7 @@ def test_engine_replay_with_preemption_bit_exact(policy, kh, gpu_blocks, S, deco
     oracle = TraceOracle(shape, gpu_blocks, kh, payload=key_words_numpy, chunk_blocks=R, **kw)
     want = oen.replay(trace, oracle, ocl.ServiceModel(**rates), 8, S, decode_us, shape.bytes_per_token)
     server = AgentServer(shape, gpu_blocks, kh, key_words_numpy, incremental_hash=True, chunk_blocks=R,
-                         link_strategy=link, **kw)
+                         link_strategy=link, native_turn=native, **kw)
     got = closedloop.replay_engine(trace, server.begin, server.finish, closedloop.ServiceModel(**rates), 8, S,
                                    decode_us, shape.bytes_per_token, shape.block_size)
     assert got["events"] == want["events"] and got["order"] == want["order"]

@@ -35,3 +35,51 @@ def test_plan_sources(monkeypatch):
     assert kh == int((10 << 30) * 0.6 // shape.block_bytes) and "capped" in why
     kh, _ = replay.plan(cfg3, trace, shape, data_plane=False)
     assert kh == cfg3.host_blocks
+
+
+def test_eakv_working_set_against_oracle_sizing_and_the_papers_printed_values():
+    """eakv_working_set (Eq. 1, Eq. 5, gamma_G, gamma_H in integers) against oracle.sizing evaluated
+    in exact fractions, and on the paper's own H20 numbers (Section 3.2, Appendix C)."""
+    import random
+    from fractions import Fraction
+    from paper_2609_33762_b200 import eakv
+    # the paper: 4,427 requests with 147,124,984 prompt tokens, A = 16, Qwen3 at TP8 (24 KiB per
+    # token per rank), GPU KV capacity 343,408 tokens, host tier 5 GiB in 1,024-token chunks (213)
+    out = eakv.eakv_working_set(num_layers=48, kv_heads=4, head_dim=128, tensor_parallel=8, block_size=1024,
+                                active_pool=16, total_prompt_tokens=147_124_984, n_requests=4427,
+                                gpu_blocks=335, host_blocks=213)
+    assert out["beta_rank_bytes"] == 24 * 1024
+    assert abs(out["working_set_bytes"] / 2**30 - 11.4) < 0.05                 # "11.4 GiB per rank"
+    assert abs(out["gamma_h"] - 2.3) < 0.05 and out["working_set_exceeds_host"] == 1
+    assert abs(out["gamma_g"] - 16 * 33_234 / (335 * 1024)) < 0.01 and out["pool_exceeds_gpu"] == 1
+    a8 = eakv.eakv_working_set(num_layers=48, kv_heads=4, head_dim=128, tensor_parallel=8, block_size=1024,
+                               active_pool=8, total_prompt_tokens=147_124_984, n_requests=4427, host_blocks=853)
+    assert abs(a8["working_set_bytes"] / 2**30 - 5.3) < 0.05                   # "5.3 GiB" at A = 8
+    assert a8["working_set_exceeds_host"] == 0                                 # a 20 GiB tier holds it
+    rng = random.Random(8)
+    for _ in range(300):
+        L, H, d, s = rng.randrange(1, 80), rng.randrange(1, 33), rng.choice([64, 128]), rng.choice([1, 2, 4])
+        tp, b = rng.choice([1, 2, 4, 8, 16]), rng.choice([1, 16, 32, 1024])
+        A, n = rng.randrange(1, 300), rng.randrange(1, 10**5)
+        total = rng.randrange(0, 10**12)
+        kg, kh = rng.randrange(0, 10**6), rng.randrange(0, 10**6)
+        got = eakv.eakv_working_set(num_layers=L, kv_heads=H, head_dim=d, elem_bytes=s, tensor_parallel=tp,
+                                    block_size=b, active_pool=A, total_prompt_tokens=total, n_requests=n,
+                                    gpu_blocks=kg, host_blocks=kh)
+        beta = sizing.beta_rank(L, d, s, H, tp)
+        n_bar = Fraction(total, n)
+        ws = sizing.working_set_bytes(A, n_bar, beta)
+        assert got["beta_rank_bytes"] == beta
+        assert got["working_set_bytes"] == ws.numerator // ws.denominator
+        assert got["working_set_blocks"] == sizing.tier_chunks(ws, b, beta).__floor__()
+        if kg:
+            g = sizing.gamma_g(A, n_bar, kg * b)
+            assert abs(got["gamma_g"] - float(g)) <= 1e-12 * max(1.0, float(g)) and got["pool_exceeds_gpu"] == (g > 1)
+        if kh:
+            h = sizing.gamma_h(ws, kh * b * beta)
+            assert abs(got["gamma_h"] - float(h)) <= 1e-12 * max(1.0, float(h))
+            assert got["working_set_exceeds_host"] == (h > 1)
+    import pytest
+    with pytest.raises(eakv.EakvError):
+        eakv.eakv_working_set(num_layers=0, kv_heads=1, head_dim=8, block_size=16, active_pool=2,
+                              total_prompt_tokens=10, n_requests=1)

@@ -139,3 +139,45 @@ def test_aborted_turn_takes_back_what_it_never_produced(eakv):
     ctx.eakv_turn_end()
     assert ctx.eakv_match(longer)[:2] == (10, 10)
     ctx.close()
+
+
+def test_requests_overlap_and_an_unstored_release_takes_its_turn_back(eakv):
+    """eakv_request_*: two requests open at once share a prefix block; a request released before
+    its store is taken back like an aborted turn; refused ids and orders."""
+    b = 4
+    ctx = cp_ctx(eakv, b, 16, 32)
+    sys_key = 900
+    a = np.asarray([sys_key, 1, 2, 3], dtype=np.uint64)
+    c = np.asarray([sys_key, 11, 12], dtype=np.uint64)
+    va = ctx.eakv_request_begin(1, 0, 4 * b + 1, a, 0, 0)
+    vc = ctx.eakv_request_begin(2, 0, 3 * b, c, 1, 1)
+    assert va["gpu_block"][0] == vc["gpu_block"][0]                    # the shared first block
+    assert vc["gpu_resident"].tolist() == [1, 0, 0] and vc["hit"].tolist() == [1, 0, 0]
+    assert va["tail_block"] >= 0 and vc["tail_block"] == -1
+    for bad in (lambda: ctx.eakv_request_begin(1, 0, 4, a[:1], 0, 2),  # id in use
+                lambda: ctx.eakv_turn_begin(0, 4, a[:1], 0, 2),        # single turn while requests are open
+                lambda: ctx.eakv_request_store(3), lambda: ctx.eakv_request_release(3)):
+        with pytest.raises(eakv.EakvError) as ei:
+            bad()
+        assert ei.value.code == eakv.E_INVAL
+    # a third request that does not fit beside the two is refused and changes nothing
+    before = ctx.eakv_get_stats()
+    big = np.arange(100, 112, dtype=np.uint64)
+    assert ctx.eakv_request_begin(3, 0, 12 * b, big, 2, 3) is None
+    assert ctx.eakv_get_stats() == before and ctx.eakv_match(big)[:2] == (0, 0)
+    ctx.eakv_request_store(1)
+    with pytest.raises(eakv.EakvError):
+        ctx.eakv_request_store(1)                                      # once per begin
+    ctx.eakv_request_release(1)                                        # finished: everything stays listed
+    assert ctx.eakv_match(a)[:2] == (4, 4)
+    # request 2 is released without a store: its two new units and blocks are taken back, the shared
+    # block (stored by request 1) stays
+    ctx.eakv_request_release(2)
+    assert ctx.eakv_match(c)[:2] == (1, 1)
+    assert ctx.eakv_get_stats()["resident"] == 4
+    # now the big request fits
+    assert ctx.eakv_request_begin(3, 0, 12 * b, big, 2, 4) is not None
+    ctx.eakv_request_store(3)
+    ctx.eakv_request_release(3)
+    assert ctx.eakv_match(big)[:2] == (12, 12)
+    ctx.close()
