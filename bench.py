@@ -54,11 +54,18 @@ def parse_args():
     ap.add_argument("--copy-path", default="bulk", choices=["vector", "bulk"])
     ap.add_argument("--copy-ctas", type=int, default=0)
     ap.add_argument("--host-ctas", type=int, default=0)
+    ap.add_argument("--host-copy-path", default="vector", choices=["vector", "bulk_load", "bulk_both"],
+                    help="device code that moves a mapped host tier (zero-copy strategy)")
+    ap.add_argument("--host-load-ctas", type=int, default=0)
+    ap.add_argument("--host-store-ctas", type=int, default=0)
     ap.add_argument("--staging-mib", type=int, default=64)
     ap.add_argument("--no-overlap", dest="overlap", action="store_false",
                     help="e2e arm: restores and host writes on one stream instead of two")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quick", action="store_true",
+                    help="main line and e2e arm only: no side measurements (strategy matrix, curve, hash, "
+                         "control plane, CPU baseline); for sweeps")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--hash-only", action="store_true",
                     help="run only the prefix-hash throughput section and print its JSON")
@@ -166,7 +173,9 @@ class Arm:
             kw.update(tier_location=eakv.TIER_PINNED_HOST,
                       link_strategy={"staged": eakv.LINK_STAGED, "zero_copy": eakv.LINK_ZERO_COPY,
                                      "copy_engine": eakv.LINK_COPY_ENGINE}[link],
-                      staging_bytes=args.staging_mib << 20, copy_ctas=args.host_ctas)
+                      staging_bytes=args.staging_mib << 20, copy_ctas=args.host_ctas,
+                      host_copy_path={"vector": 0, "bulk_load": 1, "bulk_both": 2}[args.host_copy_path],
+                      host_load_ctas=args.host_load_ctas, host_store_ctas=args.host_store_ctas)
             if link == "staged":
                 kw["copy_ctas"] = args.copy_ctas
             if tier_memory is not None:
@@ -859,16 +868,17 @@ def main():
 
     achieved = kernel_rate(r)
     kernel_name = "copy_blocks_vector_kernel" if args.copy_path == "vector" else "copy_blocks_bulk_kernel"
-    # the other device copy path on the same step (fewer steps), so both appear side by side
-    other = "vector" if args.copy_path == "bulk" else "bulk"
-    arm_o = Arm(args, pool, shape, torch, eakv, host_tier=False, device=device, copy_path=other)
-    r_o = run_arm(arm_o, prompts_dev, tables, max(2, min(args.steps, 10)), min(args.warmup, 3), dist, None)
-    arm_o.ctx.close()
-    del arm_o
     by_copy_path = {args.copy_path: {"achieved": achieved, "frac": achieved / peak,
-                                     "launches_timed": len(r["kernel"])},
-                    other: {"achieved": kernel_rate(r_o), "frac": kernel_rate(r_o) / peak,
-                            "launches_timed": len(r_o["kernel"])}}
+                                     "launches_timed": len(r["kernel"])}}
+    if not args.quick:
+        # the other device copy path on the same step (fewer steps), so both appear side by side
+        other = "vector" if args.copy_path == "bulk" else "bulk"
+        arm_o = Arm(args, pool, shape, torch, eakv, host_tier=False, device=device, copy_path=other)
+        r_o = run_arm(arm_o, prompts_dev, tables, max(2, min(args.steps, 10)), min(args.warmup, 3), dist, None)
+        arm_o.ctx.close()
+        del arm_o
+        by_copy_path[other] = {"achieved": kernel_rate(r_o), "frac": kernel_rate(r_o) / peak,
+                               "launches_timed": len(r_o["kernel"])}
     # the profile's per-block DRAM traffic was captured on the unsharded shape
     traffic = read_profile_traffic(kernel_name, m) if args.tp_shard == 1 else None
 
@@ -891,7 +901,7 @@ def main():
                           time_kernels=False) for _ in range(2)]
         pass_ms = [aggregate_over_ranks(dist, p_["ms"], p_["moved"], device) for p_ in passes]
         re_ = passes[0] if pass_ms[0][0] <= pass_ms[1][0] else passes[1]
-        layered = layered_load_probe(torch, arm, tables, shape) if rank == 0 else None
+        layered = layered_load_probe(torch, arm, tables, shape) if (rank == 0 and not args.quick) else None
         arm.ctx.close()
         del arm
         e_ms, e_moved = aggregate_over_ranks(dist, re_["ms"], re_["moved"], device)
@@ -913,7 +923,7 @@ def main():
         # the same step under every host-link strategy, side by side (fewer steps each)
         by = {args.link: {"value": e_val, "frac_of_link": e2e.get("frac_of_link"), "steps": e_steps}}
         for name in ("staged", "zero_copy", "copy_engine"):
-            if name in by:
+            if name in by or args.quick:
                 continue
             a2 = Arm(args, pool, shape, torch, eakv, host_tier=True, device=device, link=name,
                      tier_memory=tier_ptr)
@@ -924,7 +934,7 @@ def main():
             v2 = mv2 / (ms2 * 1e-3) / 1e9
             by[name] = {"value": v2, "frac_of_link": v2 / bound / max(world, 1) if bound else None, "steps": 3}
         e2e["by_strategy"] = by
-        if rank == 0:
+        if rank == 0 and not args.quick:
             e2e["curve"] = guarded(store_load_curve, torch, eakv, pool, shape, device, args,
                                    link.get("h2d"), link.get("d2h"), tier_ptr, TIER_PROMPTS * m)
         del tier_pin
@@ -944,11 +954,12 @@ def main():
         e2e = guarded(e2e_section) if dist is None else e2e_section()
         if "error" in e2e:
             e2e.update(value=None, unit=UNIT)
-    hashing = guarded(hash_throughput, torch, eakv, pool, shape, device, peak) if rank == 0 else None
-    control = guarded(control_plane_rate, eakv, pool, shape, device) if rank == 0 else None
+    side = rank == 0 and not args.quick
+    hashing = guarded(hash_throughput, torch, eakv, pool, shape, device, peak) if side else None
+    control = guarded(control_plane_rate, eakv, pool, shape, device) if side else None
 
     cpu = None
-    if rank == 0 and not args.no_cpu_baseline:
+    if rank == 0 and not args.no_cpu_baseline and not args.quick:
         g, s, dt = oracle_step_rate_c(args.cpu_seconds)
         cpu = {"value": g, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"plain C oracle: {s} steps x 2 requests x 128 blocks of 1.5 MiB in {dt:.1f} s"}

@@ -78,6 +78,13 @@ extern "C" {
                                    used for device-resident buffers only: a mapped host tier
                                    under EAKV_LINK_ZERO_COPY is always moved by the vector kernel */
 
+/* which device code moves the bytes of a mapped host tier (EAKV_LINK_ZERO_COPY, and the scattered
+ * calls that EAKV_LINK_STAGED sends directly) */
+#define EAKV_HOST_COPY_VECTOR    0  /* (default) 16-byte loads and stores over the link                */
+#define EAKV_HOST_COPY_BULK_LOAD 1  /* restores: bulk async copies host -> shared memory -> pool;
+                                       stores keep the vector kernel                                  */
+#define EAKV_HOST_COPY_BULK_BOTH 2  /* both directions through the bulk-copy ring                      */
+
 /* GPU-tier recency order of one request's blocks after eakv_gpu_tier_step (the GPU tier belongs
  * to the serving engine in the paper, Section 2; both orders are this library's model of it) */
 #define EAKV_FREE_ASCENDING 0   /* as referenced: the prompt's first block is the request's least
@@ -151,6 +158,13 @@ typedef struct eakv_config {
     int64_t telemetry_max_age_ms;  /* a report older than this is not fresh (0: any age is).  Without a
                                       fresh report -- before the first publication, too -- p_t is the
                                       working-set test of Eq. 10 alone                                    */
+    int32_t host_copy_path;        /* EAKV_HOST_COPY_*                                                    */
+    int32_t host_load_ctas;        /* CTAs of a kernel that reads the mapped host tier; 0 = copy_ctas if
+                                      set, else 64                                                        */
+    int32_t host_store_ctas;       /* CTAs of a kernel that writes it; 0 = likewise.  Restores are
+                                      non-posted reads and stores posted writes, so with both directions
+                                      busy they want different grids                                      */
+    int32_t reserved0;
 } eakv_config;
 
 typedef struct eakv_stats {

@@ -202,13 +202,20 @@ void free_all(eakv_ctx* c) {
     delete c;
 }
 
+// grid of a kernel that touches the mapped host tier: per direction if configured
+// A few SMs saturate the host link and the rest stay with the engine.  Measured with restores
+// and writes running at once (zero-copy, vector kernel, 6 GiB each way): 16 CTAs 49.5 GB/s, 32: 63.7,
+// 64: 74.1, 128: 72.6, 296: 73.2; one direction alone is flat from 32 CTAs up.
+int host_ctas(const eakv_ctx* ctx, bool to_tier) {
+    const int dir = to_tier ? ctx->cfg.host_store_ctas : ctx->cfg.host_load_ctas;
+    if (dir > 0) return dir;
+    return ctx->cfg.copy_ctas > 0 ? ctx->cfg.copy_ctas : 64;
+}
+
 // grid of the vector kernel: the configured one, else sized here
 int vector_ctas(const eakv_ctx* ctx, bool touches_host) {
     if (ctx->cfg.copy_ctas > 0) return ctx->cfg.copy_ctas;
-    // A few SMs saturate the host link and the rest stay with the engine.  Measured with restores
-    // and writes running at once (zero-copy, 6 GiB each way): 16 CTAs 49.5 GB/s, 32: 63.7, 64: 74.1,
-    // 128: 72.6, 296: 73.2; one direction alone is flat from 32 CTAs up.
-    if (touches_host) return 64;
+    (void)touches_host;
     return ctx->sm_count * copy_vector_ctas_per_sm();
 }
 
@@ -236,12 +243,18 @@ int launch_copy(eakv_ctx* ctx, const int2* d_entries, const int2* h_inline, int6
     L.group_pieces = 1;          // the bulk launcher raises it for small pieces
     L.pad0 = 0;
     cudaError_t e;
-    // bulk async copies serve device-resident buffers; a mapped host tier is always driven
-    // by the vector kernel (few CTAs, plain loads/stores over the link)
-    if (ctx->cfg.copy_path == EAKV_COPY_BULK && !touches_host)
+    // a mapped host tier gets a small grid (a few SMs saturate the link) of the vector kernel or,
+    // if configured, the bulk-copy ring; device-resident buffers get the configured copy path
+    if (touches_host) {
+        const bool bulk = ctx->cfg.host_copy_path == EAKV_HOST_COPY_BULK_BOTH ||
+                          (ctx->cfg.host_copy_path == EAKV_HOST_COPY_BULK_LOAD && !to_tier);
+        if (bulk) e = launch_copy_bulk(L, to_tier, host_ctas(ctx, to_tier), ctx->sm_count, stream);
+        else      e = launch_copy_vector(L, to_tier, host_ctas(ctx, to_tier), stream);
+    } else if (ctx->cfg.copy_path == EAKV_COPY_BULK) {
         e = launch_copy_bulk(L, to_tier, ctx->cfg.copy_ctas > 0 ? ctx->cfg.copy_ctas : 0, ctx->sm_count, stream);
-    else
-        e = launch_copy_vector(L, to_tier, vector_ctas(ctx, touches_host), stream);
+    } else {
+        e = launch_copy_vector(L, to_tier, vector_ctas(ctx, false), stream);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, e, "copy kernel launch");
     ctx->stats.kernel_launches += 1;
     return EAKV_OK;
@@ -456,6 +469,8 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
         return EAKV_E_INVAL;
     if (cfg->gpu_index_blocks < 0 || cfg->gpu_index_blocks > cfg->gpu_blocks) return EAKV_E_INVAL;
     if (cfg->telemetry_period_ms < 0 || cfg->telemetry_max_age_ms < 0) return EAKV_E_INVAL;
+    if (cfg->host_copy_path < 0 || cfg->host_copy_path > 2 || cfg->host_load_ctas < 0 || cfg->host_store_ctas < 0)
+        return EAKV_E_INVAL;
     const int64_t piece = (int64_t)cfg->block_size * cfg->kv_heads * cfg->head_dim * cfg->elem_bytes;
     if (piece % 16 != 0) return EAKV_E_INVAL;
     const int pieces = 2 * cfg->num_layers;

@@ -15,6 +15,7 @@ LINK_ZERO_COPY, LINK_STAGED, LINK_COPY_ENGINE = 0, 1, 2
 TIER_PINNED_HOST, TIER_DEVICE = 0, 1
 FREE_ASCENDING, FREE_REVERSE = 0, 1
 COPY_VECTOR, COPY_BULK = 0, 1
+HOST_COPY_VECTOR, HOST_COPY_BULK_LOAD, HOST_COPY_BULK_BOTH = 0, 1, 2
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libeakv.so")
 _lib = None
@@ -46,6 +47,8 @@ class Config(C.Structure):
         ("tier_memory", C.c_void_p),
         ("gpu_free_order", C.c_int32), ("write_behind", C.c_int32),
         ("telemetry_period_ms", C.c_int64), ("telemetry_max_age_ms", C.c_int64),
+        ("host_copy_path", C.c_int32), ("host_load_ctas", C.c_int32), ("host_store_ctas", C.c_int32),
+        ("reserved0", C.c_int32),
     ]
 
 
@@ -271,7 +274,7 @@ class Context:
                  staging_bytes=0, max_call_blocks=0, hash_scratch_blocks=0, min_staged_run_bytes=0,
                  tier_memory=0, control_plane_only=False, chunk_blocks=1,
                  gpu_free_order=FREE_ASCENDING, write_behind=False, telemetry_period_ms=0,
-                 telemetry_max_age_ms=0):
+                 telemetry_max_age_ms=0, host_copy_path=0, host_load_ctas=0, host_store_ctas=0):
         L = lib()
         cfg = Config()
         L.eakv_config_init(C.byref(cfg))
@@ -288,6 +291,8 @@ class Context:
         cfg.gpu_free_order = int(gpu_free_order)
         cfg.write_behind = int(bool(write_behind))
         cfg.telemetry_period_ms, cfg.telemetry_max_age_ms = int(telemetry_period_ms), int(telemetry_max_age_ms)
+        cfg.host_copy_path = int(host_copy_path)
+        cfg.host_load_ctas, cfg.host_store_ctas = int(host_load_ctas), int(host_store_ctas)
         cfg.hash_base, cfg.hash_seed = hash_base, hash_seed
         cfg.policy, cfg.kappa_blocks, cfg.theta_percent = policy, kappa_blocks, theta_percent
         cfg.len_window, cfg.window_ms, cfg.telemetry = len_window, window_ms, telemetry
