@@ -410,6 +410,24 @@ def hash_throughput(torch, eakv, pool, shape, device, peak_gbs, prompts=512, tok
         if i >= 3:
             ts.append(e0.elapsed_time(e1) * 1e3)
     host_us = float(np.median(ts))
+    # what a lookup costs its caller: wall time from the call to the keys being readable on the host
+    # (tokens in pinned memory in, keys in pinned memory out), next to the floor any kernel pays on
+    # this machine through Python: one trivial kernel launch plus a stream synchronize
+    keys_pin = torch.empty(8192, dtype=torch.int64).pin_memory()
+    one = torch.zeros(1, device=device)
+
+    def wall_us(fn, reps=60):
+        ts = []
+        for i in range(reps + 5):
+            t0 = time.perf_counter()
+            fn()
+            stream.synchronize()
+            if i >= 5:
+                ts.append((time.perf_counter() - t0) * 1e6)
+        return float(np.median(ts))
+    lookup = {str(n): wall_us(lambda n=n: ctx.eakv_hash_blocks(host_toks.data_ptr(), n, seed, keys_pin.data_ptr(), stream))
+              for n in (16, 1024, 4096, 65536) if n <= n_host}
+    floor_us = wall_us(lambda: one.add_(1))
     ctx.close()
     rate = prompts * tokens / (best * 1e-3)
     srate = prompts * tokens / (sustained * 1e-3)
@@ -422,6 +440,9 @@ def hash_throughput(torch, eakv, pool, shape, device, peak_gbs, prompts=512, tok
             "hbm_bound_tokens_per_s": peak_gbs * 1e9 / 4,
             "single_prompt_tokens": tokens, "single_prompt_us_median": float(np.median(single)),
             "single_call_us_by_tokens": latency,
+            "lookup_wall_us_by_tokens": lookup, "launch_and_sync_floor_us": floor_us,
+            "lookup_note": "wall time of eakv_hash_blocks + stream synchronize, tokens and keys in pinned host "
+                           "memory; the floor is one trivial kernel launch + synchronize on the same stream",
             "host_resident_prompt": {"tokens": n_host, "us": host_us, "tokens_per_s": n_host / (host_us * 1e-6),
                                      "bytes_per_s": 4 * n_host / (host_us * 1e-6),
                                      "note": "tokens read from pinned host memory through the mapping"},

@@ -86,6 +86,14 @@ __device__ __forceinline__ Pair compose(Pair first, Pair second) {
 
 // Scan of one prompt's block partials into keys, by one whole CTA.
 //   partial[0..nblk) -> keys[0..nblk),  keys[j] = keys[j-1] * A + partial[j], keys[-1] = parent
+// SHARED: the partials sit in shared memory (a prompt that fits one CTA tile never goes through
+// global scratch); otherwise they are read from global memory past L1.
+template <bool SHARED>
+__device__ __forceinline__ uint64_t load_partial(const uint64_t* p) {
+    return SHARED ? *p : __ldcg(p);
+}
+
+template <bool SHARED>
 __device__ __noinline__ void scan_prompt(const uint64_t* partial, uint64_t* keys, int64_t nblk, uint64_t parent,
                             uint64_t A, Pair* warp_tot /* smem [32] */) {
     const int tid = threadIdx.x, nthr = blockDim.x;
@@ -98,7 +106,7 @@ __device__ __noinline__ void scan_prompt(const uint64_t* partial, uint64_t* keys
     const bool in_regs = per <= kRegRun;
     if (in_regs) {
 #pragma unroll
-        for (int i = 0; i < kRegRun; ++i) run[i] = (lo + i < hi) ? __ldcg(partial + lo + i) : 0;
+        for (int i = 0; i < kRegRun; ++i) run[i] = (lo + i < hi) ? load_partial<SHARED>(partial + lo + i) : 0;
     }
     Pair mine{1, 0};
     if (in_regs) {
@@ -124,7 +132,7 @@ __device__ __noinline__ void scan_prompt(const uint64_t* partial, uint64_t* keys
         }
     } else {
         for (int64_t j = lo; j < hi; ++j) {
-            const uint64_t c = __ldcg(partial + j);
+            const uint64_t c = load_partial<SHARED>(partial + j);
             mine.a = mulmod61(mine.a, A);
             mine.c = addmod61(mulmod61(mine.c, A), c);
         }
@@ -169,7 +177,7 @@ __device__ __noinline__ void scan_prompt(const uint64_t* partial, uint64_t* keys
         }
     } else {
         for (int64_t j = lo; j < hi; ++j) {
-            h = addmod61(mulmod61(h, A), __ldcg(partial + j));
+            h = addmod61(mulmod61(h, A), load_partial<SHARED>(partial + j));
             keys[j] = h;
         }
     }
@@ -262,7 +270,7 @@ hash_blocks_kernel(HashLaunch L) {
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    scan_prompt(partial, L.keys + blk0, nblk, parent, pw[L.block_size], warp_tot);
+    scan_prompt<false>(partial, L.keys + blk0, nblk, parent, pw[L.block_size], warp_tot);
     if (tid == 0) L.counters[p] = 0;   // ready for the next launch
 }
 
@@ -362,7 +370,7 @@ hash_blocks_tpb_kernel(HashLaunch L) {
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    scan_prompt(partial, L.keys + blk0, nblk, parent, L.pow_table[b], warp_tot);
+    scan_prompt<false>(partial, L.keys + blk0, nblk, parent, L.pow_table[b], warp_tot);
     if (tid == 0) L.counters[p] = 0;
 }
 #undef EAKV_MAC3
@@ -468,6 +476,11 @@ hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
         }
         __syncthreads();     // the limb table is shared by the whole CTA
     }
+    // A single prompt that fits this one CTA (at most kHashThreads blocks) never leaves the CTA:
+    // its partials stay in shared memory and the scan follows after one barrier -- no global
+    // scratch, no fence, no ticket.
+    __shared__ uint64_t local_partial[kHashThreads];
+    const bool lone = L.tiles == nullptr && gridDim.x == 1 && nb_tile <= kHashThreads;
     uint64_t* partial = L.partial + blk0;
     for (int r = 0; r < n_sub; ++r) {
         if (r + S - 1 < n_sub) issue(r + S - 1);
@@ -504,9 +517,15 @@ hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
                     acc = addmod61(acc, fold_limb_sums(s0, s1, s2));
                 }
             }
-            __stcg(partial + first_blk + j, acc);
+            if (lone) local_partial[j] = acc;
+            else __stcg(partial + first_blk + j, acc);
         }
         __syncwarp();        // this warp refills the stage S-1 iterations from now
+    }
+    if (lone) {
+        __syncthreads();
+        scan_prompt<true>(local_partial, L.keys + blk0, nblk, parent, L.pow_block, warp_tot);
+        return;
     }
     __threadfence();
     __syncthreads();
@@ -517,7 +536,7 @@ hash_blocks_staged_kernel(const __grid_constant__ HashLaunch L) {
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    scan_prompt(partial, L.keys + blk0, nblk, parent, L.pow_block, warp_tot);
+    scan_prompt<false>(partial, L.keys + blk0, nblk, parent, L.pow_block, warp_tot);
     if (tid == 0) L.counters[p] = 0;
 }
 #undef EAKV_MAC3
