@@ -54,7 +54,7 @@ def parse_args():
     ap.add_argument("--copy-path", default="bulk", choices=["vector", "bulk"])
     ap.add_argument("--copy-ctas", type=int, default=0)
     ap.add_argument("--host-ctas", type=int, default=0)
-    ap.add_argument("--host-copy-path", default="vector", choices=["vector", "bulk_load", "bulk_both"],
+    ap.add_argument("--host-copy-path", default="bulk_load", choices=["vector", "bulk_load", "bulk_both"],
                     help="device code that moves a mapped host tier (zero-copy strategy)")
     ap.add_argument("--host-load-ctas", type=int, default=0)
     ap.add_argument("--host-store-ctas", type=int, default=0)

@@ -204,12 +204,18 @@ void free_all(eakv_ctx* c) {
 
 // grid of a kernel that touches the mapped host tier: per direction if configured
 // A few SMs saturate the host link and the rest stay with the engine.  Measured with restores
-// and writes running at once (zero-copy, vector kernel, 6 GiB each way): 16 CTAs 49.5 GB/s, 32: 63.7,
-// 64: 74.1, 128: 72.6, 296: 73.2; one direction alone is flat from 32 CTAs up.
+// and writes running at once (zero-copy, 6 GiB each way, GB/s of both directions together):
+// vector kernel both ways, one grid size: 16 CTAs 49.5, 32: 63.7, 64: 73-74, 128: 72.6, 296: 73.2;
+// restores through the bulk-copy ring (load CTAs / store CTAs): 32/64 65.0, 48/64 70.5, 64/48 73.7,
+// 64/64 78.1, 80/80 77.1, 96/64 78.8, 64/96 70.5, 64/128 63.0, 148/32 59.9 -- more writers starve
+// the read requests, which share the upstream direction with the posted writes.  One direction
+// alone is flat from 32 CTAs up (52 GB/s with either kernel).
 int host_ctas(const eakv_ctx* ctx, bool to_tier) {
     const int dir = to_tier ? ctx->cfg.host_store_ctas : ctx->cfg.host_load_ctas;
     if (dir > 0) return dir;
-    return ctx->cfg.copy_ctas > 0 ? ctx->cfg.copy_ctas : 64;
+    if (ctx->cfg.copy_ctas > 0) return ctx->cfg.copy_ctas;
+    const bool bulk_load = !to_tier && ctx->cfg.host_copy_path != EAKV_HOST_COPY_VECTOR;
+    return bulk_load ? 96 : 64;
 }
 
 // grid of the vector kernel: the configured one, else sized here
@@ -450,6 +456,7 @@ int eakv_config_init(eakv_config* cfg) {
     cfg->link_strategy = EAKV_LINK_STAGED;
     cfg->tier_location = EAKV_TIER_PINNED_HOST;
     cfg->copy_path = EAKV_COPY_BULK;
+    cfg->host_copy_path = EAKV_HOST_COPY_BULK_LOAD;
     return EAKV_OK;
 }
 

@@ -9,16 +9,15 @@
 //     D_i = #{ j < i : prev_j < p } - (p + 1).
 //
 // Steps, all data-parallel:
-//   1. prev[]: stable sort of (key, position) pairs by key (CUB radix sort, the one library
-//      primitive used here); equal neighbours give each position its predecessor.
+//   1. prev[]: stable sort of (key, position) pairs by key (a least-significant-digit radix sort
+//      written here: eight passes of 8 bits, three kernels per pass, no kernel waits for another);
+//      equal neighbours give each position its predecessor.
 //   2. a wavelet matrix over v_j = prev_j + 1 (one stable 0/1 partition per bit, built with a
 //      three-kernel exclusive scan per level: no kernel waits for another);
 //   3. one "count of values below x in a prefix" query per reference, nbits steps each.
 // The capacity curve then needs only D: a reference hits a tier of K chunks iff D < K
 // (Mattson); a request's host coverage is its leading run of hits; restored = max(0, H - G);
 // computed prefill = n - max(G, H) * b.
-#include <cub/device/device_radix_sort.cuh>
-
 #include <algorithm>
 #include <cstdint>
 #include <vector>
@@ -31,10 +30,123 @@ constexpr int kSdThreads = 256;
 constexpr int kSdItems = 4;                         // elements per thread in the scan kernels
 constexpr int kSdTile = kSdThreads * kSdItems;      // 1024 elements per CTA
 
-// ---- step 1 ---------------------------------------------------------------------------------
-__global__ void iota_kernel(int32_t* idx, int64_t n) {
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) idx[i] = (int32_t)i;
+// ---- step 1: stable LSD radix sort of (key, position) ---------------------------------------
+// One pass sorts by the 8-bit digit at `shift`.  A CTA owns a tile of kRsTile consecutive
+// elements.  (a) per-tile digit counts, stored digit-major: counts[digit][tile]; (b) one CTA per
+// digit turns its row into exclusive offsets across tiles and leaves the digit's total; (c) every
+// CTA scans the 256 totals into digit bases, then walks its tile in rounds of kRsThreads elements
+// in order, ranking equal digits by (round, warp, lane) so that the pass is stable, and scatters.
+constexpr int kRsThreads = 256;
+constexpr int kRsItems = 8;
+constexpr int kRsTile = kRsThreads * kRsItems;      // 2048 elements per CTA
+constexpr int kRsDigits = 256;
+
+__global__ void __launch_bounds__(kRsThreads)
+rs_count_kernel(const uint64_t* __restrict__ keys, int64_t n, int shift, int n_tiles,
+                int32_t* __restrict__ counts /* [256][n_tiles] */) {
+    __shared__ int hist[kRsDigits];
+    hist[threadIdx.x] = 0;
+    __syncthreads();
+    const int64_t base = (int64_t)blockIdx.x * kRsTile;
+#pragma unroll
+    for (int k = 0; k < kRsItems; ++k) {
+        const int64_t i = base + k * kRsThreads + threadIdx.x;
+        if (i < n) atomicAdd(&hist[(int)((keys[i] >> shift) & 255u)], 1);
+    }
+    __syncthreads();
+    counts[(int64_t)threadIdx.x * n_tiles + blockIdx.x] = hist[threadIdx.x];
+}
+
+// one CTA per digit: exclusive scan of its row of tile counts (in place), total to totals[digit]
+__global__ void __launch_bounds__(1024)
+rs_scan_rows_kernel(int32_t* __restrict__ counts, int n_tiles, int32_t* __restrict__ totals) {
+    __shared__ int warp_tot[32];
+    __shared__ int carry_s;
+    int32_t* row = counts + (int64_t)blockIdx.x * n_tiles;
+    if (threadIdx.x == 0) carry_s = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int base = 0; base < n_tiles; base += 1024) {
+        const int i = base + threadIdx.x;
+        const int x = i < n_tiles ? row[i] : 0;
+        int inc = x;
+        for (int d = 1; d < 32; d <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, inc, d);
+            if (lane >= d) inc += up;
+        }
+        if (lane == 31) warp_tot[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            int w = warp_tot[lane];
+            for (int d = 1; d < 32; d <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, w, d);
+                if (lane >= d) w += up;
+            }
+            warp_tot[lane] = w;
+        }
+        __syncthreads();
+        const int carry = carry_s;
+        if (i < n_tiles) row[i] = carry + (warp ? warp_tot[warp - 1] : 0) + inc - x;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry_s = carry + warp_tot[31];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) totals[blockIdx.x] = carry_s;
+}
+
+// idx_in == NULL: the value of element i is its position i (first pass)
+__global__ void __launch_bounds__(kRsThreads)
+rs_scatter_kernel(const uint64_t* __restrict__ keys_in, const int32_t* __restrict__ idx_in, int64_t n,
+                  int shift, int n_tiles, const int32_t* __restrict__ counts /* exclusive, [256][n_tiles] */,
+                  const int32_t* __restrict__ totals, uint64_t* __restrict__ keys_out,
+                  int32_t* __restrict__ idx_out) {
+    __shared__ int digit_base[kRsDigits];            // where this tile's elements of a digit start
+    __shared__ int warp_count[kRsThreads / 32][kRsDigits];
+    __shared__ int scan_tmp[kRsThreads / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    {   // exclusive scan of the 256 digit totals + this tile's offset inside each digit
+        const int t = totals[tid];
+        int inc = t;
+        for (int d = 1; d < 32; d <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, inc, d);
+            if (lane >= d) inc += up;
+        }
+        if (lane == 31) scan_tmp[warp] = inc;
+        __syncthreads();
+        int before = inc - t;
+        for (int w = 0; w < warp; ++w) before += scan_tmp[w];
+        digit_base[tid] = before + counts[(int64_t)tid * n_tiles + blockIdx.x];
+    }
+    for (int w = 0; w < kRsThreads / 32; ++w) warp_count[w][tid] = 0;
+    __syncthreads();
+    const int64_t base = (int64_t)blockIdx.x * kRsTile;
+    for (int k = 0; k < kRsItems; ++k) {
+        const int64_t i = base + k * kRsThreads + tid;
+        const bool live = i < n;
+        const uint64_t key = live ? keys_in[i] : 0;
+        const int d = live ? (int)((key >> shift) & 255u) : -1;
+        // lanes of this warp with the same digit; dead lanes (d = -1) only match each other
+        const unsigned peers = __match_any_sync(0xffffffffu, d);
+        const int rank = __popc(peers & ((1u << lane) - 1u));
+        if (live && rank == 0) warp_count[warp][d] = __popc(peers);
+        __syncthreads();
+        if (live) {
+            int off = digit_base[d] + rank;
+            for (int w = 0; w < warp; ++w) off += warp_count[w][d];
+            keys_out[off] = key;
+            idx_out[off] = idx_in ? idx_in[i] : (int32_t)i;
+        }
+        __syncthreads();
+        {   // this round's elements of digit `tid` are placed: advance the base, clear the counts
+            int sum = 0;
+            for (int w = 0; w < kRsThreads / 32; ++w) {
+                sum += warp_count[w][tid];
+                warp_count[w][tid] = 0;
+            }
+            digit_base[tid] += sum;
+        }
+        __syncthreads();
+    }
 }
 
 // sorted by (key, position): the predecessor of a position is its left neighbour with the same key
@@ -315,15 +427,15 @@ static int reuse_distances_impl(const uint64_t* keys_dev, int64_t n_refs, int64_
     const int grid1 = (int)((n + 255) / 256);
 
     int rc = EAKV_OK;
-    uint64_t* keys_sorted = nullptr;
-    int32_t *idx = nullptr, *idx_sorted = nullptr, *prev = nullptr, *zeros_before = nullptr;
-    int32_t *tile_zeros = nullptr, *level_zeros = nullptr;
+    uint64_t *keys_sorted = nullptr, *keys_tmp = nullptr;
+    int32_t *idx_tmp = nullptr, *idx_sorted = nullptr, *prev = nullptr, *zeros_before = nullptr;
+    int32_t *tile_zeros = nullptr, *level_zeros = nullptr, *rs_counts = nullptr, *rs_totals = nullptr;
     uint32_t *va = nullptr, *vb = nullptr;
-    void* sort_tmp = nullptr;
-    size_t sort_bytes = 0;
+    const int rs_tiles = (int)((n + kRsTile - 1) / kRsTile);
 
     SD_CU(cudaMalloc(&keys_sorted, n * 8));
-    SD_CU(cudaMalloc(&idx, n * 4));
+    SD_CU(cudaMalloc(&keys_tmp, n * 8));
+    SD_CU(cudaMalloc(&idx_tmp, n * 4));
     SD_CU(cudaMalloc(&idx_sorted, n * 4));
     SD_CU(cudaMalloc(&prev, n * 4));
     SD_CU(cudaMalloc(&va, n * 4));
@@ -331,13 +443,21 @@ static int reuse_distances_impl(const uint64_t* keys_dev, int64_t n_refs, int64_
     SD_CU(cudaMalloc(&zeros_before, (size_t)nbits * (n + 1) * 4));
     SD_CU(cudaMalloc(&tile_zeros, (size_t)n_tiles * 4));
     SD_CU(cudaMalloc(&level_zeros, (size_t)nbits * 4));
-    SD_CU(cub::DeviceRadixSort::SortPairs(nullptr, sort_bytes, keys_dev, keys_sorted, idx, idx_sorted,
-                                          (int)n, 0, 61, stream));
-    SD_CU(cudaMalloc(&sort_tmp, sort_bytes));
+    SD_CU(cudaMalloc(&rs_counts, (size_t)kRsDigits * rs_tiles * 4));
+    SD_CU(cudaMalloc(&rs_totals, kRsDigits * 4));
 
-    iota_kernel<<<grid1, 256, 0, stream>>>(idx, n);
-    SD_CU(cub::DeviceRadixSort::SortPairs(sort_tmp, sort_bytes, keys_dev, keys_sorted, idx, idx_sorted,
-                                          (int)n, 0, 61, stream));
+    // eight stable passes over the 61-bit keys, least significant digit first; the buffers alternate
+    // so that the last pass lands in keys_sorted / idx_sorted
+    for (int pass = 0; pass < 8; ++pass) {
+        const uint64_t* kin = pass == 0 ? keys_dev : ((pass & 1) ? keys_tmp : keys_sorted);
+        const int32_t* iin = pass == 0 ? nullptr : ((pass & 1) ? idx_tmp : idx_sorted);
+        uint64_t* kout = (pass & 1) ? keys_sorted : keys_tmp;
+        int32_t* iout = (pass & 1) ? idx_sorted : idx_tmp;
+        rs_count_kernel<<<rs_tiles, kRsThreads, 0, stream>>>(kin, n, 8 * pass, rs_tiles, rs_counts);
+        rs_scan_rows_kernel<<<kRsDigits, 1024, 0, stream>>>(rs_counts, rs_tiles, rs_totals);
+        rs_scatter_kernel<<<rs_tiles, kRsThreads, 0, stream>>>(kin, iin, n, 8 * pass, rs_tiles, rs_counts, rs_totals,
+                                                               kout, iout);
+    }
     prev_from_sorted_kernel<<<grid1, 256, 0, stream>>>(keys_sorted, idx_sorted, n, prev, va, next_dev);
     for (int l = 0; l < nbits; ++l) {
         const int shift = nbits - 1 - l;
@@ -352,9 +472,9 @@ static int reuse_distances_impl(const uint64_t* keys_dev, int64_t n_refs, int64_
     SD_CU(cudaGetLastError());
     SD_CU(cudaStreamSynchronize(stream));
 done:
-    cudaFree(keys_sorted); cudaFree(idx); cudaFree(idx_sorted); cudaFree(prev); cudaFree(va);
-    cudaFree(vb); cudaFree(zeros_before); cudaFree(tile_zeros); cudaFree(level_zeros);
-    cudaFree(sort_tmp);
+    cudaFree(keys_sorted); cudaFree(keys_tmp); cudaFree(idx_tmp); cudaFree(idx_sorted); cudaFree(prev);
+    cudaFree(va); cudaFree(vb); cudaFree(zeros_before); cudaFree(tile_zeros); cudaFree(level_zeros);
+    cudaFree(rs_counts); cudaFree(rs_totals);
     if (rc != EAKV_OK) cudaGetLastError();
     return rc;
 }

@@ -274,7 +274,7 @@ class Context:
                  staging_bytes=0, max_call_blocks=0, hash_scratch_blocks=0, min_staged_run_bytes=0,
                  tier_memory=0, control_plane_only=False, chunk_blocks=1,
                  gpu_free_order=FREE_ASCENDING, write_behind=False, telemetry_period_ms=0,
-                 telemetry_max_age_ms=0, host_copy_path=0, host_load_ctas=0, host_store_ctas=0):
+                 telemetry_max_age_ms=0, host_copy_path=HOST_COPY_BULK_LOAD, host_load_ctas=0, host_store_ctas=0):
         L = lib()
         cfg = Config()
         L.eakv_config_init(C.byref(cfg))

@@ -36,8 +36,9 @@ def variants():
     # the default: staged, but scattered slots fall back to the direct kernel
     out.append(dict(link_strategy=e.LINK_STAGED, tier_location=e.TIER_PINNED_HOST,
                     copy_path=e.COPY_BULK, min_staged_run_bytes=0))
-    # a mapped host tier moved by the bulk-copy ring (restores only, or both directions)
-    for hp in (e.HOST_COPY_BULK_LOAD, e.HOST_COPY_BULK_BOTH):
+    # a mapped host tier moved by the vector kernel both ways, or by the bulk-copy ring (restores
+    # only, which is the default, or both directions), with small explicit grids
+    for hp in (e.HOST_COPY_VECTOR, e.HOST_COPY_BULK_LOAD, e.HOST_COPY_BULK_BOTH):
         out.append(dict(link_strategy=e.LINK_ZERO_COPY, tier_location=e.TIER_PINNED_HOST, host_copy_path=hp,
                         host_load_ctas=8, host_store_ctas=4))
     # copy engine only: needs the piece arrays at one pitch, i.e. one allocation for the whole pool
