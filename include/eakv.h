@@ -48,6 +48,8 @@ extern "C" {
 #define EAKV_E_NOMEM     -4   /* host, pinned or device allocation failed */
 #define EAKV_E_CUDA      -5   /* a CUDA runtime call failed; see eakv_last_cuda_error */
 #define EAKV_E_TIMEOUT   -6   /* a bounded device-side wait gave up (bulk-copy path) */
+#define EAKV_E_BUSY      -7   /* a running request's GPU blocks do not fit beside those the other running
+                                 requests hold: nothing changed; retry after a request was released */
 
 /* write admission (Section 4, Eq. 6): save(r) = not (p_t and u > kappa) */
 #define EAKV_POLICY_WRITE_ALL          0   /* p_t = 0: plain offload                      */
@@ -308,9 +310,10 @@ int eakv_gpu_tier_release(eakv_ctx* ctx, int32_t block_id);
  * eakv_gpu_tier_step for a request that stays running: it references the keys in order in the same
  * way and then keeps every block of the prompt (and the tail block) pinned under request_id, out
  * of the recency order, so that no other request can take them.  A block already pinned by
- * another running request (a shared prefix) is shared.  EAKV_E_CAPACITY, nothing changed, when the
+ * another running request (a shared prefix) is shared.  EAKV_E_BUSY, nothing changed, when the
  * blocks nobody holds do not suffice: the caller waits, or suspends a running request with
- * eakv_gpu_tier_release_request and tries again.  eakv_gpu_tier_release_request lets a finished
+ * eakv_gpu_tier_release_request and tries again.  EAKV_E_CAPACITY when the prompt could not be held
+ * even with no other request running.  eakv_gpu_tier_release_request lets a finished
  * or suspended request's blocks go: those no other request holds re-enter the recency order at
  * the most-recent end in prompt order (tail first under EAKV_FREE_REVERSE) and keep their keys, so a
  * resumed request finds what has not been evicted meanwhile; the tail block is freed.  With one
@@ -400,9 +403,9 @@ int eakv_turn_abort(eakv_ctx* ctx);
  * running requests; Appendix A: 16) and suspends one when GPU KV memory runs out.  Any number of
  * requests may be open, each under a request_id of the caller's choosing.
  * eakv_request_begin: as eakv_turn_begin, but the prompt's GPU blocks are taken with
- * eakv_gpu_tier_acquire and stay pinned under request_id.  EAKV_E_CAPACITY, with neither tier
+ * eakv_gpu_tier_acquire and stay pinned under request_id.  EAKV_E_BUSY, with neither tier
  * changed, when they do not fit beside the running requests: wait, or suspend a running request
- * (eakv_request_release) and try again.  decided: -1 for the request's first lookup; 0 / 1 for a
+ * (eakv_request_release) and try again (EAKV_E_CAPACITY: the prompt exceeds a tier on its own).  decided: -1 for the request's first lookup; 0 / 1 for a
  * later lookup of a resumed request, carrying the skip / store choice of its first one (Appendix D;
  * see eakv_tier_step_again).  *view's arrays stay valid until the request is released.
  * eakv_request_store: after the engine has produced the blocks flagged needs_fill, eakv_store of

@@ -1018,7 +1018,8 @@ int eakv_gpu_tier_acquire(eakv_ctx* ctx, int64_t request_id, const uint64_t* has
         const int32_t s = T.find(hashes_host[j]);
         if (s < 0 || !T.is_pinned(s)) ++cost;
     }
-    if (cost > T.free_slots() + T.evictable()) return EAKV_E_CAPACITY;
+    if (n_blocks + (need_tail ? 1 : 0) > T.capacity()) return EAKV_E_CAPACITY;   // never fits
+    if (cost > T.free_slots() + T.evictable()) return EAKV_E_BUSY;               // not beside the others
     eakv_ctx::HeldRequest& h = ctx->held[request_id];
     h.blocks.resize((size_t)n_blocks);
     bool ev;
@@ -1485,6 +1486,7 @@ const char* eakv_strerror(int code) {
         case EAKV_E_NOMEM: return "out of memory";
         case EAKV_E_CUDA: return "CUDA runtime error";
         case EAKV_E_TIMEOUT: return "device-side wait timed out";
+        case EAKV_E_BUSY: return "GPU blocks held by running requests leave no room";
         default: return "unknown error";
     }
 }

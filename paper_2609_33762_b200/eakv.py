@@ -9,7 +9,7 @@ import os
 
 import numpy as np
 
-OK, E_INVAL, E_RANGE, E_CAPACITY, E_NOMEM, E_CUDA, E_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
+OK, E_INVAL, E_RANGE, E_CAPACITY, E_NOMEM, E_CUDA, E_TIMEOUT, E_BUSY = 0, -1, -2, -3, -4, -5, -6, -7
 POLICY_WRITE_ALL, POLICY_FILTER_FIXED, POLICY_FILTER_CONDITIONED = 0, 1, 2
 LINK_ZERO_COPY, LINK_STAGED, LINK_COPY_ENGINE = 0, 1, 2
 TIER_PINNED_HOST, TIER_DEVICE = 0, 1
@@ -455,7 +455,7 @@ class Context:
         rc = lib().eakv_gpu_tier_acquire(self._h, int(request_id), hp, n, int(bool(need_tail)),
                                          res.ctypes.data_as(C.c_void_p), blk.ctypes.data_as(C.c_void_p),
                                          C.byref(tail))
-        if rc == E_CAPACITY:
+        if rc == E_BUSY:
             return None
         self._check(rc, "eakv_gpu_tier_acquire")
         return res, blk, tail.value
@@ -517,7 +517,7 @@ class Context:
         rc = lib().eakv_request_begin(self._h, int(request_id), C.c_void_p(int(tokens_ptr)), int(n_tokens), kp, nk,
                                       int(agent_id), int(now_ms), -1 if decided is None else int(bool(decided)),
                                       _stream(stream), C.byref(v))
-        if rc == E_CAPACITY:
+        if rc == E_BUSY:
             return None
         self._check(rc, "eakv_request_begin")
         return self._view_dict(v)

@@ -91,7 +91,14 @@ def test_single_request_calls_are_refused_while_requests_hold_blocks(mods):
     with pytest.raises(eakv.EakvError) as ei:
         ctx.eakv_gpu_tier_acquire(7, as_keys([4]), False)     # the id is in use
     assert ei.value.code == eakv.E_INVAL
+    # too large for the tier even alone: an error, not "try again later"
+    with pytest.raises(eakv.EakvError) as ei:
+        ctx.eakv_gpu_tier_acquire(8, as_keys(range(100, 117)), False)
+    assert ei.value.code == eakv.E_CAPACITY
+    assert ctx.eakv_gpu_tier_acquire(8, as_keys(range(100, 114)), False) is None      # 14 > 16 - 4 held: busy
     ctx.eakv_gpu_tier_release_request(7)
+    assert ctx.eakv_gpu_tier_acquire(8, as_keys(range(100, 114)), False) is not None
+    ctx.eakv_gpu_tier_release_request(8)
     ctx.eakv_gpu_tier_step(as_keys([9]), False)
     ctx.close()
 
