@@ -62,31 +62,40 @@ class AgentServer:
         self.shape = shape
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
-        # data_plane=False runs keys, matching and both tiers' bookkeeping only; the pool is
-        # then a one-block placeholder and no KV bytes move
+        # data_plane=False runs keys, matching and both tiers' bookkeeping only: no KV bytes move.
+        # The bookkeeping then lives in a control-plane-only context (no tier memory, no staging),
+        # which runs the library's turn engine from keys alone; a second, minimal context on the
+        # device does nothing but hash.
         self.data_plane = data_plane
         self.pool = PagedPool(shape, gpu_blocks if data_plane else 1, device)
-        if not data_plane and "tier_memory" not in ctx_kwargs:
-            # bookkeeping-only run: adopt a token buffer so no tier-sized memory is pinned
+        common = dict(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+                      block_size=shape.block_size, elem_bytes=shape.elem_bytes)
+        if data_plane:
+            self.ctx = eakv.Context(gpu_blocks=gpu_blocks, host_blocks=host_blocks,
+                                    gpu_index_blocks=gpu_index_blocks, kv_base=self.pool.kv_base,
+                                    chunk_blocks=chunk_blocks, **common, **ctx_kwargs)
+            self.hash_ctx = self.ctx
+        else:
             self._no_tier = torch.zeros(16, dtype=torch.uint8, device=self.device)
-            ctx_kwargs["tier_memory"] = self._no_tier.data_ptr()
-            ctx_kwargs["tier_location"] = eakv.TIER_DEVICE
-        self.ctx = eakv.Context(
-            num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
-            block_size=shape.block_size, elem_bytes=shape.elem_bytes, gpu_blocks=gpu_blocks,
-            host_blocks=host_blocks, gpu_index_blocks=gpu_index_blocks, kv_base=self.pool.kv_base,
-            chunk_blocks=chunk_blocks, **ctx_kwargs)
+            hash_kw = {k: ctx_kwargs[k] for k in ("hash_base", "hash_seed", "hash_scratch_blocks") if k in ctx_kwargs}
+            self.hash_ctx = eakv.Context(gpu_blocks=1, host_blocks=1, kv_base=self.pool.kv_base,
+                                         tier_memory=self._no_tier.data_ptr(), tier_location=eakv.TIER_DEVICE,
+                                         **common, **hash_kw)
+            book_kw = {k: v for k, v in ctx_kwargs.items()
+                       if k not in ("tier_memory", "tier_location", "link_strategy", "copy_path", "copy_ctas",
+                                    "staging_bytes", "hash_scratch_blocks", "write_behind")}
+            self.ctx = eakv.Context(gpu_blocks=gpu_blocks, host_blocks=host_blocks,
+                                    gpu_index_blocks=gpu_index_blocks, kv_base=None, control_plane_only=True,
+                                    chunk_blocks=chunk_blocks, **common, **book_kw)
         self.payload = payload
         self.incremental = incremental_hash
         self.stream = torch.cuda.current_stream(self.device)
         self.b = shape.block_size
         self.R = max(1, int(chunk_blocks))
         if native_turn is None:
-            native_turn = bool(data_plane)
+            native_turn = True
         self.native_turn = native_turn     # drive turns through the library's turn engine
-        if native_turn and not data_plane:
-            raise ValueError("the two-call turn engine always moves KV bytes: it needs the data plane")
-        self.seed = self.ctx.eakv_hash_seed()
+        self.seed = self.hash_ctx.eakv_hash_seed()
         self._agent_keys = {}          # agent -> np.uint64 keys of its previous prompt
         self._timed = {"load": [], "store": []}     # (bytes, start event, end event)
         self.records = []
@@ -95,6 +104,8 @@ class AgentServer:
 
     def close(self):
         self.ctx.close()
+        if self.hash_ctx is not self.ctx:
+            self.hash_ctx.close()
 
     def _time(self, kind, nbytes):
         """Context manager bracketing one store/load call with CUDA events on its stream."""
@@ -145,8 +156,8 @@ class AgentServer:
             self._ensure_pinned(seg_len)
             self._tok_pin.numpy()[:seg_len] = tokens[start * self.b: nblk * self.b]
             parent = int(out[start - 1]) if start else self.seed
-            got = self.ctx.eakv_hash_blocks(self._tok_pin.data_ptr(), seg_len, parent,
-                                            self._keys_pin.data_ptr(), self.stream)
+            got = self.hash_ctx.eakv_hash_blocks(self._tok_pin.data_ptr(), seg_len, parent,
+                                                 self._keys_pin.data_ptr(), self.stream)
             assert got == nblk - start
             self.stream.synchronize()
             out[start:] = self._keys_pin.numpy()[:got].view(np.uint64)
@@ -159,12 +170,15 @@ class AgentServer:
         """The same turn through the library's two-call engine: lookup, bookkeeping and the
         restore happen inside eakv_turn_begin, the store inside eakv_turn_end."""
         n = len(tokens)
-        self._ensure_pinned(max(n, 1))
-        self._tok_pin.numpy()[:n] = tokens
-        known = self._agent_keys.get(agent) if self.incremental else None
-        v = self.ctx.eakv_turn_begin(self._tok_pin.data_ptr(), n, known, agent, now_ms, self.stream)
+        if self.data_plane:
+            self._ensure_pinned(max(n, 1))
+            self._tok_pin.numpy()[:n] = tokens
+            known = self._agent_keys.get(agent) if self.incremental else None
+            v = self.ctx.eakv_turn_begin(self._tok_pin.data_ptr(), n, known, agent, now_ms, self.stream)
+        else:       # bookkeeping only: the hashing context supplies every key
+            v = self.ctx.eakv_turn_begin(0, n, self.block_keys(tokens, agent), agent, now_ms)
         keys, blocks = v["keys"], v["gpu_block"]
-        if self.incremental:
+        if self.incremental and self.data_plane:
             self._agent_keys[agent] = keys
         self._fill(keys, blocks, np.nonzero(v["needs_fill"])[0])
         self.ctx.eakv_turn_end(self.stream)
@@ -250,15 +264,19 @@ class AgentServer:
     def _begin_native(self, request_id, tokens, agent, now_ms, decided):
         """The same through eakv_request_begin / eakv_request_store."""
         n = len(tokens)
-        self._ensure_pinned(max(n, 1))
-        self._tok_pin.numpy()[:n] = tokens
-        known = self._agent_keys.get(agent) if self.incremental else None
-        v = self.ctx.eakv_request_begin(request_id, self._tok_pin.data_ptr(), n, known, agent, now_ms,
-                                        decided=decided, stream=self.stream)
+        if self.data_plane:
+            self._ensure_pinned(max(n, 1))
+            self._tok_pin.numpy()[:n] = tokens
+            known = self._agent_keys.get(agent) if self.incremental else None
+            v = self.ctx.eakv_request_begin(request_id, self._tok_pin.data_ptr(), n, known, agent, now_ms,
+                                            decided=decided, stream=self.stream)
+        else:
+            v = self.ctx.eakv_request_begin(request_id, 0, n, self.block_keys(tokens, agent), agent, now_ms,
+                                            decided=decided)
         if v is None:
             return None
         keys, blocks = v["keys"], v["gpu_block"]
-        if self.incremental:
+        if self.incremental and self.data_plane:
             prev = self._agent_keys.get(agent)
             if prev is None or len(keys) >= len(prev):
                 self._agent_keys[agent] = keys

@@ -61,7 +61,7 @@ def plan(cfg, trace, shape, host_gib=None, data_plane=True, ram_fraction=0.6):
 
 def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=True,
         incremental_hash=True, device="cuda:0", link_strategy=eakv.LINK_STAGED, agents=None,
-        turns=None, server_hook=None, chunk_blocks=1, kappa=None, native_turn=False,
+        turns=None, server_hook=None, chunk_blocks=1, kappa=None, native_turn=True,
         gpu_free_order=eakv.FREE_ASCENDING, write_behind=False):
     import torch
     from eakv_workloads import CONFIGS, SHAPES, key_words_torch, make_trace
@@ -78,7 +78,7 @@ def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=Tru
                          incremental_hash=incremental_hash, policy=POLICIES[policy],
                          kappa_blocks=max(1, cfg.kappa_blocks // chunk_blocks) if kappa is None else kappa,
                          link_strategy=link_strategy, chunk_blocks=chunk_blocks,
-                         native_turn=native_turn and data_plane, gpu_free_order=gpu_free_order,
+                         native_turn=native_turn, gpu_free_order=gpu_free_order,
                          write_behind=write_behind)
     t_setup = time.perf_counter() - t0
     t0 = time.perf_counter()
@@ -89,6 +89,9 @@ def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=Tru
     if server_hook is not None:
         server_hook(server, trace)
     st = server.ctx.eakv_get_stats()
+    if server.hash_ctx is not server.ctx:            # bookkeeping-only run: the hashing context counts the hashing
+        hs = server.hash_ctx.eakv_get_stats()
+        st["tokens_hashed"], st["kernel_launches"] = hs["tokens_hashed"], hs["kernel_launches"]
     tot = server.totals
     n_req = len(server.records)
     out = {
@@ -97,7 +100,7 @@ def run(config, *, policy="write_all", host_gib=None, limit=None, data_plane=Tru
         "gpu_free_order": "reverse" if gpu_free_order == eakv.FREE_REVERSE else "ascending",
         "write_behind": bool(write_behind),
         "host_gib": kh * chunk_blocks * shape.block_bytes / GIB,
-        "host_sizing": why, "data_plane": data_plane, "native_turn": bool(native_turn and data_plane),
+        "host_sizing": why, "data_plane": data_plane, "native_turn": bool(native_turn),
         "working_set_blocks_eq5": working_set_blocks(trace, shape),
         "prompt_tokens": tot["prompt_tokens"], "computed_prefill_tokens": tot["fresh_tokens"],
         "gpu_hit_tokens": tot["gpu_hit_blocks"] * shape.block_size,
@@ -128,10 +131,10 @@ def main():
     ap.add_argument("--chunk-blocks", type=int, default=1,
                     help="host-tier chunk in GPU blocks (64 = the paper's 1,024-token chunks at block 16)")
     ap.add_argument("--kappa", type=int, default=None, help="write threshold in tier units")
-    ap.add_argument("--native-turn", action="store_true",
-                    help="drive turns through eakv_turn_begin / eakv_turn_end")
+    ap.add_argument("--single-calls", dest="native_turn", action="store_false",
+                    help="drive the single calls one by one instead of eakv_turn_begin / eakv_turn_end")
     ap.add_argument("--write-behind", action="store_true",
-                    help="with --native-turn: host writes are deferred to a stream of the context")
+                    help="host writes are deferred to a stream of the context (turn engine only)")
     ap.add_argument("--reverse-free", action="store_true",
                     help="GPU tier keeps a request's blocks tail-first in its recency order")
     args = ap.parse_args()

@@ -44,7 +44,7 @@ def eq5_blocks(trace, shape):
     return int(ws // (shape.block_size * beta))
 
 
-def run_both(cfg_name, *, policy, host_blocks, limit=None, data_plane=False, link=1, chunk_blocks=1):
+def run_both(cfg_name, *, policy, host_blocks, limit=None, data_plane=False, link=1, chunk_blocks=1, native=False):
     from paper_2609_33762_b200.harness import AgentServer
     cfg = CONFIGS[cfg_name]
     shape = SHAPES[cfg.shape]
@@ -55,7 +55,7 @@ def run_both(cfg_name, *, policy, host_blocks, limit=None, data_plane=False, lin
     oracle = TraceOracle(shape, cfg.gpu_blocks, host_blocks, **kw)
     oracle.run(trace, limit=limit)
     payload = (lambda keys, q, n: key_words_torch(keys.astype(np.int64), q, n, "cuda")) if data_plane else None
-    server = AgentServer(shape, cfg.gpu_blocks, host_blocks, payload, data_plane=data_plane, native_turn=False,
+    server = AgentServer(shape, cfg.gpu_blocks, host_blocks, payload, data_plane=data_plane, native_turn=native,
                          incremental_hash=True, link_strategy=link, **kw)
     server.run(trace, limit=limit)
     compare_records_fast(server.records, oracle.records)
@@ -103,7 +103,9 @@ def test_config3_policies_control_plane(policy, limit):
     """Fixed 32 GiB tier: conditioned admission on the full trace; write-all and the fixed
     filter (which declines every request of this trace) on a prefix."""
     cfg = CONFIGS["c3"]
-    server, oracle, *_ = run_both("c3", policy=policy, host_blocks=cfg.host_blocks, limit=limit)
+    # the conditioned run goes through the library's turn engine (bookkeeping-only context fed with the
+    # GPU's keys), the other two through the single calls
+    server, oracle, *_ = run_both("c3", policy=policy, host_blocks=cfg.host_blocks, limit=limit, native=policy == 2)
     st = oracle.host.stats
     if policy == 2:
         assert 0 < st["declined_requests"] < st["requests"] and st["pressure_requests"] > 0
