@@ -122,6 +122,14 @@ class AgentServer:
                 server._timed[kind].append((nbytes, self_t.e0, self_t.e1))
         return _T()
 
+    def _timed_since(self, e0, kind, nbytes):
+        """Close a timing bracket opened with event ``e0`` on the server's stream (turn engine: the
+        restore is enqueued inside eakv_turn_begin, the store inside eakv_turn_end)."""
+        if nbytes > 0:
+            e1 = torch.cuda.Event(enable_timing=True)
+            e1.record(self.stream)
+            self._timed[kind].append((nbytes, e0, e1))
+
     def transfer_rates(self):
         """GB/s of the store and load calls so far (device time between the events that
         bracket each call); call after a synchronize."""
@@ -174,14 +182,22 @@ class AgentServer:
             self._ensure_pinned(max(n, 1))
             self._tok_pin.numpy()[:n] = tokens
             known = self._agent_keys.get(agent) if self.incremental else None
+            e0 = torch.cuda.Event(enable_timing=True)
+            e0.record(self.stream)
             v = self.ctx.eakv_turn_begin(self._tok_pin.data_ptr(), n, known, agent, now_ms, self.stream)
+            self._timed_since(e0, "load", (v["restore_hi"] - v["restore_lo"]) * self.ctx.block_bytes)
         else:       # bookkeeping only: the hashing context supplies every key
             v = self.ctx.eakv_turn_begin(0, n, self.block_keys(tokens, agent), agent, now_ms)
         keys, blocks = v["keys"], v["gpu_block"]
         if self.incremental and self.data_plane:
             self._agent_keys[agent] = keys
         self._fill(keys, blocks, np.nonzero(v["needs_fill"])[0])
+        if self.data_plane:
+            e0 = torch.cuda.Event(enable_timing=True)
+            e0.record(self.stream)
         self.ctx.eakv_turn_end(self.stream)
+        if self.data_plane:
+            self._timed_since(e0, "store", v["n_stored_blocks"] * self.ctx.block_bytes)
         rec = self._record_from_view(v, agent, now_ms, n)
         G, H = rec["G"], rec["H"]
         return rec, G, H
