@@ -58,7 +58,7 @@ def parse_args():
                     help="device code that moves a mapped host tier (zero-copy strategy)")
     ap.add_argument("--host-load-ctas", type=int, default=0)
     ap.add_argument("--host-store-ctas", type=int, default=0)
-    ap.add_argument("--staging-mib", type=int, default=64)
+    ap.add_argument("--staging-mib", type=int, default=256)
     ap.add_argument("--no-overlap", dest="overlap", action="store_false",
                     help="e2e arm: restores and host writes on one stream instead of two")
     ap.add_argument("--no-e2e", action="store_true")

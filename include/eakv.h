@@ -117,7 +117,7 @@ typedef struct eakv_config {
     int32_t tier_location;         /* EAKV_TIER_*                                                */
     int32_t copy_path;             /* EAKV_COPY_*                                                */
     int32_t copy_ctas;             /* CTAs of the copy kernels; 0 = auto                         */
-    int64_t staging_bytes;         /* per staging buffer (two per direction); 0 = 64 MiB         */
+    int64_t staging_bytes;         /* per staging buffer (two per direction); 0 = 256 MiB        */
     int64_t max_call_blocks;       /* entries per argument-ring slot; 0 = 16384                  */
     int64_t hash_scratch_blocks;   /* block partials the hash scratch holds; 0 = 1 << 20        */
     int64_t min_staged_run_bytes;  /* EAKV_LINK_STAGED: a call whose runs of consecutive slots
