@@ -903,6 +903,31 @@ def main():
     # the profile's per-block DRAM traffic was captured on the unsharded shape
     traffic = read_profile_traffic(kernel_name, m) if args.tp_shard == 1 else None
 
+    # The same step on one tensor-parallel rank's shape (Eq. 1: a rank of TP8 holds one KV head, so its
+    # pieces are 4 KiB instead of 16 KiB; the paper states every size per rank): device tier, a pool
+    # of its own (32,768 blocks), a few steps.  A side measurement of the single-GPU line only.
+    tp8 = None
+    if args.tp_shard == 1 and not args.quick and rank == 0 and dist is None:
+        def tp8_section():
+            sh8 = shape.tp_shard(8)
+            nb8 = max(2 * m, min(32768, nb))
+            pool8 = PagedPool(sh8, nb8, device, fill=lambda q, t: t.random_(), contiguous=True)
+            perm8 = np.random.default_rng(5).permutation(nb8).astype(np.int32)
+            w8 = nb8 // (2 * m)
+            tables8 = [perm8[(i % w8) * 2 * m:(i % w8 + 1) * 2 * m] for i in range(total_steps + 1)]
+            a8 = Arm(args, pool8, sh8, torch, eakv, host_tier=False, device=device)
+            r8 = run_arm(a8, prompts_dev, tables8, max(2, min(args.steps, 10)), min(args.warmup, 3), None, None)
+            a8.ctx.close()
+            rate = kernel_rate(r8)
+            return {"kv_heads": sh8.kv_heads, "piece_bytes": sh8.piece_bytes, "block_bytes": sh8.block_bytes,
+                    "pool_blocks": nb8, "achieved": rate, "frac": rate / peak, "unit": "GB/s read+write",
+                    "value_gbps": r8["moved"] / (r8["ms"] * 1e-3) / 1e9, "launches_timed": len(r8["kernel"])}
+        try:
+            tp8 = tp8_section()
+        except Exception as exc:  # noqa: BLE001
+            tp8 = {"error": f"{type(exc).__name__}: {exc}"}
+        torch.cuda.empty_cache()
+
     # ---- end-to-end arm (pinned host tier, host tokens) ----
     def e2e_section():
         link = pinned_link_peak(torch, device) if rank == 0 else None
@@ -1011,6 +1036,7 @@ def main():
                          "kernel": kernel_name,
                          "launches_timed": len(r["kernel"]),
                          "by_copy_path": by_copy_path,
+                         "tp8_rank_shape": tp8,
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "cpu_baseline": cpu,
             "hash": hashing,

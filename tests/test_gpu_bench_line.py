@@ -39,6 +39,7 @@ def test_bench_line_on_a_small_case():
     assert set(e["by_strategy"]) == {"staged", "zero_copy", "copy_engine"}
     assert all(v["value"] > 0 for v in e["by_strategy"].values())
     assert set(r["by_copy_path"]) == {"bulk", "vector"} and all(v["achieved"] > 0 for v in r["by_copy_path"].values())
+    assert r["tp8_rank_shape"]["piece_bytes"] == 4096 and r["tp8_rank_shape"]["achieved"] > 0
     rows = e["curve"]["rows"]
     assert {(x["tier"], x["op"], x["ids"], x["mask"]) for x in rows} >= {
         ("host", "store", "random", "bernoulli"), ("host", "load", "contiguous", "ones"), ("hbm", "store", "random", "ones")}
