@@ -410,6 +410,14 @@ int eakv_turn_abort(eakv_ctx* ctx);
  * see eakv_tier_step_again).  *view's arrays stay valid until the request is released.
  * eakv_request_store: after the engine has produced the blocks flagged needs_fill, eakv_store of
  * the admitted blocks on cuda_stream (deferred under eakv_config.write_behind); once per begin.
+ * Between a request's begin and its store the units it admitted are listed in the host tier (no
+ * other request stores them again) but do not count toward another request's host prefix: their
+ * slots hold nothing yet, so that request computes those blocks itself.  After the store they are
+ * restorable; a restore by another request must be ordered after that store on the GPU (same
+ * stream, or an event), as for any store followed by a load of the same slots.  The GPU side has
+ * no such guard: a block that an open request was told to fill counts as resident for a later
+ * request with the same prefix (the two share it), so an engine that runs both must let the
+ * second one read that block only after the first one's fill (stream order or an event).
  * eakv_request_release: the request finished or is suspended: its blocks become evictable
  * (eakv_gpu_tier_release_request) and its tail block is freed.  Released before its store -- the
  * engine never produced the KV -- it is taken back like an aborted turn.

@@ -10,6 +10,7 @@
 #include <new>
 #include <string>
 #include <unordered_map>
+#include <unordered_set>
 #include <vector>
 
 #include "control_plane.h"
@@ -124,6 +125,9 @@ struct eakv_ctx {
     int64_t turn_keys_cap = 0;
     TurnState turn;                            // the one open turn of eakv_turn_begin / eakv_turn_end
     std::unordered_map<int64_t, TurnState> requests;   // open turns of running requests (eakv_request_*)
+    // tier units an open turn admitted whose store has not been enqueued yet: listed in the host
+    // index (so nobody stores them twice) but not restorable by another request
+    std::unordered_set<uint64_t> unstored_units;
 
     std::string cuda_err;
 };
@@ -1196,7 +1200,15 @@ namespace {
 // those the engine was to fill (the restored ones hold their bytes).  A block another running
 // request shares stays.  Promotions and evictions the turn caused stand.  Lets the turn's GPU
 // blocks go (pins, tail block).
+void forget_unstored(eakv_ctx* ctx, const TurnState& T) {
+    if (ctx->unstored_units.empty()) return;
+    const uint64_t* ukeys = T.unit_keys.empty() ? T.keys.data() : T.unit_keys.data();
+    for (size_t c = 0; c < T.admit_u.size(); ++c)
+        if (T.admit_u[c]) ctx->unstored_units.erase(ukeys[c]);
+}
+
 void withdraw_turn(eakv_ctx* ctx, TurnState& T, bool host_units, int gpu_mode) {
+    forget_unstored(ctx, T);
     if (host_units) {
         int64_t n = 0;
         const uint64_t* ukeys = T.unit_keys.empty() ? T.keys.data() : T.unit_keys.data();
@@ -1299,6 +1311,10 @@ int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32
     if (rc != EAKV_OK) return rc;
     rc = eakv_match(ctx, ukeys, nu, &G_unused, &Hu, nullptr, T.host_slots.data());
     if (rc != EAKV_OK) return rc;
+    // a unit that another open request admitted but has not stored yet cannot be restored
+    if (!ctx->unstored_units.empty())
+        for (int64_t c = 0; c < Hu; ++c)
+            if (ctx->unstored_units.count(ukeys[c])) { Hu = c; break; }
     int32_t tail = -1;
     if (as_request)
         rc = eakv_gpu_tier_acquire(ctx, request_id, keys, nblk, need_tail, T.resident.data(), T.block.data(), &tail);
@@ -1359,6 +1375,9 @@ int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32
             ++n_store;
         }
     }
+    if (as_request)
+        for (int64_t c = 0; c < nu; ++c)
+            if (T.admit_u[c]) ctx->unstored_units.insert(ukeys[c]);
     view->n_blocks = nblk; view->n_units = nu;
     view->gpu_prefix_blocks = G; view->host_prefix_blocks = H;
     view->restore_lo = lo; view->restore_hi = hi;
@@ -1380,6 +1399,7 @@ int turn_store_impl(eakv_ctx* ctx, TurnState& T, void* cuda_stream) {
     bool any_store = false;
     for (int64_t j = 0; j < nblk && !any_store; ++j) any_store = T.admit_b[j] != 0;
     T.stored = true;
+    forget_unstored(ctx, T);                                 // from here on a stream-ordered restore finds the bytes
     if (ctx->device < 0 || !any_store) return EAKV_OK;       // bookkeeping only, or nothing admitted
     if (!ctx->cfg.write_behind)
         return eakv_store(ctx, T.block.data(), T.admit_b.data(), T.slot_b.data(), nblk, cuda_stream);

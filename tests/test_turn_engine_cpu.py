@@ -181,3 +181,35 @@ def test_requests_overlap_and_an_unstored_release_takes_its_turn_back(eakv):
     ctx.eakv_request_release(3)
     assert ctx.eakv_match(big)[:2] == (12, 12)
     ctx.close()
+
+
+def test_units_admitted_by_an_open_request_are_not_restorable_until_it_stored(eakv):
+    """Request 1 admits the units of a prompt; before it has stored them request 2 arrives with the
+    same prompt (another GPU tier state is simulated by a tiny GPU tier that request 1 does not
+    share: different keys cannot be used, so request 2 simply repeats the prompt).  Its lookup
+    must not count the unwritten slots as host coverage, and must not store them a second time."""
+    b = 4
+    ctx = cp_ctx(eakv, b, 32, 32)
+    keys = np.arange(1, 7, dtype=np.uint64)
+    v1 = ctx.eakv_request_begin(1, 0, 6 * b, keys, 0, 0)
+    assert v1["admit"].tolist() == [1] * 6 and v1["host_prefix_blocks"] == 0
+    v2 = ctx.eakv_request_begin(2, 0, 6 * b, keys, 1, 1)
+    assert v2["hit"].tolist() == [1] * 6 and v2["admit"].tolist() == [0] * 6      # listed: no second store
+    assert v2["host_prefix_blocks"] == 0                                           # but nothing to restore yet
+    assert v2["gpu_prefix_blocks"] == 6 and v2["restore_hi"] == v2["restore_lo"]   # (the GPU blocks are shared)
+    ctx.eakv_request_store(1)
+    ctx.eakv_request_store(2)
+    v3 = ctx.eakv_request_begin(3, 0, 6 * b, keys, 2, 2)
+    assert v3["host_prefix_blocks"] == 6                                           # stored: restorable now
+    for rid in (1, 2, 3):
+        ctx.eakv_request_release(rid)
+    # a request released before its store leaves nothing pending behind
+    other = np.arange(50, 53, dtype=np.uint64)
+    ctx.eakv_request_begin(4, 0, 3 * b, other, 0, 3)
+    ctx.eakv_request_release(4)
+    v5 = ctx.eakv_request_begin(5, 0, 3 * b, other, 0, 4)
+    assert v5["admit"].tolist() == [1, 1, 1]
+    ctx.eakv_request_store(5)
+    ctx.eakv_request_release(5)
+    assert ctx.eakv_match(other)[:2] == (3, 3)
+    ctx.close()
