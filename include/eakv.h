@@ -76,9 +76,10 @@ extern "C" {
 
 /* which device code moves the bytes */
 #define EAKV_COPY_VECTOR 0      /* 16-byte vector loads/stores, coalesced                       */
-#define EAKV_COPY_BULK   1      /* 1-D bulk async copies through a shared-memory ring (default);
-                                   used for device-resident buffers only: a mapped host tier
-                                   under EAKV_LINK_ZERO_COPY is always moved by the vector kernel */
+#define EAKV_COPY_BULK   1      /* 1-D bulk async copies through a shared-memory ring (default).
+                                   copy_path selects the code for device-resident buffers (an
+                                   HBM tier, the staging buffers); what moves a mapped host tier
+                                   is selected by host_copy_path below                            */
 
 /* which device code moves the bytes of a mapped host tier (EAKV_LINK_ZERO_COPY, and the scattered
  * calls that EAKV_LINK_STAGED sends directly) */
@@ -116,7 +117,8 @@ typedef struct eakv_config {
     int32_t link_strategy;         /* EAKV_LINK_*                                                */
     int32_t tier_location;         /* EAKV_TIER_*                                                */
     int32_t copy_path;             /* EAKV_COPY_*                                                */
-    int32_t copy_ctas;             /* CTAs of the copy kernels; 0 = auto                         */
+    int32_t copy_ctas;             /* CTAs of the copy kernels; 0 = auto (device buffers: the SM count
+                                      times the kernel's resident CTAs; host tier: see host_*_ctas) */
     int64_t staging_bytes;         /* per staging buffer (two per direction); 0 = 256 MiB        */
     int64_t max_call_blocks;       /* entries per argument-ring slot; 0 = 16384                  */
     int64_t hash_scratch_blocks;   /* block partials the hash scratch holds; 0 = 1 << 20        */
