@@ -472,6 +472,16 @@ int eakv_capacity_curve(const int64_t* dist_dev, int64_t n_refs, const int64_t* 
                         int32_t n_capacities, int64_t* hits_out, int64_t* restored_out,
                         int64_t* computed_out, int64_t* cover_out, void* cuda_stream);
 
+/* Working-set sizes read off the reuse distances (Section 3.2, Section 5.4: where more host
+ * capacity stops paying).  *full_out = largest finite distance + 1, the smallest tier (in tier
+ * units) that hits every re-reference; *within_out = the smallest tier whose predicted computed
+ * prefill (as eakv_capacity_curve computes it) is within `percent` per cent of the unbounded tier's.
+ * Arguments as eakv_capacity_curve; context-free; returns after the work is done. */
+int eakv_working_set_sizes(const int64_t* dist_dev, int64_t n_refs, const int64_t* req_offsets_host,
+                           const int64_t* req_tokens_host, const int64_t* req_gpu_prefix_host,
+                           int64_t n_requests, int32_t block_size, int32_t percent,
+                           int64_t* full_out, int64_t* within_out, void* cuda_stream);
+
 /* Declined-chunk audit (Appendix D, "Reuse distance of declined chunks"; Proposition 1): of the
  * references whose miss an admission policy declined, how many could be declined at no cost --
  * their chunk is referenced next at reuse distance D >= capacity, or never again.

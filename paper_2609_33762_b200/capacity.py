@@ -75,27 +75,10 @@ def gpu_prefixes(trace, shape, gpu_blocks, stream_host, offsets, gpu_free_order=
     return G
 
 
-def working_set_within(dist_ptr, n_refs, offsets, tokens, G, block_size, ws_full, percent=1):
+def working_set_within(dist_ptr, n_refs, offsets, tokens, G, block_size, ws_full=None, percent=1):
     """Smallest tier (in blocks) whose predicted computed prefill is within ``percent`` % of the
-    unbounded tier's: 64 capacities per curve launch, narrowed until the bracket is one block wide
-    (computed prefill never grows with capacity, so the condition is monotone)."""
-    floor_tokens = int(eakv.eakv_capacity_curve(dist_ptr, n_refs, offsets, tokens, G, block_size,
-                                                [max(ws_full, 1)])["computed_tokens"][0])
-    ok = lambda c: int(c) * 100 <= floor_tokens * (100 + percent)
-    lo, hi = -1, max(ws_full, 0)            # lo fails (or is below 0), hi passes
-    while hi - lo > 1:
-        span = hi - lo
-        cand = sorted({lo + max(1, (span * i) // 65) for i in range(1, 65) if lo + max(1, (span * i) // 65) < hi})
-        if not cand:
-            break
-        out = eakv.eakv_capacity_curve(dist_ptr, n_refs, offsets, tokens, G, block_size, [max(c, 0) for c in cand])
-        passed = [c for c, v in zip(cand, out["computed_tokens"]) if ok(v)]
-        failed = [c for c, v in zip(cand, out["computed_tokens"]) if not ok(v)]
-        if passed:
-            hi = min(passed)
-        if failed:
-            lo = max([c for c in failed if c < hi] or [lo])
-    return hi
+    unbounded tier's (eakv_working_set_sizes: the search runs in the library)."""
+    return eakv.eakv_working_set_sizes(dist_ptr, n_refs, offsets, tokens, G, block_size, percent)[1]
 
 
 def model(config, host_gib, device="cuda:0", limit=None, agents=None, shared_prefix=0,
@@ -125,9 +108,7 @@ def model(config, host_gib, device="cuda:0", limit=None, agents=None, shared_pre
     t0 = time.perf_counter()
     out = eakv.eakv_capacity_curve(dist.data_ptr(), n_refs, offsets, tokens, G, shape.block_size, caps)
     t_curve = time.perf_counter() - t0
-    finite = dist[:n_refs][dist[:n_refs] >= 0]
-    ws_full = int(finite.max().item()) + 1 if finite.numel() else 0
-    ws_99 = working_set_within(dist.data_ptr(), n_refs, offsets, tokens, G, shape.block_size, ws_full)
+    ws_full, ws_99 = eakv.eakv_working_set_sizes(dist.data_ptr(), n_refs, offsets, tokens, G, shape.block_size, 1)
     # Eq. 5 and the pressure ratios of Section 3.2, integer arithmetic in the library
     sizing = eakv.eakv_working_set(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
                                    elem_bytes=shape.elem_bytes, block_size=shape.block_size,

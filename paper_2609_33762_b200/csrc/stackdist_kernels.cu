@@ -332,6 +332,15 @@ __global__ void reuse_distance_kernel(const int32_t* __restrict__ prev, int64_t 
     dist[i] = count - ((int64_t)p + 1);
 }
 
+// largest finite reuse distance of the stream (-1 if every reference is a first reference)
+__global__ void max_distance_kernel(const int64_t* __restrict__ dist, int64_t n, long long* __restrict__ out) {
+    long long m = -1;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        m = max(m, (long long)dist[i]);
+    for (int d = 16; d; d >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, d));
+    if ((threadIdx.x & 31) == 0 && m >= 0) atomicMax(out, m);
+}
+
 // ---- capacity curve ---------------------------------------------------------------------------
 // hits[c] += #{ i : 0 <= D_i < K_c }
 __global__ void curve_hits_kernel(const int64_t* __restrict__ dist, int64_t n,
@@ -610,4 +619,73 @@ done:
     cudaFree(d_off); cudaFree(d_tok); cudaFree(d_gpu); cudaFree(d_caps); cudaFree(d_out); cudaFree(d_cover);
     if (rc != EAKV_OK) cudaGetLastError();
     return rc;
+}
+
+// Working-set sizes read off the distances (Section 3.2: the capacity at which more host memory
+// stops paying).  full = largest finite reuse distance + 1, the smallest tier that hits every
+// re-reference.  within = the smallest tier whose predicted computed prefill is within `percent`
+// per cent of the unbounded tier's: computed prefill never grows with capacity, so the condition is
+// monotone and the bracket (fails, passes] is narrowed with 64 capacities per curve launch.
+extern "C" int eakv_working_set_sizes(const int64_t* dist_dev, int64_t n_refs, const int64_t* req_offsets_host,
+                                      const int64_t* req_tokens_host, const int64_t* req_gpu_prefix_host,
+                                      int64_t n_requests, int32_t block_size, int32_t percent,
+                                      int64_t* full_out, int64_t* within_out, void* cuda_stream) {
+    if (n_refs < 0 || n_requests < 0 || block_size <= 0 || percent < 0 || !full_out || !within_out)
+        return EAKV_E_INVAL;
+    if (n_refs > 0 && !dist_dev) return EAKV_E_INVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int rc = EAKV_OK;
+    long long* d_max = nullptr;
+    long long h_max = -1;
+    int dev = 0, sms = 148;
+    SD_CU(cudaMalloc(&d_max, 8));
+    SD_CU(cudaMemcpyAsync(d_max, &h_max, 8, cudaMemcpyHostToDevice, stream));
+    if (n_refs > 0) {
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        max_distance_kernel<<<(int)std::min<int64_t>((n_refs + 255) / 256, (int64_t)sms * 8), 256, 0, stream>>>(
+            dist_dev, n_refs, d_max);
+        SD_CU(cudaGetLastError());
+    }
+    SD_CU(cudaMemcpyAsync(&h_max, d_max, 8, cudaMemcpyDeviceToHost, stream));
+    SD_CU(cudaStreamSynchronize(stream));
+done:
+    cudaFree(d_max);
+    if (rc != EAKV_OK) {
+        cudaGetLastError();
+        return rc;
+    }
+    const int64_t full = h_max + 1;
+    *full_out = full;
+    auto computed_at = [&](const std::vector<int64_t>& caps, std::vector<int64_t>& out) -> int {
+        std::vector<int64_t> hits(caps.size()), restored(caps.size());
+        out.resize(caps.size());
+        return eakv_capacity_curve(dist_dev, n_refs, req_offsets_host, req_tokens_host, req_gpu_prefix_host,
+                                   n_requests, block_size, caps.data(), (int32_t)caps.size(), hits.data(),
+                                   restored.data(), out.data(), nullptr, cuda_stream);
+    };
+    std::vector<int64_t> caps{std::max<int64_t>(full, 1)}, computed;
+    rc = computed_at(caps, computed);
+    if (rc != EAKV_OK) return rc;
+    const __int128 floor_tokens = computed[0];
+    auto passes = [&](int64_t c) { return (__int128)c * 100 <= floor_tokens * (100 + percent); };
+    int64_t lo = -1, hi = std::max<int64_t>(full, 0);              // lo fails (or is below 0), hi passes
+    while (hi - lo > 1) {
+        const int64_t span = hi - lo;
+        caps.clear();
+        for (int i = 1; i <= 64; ++i) {
+            const int64_t c = lo + std::max<int64_t>(1, (int64_t)((__int128)span * i / 65));
+            if (c < hi && (caps.empty() || c > caps.back())) caps.push_back(c);
+        }
+        if (caps.empty()) break;
+        std::vector<int64_t> query(caps);
+        for (int64_t& c : query) c = std::max<int64_t>(c, 0);
+        rc = computed_at(query, computed);
+        if (rc != EAKV_OK) return rc;
+        for (size_t i = 0; i < caps.size(); ++i) {
+            if (passes(computed[i])) { hi = caps[i]; break; }      // the first that passes bounds from above
+            lo = caps[i];                                          // everything before it fails
+        }
+    }
+    *within_out = hi;
+    return EAKV_OK;
 }

@@ -111,7 +111,7 @@ EXPORTS = [
     "eakv_selfcheck_limits", "eakv_selfcheck_wait_probe",
     "eakv_gpu_tier_acquire", "eakv_gpu_tier_release_request", "eakv_tier_step_again",
     "eakv_declined_audit", "eakv_working_set",
-    "eakv_request_begin", "eakv_request_store", "eakv_request_release",
+    "eakv_request_begin", "eakv_request_store", "eakv_request_release", "eakv_working_set_sizes",
 ]
 STATIC_MAX_BLOCKS = 65536
 
@@ -149,6 +149,7 @@ def lib():
     L.eakv_reuse_distances.argtypes = [vp, i64, vp, vp]
     L.eakv_capacity_curve.argtypes = [vp, i64, vp, vp, vp, i64, i32, vp, i32, vp, vp, vp, vp, vp]
     L.eakv_declined_audit.argtypes = [vp, vp, i64, i64, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), vp, vp]
+    L.eakv_working_set_sizes.argtypes = [vp, i64, vp, vp, vp, i64, i32, i32, C.POINTER(i64), C.POINTER(i64), vp]
     L.eakv_working_set.argtypes = [C.POINTER(WorkingSetIn), C.POINTER(WorkingSetOut)]
     L.eakv_turn_begin.argtypes = [vp, vp, i64, vp, i64, i64, i64, vp, C.POINTER(TurnView)]
     L.eakv_turn_end.argtypes = [vp, vp]
@@ -228,6 +229,22 @@ def eakv_declined_audit(keys_dev, declined_dev, n_refs, capacity, next_dist_dev=
     if rc != OK:
         raise EakvError(rc, "eakv_declined_audit")
     return d.value, m.value, nv.value
+
+
+def eakv_working_set_sizes(dist_dev, n_refs, req_offsets, req_tokens, req_gpu_prefix, block_size, percent=1,
+                           stream=None):
+    """(full, within): smallest tier that hits every re-reference, and smallest tier whose predicted
+    computed prefill is within ``percent`` % of the unbounded tier's."""
+    off, offp = _np(req_offsets, np.int64)
+    tok, tokp = _np(req_tokens, np.int64)
+    gpu, gpup = _np(req_gpu_prefix, np.int64)
+    full, within = C.c_int64(0), C.c_int64(0)
+    rc = lib().eakv_working_set_sizes(C.c_void_p(int(dist_dev)), int(n_refs), offp, tokp, gpup, len(off) - 1,
+                                      int(block_size), int(percent), C.byref(full), C.byref(within),
+                                      _stream(stream))
+    if rc != OK:
+        raise EakvError(rc, "eakv_working_set_sizes")
+    return full.value, within.value
 
 
 def eakv_working_set(*, num_layers, kv_heads, head_dim, block_size, active_pool, total_prompt_tokens,

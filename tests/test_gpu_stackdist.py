@@ -87,12 +87,12 @@ def test_capacity_curve_on_config0():
     assert np.all(np.diff(out["hits"]) >= 0)             # hits are monotone in capacity
     # smallest tier within 1 % (and 10 %) of the unbounded tier's computed prefill: GPU narrowing
     # against the oracle's plain scan over every capacity
-    from paper_2609_33762_b200 import capacity
     ws_full = sd.working_set_full(sd.reuse_distances(stream))
-    for pct in (1, 10):
-        got = capacity.working_set_within(dist_dev.data_ptr(), len(stream), offsets, n_tok, G,
-                                          shape.block_size, ws_full, percent=pct)
-        assert got == sd.working_set_within(req_keys, n_tok, G, shape.block_size, percent=pct)
+    for pct in (0, 1, 10):
+        full, within = eakv.eakv_working_set_sizes(dist_dev.data_ptr(), len(stream), offsets, n_tok, G,
+                                                   shape.block_size, pct)
+        assert full == ws_full
+        assert within == sd.working_set_within(req_keys, n_tok, G, shape.block_size, percent=pct)
 
 
 def test_config3_prefix_distances_and_product_tier_agree():
