@@ -105,7 +105,7 @@ cudaError_t launch_copy_vector(const CopyLaunch& L, bool to_tier, int ctas, cuda
 // ---------------------------------------------------------------------------------------
 // Bulk path: one thread per CTA drives a ring of shared-memory stages with 1-D bulk async
 // copies (global -> shared completing on an mbarrier, shared -> global in bulk groups).
-// No multicast, no tensor maps; every address and size is a multiple of 16 bytes.
+// Plain per-CTA bulk copies, no tensor maps; every address and size is a multiple of 16 bytes.
 // Every wait is bounded: on giving up the thread raises *error_flag, drains what it has
 // in flight (bounded again) and returns.
 // ---------------------------------------------------------------------------------------
