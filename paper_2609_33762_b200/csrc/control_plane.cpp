@@ -2,57 +2,51 @@
 
 namespace eakv {
 
-static inline uint64_t mix64(uint64_t x) {
-    x ^= x >> 31;
-    x *= 0x7fb5d329728ea185ull;
-    x ^= x >> 27;
-    x *= 0x81dadef4bc2dd44dull;
-    x ^= x >> 33;
-    return x;
-}
-
 KeyedLru::KeyedLru(int64_t capacity)
-    : cap_(capacity), resident_(0), key_(capacity), prev_(capacity, -1), next_(capacity, -1),
+    : cap_(capacity), resident_(0), node_(capacity, Node{0, -1, -1}),
       state_(capacity, 0), pin_count_(capacity, 0), lru_(-1), mru_(-1) {
     free_.reserve(capacity);
     for (int64_t s = capacity - 1; s >= 0; --s) free_.push_back((int32_t)s);
     size_t n = 16;
     while (n < (size_t)capacity * 2 + 2) n <<= 1;
-    table_.assign(n, 0);
+    table_.assign(n, Entry{0, 0});
     mask_ = n - 1;
 }
 
-size_t KeyedLru::home(uint64_t key) const { return (size_t)mix64(key) & mask_; }
-
 int32_t KeyedLru::find(uint64_t key) const {
-    size_t i = home(key);
+    const uint64_t h = hash(key);
+    const uint32_t tag = (uint32_t)h;
+    size_t i = (size_t)h & mask_;
     while (true) {
-        int32_t v = table_[i];
-        if (v == 0) return -1;
-        if (key_[v - 1] == key) return v - 1;
+        const Entry e = table_[i];
+        if (e.v == 0) return -1;
+        if (e.tag == tag && node_[e.v - 1].key == key) return e.v - 1;
         i = (i + 1) & mask_;
     }
 }
 
 void KeyedLru::table_put(uint64_t key, int32_t slot) {
-    size_t i = home(key);
-    while (table_[i] != 0) i = (i + 1) & mask_;
-    table_[i] = slot + 1;
+    const uint64_t h = hash(key);
+    size_t i = (size_t)h & mask_;
+    while (table_[i].v != 0) i = (i + 1) & mask_;
+    table_[i] = Entry{(uint32_t)h, slot + 1};
 }
 
 // linear probing with backward-shift deletion
 void KeyedLru::table_erase(uint64_t key) {
-    size_t i = home(key);
+    const uint64_t hk = hash(key);
+    const uint32_t tag = (uint32_t)hk;
+    size_t i = (size_t)hk & mask_;
     while (true) {
-        int32_t v = table_[i];
-        if (v == 0) return;
-        if (key_[v - 1] == key) break;
+        const Entry e = table_[i];
+        if (e.v == 0) return;
+        if (e.tag == tag && node_[e.v - 1].key == key) break;
         i = (i + 1) & mask_;
     }
     size_t hole = i;
     size_t j = (i + 1) & mask_;
-    while (table_[j] != 0) {
-        size_t h = home(key_[table_[j] - 1]);
+    while (table_[j].v != 0) {
+        const size_t h = (size_t)table_[j].tag & mask_;
         // can the entry at j move into the hole?  yes unless its home lies cyclically in (hole, j]
         bool stays = (hole <= j) ? (h > hole && h <= j) : (h > hole || h <= j);
         if (!stays) {
@@ -61,20 +55,20 @@ void KeyedLru::table_erase(uint64_t key) {
         }
         j = (j + 1) & mask_;
     }
-    table_[hole] = 0;
+    table_[hole] = Entry{0, 0};
 }
 
 void KeyedLru::unlink(int32_t s) {
-    int32_t p = prev_[s], n = next_[s];
-    if (p >= 0) next_[p] = n; else lru_ = n;
-    if (n >= 0) prev_[n] = p; else mru_ = p;
-    prev_[s] = next_[s] = -1;
+    int32_t p = node_[s].prev, n = node_[s].next;
+    if (p >= 0) node_[p].next = n; else lru_ = n;
+    if (n >= 0) node_[n].prev = p; else mru_ = p;
+    node_[s].prev = node_[s].next = -1;
 }
 
 void KeyedLru::push_mru(int32_t s) {
-    prev_[s] = mru_;
-    next_[s] = -1;
-    if (mru_ >= 0) next_[mru_] = s; else lru_ = s;
+    node_[s].prev = mru_;
+    node_[s].next = -1;
+    if (mru_ >= 0) node_[mru_].next = s; else lru_ = s;
     mru_ = s;
 }
 
@@ -86,12 +80,18 @@ void KeyedLru::promote(int32_t s) {
 
 int32_t KeyedLru::evict_lru(uint64_t* victim_key) {
     int32_t v = lru_;
-    *victim_key = key_[v];
-    table_erase(key_[v]);
+    *victim_key = node_[v].key;
+    table_erase(node_[v].key);
     unlink(v);
     state_[v] = 0;
     --resident_;
     free_.push_back(v);
+    // the next victims are known: bring in the table line of the next one and the node of the one after
+    if (lru_ >= 0) {
+        const Node& n = node_[lru_];
+        __builtin_prefetch(&table_[(size_t)hash(n.key) & mask_], 1);
+        if (n.next >= 0) __builtin_prefetch(&node_[n.next], 1);
+    }
     return v;
 }
 
@@ -103,7 +103,7 @@ int32_t KeyedLru::insert(uint64_t key, bool* evicted, uint64_t* victim_key, int3
     }
     int32_t s = free_.back();
     free_.pop_back();
-    key_[s] = key;
+    node_[s].key = key;
     state_[s] = 1;
     table_put(key, s);
     push_mru(s);
@@ -155,9 +155,9 @@ void KeyedLru::release_unkeyed(int32_t s) {
 
 int64_t KeyedLru::export_order(uint64_t* keys, int32_t* slots, int64_t capacity) const {
     int64_t n = 0;
-    for (int32_t s = lru_; s >= 0; s = next_[s], ++n) {
+    for (int32_t s = lru_; s >= 0; s = node_[s].next, ++n) {
         if (n < capacity) {
-            if (keys) keys[n] = key_[s];
+            if (keys) keys[n] = node_[s].key;
             if (slots) slots[n] = s;
         }
     }
@@ -171,7 +171,7 @@ bool KeyedLru::import_order(const uint64_t* keys, const int32_t* slots, int64_t 
     for (; done < n; ++done) {
         const int32_t s = slots[done];
         if (s < 0 || s >= cap_ || state_[s] != 0 || find(keys[done]) >= 0) { ok = false; break; }
-        key_[s] = keys[done];
+        node_[s].key = keys[done];
         state_[s] = 1;
         table_put(keys[done], s);
         push_mru(s);
@@ -180,7 +180,7 @@ bool KeyedLru::import_order(const uint64_t* keys, const int32_t* slots, int64_t 
     if (!ok) {                     // undo: back to the empty tier
         for (int64_t i = 0; i < done; ++i) {
             const int32_t s = slots[i];
-            table_erase(key_[s]);
+            table_erase(node_[s].key);
             unlink(s);
             state_[s] = 0;
         }
@@ -208,7 +208,7 @@ void Admission::publish(int64_t now_ms, int64_t resident_now) {
     if (t < period_ms_ || t <= report_time_) return;
     // every earlier request came before t, so the tier as it stands is what that publication saw
     int64_t e = 0;
-    for (int64_t x : evict_times_) e += (x > t - window_ms_ && x < t);
+    for (const EvictRun& r : evict_runs_) e += (r.time > t - window_ms_ && r.time < t) ? r.count : 0;
     report_time_ = t;
     report_resident_ = resident_now;
     report_evicted_ = e;
@@ -223,7 +223,10 @@ bool Admission::pressure(int64_t agent, int64_t n_tokens, int64_t now_ms, int64_
         lengths_.pop_front();
     }
     const int64_t lo = now_ms - window_ms_;
-    while (!evict_times_.empty() && evict_times_.front() <= lo) evict_times_.pop_front();
+    while (!evict_runs_.empty() && evict_runs_.front().time <= lo) {
+        evict_count_ -= evict_runs_.front().count;
+        evict_runs_.pop_front();
+    }
     if (policy_ == 0) return false;
     if (policy_ == 1) return true;
     int64_t active = 0;
@@ -240,7 +243,7 @@ bool Admission::pressure(int64_t agent, int64_t n_tokens, int64_t now_ms, int64_
                report_evicted_ > 0;
     }
     const bool full = (__int128)100 * resident_now >= (__int128)theta_percent_ * host_blocks_;
-    const bool evicting = !evict_times_.empty();
+    const bool evicting = !evict_runs_.empty();
     return estimate && full && evicting;
 }
 
@@ -251,8 +254,8 @@ int64_t Admission::export_state(int64_t* out, int64_t capacity) const {
     for (const auto& kv : ordered) { v.push_back(kv.first); v.push_back(kv.second); }
     v.push_back((int64_t)lengths_.size());
     for (int64_t x : lengths_) v.push_back(x);
-    v.push_back((int64_t)evict_times_.size());
-    for (int64_t x : evict_times_) v.push_back(x);
+    v.push_back(evict_count_);
+    for (const EvictRun& r : evict_runs_) v.insert(v.end(), (size_t)r.count, r.time);
     v.push_back(report_time_);
     v.push_back(report_resident_);
     v.push_back(report_evicted_);
@@ -265,7 +268,8 @@ bool Admission::import_state(const int64_t* in, int64_t n) {
     auto take = [&](int64_t* x) { if (i >= n) return false; *x = in[i++]; return true; };
     int64_t na = 0, nl = 0, ne = 0;
     std::unordered_map<int64_t, int64_t> agents;
-    std::deque<int64_t> lengths, evs;
+    std::deque<int64_t> lengths;
+    std::deque<EvictRun> evs;
     int64_t sum = 0;
     if (!take(&na) || na < 0 || na > (n - i) / 2) return false;
     for (int64_t k = 0; k < na; ++k) {
@@ -284,7 +288,8 @@ bool Admission::import_state(const int64_t* in, int64_t n) {
     for (int64_t k = 0; k < ne; ++k) {
         int64_t x = 0;
         if (!take(&x)) return false;
-        evs.push_back(x);
+        if (!evs.empty() && evs.back().time == x) evs.back().count += 1;
+        else evs.push_back(EvictRun{x, 1});
     }
     int64_t rt = -1, rr = 0, re = 0;
     if (!take(&rt) || !take(&rr) || !take(&re) || rt < -1 || rr < 0 || re < 0) return false;
@@ -294,7 +299,8 @@ bool Admission::import_state(const int64_t* in, int64_t n) {
     agent_last_.swap(agents);
     lengths_.swap(lengths);
     length_sum_ = sum;
-    evict_times_.swap(evs);
+    evict_runs_.swap(evs);
+    evict_count_ = ne;
     return true;
 }
 

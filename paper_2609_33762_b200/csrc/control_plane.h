@@ -3,8 +3,10 @@
 // KeyedLru implements the paper's LRU reference model (Appendix D): residents in recency
 // order, hit -> most-recent end, admitted miss -> insert at the most-recent end after
 // evicting the least-recent resident when full.  Storage is flat: an open-addressing
-// table maps a 61-bit key to a slot; recency links live in arrays indexed by slot; free
-// slots come from a stack that first yields 0, 1, 2, ... and reuses an evicted slot next.
+// table maps a 61-bit key to a slot (each entry carries 32 bits of the key's hash, so a probe
+// reads the key array only on a tag match and a deletion never does); recency links live in
+// arrays indexed by slot; free slots come from a stack that first yields 0, 1, 2, ... and reuses
+// an evicted slot next.
 #pragma once
 #include <cstdint>
 #include <deque>
@@ -46,6 +48,21 @@ public:
     bool is_pinned(int32_t slot) const { return pin_count_[slot] > 0; }
     int64_t evictable() const { return resident_ - pinned_; }
     int64_t free_slots() const { return (int64_t)free_.size(); }
+    // Hints for a caller that knows its keys ahead of the walk; they change nothing.  Call them in
+    // this order a few references apart: the table line of a key; then the node of the slot its
+    // home entry names; then that node's two neighbours in the recency order.
+    void prefetch_table(uint64_t key) const { __builtin_prefetch(&table_[(size_t)hash(key) & mask_]); }
+    void prefetch_node(uint64_t key) const {
+        const Entry e = table_[(size_t)hash(key) & mask_];
+        if (e.v) __builtin_prefetch(&node_[e.v - 1], 1);
+    }
+    void prefetch_neighbours(uint64_t key) const {
+        const Entry e = table_[(size_t)hash(key) & mask_];
+        if (!e.v) return;
+        const Node& n = node_[e.v - 1];
+        if (n.prev >= 0) __builtin_prefetch(&node_[n.prev], 1);
+        if (n.next >= 0) __builtin_prefetch(&node_[n.next], 1);
+    }
     // Residents in recency order, least recent first, into keys[]/slots[] (either may be NULL);
     // returns how many there are (at most `capacity` are written).
     int64_t export_order(uint64_t* keys, int32_t* slots, int64_t capacity) const;
@@ -56,23 +73,37 @@ public:
     bool import_order(const uint64_t* keys, const int32_t* slots, int64_t n);
 
 private:
+    struct Entry {
+        uint32_t tag;                  // low 32 bits of the key's hash: the home position is tag & mask_
+        int32_t v;                     // slot + 1, 0 = empty
+    };
     void table_put(uint64_t key, int32_t slot);
     void table_erase(uint64_t key);
-    size_t home(uint64_t key) const;
+    static uint64_t hash(uint64_t x) {
+        x ^= x >> 31;
+        x *= 0x7fb5d329728ea185ull;
+        x ^= x >> 27;
+        x *= 0x81dadef4bc2dd44dull;
+        x ^= x >> 33;
+        return x;
+    }
+    struct Node {                      // by slot: key and recency links share a cache line
+        uint64_t key;
+        int32_t prev, next;            // -1 ends
+    };
     void unlink(int32_t slot);
     void push_mru(int32_t slot);
     int32_t evict_lru(uint64_t* victim_key);
 
     int64_t cap_, resident_;
-    std::vector<uint64_t> key_;        // by slot
-    std::vector<int32_t> prev_, next_; // by slot; -1 ends
+    std::vector<Node> node_;
     std::vector<uint8_t> state_;       // 0 free, 1 keyed resident, 2 unkeyed taken
     std::vector<int32_t> pin_count_;   // holders per slot
     int64_t pinned_ = 0;               // residents with at least one holder
     int32_t lru_, mru_;
     std::vector<int32_t> free_;        // stack
-    std::vector<int32_t> table_;       // slot + 1, 0 = empty
-    size_t mask_;
+    std::vector<Entry> table_;         // at most half full
+    size_t mask_;                      // table size - 1 (at most 2^32 - 1: capacities are below 2^31)
 };
 
 // Pressure signal of Eq. 10 over virtual time, all integers:
@@ -94,7 +125,11 @@ public:
     // registers the request (agent activity, prompt length), expires old evictions and
     // returns p_t; call once per request before the walk
     bool pressure(int64_t agent, int64_t n_tokens, int64_t now_ms, int64_t resident_now);
-    void note_eviction(int64_t now_ms) { evict_times_.push_back(now_ms); }
+    void note_eviction(int64_t now_ms) {
+        ++evict_count_;
+        if (!evict_runs_.empty() && evict_runs_.back().time == now_ms) evict_runs_.back().count += 1;
+        else evict_runs_.push_back(EvictRun{now_ms, 1});
+    }
     int32_t kappa() const { return kappa_; }
     // The windows as a flat list of int64: n_agents, (agent, last time) pairs in ascending agent
     // order, n_lengths, the prompt lengths oldest first, n_evictions, the eviction times oldest
@@ -112,7 +147,9 @@ private:
     std::unordered_map<int64_t, int64_t> agent_last_;
     std::deque<int64_t> lengths_;
     int64_t length_sum_;
-    std::deque<int64_t> evict_times_;
+    struct EvictRun { int64_t time, count; };     // evictions of one request share its time
+    std::deque<EvictRun> evict_runs_;             // oldest first
+    int64_t evict_count_ = 0;                     // sum of the counts
 };
 
 }  // namespace eakv

@@ -879,8 +879,22 @@ static int tier_step_impl(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_
 
     KeyedLru& T = *ctx->host_tier;
     ctx->adm->publish(now_ms, T.resident());
+    // the keys are known ahead of the walk: table line, node and the node's neighbours are asked
+    // for 12, 8 and 4 references early (hints only)
+    auto hint = [&](int64_t j) {
+        if (j + 12 < n_blocks) T.prefetch_table(hashes_host[j + 12]);
+        if (j + 8 < n_blocks) T.prefetch_node(hashes_host[j + 8]);
+        if (j + 4 < n_blocks) T.prefetch_neighbours(hashes_host[j + 4]);
+    };
+    for (int64_t j = 0; j < std::min<int64_t>(12, n_blocks); ++j) T.prefetch_table(hashes_host[j]);
+    // leading hits: their slots stay valid until the walk reaches the first miss (hits only promote)
     int64_t H = 0;
-    while (H < n_blocks && T.find(hashes_host[H]) >= 0) ++H;
+    for (; H < n_blocks; ++H) {
+        hint(H);
+        const int32_t s = T.find(hashes_host[H]);
+        if (s < 0) break;
+        slot_out[H] = s;
+    }
     const bool first = decided < 0;
     const bool p = first ? ctx->adm->pressure(agent_id, n_tokens, now_ms, T.resident()) : false;
     const int64_t cb = ctx->chunk_tokens;                 // tokens per tier unit
@@ -896,7 +910,8 @@ static int tier_step_impl(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_
     for (int64_t j = 0; j < n_blocks; ++j) {
         const uint64_t key = hashes_host[j];
         st.references += 1;
-        const int32_t s = T.find(key);
+        if (j >= H) hint(j);
+        const int32_t s = j < H ? slot_out[j] : T.find(key);
         if (s >= 0) {
             T.promote(s);
             hit_out[j] = 1; admit_out[j] = 0; slot_out[j] = s;
