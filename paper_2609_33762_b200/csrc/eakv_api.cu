@@ -849,12 +849,17 @@ int eakv_match(const eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_block
                int32_t* gpu_block_ids_out, int32_t* host_slots_out) {
     if (!ctx || n_blocks < 0 || (n_blocks > 0 && !hashes_host)) return EAKV_E_INVAL;
     int64_t G = 0, H = 0;
+    // each walk asks for the table line and the node of the keys 8 and 4 references ahead (hints only)
     for (; G < n_blocks; ++G) {
+        if (G + 8 < n_blocks) ctx->gpu_tier->prefetch_table(hashes_host[G + 8]);
+        if (G + 4 < n_blocks) ctx->gpu_tier->prefetch_node(hashes_host[G + 4]);
         const int32_t s = ctx->gpu_tier->find(hashes_host[G]);
         if (s < 0) break;
         if (gpu_block_ids_out) gpu_block_ids_out[G] = s;
     }
     for (; H < n_blocks; ++H) {
+        if (H + 8 < n_blocks) ctx->host_tier->prefetch_table(hashes_host[H + 8]);
+        if (H + 4 < n_blocks) ctx->host_tier->prefetch_node(hashes_host[H + 4]);
         const int32_t s = ctx->host_tier->find(hashes_host[H]);
         if (s < 0) break;
         if (host_slots_out) host_slots_out[H] = s;
