@@ -181,7 +181,7 @@ def lib():
 
 def _np(a, dtype):
     a = np.ascontiguousarray(a, dtype=dtype)
-    return a, a.ctypes.data_as(C.c_void_p)
+    return a, a.ctypes.data
 
 
 def _stream(s):
@@ -271,7 +271,7 @@ def eakv_capacity_curve(dist_dev, n_refs, req_offsets, req_tokens, req_gpu_prefi
     restored = np.zeros(Cn, dtype=np.int64)
     computed = np.zeros(Cn, dtype=np.int64)
     cover = np.zeros((Cn, J), dtype=np.int64) if want_cover else None
-    vp = lambda a: a.ctypes.data_as(C.c_void_p)
+    vp = lambda a: a.ctypes.data
     rc = lib().eakv_capacity_curve(C.c_void_p(int(dist_dev)), int(n_refs), offp, tokp, gpup, J,
                                    int(block_size), capsp, Cn, vp(hits), vp(restored), vp(computed),
                                    vp(cover) if want_cover else None, _stream(stream))
@@ -375,7 +375,7 @@ class Context:
         out = np.zeros(n_prompts + 1, dtype=np.int64)
         rc = lib().eakv_hash_blocks_batched(self._h, C.c_void_p(int(tokens_dev)), off_p, n_prompts,
                                             par_p, C.c_void_p(int(hashes_dev)),
-                                            out.ctypes.data_as(C.c_void_p), _stream(stream))
+                                            out.ctypes.data, _stream(stream))
         self._check(rc, "eakv_hash_blocks_batched")
         return out
 
@@ -387,7 +387,7 @@ class Context:
         gids = np.full(n, -1, dtype=np.int32)
         slots = np.full(n, -1, dtype=np.int32)
         rc = lib().eakv_match(self._h, hp, n, C.byref(G), C.byref(H),
-                              gids.ctypes.data_as(C.c_void_p), slots.ctypes.data_as(C.c_void_p))
+                              gids.ctypes.data, slots.ctypes.data)
         self._check(rc, "eakv_match")
         return G.value, H.value, gids[:G.value], slots[:H.value]
 
@@ -397,7 +397,7 @@ class Context:
         self._check(lib().eakv_tier_export(self._h, None, None, 0, C.byref(n)), "eakv_tier_export")
         keys = np.zeros(n.value, dtype=np.uint64)
         slots = np.zeros(n.value, dtype=np.int32)
-        rc = lib().eakv_tier_export(self._h, keys.ctypes.data_as(C.c_void_p), slots.ctypes.data_as(C.c_void_p),
+        rc = lib().eakv_tier_export(self._h, keys.ctypes.data, slots.ctypes.data,
                                     n.value, C.byref(n))
         self._check(rc, "eakv_tier_export")
         return keys, slots
@@ -414,7 +414,7 @@ class Context:
         n = C.c_int64(0)
         self._check(lib().eakv_admission_export(self._h, None, 0, C.byref(n)), "eakv_admission_export")
         vals = np.zeros(n.value, dtype=np.int64)
-        self._check(lib().eakv_admission_export(self._h, vals.ctypes.data_as(C.c_void_p), n.value, C.byref(n)),
+        self._check(lib().eakv_admission_export(self._h, vals.ctypes.data, n.value, C.byref(n)),
                     "eakv_admission_export")
         return vals
 
@@ -434,7 +434,7 @@ class Context:
         es = np.zeros(n, dtype=np.int32)
         nev = C.c_int64(n)
         info = StepInfo()
-        vp = lambda a: a.ctypes.data_as(C.c_void_p)
+        vp = lambda a: a.ctypes.data
         if decided is None:
             rc = lib().eakv_tier_step(self._h, hp, n, int(agent_id), int(n_tokens), int(now_ms),
                                       vp(hit), vp(admit), vp(slot), vp(ek), vp(es), C.byref(nev),
@@ -456,8 +456,8 @@ class Context:
         blk = np.zeros(n, dtype=np.int32)
         tail = C.c_int32(-1)
         rc = lib().eakv_gpu_tier_step(self._h, hp, n, int(bool(need_tail)),
-                                      res.ctypes.data_as(C.c_void_p),
-                                      blk.ctypes.data_as(C.c_void_p), C.byref(tail))
+                                      res.ctypes.data,
+                                      blk.ctypes.data, C.byref(tail))
         self._check(rc, "eakv_gpu_tier_step")
         return res, blk, tail.value
 
@@ -470,7 +470,7 @@ class Context:
         blk = np.zeros(n, dtype=np.int32)
         tail = C.c_int32(-1)
         rc = lib().eakv_gpu_tier_acquire(self._h, int(request_id), hp, n, int(bool(need_tail)),
-                                         res.ctypes.data_as(C.c_void_p), blk.ctypes.data_as(C.c_void_p),
+                                         res.ctypes.data, blk.ctypes.data,
                                          C.byref(tail))
         if rc == E_BUSY:
             return None
