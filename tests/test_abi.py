@@ -93,3 +93,23 @@ def test_no_cpu_fallback_without_a_gpu(lib):
         eakv.Context(num_layers=4, kv_heads=2, head_dim=64, block_size=16, gpu_blocks=8,
                      host_blocks=8, kv_base=ptrs)
     assert ei.value.code == eakv.E_CUDA
+
+
+def test_a_plain_c_client_compiles_and_links(tmp_path):
+    """The header is a C99 header and the library resolves every call a C client makes
+    (tests/c_client/five_calls.c; it is run on a GPU by tests/test_gpu_c_client.py)."""
+    import shutil
+    import subprocess
+    cuda = os.environ.get("CUDA_HOME", "/usr/local/cuda")
+    if shutil.which("gcc") is None or not os.path.exists(os.path.join(cuda, "include", "cuda_runtime_api.h")):
+        pytest.skip("gcc or the CUDA headers are missing")
+    here = os.path.dirname(os.path.abspath(__file__))
+    root = os.path.dirname(here)
+    pkg = os.path.join(root, "paper_2609_33762_b200")
+    exe = os.path.join(str(tmp_path), "five_calls")
+    cmd = ["gcc", "-std=c99", "-Wall", "-Werror", "-O1", os.path.join(here, "c_client", "five_calls.c"),
+           "-I" + os.path.join(root, "include"), "-I" + os.path.join(cuda, "include"),
+           "-L" + pkg, "-leakv", "-L" + os.path.join(cuda, "lib64"), "-lcudart", "-Wl,-rpath," + pkg, "-o", exe]
+    run = subprocess.run(cmd, capture_output=True, text=True)
+    assert run.returncode == 0, run.stderr
+    assert os.path.exists(exe)
