@@ -111,7 +111,7 @@ private:
 //   full      100 * resident >= theta_percent * K_H
 //   evicting  evictions in (now - window, now] > 0
 // With a report period the last two are read from the latest published report instead, if one
-// exists and is not older than the maximum age; otherwise the estimate alone decides.
+// exists and is not older than the maximum age; otherwise p_t is the working-set test by itself.
 class Admission {
 public:
     Admission(int32_t policy, int32_t kappa_blocks, int32_t theta_percent, int64_t window_ms,

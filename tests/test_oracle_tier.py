@@ -371,8 +371,8 @@ def test_published_reports_hand_case():
     for x in (t, sync):
         r = x.step([1, 2, 3, 4], 40, agent=0, now_ms=100)
         assert r.save and not r.pressure
-    # 200 ms: no report has been published yet (the first one comes at 1,000 ms): the estimate
-    # alone decides, and it says pressure.  Read synchronously, the tier is full but has not
+    # 200 ms: no report has been published yet (the first one comes at 1,000 ms): p_t is
+    # the working-set test by itself, and it says pressure.  Read synchronously, the tier is full but has not
     # evicted anything, so there is no pressure.
     r = t.step([5, 6], 40, agent=1, now_ms=200)
     assert r.pressure and not r.save and r.admit == [0, 0] and t.report is None
@@ -411,7 +411,7 @@ def test_stale_report_falls_back_to_the_estimate():
     r = t.step([4], 100, agent=1, now_ms=12_000)
     assert t.report == (10_000, 3, 0) and not r.pressure and r.save
     # 16,500 ms: the same report is 6.5 s old and no newer one exists (the next comes at 20,000 ms):
-    # not fresh, so the estimate alone decides: (2-1) * 212 > 16 * 3 -> pressure, declined
+    # not fresh, so p_t is the working-set test only: (2-1) * 212 > 16 * 3 -> pressure, declined
     r = t.step([5], 100, agent=0, now_ms=16_500)
     assert t.report == (10_000, 3, 0) and r.pressure and not r.save and r.new_chunks == 25
     # with no age limit the old report is still used: no pressure
