@@ -84,7 +84,7 @@ CONFIGS = {
     # sibling of C0 with a host tier large enough that restores happen
     "c0_big_tier": TraceConfig("c0_big_tier", "tiny", 0, 8, 12, 512, 200.0, 1.0, 2048,
                                interleave="round_robin", gpu_blocks=128, host_blocks=1024),
-    # C2: 32 agents x 40 turns, tier sized to the working-set estimate (at run time)
+    # C2: 32 agents x 40 turns, tier capacity = the Eq. 5 working-set size (computed at run time)
     "c2": TraceConfig("c2", "qwen3_30b_a3b", 2, 32, 40, 4096, 1500.0, 1.2, 65536,
                       interleave="tool_gap",
                       gpu_blocks=(20 * GIB) // SHAPES["qwen3_30b_a3b"].block_bytes,

@@ -152,7 +152,7 @@ typedef struct eakv_config {
                                       wait at eakv_turn_begin).  Call eakv_sync
                                       before reading the tier on the host                              */
     int64_t telemetry_period_ms;   /* Appendix D, pressure signal and parameter table (report interval 1 s,
-                                      maximum age of a fresh report 5 s).  0: the occupancy and eviction
+                                      a report counts as fresh for 5 s).  0: the occupancy and eviction
                                       terms of Eq. 10 are read from the tier itself at every request.
                                       P > 0: they are read from the latest published report.  Reports are
                                       published at the virtual times P, 2P, ... (now_ms of eakv_tier_step);
@@ -308,7 +308,7 @@ int eakv_gpu_tier_step(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_blo
 int eakv_gpu_tier_release(eakv_ctx* ctx, int32_t block_id);
 
 /* Several requests at once (Section 2: the engine runs up to a cap of requests at the same time
- * and suspends one when GPU KV memory runs out; Appendix A: cap 16).  eakv_gpu_tier_acquire is
+ * and suspends one if their KV no longer fits on the GPU; Appendix A: cap 16).  eakv_gpu_tier_acquire is
  * eakv_gpu_tier_step for a request that stays running: it references the keys in order in the same
  * way and then keeps every block of the prompt (and the tail block) pinned under request_id, out
  * of the recency order, so that no other request can take them.  A block already pinned by
@@ -327,8 +327,8 @@ int eakv_gpu_tier_acquire(eakv_ctx* ctx, int64_t request_id, const uint64_t* has
                           int32_t* tail_block_out);
 int eakv_gpu_tier_release_request(eakv_ctx* ctx, int64_t request_id);
 
-/* Store (Section 2 host writes; Appendix D: copy only absent chunks, from their original
- * GPU KV locations): for every j with admit_mask[j] != 0 copy all 2L pieces of pool block
+/* Store (Section 2 host writes; Appendix D: a chunk is copied only if the tier lacks it, straight
+ * out of the paged blocks that hold it): for every j with admit_mask[j] != 0 copy all 2L pieces of pool block
  * block_table[j] to tier slot host_slots[j].  admit_mask NULL = all admitted.
  *   block_table, host_slots host int32[n_blocks]; admit_mask host uint8[n_blocks] or NULL
  * Entries with admit 0 are ignored (their ids are not validated).  Asynchronous on
@@ -402,7 +402,7 @@ int eakv_turn_end(eakv_ctx* ctx, void* cuda_stream);
 int eakv_turn_abort(eakv_ctx* ctx);
 
 /* The same turn for an engine that runs several requests at once (Section 2: the engine's cap on
- * running requests; Appendix A: 16) and suspends one when GPU KV memory runs out.  Any number of
+ * running requests; Appendix A: 16) and suspends one if their KV no longer fits on the GPU.  Any number of
  * requests may be open, each under a request_id of the caller's choosing.
  * eakv_request_begin: as eakv_turn_begin, but the prompt's GPU blocks are taken with
  * eakv_gpu_tier_acquire and stay pinned under request_id.  EAKV_E_BUSY, with neither tier
@@ -484,7 +484,7 @@ int eakv_working_set_sizes(const int64_t* dist_dev, int64_t n_refs, const int64_
 
 /* Declined-chunk audit (Appendix D, "Reuse distance of declined chunks"; Proposition 1): of the
  * references whose miss an admission policy declined, how many could be declined at no cost --
- * their chunk is referenced next at reuse distance D >= capacity, or never again.
+ * the chunk's next reference has reuse distance D >= capacity, or there is none.
  *   keys_dev      device uint64[n_refs], the tier's reference stream (values below 2^61)
  *   declined_dev  device uint8[n_refs], non-zero where the miss was declined
  *   capacity      K_H in tier units

@@ -1,6 +1,6 @@
 """Which declined writes could the tier afford to decline?  (Section 5.5 and Appendix D,
 "Reuse distance of declined chunks": a declined chunk meets the condition of Proposition 1
-when its next reference lies at reuse distance D >= K_H, or never comes.)
+if the chunk's next reference has D >= K_H, or if there is no next reference.)
 
 Also the threshold sensitivity of Appendix D: for a write threshold kappa under fixed
 admission (every request under pressure), which requests are filtered and what share of

@@ -1,11 +1,10 @@
 """Closed-loop replay with a service-time model (test infrastructure, CPU only).
 
 Section 2 ("A closed-loop workload"), Section 5.1 and Appendix B ("Workload construction",
-"Timing boundary"): tasks enter the active pool of size A in their listed order; a task's
-next call becomes eligible once its previous response has finished and the recorded
-inter-call interval has elapsed; when a task's last call finishes the next waiting task
-enters the pool; makespan is the completion time of the last task and includes every
-inter-call interval.  Serving decisions therefore change the order in which the tiers see
+"Timing boundary"): A tasks are active at a time, admitted in list order; a task may issue call
+k+1 only after call k's response is complete and the recorded gap between the two has gone by;
+a task that has finished all of its calls frees its place for the next one in the list; the
+makespan is when the last response of all completes, gaps included.  Serving decisions therefore change the order in which the tiers see
 the calls.
 
 The engine here is this build's reading (the paper runs a real engine): one call at a time,

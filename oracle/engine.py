@@ -3,8 +3,8 @@
 
 What the paper fixes (Section 2, "A closed-loop workload"; Appendix A; Appendix C): tasks in an
 active pool of size A issue their next call after the previous response and the recorded
-interval; the serving engine separately caps how many requests it runs at once (16 in the
-paper's setup); a request the engine suspends when GPU KV memory runs out is later resumed by
+interval; the engine has a limit of its own on concurrently running requests (16 in the
+paper's setup); if the GPU cannot hold the KV of all of them it suspends one, which later resumes by
 recomputing its KV, and the tokens recomputed that way (J) add to computed prefill.  The store
 or skip choice of a request's first lookup is kept for its later lookups, including those after
 a preemption (Appendix D).

@@ -1,8 +1,8 @@
 """Longest cached prefix (Section 2 "Exact-prefix reuse"; Appendix C "Prefix coverage
 from a reference stream", and the restore equation R_j = max{0, H_j - G_j} there).
 
-A lookup walks the block keys from the start and stops at the first absent one: later
-isolated resident blocks do not extend the recoverable prefix.
+A lookup walks the block keys from the start and stops at the first absent one: a resident
+block behind a gap does not count, since only an unbroken prefix can be restored.
 """
 
 

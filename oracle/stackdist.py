@@ -1,7 +1,7 @@
 """Stack-distance capacity model (Section 3.2, Eq. 4; Appendix C "Prefix coverage from
 a reference stream").
 
-The reuse distance D of a reference counts the distinct *other* chunks referenced
+The reuse distance D of a reference is the number of different chunks, *other* than this one, touched
 strictly between it and the previous reference to the same chunk (infinite on a first
 reference).  Under a fully associative LRU tier that admits every miss, a reference
 hits exactly when D < K (Mattson's inclusion property).  Host coverage of a request is

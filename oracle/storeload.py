@@ -1,5 +1,5 @@
 """Store and load of KV blocks as opaque bytes (Section 2: host writes and restores;
-Appendix D: only absent chunks are copied, from their original GPU KV locations).
+Appendix D: a chunk is copied only if the tier lacks it, straight out of the paged blocks that hold it).
 
 Layouts
   pool : list of 2L numpy uint8 arrays, pool[2*l + kv] has shape [NB, piece_bytes]

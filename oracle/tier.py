@@ -1,13 +1,13 @@
 """Host-tier reference model and write admission.
 
 Reference model (Appendix D, "Reference model" and "Recency order of the host tier"):
-the tier starts empty and holds at most K_H chunks in recency order.  A reference to a
-resident chunk hits and moves it to the most-recent end.  A miss that is admitted
-inserts the chunk at the most-recent end, first evicting the least-recent chunk when
-K_H chunks are resident; a declined miss leaves the tier unchanged.
+an LRU list of capacity K_H chunks, empty at time zero.  Referencing a resident chunk is a hit
+and makes it the most recent entry.  An admitted miss appends the chunk as the most recent entry;
+if the list already has K_H entries its least recent one is dropped first.  A miss that is
+declined changes nothing.
 
-Write rule (Eq. 6): a request with n prompt tokens of which the host holds the first h
-needs u = floor(n/b) - floor(h/b) new full chunks and save(r) = not (p_t and u > kappa),
+Write rule (Eq. 6): with n prompt tokens and a host-resident prefix of h tokens, the request
+would add u = floor(n/b) - floor(h/b) full chunks, and save(r) = not (p_t and u > kappa),
 decided once per request.  p_t is 0 for plain offload (write-all), 1 for fixed write
 admission, and the pressure signal of Eq. 10 for capacity-conditioned admission:
 p_t = [ (A_t - 1) N_t beta > C_H ] and [ o_t >= theta and e_t > 0 ].  Copy-time
@@ -24,9 +24,8 @@ Readings taken where the paper is silent (integers only, virtual time in ms):
   * a request with more full chunks than K_H is refused and changes nothing.
 
 Tier reports (Appendix D, "Pressure signal" and the parameter table: the tier publishes the number
-of registered chunks, K_H and e_t every second; a report older than 5 seconds is not fresh; when
-no fresh report exists, before the first publication for instance, the first factor alone
-decides).  With ``telemetry_period_ms`` = P > 0 the second factor is read from the latest report
+of registered chunks, K_H and e_t every second; a report older than 5 seconds is not fresh; with
+nothing fresh to read (nothing published yet, say) p_t reduces to its working-set factor).  With ``telemetry_period_ms`` = P > 0 the second factor is read from the latest report
 instead of from the tier itself: reports are published at the virtual times P, 2P, 3P, ...; the
 report of time t describes the tier as the requests before t left it (registered chunks, and the
 evictions with a time in (t - W, t)); a request at time ``now`` reads the report of time
@@ -138,8 +137,8 @@ class HostTier:
     # ---- one request ----------------------------------------------------------------------
     def step(self, keys, n_tokens, agent, now_ms, decided=None):
         """``decided``: None for the request's first lookup.  A later lookup of the same request
-        (after a preemption; Appendix D: the store/skip choice is kept for later lookups of the
-        same request) passes the choice made then: the walk is the same, but the request is not
+        (after a preemption; Appendix D: the store/skip choice made at the first lookup
+        also holds for the request's further lookups) passes the choice made then: the walk is the same, but the request is not
         registered again in the activity and prompt-length windows, which count first lookups."""
         if len(keys) > self.K:
             raise CapacityError("request references more blocks than the tier holds")

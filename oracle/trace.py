@@ -79,8 +79,8 @@ class GpuTier:
             self.free.append(block_id)
 
     # ---- several requests at once: a running request's blocks cannot be evicted -------------
-    # (Section 2: the engine runs several requests at once and suspends one when GPU KV memory
-    # runs out.)  A pinned block is out of the recency order; when its last holder lets go it
+    # (Section 2: the engine runs several requests at once and suspends one if their KV no
+    # longer fits on the GPU.)  A pinned block is out of the recency order; when its last holder lets go it
     # re-enters at the most-recent end.  acquire() followed at once by release_request() leaves
     # the tier exactly as step() does.
     def fits(self, keys, need_tail):

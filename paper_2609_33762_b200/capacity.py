@@ -4,7 +4,7 @@ and the working-set sizes that go with them.
 
     python -m paper_2609_33762_b200.capacity --config c2 --host-gib 8,16,32,64,128,256
 
-The reference stream (every request references the full blocks of its prompt, in request
+The reference stream (each request touches all full blocks of its prompt, in request
 order) is built from one batched hash launch: prompts only grow by appends, so a request's
 keys are a prefix of its agent's final key list.
 """

@@ -1,10 +1,9 @@
 """Closed-loop replay: the order of the calls follows from how long each one takes.
 
-Section 2 ("A closed-loop workload"), Section 5.1 and Appendix B of the paper: tasks enter an
-active pool of size A in their listed order, a task's next call becomes eligible when its
-previous response has finished and the recorded inter-call interval has passed, a finished
-task hands its place to the next waiting one, and makespan is the completion time of the
-last task.  The engine is one call at a time, first come first served by eligibility (lower
+Section 2 ("A closed-loop workload"), Section 5.1 and Appendix B of the paper: A tasks are
+active at a time, admitted in list order; a task may issue its next call only after the previous
+response is complete and the recorded gap has gone by; a finished task frees its place for the
+next one in the list; the makespan is when the last response of all completes.  The engine is one call at a time, first come first served by eligibility (lower
 task id first among equals).  A call's response time follows Eq. 2 in integer microseconds:
 
     overhead + ceil(computed_tokens * t_pf) + [restored > 0] (tau_load + ceil(restored_bytes / B_H2D))
@@ -100,8 +99,8 @@ class ClosedLoop:
 class EngineLoop:
     """Closed loop against an engine that runs up to ``running_cap`` requests at once (Section 2 and
     Appendix A of the paper: the engine's own cap on running requests, 16 there, beside the active
-    pool) and suspends a running request when GPU KV memory runs out, to resume it later by
-    recomputing its KV (Section 2; the recomputed tokens are the J terms of Appendix C).
+    pool) and suspends a running request if the GPU cannot hold every running request's KV, to resume
+    it later by recomputing its KV (Section 2; the recomputed tokens are the J terms of Appendix C).
 
     The engine model: a response is a prefill phase, served one request at a time, followed by
     ``decode_us`` of decoding during which the request stays running (its GPU blocks stay pinned)
@@ -382,7 +381,7 @@ def main():
     ap.add_argument("--turns", type=int, default=None)
     ap.add_argument("--running-cap", type=int, default=None,
                     help="engine model: this many requests run at once, GPU blocks pinned while they run, "
-                         "preemption when GPU KV memory runs out (default: one call at a time)")
+                         "preemption if the GPU pool cannot hold all running requests (default: one call at a time)")
     ap.add_argument("--decode-ms", type=float, default=2000.0, help="engine model: decoding time per call")
     ap.add_argument("--gpu-gib", type=float, default=None, help="GPU KV tier size (default: the configuration's)")
     args = ap.parse_args()

@@ -1,8 +1,8 @@
 // Stack-distance capacity model on the GPU (Section 3.2, Eq. 4; Appendix C "Prefix coverage
 // from a reference stream").
 //
-// Reuse distance of reference i with previous reference p to the same chunk: the number of
-// distinct other chunks referenced strictly between them.  A position j in (p, i) is the
+// Reuse distance of reference i with previous reference p to the same chunk: how many different
+// chunks, other than this one, are touched strictly between the two.  A position j in (p, i) is the
 // first reference to its chunk inside that window exactly when its own previous reference lies
 // before p, and every j <= p trivially has prev_j < p, so
 //
@@ -16,7 +16,7 @@
 //      three-kernel exclusive scan per level: no kernel waits for another);
 //   3. one "count of values below x in a prefix" query per reference, nbits steps each.
 // The capacity curve then needs only D: a reference hits a tier of K chunks iff D < K
-// (Mattson); a request's host coverage is its leading run of hits; restored = max(0, H - G);
+// (Mattson); the host-covered prefix of a request = its leading run of hits; restored = max(0, H - G);
 // computed prefill = n - max(G, H) * b.
 #include <algorithm>
 #include <cstdint>

@@ -7,7 +7,7 @@ plus the achieved store/load rates.
     python -m paper_2609_33762_b200.replay --config c4 --host-gib 64 --limit 2000
 
 Sizing follows the paper's rule: working-set scale (A - 1) * N_mean * beta (Eq. 5) for
-configurations that ask for a tier "sized to the working set", capped by the pinned memory
+configurations whose tier capacity is defined as that working-set size, capped by the pinned memory
 the box can spare.  With --no-data-plane only keys, matching and both tiers' bookkeeping run.
 """
 from __future__ import annotations

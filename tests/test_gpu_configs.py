@@ -86,7 +86,7 @@ def check_sampled_bytes(server, oracle, shape, n=48):
 
 
 def test_config2_full_trace_control_plane():
-    """Write-all, tier sized to the working-set scale of Eq. 5, all 1,280 requests."""
+    """Write-all, tier capacity = the Eq. 5 working-set size, all 1,280 requests."""
     from paper_2609_33762_b200 import replay
     cfg = CONFIGS["c2"]
     shape = SHAPES[cfg.shape]

@@ -258,7 +258,7 @@ def test_closed_loop_replay_bit_exact(policy, kh, pool, native):
     (0, 64, 136, 4, 50_000, 4, 1)])
 def test_engine_replay_with_preemption_bit_exact(policy, kh, gpu_blocks, S, decode_us, R, link, native):
     """The engine model (several running requests with pinned GPU blocks, suspension when GPU KV
-    memory runs out, resumption by restoring and recomputing) on the GPU path with bytes: every
+    memory is short, resumption by restoring and recomputing) on the GPU path with bytes: every
     scheduler event, every record of every first and resumed lookup, J, and every resident byte of
     both tiers equal the oracle's."""
     from oracle import closedloop as ocl
