@@ -237,6 +237,28 @@ def test_bad_shapes_rejected_at_create():
     assert ei.value.code == e.E_INVAL
 
 
+def test_a_tier_that_cannot_be_allocated_is_refused_cleanly():
+    """A 3 TiB tier in HBM (2 M slots of 1.5 MiB): the one device allocation of that size is refused
+    by the runtime at once, create returns EAKV_E_NOMEM after freeing what it had, and the device
+    is as usable as before (a working context right after it)."""
+    e = eakv()
+    shape = SHAPES["qwen3_30b_a3b"]
+    t = torch.zeros(2 * shape.piece_bytes // 2, dtype=torch.int16, device="cuda")
+    free_before = torch.cuda.mem_get_info()[0]
+    with pytest.raises(e.EakvError) as ei:
+        e.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+                  block_size=shape.block_size, gpu_blocks=2, host_blocks=1 << 21,
+                  kv_base=[t.data_ptr()] * shape.pieces_per_block, tier_location=e.TIER_DEVICE)
+    assert ei.value.code == e.E_NOMEM
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] >= free_before - (64 << 20)      # nothing of the attempt is left
+    rig = Rig(SHAPE_CASES["tiny"], 8, 4, 11, tier_location=1)
+    rig.store(np.array([1, 3], np.int32), None, np.array([0, 2], np.int32))
+    rig.load(np.array([0, 2], np.int32), np.array([5, 6], np.int32))
+    rig.check()
+    rig.close()
+
+
 @pytest.mark.parametrize("kw", [
     dict(tier_location=1, copy_path=1), dict(tier_location=1, copy_path=0),
     dict(tier_location=0, link_strategy=0),
@@ -334,6 +356,28 @@ def test_layer_group_event_means_the_group_has_landed(name, group, contiguous_sl
         for i, q in enumerate(range(q0, q1)):
             assert np.array_equal(got[i], rig.pool_np[q][dst]), (g, q)
     stream.synchronize()
+    rig.check()
+    rig.close()
+
+
+def test_a_tier_that_cannot_be_allocated_is_refused_cleanly():
+    """A 3 TiB tier in HBM (2 M slots of 1.5 MiB): the one device allocation of that size is refused
+    by the runtime at once, create returns EAKV_E_NOMEM after freeing what it had, and the device
+    is as usable as before (a working context right after it)."""
+    e = eakv()
+    shape = SHAPES["qwen3_30b_a3b"]
+    t = torch.zeros(2 * shape.piece_bytes // 2, dtype=torch.int16, device="cuda")
+    free_before = torch.cuda.mem_get_info()[0]
+    with pytest.raises(e.EakvError) as ei:
+        e.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+                  block_size=shape.block_size, gpu_blocks=2, host_blocks=1 << 21,
+                  kv_base=[t.data_ptr()] * shape.pieces_per_block, tier_location=e.TIER_DEVICE)
+    assert ei.value.code == e.E_NOMEM
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] >= free_before - (64 << 20)      # nothing of the attempt is left
+    rig = Rig(SHAPE_CASES["tiny"], 8, 4, 11, tier_location=1)
+    rig.store(np.array([1, 3], np.int32), None, np.array([0, 2], np.int32))
+    rig.load(np.array([0, 2], np.int32), np.array([5, 6], np.int32))
     rig.check()
     rig.close()
 
