@@ -414,7 +414,12 @@ int eakv_turn_abort(eakv_ctx* ctx);
  * the admitted blocks on cuda_stream (deferred under eakv_config.write_behind); once per begin.
  * Between a request's begin and its store the units it admitted are listed in the host tier (no
  * other request stores them again) but do not count toward another request's host prefix: their
- * slots hold nothing yet, so that request computes those blocks itself.  After the store they are
+ * slots hold nothing yet, so that request computes those blocks itself.  If another request's
+ * lookup evicts such a unit before its store, the slot has a new owner and the store leaves that
+ * unit out (view->n_stored_blocks counts what was admitted at the lookup; eakv_stats.blocks_stored
+ * what was written); the bookkeeping is that of the reference model either way, which registers a
+ * write at its lookup.  A release before the store takes back only the units the request still
+ * owns.  After the store they are
  * restorable; a restore by another request must be ordered after that store on the GPU (same
  * stream, or an event), as for any store followed by a load of the same slots.  The GPU side has
  * no such guard: a block that an open request was told to fill counts as resident for a later

@@ -153,6 +153,8 @@ class TraceOracle:
                          for _ in range(shape.pieces_per_block)]
             self.tier = np.zeros((host_blocks * self.R, shape.pieces_per_block, P), dtype=np.uint8)
         self.records = []
+        self.pending = {}        # unit key -> the open request that admitted it and has not written it yet
+        self.open = {}           # request id -> what its deferred store still needs
         self.totals = dict(prompt_tokens=0, fresh_tokens=0, loaded_blocks=0, stored_blocks=0,
                            gpu_hit_blocks=0, host_hit_blocks=0)
 
@@ -211,11 +213,18 @@ class TraceOracle:
         return rec
 
     # ---- requests that overlap: begin pins the GPU blocks, finish lets them go ---------------
-    def begin(self, request_id, tokens, agent, now_ms, keys=None, decided=None):
+    def begin(self, request_id, tokens, agent, now_ms, keys=None, decided=None, defer_store=False):
         """The same turn as ``turn`` up to and including the store, with the request's GPU blocks
         pinned until ``finish``.  Returns None, with nothing changed, if the GPU tier cannot hold
         the request beside the running ones.  ``decided``: the save decision of the request's
-        first lookup when this is a later one (a resumed request), else None."""
+        first lookup when this is a later one (a resumed request), else None.
+
+        ``defer_store``: the host write happens later, at ``store(request_id)`` (an engine writes a
+        request's KV once it has computed it, and other requests may be looked up in between).
+        The bookkeeping is that of the reference model all the same, every write registered at its
+        lookup; what changes is physical: a unit whose bytes are not there yet cannot be restored,
+        so another request's host prefix ends before the first such unit, and a unit that a later
+        lookup evicts before its bytes arrive is never written (its slot has a new owner)."""
         n = len(tokens)
         if keys is None:
             keys = ohash.hash_blocks(tokens, self.b, self.hash_seed, self.hash_base)
@@ -230,9 +239,15 @@ class TraceOracle:
         R = self.R
         chunk_keys = keys[R - 1::R]
         Hc = self.host.leading_run(chunk_keys)
+        for c in range(Hc):
+            if chunk_keys[c] in self.pending:          # listed, but its bytes have not been written yet
+                Hc = c
+                break
         H = Hc * R
         host_slots = [self.host.slot_of(k) * R + i for k in chunk_keys[:Hc] for i in range(R)]
         res = self.host.step(chunk_keys, n, agent, now_ms, decided=decided)
+        for k, _ in res.evicted:
+            self.pending.pop(k, None)                  # a pending write lost its slot
         resident, gpu_ids, tail = self.gpu.acquire(request_id, keys, need_tail)
         cover = max(G, H)
         lo, hi = (G, H) if H > G else (G, G)
@@ -251,7 +266,14 @@ class TraceOracle:
                     words = self.payload([keys[j] for j in fill], q, W)
                     for r, j in enumerate(fill):
                         self.pool[q][gpu_ids[j], :] = words[r].view(np.uint8)
-            storeload.store(self.pool, self.tier, gpu_ids, admit_b, slot_b)
+            if not defer_store:
+                storeload.store(self.pool, self.tier, gpu_ids, admit_b, slot_b)
+        if defer_store:
+            for c, a in enumerate(res.admit):
+                if a:
+                    self.pending[chunk_keys[c]] = request_id
+            self.open[request_id] = dict(chunk_keys=chunk_keys, admit=list(res.admit), gpu_ids=gpu_ids,
+                                         admit_b=admit_b, slot_b=slot_b)
         rec = dict(agent=agent, now_ms=now_ms, n_tokens=n, keys=keys, G=G, H=H,
                    new_chunks=res.new_chunks, pressure=res.pressure, save=res.save,
                    hit=res.hit, admit=res.admit, slot=res.slot, evicted=res.evicted,
@@ -271,8 +293,27 @@ class TraceOracle:
         self.records.append(rec)
         return rec
 
+    def store(self, request_id):
+        """The deferred host write of ``begin(..., defer_store=True)``: the admitted units that are
+        still this request's (no later lookup evicted them) are written; returns how many blocks."""
+        o = self.open.pop(request_id)
+        R = self.R
+        admit_b = list(o["admit_b"])
+        for c, a in enumerate(o["admit"]):
+            if not a:
+                continue
+            if self.pending.get(o["chunk_keys"][c]) == request_id:
+                del self.pending[o["chunk_keys"][c]]
+            else:
+                for i in range(R):
+                    admit_b[c * R + i] = 0
+        if self.payload is not None:
+            storeload.store(self.pool, self.tier, o["gpu_ids"], admit_b, o["slot_b"])
+        return sum(admit_b)
+
     def finish(self, request_id):
         """The request finished, or the engine suspended it: its blocks become evictable."""
+        assert request_id not in self.open, "store first"
         self.gpu.release_request(request_id)
 
     def run(self, trace, limit=None):

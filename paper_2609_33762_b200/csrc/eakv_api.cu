@@ -54,9 +54,10 @@ struct TurnState {
     std::vector<uint64_t> keys, unit_keys, evicted_keys;
     std::vector<int32_t> block, slot_u, slot_b, evicted_slots, host_slots;
     std::vector<uint8_t> resident, fill, hit, admit_u, admit_b;
+    std::vector<uint8_t> owned_u;      // units this turn admitted and still has to write (see claim_units)
     int64_t request_id = kNoRequest;
     int32_t tail = -1;
-    bool open = false, stored = false;
+    bool open = false, stored = false, claimed = false;
 };
 }  // namespace
 
@@ -127,7 +128,10 @@ struct eakv_ctx {
     std::unordered_map<int64_t, TurnState> requests;   // open turns of running requests (eakv_request_*)
     // tier units an open turn admitted whose store has not been enqueued yet: listed in the host
     // index (so nobody stores them twice) but not restorable by another request
-    std::unordered_set<uint64_t> unstored_units;
+    // units an open request admitted and has not written yet -> that request.  An eviction takes a
+    // unit out of here: its slot belongs to someone else from then on and is never written by the
+    // request that lost it.
+    std::unordered_map<uint64_t, int64_t> unstored_units;
 
     std::string cuda_err;
 };
@@ -927,6 +931,7 @@ static int tier_step_impl(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_
             int32_t vslot = -1;
             const int32_t ns = T.insert(key, &ev, &vkey, &vslot);
             if (ev) {
+                if (!ctx->unstored_units.empty()) ctx->unstored_units.erase(vkey);   // a pending write lost its slot
                 if (evicted_keys_out) evicted_keys_out[n_ev] = vkey;
                 if (evicted_slots_out) evicted_slots_out[n_ev] = vslot;
                 ++n_ev;
@@ -1220,21 +1225,37 @@ namespace {
 // those the engine was to fill (the restored ones hold their bytes).  A block another running
 // request shares stays.  Promotions and evictions the turn caused stand.  Lets the turn's GPU
 // blocks go (pins, tail block).
-void forget_unstored(eakv_ctx* ctx, const TurnState& T) {
-    if (ctx->unstored_units.empty()) return;
+// Which of the units the turn admitted are still its own to write (owned_u), once per turn.  A
+// single turn owns all of them: nothing comes between its begin and its end.  A request owns those
+// that no other request's lookup has evicted since its own (the reference model saw this request's
+// write at its lookup, so a later eviction simply overwrote it); they leave the pending set here.
+void claim_units(eakv_ctx* ctx, TurnState& T) {
+    if (T.claimed) return;
+    T.claimed = true;
     const uint64_t* ukeys = T.unit_keys.empty() ? T.keys.data() : T.unit_keys.data();
-    for (size_t c = 0; c < T.admit_u.size(); ++c)
-        if (T.admit_u[c]) ctx->unstored_units.erase(ukeys[c]);
+    T.owned_u.assign(T.admit_u.size(), 0);
+    for (size_t c = 0; c < T.admit_u.size(); ++c) {
+        if (!T.admit_u[c]) continue;
+        if (T.request_id == kNoRequest) {
+            T.owned_u[c] = 1;
+            continue;
+        }
+        auto it = ctx->unstored_units.find(ukeys[c]);
+        if (it != ctx->unstored_units.end() && it->second == T.request_id) {
+            T.owned_u[c] = 1;
+            ctx->unstored_units.erase(it);
+        }
+    }
 }
 
 void withdraw_turn(eakv_ctx* ctx, TurnState& T, bool host_units, int gpu_mode) {
-    forget_unstored(ctx, T);
+    claim_units(ctx, T);
     if (host_units) {
         int64_t n = 0;
         const uint64_t* ukeys = T.unit_keys.empty() ? T.keys.data() : T.unit_keys.data();
         // last admitted first, so that the free stack hands the slots out again in the same order
-        for (size_t c = T.admit_u.size(); c-- > 0;)
-            if (T.admit_u[c] && ctx->host_tier->erase(ukeys[c]) >= 0) ++n;
+        for (size_t c = T.owned_u.size(); c-- > 0;)
+            if (T.owned_u[c] && ctx->host_tier->erase(ukeys[c]) >= 0) ++n;
         ctx->stats.admitted -= n;
         ctx->stats.resident = ctx->host_tier->resident();
     }
@@ -1324,6 +1345,8 @@ int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32
     T.request_id = request_id;
     T.tail = -1;
     T.stored = false;
+    T.claimed = false;
+    T.owned_u.clear();
     // lookups (they change nothing), then the GPU side -- a running request whose blocks do not fit
     // beside the others is refused here with both tiers untouched -- then the host tier
     int64_t G = 0, G_unused = 0, Hu = 0;
@@ -1397,7 +1420,7 @@ int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32
     }
     if (as_request)
         for (int64_t c = 0; c < nu; ++c)
-            if (T.admit_u[c]) ctx->unstored_units.insert(ukeys[c]);
+            if (T.admit_u[c]) ctx->unstored_units[ukeys[c]] = request_id;
     view->n_blocks = nblk; view->n_units = nu;
     view->gpu_prefix_blocks = G; view->host_prefix_blocks = H;
     view->restore_lo = lo; view->restore_hi = hi;
@@ -1416,10 +1439,16 @@ int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32
 // the store of an open turn's admitted blocks (directly, or deferred on the context's stream)
 int turn_store_impl(eakv_ctx* ctx, TurnState& T, void* cuda_stream) {
     const int64_t nblk = (int64_t)T.block.size();
+    T.stored = true;
+    claim_units(ctx, T);                                     // from here on a stream-ordered restore finds the bytes
+    // a unit that another request's lookup evicted in the meantime is not written: its slot is not
+    // this request's any more
+    const int64_t R = ctx->chunk_tokens / ctx->cfg.block_size;
+    for (size_t c = 0; c < T.admit_u.size(); ++c)
+        if (T.admit_u[c] && !T.owned_u[c])
+            for (int64_t i = 0; i < R; ++i) T.admit_b[c * R + i] = 0;
     bool any_store = false;
     for (int64_t j = 0; j < nblk && !any_store; ++j) any_store = T.admit_b[j] != 0;
-    T.stored = true;
-    forget_unstored(ctx, T);                                 // from here on a stream-ordered restore finds the bytes
     if (ctx->device < 0 || !any_store) return EAKV_OK;       // bookkeeping only, or nothing admitted
     if (!ctx->cfg.write_behind)
         return eakv_store(ctx, T.block.data(), T.admit_b.data(), T.slot_b.data(), nblk, cuda_stream);

@@ -202,16 +202,20 @@ class AgentServer:
         G, H = rec["G"], rec["H"]
         return rec, G, H
 
-    def begin(self, request_id, tokens, agent, now_ms, decided=None):
+    def begin(self, request_id, tokens, agent, now_ms, decided=None, defer_store=False):
         """A turn of a request that stays running: the same steps as ``turn`` up to and including
         the store, with the request's GPU blocks pinned under ``request_id`` until ``finish``
         (eakv_gpu_tier_acquire).  Returns None, with nothing changed, when the blocks do not fit
         beside the running requests.  ``decided``: None for the request's first lookup, else the
-        store/skip choice made then (a resumed request: eakv_tier_step_again)."""
+        store/skip choice made then (a resumed request: eakv_tier_step_again).  ``defer_store``
+        (turn engine only): the host write waits for ``store(request_id)``, as in an engine that
+        looks other requests up while this one computes."""
         tokens = np.asarray(tokens, dtype=np.int32)
         n = len(tokens)
         if self.native_turn:
-            return self._begin_native(request_id, tokens, agent, now_ms, decided)
+            return self._begin_native(request_id, tokens, agent, now_ms, decided, defer_store)
+        if defer_store:
+            raise ValueError("defer_store needs the turn engine (native_turn)")
         keys = self.block_keys(tokens, agent)
         nblk = len(keys)
         R = self.R
@@ -277,7 +281,11 @@ class AgentServer:
         self.records.append(rec)
         return rec
 
-    def _begin_native(self, request_id, tokens, agent, now_ms, decided):
+    def store(self, request_id):
+        """The deferred host write of ``begin(..., defer_store=True)`` (eakv_request_store)."""
+        self.ctx.eakv_request_store(request_id, self.stream if self.data_plane else None)
+
+    def _begin_native(self, request_id, tokens, agent, now_ms, decided, defer_store=False):
         """The same through eakv_request_begin / eakv_request_store."""
         n = len(tokens)
         if self.data_plane:
@@ -297,7 +305,8 @@ class AgentServer:
             if prev is None or len(keys) >= len(prev):
                 self._agent_keys[agent] = keys
         self._fill(keys, blocks, np.nonzero(v["needs_fill"])[0])
-        self.ctx.eakv_request_store(request_id, self.stream)
+        if not defer_store:
+            self.ctx.eakv_request_store(request_id, self.stream)
         rec = self._record_from_view(v, agent, now_ms, n)
         rec.update(request_id=request_id, resumed=decided is not None)
         t = self.totals

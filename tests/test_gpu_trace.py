@@ -291,6 +291,58 @@ def test_engine_replay_with_preemption_bit_exact(policy, kh, gpu_blocks, S, deco
     server.close()
 
 
+@pytest.mark.parametrize("R,link,seed,write_behind", [(1, 1, 5, False), (1, 0, 6, False), (2, 1, 7, False),
+                                                       (1, 1, 8, True)])
+def test_deferred_stores_interleaved_with_other_lookups_with_bytes(R, link, seed, write_behind):
+    """Requests whose host write comes only after other requests have been looked up
+    (eakv_request_begin ... eakv_request_store): a unit that a later lookup evicted before its
+    bytes arrived must not be written, or the slot's new owner would read a stranger's KV.  Every
+    record equals the oracle's, and after every store each listed unit whose write is not pending
+    holds the oracle's bytes (which tests/test_oracle_deferred_store.py pins to the payload)."""
+    from deferred_util import drive, operations
+    from paper_2609_33762_b200.harness import AgentServer
+    shape = SHAPES["tiny"]
+    b = shape.block_size
+    gpu_blocks, kh = 200, 96 // R
+    oracle = TraceOracle(shape, gpu_blocks, kh, payload=key_words_numpy, chunk_blocks=R)
+    server = AgentServer(shape, gpu_blocks, kh, key_words_numpy, incremental_hash=False, chunk_blocks=R,
+                         link_strategy=link, native_turn=True, write_behind=write_behind)
+    seen = dict(begins=0, skipped=0)
+
+    def check_listed_bytes():
+        server.ctx.eakv_sync()
+        tier = server.ctx.tier_host_view()
+        for ukey, slot in oracle.host.order.items():
+            if ukey not in oracle.pending:
+                for i in range(R):
+                    assert np.array_equal(tier[slot * R + i], oracle.tier[slot * R + i]), (ukey, slot, i)
+
+    def on_begin(rid, agent, tokens, now):
+        w = oracle.begin(rid, tokens, agent, now, defer_store=True)
+        g = server.begin(rid, tokens, agent, now, defer_store=True)
+        assert (g is None) == (w is None)
+        if g is None:
+            return False
+        seen["begins"] += 1
+        compare_records([g], [w])
+        return True
+
+    def on_store(rid):
+        admitted = sum(oracle.open[rid]["admit_b"])
+        seen["skipped"] += admitted - oracle.store(rid)
+        server.store(rid)
+        check_listed_bytes()
+
+    def on_finish(rid):
+        oracle.finish(rid)
+        server.finish(rid)
+
+    drive(operations(seed, 260, b, 60 * b, max_open=4), on_begin, on_store, on_finish)
+    assert seen["begins"] > 60 and seen["skipped"] > 0          # evicted-before-written did occur
+    compare_bytes(server, oracle)
+    server.close()
+
+
 def test_warm_restart_with_adopted_tier_memory():
     """Half of the trace, then the process 'restarts': the host tier's index is exported, the
     context destroyed, a new one adopts the same pinned tier memory and imports the index.  The

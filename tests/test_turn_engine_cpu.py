@@ -213,3 +213,84 @@ def test_units_admitted_by_an_open_request_are_not_restorable_until_it_stored(ea
     ctx.eakv_request_release(5)
     assert ctx.eakv_match(other)[:2] == (3, 3)
     ctx.close()
+
+
+@pytest.mark.parametrize("R,seed", [(1, 5), (1, 6), (2, 7), (4, 8)])
+def test_deferred_stores_interleaved_with_other_lookups_equal_the_oracle(eakv, R, seed):
+    """eakv_request_begin ... (other requests' lookups) ... eakv_request_store: every view equals
+    the oracle's deferred-store record, and the tier's final recency order and slots are equal.
+    (The bytes of the same interleavings are checked on the GPU.)"""
+    from deferred_util import drive, operations
+    shape = SHAPES["tiny"]
+    b = shape.block_size
+    kh = 160 // R
+    oracle = TraceOracle(shape, 160, kh, chunk_blocks=R)
+    ctx = cp_ctx(eakv, b, 160, kh, chunk_blocks=R)
+    seen = dict(begins=0, refused=0)
+
+    def on_begin(rid, agent, tokens, now):
+        w = oracle.begin(rid, tokens, agent, now, defer_store=True)
+        v = ctx.eakv_request_begin(rid, 0, len(tokens), keys_of(tokens, b), agent, now)
+        assert (v is None) == (w is None)
+        if v is None:
+            seen["refused"] += 1
+            return False
+        seen["begins"] += 1
+        compare_view(v, w, R)
+        return True
+
+    def on_store(rid):
+        oracle.store(rid)
+        ctx.eakv_request_store(rid)
+
+    def on_finish(rid):
+        oracle.finish(rid)
+        ctx.eakv_request_release(rid)
+
+    drive(operations(seed, 500, b, 60 * b, max_open=4), on_begin, on_store, on_finish)
+    keys, slots = ctx.eakv_tier_export()
+    assert list(zip(keys.tolist(), slots.tolist())) == list(oracle.host.order.items())
+    assert seen["begins"] > 100
+    ctx.close()
+
+
+def test_a_release_before_the_store_takes_back_only_units_the_request_still_owns(eakv):
+    """Request 1 admits six units; request 2's lookup evicts four of them unwritten and reuses
+    their slots; request 3 admits two of the evicted keys again.  Request 1, released without a
+    store, may take back only the two units it still owns: not request 3's, although they carry
+    keys request 1 once admitted, and not the slots request 2 now owns."""
+    b = 4
+    ctx = cp_ctx(eakv, b, 64, 8)
+    k1 = np.arange(1, 7, dtype=np.uint64)
+    k2 = np.arange(11, 17, dtype=np.uint64)
+    v1 = ctx.eakv_request_begin(1, 0, 6 * b, k1, 0, 0)
+    assert v1["slot"].tolist() == [0, 1, 2, 3, 4, 5]
+    v2 = ctx.eakv_request_begin(2, 0, 6 * b, k2, 1, 1)
+    assert v2["slot"].tolist() == [6, 7, 0, 1, 2, 3] and v2["evicted_keys"].tolist() == [1, 2, 3, 4]
+    ctx.eakv_request_store(2)
+    # keys 1, 2 come back through request 3 (evicting request 1's last two units, 5 and 6)
+    k3 = np.asarray([1, 2], dtype=np.uint64)
+    v3 = ctx.eakv_request_begin(3, 0, 2 * b, k3, 2, 2)
+    assert v3["admit"].tolist() == [1, 1] and v3["evicted_keys"].tolist() == [5, 6]
+    # request 1 owns nothing any more: its release changes no listing
+    before = ctx.eakv_tier_export()
+    ctx.eakv_request_release(1)
+    after = ctx.eakv_tier_export()
+    assert before[0].tolist() == after[0].tolist() and before[1].tolist() == after[1].tolist()
+    ctx.eakv_request_store(3)
+    assert ctx.eakv_match(k3)[1] == 2 and ctx.eakv_match(k2)[1] == 6
+    for rid in (2, 3):
+        ctx.eakv_request_release(rid)
+    # and a request that still owns some of its units takes back exactly those
+    k4 = np.arange(21, 25, dtype=np.uint64)
+    k5 = np.arange(31, 37, dtype=np.uint64)
+    ctx.eakv_request_begin(4, 0, 4 * b, k4, 0, 3)          # evicts 11..14
+    v5 = ctx.eakv_request_begin(5, 0, 6 * b, k5, 1, 4)     # evicts 15, 16, 1, 2, then 21, 22 of request 4
+    assert v5["evicted_keys"].tolist() == [15, 16, 1, 2, 21, 22]
+    ctx.eakv_request_release(4)                            # owns 23, 24 only
+    keys = ctx.eakv_tier_export()[0].tolist()
+    assert keys == [31, 32, 33, 34, 35, 36]
+    ctx.eakv_request_store(5)
+    ctx.eakv_request_release(5)
+    assert ctx.eakv_match(k5)[1] == 6
+    ctx.close()
