@@ -576,7 +576,13 @@ int eakv_sync(eakv_ctx* ctx);
  * slot of a skipped entry receives whatever that part of the staging buffer held).
  * eakv_selfcheck_wait_probe: enqueues a one-thread kernel that waits, with a short poll limit, on a
  * barrier nothing arrives at, gives up and raises the word: the next eakv_sync returns
- * EAKV_E_TIMEOUT and the context stays usable. */
+ * EAKV_E_TIMEOUT and the context stays usable.
+ * eakv_selfcheck_fail_next_transfer: a failure made on the host, for the paths that only a CUDA
+ * error reaches otherwise: the next restore step of eakv_turn_begin / eakv_request_begin, or the
+ * next store step of eakv_turn_end / eakv_request_store, returns `code` (a negative EAKV_E_*; 0
+ * disarms) with nothing enqueued, once.  The call then behaves as after a real failure at that
+ * point: what the turn registered is withdrawn.  Works on bookkeeping-only contexts too. */
+int eakv_selfcheck_fail_next_transfer(eakv_ctx* ctx, int32_t code);
 int eakv_selfcheck_limits(eakv_ctx* ctx, int64_t gpu_blocks, int64_t tier_slots, int64_t hash_blocks);
 int eakv_selfcheck_wait_probe(eakv_ctx* ctx, void* cuda_stream);
 

@@ -132,6 +132,7 @@ struct eakv_ctx {
     // unit out of here: its slot belongs to someone else from then on and is never written by the
     // request that lost it.
     std::unordered_map<uint64_t, int64_t> unstored_units;
+    int fail_next_transfer = 0;        // self-test: the next restore / store step returns this code instead
 
     std::string cuda_err;
 };
@@ -680,6 +681,21 @@ int eakv_selfcheck_limits(eakv_ctx* ctx, int64_t gpu_blocks, int64_t tier_slots,
     ctx->check_hash_blocks = hash_blocks;
     return EAKV_OK;
 }
+
+int eakv_selfcheck_fail_next_transfer(eakv_ctx* ctx, int32_t code) {
+    if (!ctx || code > 0) return EAKV_E_INVAL;
+    ctx->fail_next_transfer = code;
+    return EAKV_OK;
+}
+
+namespace {
+// the injected failure of eakv_selfcheck_fail_next_transfer, once
+int injected_failure(eakv_ctx* ctx) {
+    const int rc = ctx->fail_next_transfer;
+    ctx->fail_next_transfer = 0;
+    return rc;
+}
+}  // namespace
 
 int eakv_selfcheck_wait_probe(eakv_ctx* ctx, void* cuda_stream) {
     if (!ctx || ctx->device < 0) return EAKV_E_INVAL;
@@ -1374,6 +1390,11 @@ int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32
         withdraw_turn(ctx, T, false, 1);
         return rc;
     }
+    // the units this request admitted are its own to write until another lookup evicts them (before
+    // anything below can fail: a withdrawal takes back what is registered here)
+    if (as_request)
+        for (int64_t c = 0; c < nu; ++c)
+            if (T.admit_u[c]) ctx->unstored_units[ukeys[c]] = request_id;
     if (ctx->wb_pending) {
         bool reused = tail >= 0 && ctx->wb_blocks[tail];
         for (int64_t j = 0; j < nblk && !reused; ++j)
@@ -1391,12 +1412,14 @@ int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32
     const int64_t H = Hu * R;
     const int64_t cover = std::max(G, H);
     const int64_t lo = G, hi = H > G ? H : G;
-    if (hi > lo && !bookkeeping_only) {
+    if (hi > lo) {
         // block slots of the restored blocks: chunk slot * R + position inside the chunk
         std::vector<int32_t> slots((size_t)(hi - lo));
         for (int64_t j = lo; j < hi; ++j)
             slots[j - lo] = (int32_t)((int64_t)T.host_slots[j / R] * R + j % R);
-        rc = eakv_load(ctx, slots.data(), T.block.data() + lo, hi - lo, cuda_stream);
+        rc = injected_failure(ctx);
+        if (rc == EAKV_OK && !bookkeeping_only)
+            rc = eakv_load(ctx, slots.data(), T.block.data() + lo, hi - lo, cuda_stream);
         if (rc != EAKV_OK) {
             // nothing of this turn was restored or will be computed: neither tier may list it
             withdraw_turn(ctx, T, true, 1);
@@ -1418,9 +1441,6 @@ int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32
             ++n_store;
         }
     }
-    if (as_request)
-        for (int64_t c = 0; c < nu; ++c)
-            if (T.admit_u[c]) ctx->unstored_units[ukeys[c]] = request_id;
     view->n_blocks = nblk; view->n_units = nu;
     view->gpu_prefix_blocks = G; view->host_prefix_blocks = H;
     view->restore_lo = lo; view->restore_hi = hi;
@@ -1449,7 +1469,9 @@ int turn_store_impl(eakv_ctx* ctx, TurnState& T, void* cuda_stream) {
             for (int64_t i = 0; i < R; ++i) T.admit_b[c * R + i] = 0;
     bool any_store = false;
     for (int64_t j = 0; j < nblk && !any_store; ++j) any_store = T.admit_b[j] != 0;
-    if (ctx->device < 0 || !any_store) return EAKV_OK;       // bookkeeping only, or nothing admitted
+    if (!any_store) return EAKV_OK;                          // nothing to write
+    if (const int inj = injected_failure(ctx)) return inj;
+    if (ctx->device < 0) return EAKV_OK;                     // bookkeeping only
     if (!ctx->cfg.write_behind)
         return eakv_store(ctx, T.block.data(), T.admit_b.data(), T.slot_b.data(), nblk, cuda_stream);
     // deferred write: on the context's stream, after what precedes it on the caller's stream

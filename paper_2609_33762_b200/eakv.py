@@ -111,7 +111,7 @@ EXPORTS = [
     "eakv_selfcheck_limits", "eakv_selfcheck_wait_probe",
     "eakv_gpu_tier_acquire", "eakv_gpu_tier_release_request", "eakv_tier_step_again",
     "eakv_declined_audit", "eakv_working_set",
-    "eakv_request_begin", "eakv_request_store", "eakv_request_release", "eakv_working_set_sizes",
+    "eakv_request_begin", "eakv_request_store", "eakv_request_release", "eakv_working_set_sizes", "eakv_selfcheck_fail_next_transfer",
 ]
 STATIC_MAX_BLOCKS = 65536
 
@@ -149,6 +149,7 @@ def lib():
     L.eakv_reuse_distances.argtypes = [vp, i64, vp, vp]
     L.eakv_capacity_curve.argtypes = [vp, i64, vp, vp, vp, i64, i32, vp, i32, vp, vp, vp, vp, vp]
     L.eakv_declined_audit.argtypes = [vp, vp, i64, i64, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), vp, vp]
+    L.eakv_selfcheck_fail_next_transfer.argtypes = [vp, i32]
     L.eakv_working_set_sizes.argtypes = [vp, i64, vp, vp, vp, i64, i32, i32, C.POINTER(i64), C.POINTER(i64), vp]
     L.eakv_working_set.argtypes = [C.POINTER(WorkingSetIn), C.POINTER(WorkingSetOut)]
     L.eakv_turn_begin.argtypes = [vp, vp, i64, vp, i64, i64, i64, vp, C.POINTER(TurnView)]
@@ -538,6 +539,9 @@ class Context:
             return None
         self._check(rc, "eakv_request_begin")
         return self._view_dict(v)
+
+    def eakv_selfcheck_fail_next_transfer(self, code):
+        self._check(lib().eakv_selfcheck_fail_next_transfer(self._h, int(code)), "eakv_selfcheck_fail_next_transfer")
 
     def eakv_request_store(self, request_id, stream=None):
         self._check(lib().eakv_request_store(self._h, int(request_id), _stream(stream)), "eakv_request_store")

@@ -294,3 +294,84 @@ def test_a_release_before_the_store_takes_back_only_units_the_request_still_owns
     ctx.eakv_request_release(5)
     assert ctx.eakv_match(k5)[1] == 6
     ctx.close()
+
+
+def test_injected_transfer_failures_withdraw_what_the_turn_registered(eakv):
+    """The paths that only a CUDA error reaches otherwise, with a failure made on the host
+    (eakv_selfcheck_fail_next_transfer): a restore that fails in begin and a store that fails in
+    end / request_store leave no key listed whose bytes were never written, close the turn, and
+    leave the context usable."""
+    b = 4
+    E = eakv
+    p = np.arange(1, 7, dtype=np.uint64)                    # 6 blocks, stored by the first turn
+    q = np.arange(101, 111, dtype=np.uint64)                # pushes them out of the 10-block GPU tier
+    grown = np.concatenate([p, np.arange(7, 10, dtype=np.uint64)])
+
+    def fresh():
+        ctx = cp_ctx(eakv, b, 10, 64)
+        for keys, agent in ((p, 0), (q, 1)):
+            ctx.eakv_turn_begin(0, len(keys) * b, keys, agent, 0)
+            ctx.eakv_turn_end()
+        assert ctx.eakv_match(grown)[:2] == (0, 6)
+        return ctx
+
+    # restore fails in eakv_turn_begin
+    ctx = fresh()
+    listed = ctx.eakv_tier_export()[0].tolist()
+    ctx.eakv_selfcheck_fail_next_transfer(E.E_CUDA)
+    with pytest.raises(E.EakvError) as ei:
+        ctx.eakv_turn_begin(0, len(grown) * b, grown, 0, 1)
+    assert ei.value.code == E.E_CUDA
+    with pytest.raises(E.EakvError):
+        ctx.eakv_turn_end()                                   # no turn is open
+    assert sorted(ctx.eakv_tier_export()[0].tolist()) == sorted(listed)      # the three new units are gone
+    assert ctx.eakv_match(grown)[:2] == (0, 6)               # and no block of it is keyed on the GPU
+    v = ctx.eakv_turn_begin(0, len(grown) * b, grown, 0, 2)  # the same turn again goes through
+    assert (v["host_prefix_blocks"], v["admit"].tolist()) == (6, [0] * 6 + [1] * 3)
+    ctx.eakv_turn_end()
+    assert ctx.eakv_match(grown)[1] == 9
+    ctx.close()
+
+    # store fails in eakv_turn_end
+    ctx = fresh()
+    ctx.eakv_turn_begin(0, len(grown) * b, grown, 0, 1)
+    ctx.eakv_selfcheck_fail_next_transfer(E.E_CUDA)
+    with pytest.raises(E.EakvError) as ei:
+        ctx.eakv_turn_end()
+    assert ei.value.code == E.E_CUDA
+    assert ctx.eakv_match(grown)[1] == 6                     # restored prefix stays, unwritten units do not
+    with pytest.raises(E.EakvError):
+        ctx.eakv_turn_abort()
+    ctx.close()
+
+    # the same for overlapping requests, with another request open meanwhile
+    ctx = cp_ctx(eakv, b, 64, 64)
+    other = np.arange(201, 205, dtype=np.uint64)
+    ctx.eakv_request_begin(9, 0, 4 * b, other, 3, 0)
+    ctx.eakv_request_begin(1, 0, 6 * b, p, 0, 0)
+    ctx.eakv_selfcheck_fail_next_transfer(E.E_CUDA)
+    with pytest.raises(E.EakvError):
+        ctx.eakv_request_store(1)
+    assert ctx.eakv_match(p)[1] == 0                          # nothing of request 1 is listed
+    with pytest.raises(E.EakvError):
+        ctx.eakv_request_release(1)                           # the failure closed it
+    ctx.eakv_request_store(9)
+    ctx.eakv_request_release(9)
+    assert ctx.eakv_match(other)[1] == 4
+    # restore fails in eakv_request_begin: the units it admitted (registered as its own) go too
+    ctx2 = cp_ctx(eakv, b, 10, 64)
+    for keys, agent in ((p, 0), (q, 1)):
+        ctx2.eakv_turn_begin(0, len(keys) * b, keys, agent, 0)
+        ctx2.eakv_turn_end()
+    ctx2.eakv_selfcheck_fail_next_transfer(E.E_NOMEM)
+    with pytest.raises(E.EakvError) as ei:
+        ctx2.eakv_request_begin(5, 0, len(grown) * b, grown, 0, 1)
+    assert ei.value.code == E.E_NOMEM
+    assert ctx2.eakv_match(grown)[:2] == (0, 6)
+    v = ctx2.eakv_request_begin(6, 0, len(grown) * b, grown, 0, 2)
+    assert v["admit"].tolist() == [0] * 6 + [1] * 3
+    ctx2.eakv_request_store(6)
+    ctx2.eakv_request_release(6)
+    assert ctx2.eakv_match(grown)[1] == 9
+    ctx2.close()
+    ctx.close()
