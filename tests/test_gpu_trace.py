@@ -456,6 +456,64 @@ def test_write_behind_orders_block_reuse_and_slot_reads():
     ctx.close()
 
 
+def test_a_failed_store_or_restore_leaves_no_stale_slot_readable():
+    """With bytes: a store that fails in eakv_turn_end (made to fail on the host) withdraws the
+    turn's units, so that the same prompt afterwards is computed and stored again rather than
+    restored from slots that were never written; a restore that fails in eakv_turn_begin
+    withdraws that turn, and the retry restores the right bytes."""
+    from paper_2609_33762_b200 import eakv
+    from paper_2609_33762_b200.harness import PagedPool
+    shape = SHAPES["tiny"]
+    nb, kh, m = 24, 64, 12
+    pool = PagedPool(shape, nb, "cuda:0")
+    ctx = eakv.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+                       block_size=shape.block_size, gpu_blocks=nb, host_blocks=kh, kv_base=pool.kv_base)
+    stream = torch.cuda.current_stream()
+    rng = np.random.default_rng(78)
+    n = m * shape.block_size
+    prompts = [torch.from_numpy(rng.integers(0, 50000, size=n, dtype=np.int32)).pin_memory() for _ in range(3)]
+
+    def begin(p, value):
+        v = ctx.eakv_turn_begin(prompts[p].data_ptr(), n, None, p, 0, stream)
+        ids = torch.as_tensor(v["gpu_block"][v["needs_fill"] != 0].astype(np.int64), device="cuda")
+        for piece in pool.pieces:
+            piece[ids] = value
+        return v
+
+    tier = ctx.tier_host_view().view(np.uint16)
+    tier[:] = 0x7777                                    # what a never-written slot would return
+    a = begin(0, 0x1111)
+    ctx.eakv_selfcheck_fail_next_transfer(eakv.E_CUDA)
+    with pytest.raises(eakv.EakvError):
+        ctx.eakv_turn_end(stream)
+    ctx.eakv_sync()
+    assert (tier[a["slot"]] == 0x7777).all()            # nothing was written ...
+    assert ctx.eakv_match(a["keys"])[1] == 0            # ... and nothing is listed
+    for p, value in ((1, 0x2222), (2, 0x3333)):         # two other prompts take prompt 0 off the GPU
+        begin(p, value)
+        ctx.eakv_turn_end(stream)
+    a2 = begin(0, 0x4444)                               # computed again (not restored), stored now
+    assert a2["restore_hi"] == a2["restore_lo"] and a2["n_fill"] == m and a2["n_stored_blocks"] == m
+    ctx.eakv_turn_end(stream)
+    begin(1, 0x5555)                                    # (prompt 1 is restored: nothing to fill)
+    ctx.eakv_turn_end(stream)
+    begin(2, 0x6666)
+    ctx.eakv_turn_end(stream)
+    # prompt 0 is off the GPU again: its restore is made to fail once, then retried
+    ctx.eakv_selfcheck_fail_next_transfer(eakv.E_CUDA)
+    with pytest.raises(eakv.EakvError):
+        ctx.eakv_turn_begin(prompts[0].data_ptr(), n, None, 0, 0, stream)
+    assert ctx.eakv_match(a["keys"])[:2] == (0, m)      # still only on the host
+    a3 = begin(0, 0x0BAD)
+    assert a3["restore_hi"] - a3["restore_lo"] == m and a3["n_fill"] == 0
+    ctx.eakv_turn_end(stream)
+    ctx.eakv_sync()
+    ids = torch.as_tensor(a3["gpu_block"].astype(np.int64), device="cuda")
+    for piece in pool.pieces:
+        assert bool((piece[ids].view(torch.int16) == 0x4444).all())
+    ctx.close()
+
+
 def test_write_behind_orders_a_direct_load_of_pending_slots():
     """eakv_load of slots that a deferred write is still filling, into GPU blocks the write does
     not touch: only the slot marks can make it wait, and it must return the written bytes."""
