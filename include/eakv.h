@@ -427,7 +427,9 @@ int eakv_turn_abort(eakv_ctx* ctx);
  * second one read that block only after the first one's fill (stream order or an event).
  * eakv_request_release: the request finished or is suspended: its blocks become evictable
  * (eakv_gpu_tier_release_request) and its tail block is freed.  Released before its store -- the
- * engine never produced the KV -- it is taken back like an aborted turn.
+ * engine never produced the KV -- it is taken back like an aborted turn; a block it was told to fill
+ * that another open request shares stays keyed for that request, which was told the block is
+ * resident: the engine must then produce it on that request's behalf (or release that request too).
  * Errors: EAKV_E_INVAL for a request_id that is already open (begin) or not open (store, release),
  * for a second store, and while a single turn (eakv_turn_begin) is open; failures after the
  * bookkeeping are handled as in eakv_turn_begin / eakv_turn_end and close the request. */
