@@ -478,7 +478,7 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
         return EAKV_E_INVAL;
     if (cfg->block_size > kHashMaxBlockSize) return EAKV_E_INVAL;
     const int64_t chunk_blocks = cfg->chunk_blocks > 0 ? cfg->chunk_blocks : 1;
-    if (cfg->gpu_blocks > INT32_MAX || cfg->host_blocks * chunk_blocks > INT32_MAX) return EAKV_E_INVAL;
+    if (cfg->gpu_blocks > INT32_MAX || cfg->host_blocks > INT32_MAX / chunk_blocks) return EAKV_E_INVAL;
     if (cfg->policy < 0 || cfg->policy > 2 || cfg->link_strategy < 0 || cfg->link_strategy > 2 ||
         cfg->tier_location < 0 || cfg->tier_location > 1 || cfg->copy_path < 0 || cfg->copy_path > 1 ||
         cfg->gpu_free_order < 0 || cfg->gpu_free_order > 1)

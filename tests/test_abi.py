@@ -81,6 +81,13 @@ def test_create_rejects_bad_config_before_touching_cuda(lib):
     assert lib.eakv_create(C.byref(cfg), C.byref(h)) == eakv.E_INVAL      # empty shape
     assert lib.eakv_create(None, C.byref(h)) == eakv.E_INVAL
     assert not h.value
+    # sizes beyond 32-bit ids are refused, also where host_blocks * chunk_blocks would wrap around
+    for hb, cb in ((1 << 31, 1), (1 << 62, 4), ((1 << 31) // 64 + 1, 64)):
+        cfg = eakv.Config()
+        lib.eakv_config_init(C.byref(cfg))
+        cfg.num_layers, cfg.kv_heads, cfg.head_dim, cfg.block_size = 1, 1, 8, 16
+        cfg.gpu_blocks, cfg.host_blocks, cfg.chunk_blocks, cfg.control_plane_only = 4, hb, cb, 1
+        assert lib.eakv_create(C.byref(cfg), C.byref(h)) == eakv.E_INVAL and not h.value
 
 
 def test_no_cpu_fallback_without_a_gpu(lib):
