@@ -1235,12 +1235,6 @@ int eakv_load_layers(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* bl
 // ------------------------------------------------------------------------------------------
 namespace {
 
-// Take back what an open turn registered but will never produce.  host_units: the tier units the
-// turn admitted leave the host index (their slots were never written).  gpu_mode 1: every GPU
-// block the turn newly keyed leaves the GPU index (nothing was restored or computed); 2: only
-// those the engine was to fill (the restored ones hold their bytes).  A block another running
-// request shares stays.  Promotions and evictions the turn caused stand.  Lets the turn's GPU
-// blocks go (pins, tail block).
 // Which of the units the turn admitted are still its own to write (owned_u), once per turn.  A
 // single turn owns all of them: nothing comes between its begin and its end.  A request owns those
 // that no other request's lookup has evicted since its own (the reference model saw this request's
@@ -1264,6 +1258,13 @@ void claim_units(eakv_ctx* ctx, TurnState& T) {
     }
 }
 
+// Take back what an open turn registered but will never produce.  host_units: the tier units the
+// turn admitted and still owns (claim_units) leave the host index (their slots were never written).
+// gpu_mode 1: every GPU
+// block the turn newly keyed leaves the GPU index (nothing was restored or computed); 2: only
+// those the engine was to fill (the restored ones hold their bytes).  A block another running
+// request shares stays.  Promotions and evictions the turn caused stand.  Lets the turn's GPU
+// blocks go (pins, tail block).
 void withdraw_turn(eakv_ctx* ctx, TurnState& T, bool host_units, int gpu_mode) {
     claim_units(ctx, T);
     if (host_units) {
