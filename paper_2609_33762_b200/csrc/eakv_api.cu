@@ -139,6 +139,19 @@ struct eakv_ctx {
 
 namespace {
 
+// Can kernels of this process read the address?  Device, managed and registered (pinned) host
+// memory: yes.  Ordinary host memory: no -- a kernel given such a pointer takes an illegal-address
+// fault that costs the whole CUDA context, so the calls that hand a caller's pointer to a kernel
+// ask first and refuse with EAKV_E_INVAL.
+bool device_readable(const void* p) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeHost || at.type == cudaMemoryTypeManaged;
+}
+
 int cuda_fail(eakv_ctx* c, cudaError_t e, const char* what) {
     if (c) {
         c->cuda_err = std::string(what) + ": " + cudaGetErrorString(e);
@@ -731,6 +744,7 @@ int eakv_hash_blocks(eakv_ctx* ctx, const int32_t* tokens_dev, int64_t n_tokens,
     if (!tokens_dev || !hashes_dev) return EAKV_E_INVAL;
     if (((uintptr_t)tokens_dev & 3) || ((uintptr_t)hashes_dev & 7)) return EAKV_E_INVAL;
     DeviceGuard g(ctx->device);
+    if (!device_readable(tokens_dev) || !device_readable(hashes_dev)) return EAKV_E_INVAL;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const bool generic = hash_thread_per_block(b);
     const bool vec = (b % 4) == 0 && (((uintptr_t)tokens_dev & 15) == 0);
@@ -795,6 +809,7 @@ int eakv_hash_blocks_batched(eakv_ctx* ctx, const int32_t* tokens_dev,
     if (!tokens_dev || !hashes_dev) return EAKV_E_INVAL;
     if (((uintptr_t)tokens_dev & 3) || ((uintptr_t)hashes_dev & 7)) return EAKV_E_INVAL;
     DeviceGuard g(ctx->device);
+    if (!device_readable(tokens_dev) || !device_readable(hashes_dev)) return EAKV_E_INVAL;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const bool generic = hash_thread_per_block(b);
     bool vec = (b % 4) == 0 && (((uintptr_t)tokens_dev & 15) == 0);
@@ -1310,6 +1325,7 @@ int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32
     // a context without a device cannot hash: the caller supplies every key
     if (bookkeeping_only && n_known < nblk) return EAKV_E_INVAL;
     if (nblk > n_known && !tokens) return EAKV_E_INVAL;
+    if (nblk > n_known && !bookkeeping_only && !device_readable(tokens)) return EAKV_E_INVAL;   // (ordinary host memory)
     // everything that can be refused without a CUDA error is refused here, before either tier changes
     if (nu > ctx->host_tier->capacity()) return EAKV_E_CAPACITY;
     if (!as_request && nblk + (need_tail ? 1 : 0) + ctx->gpu_unkeyed > ctx->gpu_tier->capacity())

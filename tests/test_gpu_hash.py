@@ -240,3 +240,33 @@ def test_hash_self_check_reports_range_and_recovers():
         ctx.eakv_selfcheck_limits()
         assert gpu_keys(ctx, toks) == oh.hash_blocks(toks.tolist(), b)
         ctx.close()
+
+
+def test_ordinary_host_memory_is_refused_not_dereferenced():
+    """A token or key pointer into ordinary (pageable) host memory would cost the CUDA context if a
+    kernel read it: the calls ask the runtime what the address is and return EAKV_E_INVAL without
+    launching.  Pinned host memory and device memory go through, with the oracle's keys."""
+    from paper_2609_33762_b200 import eakv
+    b = 16
+    ctx = hash_ctx(b)
+    toks = np.random.default_rng(13).integers(0, 151936, size=40 * b, dtype=np.int32)
+    want = oh.hash_blocks(toks.tolist(), b)
+    out = torch.zeros(40, dtype=torch.int64, device="cuda")
+    pageable_out = np.zeros(40, dtype=np.uint64)
+    dev = torch.from_numpy(toks).cuda()
+    for tok_ptr, out_ptr in ((toks.ctypes.data, out.data_ptr()), (dev.data_ptr(), pageable_out.ctypes.data)):
+        with pytest.raises(eakv.EakvError) as ei:
+            ctx.eakv_hash_blocks(tok_ptr, len(toks), ctx.eakv_hash_seed(), out_ptr)
+        assert ei.value.code == eakv.E_INVAL
+    with pytest.raises(eakv.EakvError) as ei:
+        ctx.eakv_turn_begin(toks.ctypes.data, len(toks), None, 0, 0)
+    assert ei.value.code == eakv.E_INVAL
+    ctx.eakv_sync()                                           # nothing was launched, nothing is wrong
+    pinned = torch.from_numpy(toks).pin_memory()
+    pinned_out = torch.zeros(40, dtype=torch.int64).pin_memory()
+    ctx.eakv_hash_blocks(pinned.data_ptr(), len(toks), ctx.eakv_hash_seed(), pinned_out.data_ptr())
+    ctx.eakv_sync()
+    torch.cuda.synchronize()
+    assert [int(x) for x in pinned_out.numpy().view(np.uint64)] == [int(k) for k in want]
+    assert gpu_keys(ctx, toks) == want
+    ctx.close()
