@@ -574,6 +574,13 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
     } while (0)
 
     if (!cfg->control_plane_only) {
+        // the pool and an adopted tier are read and written by kernels: refuse addresses they cannot reach
+        bool reachable = !cfg->tier_memory || device_readable(cfg->tier_memory);
+        for (int q = 0; q < pieces && reachable; ++q) reachable = device_readable(cfg->kv_base[q]);
+        if (!reachable) {
+            free_all(ctx);
+            return EAKV_E_INVAL;
+        }
         CUC(cudaGetDevice(&ctx->device));
         CUC(cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device));
         CUC(hash_kernels_init());

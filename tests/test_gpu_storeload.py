@@ -224,6 +224,13 @@ def test_bad_shapes_rejected_at_create():
         with pytest.raises(e.EakvError) as ei:
             e.Context(**{**base, **patch})
         assert ei.value.code == e.E_INVAL
+    # a pool (or an adopted tier) in ordinary host memory: kernels cannot reach it
+    host = np.zeros(4096, dtype=np.uint8)
+    hp = (host.ctypes.data + 15) // 16 * 16
+    for patch in (dict(kv_base=[hp, hp]), dict(tier_memory=hp)):
+        with pytest.raises(e.EakvError) as ei:
+            e.Context(**{**base, **patch})
+        assert ei.value.code == e.E_INVAL
     # Copy engine alone: the pitch between piece arrays (2 GiB here: 131,072 blocks of 16 KiB) is
     # above what a strided copy-engine transfer accepts, so the configuration is refused at create
     # rather than failing on every later call.  The pool addresses are only compared, never
