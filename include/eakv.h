@@ -16,8 +16,9 @@
  *     before the call returns.  "device" pointers must be dereferenceable by kernels of
  *     the context's GPU (device memory, or pinned host memory under unified addressing).
  *     The calls that pass a caller's token or key pointer to a kernel (eakv_hash_blocks,
- *     eakv_hash_blocks_batched, eakv_turn_begin, eakv_request_begin) ask the runtime what the
- *     address is and return EAKV_E_INVAL for ordinary host memory instead of launching.
+ *     eakv_hash_blocks_batched, eakv_hash_blocks_static, eakv_turn_begin, eakv_request_begin,
+ *     the capacity-model entry points) and eakv_create (pool, adopted tier) ask the runtime what
+ *     the address is and return EAKV_E_INVAL for ordinary host memory instead of launching.
  *   - The caller owns every buffer it passes.  The context owns its tier memory (unless
  *     adopted, see eakv_config.tier_memory), staging buffers, argument rings and side
  *     streams.

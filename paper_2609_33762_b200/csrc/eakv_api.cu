@@ -126,11 +126,10 @@ struct eakv_ctx {
     int64_t turn_keys_cap = 0;
     TurnState turn;                            // the one open turn of eakv_turn_begin / eakv_turn_end
     std::unordered_map<int64_t, TurnState> requests;   // open turns of running requests (eakv_request_*)
-    // tier units an open turn admitted whose store has not been enqueued yet: listed in the host
-    // index (so nobody stores them twice) but not restorable by another request
     // units an open request admitted and has not written yet -> that request.  An eviction takes a
     // unit out of here: its slot belongs to someone else from then on and is never written by the
-    // request that lost it.
+    // request that lost it.  While listed here a unit is in the host index (nobody stores it twice)
+    // but no other request can restore it.
     std::unordered_map<uint64_t, int64_t> unstored_units;
     int fail_next_transfer = 0;        // self-test: the next restore / store step returns this code instead
 
@@ -138,19 +137,6 @@ struct eakv_ctx {
 };
 
 namespace {
-
-// Can kernels of this process read the address?  Device, managed and registered (pinned) host
-// memory: yes.  Ordinary host memory: no -- a kernel given such a pointer takes an illegal-address
-// fault that costs the whole CUDA context, so the calls that hand a caller's pointer to a kernel
-// ask first and refuse with EAKV_E_INVAL.
-bool device_readable(const void* p) {
-    cudaPointerAttributes at;
-    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) {
-        cudaGetLastError();
-        return false;
-    }
-    return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeHost || at.type == cudaMemoryTypeManaged;
-}
 
 int cuda_fail(eakv_ctx* c, cudaError_t e, const char* what) {
     if (c) {

@@ -139,4 +139,17 @@ cudaError_t launch_wait_probe(int* error_flag, cudaStream_t stream);
 cudaError_t copy_kernels_init();
 int copy_vector_ctas_per_sm();
 
+// Can kernels of this process read the address?  Device, managed and registered (pinned) host
+// memory: yes.  Ordinary host memory: no -- a kernel given such a pointer takes an illegal-address
+// fault that costs the whole CUDA context, so the calls that hand a caller's pointer to a kernel
+// ask first and refuse with EAKV_E_INVAL.
+inline bool device_readable(const void* p) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeHost || at.type == cudaMemoryTypeManaged;
+}
+
 }  // namespace eakv

@@ -978,6 +978,7 @@ extern "C" int eakv_hash_blocks_static(const int32_t* tokens_dev, int64_t n_toke
     if (nblk == 0) return EAKV_OK;
     if (!tokens_dev || !hashes_dev) return EAKV_E_INVAL;
     if (((uintptr_t)tokens_dev & 3) || ((uintptr_t)hashes_dev & 7)) return EAKV_E_INVAL;
+    if (!device_readable(tokens_dev) || !device_readable(hashes_dev)) return EAKV_E_INVAL;   // (a query, no allocation)
 
     unsigned char* scratch = static_scratch(nullptr);
     if (!scratch) return EAKV_E_CUDA;

@@ -23,6 +23,7 @@
 #include <vector>
 
 #include "../../include/eakv.h"
+#include "eakv_internal.h"
 
 namespace eakv {
 
@@ -493,6 +494,7 @@ extern "C" int eakv_reuse_distances(const uint64_t* keys_dev, int64_t n_refs, in
     if (n_refs < 0 || n_refs > 0x7ffffff0LL) return EAKV_E_INVAL;
     if (n_refs == 0) return EAKV_OK;
     if (!keys_dev || !dist_dev) return EAKV_E_INVAL;
+    if (!device_readable(keys_dev) || !device_readable(dist_dev)) return EAKV_E_INVAL;
     return reuse_distances_impl(keys_dev, n_refs, dist_dev, nullptr, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -504,6 +506,9 @@ extern "C" int eakv_declined_audit(const uint64_t* keys_dev, const uint8_t* decl
     *declined_out = *meets_out = *never_out = 0;
     if (n_refs == 0) return EAKV_OK;
     if (!keys_dev || !declined_dev) return EAKV_E_INVAL;
+    if (!device_readable(keys_dev) || !device_readable(declined_dev) ||
+        (next_dist_dev && !device_readable(next_dist_dev)))
+        return EAKV_E_INVAL;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     int rc = EAKV_OK;
     int64_t* dist = nullptr;
@@ -571,6 +576,7 @@ extern "C" int eakv_capacity_curve(const int64_t* dist_dev, int64_t n_refs,
         return EAKV_E_INVAL;
     if (n_requests > 0 && (!req_tokens_host || !req_gpu_prefix_host)) return EAKV_E_INVAL;
     if (n_refs > 0 && !dist_dev) return EAKV_E_INVAL;
+    if (n_refs > 0 && !device_readable(dist_dev)) return EAKV_E_INVAL;
     if (req_offsets_host[0] != 0 || req_offsets_host[n_requests] != n_refs) return EAKV_E_INVAL;
     for (int64_t r = 0; r < n_requests; ++r)
         if (req_offsets_host[r + 1] < req_offsets_host[r]) return EAKV_E_INVAL;
@@ -633,6 +639,7 @@ extern "C" int eakv_working_set_sizes(const int64_t* dist_dev, int64_t n_refs, c
     if (n_refs < 0 || n_requests < 0 || block_size <= 0 || percent < 0 || !full_out || !within_out)
         return EAKV_E_INVAL;
     if (n_refs > 0 && !dist_dev) return EAKV_E_INVAL;
+    if (n_refs > 0 && !device_readable(dist_dev)) return EAKV_E_INVAL;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     int rc = EAKV_OK;
     long long* d_max = nullptr;
