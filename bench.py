@@ -475,9 +475,46 @@ def control_plane_rate(eakv, pool, shape, device, requests=400, blocks=4096):
         refs += blocks
     st = ctx.eakv_get_stats()
     ctx.close()
-    return {"match_refs_per_s": refs / t_match, "tier_step_refs_per_s": refs / t_step,
-            "references": refs, "hits": st["hits"], "evicted": st["evicted"],
-            "note": "through the Python binding, one thread"}
+    out = {"match_refs_per_s": refs / t_match, "tier_step_refs_per_s": refs / t_step,
+           "references": refs, "hits": st["hits"], "evicted": st["evicted"],
+           "note": "through the Python binding, one thread"}
+    out["turn"] = turn_overhead(eakv, device)
+    return out
+
+
+def turn_overhead(eakv, device, prompt_blocks=3072, appended_blocks=192, reps=20):
+    """Wall time of one whole turn through eakv_turn_begin + eakv_turn_end when nothing has to move:
+    a 48k-token prompt of which the last 3k tokens are new since the previous turn (their keys are
+    hashed on the GPU, the others are passed in), every block resident on the GPU, the write
+    declined.  What is left is the library's own cost per turn: hashing, the lookups and both
+    tiers' bookkeeping over 3,072 blocks.  (A KV shape of 512 bytes per block keeps the pool small;
+    the control plane does not depend on it.)"""
+    import torch
+    b, nb = 16, 2 * prompt_blocks
+    piece = b * 1 * 8 * 2
+    pool = [torch.zeros(nb * piece // 2, dtype=torch.int16, device=device) for _ in range(2)]
+    ctx = eakv.Context(num_layers=1, kv_heads=1, head_dim=8, block_size=b, gpu_blocks=nb,
+                       host_blocks=2 * prompt_blocks, kv_base=[t.data_ptr() for t in pool],
+                       tier_location=eakv.TIER_DEVICE, policy=eakv.POLICY_FILTER_FIXED, kappa_blocks=0)
+    stream = torch.cuda.current_stream(device)
+    tok = torch.randint(0, 150000, (prompt_blocks * b,), dtype=torch.int32).pin_memory()
+    n_prev = (prompt_blocks - appended_blocks) * b
+    v = ctx.eakv_turn_begin(tok.data_ptr(), n_prev, None, 0, 0, stream)
+    ctx.eakv_turn_end(stream)
+    known = v["keys"]
+    times = []
+    for i in range(reps + 3):
+        t0 = time.perf_counter()
+        v = ctx.eakv_turn_begin(tok.data_ptr(), prompt_blocks * b, known, 0, i + 1, stream)
+        ctx.eakv_turn_end(stream)
+        times.append(time.perf_counter() - t0)
+    ctx.eakv_sync()
+    assert v["gpu_prefix_blocks"] == prompt_blocks and v["n_stored_blocks"] == 0
+    ctx.close()
+    return {"wall_us_median": float(np.median(times[3:])) * 1e6, "prompt_tokens": prompt_blocks * b,
+            "appended_tokens": appended_blocks * b,
+            "note": "eakv_turn_begin + eakv_turn_end, prompt resident on the GPU, write declined: "
+                    "hash of the appended tokens + lookups + bookkeeping of 3,072 blocks"}
 
 
 def layered_load_probe(torch, arm, tables, shape, layers_per_group=12):
