@@ -1373,23 +1373,25 @@ int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32
     T.stored = false;
     T.claimed = false;
     T.owned_u.clear();
-    // lookups (they change nothing), then the GPU side -- a running request whose blocks do not fit
-    // beside the others is refused here with both tiers untouched -- then the host tier
-    int64_t G = 0, G_unused = 0, Hu = 0;
-    int rc = eakv_match(ctx, keys, nblk, &G, nullptr, nullptr, nullptr);
-    if (rc != EAKV_OK) return rc;
-    rc = eakv_match(ctx, ukeys, nu, &G_unused, &Hu, nullptr, T.host_slots.data());
-    if (rc != EAKV_OK) return rc;
-    // a unit that another open request admitted but has not stored yet cannot be restored
-    if (!ctx->unstored_units.empty())
-        for (int64_t c = 0; c < Hu; ++c)
-            if (ctx->unstored_units.count(ukeys[c])) { Hu = c; break; }
+    // The GPU side first -- a running request whose blocks do not fit beside the others is refused
+    // here with both tiers untouched -- then the host tier.  Each walk also answers the lookup: up to
+    // its first miss a walk only promotes, so the leading run of keys it found resident is the
+    // longest cached prefix as it stood before the turn (G; H with the slots of those units).
     int32_t tail = -1;
+    int rc;
     if (as_request)
         rc = eakv_gpu_tier_acquire(ctx, request_id, keys, nblk, need_tail, T.resident.data(), T.block.data(), &tail);
     else
         rc = eakv_gpu_tier_step(ctx, keys, nblk, need_tail, T.resident.data(), T.block.data(), &tail);
     if (rc != EAKV_OK) return rc;
+    int64_t G = 0;
+    while (G < nblk && T.resident[G]) ++G;
+    // a unit that another open request admitted but has not stored yet cannot be restored (read
+    // before this turn's own admissions join that set)
+    int64_t pending_from = nu;
+    if (!ctx->unstored_units.empty())
+        for (int64_t c = 0; c < nu; ++c)
+            if (ctx->unstored_units.count(ukeys[c])) { pending_from = c; break; }
     T.tail = tail;
     T.open = true;
     int64_t n_ev = nu;
@@ -1400,6 +1402,8 @@ int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32
         withdraw_turn(ctx, T, false, 1);
         return rc;
     }
+    int64_t Hu = std::min<int64_t>(info.host_prefix_blocks, pending_from);
+    for (int64_t c = 0; c < Hu; ++c) T.host_slots[c] = T.slot_u[c];
     // the units this request admitted are its own to write until another lookup evicts them (before
     // anything below can fail: a withdrawal takes back what is registered here)
     if (as_request)
