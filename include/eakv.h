@@ -456,6 +456,21 @@ int eakv_load_layers(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* bl
                      int64_t n_blocks, int32_t layers_per_group, void* const* events,
                      int32_t n_events, void* cuda_stream);
 
+/* Layer-pipelined host write (Section 3.1: write costs are part of what a response waits for
+ * beyond its prefill; an engine that produces KV layer by layer can let the write of the first
+ * layers run under the compute of the later ones).  Same result as eakv_store, but the 2L pieces
+ * of every admitted block are moved in ascending groups of layers_per_group layers, and before
+ * group g is read cuda_stream waits for ready_events[g].
+ *   ready_events  host array of n_events cudaEvent_t handles (as void*) or NULL entries (no wait);
+ *                 n_events must equal ceil(num_layers / layers_per_group).  The producer must
+ *                 have recorded event g (cudaEventRecord already called, on its own stream,
+ *                 behind the work that completes those layers of the blocks in block_table)
+ *                 before this call: a wait on an event that was never recorded does not wait.
+ * Errors as eakv_store, plus EAKV_E_INVAL for a wrong n_events. */
+int eakv_store_layers(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_mask,
+                      const int32_t* host_slots, int64_t n_blocks, int32_t layers_per_group,
+                      void* const* ready_events, int32_t n_events, void* cuda_stream);
+
 /* Reuse (stack) distances of a reference stream (Section 3.2, Eq. 4): dist[i] = number of
  * distinct other keys referenced strictly between reference i and the previous reference to
  * the same key, or -1 on a first reference.  Under a fully associative LRU tier of K chunks

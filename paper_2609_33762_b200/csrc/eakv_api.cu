@@ -1238,6 +1238,48 @@ int eakv_load_layers(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* bl
     return EAKV_OK;
 }
 
+int eakv_store_layers(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_mask,
+                      const int32_t* host_slots, int64_t n_blocks, int32_t layers_per_group,
+                      void* const* ready_events, int32_t n_events, void* cuda_stream) {
+    if (!ctx || n_blocks < 0 || ctx->device < 0 || layers_per_group <= 0) return EAKV_E_INVAL;
+    const int L = ctx->cfg.num_layers;
+    const int groups = (L + layers_per_group - 1) / layers_per_group;
+    if (n_events != groups || (groups > 0 && !ready_events)) return EAKV_E_INVAL;
+    if (n_blocks > 0 && (!block_table || !host_slots)) return EAKV_E_INVAL;
+    next_epoch(ctx);
+    std::vector<int2>& ent = ctx->scratch_entries;
+    ent.clear();
+    for (int64_t j = 0; j < n_blocks; ++j) {
+        if (admit_mask && !admit_mask[j]) continue;
+        const int32_t blk = block_table[j], slot = host_slots[j];
+        if (blk < 0 || blk >= ctx->cfg.gpu_blocks || slot < 0 || slot >= ctx->tier_slots)
+            return EAKV_E_RANGE;
+        if (ctx->slot_stamp[slot] == ctx->epoch) return EAKV_E_INVAL;
+        ctx->slot_stamp[slot] = ctx->epoch;
+        ent.push_back(make_int2(blk, slot));
+    }
+    const int64_t m = (int64_t)ent.size();
+    DeviceGuard g(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (m > 0) {
+        const int rcw = wait_write_behind(ctx, stream);
+        if (rcw != EAKV_OK) return rcw;
+    }
+    for (int grp = 0; grp < groups; ++grp) {
+        const int l0 = grp * layers_per_group;
+        const int l1 = std::min(L, l0 + layers_per_group);
+        // the group's layers are read only after the producer has said they are complete
+        if (ready_events[grp]) CU(cudaStreamWaitEvent(stream, static_cast<cudaEvent_t>(ready_events[grp]), 0));
+        if (m > 0) {
+            int rc = move_blocks(ctx, ent, true, stream, 2 * l0, 2 * (l1 - l0));
+            if (rc != EAKV_OK) return rc;
+        }
+    }
+    ctx->stats.blocks_stored += m;
+    ctx->stats.bytes_stored += m * ctx->block_bytes;
+    return EAKV_OK;
+}
+
 // ------------------------------------------------------------------------------------------
 // turns: one at a time (eakv_turn_*), or several running requests at once (eakv_request_*)
 // ------------------------------------------------------------------------------------------

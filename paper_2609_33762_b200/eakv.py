@@ -111,7 +111,7 @@ EXPORTS = [
     "eakv_selfcheck_limits", "eakv_selfcheck_wait_probe",
     "eakv_gpu_tier_acquire", "eakv_gpu_tier_release_request", "eakv_tier_step_again",
     "eakv_declined_audit", "eakv_working_set",
-    "eakv_request_begin", "eakv_request_store", "eakv_request_release", "eakv_working_set_sizes", "eakv_selfcheck_fail_next_transfer",
+    "eakv_request_begin", "eakv_request_store", "eakv_request_release", "eakv_working_set_sizes", "eakv_selfcheck_fail_next_transfer", "eakv_store_layers",
 ]
 STATIC_MAX_BLOCKS = 65536
 
@@ -150,6 +150,7 @@ def lib():
     L.eakv_capacity_curve.argtypes = [vp, i64, vp, vp, vp, i64, i32, vp, i32, vp, vp, vp, vp, vp]
     L.eakv_declined_audit.argtypes = [vp, vp, i64, i64, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), vp, vp]
     L.eakv_selfcheck_fail_next_transfer.argtypes = [vp, i32]
+    L.eakv_store_layers.argtypes = [vp, vp, vp, vp, i64, i32, vp, i32, vp]
     L.eakv_working_set_sizes.argtypes = [vp, i64, vp, vp, vp, i64, i32, i32, C.POINTER(i64), C.POINTER(i64), vp]
     L.eakv_working_set.argtypes = [C.POINTER(WorkingSetIn), C.POINTER(WorkingSetOut)]
     L.eakv_turn_begin.argtypes = [vp, vp, i64, vp, i64, i64, i64, vp, C.POINTER(TurnView)]
@@ -509,6 +510,19 @@ class Context:
         rc = lib().eakv_load_layers(self._h, hsp, btp, len(bt), int(layers_per_group),
                                     C.cast(ev, C.c_void_p), len(events), _stream(stream))
         self._check(rc, "eakv_load_layers")
+
+    def eakv_store_layers(self, block_table, admit_mask, host_slots, layers_per_group, ready_events, stream=None):
+        """``ready_events``: per layer group a cudaEvent_t handle as integer (already recorded by the
+        producer) or None for no wait."""
+        bt, btp = _np(block_table, np.int32)
+        hs, hsp = _np(host_slots, np.int32)
+        amp = None
+        if admit_mask is not None:
+            am, amp = _np(admit_mask, np.uint8)
+        ev = (C.c_void_p * max(len(ready_events), 1))(*[None if e is None else int(e) for e in ready_events])
+        rc = lib().eakv_store_layers(self._h, btp, amp, hsp, len(bt), int(layers_per_group),
+                                     C.cast(ev, C.c_void_p), len(ready_events), _stream(stream))
+        self._check(rc, "eakv_store_layers")
 
     def eakv_turn_begin(self, tokens_ptr, n_tokens, known_keys, agent_id, now_ms, stream=None):
         """First half of a turn; returns a dict of the view's scalars and (copied) arrays."""

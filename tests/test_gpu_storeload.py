@@ -244,6 +244,93 @@ def test_bad_shapes_rejected_at_create():
     assert ei.value.code == e.E_INVAL
 
 
+@pytest.mark.parametrize("kw", [
+    dict(tier_location=1, copy_path=1), dict(tier_location=1, copy_path=0),
+    dict(tier_location=0, link_strategy=0),
+    dict(tier_location=0, link_strategy=1, min_staged_run_bytes=-1),
+    dict(tier_location=0, link_strategy=1),
+    dict(tier_location=0, link_strategy=2, contiguous_pool=True),
+], ids=["hbm-bulk", "hbm-vector", "host-zero-copy", "host-staged", "host-default", "host-copy-engine"])
+@pytest.mark.parametrize("name,group", [("qwen", 12), ("qwen", 5), ("tiny", 1), ("ragged", 2), ("qwen_tp8", 5),
+                                        ("small", 1)])
+def test_layer_pipelined_store(name, group, kw):
+    """eakv_store_layers writes the same bytes as eakv_store, in layer groups (masked entries
+    untouched, errors as for the plain store)."""
+    e = eakv()
+    shape = SHAPE_CASES[name]
+    nb, kh = (64, 48) if shape.block_bytes <= (1 << 21) else (24, 20)
+    rig = Rig(shape, nb, kh, seed=22, staging_bytes=3 * shape.block_bytes, **kw)
+    rng = rig.rng
+    groups = -(-shape.num_layers // group)
+    none = [None] * groups
+    m = min(nb, kh) - 5
+    table = rng.permutation(nb)[:m].astype(np.int32)
+    slots = rng.permutation(kh)[:m].astype(np.int32)
+    admit = (rng.random(m) < 0.7).astype(np.uint8)
+    stream = torch.cuda.Stream()
+    rig.ctx.eakv_store_layers(table, admit, slots, group, none, stream)
+    osl.store(rig.pool_np, rig.tier_np, table, admit, slots)
+    stream.synchronize()
+    rig.check()
+    # contiguous slots without a mask, and an empty call
+    rig.ctx.eakv_store_layers(np.arange(8, dtype=np.int32)[::-1].copy(), None, np.arange(8, dtype=np.int32),
+                              group, none, stream)
+    osl.store(rig.pool_np, rig.tier_np, list(range(8))[::-1], [1] * 8, list(range(8)))
+    rig.ctx.eakv_store_layers(np.zeros(0, np.int32), None, np.zeros(0, np.int32), group, none, stream)
+    stream.synchronize()
+    rig.check()
+    assert rig.ctx.eakv_get_stats()["blocks_stored"] == int(admit.sum()) + 8
+    for bad, code in (((table, admit, slots, group, none + [None]), e.E_INVAL),                     # events
+                      ((np.array([0, 1], np.int32), None, np.array([3, 3], np.int32), group, none), e.E_INVAL),
+                      ((np.array([nb], np.int32), None, np.array([0], np.int32), group, none), e.E_RANGE)):
+        with pytest.raises(e.EakvError) as ei:
+            rig.ctx.eakv_store_layers(*bad, stream)
+        assert ei.value.code == code
+    rig.check()
+    rig.close()
+
+
+@pytest.mark.parametrize("kw", [
+    dict(tier_location=1, copy_path=1),
+    dict(tier_location=0, link_strategy=0),
+    dict(tier_location=0, link_strategy=1, min_staged_run_bytes=-1),
+    dict(tier_location=0, link_strategy=2, contiguous_pool=True),
+], ids=["hbm-bulk", "host-zero-copy", "host-staged", "host-copy-engine"])
+@pytest.mark.parametrize("name,group", [("qwen", 12), ("qwen_tp8", 16)])
+def test_layer_pipelined_store_waits_for_each_group(name, group, kw):
+    """The contract of eakv_store_layers: group g is read only after ready_events[g].  A producer
+    stream fills the layers group by group, each fill held back by a delay and followed by its
+    event; the store is enqueued on another stream right away.  The tier must hold what the
+    producer wrote, not what the blocks held when the store was enqueued."""
+    shape = SHAPE_CASES[name]
+    nb, kh, m = 64, 48, 40
+    rig = Rig(shape, nb, kh, seed=34, staging_bytes=4 * shape.block_bytes, **kw)
+    rng = rig.rng
+    groups = -(-shape.num_layers // group)
+    table = rng.permutation(nb)[:m].astype(np.int32)
+    slots = rng.permutation(kh)[:m].astype(np.int32)
+    ids = torch.as_tensor(table.astype(np.int64), device="cuda")
+    fresh = [torch.from_numpy(rng.integers(0, 256, size=(m, shape.piece_bytes), dtype=np.uint8)).cuda()
+             for _ in range(shape.pieces_per_block)]
+    producer, io = torch.cuda.Stream(), torch.cuda.Stream()
+    events = [torch.cuda.Event() for _ in range(groups)]
+    torch.cuda.synchronize()
+    with torch.cuda.stream(producer):
+        for g in range(groups):
+            torch.cuda._sleep(20_000_000)                       # ~10 ms: the store is enqueued long before
+            for q in range(2 * g * group, min(2 * (g + 1) * group, shape.pieces_per_block)):
+                rig.pool_dev[q].view(torch.uint8).view(nb, -1)[ids] = fresh[q]
+            events[g].record(producer)
+    rig.ctx.eakv_store_layers(table, None, slots, group, [ev.cuda_event for ev in events], io)
+    for q in range(shape.pieces_per_block):
+        rig.pool_np[q][table] = fresh[q].cpu().numpy()
+    osl.store(rig.pool_np, rig.tier_np, table, [1] * m, slots)
+    io.synchronize()
+    producer.synchronize()
+    rig.check()
+    rig.close()
+
+
 def test_a_tier_that_cannot_be_allocated_is_refused_cleanly():
     """A 3 TiB tier in HBM (2 M slots of 1.5 MiB): the one device allocation of that size is refused
     by the runtime at once, create returns EAKV_E_NOMEM after freeing what it had, and the device
@@ -363,6 +450,93 @@ def test_layer_group_event_means_the_group_has_landed(name, group, contiguous_sl
         for i, q in enumerate(range(q0, q1)):
             assert np.array_equal(got[i], rig.pool_np[q][dst]), (g, q)
     stream.synchronize()
+    rig.check()
+    rig.close()
+
+
+@pytest.mark.parametrize("kw", [
+    dict(tier_location=1, copy_path=1), dict(tier_location=1, copy_path=0),
+    dict(tier_location=0, link_strategy=0),
+    dict(tier_location=0, link_strategy=1, min_staged_run_bytes=-1),
+    dict(tier_location=0, link_strategy=1),
+    dict(tier_location=0, link_strategy=2, contiguous_pool=True),
+], ids=["hbm-bulk", "hbm-vector", "host-zero-copy", "host-staged", "host-default", "host-copy-engine"])
+@pytest.mark.parametrize("name,group", [("qwen", 12), ("qwen", 5), ("tiny", 1), ("ragged", 2), ("qwen_tp8", 5),
+                                        ("small", 1)])
+def test_layer_pipelined_store(name, group, kw):
+    """eakv_store_layers writes the same bytes as eakv_store, in layer groups (masked entries
+    untouched, errors as for the plain store)."""
+    e = eakv()
+    shape = SHAPE_CASES[name]
+    nb, kh = (64, 48) if shape.block_bytes <= (1 << 21) else (24, 20)
+    rig = Rig(shape, nb, kh, seed=22, staging_bytes=3 * shape.block_bytes, **kw)
+    rng = rig.rng
+    groups = -(-shape.num_layers // group)
+    none = [None] * groups
+    m = min(nb, kh) - 5
+    table = rng.permutation(nb)[:m].astype(np.int32)
+    slots = rng.permutation(kh)[:m].astype(np.int32)
+    admit = (rng.random(m) < 0.7).astype(np.uint8)
+    stream = torch.cuda.Stream()
+    rig.ctx.eakv_store_layers(table, admit, slots, group, none, stream)
+    osl.store(rig.pool_np, rig.tier_np, table, admit, slots)
+    stream.synchronize()
+    rig.check()
+    # contiguous slots without a mask, and an empty call
+    rig.ctx.eakv_store_layers(np.arange(8, dtype=np.int32)[::-1].copy(), None, np.arange(8, dtype=np.int32),
+                              group, none, stream)
+    osl.store(rig.pool_np, rig.tier_np, list(range(8))[::-1], [1] * 8, list(range(8)))
+    rig.ctx.eakv_store_layers(np.zeros(0, np.int32), None, np.zeros(0, np.int32), group, none, stream)
+    stream.synchronize()
+    rig.check()
+    assert rig.ctx.eakv_get_stats()["blocks_stored"] == int(admit.sum()) + 8
+    for bad, code in (((table, admit, slots, group, none + [None]), e.E_INVAL),                     # events
+                      ((np.array([0, 1], np.int32), None, np.array([3, 3], np.int32), group, none), e.E_INVAL),
+                      ((np.array([nb], np.int32), None, np.array([0], np.int32), group, none), e.E_RANGE)):
+        with pytest.raises(e.EakvError) as ei:
+            rig.ctx.eakv_store_layers(*bad, stream)
+        assert ei.value.code == code
+    rig.check()
+    rig.close()
+
+
+@pytest.mark.parametrize("kw", [
+    dict(tier_location=1, copy_path=1),
+    dict(tier_location=0, link_strategy=0),
+    dict(tier_location=0, link_strategy=1, min_staged_run_bytes=-1),
+    dict(tier_location=0, link_strategy=2, contiguous_pool=True),
+], ids=["hbm-bulk", "host-zero-copy", "host-staged", "host-copy-engine"])
+@pytest.mark.parametrize("name,group", [("qwen", 12), ("qwen_tp8", 16)])
+def test_layer_pipelined_store_waits_for_each_group(name, group, kw):
+    """The contract of eakv_store_layers: group g is read only after ready_events[g].  A producer
+    stream fills the layers group by group, each fill held back by a delay and followed by its
+    event; the store is enqueued on another stream right away.  The tier must hold what the
+    producer wrote, not what the blocks held when the store was enqueued."""
+    shape = SHAPE_CASES[name]
+    nb, kh, m = 64, 48, 40
+    rig = Rig(shape, nb, kh, seed=34, staging_bytes=4 * shape.block_bytes, **kw)
+    rng = rig.rng
+    groups = -(-shape.num_layers // group)
+    table = rng.permutation(nb)[:m].astype(np.int32)
+    slots = rng.permutation(kh)[:m].astype(np.int32)
+    ids = torch.as_tensor(table.astype(np.int64), device="cuda")
+    fresh = [torch.from_numpy(rng.integers(0, 256, size=(m, shape.piece_bytes), dtype=np.uint8)).cuda()
+             for _ in range(shape.pieces_per_block)]
+    producer, io = torch.cuda.Stream(), torch.cuda.Stream()
+    events = [torch.cuda.Event() for _ in range(groups)]
+    torch.cuda.synchronize()
+    with torch.cuda.stream(producer):
+        for g in range(groups):
+            torch.cuda._sleep(20_000_000)                       # ~10 ms: the store is enqueued long before
+            for q in range(2 * g * group, min(2 * (g + 1) * group, shape.pieces_per_block)):
+                rig.pool_dev[q].view(torch.uint8).view(nb, -1)[ids] = fresh[q]
+            events[g].record(producer)
+    rig.ctx.eakv_store_layers(table, None, slots, group, [ev.cuda_event for ev in events], io)
+    for q in range(shape.pieces_per_block):
+        rig.pool_np[q][table] = fresh[q].cpu().numpy()
+    osl.store(rig.pool_np, rig.tier_np, table, [1] * m, slots)
+    io.synchronize()
+    producer.synchronize()
     rig.check()
     rig.close()
 
