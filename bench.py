@@ -547,6 +547,35 @@ def layered_load_probe(torch, arm, tables, shape, layers_per_group=12):
     return out
 
 
+def layered_store_probe(torch, arm, tables, shape, layers_per_group=12):
+    """Write 4,096 blocks to the pinned tier whole, and in layer groups behind per-group events of
+    a producer (already complete here, so the figures are the write alone): the layered form
+    costs nothing extra, and under a real producer its first groups run beneath the compute."""
+    m = arm.m
+    slots = np.arange(m, dtype=np.int32)
+    table = tables[0][:m]
+    st = torch.cuda.Stream(arm.device)
+    groups = -(-shape.num_layers // layers_per_group)
+    evs = [torch.cuda.Event() for _ in range(groups)]
+    for ev in evs:
+        ev.record(st)
+    out = {}
+    for mode in ("plain", "layered"):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        if mode == "plain":
+            arm.ctx.eakv_store(table, None, slots, st)
+        else:
+            arm.ctx.eakv_store_layers(table, None, slots, layers_per_group, [ev.cuda_event for ev in evs], st)
+        e1.record(st)
+        torch.cuda.synchronize()
+        out[mode + "_ms"] = e0.elapsed_time(e1)
+    out["layers_per_group"] = layers_per_group
+    out["blocks"] = m
+    return out
+
+
 def store_load_curve(torch, eakv, pool, shape, device, args, h2d_peak, d2h_peak, tier_ptr=None,
                      tier_blocks=4096, reps=5):
     """The microbench's curve: 1 to 4,096 blocks per call, block ids contiguous or uniform-random
@@ -985,6 +1014,7 @@ def main():
         pass_ms = [aggregate_over_ranks(dist, p_["ms"], p_["moved"], device) for p_ in passes]
         re_ = passes[0] if pass_ms[0][0] <= pass_ms[1][0] else passes[1]
         layered = layered_load_probe(torch, arm, tables, shape) if (rank == 0 and not args.quick) else None
+        layered_st = layered_store_probe(torch, arm, tables, shape) if (rank == 0 and not args.quick) else None
         arm.ctx.close()
         del arm
         e_ms, e_moved = aggregate_over_ranks(dist, re_["ms"], re_["moved"], device)
@@ -994,6 +1024,7 @@ def main():
                "ms_per_step": e_ms / e_steps, "link_strategy": args.link,
                "passes_gbps": [mv / (ms_ * 1e-3) / 1e9 for ms_, mv in pass_ms]}
         e2e["layered_load"] = layered
+        e2e["layered_store"] = layered_st
         serial = bound = None
         if link:
             # one direction at a time: harmonic mean of the two; both at once: the measured
