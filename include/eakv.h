@@ -403,6 +403,11 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
                     const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
                     void* cuda_stream, eakv_turn_view* view);
 int eakv_turn_end(eakv_ctx* ctx, void* cuda_stream);
+/* eakv_turn_end with the host write in layer groups (eakv_store_layers: group g is read only
+ * after ready_events[g], which the engine recorded behind the work that completes those layers).
+ * A wrong n_events is refused with EAKV_E_INVAL and the turn stays open. */
+int eakv_turn_end_layers(eakv_ctx* ctx, int32_t layers_per_group, void* const* ready_events,
+                         int32_t n_events, void* cuda_stream);
 int eakv_turn_abort(eakv_ctx* ctx);
 
 /* The same turn for an engine that runs several requests at once (Section 2: the engine's cap on
@@ -441,6 +446,9 @@ int eakv_request_begin(eakv_ctx* ctx, int64_t request_id, const int32_t* tokens,
                        const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
                        int32_t decided, void* cuda_stream, eakv_turn_view* view);
 int eakv_request_store(eakv_ctx* ctx, int64_t request_id, void* cuda_stream);
+/* eakv_request_store in layer groups, as eakv_turn_end_layers. */
+int eakv_request_store_layers(eakv_ctx* ctx, int64_t request_id, int32_t layers_per_group,
+                              void* const* ready_events, int32_t n_events, void* cuda_stream);
 int eakv_request_release(eakv_ctx* ctx, int64_t request_id);
 
 /* Layer-pipelined restore (Section 3.1, Eq. 2: the fixed restoration overhead tau_load is

@@ -1512,8 +1512,22 @@ int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32
     return EAKV_OK;
 }
 
-// the store of an open turn's admitted blocks (directly, or deferred on the context's stream)
-int turn_store_impl(eakv_ctx* ctx, TurnState& T, void* cuda_stream) {
+// the store of an open turn's admitted blocks (directly, or deferred on the context's stream);
+// layers_per_group > 0: in layer groups behind the producer's events (eakv_store_layers)
+int turn_store_impl(eakv_ctx* ctx, TurnState& T, void* cuda_stream, int32_t layers_per_group = 0,
+                    void* const* ready_events = nullptr, int32_t n_events = 0) {
+    if (layers_per_group < 0) return EAKV_E_INVAL;
+    if (layers_per_group > 0) {      // refused before the turn counts as stored
+        const int groups = (ctx->cfg.num_layers + layers_per_group - 1) / layers_per_group;
+        if (n_events != groups || !ready_events) return EAKV_E_INVAL;
+    }
+    auto write = [&](void* on_stream) {
+        const int64_t n = (int64_t)T.block.size();
+        if (layers_per_group > 0)
+            return eakv_store_layers(ctx, T.block.data(), T.admit_b.data(), T.slot_b.data(), n, layers_per_group,
+                                     ready_events, n_events, on_stream);
+        return eakv_store(ctx, T.block.data(), T.admit_b.data(), T.slot_b.data(), n, on_stream);
+    };
     const int64_t nblk = (int64_t)T.block.size();
     T.stored = true;
     claim_units(ctx, T);                                     // from here on a stream-ordered restore finds the bytes
@@ -1528,8 +1542,7 @@ int turn_store_impl(eakv_ctx* ctx, TurnState& T, void* cuda_stream) {
     if (!any_store) return EAKV_OK;                          // nothing to write
     if (const int inj = injected_failure(ctx)) return inj;
     if (ctx->device < 0) return EAKV_OK;                     // bookkeeping only
-    if (!ctx->cfg.write_behind)
-        return eakv_store(ctx, T.block.data(), T.admit_b.data(), T.slot_b.data(), nblk, cuda_stream);
+    if (!ctx->cfg.write_behind) return write(cuda_stream);
     // deferred write: on the context's stream, after what precedes it on the caller's stream
     DeviceGuard g(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -1542,7 +1555,7 @@ int turn_store_impl(eakv_ctx* ctx, TurnState& T, void* cuda_stream) {
     }
     CU(cudaEventRecord(ctx->wb_fence, stream));
     CU(cudaStreamWaitEvent(ctx->wb_stream, ctx->wb_fence, 0));
-    int r = eakv_store(ctx, T.block.data(), T.admit_b.data(), T.slot_b.data(), nblk, ctx->wb_stream);
+    int r = write(ctx->wb_stream);
     if (r != EAKV_OK) return r;
     CU(cudaEventRecord(ctx->wb_done, ctx->wb_stream));
     for (int64_t j = 0; j < nblk; ++j)
@@ -1567,8 +1580,14 @@ int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
 }
 
 int eakv_turn_end(eakv_ctx* ctx, void* cuda_stream) {
+    return eakv_turn_end_layers(ctx, 0, nullptr, 0, cuda_stream);
+}
+
+int eakv_turn_end_layers(eakv_ctx* ctx, int32_t layers_per_group, void* const* ready_events, int32_t n_events,
+                         void* cuda_stream) {
     if (!ctx || !ctx->turn.open) return EAKV_E_INVAL;
-    const int rc = turn_store_impl(ctx, ctx->turn, cuda_stream);
+    const int rc = turn_store_impl(ctx, ctx->turn, cuda_stream, layers_per_group, ready_events, n_events);
+    if (rc == EAKV_E_INVAL && !ctx->turn.stored) return rc;                   // bad arguments: the turn stays open
     // a store that could not be enqueued leaves slots unwritten: their keys must not stay listed
     withdraw_turn(ctx, ctx->turn, rc != EAKV_OK, 0);
     return rc;
@@ -1594,10 +1613,16 @@ int eakv_request_begin(eakv_ctx* ctx, int64_t request_id, const int32_t* tokens,
 }
 
 int eakv_request_store(eakv_ctx* ctx, int64_t request_id, void* cuda_stream) {
+    return eakv_request_store_layers(ctx, request_id, 0, nullptr, 0, cuda_stream);
+}
+
+int eakv_request_store_layers(eakv_ctx* ctx, int64_t request_id, int32_t layers_per_group,
+                              void* const* ready_events, int32_t n_events, void* cuda_stream) {
     if (!ctx) return EAKV_E_INVAL;
     auto it = ctx->requests.find(request_id);
     if (it == ctx->requests.end() || it->second.stored) return EAKV_E_INVAL;
-    const int rc = turn_store_impl(ctx, it->second, cuda_stream);
+    const int rc = turn_store_impl(ctx, it->second, cuda_stream, layers_per_group, ready_events, n_events);
+    if (rc == EAKV_E_INVAL && !it->second.stored) return rc;                  // bad arguments: the request stays open
     if (rc != EAKV_OK) {
         withdraw_turn(ctx, it->second, true, 0);
         ctx->requests.erase(it);

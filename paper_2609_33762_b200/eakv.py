@@ -111,7 +111,7 @@ EXPORTS = [
     "eakv_selfcheck_limits", "eakv_selfcheck_wait_probe",
     "eakv_gpu_tier_acquire", "eakv_gpu_tier_release_request", "eakv_tier_step_again",
     "eakv_declined_audit", "eakv_working_set",
-    "eakv_request_begin", "eakv_request_store", "eakv_request_release", "eakv_working_set_sizes", "eakv_selfcheck_fail_next_transfer", "eakv_store_layers",
+    "eakv_request_begin", "eakv_request_store", "eakv_request_release", "eakv_working_set_sizes", "eakv_selfcheck_fail_next_transfer", "eakv_store_layers", "eakv_turn_end_layers", "eakv_request_store_layers",
 ]
 STATIC_MAX_BLOCKS = 65536
 
@@ -151,6 +151,8 @@ def lib():
     L.eakv_declined_audit.argtypes = [vp, vp, i64, i64, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), vp, vp]
     L.eakv_selfcheck_fail_next_transfer.argtypes = [vp, i32]
     L.eakv_store_layers.argtypes = [vp, vp, vp, vp, i64, i32, vp, i32, vp]
+    L.eakv_turn_end_layers.argtypes = [vp, i32, vp, i32, vp]
+    L.eakv_request_store_layers.argtypes = [vp, i64, i32, vp, i32, vp]
     L.eakv_working_set_sizes.argtypes = [vp, i64, vp, vp, vp, i64, i32, i32, C.POINTER(i64), C.POINTER(i64), vp]
     L.eakv_working_set.argtypes = [C.POINTER(WorkingSetIn), C.POINTER(WorkingSetOut)]
     L.eakv_turn_begin.argtypes = [vp, vp, i64, vp, i64, i64, i64, vp, C.POINTER(TurnView)]
@@ -559,6 +561,22 @@ class Context:
 
     def eakv_request_store(self, request_id, stream=None):
         self._check(lib().eakv_request_store(self._h, int(request_id), _stream(stream)), "eakv_request_store")
+
+    @staticmethod
+    def _event_array(ready_events):
+        return (C.c_void_p * max(len(ready_events), 1))(*[None if e is None else int(e) for e in ready_events])
+
+    def eakv_request_store_layers(self, request_id, layers_per_group, ready_events, stream=None):
+        ev = self._event_array(ready_events)
+        rc = lib().eakv_request_store_layers(self._h, int(request_id), int(layers_per_group), C.cast(ev, C.c_void_p),
+                                             len(ready_events), _stream(stream))
+        self._check(rc, "eakv_request_store_layers")
+
+    def eakv_turn_end_layers(self, layers_per_group, ready_events, stream=None):
+        ev = self._event_array(ready_events)
+        rc = lib().eakv_turn_end_layers(self._h, int(layers_per_group), C.cast(ev, C.c_void_p),
+                                        len(ready_events), _stream(stream))
+        self._check(rc, "eakv_turn_end_layers")
 
     def eakv_request_release(self, request_id):
         self._check(lib().eakv_request_release(self._h, int(request_id)), "eakv_request_release")

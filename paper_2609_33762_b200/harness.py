@@ -53,13 +53,18 @@ class PagedPool:
 class AgentServer:
     def __init__(self, shape, gpu_blocks, host_blocks, payload, *, device="cuda:0",
                  gpu_index_blocks=0, incremental_hash=False, data_plane=True, chunk_blocks=1,
-                 native_turn=None, **ctx_kwargs):
+                 native_turn=None, store_layers=0, **ctx_kwargs):
         """``payload(keys, q, n_words)`` returns the int16/uint16 words of piece q for the
         blocks with these keys, as a numpy array or a tensor on ``device``.  With
         ``chunk_blocks`` = R > 1 the host tier works in chunks of R blocks (``host_blocks``
         then counts chunks): one key per full chunk goes to the tier step, and chunk slot s
-        maps to block slots s*R .. s*R+R-1 for store and load."""
+        maps to block slots s*R .. s*R+R-1 for store and load.  ``store_layers`` = g > 0 (turn
+        engine, data plane): the "prefill" runs on a stream of its own, g layers at a time with an
+        event after each group, and the host write follows it group by group
+        (eakv_turn_end_layers / eakv_request_store_layers)."""
         self.shape = shape
+        self.store_layers = int(store_layers)
+        self._fill_stream = None
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         # data_plane=False runs keys, matching and both tiers' bookkeeping only: no KV bytes move.
@@ -90,6 +95,7 @@ class AgentServer:
         self.payload = payload
         self.incremental = incremental_hash
         self.stream = torch.cuda.current_stream(self.device)
+        self._ready = {}
         self.b = shape.block_size
         self.R = max(1, int(chunk_blocks))
         if native_turn is None:
@@ -191,11 +197,15 @@ class AgentServer:
         keys, blocks = v["keys"], v["gpu_block"]
         if self.incremental and self.data_plane:
             self._agent_keys[agent] = keys
-        self._fill(keys, blocks, np.nonzero(v["needs_fill"])[0])
+        ready = self._fill(keys, blocks, np.nonzero(v["needs_fill"])[0])
         if self.data_plane:
             e0 = torch.cuda.Event(enable_timing=True)
             e0.record(self.stream)
-        self.ctx.eakv_turn_end(self.stream)
+        if ready is None:
+            self.ctx.eakv_turn_end(self.stream)
+        else:
+            self.ctx.eakv_turn_end_layers(self.store_layers, ready, self.stream)
+            self.stream.wait_stream(self._fill_stream)
         if self.data_plane:
             self._timed_since(e0, "store", v["n_stored_blocks"] * self.ctx.block_bytes)
         rec = self._record_from_view(v, agent, now_ms, n)
@@ -283,7 +293,14 @@ class AgentServer:
 
     def store(self, request_id):
         """The deferred host write of ``begin(..., defer_store=True)`` (eakv_request_store)."""
-        self.ctx.eakv_request_store(request_id, self.stream if self.data_plane else None)
+        self._request_store(request_id, self._ready.pop(request_id, None))
+
+    def _request_store(self, request_id, ready):
+        if ready is None:
+            self.ctx.eakv_request_store(request_id, self.stream if self.data_plane else None)
+        else:
+            self.ctx.eakv_request_store_layers(request_id, self.store_layers, ready, self.stream)
+            self.stream.wait_stream(self._fill_stream)
 
     def _begin_native(self, request_id, tokens, agent, now_ms, decided, defer_store=False):
         """The same through eakv_request_begin / eakv_request_store."""
@@ -304,9 +321,11 @@ class AgentServer:
             prev = self._agent_keys.get(agent)
             if prev is None or len(keys) >= len(prev):
                 self._agent_keys[agent] = keys
-        self._fill(keys, blocks, np.nonzero(v["needs_fill"])[0])
-        if not defer_store:
-            self.ctx.eakv_request_store(request_id, self.stream)
+        ready = self._fill(keys, blocks, np.nonzero(v["needs_fill"])[0])
+        if defer_store:
+            self._ready[request_id] = ready
+        else:
+            self._request_store(request_id, ready)
         rec = self._record_from_view(v, agent, now_ms, n)
         rec.update(request_id=request_id, resumed=decided is not None)
         t = self.totals
@@ -323,14 +342,37 @@ class AgentServer:
         return rec
 
     def _fill(self, keys, blocks, fill):
-        """The engine's part: produce the KV of the blocks the library flagged (synthetic payload)."""
-        if len(fill) and self.data_plane:
-            ids = torch.as_tensor(blocks[fill].astype(np.int64), device=self.device)
-            for q, piece in enumerate(self.pool.pieces):
-                w = self.payload(keys[fill], q, self.pool.words)
-                if isinstance(w, np.ndarray):
-                    w = torch.from_numpy(w.view(np.int16)).to(self.device)
-                piece[ids] = w.view(torch.int16)
+        """The engine's part: produce the KV of the blocks the library flagged (synthetic payload).
+        With ``store_layers`` the layers are produced on a stream of their own, a group at a time,
+        and the handles of the per-group events are returned for the layered host write."""
+        layered = self.store_layers > 0 and self.data_plane and self.native_turn
+        if not layered:
+            if len(fill) and self.data_plane:
+                ids = torch.as_tensor(blocks[fill].astype(np.int64), device=self.device)
+                for q, piece in enumerate(self.pool.pieces):
+                    w = self.payload(keys[fill], q, self.pool.words)
+                    if isinstance(w, np.ndarray):
+                        w = torch.from_numpy(w.view(np.int16)).to(self.device)
+                    piece[ids] = w.view(torch.int16)
+            return None
+        if self._fill_stream is None:
+            self._fill_stream = torch.cuda.Stream(self.device)
+        g = self.store_layers
+        groups = -(-self.shape.num_layers // g)
+        events = [torch.cuda.Event() for _ in range(groups)]
+        self._fill_events = events                      # kept alive until the next fill
+        ids = torch.as_tensor(blocks[fill].astype(np.int64), device=self.device) if len(fill) else None
+        self._fill_stream.wait_stream(self.stream)      # the blocks may still be read by earlier work
+        with torch.cuda.stream(self._fill_stream):
+            for grp in range(groups):
+                for q in range(2 * grp * g, min(2 * (grp + 1) * g, len(self.pool.pieces))):
+                    if ids is not None:
+                        w = self.payload(keys[fill], q, self.pool.words)
+                        if isinstance(w, np.ndarray):
+                            w = torch.from_numpy(w.view(np.int16)).to(self.device)
+                        self.pool.pieces[q][ids] = w.view(torch.int16)
+                events[grp].record(self._fill_stream)
+        return [ev.cuda_event for ev in events]
 
     @staticmethod
     def _record_from_view(v, agent, now_ms, n):

@@ -291,9 +291,9 @@ def test_engine_replay_with_preemption_bit_exact(policy, kh, gpu_blocks, S, deco
     server.close()
 
 
-@pytest.mark.parametrize("R,link,seed,write_behind", [(1, 1, 5, False), (1, 0, 6, False), (2, 1, 11, False),
-                                                       (1, 1, 8, True)])
-def test_deferred_stores_interleaved_with_other_lookups_with_bytes(R, link, seed, write_behind):
+@pytest.mark.parametrize("R,link,seed,write_behind,layers", [(1, 1, 5, False, 0), (1, 0, 6, False, 0), (2, 1, 11, False, 0),
+                                                              (1, 1, 8, True, 0), (1, 1, 6, False, 2)])
+def test_deferred_stores_interleaved_with_other_lookups_with_bytes(R, link, seed, write_behind, layers):
     """Requests whose host write comes only after other requests have been looked up
     (eakv_request_begin ... eakv_request_store): a unit that a later lookup evicted before its
     bytes arrived must not be written, or the slot's new owner would read a stranger's KV.  Every
@@ -306,7 +306,7 @@ def test_deferred_stores_interleaved_with_other_lookups_with_bytes(R, link, seed
     gpu_blocks, kh = 200, 64 // R               # a tier a few running requests overrun
     oracle = TraceOracle(shape, gpu_blocks, kh, payload=key_words_numpy, chunk_blocks=R)
     server = AgentServer(shape, gpu_blocks, kh, key_words_numpy, incremental_hash=False, chunk_blocks=R,
-                         link_strategy=link, native_turn=True, write_behind=write_behind)
+                         link_strategy=link, native_turn=True, write_behind=write_behind, store_layers=layers)
     seen = dict(begins=0, skipped=0)
 
     def check_listed_bytes():
@@ -339,6 +339,29 @@ def test_deferred_stores_interleaved_with_other_lookups_with_bytes(R, link, seed
 
     drive(operations(seed, 260, b, 60 * b, max_open=4), on_begin, on_store, on_finish)
     assert seen["begins"] > 60 and seen["skipped"] > 0          # evicted-before-written did occur
+    compare_bytes(server, oracle)
+    server.close()
+
+
+@pytest.mark.parametrize("cfg_name,R,policy,link,group,write_behind", [
+    ("c0", 1, 0, 1, 1, False), ("c0", 1, 2, 0, 3, False), ("c0_big_tier", 4, 0, 1, 2, False), ("c0", 1, 0, 1, 4, True)])
+def test_turn_engine_with_layered_host_writes_bit_exact(cfg_name, R, policy, link, group, write_behind):
+    """The turn engine with the prefill on a stream of its own, a layer group at a time, and the
+    host write following it group by group (eakv_turn_end_layers): records and every resident byte
+    equal the oracle's."""
+    from paper_2609_33762_b200.harness import AgentServer
+    cfg = CONFIGS[cfg_name]
+    shape = SHAPES[cfg.shape]
+    trace = make_trace(cfg)
+    kh = cfg.host_blocks // R
+    kw = dict(policy=policy, kappa_blocks=20, window_ms=40, len_window=16)
+    oracle = TraceOracle(shape, cfg.gpu_blocks, kh, payload=key_words_numpy, chunk_blocks=R, **kw)
+    oracle.run(trace)
+    server = AgentServer(shape, cfg.gpu_blocks, kh, key_words_numpy, native_turn=True, incremental_hash=True,
+                         chunk_blocks=R, link_strategy=link, store_layers=group, write_behind=write_behind, **kw)
+    server.run(trace)
+    compare_records(server.records, oracle.records)
+    assert server.totals == oracle.totals and oracle.totals["stored_blocks"] > 0
     compare_bytes(server, oracle)
     server.close()
 
