@@ -204,7 +204,7 @@ class AgentServer:
         if ready is None:
             self.ctx.eakv_turn_end(self.stream)
         else:
-            self.ctx.eakv_turn_end_layers(self.store_layers, ready, self.stream)
+            self.ctx.eakv_turn_end_layers(self.store_layers, [ev.cuda_event for ev in ready], self.stream)
             self.stream.wait_stream(self._fill_stream)
         if self.data_plane:
             self._timed_since(e0, "store", v["n_stored_blocks"] * self.ctx.block_bytes)
@@ -299,7 +299,8 @@ class AgentServer:
         if ready is None:
             self.ctx.eakv_request_store(request_id, self.stream if self.data_plane else None)
         else:
-            self.ctx.eakv_request_store_layers(request_id, self.store_layers, ready, self.stream)
+            self.ctx.eakv_request_store_layers(request_id, self.store_layers, [ev.cuda_event for ev in ready],
+                                               self.stream)
             self.stream.wait_stream(self._fill_stream)
 
     def _begin_native(self, request_id, tokens, agent, now_ms, decided, defer_store=False):
@@ -344,7 +345,7 @@ class AgentServer:
     def _fill(self, keys, blocks, fill):
         """The engine's part: produce the KV of the blocks the library flagged (synthetic payload).
         With ``store_layers`` the layers are produced on a stream of their own, a group at a time,
-        and the handles of the per-group events are returned for the layered host write."""
+        and the per-group events are returned for the layered host write."""
         layered = self.store_layers > 0 and self.data_plane and self.native_turn
         if not layered:
             if len(fill) and self.data_plane:
@@ -359,8 +360,7 @@ class AgentServer:
             self._fill_stream = torch.cuda.Stream(self.device)
         g = self.store_layers
         groups = -(-self.shape.num_layers // g)
-        events = [torch.cuda.Event() for _ in range(groups)]
-        self._fill_events = events                      # kept alive until the next fill
+        events = [torch.cuda.Event() for _ in range(groups)]    # (the caller keeps them until the store is enqueued)
         ids = torch.as_tensor(blocks[fill].astype(np.int64), device=self.device) if len(fill) else None
         self._fill_stream.wait_stream(self.stream)      # the blocks may still be read by earlier work
         with torch.cuda.stream(self._fill_stream):
@@ -372,7 +372,7 @@ class AgentServer:
                             w = torch.from_numpy(w.view(np.int16)).to(self.device)
                         self.pool.pieces[q][ids] = w.view(torch.int16)
                 events[grp].record(self._fill_stream)
-        return [ev.cuda_event for ev in events]
+        return events
 
     @staticmethod
     def _record_from_view(v, agent, now_ms, n):
@@ -386,6 +386,7 @@ class AgentServer:
 
     def finish(self, request_id):
         """The request finished, or the engine suspended it: its GPU blocks become evictable."""
+        self._ready.pop(request_id, None)
         if self.native_turn:
             self.ctx.eakv_request_release(request_id)
         else:
