@@ -375,3 +375,28 @@ def test_injected_transfer_failures_withdraw_what_the_turn_registered(eakv):
     assert ctx2.eakv_match(grown)[1] == 9
     ctx2.close()
     ctx.close()
+
+
+def test_layered_end_refuses_a_wrong_event_count_and_keeps_the_turn_open(eakv):
+    """eakv_turn_end_layers / eakv_request_store_layers: one event per layer group; a wrong count
+    is refused before anything happens, and the turn can still be ended."""
+    b = 4
+    ctx = eakv.Context(num_layers=5, kv_heads=1, head_dim=8, block_size=b, gpu_blocks=32, host_blocks=32,
+                       kv_base=None, control_plane_only=True)
+    keys = np.arange(1, 5, dtype=np.uint64)
+    ctx.eakv_turn_begin(0, 4 * b, keys, 0, 0)
+    for bad in ([None], [None] * 4):                      # 5 layers in groups of 2 -> 3 events
+        with pytest.raises(eakv.EakvError) as ei:
+            ctx.eakv_turn_end_layers(2, bad)
+        assert ei.value.code == eakv.E_INVAL
+    ctx.eakv_turn_end_layers(2, [None] * 3)
+    assert ctx.eakv_match(keys)[1] == 4
+    more = np.arange(1, 7, dtype=np.uint64)
+    ctx.eakv_request_begin(7, 0, 6 * b, more, 0, 1)
+    with pytest.raises(eakv.EakvError) as ei:
+        ctx.eakv_request_store_layers(7, 5, [None] * 2)   # one group of 5 layers -> 1 event
+    assert ei.value.code == eakv.E_INVAL
+    ctx.eakv_request_store_layers(7, 5, [None])
+    ctx.eakv_request_release(7)
+    assert ctx.eakv_match(more)[1] == 6
+    ctx.close()
