@@ -402,6 +402,14 @@ typedef struct eakv_turn_view {
 int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
                     const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
                     void* cuda_stream, eakv_turn_view* view);
+/* eakv_turn_begin with the restore in layer groups (eakv_load_layers): events[g] is recorded on
+ * cuda_stream once group g of the restored blocks has landed -- also when the turn restores
+ * nothing, so that a consumer may always wait on them.  A wrong n_events or a NULL event is
+ * refused with EAKV_E_INVAL before anything changes.  (A bookkeeping-only context records nothing.) */
+int eakv_turn_begin_layers(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
+                           const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
+                           int32_t layers_per_group, void* const* events, int32_t n_events,
+                           void* cuda_stream, eakv_turn_view* view);
 int eakv_turn_end(eakv_ctx* ctx, void* cuda_stream);
 /* eakv_turn_end with the host write in layer groups (eakv_store_layers: group g is read only
  * after ready_events[g], which the engine recorded behind the work that completes those layers).
@@ -445,6 +453,11 @@ int eakv_turn_abort(eakv_ctx* ctx);
 int eakv_request_begin(eakv_ctx* ctx, int64_t request_id, const int32_t* tokens, int64_t n_tokens,
                        const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
                        int32_t decided, void* cuda_stream, eakv_turn_view* view);
+/* eakv_request_begin with the restore in layer groups, as eakv_turn_begin_layers. */
+int eakv_request_begin_layers(eakv_ctx* ctx, int64_t request_id, const int32_t* tokens, int64_t n_tokens,
+                              const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
+                              int32_t decided, int32_t layers_per_group, void* const* events, int32_t n_events,
+                              void* cuda_stream, eakv_turn_view* view);
 int eakv_request_store(eakv_ctx* ctx, int64_t request_id, void* cuda_stream);
 /* eakv_request_store in layer groups, as eakv_turn_end_layers. */
 int eakv_request_store_layers(eakv_ctx* ctx, int64_t request_id, int32_t layers_per_group,

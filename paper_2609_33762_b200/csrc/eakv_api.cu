@@ -1348,9 +1348,17 @@ void withdraw_turn(eakv_ctx* ctx, TurnState& T, bool host_units, int gpu_mode) {
 // decided < 0: the request's first lookup; 0 / 1: a later lookup with that store/skip choice
 int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32_t* tokens, int64_t n_tokens,
                     const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms, int decided,
-                    void* cuda_stream, eakv_turn_view* view) {
+                    void* cuda_stream, eakv_turn_view* view, int32_t layers_per_group = 0,
+                    void* const* events = nullptr, int32_t n_events = 0) {
     const bool as_request = request_id != kNoRequest;
     const bool bookkeeping_only = ctx->device < 0;
+    if (layers_per_group < 0) return EAKV_E_INVAL;
+    if (layers_per_group > 0) {                   // the restore in layer groups: one event per group
+        const int groups = (ctx->cfg.num_layers + layers_per_group - 1) / layers_per_group;
+        if (n_events != groups || !events) return EAKV_E_INVAL;
+        for (int g = 0; g < groups; ++g)
+            if (!events[g]) return EAKV_E_INVAL;
+    }
     const int b = ctx->cfg.block_size;
     const int64_t R = ctx->chunk_tokens / b;
     const int64_t nblk = n_tokens / b;
@@ -1468,14 +1476,19 @@ int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32
     const int64_t H = Hu * R;
     const int64_t cover = std::max(G, H);
     const int64_t lo = G, hi = H > G ? H : G;
-    if (hi > lo) {
+    if (hi > lo || (layers_per_group > 0 && !bookkeeping_only)) {
         // block slots of the restored blocks: chunk slot * R + position inside the chunk
         std::vector<int32_t> slots((size_t)(hi - lo));
         for (int64_t j = lo; j < hi; ++j)
             slots[j - lo] = (int32_t)((int64_t)T.host_slots[j / R] * R + j % R);
-        rc = injected_failure(ctx);
-        if (rc == EAKV_OK && !bookkeeping_only)
-            rc = eakv_load(ctx, slots.data(), T.block.data() + lo, hi - lo, cuda_stream);
+        rc = hi > lo ? injected_failure(ctx) : EAKV_OK;
+        if (rc == EAKV_OK && !bookkeeping_only) {
+            if (layers_per_group > 0)      // (with nothing to restore the events are recorded all the same)
+                rc = eakv_load_layers(ctx, slots.data(), T.block.data() + lo, hi - lo, layers_per_group, events,
+                                      n_events, cuda_stream);
+            else
+                rc = eakv_load(ctx, slots.data(), T.block.data() + lo, hi - lo, cuda_stream);
+        }
         if (rc != EAKV_OK) {
             // nothing of this turn was restored or will be computed: neither tier may list it
             withdraw_turn(ctx, T, true, 1);
@@ -1572,11 +1585,19 @@ int turn_store_impl(eakv_ctx* ctx, TurnState& T, void* cuda_stream, int32_t laye
 int eakv_turn_begin(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
                     const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
                     void* cuda_stream, eakv_turn_view* view) {
+    return eakv_turn_begin_layers(ctx, tokens, n_tokens, known_keys, n_known, agent_id, now_ms, 0, nullptr, 0,
+                                  cuda_stream, view);
+}
+
+int eakv_turn_begin_layers(eakv_ctx* ctx, const int32_t* tokens, int64_t n_tokens,
+                           const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
+                           int32_t layers_per_group, void* const* events, int32_t n_events,
+                           void* cuda_stream, eakv_turn_view* view) {
     if (!ctx || !view || n_tokens < 0 || n_known < 0) return EAKV_E_INVAL;
     if (ctx->turn.open || !ctx->held.empty()) return EAKV_E_INVAL;
     if (n_known > 0 && !known_keys) return EAKV_E_INVAL;
     return turn_begin_impl(ctx, ctx->turn, kNoRequest, tokens, n_tokens, known_keys, n_known, agent_id, now_ms,
-                           -1, cuda_stream, view);
+                           -1, cuda_stream, view, layers_per_group, events, n_events);
 }
 
 int eakv_turn_end(eakv_ctx* ctx, void* cuda_stream) {
@@ -1602,12 +1623,21 @@ int eakv_turn_abort(eakv_ctx* ctx) {
 int eakv_request_begin(eakv_ctx* ctx, int64_t request_id, const int32_t* tokens, int64_t n_tokens,
                        const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
                        int32_t decided, void* cuda_stream, eakv_turn_view* view) {
+    return eakv_request_begin_layers(ctx, request_id, tokens, n_tokens, known_keys, n_known, agent_id, now_ms,
+                                     decided, 0, nullptr, 0, cuda_stream, view);
+}
+
+int eakv_request_begin_layers(eakv_ctx* ctx, int64_t request_id, const int32_t* tokens, int64_t n_tokens,
+                              const uint64_t* known_keys, int64_t n_known, int64_t agent_id, int64_t now_ms,
+                              int32_t decided, int32_t layers_per_group, void* const* events, int32_t n_events,
+                              void* cuda_stream, eakv_turn_view* view) {
     if (!ctx || !view || n_tokens < 0 || n_known < 0 || request_id == kNoRequest) return EAKV_E_INVAL;
     if (ctx->turn.open || ctx->requests.count(request_id) || ctx->held.count(request_id)) return EAKV_E_INVAL;
     if (n_known > 0 && !known_keys) return EAKV_E_INVAL;
     TurnState& T = ctx->requests[request_id];
     const int rc = turn_begin_impl(ctx, T, request_id, tokens, n_tokens, known_keys, n_known, agent_id, now_ms,
-                                   decided < 0 ? -1 : (decided ? 1 : 0), cuda_stream, view);
+                                   decided < 0 ? -1 : (decided ? 1 : 0), cuda_stream, view, layers_per_group,
+                                   events, n_events);
     if (rc != EAKV_OK) ctx->requests.erase(request_id);
     return rc;
 }

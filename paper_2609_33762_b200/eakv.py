@@ -112,6 +112,7 @@ EXPORTS = [
     "eakv_gpu_tier_acquire", "eakv_gpu_tier_release_request", "eakv_tier_step_again",
     "eakv_declined_audit", "eakv_working_set",
     "eakv_request_begin", "eakv_request_store", "eakv_request_release", "eakv_working_set_sizes", "eakv_selfcheck_fail_next_transfer", "eakv_store_layers", "eakv_turn_end_layers", "eakv_request_store_layers",
+    "eakv_turn_begin_layers", "eakv_request_begin_layers",
 ]
 STATIC_MAX_BLOCKS = 65536
 
@@ -152,6 +153,8 @@ def lib():
     L.eakv_selfcheck_fail_next_transfer.argtypes = [vp, i32]
     L.eakv_store_layers.argtypes = [vp, vp, vp, vp, i64, i32, vp, i32, vp]
     L.eakv_turn_end_layers.argtypes = [vp, i32, vp, i32, vp]
+    L.eakv_turn_begin_layers.argtypes = [vp, vp, i64, vp, i64, i64, i64, i32, vp, i32, vp, vp]
+    L.eakv_request_begin_layers.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i32, i32, vp, i32, vp, vp]
     L.eakv_request_store_layers.argtypes = [vp, i64, i32, vp, i32, vp]
     L.eakv_working_set_sizes.argtypes = [vp, i64, vp, vp, vp, i64, i32, i32, C.POINTER(i64), C.POINTER(i64), vp]
     L.eakv_working_set.argtypes = [C.POINTER(WorkingSetIn), C.POINTER(WorkingSetOut)]
@@ -526,20 +529,28 @@ class Context:
                                      C.cast(ev, C.c_void_p), len(ready_events), _stream(stream))
         self._check(rc, "eakv_store_layers")
 
-    def eakv_turn_begin(self, tokens_ptr, n_tokens, known_keys, agent_id, now_ms, stream=None):
-        """First half of a turn; returns a dict of the view's scalars and (copied) arrays."""
+    def eakv_turn_begin(self, tokens_ptr, n_tokens, known_keys, agent_id, now_ms, stream=None, layers=None):
+        """First half of a turn; returns a dict of the view's scalars and (copied) arrays.
+        ``layers`` = (layers_per_group, events): the restore runs in layer groups and records one
+        event per group (eakv_turn_begin_layers)."""
         kp, nk = None, 0
         if known_keys is not None and len(known_keys):
             kk, kp = _np(known_keys, np.uint64)
             nk = len(kk)
         v = TurnView()
-        rc = lib().eakv_turn_begin(self._h, C.c_void_p(int(tokens_ptr)), int(n_tokens), kp, nk,
-                                   int(agent_id), int(now_ms), _stream(stream), C.byref(v))
+        if layers is None:
+            rc = lib().eakv_turn_begin(self._h, C.c_void_p(int(tokens_ptr)), int(n_tokens), kp, nk,
+                                       int(agent_id), int(now_ms), _stream(stream), C.byref(v))
+        else:
+            ev = self._event_array(layers[1])
+            rc = lib().eakv_turn_begin_layers(self._h, C.c_void_p(int(tokens_ptr)), int(n_tokens), kp, nk,
+                                              int(agent_id), int(now_ms), int(layers[0]), C.cast(ev, C.c_void_p),
+                                              len(layers[1]), _stream(stream), C.byref(v))
         self._check(rc, "eakv_turn_begin")
         return self._view_dict(v)
 
     def eakv_request_begin(self, request_id, tokens_ptr, n_tokens, known_keys, agent_id, now_ms,
-                           decided=None, stream=None):
+                           decided=None, stream=None, layers=None):
         """First half of a running request's turn (its GPU blocks stay pinned until
         eakv_request_release); None when the blocks do not fit beside the running requests.
         ``decided``: None for the first lookup, else the store/skip choice made then."""
@@ -548,9 +559,15 @@ class Context:
             kk, kp = _np(known_keys, np.uint64)
             nk = len(kk)
         v = TurnView()
-        rc = lib().eakv_request_begin(self._h, int(request_id), C.c_void_p(int(tokens_ptr)), int(n_tokens), kp, nk,
-                                      int(agent_id), int(now_ms), -1 if decided is None else int(bool(decided)),
-                                      _stream(stream), C.byref(v))
+        d = -1 if decided is None else int(bool(decided))
+        if layers is None:
+            rc = lib().eakv_request_begin(self._h, int(request_id), C.c_void_p(int(tokens_ptr)), int(n_tokens), kp, nk,
+                                          int(agent_id), int(now_ms), d, _stream(stream), C.byref(v))
+        else:
+            ev = self._event_array(layers[1])
+            rc = lib().eakv_request_begin_layers(self._h, int(request_id), C.c_void_p(int(tokens_ptr)), int(n_tokens),
+                                                 kp, nk, int(agent_id), int(now_ms), d, int(layers[0]),
+                                                 C.cast(ev, C.c_void_p), len(layers[1]), _stream(stream), C.byref(v))
         if rc == E_BUSY:
             return None
         self._check(rc, "eakv_request_begin")

@@ -53,7 +53,7 @@ class PagedPool:
 class AgentServer:
     def __init__(self, shape, gpu_blocks, host_blocks, payload, *, device="cuda:0",
                  gpu_index_blocks=0, incremental_hash=False, data_plane=True, chunk_blocks=1,
-                 native_turn=None, store_layers=0, **ctx_kwargs):
+                 native_turn=None, store_layers=0, load_layers=0, **ctx_kwargs):
         """``payload(keys, q, n_words)`` returns the int16/uint16 words of piece q for the
         blocks with these keys, as a numpy array or a tensor on ``device``.  With
         ``chunk_blocks`` = R > 1 the host tier works in chunks of R blocks (``host_blocks``
@@ -61,9 +61,13 @@ class AgentServer:
         maps to block slots s*R .. s*R+R-1 for store and load.  ``store_layers`` = g > 0 (turn
         engine, data plane): the "prefill" runs on a stream of its own, g layers at a time with an
         event after each group, and the host write follows it group by group
-        (eakv_turn_end_layers / eakv_request_store_layers)."""
+        (eakv_turn_end_layers / eakv_request_store_layers).  ``load_layers`` = g > 0: the restore
+        runs in groups of g layers with one event per group (eakv_turn_begin_layers /
+        eakv_request_begin_layers); ``last_restore_events`` holds the latest turn's events."""
         self.shape = shape
         self.store_layers = int(store_layers)
+        self.load_layers = int(load_layers)
+        self.last_restore_events = []
         self._fill_stream = None
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
@@ -190,7 +194,8 @@ class AgentServer:
             known = self._agent_keys.get(agent) if self.incremental else None
             e0 = torch.cuda.Event(enable_timing=True)
             e0.record(self.stream)
-            v = self.ctx.eakv_turn_begin(self._tok_pin.data_ptr(), n, known, agent, now_ms, self.stream)
+            v = self.ctx.eakv_turn_begin(self._tok_pin.data_ptr(), n, known, agent, now_ms, self.stream,
+                                         layers=self._restore_layers())
             self._timed_since(e0, "load", (v["restore_hi"] - v["restore_lo"]) * self.ctx.block_bytes)
         else:       # bookkeeping only: the hashing context supplies every key
             v = self.ctx.eakv_turn_begin(0, n, self.block_keys(tokens, agent), agent, now_ms)
@@ -291,6 +296,16 @@ class AgentServer:
         self.records.append(rec)
         return rec
 
+    def _restore_layers(self):
+        """(layers per group, event handles) for a layered restore, or None."""
+        if self.load_layers <= 0:
+            return None
+        groups = -(-self.shape.num_layers // self.load_layers)
+        self.last_restore_events = [torch.cuda.Event() for _ in range(groups)]
+        for ev in self.last_restore_events:
+            ev.record(self.stream)                       # materialises the handle
+        return self.load_layers, [ev.cuda_event for ev in self.last_restore_events]
+
     def store(self, request_id):
         """The deferred host write of ``begin(..., defer_store=True)`` (eakv_request_store)."""
         self._request_store(request_id, self._ready.pop(request_id, None))
@@ -311,7 +326,7 @@ class AgentServer:
             self._tok_pin.numpy()[:n] = tokens
             known = self._agent_keys.get(agent) if self.incremental else None
             v = self.ctx.eakv_request_begin(request_id, self._tok_pin.data_ptr(), n, known, agent, now_ms,
-                                            decided=decided, stream=self.stream)
+                                            decided=decided, stream=self.stream, layers=self._restore_layers())
         else:
             v = self.ctx.eakv_request_begin(request_id, 0, n, self.block_keys(tokens, agent), agent, now_ms,
                                             decided=decided)

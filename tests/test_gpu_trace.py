@@ -306,7 +306,8 @@ def test_deferred_stores_interleaved_with_other_lookups_with_bytes(R, link, seed
     gpu_blocks, kh = 200, 64 // R               # a tier a few running requests overrun
     oracle = TraceOracle(shape, gpu_blocks, kh, payload=key_words_numpy, chunk_blocks=R)
     server = AgentServer(shape, gpu_blocks, kh, key_words_numpy, incremental_hash=False, chunk_blocks=R,
-                         link_strategy=link, native_turn=True, write_behind=write_behind, store_layers=layers)
+                         link_strategy=link, native_turn=True, write_behind=write_behind, store_layers=layers,
+                         load_layers=layers)
     seen = dict(begins=0, skipped=0)
 
     def check_listed_bytes():
@@ -346,9 +347,9 @@ def test_deferred_stores_interleaved_with_other_lookups_with_bytes(R, link, seed
 @pytest.mark.parametrize("cfg_name,R,policy,link,group,write_behind", [
     ("c0", 1, 0, 1, 1, False), ("c0", 1, 2, 0, 3, False), ("c0_big_tier", 4, 0, 1, 2, False), ("c0", 1, 0, 1, 4, True)])
 def test_turn_engine_with_layered_host_writes_bit_exact(cfg_name, R, policy, link, group, write_behind):
-    """The turn engine with the prefill on a stream of its own, a layer group at a time, and the
-    host write following it group by group (eakv_turn_end_layers): records and every resident byte
-    equal the oracle's."""
+    """The turn engine with the prefill on a stream of its own, a layer group at a time, the host
+    write following it group by group (eakv_turn_end_layers), and the restore in layer groups with
+    one event each (eakv_turn_begin_layers): records and every resident byte equal the oracle's."""
     from paper_2609_33762_b200.harness import AgentServer
     cfg = CONFIGS[cfg_name]
     shape = SHAPES[cfg.shape]
@@ -358,8 +359,12 @@ def test_turn_engine_with_layered_host_writes_bit_exact(cfg_name, R, policy, lin
     oracle = TraceOracle(shape, cfg.gpu_blocks, kh, payload=key_words_numpy, chunk_blocks=R, **kw)
     oracle.run(trace)
     server = AgentServer(shape, cfg.gpu_blocks, kh, key_words_numpy, native_turn=True, incremental_hash=True,
-                         chunk_blocks=R, link_strategy=link, store_layers=group, write_behind=write_behind, **kw)
+                         chunk_blocks=R, link_strategy=link, store_layers=group, load_layers=group,
+                         write_behind=write_behind, **kw)
     server.run(trace)
+    assert len(server.last_restore_events) == -(-shape.num_layers // group)
+    for ev in server.last_restore_events:
+        ev.synchronize()
     compare_records(server.records, oracle.records)
     assert server.totals == oracle.totals and oracle.totals["stored_blocks"] > 0
     compare_bytes(server, oracle)
