@@ -400,3 +400,23 @@ def test_layered_end_refuses_a_wrong_event_count_and_keeps_the_turn_open(eakv):
     ctx.eakv_request_release(7)
     assert ctx.eakv_match(more)[1] == 6
     ctx.close()
+
+
+def test_layered_begin_refuses_bad_events_before_anything_changes(eakv):
+    b = 4
+    ctx = eakv.Context(num_layers=5, kv_heads=1, head_dim=8, block_size=b, gpu_blocks=32, host_blocks=32,
+                       kv_base=None, control_plane_only=True)
+    keys = np.arange(1, 5, dtype=np.uint64)
+    before = ctx.eakv_get_stats()
+    for bad in ((2, [1, 2]), (2, [1, None, 3]), (5, [])):          # 3 events needed; a NULL one; 1 needed
+        with pytest.raises(eakv.EakvError) as ei:
+            ctx.eakv_turn_begin(0, 4 * b, keys, 0, 0, layers=bad)
+        assert ei.value.code == eakv.E_INVAL
+        with pytest.raises(eakv.EakvError) as ei:
+            ctx.eakv_request_begin(3, 0, 4 * b, keys, 0, 0, layers=bad)
+        assert ei.value.code == eakv.E_INVAL
+    assert ctx.eakv_get_stats() == before and ctx.eakv_match(keys)[:2] == (0, 0)
+    v = ctx.eakv_turn_begin(0, 4 * b, keys, 0, 0, layers=(2, [1, 2, 3]))     # (bookkeeping only: never touched)
+    assert v["admit"].tolist() == [1] * 4
+    ctx.eakv_turn_end()
+    ctx.close()
