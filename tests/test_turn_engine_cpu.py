@@ -420,3 +420,77 @@ def test_layered_begin_refuses_bad_events_before_anything_changes(eakv):
     assert v["admit"].tolist() == [1] * 4
     ctx.eakv_turn_end()
     ctx.close()
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_every_listed_unit_is_written_or_pending_under_random_begin_store_release(eakv, seed):
+    """Requests begin, store and are released in random order, some of them released before their
+    store.  A model of which slot holds whose bytes follows the views: a slot is written by the
+    store of the request that owns it, an eviction forgets it, a release before the store takes
+    the owner's pending units back.  After every call the tier lists exactly the written and the
+    pending units at those slots, and a restore only ever reads a written slot of the right key."""
+    import random
+    from deferred_util import Prompts
+    rng = random.Random(1000 + seed)
+    b = 4
+    R = rng.choice([1, 1, 2, 4])
+    kh = 60 // R + 1 + rng.choice([0, 10, 40]) // R
+    nb = rng.choice([130, 160, 220])
+    ctx = cp_ctx(eakv, b, nb, kh, chunk_blocks=R, policy=rng.choice([0, 2]), kappa_blocks=max(1, 8 // R),
+                 window_ms=20_000, len_window=8)
+    prompts = Prompts(rng, b, agents=6)
+    written, pending, begun, stored, busy = {}, {}, {}, set(), set()
+    rid = now = restored = withdrawn = 0
+    for step in range(400):
+        now += rng.randrange(0, 3000)
+        choices = []
+        if len(begun) < 5 and len(busy) < 6:
+            choices += ["begin"] * 3
+        if any(r not in stored for r in begun):
+            choices += ["store"] * 2
+        if begun:
+            choices += ["release"] * 2
+        op = rng.choice(choices)
+        if op == "begin":
+            agent = rng.choice([a for a in range(6) if a not in busy])
+            rid += 1
+            toks = prompts.next_prompt(agent, 60 * b)
+            keys = keys_of(toks, b)
+            v = ctx.eakv_request_begin(rid, 0, len(toks), keys, agent, now)
+            if v is None:
+                continue
+            ukeys = [int(k) for k in keys[R - 1::R]]
+            for k in v["evicted_keys"].tolist():
+                written.pop(k, None)
+                pending.pop(k, None)
+            if v["restore_hi"] > v["restore_lo"]:
+                for c in range(v["restore_lo"] // R, -(-v["restore_hi"] // R)):
+                    assert written.get(ukeys[c]) == int(v["slot"][c]), "restore of a slot that was never written"
+                    restored += 1
+            for c, a in enumerate(v["admit"].tolist()):
+                if a:
+                    pending[ukeys[c]] = (rid, int(v["slot"][c]))
+            begun[rid] = agent
+            busy.add(agent)
+        elif op == "store":
+            r = rng.choice([r for r in begun if r not in stored])
+            ctx.eakv_request_store(r)
+            stored.add(r)
+            for k, (owner, s) in list(pending.items()):
+                if owner == r:
+                    written[k] = s
+                    del pending[k]
+        else:
+            r = rng.choice(list(begun))
+            ctx.eakv_request_release(r)
+            if r not in stored:
+                for k, (owner, s) in list(pending.items()):
+                    if owner == r:
+                        del pending[k]
+                        withdrawn += 1
+            stored.discard(r)
+            busy.discard(begun.pop(r))
+        ek, es = ctx.eakv_tier_export()
+        assert dict(zip(ek.tolist(), es.tolist())) == {**written, **{k: s for k, (_, s) in pending.items()}}, step
+    assert withdrawn > 0
+    ctx.close()
