@@ -484,6 +484,103 @@ def test_write_behind_orders_block_reuse_and_slot_reads():
     ctx.close()
 
 
+@pytest.mark.parametrize("R,link,seed", [(1, 1, 21), (2, 0, 22), (1, 1, 23)])
+def test_written_units_hold_their_payload_under_random_begin_store_release(R, link, seed):
+    """Requests begin, store and are released in random order on the GPU path with bytes, some of
+    them released before their store (their pending units are taken back).  A model follows the
+    views (a slot is written by the store of the request that owns it; an eviction forgets it);
+    after every store each written unit's slot must hold the payload of its blocks' keys, and
+    every restored GPU block the payload of the key it was restored for."""
+    import random
+    from deferred_util import Prompts
+    from paper_2609_33762_b200.harness import AgentServer
+    shape = SHAPES["tiny"]
+    b = shape.block_size
+    W = shape.piece_bytes // 2
+    rng = random.Random(seed)
+    kh, nb = 64 // R + 4, 220
+    server = AgentServer(shape, nb, kh, key_words_numpy, incremental_hash=False, chunk_blocks=R,
+                         link_strategy=link, native_turn=True)
+    prompts = Prompts(rng, b, agents=6)
+    written, pending, begun, stored, busy, unit_blocks = {}, {}, {}, set(), set(), {}
+    rid = now = withdrawn = restored = 0
+
+    def payload_of(keys):
+        return [key_words_numpy(np.asarray(keys, dtype=np.uint64), q, W) for q in range(shape.pieces_per_block)]
+
+    def check_written():
+        server.ctx.eakv_sync()
+        tier = server.ctx.tier_host_view().view(np.uint16)
+        for ukey, slot in written.items():
+            want = payload_of(unit_blocks[ukey])
+            for i in range(R):
+                for q in range(shape.pieces_per_block):
+                    assert np.array_equal(tier[slot * R + i, q], want[q][i]), (ukey, slot, i, q)
+
+    for step in range(220):
+        now += rng.randrange(0, 3000)
+        choices = []
+        if len(begun) < 4 and len(busy) < 6:
+            choices += ["begin"] * 3
+        if any(r not in stored for r in begun):
+            choices += ["store"] * 2
+        if begun:
+            choices += ["release"] * 2
+        op = rng.choice(choices)
+        if op == "begin":
+            agent = rng.choice([a for a in range(6) if a not in busy])
+            rid += 1
+            toks = prompts.next_prompt(agent, 60 * b)
+            rec = server.begin(rid, toks, agent, now, defer_store=True)
+            if rec is None:
+                continue
+            keys = [int(k) for k in rec["keys"]]
+            ukeys = keys[R - 1::R]
+            for c, uk in enumerate(ukeys):
+                unit_blocks[uk] = keys[c * R:(c + 1) * R]
+            for k, _ in rec["evicted"]:
+                written.pop(int(k), None)
+                pending.pop(int(k), None)
+            if rec["loaded"]:
+                lo = rec["G"]
+                ids = torch.as_tensor(np.asarray(rec["gpu_block"][lo:lo + rec["loaded"]], dtype=np.int64), device="cuda")
+                want = payload_of(keys[lo:lo + rec["loaded"]])
+                torch.cuda.synchronize()
+                for q in (0, shape.pieces_per_block - 1):
+                    got = server.pool.pieces[q][ids].cpu().numpy().view(np.uint16)
+                    assert np.array_equal(got, want[q])
+                restored += rec["loaded"]
+            for c, a in enumerate(rec["admit"]):
+                if a:
+                    pending[ukeys[c]] = (rid, int(rec["slot"][c]))
+            begun[rid] = agent
+            busy.add(agent)
+        elif op == "store":
+            r = rng.choice([r for r in begun if r not in stored])
+            server.store(r)
+            stored.add(r)
+            for k, (owner, sl) in list(pending.items()):
+                if owner == r:
+                    written[k] = sl
+                    del pending[k]
+            check_written()
+        else:
+            r = rng.choice(list(begun))
+            server.finish(r)
+            if r not in stored:
+                for k, (owner, sl) in list(pending.items()):
+                    if owner == r:
+                        del pending[k]
+                        withdrawn += 1
+            stored.discard(r)
+            busy.discard(begun.pop(r))
+    check_written()
+    ek, es = server.ctx.eakv_tier_export()
+    assert dict(zip(ek.tolist(), es.tolist())) == {**written, **{k: sl for k, (_, sl) in pending.items()}}
+    assert withdrawn > 0 and restored > 0
+    server.close()
+
+
 def test_a_failed_store_or_restore_leaves_no_stale_slot_readable():
     """With bytes: a store that fails in eakv_turn_end (made to fail on the host) withdraws the
     turn's units, so that the same prompt afterwards is computed and stored again rather than
