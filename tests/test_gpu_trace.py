@@ -498,7 +498,7 @@ def test_written_units_hold_their_payload_under_random_begin_store_release(R, li
     b = shape.block_size
     W = shape.piece_bytes // 2
     rng = random.Random(seed)
-    kh, nb = 64 // R + 4, 220
+    kh, nb, max_blocks = 120 // R, 60, 30       # the host tier outlives the GPU tier (restores) and still evicts
     server = AgentServer(shape, nb, kh, key_words_numpy, incremental_hash=False, chunk_blocks=R,
                          link_strategy=link, native_turn=True)
     prompts = Prompts(rng, b, agents=6)
@@ -517,7 +517,7 @@ def test_written_units_hold_their_payload_under_random_begin_store_release(R, li
                 for q in range(shape.pieces_per_block):
                     assert np.array_equal(tier[slot * R + i, q], want[q][i]), (ukey, slot, i, q)
 
-    for step in range(220):
+    for step in range(300):
         now += rng.randrange(0, 3000)
         choices = []
         if len(begun) < 4 and len(busy) < 6:
@@ -530,7 +530,7 @@ def test_written_units_hold_their_payload_under_random_begin_store_release(R, li
         if op == "begin":
             agent = rng.choice([a for a in range(6) if a not in busy])
             rid += 1
-            toks = prompts.next_prompt(agent, 60 * b)
+            toks = prompts.next_prompt(agent, max_blocks * b)
             rec = server.begin(rid, toks, agent, now, defer_store=True)
             if rec is None:
                 continue
