@@ -104,7 +104,7 @@ def test_no_cpu_fallback_without_a_gpu(lib):
 
 def test_a_plain_c_client_compiles_and_links(tmp_path):
     """The header is a C99 header and the library resolves every call a C client makes
-    (tests/c_client/five_calls.c; it is run on a GPU by tests/test_gpu_c_client.py)."""
+    (tests/c_client/five_calls.c and turn_calls.c; they are run on a GPU by tests/test_gpu_c_client.py)."""
     import shutil
     import subprocess
     cuda = os.environ.get("CUDA_HOME", "/usr/local/cuda")
@@ -113,10 +113,11 @@ def test_a_plain_c_client_compiles_and_links(tmp_path):
     here = os.path.dirname(os.path.abspath(__file__))
     root = os.path.dirname(here)
     pkg = os.path.join(root, "paper_2609_33762_b200")
-    exe = os.path.join(str(tmp_path), "five_calls")
-    cmd = ["gcc", "-std=c99", "-Wall", "-Werror", "-O1", os.path.join(here, "c_client", "five_calls.c"),
-           "-I" + os.path.join(root, "include"), "-I" + os.path.join(cuda, "include"),
-           "-L" + pkg, "-leakv", "-L" + os.path.join(cuda, "lib64"), "-lcudart", "-Wl,-rpath," + pkg, "-o", exe]
-    run = subprocess.run(cmd, capture_output=True, text=True)
-    assert run.returncode == 0, run.stderr
-    assert os.path.exists(exe)
+    for name in ("five_calls", "turn_calls"):
+        exe = os.path.join(str(tmp_path), name)
+        cmd = ["gcc", "-std=c99", "-Wall", "-Werror", "-O1", os.path.join(here, "c_client", name + ".c"),
+               "-I" + os.path.join(root, "include"), "-I" + os.path.join(cuda, "include"),
+               "-L" + pkg, "-leakv", "-L" + os.path.join(cuda, "lib64"), "-lcudart", "-Wl,-rpath," + pkg, "-o", exe]
+        run = subprocess.run(cmd, capture_output=True, text=True)
+        assert run.returncode == 0, run.stderr
+        assert os.path.exists(exe)

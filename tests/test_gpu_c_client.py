@@ -19,9 +19,9 @@ PKG = os.path.join(ROOT, "paper_2609_33762_b200")
 CUDA = os.environ.get("CUDA_HOME", "/usr/local/cuda")
 
 
-def build_client(out_dir):
-    exe = os.path.join(str(out_dir), "five_calls")
-    cmd = ["gcc", "-std=c99", "-Wall", "-Werror", "-O1", os.path.join(HERE, "c_client", "five_calls.c"),
+def build_client(out_dir, name="five_calls"):
+    exe = os.path.join(str(out_dir), name)
+    cmd = ["gcc", "-std=c99", "-Wall", "-Werror", "-O1", os.path.join(HERE, "c_client", name + ".c"),
            "-I" + os.path.join(ROOT, "include"), "-I" + os.path.join(CUDA, "include"),
            "-L" + PKG, "-leakv", "-L" + os.path.join(CUDA, "lib64"), "-lcudart",
            "-Wl,-rpath," + PKG, "-Wl,-rpath," + os.path.join(CUDA, "lib64"), "-o", exe]
@@ -45,3 +45,22 @@ def test_plain_c_client_runs_the_five_calls(tmp_path):
     assert lines["match2"] == "0 6"                              # every block is now a host hit
     assert lines["roundtrip"] == "ok" and lines["untouched"] == "ok"
     assert lines["stats"] == "stored=6 loaded=6"
+
+
+def test_plain_c_client_runs_the_turn_engine(tmp_path):
+    """tests/c_client/turn_calls.c: three turns through eakv_turn_begin / eakv_turn_end, the third
+    one restored from the host tier inside the library; the view it prints is what the paper's
+    definitions give for those prompts, and the new block's key is the oracle's."""
+    require_gpu()
+    exe = build_client(tmp_path, "turn_calls")
+    run = subprocess.run([exe], capture_output=True, text=True, timeout=300)
+    assert run.returncode == 0, run.stdout + run.stderr
+    lines = dict(l.split(" ", 1) for l in run.stdout.strip().splitlines())
+    # 6 blocks + 4 tokens, nothing cached; then 8 other blocks fill the 8-block GPU tier; then the
+    # first prompt with 7 full blocks: 6 from the host, one new
+    assert lines["turn1"] == "blocks=6 G=0 H=0 restore=0..0 fresh=100 fill=6 store=6 tail=1"
+    assert lines["turn2"] == "blocks=8 G=0 H=0 restore=0..0 fresh=128 fill=8 store=8 tail=0"
+    assert lines["turn3"] == "blocks=7 G=0 H=6 restore=0..6 fresh=16 fill=1 store=1 tail=0"
+    assert lines["restored"] == "ok"
+    tokens = [(i * 2246822519 % (1 << 32)) % 40000 for i in range(7 * 16)]
+    assert int(lines["key7"], 16) == int(ohash.hash_blocks(tokens, 16)[6])
