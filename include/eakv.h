@@ -286,6 +286,8 @@ int eakv_tier_step_again(eakv_ctx* ctx, const uint64_t* hashes_host, int64_t n_b
  * with the process), the counters, and the admission windows, which have a pair of calls of their
  * own below (without them they restart empty and capacity-conditioned admission may decide
  * differently until they refill).
+ * The list names every unit the index holds, including those an open turn or request has admitted
+ * but not written yet: for a restart, export when no turn or request is open (and after eakv_sync).
  * E_INVAL: tier not empty, a repeated key or slot, a slot outside the tier; nothing changes. */
 int eakv_tier_export(const eakv_ctx* ctx, uint64_t* keys_host_out, int32_t* slots_host_out,
                      int64_t capacity, int64_t* n_out);
