@@ -122,6 +122,15 @@ struct eakv_ctx {
     bool wb_pending = false;
     std::vector<uint8_t> wb_blocks;     // by GPU block: a pending write still reads it
     std::vector<uint8_t> wb_slots;      // by tier slot: a pending write still fills it
+    // restores in flight: a later store into a slot that a restore on another stream may still be
+    // reading waits for rd_done (the paper's tier frees no chunk that a transfer still references;
+    // here the bookkeeping may hand the slot on, and the write is ordered behind the read instead)
+    static constexpr int kRdRing = 16;  // events of the latest restores, by sequence number modulo this
+    cudaEvent_t rd_ev[kRdRing] = {};
+    cudaStream_t rd_ev_stream[kRdRing] = {};
+    uint64_t rd_ev_seq[kRdRing] = {};   // sequence number of the restore the event was last recorded behind
+    uint64_t rd_next = 1;               // sequence number of the next restore
+    std::vector<uint64_t> rd_slot_seq;  // by tier slot: the last restore that reads it (0: none)
     uint64_t* turn_keys = nullptr;            // pinned + mapped; the hash kernel writes it directly
     int64_t turn_keys_cap = 0;
     TurnState turn;                            // the one open turn of eakv_turn_begin / eakv_turn_end
@@ -200,6 +209,8 @@ void free_all(eakv_ctx* c) {
     if (c->wb_stream) cudaStreamDestroy(c->wb_stream);
     if (c->wb_fence) cudaEventDestroy(c->wb_fence);
     if (c->wb_done) cudaEventDestroy(c->wb_done);
+    for (cudaEvent_t e : c->rd_ev)
+        if (e) cudaEventDestroy(e);
     if (c->tier && c->tier_owned) {
         if (c->cfg.tier_location == EAKV_TIER_DEVICE) cudaFree(c->tier);
         else cudaFreeHost(c->tier);
@@ -335,6 +346,45 @@ int wait_write_behind(eakv_ctx* ctx, cudaStream_t stream) {
     }
     cudaGetLastError();            // cudaErrorNotReady is not an error here
     CU(cudaStreamWaitEvent(stream, ctx->wb_done, 0));
+    return EAKV_OK;
+}
+
+// Restores in flight (see eakv_ctx::rd_ev).  Every restore gets a sequence number; an event is
+// recorded behind it in ring slot (number mod ring size), and its slots remember the number.
+// When a ring slot is reused, the new restore's event is recorded behind a wait for the old one, so
+// whatever event a ring slot holds completes only after every earlier restore that used the slot.
+// A store looks at the numbers of the slots it overwrites and waits for those restores' events,
+// unless they were recorded on the store's own stream (already in order) or have completed.
+int restore_enqueued(eakv_ctx* ctx, const std::vector<int2>& ent, cudaStream_t stream) {
+    if (ctx->rd_slot_seq.empty()) ctx->rd_slot_seq.assign((size_t)ctx->tier_slots, 0);
+    const uint64_t seq = ctx->rd_next++;
+    const int idx = (int)(seq % eakv_ctx::kRdRing);
+    if (!ctx->rd_ev[idx]) CU(cudaEventCreateWithFlags(&ctx->rd_ev[idx], cudaEventDisableTiming));
+    else if (ctx->rd_ev_stream[idx] != stream) CU(cudaStreamWaitEvent(stream, ctx->rd_ev[idx], 0));
+    CU(cudaEventRecord(ctx->rd_ev[idx], stream));
+    ctx->rd_ev_stream[idx] = stream;
+    ctx->rd_ev_seq[idx] = seq;
+    for (const int2& e : ent) ctx->rd_slot_seq[e.y] = seq;
+    return EAKV_OK;
+}
+
+int store_after_restores(eakv_ctx* ctx, const std::vector<int2>& ent, cudaStream_t stream) {
+    if (ctx->rd_slot_seq.empty()) return EAKV_OK;          // nothing was ever restored
+    bool need[eakv_ctx::kRdRing] = {};
+    bool any = false;
+    for (const int2& e : ent) {
+        const uint64_t q = ctx->rd_slot_seq[e.y];
+        if (q) { need[q % eakv_ctx::kRdRing] = true; any = true; }
+    }
+    if (!any) return EAKV_OK;
+    for (int idx = 0; idx < eakv_ctx::kRdRing; ++idx) {
+        if (!need[idx] || ctx->rd_ev_stream[idx] == stream) continue;
+        if (cudaEventQuery(ctx->rd_ev[idx]) == cudaSuccess) continue;
+        cudaGetLastError();                                // cudaErrorNotReady is not an error here
+        CU(cudaStreamWaitEvent(stream, ctx->rd_ev[idx], 0));
+    }
+    // the slots are about to hold other bytes: their old readers no longer matter once this store is ordered
+    for (const int2& e : ent) ctx->rd_slot_seq[e.y] = 0;
     return EAKV_OK;
 }
 
@@ -1153,6 +1203,8 @@ int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_m
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     int rc = wait_write_behind(ctx, stream);
     if (rc != EAKV_OK) return rc;
+    rc = store_after_restores(ctx, ent, stream);
+    if (rc != EAKV_OK) return rc;
     rc = move_blocks(ctx, ent, true, stream, 0, ctx->pieces);
     if (rc != EAKV_OK) return rc;
     ctx->stats.blocks_stored += m;
@@ -1187,6 +1239,8 @@ int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_tab
         if (rc != EAKV_OK) return rc;
     }
     rc = move_blocks(ctx, ent, false, stream, 0, ctx->pieces);
+    if (rc != EAKV_OK) return rc;
+    rc = restore_enqueued(ctx, ent, stream);
     if (rc != EAKV_OK) return rc;
     ctx->stats.blocks_loaded += m;
     ctx->stats.bytes_loaded += m * ctx->block_bytes;
@@ -1233,6 +1287,10 @@ int eakv_load_layers(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* bl
         }
         CU(cudaEventRecord(static_cast<cudaEvent_t>(events[grp]), stream));
     }
+    if (n_blocks > 0) {
+        const int rcr = restore_enqueued(ctx, ent, stream);
+        if (rcr != EAKV_OK) return rcr;
+    }
     ctx->stats.blocks_loaded += n_blocks;
     ctx->stats.bytes_loaded += n_blocks * ctx->block_bytes;
     return EAKV_OK;
@@ -1262,7 +1320,9 @@ int eakv_store_layers(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* 
     DeviceGuard g(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (m > 0) {
-        const int rcw = wait_write_behind(ctx, stream);
+        int rcw = wait_write_behind(ctx, stream);
+        if (rcw != EAKV_OK) return rcw;
+        rcw = store_after_restores(ctx, ent, stream);
         if (rcw != EAKV_OK) return rcw;
     }
     for (int grp = 0; grp < groups; ++grp) {

@@ -669,6 +669,47 @@ def test_write_behind_orders_a_direct_load_of_pending_slots():
     ctx.close()
 
 
+@pytest.mark.parametrize("link", [1, 0], ids=["staged", "zero-copy"])
+def test_a_store_waits_for_a_restore_on_another_stream_that_reads_its_slots(link):
+    """The bookkeeping may hand a slot on while a restore enqueued on another stream still reads it
+    (several lookups can pass while 0.9 GiB cross the link).  The library orders the write behind
+    that read: the restore must deliver the old bytes, the tier must end up with the new ones."""
+    from paper_2609_33762_b200 import eakv
+    from paper_2609_33762_b200.harness import PagedPool
+    shape = SHAPES["qwen3_30b_a3b"]
+    nb, kh, m = 2000, 700, 640
+    pool = PagedPool(shape, nb, "cuda:0")
+    ctx = eakv.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
+                       block_size=shape.block_size, gpu_blocks=nb, host_blocks=kh, kv_base=pool.kv_base,
+                       link_strategy=link)
+    a, b_, c = (np.arange(m, dtype=np.int32) + k * m for k in range(3))       # three disjoint block sets
+    slots = np.arange(m, dtype=np.int32)
+    for blocks, value in ((a, 0x1111), (b_, 0x2222), (c, 0x3333)):
+        ids = torch.as_tensor(blocks.astype(np.int64), device="cuda")
+        for piece in pool.pieces:
+            piece[ids] = value
+    torch.cuda.synchronize()
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    ctx.eakv_store(a, None, slots, sa)                   # the slots hold 0x1111
+    ctx.eakv_sync()
+    ctx.eakv_load(slots, c, sa)                          # restore them into set c on one stream ...
+    ctx.eakv_store(b_, None, slots[::-1].copy(), sb)     # ... and at once overwrite them from another
+    ctx.eakv_sync()
+    torch.cuda.synchronize()
+    ids = torch.as_tensor(c.astype(np.int64), device="cuda")
+    for piece in pool.pieces[::7]:
+        assert bool((piece[ids].view(torch.int16) == 0x1111).all())
+    tier = ctx.tier_host_view().view(np.uint16)
+    assert (tier[slots] == 0x2222).all()
+    # the same stream needs no wait and a later restore sees the new bytes
+    ctx.eakv_load(slots, a, sb)
+    ctx.eakv_sync()
+    ids = torch.as_tensor(a.astype(np.int64), device="cuda")
+    for piece in pool.pieces[::7]:
+        assert bool((piece[ids].view(torch.int16) == 0x2222).all())
+    ctx.close()
+
+
 def test_random_traces_with_bytes_across_options():
     """Small random traces with KV bytes through combinations of policy, chunking, link strategy,
     copy path, GPU free order, the turn engine and deferred writes: records and resident bytes
