@@ -28,7 +28,11 @@
  *   - A context is not thread-safe.  Two calls of the same kind (hash, store, load) on
  *     one context must be ordered with respect to each other (same stream, or an event
  *     between them): each kind has one set of scratch / staging buffers.  A store and a
- *     load may run concurrently on two streams when they touch different slots/blocks.
+ *     load may run concurrently on two streams.  Where they meet in a tier slot the library
+ *     orders them itself: a store into a slot that a restore enqueued earlier (on another
+ *     stream) still reads waits for that restore, and a restore of a slot that a store enqueued
+ *     earlier still fills waits for that store.  GPU blocks are the caller's: a block must not
+ *     be overwritten while a store enqueued on another stream still reads it.
  *   - Layouts: the paged pool is 2L separate arrays, kv_base[2*l] = layer l's K and
  *     kv_base[2*l+1] = its V, each [gpu_blocks][block_size][kv_heads][head_dim] of
  *     elem_bytes-sized elements; one such [block_size][kv_heads][head_dim] slab is a
@@ -439,8 +443,7 @@ int eakv_turn_abort(eakv_ctx* ctx);
  * what was written); the bookkeeping is that of the reference model either way, which registers a
  * write at its lookup.  A release before the store takes back only the units the request still
  * owns.  After the store they are
- * restorable; a restore by another request must be ordered after that store on the GPU (same
- * stream, or an event), as for any store followed by a load of the same slots.  The GPU side has
+ * restorable (a restore enqueued on another stream waits for that store).  The GPU side has
  * no such guard: a block that an open request was told to fill counts as resident for a later
  * request with the same prefix (the two share it), so an engine that runs both must let the
  * second one read that block only after the first one's fill (stream order or an event).

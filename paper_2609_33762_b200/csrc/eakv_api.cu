@@ -61,6 +61,60 @@ struct TurnState {
 };
 }  // namespace
 
+// Which transfers of one direction may still be running, by tier slot.  Every transfer gets a
+// sequence number; an event is recorded behind it in ring slot (number mod ring size) and the tier
+// slots it touches remember the number.  When a ring slot is reused, the new event is recorded
+// behind a wait for the old one, so whatever event a ring slot holds completes only after every
+// earlier transfer that used that ring slot.  `done` trails the numbers known to be complete.
+struct SlotOrder {
+    static constexpr int kRing = 16;
+    cudaEvent_t ev[kRing] = {};
+    cudaStream_t ev_stream[kRing] = {};
+    uint64_t next = 1, done = 0;
+    std::vector<uint64_t> slot_seq;        // by tier slot: the last transfer that touched it (0: none)
+
+    // after a transfer over the slots ent[].y was enqueued on `stream`
+    cudaError_t enqueued(const std::vector<int2>& ent, int64_t tier_slots, cudaStream_t stream) {
+        if (slot_seq.empty()) slot_seq.assign((size_t)tier_slots, 0);
+        const uint64_t seq = next++;
+        const int idx = (int)(seq % kRing);
+        cudaError_t e = cudaSuccess;
+        if (!ev[idx]) e = cudaEventCreateWithFlags(&ev[idx], cudaEventDisableTiming);
+        else if (ev_stream[idx] != stream) e = cudaStreamWaitEvent(stream, ev[idx], 0);
+        if (e != cudaSuccess) return e;
+        e = cudaEventRecord(ev[idx], stream);
+        if (e != cudaSuccess) return e;
+        ev_stream[idx] = stream;
+        for (const int2& x : ent) slot_seq[x.y] = seq;
+        return cudaSuccess;
+    }
+    // before a transfer of the other direction over these slots is enqueued on `stream`: wait for
+    // the transfers that touched them, unless complete or recorded on `stream` itself (in order)
+    cudaError_t order_after(const std::vector<int2>& ent, cudaStream_t stream, bool forget) {
+        if (slot_seq.empty()) return cudaSuccess;
+        while (done + 1 < next && cudaEventQuery(ev[(done + 1) % kRing]) == cudaSuccess) ++done;
+        cudaGetLastError();                                // cudaErrorNotReady is not an error here
+        bool need[kRing] = {};
+        bool any = false;
+        for (const int2& x : ent) {
+            const uint64_t q = slot_seq[x.y];
+            if (q > done) { need[q % kRing] = true; any = true; }
+            if (forget) slot_seq[x.y] = 0;
+        }
+        if (!any) return cudaSuccess;
+        for (int idx = 0; idx < kRing; ++idx) {
+            if (!need[idx] || ev_stream[idx] == stream) continue;
+            const cudaError_t e = cudaStreamWaitEvent(stream, ev[idx], 0);
+            if (e != cudaSuccess) return e;
+        }
+        return cudaSuccess;
+    }
+    void destroy() {
+        for (cudaEvent_t& e : ev)
+            if (e) { cudaEventDestroy(e); e = nullptr; }
+    }
+};
+
 struct eakv_ctx {
     eakv_config cfg;
     int device = 0;
@@ -122,15 +176,12 @@ struct eakv_ctx {
     bool wb_pending = false;
     std::vector<uint8_t> wb_blocks;     // by GPU block: a pending write still reads it
     std::vector<uint8_t> wb_slots;      // by tier slot: a pending write still fills it
-    // restores in flight: a later store into a slot that a restore on another stream may still be
-    // reading waits for rd_done (the paper's tier frees no chunk that a transfer still references;
-    // here the bookkeeping may hand the slot on, and the write is ordered behind the read instead)
-    static constexpr int kRdRing = 16;  // events of the latest restores, by sequence number modulo this
-    cudaEvent_t rd_ev[kRdRing] = {};
-    cudaStream_t rd_ev_stream[kRdRing] = {};
-    uint64_t rd_ev_seq[kRdRing] = {};   // sequence number of the restore the event was last recorded behind
-    uint64_t rd_next = 1;               // sequence number of the next restore
-    std::vector<uint64_t> rd_slot_seq;  // by tier slot: the last restore that reads it (0: none)
+    // Transfers in flight, by tier slot: a store into a slot that a restore on another stream may
+    // still be reading waits for that restore, and a restore of a slot that a store on another
+    // stream may still be writing waits for that store (the paper's tier frees no chunk that a
+    // transfer still references; here the bookkeeping may hand the slot on, and the streams are
+    // ordered instead).
+    SlotOrder restores, stores;
     uint64_t* turn_keys = nullptr;            // pinned + mapped; the hash kernel writes it directly
     int64_t turn_keys_cap = 0;
     TurnState turn;                            // the one open turn of eakv_turn_begin / eakv_turn_end
@@ -209,8 +260,8 @@ void free_all(eakv_ctx* c) {
     if (c->wb_stream) cudaStreamDestroy(c->wb_stream);
     if (c->wb_fence) cudaEventDestroy(c->wb_fence);
     if (c->wb_done) cudaEventDestroy(c->wb_done);
-    for (cudaEvent_t e : c->rd_ev)
-        if (e) cudaEventDestroy(e);
+    c->restores.destroy();
+    c->stores.destroy();
     if (c->tier && c->tier_owned) {
         if (c->cfg.tier_location == EAKV_TIER_DEVICE) cudaFree(c->tier);
         else cudaFreeHost(c->tier);
@@ -346,45 +397,6 @@ int wait_write_behind(eakv_ctx* ctx, cudaStream_t stream) {
     }
     cudaGetLastError();            // cudaErrorNotReady is not an error here
     CU(cudaStreamWaitEvent(stream, ctx->wb_done, 0));
-    return EAKV_OK;
-}
-
-// Restores in flight (see eakv_ctx::rd_ev).  Every restore gets a sequence number; an event is
-// recorded behind it in ring slot (number mod ring size), and its slots remember the number.
-// When a ring slot is reused, the new restore's event is recorded behind a wait for the old one, so
-// whatever event a ring slot holds completes only after every earlier restore that used the slot.
-// A store looks at the numbers of the slots it overwrites and waits for those restores' events,
-// unless they were recorded on the store's own stream (already in order) or have completed.
-int restore_enqueued(eakv_ctx* ctx, const std::vector<int2>& ent, cudaStream_t stream) {
-    if (ctx->rd_slot_seq.empty()) ctx->rd_slot_seq.assign((size_t)ctx->tier_slots, 0);
-    const uint64_t seq = ctx->rd_next++;
-    const int idx = (int)(seq % eakv_ctx::kRdRing);
-    if (!ctx->rd_ev[idx]) CU(cudaEventCreateWithFlags(&ctx->rd_ev[idx], cudaEventDisableTiming));
-    else if (ctx->rd_ev_stream[idx] != stream) CU(cudaStreamWaitEvent(stream, ctx->rd_ev[idx], 0));
-    CU(cudaEventRecord(ctx->rd_ev[idx], stream));
-    ctx->rd_ev_stream[idx] = stream;
-    ctx->rd_ev_seq[idx] = seq;
-    for (const int2& e : ent) ctx->rd_slot_seq[e.y] = seq;
-    return EAKV_OK;
-}
-
-int store_after_restores(eakv_ctx* ctx, const std::vector<int2>& ent, cudaStream_t stream) {
-    if (ctx->rd_slot_seq.empty()) return EAKV_OK;          // nothing was ever restored
-    bool need[eakv_ctx::kRdRing] = {};
-    bool any = false;
-    for (const int2& e : ent) {
-        const uint64_t q = ctx->rd_slot_seq[e.y];
-        if (q) { need[q % eakv_ctx::kRdRing] = true; any = true; }
-    }
-    if (!any) return EAKV_OK;
-    for (int idx = 0; idx < eakv_ctx::kRdRing; ++idx) {
-        if (!need[idx] || ctx->rd_ev_stream[idx] == stream) continue;
-        if (cudaEventQuery(ctx->rd_ev[idx]) == cudaSuccess) continue;
-        cudaGetLastError();                                // cudaErrorNotReady is not an error here
-        CU(cudaStreamWaitEvent(stream, ctx->rd_ev[idx], 0));
-    }
-    // the slots are about to hold other bytes: their old readers no longer matter once this store is ordered
-    for (const int2& e : ent) ctx->rd_slot_seq[e.y] = 0;
     return EAKV_OK;
 }
 
@@ -1203,10 +1215,10 @@ int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_m
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     int rc = wait_write_behind(ctx, stream);
     if (rc != EAKV_OK) return rc;
-    rc = store_after_restores(ctx, ent, stream);
-    if (rc != EAKV_OK) return rc;
+    CU(ctx->restores.order_after(ent, stream, true));    // the slots are about to hold other bytes
     rc = move_blocks(ctx, ent, true, stream, 0, ctx->pieces);
     if (rc != EAKV_OK) return rc;
+    CU(ctx->stores.enqueued(ent, ctx->tier_slots, stream));
     ctx->stats.blocks_stored += m;
     ctx->stats.bytes_stored += m * ctx->block_bytes;
     return EAKV_OK;
@@ -1238,10 +1250,10 @@ int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_tab
         if (touches) rc = wait_write_behind(ctx, stream);
         if (rc != EAKV_OK) return rc;
     }
+    CU(ctx->stores.order_after(ent, stream, false));
     rc = move_blocks(ctx, ent, false, stream, 0, ctx->pieces);
     if (rc != EAKV_OK) return rc;
-    rc = restore_enqueued(ctx, ent, stream);
-    if (rc != EAKV_OK) return rc;
+    CU(ctx->restores.enqueued(ent, ctx->tier_slots, stream));
     ctx->stats.blocks_loaded += m;
     ctx->stats.bytes_loaded += m * ctx->block_bytes;
     return EAKV_OK;
@@ -1278,6 +1290,7 @@ int eakv_load_layers(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* bl
             if (rcw != EAKV_OK) return rcw;
         }
     }
+    if (n_blocks > 0) CU(ctx->stores.order_after(ent, stream, false));
     for (int grp = 0; grp < groups; ++grp) {
         const int l0 = grp * layers_per_group;
         const int l1 = std::min(L, l0 + layers_per_group);
@@ -1287,10 +1300,7 @@ int eakv_load_layers(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* bl
         }
         CU(cudaEventRecord(static_cast<cudaEvent_t>(events[grp]), stream));
     }
-    if (n_blocks > 0) {
-        const int rcr = restore_enqueued(ctx, ent, stream);
-        if (rcr != EAKV_OK) return rcr;
-    }
+    if (n_blocks > 0) CU(ctx->restores.enqueued(ent, ctx->tier_slots, stream));
     ctx->stats.blocks_loaded += n_blocks;
     ctx->stats.bytes_loaded += n_blocks * ctx->block_bytes;
     return EAKV_OK;
@@ -1322,8 +1332,7 @@ int eakv_store_layers(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* 
     if (m > 0) {
         int rcw = wait_write_behind(ctx, stream);
         if (rcw != EAKV_OK) return rcw;
-        rcw = store_after_restores(ctx, ent, stream);
-        if (rcw != EAKV_OK) return rcw;
+        CU(ctx->restores.order_after(ent, stream, true));
     }
     for (int grp = 0; grp < groups; ++grp) {
         const int l0 = grp * layers_per_group;
@@ -1335,6 +1344,7 @@ int eakv_store_layers(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* 
             if (rc != EAKV_OK) return rc;
         }
     }
+    if (m > 0) CU(ctx->stores.enqueued(ent, ctx->tier_slots, stream));
     ctx->stats.blocks_stored += m;
     ctx->stats.bytes_stored += m * ctx->block_bytes;
     return EAKV_OK;

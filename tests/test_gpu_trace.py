@@ -673,7 +673,8 @@ def test_write_behind_orders_a_direct_load_of_pending_slots():
 def test_a_store_waits_for_a_restore_on_another_stream_that_reads_its_slots(link):
     """The bookkeeping may hand a slot on while a restore enqueued on another stream still reads it
     (several lookups can pass while 0.9 GiB cross the link).  The library orders the write behind
-    that read: the restore must deliver the old bytes, the tier must end up with the new ones."""
+    that read: the restore must deliver the old bytes, the tier must end up with the new ones.
+    Likewise a restore enqueued on another stream while a store still fills its slots waits for it."""
     from paper_2609_33762_b200 import eakv
     from paper_2609_33762_b200.harness import PagedPool
     shape = SHAPES["qwen3_30b_a3b"]
@@ -707,6 +708,14 @@ def test_a_store_waits_for_a_restore_on_another_stream_that_reads_its_slots(link
     ids = torch.as_tensor(a.astype(np.int64), device="cuda")
     for piece in pool.pieces[::7]:
         assert bool((piece[ids].view(torch.int16) == 0x2222).all())
+    # and the other way round: a restore, on another stream, of slots that a store is still filling
+    ctx.eakv_store(c, None, slots, sa)                   # (set c holds 0x1111 since the first restore)
+    ctx.eakv_load(slots[::-1].copy(), b_, sb)
+    ctx.eakv_sync()
+    torch.cuda.synchronize()
+    ids = torch.as_tensor(b_.astype(np.int64), device="cuda")
+    for piece in pool.pieces[::7]:
+        assert bool((piece[ids].view(torch.int16) == 0x1111).all())
     ctx.close()
 
 
