@@ -31,8 +31,12 @@
  *     load may run concurrently on two streams.  Where they meet in a tier slot the library
  *     orders them itself: a store into a slot that a restore enqueued earlier (on another
  *     stream) still reads waits for that restore, and a restore of a slot that a store enqueued
- *     earlier still fills waits for that store.  GPU blocks are the caller's: a block must not
- *     be overwritten while a store enqueued on another stream still reads it.
+ *     earlier still fills waits for that store.  The same holds for pool blocks the library
+ *     itself overwrites: a restore into a block that a store enqueued earlier on another stream
+ *     still reads waits for that store, and eakv_turn_begin / eakv_request_begin make
+ *     cuda_stream wait for such stores of the blocks the turn is handed (so an engine that fills
+ *     them behind cuda_stream is ordered too).  Any other write of the engine into a block that a
+ *     store still reads is the caller's to order.
  *   - Layouts: the paged pool is 2L separate arrays, kv_base[2*l] = layer l's K and
  *     kv_base[2*l+1] = its V, each [gpu_blocks][block_size][kv_heads][head_dim] of
  *     elem_bytes-sized elements; one such [block_size][kv_heads][head_dim] slab is a

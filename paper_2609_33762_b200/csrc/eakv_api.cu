@@ -68,6 +68,7 @@ struct TurnState {
 // earlier transfer that used that ring slot.  `done` trails the numbers known to be complete.
 struct SlotOrder {
     static constexpr int kRing = 16;
+    bool by_block = false;                 // index by pool block (ent[].x) instead of tier slot (ent[].y)
     cudaEvent_t ev[kRing] = {};
     cudaStream_t ev_stream[kRing] = {};
     uint64_t next = 1, done = 0;
@@ -85,7 +86,7 @@ struct SlotOrder {
         e = cudaEventRecord(ev[idx], stream);
         if (e != cudaSuccess) return e;
         ev_stream[idx] = stream;
-        for (const int2& x : ent) slot_seq[x.y] = seq;
+        for (const int2& x : ent) slot_seq[by_block ? x.x : x.y] = seq;
         return cudaSuccess;
     }
     // before a transfer of the other direction over these slots is enqueued on `stream`: wait for
@@ -97,9 +98,9 @@ struct SlotOrder {
         bool need[kRing] = {};
         bool any = false;
         for (const int2& x : ent) {
-            const uint64_t q = slot_seq[x.y];
+            uint64_t& q = slot_seq[by_block ? x.x : x.y];
             if (q > done) { need[q % kRing] = true; any = true; }
-            if (forget) slot_seq[x.y] = 0;
+            if (forget) q = 0;
         }
         if (!any) return cudaSuccess;
         for (int idx = 0; idx < kRing; ++idx) {
@@ -182,6 +183,9 @@ struct eakv_ctx {
     // transfer still references; here the bookkeeping may hand the slot on, and the streams are
     // ordered instead).
     SlotOrder restores, stores;
+    // the same for pool blocks: a restore into (or an engine's fill of) a block that a store on
+    // another stream may still be reading waits for that store
+    SlotOrder block_reads;
     uint64_t* turn_keys = nullptr;            // pinned + mapped; the hash kernel writes it directly
     int64_t turn_keys_cap = 0;
     TurnState turn;                            // the one open turn of eakv_turn_begin / eakv_turn_end
@@ -262,6 +266,7 @@ void free_all(eakv_ctx* c) {
     if (c->wb_done) cudaEventDestroy(c->wb_done);
     c->restores.destroy();
     c->stores.destroy();
+    c->block_reads.destroy();
     if (c->tier && c->tier_owned) {
         if (c->cfg.tier_location == EAKV_TIER_DEVICE) cudaFree(c->tier);
         else cudaFreeHost(c->tier);
@@ -635,6 +640,7 @@ int eakv_create(const eakv_config* cfg, eakv_ctx** out) {
         CUC(copy_kernels_init());
     }
 
+    ctx->block_reads.by_block = true;
     try {
         ctx->host_tier = new KeyedLru(cfg->host_blocks);
         ctx->gpu_tier = new KeyedLru(cfg->gpu_index_blocks ? cfg->gpu_index_blocks : cfg->gpu_blocks);
@@ -1219,6 +1225,7 @@ int eakv_store(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* admit_m
     rc = move_blocks(ctx, ent, true, stream, 0, ctx->pieces);
     if (rc != EAKV_OK) return rc;
     CU(ctx->stores.enqueued(ent, ctx->tier_slots, stream));
+    CU(ctx->block_reads.enqueued(ent, ctx->cfg.gpu_blocks, stream));
     ctx->stats.blocks_stored += m;
     ctx->stats.bytes_stored += m * ctx->block_bytes;
     return EAKV_OK;
@@ -1251,6 +1258,7 @@ int eakv_load(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* block_tab
         if (rc != EAKV_OK) return rc;
     }
     CU(ctx->stores.order_after(ent, stream, false));
+    CU(ctx->block_reads.order_after(ent, stream, true));   // the blocks are about to hold other bytes
     rc = move_blocks(ctx, ent, false, stream, 0, ctx->pieces);
     if (rc != EAKV_OK) return rc;
     CU(ctx->restores.enqueued(ent, ctx->tier_slots, stream));
@@ -1290,7 +1298,10 @@ int eakv_load_layers(eakv_ctx* ctx, const int32_t* host_slots, const int32_t* bl
             if (rcw != EAKV_OK) return rcw;
         }
     }
-    if (n_blocks > 0) CU(ctx->stores.order_after(ent, stream, false));
+    if (n_blocks > 0) {
+        CU(ctx->stores.order_after(ent, stream, false));
+        CU(ctx->block_reads.order_after(ent, stream, true));
+    }
     for (int grp = 0; grp < groups; ++grp) {
         const int l0 = grp * layers_per_group;
         const int l1 = std::min(L, l0 + layers_per_group);
@@ -1344,7 +1355,10 @@ int eakv_store_layers(eakv_ctx* ctx, const int32_t* block_table, const uint8_t* 
             if (rc != EAKV_OK) return rc;
         }
     }
-    if (m > 0) CU(ctx->stores.enqueued(ent, ctx->tier_slots, stream));
+    if (m > 0) {
+        CU(ctx->stores.enqueued(ent, ctx->tier_slots, stream));
+        CU(ctx->block_reads.enqueued(ent, ctx->cfg.gpu_blocks, stream));
+    }
     ctx->stats.blocks_stored += m;
     ctx->stats.bytes_stored += m * ctx->block_bytes;
     return EAKV_OK;
@@ -1529,6 +1543,20 @@ int turn_begin_impl(eakv_ctx* ctx, TurnState& T, int64_t request_id, const int32
     if (as_request)
         for (int64_t c = 0; c < nu; ++c)
             if (T.admit_u[c]) ctx->unstored_units[ukeys[c]] = request_id;
+    if (!bookkeeping_only) {
+        // blocks this turn will overwrite (restore or the engine's fill, both behind cuda_stream) may
+        // still be read by a store that another stream carries: cuda_stream waits for it
+        std::vector<int2>& nw = ctx->scratch_entries;
+        nw.clear();
+        if (tail >= 0) nw.push_back(make_int2(tail, 0));
+        for (int64_t j = 0; j < nblk; ++j)
+            if (!T.resident[j]) nw.push_back(make_int2(T.block[j], 0));
+        const cudaError_t eo = ctx->block_reads.order_after(nw, static_cast<cudaStream_t>(cuda_stream), true);
+        if (eo != cudaSuccess) {
+            withdraw_turn(ctx, T, true, 1);
+            return cuda_fail(ctx, eo, "ordering behind a store that still reads the turn's blocks");
+        }
+    }
     if (ctx->wb_pending) {
         bool reused = tail >= 0 && ctx->wb_blocks[tail];
         for (int64_t j = 0; j < nblk && !reused; ++j)

@@ -678,7 +678,7 @@ def test_a_store_waits_for_a_restore_on_another_stream_that_reads_its_slots(link
     from paper_2609_33762_b200 import eakv
     from paper_2609_33762_b200.harness import PagedPool
     shape = SHAPES["qwen3_30b_a3b"]
-    nb, kh, m = 2000, 700, 640
+    nb, kh, m = 2000, 1300, 640
     pool = PagedPool(shape, nb, "cuda:0")
     ctx = eakv.Context(num_layers=shape.num_layers, kv_heads=shape.kv_heads, head_dim=shape.head_dim,
                        block_size=shape.block_size, gpu_blocks=nb, host_blocks=kh, kv_base=pool.kv_base,
@@ -716,6 +716,23 @@ def test_a_store_waits_for_a_restore_on_another_stream_that_reads_its_slots(link
     ids = torch.as_tensor(b_.astype(np.int64), device="cuda")
     for piece in pool.pieces[::7]:
         assert bool((piece[ids].view(torch.int16) == 0x1111).all())
+    # pool blocks: a restore into blocks that a store on another stream still reads waits for it
+    slots2 = slots + m
+    ids_c = torch.as_tensor(c.astype(np.int64), device="cuda")
+    for piece in pool.pieces:
+        piece[ids_c] = 0x5555
+    torch.cuda.synchronize()
+    ctx.eakv_store(c, None, slots2, sa)                  # a second set of slots holds 0x5555
+    ctx.eakv_sync()
+    ctx.eakv_store(a, None, slots, sa)                   # set a (0x2222) on its way to the first slots ...
+    ctx.eakv_load(slots2, a[::-1].copy(), sb)            # ... while another stream restores into set a
+    ctx.eakv_sync()
+    torch.cuda.synchronize()
+    tier = ctx.tier_host_view().view(np.uint16)
+    assert (tier[slots] == 0x2222).all()                 # the store read set a before it changed
+    ids = torch.as_tensor(a.astype(np.int64), device="cuda")
+    for piece in pool.pieces[::7]:
+        assert bool((piece[ids].view(torch.int16) == 0x5555).all())
     ctx.close()
 
 
