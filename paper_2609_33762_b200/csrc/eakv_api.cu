@@ -179,9 +179,9 @@ struct eakv_ctx {
     std::vector<uint8_t> wb_slots;      // by tier slot: a pending write still fills it
     // Transfers in flight, by tier slot: a store into a slot that a restore on another stream may
     // still be reading waits for that restore, and a restore of a slot that a store on another
-    // stream may still be writing waits for that store (the paper's tier frees no chunk that a
-    // transfer still references; here the bookkeeping may hand the slot on, and the streams are
-    // ordered instead).
+    // stream may still be writing waits for that store (Appendix D: the paper's tier exempts a
+    // chunk with a copy in flight from eviction; here the bookkeeping may hand the slot on, and the
+    // streams are ordered instead).
     SlotOrder restores, stores;
     // the same for pool blocks: a restore into (or an engine's fill of) a block that a store on
     // another stream may still be reading waits for that store
