@@ -77,6 +77,9 @@ struct SlotOrder {
     // after a transfer over the slots ent[].y was enqueued on `stream`
     cudaError_t enqueued(const std::vector<int2>& ent, int64_t tier_slots, cudaStream_t stream) {
         if (slot_seq.empty()) slot_seq.assign((size_t)tier_slots, 0);
+        // keep `done` moving also when nothing of the other direction asks for a long time
+        for (int i = 0; i < 4 && done + 1 < next && cudaEventQuery(ev[(done + 1) % kRing]) == cudaSuccess; ++i) ++done;
+        cudaGetLastError();                                // cudaErrorNotReady is not an error here
         const uint64_t seq = next++;
         const int idx = (int)(seq % kRing);
         cudaError_t e = cudaSuccess;
