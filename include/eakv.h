@@ -578,6 +578,27 @@ typedef struct eakv_working_set_out {
 } eakv_working_set_out;
 int eakv_working_set(const eakv_working_set_in* in, eakv_working_set_out* out);
 
+/* Offload benefit of Section 3.1, Eq. 2, in integers (host only, no CUDA call): restoring a prefix
+ * of n tokens costs T_load(n) = n * beta_rank / B_H2D + tau_load, recomputing it T_rec(n) = n * t_pf;
+ * OBR(n) = 1 - T_load(n) / T_rec(n).  Times in picoseconds (the paper's 0.86 us of restore per
+ * token is 860,000).  obr_long_prefix is the limit 1 - beta_rank / (B_H2D * t_pf); break_even_tokens
+ * the shortest prefix whose restore is not slower than its recomputation, -1 if there is none. */
+typedef struct eakv_offload_in {
+    int64_t prefix_tokens;           /* n                                           */
+    int64_t beta_rank_bytes;         /* KV bytes per token and rank (Eq. 1)         */
+    int64_t t_prefill_ps;            /* t_pf: prefill time per token, picoseconds   */
+    int64_t h2d_bytes_per_s;         /* B_H2D                                       */
+    int64_t tau_load_ps;             /* fixed cost of one restoration, picoseconds  */
+} eakv_offload_in;
+typedef struct eakv_offload_out {
+    int64_t t_load_ps, t_rec_ps;
+    int64_t break_even_tokens;
+    double obr, obr_long_prefix;
+    int32_t restore_is_faster;       /* T_load(n) < T_rec(n), compared exactly       */
+    int32_t reserved;
+} eakv_offload_out;
+int eakv_offload_benefit(const eakv_offload_in* in, eakv_offload_out* out);
+
 /* Block keys without a context and without any allocation.  (The paper has no counterpart;
  * this exists for callers that cannot request device memory: code living inside a serving
  * process whose engine has already claimed the GPU's memory, where an allocation may fail or

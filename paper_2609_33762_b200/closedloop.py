@@ -329,14 +329,18 @@ def run(config, *, policy="write_all", host_gib=None, active_pool=None, model=Se
     st = server.ctx.eakv_get_stats()
     tot = server.totals
     queue_us = sum(o[3] - o[2] for o in order)
+    benefit = eakv.eakv_offload_benefit(prefix_tokens=max(1, trace.total_prompt_tokens // max(1, len(trace.requests))),
+                                        beta_rank_bytes=shape.bytes_per_token, t_prefill_ps=model.t_pf_ns * 1000,
+                                        h2d_bytes_per_s=model.h2d_bytes_per_us * 1_000_000,
+                                        tau_load_ps=model.tau_load_us * 1_000_000)
     out = {
         "config": config, "policy": policy, "active_pool": A, "tasks": len(trace.agent_tokens),
         "requests": len(order), "host_gib": kh * chunk_blocks * shape.block_bytes / GIB,
         "host_sizing": why, "chunk_blocks": chunk_blocks, "theta_percent": theta,
         "data_plane": data_plane, "measured_transfers": measured_transfers,
         "service_model": model.__dict__,
-        # Eq. 2 for long prefixes: OBR -> 1 - beta / (B_H2D * t_pf)
-        "obr_long_prefix": 1.0 - shape.bytes_per_token / model.h2d_bytes_per_us / (model.t_pf_ns / 1000.0),
+        # Eq. 2: the long-prefix limit of OBR and the prefix length from which a restore pays (eakv_offload_benefit)
+        "offload_benefit": {k: benefit[k] for k in ("obr_long_prefix", "break_even_tokens")},
         "makespan_s": makespan / 1e6, "mean_queue_delay_ms": queue_us / max(1, len(order)) / 1e3,
         "engine_busy_s": {k[:-3]: v / 1e6 for k, v in busy.items()},
         "prompt_tokens": tot["prompt_tokens"], "computed_prefill_tokens": tot["fresh_tokens"],

@@ -19,6 +19,7 @@
 // (Mattson); the host-covered prefix of a request = its leading run of hits; restored = max(0, H - G);
 // computed prefill = n - max(G, H) * b.
 #include <algorithm>
+#include <climits>
 #include <cstdint>
 #include <vector>
 
@@ -561,6 +562,35 @@ extern "C" int eakv_working_set(const eakv_working_set_in* in, eakv_working_set_
     out->gamma_h = h_den ? (double)num / (double)h_den : 0.0;
     out->pool_exceeds_gpu = g_den ? (g_num > g_den) : 0;
     out->working_set_exceeds_host = h_den ? (num > h_den) : 0;
+    return EAKV_OK;
+}
+
+extern "C" int eakv_offload_benefit(const eakv_offload_in* in, eakv_offload_out* out) {
+    if (!in || !out) return EAKV_E_INVAL;
+    if (in->prefix_tokens <= 0 || in->beta_rank_bytes <= 0 || in->t_prefill_ps <= 0 ||
+        in->h2d_bytes_per_s <= 0 || in->tau_load_ps < 0)
+        return EAKV_E_INVAL;
+    typedef __int128 wide;
+    const wide ps = 1000000000000ll;
+    // Eq. 2: T_load(n) = n * beta / B_H2D + tau_load,  T_rec(n) = n * t_pf  (picoseconds, floor)
+    const wide load = (wide)in->prefix_tokens * in->beta_rank_bytes * ps / in->h2d_bytes_per_s + in->tau_load_ps;
+    const wide rec = (wide)in->prefix_tokens * in->t_prefill_ps;
+    const wide lim = (wide)INT64_MAX;
+    out->t_load_ps = (int64_t)std::min(load, lim);
+    out->t_rec_ps = (int64_t)std::min(rec, lim);
+    out->obr = 1.0 - (double)load / (double)rec;
+    out->restore_is_faster = load < rec;
+    // per token: beta / B_H2D against t_pf, compared as beta * 10^12 against t_pf * B_H2D; the fixed
+    // cost tau is repaid after n* = ceil(tau * B_H2D / (t_pf * B_H2D - beta * 10^12)) tokens
+    const wide load_b = (wide)in->beta_rank_bytes * ps;
+    const wide rec_b = (wide)in->t_prefill_ps * in->h2d_bytes_per_s;
+    out->obr_long_prefix = 1.0 - (double)load_b / (double)rec_b;
+    if (load_b >= rec_b) {
+        out->break_even_tokens = -1;                 // a restored token never costs less than a computed one
+    } else {
+        const wide gain = rec_b - load_b;
+        out->break_even_tokens = (int64_t)std::min(((wide)in->tau_load_ps * in->h2d_bytes_per_s + gain - 1) / gain, lim);
+    }
     return EAKV_OK;
 }
 

@@ -68,6 +68,17 @@ class StepInfo(C.Structure):
                 ("pressure", C.c_int32), ("save", C.c_int32)]
 
 
+class OffloadIn(C.Structure):
+    _fields_ = [("prefix_tokens", C.c_int64), ("beta_rank_bytes", C.c_int64), ("t_prefill_ps", C.c_int64),
+                ("h2d_bytes_per_s", C.c_int64), ("tau_load_ps", C.c_int64)]
+
+
+class OffloadOut(C.Structure):
+    _fields_ = [("t_load_ps", C.c_int64), ("t_rec_ps", C.c_int64), ("break_even_tokens", C.c_int64),
+                ("obr", C.c_double), ("obr_long_prefix", C.c_double), ("restore_is_faster", C.c_int32),
+                ("reserved", C.c_int32)]
+
+
 class WorkingSetIn(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("num_layers", "kv_heads", "head_dim", "elem_bytes", "tensor_parallel",
                                          "block_size")] + \
@@ -112,7 +123,7 @@ EXPORTS = [
     "eakv_gpu_tier_acquire", "eakv_gpu_tier_release_request", "eakv_tier_step_again",
     "eakv_declined_audit", "eakv_working_set",
     "eakv_request_begin", "eakv_request_store", "eakv_request_release", "eakv_working_set_sizes", "eakv_selfcheck_fail_next_transfer", "eakv_store_layers", "eakv_turn_end_layers", "eakv_request_store_layers",
-    "eakv_turn_begin_layers", "eakv_request_begin_layers",
+    "eakv_turn_begin_layers", "eakv_request_begin_layers", "eakv_offload_benefit",
 ]
 STATIC_MAX_BLOCKS = 65536
 
@@ -156,6 +167,7 @@ def lib():
     L.eakv_turn_begin_layers.argtypes = [vp, vp, i64, vp, i64, i64, i64, i32, vp, i32, vp, vp]
     L.eakv_request_begin_layers.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i32, i32, vp, i32, vp, vp]
     L.eakv_request_store_layers.argtypes = [vp, i64, i32, vp, i32, vp]
+    L.eakv_offload_benefit.argtypes = [C.POINTER(OffloadIn), C.POINTER(OffloadOut)]
     L.eakv_working_set_sizes.argtypes = [vp, i64, vp, vp, vp, i64, i32, i32, C.POINTER(i64), C.POINTER(i64), vp]
     L.eakv_working_set.argtypes = [C.POINTER(WorkingSetIn), C.POINTER(WorkingSetOut)]
     L.eakv_turn_begin.argtypes = [vp, vp, i64, vp, i64, i64, i64, vp, C.POINTER(TurnView)]
@@ -236,6 +248,17 @@ def eakv_declined_audit(keys_dev, declined_dev, n_refs, capacity, next_dist_dev=
     if rc != OK:
         raise EakvError(rc, "eakv_declined_audit")
     return d.value, m.value, nv.value
+
+
+def eakv_offload_benefit(*, prefix_tokens, beta_rank_bytes, t_prefill_ps, h2d_bytes_per_s, tau_load_ps=0):
+    """Eq. 2: restore time, recompute time (picoseconds), OBR(n), its long-prefix limit and the
+    break-even prefix length."""
+    i = OffloadIn(int(prefix_tokens), int(beta_rank_bytes), int(t_prefill_ps), int(h2d_bytes_per_s), int(tau_load_ps))
+    o = OffloadOut()
+    rc = lib().eakv_offload_benefit(C.byref(i), C.byref(o))
+    if rc != OK:
+        raise EakvError(rc, "eakv_offload_benefit")
+    return {f: getattr(o, f) for f, _ in OffloadOut._fields_ if f != "reserved"}
 
 
 def eakv_working_set_sizes(dist_dev, n_refs, req_offsets, req_tokens, req_gpu_prefix, block_size, percent=1,

@@ -1,6 +1,8 @@
 """Host logic of the replay and capacity drivers that needs no GPU: tier sizing by the
 working-set scale (Eq. 5) agrees with the oracle's arithmetic, and the plan honours the
 configuration, explicit requests and the host-memory cap."""
+import pytest
+
 from eakv_workloads import CONFIGS, SHAPES, make_trace
 from oracle import sizing
 from paper_2609_33762_b200 import replay
@@ -83,3 +85,43 @@ def test_eakv_working_set_against_oracle_sizing_and_the_papers_printed_values():
     with pytest.raises(eakv.EakvError):
         eakv.eakv_working_set(num_layers=0, kv_heads=1, head_dim=8, block_size=16, active_pool=2,
                               total_prompt_tokens=10, n_requests=1)
+
+
+def test_eakv_offload_benefit_against_the_oracle_and_the_papers_ratio():
+    """Eq. 2 in the library (integers, picoseconds) against oracle.sizing.obr / load_time, on the
+    paper's own deployment (24 KiB per token and rank, 26.6 GiB/s: 0.86 us of restore per token
+    against 5.6 us of prefill, OBR > 0.84) and on random inputs; the break-even length is the first
+    n at which the restore is not slower."""
+    import math
+    import random
+    from oracle import sizing as sz
+    from paper_2609_33762_b200 import build, eakv
+    build.build()
+    GIB = 1 << 30
+    beta = sz.beta_rank(48, 128, 2, 4, 8)
+    bw = int(26.6 * GIB)
+    t_pf_ps = round(6.6e9 / (8 * 148e12) * 1e12)
+    o = eakv.eakv_offload_benefit(prefix_tokens=10**9, beta_rank_bytes=beta, t_prefill_ps=t_pf_ps, h2d_bytes_per_s=bw)
+    assert round(o["t_load_ps"] / 10**9 / 1e6, 2) == 0.86 and round(t_pf_ps / 1e6, 1) == 5.6
+    assert o["obr"] > 0.84 and math.isclose(o["obr"], 1 - 0.86 / 5.6, abs_tol=0.01)
+    assert math.isclose(o["obr_long_prefix"], o["obr"], abs_tol=1e-9) and o["break_even_tokens"] == 0
+    rng = random.Random(4)
+    for _ in range(200):
+        n = rng.randrange(1, 200_000)
+        b_ = rng.randrange(1 << 10, 1 << 19)
+        t = rng.randrange(100_000, 20_000_000)
+        w = rng.randrange(1 << 30, 1 << 37)
+        tau = rng.randrange(0, 400_000_000)
+        o = eakv.eakv_offload_benefit(prefix_tokens=n, beta_rank_bytes=b_, t_prefill_ps=t, h2d_bytes_per_s=w, tau_load_ps=tau)
+        want = sz.obr(n, t * 1e-12, b_, w, tau_load=tau * 1e-12)
+        assert math.isclose(o["obr"], want, rel_tol=1e-9, abs_tol=1e-9)
+        assert math.isclose(o["t_load_ps"], sz.load_time(n, b_, w, tau * 1e-12) * 1e12, rel_tol=1e-9, abs_tol=1.0)
+        assert o["restore_is_faster"] == (o["t_load_ps"] < o["t_rec_ps"]) or abs(o["t_load_ps"] - o["t_rec_ps"]) <= 1
+        ne = o["break_even_tokens"]
+        gain = t * w - b_ * 10**12                     # per token, times B_H2D
+        if gain <= 0:
+            assert ne == -1
+        else:
+            assert ne * gain >= tau * w and (ne == 0 or (ne - 1) * gain < tau * w)
+    with pytest.raises(eakv.EakvError):
+        eakv.eakv_offload_benefit(prefix_tokens=0, beta_rank_bytes=1, t_prefill_ps=1, h2d_bytes_per_s=1)
